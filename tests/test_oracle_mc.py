@@ -1,0 +1,49 @@
+"""Monte Carlo pins: the guarded plan keeps Theorem 1's budget; Algorithm 1's t = 1 step does not."""
+import numpy as np
+import pytest
+
+from oracle import mc, plan, rank_law
+
+
+def test_simulated_rank_follows_lemma_1():
+    rng = np.random.default_rng(0)
+    N, S, t = 4096, 64, 3
+    R = mc.simulate_ranks(N, S, t, 4000, rng)
+    assert R.mean() == pytest.approx(rank_law.nhg_mean(N, S, t), rel=0.03)
+    assert R.var() == pytest.approx(rank_law.nhg_var(N, S, t), rel=0.12)
+    assert R.min() >= t and R.max() <= N - S + t
+
+
+def test_guarded_plan_meets_the_budget_on_small_rows():
+    rng = np.random.default_rng(1)
+    N, k, eps = 1 << 16, 64, 2e-2                                   # large eps so a few thousand trials resolve it
+    p = plan.plan_guarded(N, k, eps, s_min=2048, s_max=2048)
+    for placement in ("random", "sorted"):
+        R = mc.simulate_ranks(N, p.m, p.r, 3000, rng, placement)
+        rate = np.mean((R < k) | (R > p.capacity))
+        assert rate <= eps + 3 * np.sqrt(eps / 3000)
+
+
+def test_literal_sparse_rule_breaks_the_budget():
+    rng = np.random.default_rng(2)
+    N, k, eps = 1 << 16, 64, 1e-3
+    S, t, M = plan.plan_paper(N, k, eps, s_min=2048, s_max=2048)
+    assert t == 1                                                    # alpha S = 2 < -ln(eps/2)
+    R = mc.simulate_ranks(N, S, t, 500, rng)
+    assert np.mean(R < k) > 0.5                                      # ~ 1 - exp(-alpha S) = 0.86, not exp(-alpha S)
+
+
+@pytest.mark.parametrize("N,k,eps", [(1 << 20, 64, 1e-3), (1 << 26, 256, 1e-2), (1 << 26, 4096, 1e-2), (1 << 29, 131072, 1e-3)])
+def test_failure_rates_at_the_benchmark_shapes(N, k, eps):
+    rng = np.random.default_rng(3)
+    trials = 400_000
+    p = plan.plan_guarded(N, k, eps)
+    fa, fb = mc.failure_rate_exchangeable(N, p.m, p.r, k, p.capacity, trials, rng)
+    sigma = np.sqrt(eps / trials)
+    assert fa + fb <= eps + 4 * sigma
+    assert fa == pytest.approx(rank_law.p_recall_fail_srs(N, p.m, p.r, k), abs=4 * sigma)
+    assert fb == pytest.approx(rank_law.p_overflow_srs(N, p.m, p.r, p.capacity), abs=4 * sigma)
+    # Algorithm 1 as printed, same shape: at least one of its failure modes is far over budget
+    S, t, M = plan.plan_paper(N, k, eps)
+    ga, gb = mc.failure_rate_exchangeable(N, S, t, k, M, 20_000, rng)
+    assert ga + gb > eps

@@ -1,0 +1,73 @@
+"""Pins for oracle.stages: the four stages of Section 3 run on NumPy arrays."""
+import numpy as np
+import pytest
+
+from oracle import philox, stages, topk
+
+
+def test_success_branch_returns_the_exact_topk():
+    rng = np.random.default_rng(0)
+    hits = 0
+    for seed in range(40):
+        x = rng.standard_normal(4096).astype(np.float32)
+        res = stages.run_row(x, k=20, m=256, r=4, capacity=400, k_accept=20, seed=seed)
+        v, i = topk.topk_row(x, 20)
+        assert np.array_equal(res.idx, i) and np.array_equal(res.vals, v)          # always exact, whichever branch
+        if res.status == stages.STATUS_OK:
+            hits += 1
+            assert 20 <= res.survivors <= 400
+    assert hits > 20
+
+
+def test_survivor_count_is_the_rank_of_tau():
+    x = np.random.default_rng(1).permutation(5000).astype(np.float32)              # distinct values
+    s_idx = philox.sample_indices(5000, 100, seed=9)
+    tau = stages.threshold(x, s_idx, 3)
+    assert tau == np.sort(x[s_idx])[::-1][2]
+    R = stages.count_survivors(x, tau)
+    assert R == int(np.flatnonzero(np.sort(x)[::-1] == tau)[0]) + 1                # Lemma 1's R: rank 1 = largest
+    assert np.array_equal(stages.survivor_set(x, tau), np.flatnonzero(x >= tau))
+
+
+def test_failure_branches_by_construction():
+    x = np.arange(1000, dtype=np.float32)
+    # capacity too small for the survivors of a low threshold -> overflow
+    res = stages.run_row(x, k=5, m=10, r=10, capacity=5, k_accept=5, seed=1)
+    assert res.status == stages.STATUS_OVERFLOW and res.survivors > 5
+    assert np.array_equal(res.idx, np.arange(999, 994, -1))
+    # threshold = sample maximum, k larger than what survives -> insufficient recall
+    res = stages.run_row(x, k=400, m=10, r=1, capacity=1000, k_accept=400, seed=1)
+    assert res.status == stages.STATUS_RECALL and res.survivors < 400
+    assert np.array_equal(res.idx, np.arange(999, 599, -1))
+    # all-equal input: every element passes "x >= tau" -> overflow, answer = lowest indices
+    z = np.zeros(300, dtype=np.float32)
+    res = stages.run_row(z, k=7, m=20, r=2, capacity=50, k_accept=7, seed=3)
+    assert res.status == stages.STATUS_OVERFLOW and res.survivors == 300
+    assert np.array_equal(res.idx, np.arange(7))
+    # direct mode
+    res = stages.run_row(x, k=3, m=0, r=0, capacity=0, k_accept=3, seed=0, mode=1)
+    assert res.status == stages.STATUS_DIRECT and res.idx.tolist() == [999, 998, 997]
+
+
+def test_relaxed_mode_returns_a_padded_prefix():
+    x = np.arange(1000, dtype=np.float32)
+    for seed in range(20):
+        res = stages.run_row(x, k=100, m=50, r=3, capacity=1000, k_accept=20, seed=seed)
+        if res.status == stages.STATUS_OK and res.survivors < 100:
+            R = res.survivors
+            assert np.array_equal(res.idx[:R], np.arange(999, 999 - R, -1))        # prefix of the exact answer
+            assert np.all(res.idx[R:] == -1) and np.all(np.isneginf(res.vals[R:]))
+            return
+    pytest.fail("no seed produced a short buffer")
+
+
+def test_bf16_rows_and_nan_are_kept():
+    rng = np.random.default_rng(3)
+    f = rng.standard_normal(2000).astype(np.float32)
+    b = (f.view(np.uint32) >> 16).astype(np.uint16)
+    res = stages.run_row(b, k=10, m=64, r=4, capacity=2000, k_accept=10, seed=5)
+    v, i = topk.topk_row(b, 10)
+    assert np.array_equal(res.idx, i) and np.array_equal(res.vals, v)
+    g = f.copy(); g[17] = np.nan
+    tau = np.float32(1.0)
+    assert 17 in stages.survivor_set(g, tau)                                       # not (NaN < tau)
