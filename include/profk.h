@@ -1,0 +1,207 @@
+/*
+ * profk.h -- C ABI of the Prof-K top-k library for NVIDIA B200 (sm_100a).
+ *
+ * Prof-K (Section 3 of the paper, "The Prof-K algorithm") returns the k largest
+ * entries of each row of a rows x N matrix together with their indices by
+ *   1. drawing a small sample of S positions,
+ *   2. taking the t-th largest sampled value as threshold tau,
+ *   3. streaming the row once and appending every element x_i >= tau to a
+ *      candidate buffer of capacity M,
+ *   4. running an exact top-k on that buffer; when fewer than k candidates were
+ *      kept or the buffer overflowed, an exact top-k of the whole row replaces it.
+ * In this library every stage, the check of step 4 and the exact replacement
+ * run on the GPU; no call copies anything to the host or waits for the device.
+ *
+ * Conventions for every entry point
+ *   - Pointers marked [device] are device addresses valid on the current CUDA
+ *     device; [host] are ordinary host addresses.  The library never allocates,
+ *     frees or keeps device memory: inputs, outputs and the workspace belong to
+ *     the caller.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Work is only enqueued; results are valid once the caller has
+ *     synchronised the stream.
+ *   - Return value: PROFK_OK (0) or a negative profk_status_t.  No exception
+ *     crosses the boundary.  A repaired failure of the probabilistic filter is
+ *     not an error: it shows only in the per-row statistics.
+ *   - Layout: `in` is row-major, contiguous, rows x N; element (row, i) is at
+ *     in[row * N + i].  Outputs are rows x k.  Indices are 0-based positions
+ *     inside the row.  Each output row is ordered by value descending, equal
+ *     values by index ascending; values are ordered through the total order
+ *     -NaN < -inf < ... < -0 < +0 < ... < +inf < +NaN of their bit patterns.
+ *   - Limits: 1 <= k <= N <= 2^32 - 2^24 per row, rows >= 1, rows * capacity < 2^40.
+ *   - Two calls that use the same workspace must not overlap on the device.
+ */
+#ifndef PROFK_H
+#define PROFK_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum profk_status {
+    PROFK_OK = 0,
+    PROFK_EINVAL = -1,     /* bad argument (range, null pointer, alignment) */
+    PROFK_EWORKSPACE = -2, /* no workspace registered on this device, or it is too small */
+    PROFK_ECUDA = -3,      /* a CUDA runtime call or launch reported an error */
+    PROFK_ETIMEOUT = -4    /* (statistics only) a bounded device-side wait gave up */
+} profk_status_t;
+
+typedef enum profk_dtype { PROFK_F32 = 0, PROFK_BF16 = 1 } profk_dtype_t;
+
+/* Per-row outcome of the count check of stage 4. */
+enum {
+    PROFK_ROW_OK = 0,       /* k_accept <= R <= capacity: answer refined from the buffer   */
+    PROFK_ROW_RECALL = 1,   /* R < k_accept: too few candidates, exact selection ran       */
+    PROFK_ROW_OVERFLOW = 2, /* R > capacity: buffer overflowed, exact selection ran        */
+    PROFK_ROW_DIRECT = 3    /* plan mode 1: exact selection without sampling or filtering  */
+};
+
+/*
+ * The parameters (S, t, M) of Section 4 / Algorithm 1, as this library chooses them.
+ *   m         sample size S: Algorithm 1 steps 1-4 (Eq. optimal_S with log2 k,
+ *             rounded, clamped to [s_min, s_max]) and never more than N.
+ *   r         sample rank t (1-based): the smallest rank whose recall-failure
+ *             bound Pr(R < k_accept) is <= eps/2.  Algorithm 1's last step
+ *             (t <- 1 in the sparse regime) is NOT applied: it breaks the eps
+ *             budget of Theorem 1 that this plan keeps.
+ *   capacity  buffer capacity M: max(ceil(Eq. M), smallest M whose overflow
+ *             bound Pr(R > M) is <= eps/2), never more than N.
+ *   k_accept  k in exact mode (recall == 1), ceil(recall * k) in relaxed mode.
+ *   mode      0 = sample / filter / refine; 1 = direct exact selection, chosen
+ *             when 2 * capacity >= N or N <= 2 * m (the filter would not pay).
+ *   z, alpha  Algorithm 1's z = 2 Phi^{-1}(1 - eps/2) and alpha = k / N.
+ *   p_recall_fail, p_overflow   the two bounds for the returned (m, r, capacity).
+ * Both bounds are binomial tail bounds valid for the stratified sampler the
+ * library uses (one uniform draw from each of m equal strata of the row).
+ */
+typedef struct profk_plan {
+    int64_t m;
+    int64_t r;
+    int64_t capacity;
+    int64_t k_accept;
+    int32_t mode;
+    int32_t reserved;
+    double z;
+    double alpha;
+    double p_recall_fail;
+    double p_overflow;
+} profk_plan_t;
+
+/* Tuning inputs of Algorithm 1; profk_plan uses the paper's defaults
+ * s_min = 32768, s_max = 131072, cost_ratio (tau_B / tau_A) = 1. */
+typedef struct profk_tuning {
+    int64_t s_min;
+    int64_t s_max;
+    double cost_ratio;
+} profk_tuning_t;
+
+/* What happened to one row (read back with profk_read_stats). */
+typedef struct profk_row_stats {
+    uint32_t tau_bits;   /* threshold tau: fp32 bit pattern, or bf16 pattern in the low 16 bits */
+    uint32_t survivors;  /* R = |{i : x_i >= tau}|; exact when <= capacity, otherwise only "> capacity" */
+    uint32_t capacity;   /* M used for the row */
+    uint32_t status;     /* PROFK_ROW_*; bit 31 set = a device-side wait timed out (result invalid) */
+} profk_row_stats_t;
+
+/*
+ * Host, pure: Algorithm 1 with the guard described at profk_plan_t.
+ *   N, k      row length and selection size, 1 <= k <= N <= 2^32 - 2^24
+ *   eps       total failure budget, 0 < eps < 1 (the paper's default is 1e-3)
+ *   recall    1.0 = exact mode; rho in (0,1) = relaxed mode (accept ceil(rho k) survivors)
+ *   out       [host] receives the plan
+ * Returns PROFK_EINVAL on a bad argument.  profk_plan_ex takes the tuning
+ * inputs explicitly (NULL = defaults).
+ */
+int profk_plan(int64_t N, int64_t k, double eps, double recall, profk_plan_t* out);
+int profk_plan_ex(int64_t N, int64_t k, double eps, double recall, const profk_tuning_t* tuning,
+                  profk_plan_t* out);
+
+/*
+ * Workspace.  profk_workspace_bytes gives the size the calls below need for
+ * `rows` rows with buffer capacity `capacity` and selection size k (take
+ * capacity from profk_plan; it does not depend on the element type).
+ * profk_set_workspace registers a caller-owned device allocation (256-byte
+ * aligned) for the current device; it stays registered until replaced or
+ * cleared with (NULL, 0).  Its contents need no initialisation and are
+ * overwritten by every call.
+ */
+int profk_workspace_bytes(int64_t rows, int64_t capacity, int64_t k, size_t* bytes /* [host] */);
+int profk_set_workspace(void* dev_ptr /* [device] */, size_t bytes);
+
+/*
+ * Top-k of every row (the problem statement of Section 3), all four stages on
+ * the GPU.  Equivalent to profk_plan followed by profk_topk_planned_*.
+ *   in        [device] rows x N elements, fp32 / bf16, aligned to the element size
+ *   seed      keys the Philox4x32-10 sample; in exact mode the result does not
+ *             depend on it, only tau, the buffer and the repair decision do
+ *   out_vals  [device] rows x k, same element type as `in`
+ *   out_idx   [device] rows x k int64
+ * Relaxed mode (recall < 1): a row whose buffer holds R < k (but >= k_accept)
+ * candidates returns its R best in order followed by padding (value -inf,
+ * index -1); the result is always a prefix of the exact answer.
+ * Errors: PROFK_EINVAL, PROFK_EWORKSPACE, PROFK_ECUDA.
+ */
+int profk_topk_f32(const float* in, int64_t rows, int64_t N, int64_t k, double eps, double recall,
+                   uint64_t seed, void* stream, float* out_vals, int64_t* out_idx);
+int profk_topk_bf16(const void* in, int64_t rows, int64_t N, int64_t k, double eps, double recall,
+                    uint64_t seed, void* stream, void* out_vals, int64_t* out_idx);
+
+/*
+ * Same with the plan given explicitly (stages 1-4 of Section 3 with the
+ * caller's S = m, t = r, M = capacity).  Any plan returns the exact answer,
+ * because the count check repairs a bad one: capacity == k forces overflows,
+ * r == 1 with a large m forces recall failures, mode == 1 skips the filter.
+ * Requires 1 <= r <= m <= min(N, 262144), k <= capacity <= N,
+ * 1 <= k_accept <= k (mode 0).
+ */
+int profk_topk_planned_f32(const float* in, int64_t rows, int64_t N, int64_t k, const profk_plan_t* plan,
+                           uint64_t seed, void* stream, float* out_vals, int64_t* out_idx);
+int profk_topk_planned_bf16(const void* in, int64_t rows, int64_t N, int64_t k, const profk_plan_t* plan,
+                            uint64_t seed, void* stream, void* out_vals, int64_t* out_idx);
+
+/*
+ * Stage 3 alone (the filtering scan of Section 3): for every row append the
+ * elements with x_i >= tau[row] to the row's buffer and count them.
+ *   tau        [device] rows thresholds of the element type
+ *   buf_keys   [device] rows x capacity uint64 candidate records (see below)
+ *   counts     [device] rows uint32, must be zero on entry; on return the
+ *              number of survivors (exact if <= capacity, else some value > capacity)
+ * A candidate record packs the complemented order key of the value in the high
+ * 32 bits (bf16: key in bits 63..48) and the index in the low 32 bits, so that
+ * ascending records are "value descending, index ascending".  Records are
+ * appended in no particular order.  Needs no workspace.
+ */
+int profk_filter_f32(const float* in, int64_t rows, int64_t N, const float* tau, int64_t capacity,
+                     uint64_t* buf_keys, uint32_t* counts, void* stream);
+int profk_filter_bf16(const void* in, int64_t rows, int64_t N, const void* tau, int64_t capacity,
+                      uint64_t* buf_keys, uint32_t* counts, void* stream);
+
+/*
+ * Stages 1-2 alone (sampling and threshold estimation of Section 3): tau[row]
+ * = the r-th largest of m stratified Philox samples of the row.  Also writes
+ * the sampled indices when sample_idx != NULL ([device] rows x m uint32).
+ */
+int profk_sample_threshold_f32(const float* in, int64_t rows, int64_t N, int64_t m, int64_t r, uint64_t seed,
+                               float* tau, uint32_t* sample_idx, void* stream);
+int profk_sample_threshold_bf16(const void* in, int64_t rows, int64_t N, int64_t m, int64_t r, uint64_t seed,
+                                void* tau, uint32_t* sample_idx, void* stream);
+
+/*
+ * Copies the statistics of the last call that used the registered workspace to
+ * the host and waits for `stream`.  out: [host] rows entries.
+ */
+int profk_read_stats(void* stream, int64_t rows, profk_row_stats_t* out);
+
+/* Number of kernels the last profk_topk* call on this thread enqueued. */
+int profk_last_launch_count(void);
+
+/* Static text for a status code. */
+const char* profk_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PROFK_H */

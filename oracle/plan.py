@@ -56,8 +56,11 @@ COST_RATIO_DEFAULT = 1.0     # tau_B / tau_A, Algorithm 1 default
 
 # ----------------------------------------------------------------------------- equations
 def z_one_sided(eps_part: float) -> float:
-    """z_A = Phi^{-1}(1 - eps_A) (Section 4, 'Controlling insufficient recall')."""
-    return float(stats.norm.ppf(1.0 - eps_part))
+    """z_A = Phi^{-1}(1 - eps_A) (Section 4, 'Controlling insufficient recall').
+
+    Evaluated as the upper-tail quantile of eps_A, which is the same number without the
+    rounding of 1 - eps_A (that rounding costs ~1e-11 of z at eps = 1e-6)."""
+    return float(stats.norm.isf(eps_part))
 
 
 def z_total(eps: float) -> float:

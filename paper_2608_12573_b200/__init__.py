@@ -1,0 +1,234 @@
+"""Prof-K one-pass probabilistic top-k for NVIDIA B200: thin Python binding of the C ABI.
+
+Every function here only marshals arguments (torch tensors -> device pointers, the
+current CUDA stream) into the `extern "C"` entry points declared in `include/profk.h`;
+all arithmetic of the method runs inside the CUDA library `libprofk.so`, which is built
+in-tree by `paper_2608_12573_b200._build.build()`.  There is no CPU fallback: a call
+raises when the library is missing or reports an error.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+_LIB = None
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libprofk.so")
+
+EXPORTS = [
+    "profk_plan", "profk_plan_ex", "profk_workspace_bytes", "profk_set_workspace",
+    "profk_topk_f32", "profk_topk_bf16", "profk_topk_planned_f32", "profk_topk_planned_bf16",
+    "profk_filter_f32", "profk_filter_bf16", "profk_sample_threshold_f32", "profk_sample_threshold_bf16",
+    "profk_read_stats", "profk_last_launch_count", "profk_strerror",
+]
+
+ROW_OK, ROW_RECALL, ROW_OVERFLOW, ROW_DIRECT = 0, 1, 2, 3
+
+
+class ProfkError(RuntimeError):
+    pass
+
+
+class _PlanStruct(ctypes.Structure):
+    _fields_ = [("m", ctypes.c_int64), ("r", ctypes.c_int64), ("capacity", ctypes.c_int64),
+                ("k_accept", ctypes.c_int64), ("mode", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("z", ctypes.c_double), ("alpha", ctypes.c_double),
+                ("p_recall_fail", ctypes.c_double), ("p_overflow", ctypes.c_double)]
+
+
+class _TuningStruct(ctypes.Structure):
+    _fields_ = [("s_min", ctypes.c_int64), ("s_max", ctypes.c_int64), ("cost_ratio", ctypes.c_double)]
+
+
+class _StatsStruct(ctypes.Structure):
+    _fields_ = [("tau_bits", ctypes.c_uint32), ("survivors", ctypes.c_uint32),
+                ("capacity", ctypes.c_uint32), ("status", ctypes.c_uint32)]
+
+
+@dataclass
+class Plan:
+    m: int
+    r: int
+    capacity: int
+    k_accept: int
+    mode: int
+    z: float = 0.0
+    alpha: float = 0.0
+    p_recall_fail: float = 0.0
+    p_overflow: float = 0.0
+
+    def _struct(self) -> _PlanStruct:
+        return _PlanStruct(self.m, self.r, self.capacity, self.k_accept, self.mode, 0,
+                           self.z, self.alpha, self.p_recall_fail, self.p_overflow)
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded CUDA library; raises if it has not been built."""
+    global _LIB
+    if _LIB is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ProfkError(f"{_LIB_PATH} is missing: run paper_2608_12573_b200._build.build() "
+                             "(there is no fallback implementation)")
+        _LIB = ctypes.CDLL(_LIB_PATH)
+        _LIB.profk_strerror.restype = ctypes.c_char_p
+        _LIB.profk_strerror.argtypes = [ctypes.c_int]
+        for name in EXPORTS:
+            getattr(_LIB, name)          # fail now if a symbol is absent
+    return _LIB
+
+
+def _check(code: int, what: str) -> None:
+    if code != 0:
+        raise ProfkError(f"{what}: {lib().profk_strerror(code).decode()} ({code})")
+
+
+def plan(N: int, k: int, eps: float = 1e-3, recall: float = 1.0, s_min: int | None = None,
+         s_max: int | None = None, cost_ratio: float | None = None) -> Plan:
+    """`profk_plan` / `profk_plan_ex`: the parameters (S, t, M) for one row of length N."""
+    out = _PlanStruct()
+    if s_min is None and s_max is None and cost_ratio is None:
+        code = lib().profk_plan(ctypes.c_int64(N), ctypes.c_int64(k), ctypes.c_double(eps),
+                                ctypes.c_double(recall), ctypes.byref(out))
+    else:
+        tun = _TuningStruct(32768 if s_min is None else s_min, 131072 if s_max is None else s_max,
+                            1.0 if cost_ratio is None else cost_ratio)
+        code = lib().profk_plan_ex(ctypes.c_int64(N), ctypes.c_int64(k), ctypes.c_double(eps),
+                                   ctypes.c_double(recall), ctypes.byref(tun), ctypes.byref(out))
+    _check(code, "profk_plan")
+    return Plan(out.m, out.r, out.capacity, out.k_accept, out.mode, out.z, out.alpha,
+                out.p_recall_fail, out.p_overflow)
+
+
+def workspace_bytes(rows: int, capacity: int, k: int) -> int:
+    n = ctypes.c_size_t()
+    _check(lib().profk_workspace_bytes(ctypes.c_int64(rows), ctypes.c_int64(capacity), ctypes.c_int64(k),
+                                       ctypes.byref(n)), "profk_workspace_bytes")
+    return int(n.value)
+
+
+_workspaces: dict = {}     # device index -> torch tensor kept alive while registered
+
+
+def ensure_workspace(rows: int, capacity: int, k: int, device) -> None:
+    """Allocate (through torch) and register a workspace large enough for the shape."""
+    import torch
+
+    need = workspace_bytes(rows, capacity, k)
+    dev = torch.device(device)
+    idx = dev.index if dev.index is not None else torch.cuda.current_device()
+    cur = _workspaces.get(idx)
+    if cur is None or cur.numel() < need:
+        with torch.cuda.device(idx):
+            buf = torch.empty(max(need, 1 << 20), dtype=torch.uint8, device=dev)
+            _check(lib().profk_set_workspace(ctypes.c_void_p(buf.data_ptr()), ctypes.c_size_t(buf.numel())),
+                   "profk_set_workspace")
+        _workspaces[idx] = buf
+
+
+def _stream_ptr():
+    import torch
+
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _suffix(x) -> str:
+    import torch
+
+    if x.dtype == torch.float32:
+        return "f32"
+    if x.dtype == torch.bfloat16:
+        return "bf16"
+    raise ProfkError(f"unsupported dtype {x.dtype}: float32 and bfloat16 only")
+
+
+def _rows_view(x):
+    if not x.is_cuda:
+        raise ProfkError("input must be a CUDA tensor")
+    if x.dim() == 1:
+        x = x.unsqueeze(0)
+    if x.dim() != 2 or not x.is_contiguous():
+        raise ProfkError("input must be a contiguous (N,) or (rows, N) tensor")
+    return x
+
+
+def topk(x, k: int, eps: float = 1e-3, recall: float = 1.0, seed: int = 0, plan_override: Plan | None = None,
+         out=None):
+    """`profk_topk_*` / `profk_topk_planned_*` on the current stream.
+
+    x: CUDA tensor (N,) or (rows, N), float32 or bfloat16.  Returns (values, indices) with
+    shapes (rows, k) (or (k,) for 1-D input); nothing is synchronised.
+    """
+    import torch
+
+    one_d = x.dim() == 1
+    x2 = _rows_view(x)
+    rows, n = x2.shape
+    pl = plan_override if plan_override is not None else plan(n, k, eps, recall)
+    ensure_workspace(rows, pl.capacity, k, x2.device)
+    if out is None:
+        vals = torch.empty((rows, k), dtype=x2.dtype, device=x2.device)
+        idx = torch.empty((rows, k), dtype=torch.int64, device=x2.device)
+    else:
+        vals, idx = out
+    sfx = _suffix(x2)
+    with torch.cuda.device(x2.device):
+        if plan_override is None:
+            fn = getattr(lib(), f"profk_topk_{sfx}")
+            code = fn(ctypes.c_void_p(x2.data_ptr()), ctypes.c_int64(rows), ctypes.c_int64(n), ctypes.c_int64(k),
+                      ctypes.c_double(eps), ctypes.c_double(recall), ctypes.c_uint64(seed), _stream_ptr(),
+                      ctypes.c_void_p(vals.data_ptr()), ctypes.c_void_p(idx.data_ptr()))
+        else:
+            st = pl._struct()
+            fn = getattr(lib(), f"profk_topk_planned_{sfx}")
+            code = fn(ctypes.c_void_p(x2.data_ptr()), ctypes.c_int64(rows), ctypes.c_int64(n), ctypes.c_int64(k),
+                      ctypes.byref(st), ctypes.c_uint64(seed), _stream_ptr(),
+                      ctypes.c_void_p(vals.data_ptr()), ctypes.c_void_p(idx.data_ptr()))
+    _check(code, "profk_topk")
+    if one_d:
+        return vals[0], idx[0]
+    return vals, idx
+
+
+def filter_pass(x, tau, capacity: int):
+    """`profk_filter_*`: stage 3 alone.  Returns (records uint64 as int64 tensor (rows, capacity), counts int32 (rows,))."""
+    import torch
+
+    x2 = _rows_view(x)
+    rows, n = x2.shape
+    tau = tau.reshape(rows).contiguous()
+    buf = torch.empty((rows, capacity), dtype=torch.int64, device=x2.device)
+    counts = torch.zeros(rows, dtype=torch.int32, device=x2.device)
+    fn = getattr(lib(), f"profk_filter_{_suffix(x2)}")
+    with torch.cuda.device(x2.device):
+        code = fn(ctypes.c_void_p(x2.data_ptr()), ctypes.c_int64(rows), ctypes.c_int64(n), ctypes.c_void_p(tau.data_ptr()),
+                  ctypes.c_int64(capacity), ctypes.c_void_p(buf.data_ptr()), ctypes.c_void_p(counts.data_ptr()), _stream_ptr())
+    _check(code, "profk_filter")
+    return buf, counts
+
+
+def sample_threshold(x, m: int, r: int, seed: int, want_indices: bool = False):
+    """`profk_sample_threshold_*`: stages 1-2 alone.  Returns tau (rows,) and optionally the sampled indices."""
+    import torch
+
+    x2 = _rows_view(x)
+    rows, n = x2.shape
+    tau = torch.empty(rows, dtype=x2.dtype, device=x2.device)
+    sidx = torch.empty((rows, m), dtype=torch.int32, device=x2.device) if want_indices else None
+    fn = getattr(lib(), f"profk_sample_threshold_{_suffix(x2)}")
+    with torch.cuda.device(x2.device):
+        code = fn(ctypes.c_void_p(x2.data_ptr()), ctypes.c_int64(rows), ctypes.c_int64(n), ctypes.c_int64(m),
+                  ctypes.c_int64(r), ctypes.c_uint64(seed), ctypes.c_void_p(tau.data_ptr()),
+                  ctypes.c_void_p(sidx.data_ptr() if want_indices else None), _stream_ptr())
+    _check(code, "profk_sample_threshold")
+    return (tau, sidx) if want_indices else tau
+
+
+def read_stats(rows: int):
+    """`profk_read_stats`: list of (tau_bits, survivors, capacity, status) for the last call; synchronises."""
+    arr = (_StatsStruct * rows)()
+    _check(lib().profk_read_stats(_stream_ptr(), ctypes.c_int64(rows), arr), "profk_read_stats")
+    return [(s.tau_bits, s.survivors, s.capacity, s.status) for s in arr]
+
+
+def last_launch_count() -> int:
+    return int(lib().profk_last_launch_count())

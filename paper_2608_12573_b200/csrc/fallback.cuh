@@ -1,0 +1,214 @@
+// Count check and exact replacement (Section 3, "Refinement": "if fewer than k candidates
+// are collected, or if the buffer overflows ..., falls back to an exact top-k computation
+// on the full input").  The decision is taken on the device: this kernel reads the
+// per-row survivor counters, and for every row that failed it selects the exact top-k of
+// the whole row into the row's candidate buffer, so that the refine kernel that follows
+// orders the buffer the same way for every row.
+//
+// The exact selection is a most-significant-digit radix select over 64-bit candidate
+// records (value key, then index), 11 bits per pass, run by the whole grid with a grid
+// barrier after each pass.  The kernel is launched cooperatively so that all CTAs are
+// co-resident; every wait is bounded and reports through the workspace header.
+#pragma once
+
+#include "rowscan.cuh"
+#include "sample_select.cuh"
+
+namespace profk {
+
+constexpr int FB_THREADS = 512;
+constexpr int FB_UNROLL = 4;
+constexpr int FB_BINS = 2048;
+constexpr int FB_PASSES = 6;                // 5 x 11 bits + 9 bits = 64
+constexpr uint32_t SPIN_LIMIT = 1u << 24;   // polls (each ~100 ns apart) before a wait gives up
+
+enum : uint32_t { ROW_OK = 0, ROW_RECALL = 1, ROW_OVERFLOW = 2, ROW_DIRECT = 3, ROW_TIMEOUT_BIT = 0x80000000u };
+
+template <typename T> struct FallbackParams {
+    const T* in;
+    uint64_t N;
+    uint64_t rows;
+    uint32_t k;
+    uint32_t k_accept;
+    uint32_t capacity;
+    int mode;                 // 1 = every row takes the exact path
+    RowCtl* ctl;
+    WsHeader* header;
+    uint32_t* ghist;          // FB_PASSES x FB_BINS global histogram
+    uint64_t* buf;            // rows x capacity records
+    uint64_t tiles_per_row;
+};
+
+// Sense-free generation barrier over all CTAs of a co-resident grid.  Returns false when
+// the wait gave up (or an earlier one did); the caller then leaves the kernel.
+__device__ __forceinline__ bool grid_barrier(WsHeader* h, uint32_t& gen) {
+    __shared__ uint32_t s_ok;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t ok = 1;
+        __threadfence();
+        const uint32_t arrived = atomicAdd(&h->bar_count, 1u);
+        if (arrived == gridDim.x - 1) {
+            atomicExch(&h->bar_count, 0u);
+            __threadfence();
+            atomicAdd(&h->bar_gen, 1u);
+        } else {
+            uint32_t polls = 0;
+            while (*((volatile uint32_t*)&h->bar_gen) == gen) {
+                __nanosleep(64);
+                if (++polls > SPIN_LIMIT) { atomicExch(&h->error, 1u); ok = 0; break; }
+            }
+        }
+        __threadfence();
+        if (*((volatile uint32_t*)&h->error) != 0) ok = 0;
+        s_ok = ok;
+    }
+    __syncthreads();
+    gen += 1;
+    return s_ok != 0;
+}
+
+// Visits every element of `row` that falls to this CTA (tiles blockIdx.x, +gridDim.x, ...):
+// f(record, valid) is called by all 32 lanes of each warp together.
+template <typename T, typename F>
+__device__ __forceinline__ void for_each_record(const FallbackParams<T>& p, uint64_t row, F&& f) {
+    using V = typename Elem<T>::vec_t;
+    constexpr int VEC = Elem<T>::VEC;
+    constexpr uint32_t TILE_VECTORS = FB_THREADS * FB_UNROLL;
+    const RowView<T> rv = row_view(p.in, p.N, row);
+    for (uint64_t tile = blockIdx.x; tile < p.tiles_per_row; tile += gridDim.x) {
+        V v[FB_UNROLL];
+        bool inside[FB_UNROLL];
+#pragma unroll
+        for (int u = 0; u < FB_UNROLL; ++u)
+            v[u] = load_row_vector(rv, p.N, tile * TILE_VECTORS + (uint64_t)u * FB_THREADS + threadIdx.x, &inside[u]);
+#pragma unroll
+        for (int u = 0; u < FB_UNROLL; ++u) {
+            const uint64_t q = tile * TILE_VECTORS + (uint64_t)u * FB_THREADS + threadIdx.x;
+            const int64_t i0 = (int64_t)(q * VEC) - (int64_t)rv.mis;
+#pragma unroll
+            for (int l = 0; l < VEC; ++l) {
+                const int64_t i = i0 + l;
+                const bool valid = inside[u] && i >= 0 && i < (int64_t)p.N;
+                f(make_record(Elem<T>::key(vec_elem(v[u], l)), (uint32_t)i), valid);
+            }
+        }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackParams<T> p) {
+    __shared__ uint32_t sh_hist[FB_BINS];
+    __shared__ uint32_t warp_sums[32];
+    __shared__ uint32_t flag_masks[FB_THREADS / 32];
+    __shared__ uint32_t s_digit, s_before, s_cnt;
+
+    const unsigned tid = threadIdx.x, lane = lane_id(), warp = tid >> 5;
+    pdl_launch_dependents();
+
+    uint32_t gen = *((volatile uint32_t*)&p.header->bar_gen);   // read before this CTA's first arrival
+
+    for (uint64_t chunk = 0; chunk < p.rows; chunk += FB_THREADS) {
+        // ---- count check for FB_THREADS rows at a time; every CTA takes the same decisions ----
+        const uint64_t r = chunk + tid;
+        bool failed = false;
+        if (r < p.rows) {
+            const uint32_t R = p.ctl[r].count;
+            uint32_t status = ROW_OK;
+            if (p.mode == 1) status = ROW_DIRECT;
+            else if (R > p.capacity) status = ROW_OVERFLOW;
+            else if (R < p.k_accept) status = ROW_RECALL;
+            failed = status != ROW_OK;
+            if (blockIdx.x == 0) {
+                p.ctl[r].status = status;
+                p.ctl[r].n_final = failed ? p.k : R;
+            }
+        }
+        const unsigned m = __ballot_sync(FULL_MASK, failed);
+        if (lane == 0) flag_masks[warp] = m;
+        __syncthreads();
+
+        for (unsigned w = 0; w < FB_THREADS / 32; ++w) {
+            unsigned mask = flag_masks[w];
+            while (mask) {
+                const unsigned b = __ffs(mask) - 1;
+                mask &= mask - 1;
+                const uint64_t row = chunk + w * 32 + b;
+
+                // ---- exact selection of the k smallest records of `row` ----
+                if (!grid_barrier(p.header, gen)) return;          // previous row's histogram reads are over
+                for (uint32_t i = blockIdx.x * FB_THREADS + tid; i < FB_PASSES * FB_BINS; i += gridDim.x * FB_THREADS)
+                    p.ghist[i] = 0;
+                if (!grid_barrier(p.header, gen)) return;
+
+                uint64_t prefix = 0;       // selected high bits, right-aligned
+                uint32_t need = p.k;       // rank (from the smallest record) inside the prefix class
+                uint64_t limit = ~0ull;    // records <= limit are the answer
+                for (int pass = 0; pass < FB_PASSES; ++pass) {
+                    const int shift = pass < 5 ? 53 - 11 * pass : 0;
+                    const int width = pass < 5 ? 11 : 9;
+                    const uint32_t nbins = 1u << width;
+                    for (uint32_t i = tid; i < nbins; i += FB_THREADS) sh_hist[i] = 0;
+                    __syncthreads();
+                    for_each_record(p, row, [&](uint64_t rec, bool valid) {
+                        const bool in_class = valid && (pass == 0 || (rec >> (shift + width)) == prefix);
+                        const uint32_t digit = in_class ? (uint32_t)(rec >> shift) & (nbins - 1) : 0xFFFFFFFFu;
+                        const unsigned peers = __match_any_sync(FULL_MASK, digit);
+                        if (in_class && lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&sh_hist[digit], __popc(peers));
+                    });
+                    __syncthreads();
+                    uint32_t* gh = p.ghist + pass * FB_BINS;
+                    for (uint32_t i = tid; i < nbins; i += FB_THREADS) {
+                        const uint32_t c = sh_hist[i];
+                        if (c) atomicAdd(&gh[i], c);
+                    }
+                    if (!grid_barrier(p.header, gen)) return;
+
+                    // Every CTA finds the bin that holds the need-th smallest record of the class.
+                    constexpr int PER = FB_BINS / FB_THREADS;                   // bins per thread
+                    uint32_t c[PER], sum = 0;
+#pragma unroll
+                    for (int j = 0; j < PER; ++j) {
+                        const uint32_t bin = tid * PER + j;
+                        c[j] = bin < nbins ? __ldcg(&gh[bin]) : 0;
+                        sum += c[j];
+                    }
+                    uint32_t before = block_inclusive_scan(sum, warp_sums) - sum;
+#pragma unroll
+                    for (int j = 0; j < PER; ++j) {
+                        if (before < need && need <= before + c[j]) { s_digit = tid * PER + j; s_before = before; s_cnt = c[j]; }
+                        before += c[j];
+                    }
+                    __syncthreads();
+                    prefix = (prefix << width) | s_digit;
+                    need -= s_before;
+                    const bool whole_bin = (s_cnt == need);
+                    __syncthreads();
+                    if (whole_bin || pass == FB_PASSES - 1) {
+                        limit = ((prefix + 1) << shift) - 1;        // wraps to all-ones when the class is the last one
+                        break;
+                    }
+                }
+
+                // ---- collect the k records <= limit into the row's buffer ----
+                uint64_t* dst = p.buf + row * (uint64_t)p.capacity;
+                uint32_t* counter = &p.ctl[row].collect;
+                const unsigned lt_mask = (1u << lane) - 1u;
+                for_each_record(p, row, [&](uint64_t rec, bool valid) {
+                    const bool take = valid && rec <= limit;
+                    const unsigned bal = __ballot_sync(FULL_MASK, take);
+                    if (bal) {
+                        unsigned base = 0;
+                        if (lane == 0) base = atomicAdd(counter, __popc(bal));
+                        base = __shfl_sync(FULL_MASK, base, 0);
+                        const unsigned pos = base + __popc(bal & lt_mask);
+                        if (take && pos < p.capacity) dst[pos] = rec;
+                    }
+                });
+            }
+        }
+        __syncthreads();   // flag_masks is rewritten by the next chunk
+    }
+}
+
+}  // namespace profk

@@ -1,0 +1,137 @@
+// Stage 3, the filtering scan (Section 3, "Filtering"): stream every row once and append
+// each element with x_i >= tau to the row's candidate buffer.
+//
+// The kernel is bound by HBM bandwidth: one 128-bit load per VEC elements, one compare
+// per element, and nothing else on the common path.  Survivors are rare (1e-3 .. 1e-5 of
+// the elements), so the append is a warp-cooperative slow path taken only when some lane
+// of the warp saw a survivor: a warp prefix sum and one global atomic per warp.
+#pragma once
+
+#include "rowscan.cuh"
+
+namespace profk {
+
+template <typename T> struct FilterParams {
+    const T* in;
+    uint64_t N;
+    uint64_t rows;
+    const T* tau;            // rows thresholds
+    uint32_t capacity;       // records per row buffer
+    uint64_t* buf;           // rows x capacity records
+    uint32_t* counts;        // per-row survivor counter (stride in 32-bit words)
+    uint32_t count_stride;
+    uint64_t tiles_per_row;
+    uint64_t total_tiles;
+    int use_pdl;             // 1 = launched as a programmatic dependent of the threshold kernel
+};
+
+// not (x < tau) for every lane of a vector, OR-ed: does the vector hold any survivor?
+__device__ __forceinline__ bool vec_any_pass(const float4& v, float tau) {
+    return !(v.x < tau) | !(v.y < tau) | !(v.z < tau) | !(v.w < tau);
+}
+__device__ __forceinline__ bool vec_any_pass(const uint4& v, __nv_bfloat16 tau) {
+    const __nv_bfloat162 t2 = __halves2bfloat162(tau, tau);
+    const unsigned a = __hlt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&v.x), t2);
+    const unsigned b = __hlt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&v.y), t2);
+    const unsigned c = __hlt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&v.z), t2);
+    const unsigned d = __hlt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&v.w), t2);
+    return (a & b & c & d) != 0xFFFFFFFFu;    // some lane is not below tau
+}
+
+template <typename T, int THREADS, int UNROLL>
+__global__ void __launch_bounds__(THREADS) filter_kernel(const FilterParams<T> p) {
+    using V = typename Elem<T>::vec_t;
+    constexpr int VEC = Elem<T>::VEC;
+    constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
+
+    const unsigned lane = lane_id();
+
+    uint64_t tile = blockIdx.x;
+    if (tile >= p.total_tiles) return;
+
+    // Decode the first tile and issue its loads before waiting on the threshold kernel:
+    // the input does not depend on it.
+    uint64_t row = tile / p.tiles_per_row;
+    uint64_t trow = tile - row * p.tiles_per_row;
+    RowView<T> rv = row_view(p.in, p.N, row);
+    V v[UNROLL];
+    bool inside[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u)
+        v[u] = load_row_vector(rv, p.N, trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x, &inside[u]);
+
+    if (p.use_pdl) pdl_wait();
+
+    uint64_t skip_row = ~0ull;    // row whose buffer this warp has seen overflow: nothing more to append
+    while (true) {
+        const T tau = p.tau[row];
+        bool hit = false;
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) hit |= (inside[u] && vec_any_pass(v[u], tau));
+
+        if (__any_sync(FULL_MASK, hit) && row != skip_row) {
+            // Slow path: exact per-element test; a warp-wide prefix sum of the per-lane
+            // survivor counts places every lane's records behind one atomic per warp.
+            const float tau_f = Elem<T>::as_float(tau);
+            unsigned mine[UNROLL];          // per vector: bit l set = element l survives
+            unsigned cnt = 0;
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                mine[u] = 0;
+                const uint64_t q = trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
+                const int64_t i0 = (int64_t)(q * VEC) - (int64_t)rv.mis;
+#pragma unroll
+                for (int l = 0; l < VEC; ++l) {
+                    const int64_t i = i0 + l;
+                    const bool ok = inside[u] && i >= 0 && i < (int64_t)p.N &&
+                                    !(Elem<T>::as_float(vec_elem(v[u], l)) < tau_f);
+                    if (ok) mine[u] |= 1u << l;
+                }
+                cnt += __popc(mine[u]);
+            }
+            unsigned incl = cnt;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const unsigned nb = __shfl_up_sync(FULL_MASK, incl, d);
+                if (lane >= (unsigned)d) incl += nb;
+            }
+            const unsigned total = __shfl_sync(FULL_MASK, incl, 31);
+            unsigned base = 0;
+            if (lane == 0 && total) base = atomicAdd(p.counts + row * p.count_stride, total);
+            base = __shfl_sync(FULL_MASK, base, 0);
+            unsigned pos = base + incl - cnt;
+            uint64_t* dst = p.buf + row * (uint64_t)p.capacity;
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                if (mine[u]) {
+                    const uint64_t q = trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
+                    const int64_t i0 = (int64_t)(q * VEC) - (int64_t)rv.mis;
+#pragma unroll
+                    for (int l = 0; l < VEC; ++l) {
+                        if (mine[u] & (1u << l)) {
+                            if (pos < p.capacity)
+                                dst[pos] = make_record(Elem<T>::key(vec_elem(v[u], l)), (uint32_t)(i0 + l));
+                            ++pos;
+                        }
+                    }
+                }
+            }
+            if ((uint64_t)base + total > p.capacity) skip_row = row;   // overflow: the exact path will redo this row
+        }
+
+        // Next tile of this CTA; tiles of a row already known to overflow are not even loaded.
+        uint64_t nrow;
+        do {
+            tile += gridDim.x;
+            if (tile >= p.total_tiles) return;
+            nrow = tile / p.tiles_per_row;
+        } while (nrow == skip_row);
+        trow = tile - nrow * p.tiles_per_row;
+        if (nrow != row) { row = nrow; rv = row_view(p.in, p.N, row); }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u)
+            v[u] = load_row_vector(rv, p.N, trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x, &inside[u]);
+    }
+}
+
+}  // namespace profk

@@ -1,0 +1,406 @@
+// C ABI of the library (see profk.h): argument checks, workspace layout and the launch
+// sequence  threshold -> filter -> count check / exact replacement -> refine.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <tuple>
+#include <vector>
+
+#include "fallback.cuh"
+#include "filter.cuh"
+#include "profk.h"
+#include "refine.cuh"
+#include "sample_select.cuh"
+
+using namespace profk;
+
+namespace {
+
+constexpr int FILTER_THREADS = 512;
+constexpr int FILTER_UNROLL = 4;
+constexpr uint32_t SORT_CAP_MAX = 8192;          // largest k the single-CTA refine orders in shared memory
+constexpr size_t REFINE_SMEM_MAX = 200 * 1024;   // dynamic shared memory the refine kernel may ask for
+constexpr int64_t N_MAX = 4278190080LL;          // 2^32 - 2^24
+constexpr int64_t M_MAX = 262144;                // largest sample the cluster select holds (8 CTAs x 32768 keys)
+
+thread_local int g_launches = 0;
+
+struct DeviceInfo {
+    int sm_count = 0;
+    int filter_blocks_per_sm[2] = {0, 0};     // by dtype
+    int fallback_blocks_per_sm[2] = {0, 0};
+    bool ready = false;
+};
+
+struct Workspace { void* ptr = nullptr; size_t bytes = 0; };
+
+std::mutex g_mutex;
+std::map<int, DeviceInfo> g_devinfo;
+std::map<int, Workspace> g_workspace;
+std::map<std::tuple<int64_t, int64_t, double, double>, profk_plan_t> g_plan_cache;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct WsLayout {
+    size_t off_header, off_ghist, off_ctl, off_tau, off_buf, total;
+};
+
+WsLayout ws_layout(int64_t rows, int64_t capacity) {
+    WsLayout l;
+    l.off_header = 0;
+    l.off_ghist = sizeof(WsHeader);
+    l.off_ctl = align_up(l.off_ghist + (size_t)FB_PASSES * FB_BINS * sizeof(uint32_t), 256);
+    l.off_tau = align_up(l.off_ctl + (size_t)rows * sizeof(RowCtl), 256);
+    l.off_buf = align_up(l.off_tau + (size_t)rows * 4, 256);
+    l.total = align_up(l.off_buf + (size_t)rows * (size_t)capacity * sizeof(uint64_t), 256);
+    return l;
+}
+
+#define CUDA_TRY(expr)                                   \
+    do {                                                 \
+        cudaError_t _e = (expr);                         \
+        if (_e != cudaSuccess) { (void)cudaGetLastError(); return PROFK_ECUDA; } \
+    } while (0)
+
+template <typename T> constexpr int dtype_index() { return sizeof(T) == 4 ? 0 : 1; }
+
+template <typename T> int ensure_device_info(int dev, DeviceInfo* out) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceInfo& di = g_devinfo[dev];
+    if (!di.ready) {
+        CUDA_TRY(cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev));
+        di.ready = true;
+    }
+    const int d = dtype_index<T>();
+    if (di.filter_blocks_per_sm[d] == 0) {
+        int nb = 0;
+        CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL>,
+                                                                 FILTER_THREADS, 0));
+        di.filter_blocks_per_sm[d] = std::max(nb, 1);
+        CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fallback_kernel<T>, FB_THREADS, 0));
+        di.fallback_blocks_per_sm[d] = std::max(nb, 1);
+        CUDA_TRY(cudaFuncSetAttribute(sample_select_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
+        CUDA_TRY(cudaFuncSetAttribute(refine_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFINE_SMEM_MAX));
+    }
+    *out = di;
+    return PROFK_OK;
+}
+
+__global__ void init_ctl_kernel(RowCtl* ctl, uint64_t rows, WsHeader* header, uint32_t capacity) {
+    const uint64_t r = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < rows) {
+        RowCtl* c = ctl + r;
+        c->tau_bits = 0; c->count = 0; c->collect = 0; c->status = 0; c->n_final = 0; c->capacity = capacity;
+    }
+    if (r == 0) { header->bar_count = 0; header->error = 0; }
+}
+
+// Cluster size for the threshold kernel: spread one row's gather over several SMs when
+// there are few rows; never more keys per CTA than its shared memory holds.
+int pick_cluster(int64_t rows, int64_t m) {
+    int c = rows <= 18 ? 8 : rows <= 37 ? 4 : rows <= 74 ? 2 : 1;
+    while (c < 8 && (m + c - 1) / c > 32768) c *= 2;
+    return c;
+}
+
+template <typename T>
+int launch_sample_select(const T* in, int64_t rows, int64_t N, int64_t m, int64_t r, uint64_t seed, T* tau, RowCtl* ctl,
+                         WsHeader* header, uint32_t capacity, uint32_t* sample_idx, cudaStream_t st) {
+    const int csize = pick_cluster(rows, m);
+    SelectParams<T> sp;
+    sp.in = in; sp.N = (uint64_t)N; sp.S = (uint32_t)m; sp.t = (uint32_t)r; sp.seed = seed;
+    sp.per_cta = (uint32_t)((m + csize - 1) / csize);
+    sp.tau = tau; sp.ctl = ctl; sp.header = header; sp.capacity = capacity; sp.sample_idx = sample_idx;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(rows * csize));
+    cfg.blockDim = dim3(SEL_THREADS);
+    cfg.dynamicSmemBytes = (size_t)sp.per_cta * sizeof(uint32_t);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, sample_select_kernel<T>, sp));
+    ++g_launches;
+    return PROFK_OK;
+}
+
+template <typename T>
+int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, const T* tau, int64_t capacity, uint64_t* buf,
+                  uint32_t* counts, uint32_t count_stride, bool pdl, cudaStream_t st) {
+    FilterParams<T> fp;
+    fp.in = in; fp.N = (uint64_t)N; fp.rows = (uint64_t)rows; fp.tau = tau; fp.capacity = (uint32_t)capacity;
+    fp.buf = buf; fp.counts = counts; fp.count_stride = count_stride;
+    fp.tiles_per_row = tiles_per_row<T>((uint64_t)N, FILTER_THREADS * FILTER_UNROLL);
+    fp.total_tiles = fp.tiles_per_row * (uint64_t)rows;
+    fp.use_pdl = pdl ? 1 : 0;
+    const uint64_t max_grid = (uint64_t)di.sm_count * di.filter_blocks_per_sm[dtype_index<T>()];
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)std::min<uint64_t>(fp.total_tiles, max_grid));
+    cfg.blockDim = dim3(FILTER_THREADS);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL>, fp));
+    ++g_launches;
+    return PROFK_OK;
+}
+
+template <typename T>
+int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_plan_t* plan, uint64_t seed, void* stream,
+                 T* out_vals, int64_t* out_idx) {
+    g_launches = 0;
+    if (!in || !out_vals || !out_idx || !plan) return PROFK_EINVAL;
+    if (rows < 1 || N < 1 || N > N_MAX || k < 1 || k > N) return PROFK_EINVAL;
+    if (((uintptr_t)in % sizeof(T)) || ((uintptr_t)out_vals % sizeof(T)) || ((uintptr_t)out_idx % 8)) return PROFK_EINVAL;
+    const int64_t capacity = plan->capacity;
+    if (capacity < k || capacity > N || rows * capacity >= (1LL << 40)) return PROFK_EINVAL;
+    if (plan->mode != 0 && plan->mode != 1) return PROFK_EINVAL;
+    if (plan->mode == 0) {
+        if (plan->m < 1 || plan->m > std::min<int64_t>(N, M_MAX) || plan->r < 1 || plan->r > plan->m) return PROFK_EINVAL;
+        if (plan->k_accept < 1 || plan->k_accept > k) return PROFK_EINVAL;
+    }
+    if (k > SORT_CAP_MAX) return PROFK_EINVAL;   // larger selections need the multi-CTA sort
+
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    DeviceInfo di;
+    int rc = ensure_device_info<T>(dev, &di);
+    if (rc != PROFK_OK) return rc;
+
+    Workspace ws;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        ws = g_workspace[dev];
+    }
+    const WsLayout lay = ws_layout(rows, capacity);
+    if (!ws.ptr || ws.bytes < lay.total) return PROFK_EWORKSPACE;
+    unsigned char* base = static_cast<unsigned char*>(ws.ptr);
+    WsHeader* header = reinterpret_cast<WsHeader*>(base + lay.off_header);
+    uint32_t* ghist = reinterpret_cast<uint32_t*>(base + lay.off_ghist);
+    RowCtl* ctl = reinterpret_cast<RowCtl*>(base + lay.off_ctl);
+    T* tau = reinterpret_cast<T*>(base + lay.off_tau);
+    uint64_t* buf = reinterpret_cast<uint64_t*>(base + lay.off_buf);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    if (plan->mode == 0) {
+        rc = launch_sample_select<T>(in, rows, N, plan->m, plan->r, seed, tau, ctl, header, (uint32_t)capacity, nullptr, st);
+        if (rc != PROFK_OK) return rc;
+        rc = launch_filter<T>(di, in, rows, N, tau, capacity, buf, &ctl[0].count, sizeof(RowCtl) / 4, true, st);
+        if (rc != PROFK_OK) return rc;
+    } else {
+        init_ctl_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(ctl, (uint64_t)rows, header, (uint32_t)capacity);
+        CUDA_TRY(cudaGetLastError());
+        ++g_launches;
+    }
+
+    {   // count check + exact replacement of failed rows (cooperative: all CTAs co-resident)
+        FallbackParams<T> fb;
+        fb.in = in; fb.N = (uint64_t)N; fb.rows = (uint64_t)rows; fb.k = (uint32_t)k;
+        fb.k_accept = (uint32_t)(plan->mode == 0 ? plan->k_accept : k);
+        fb.capacity = (uint32_t)capacity; fb.mode = plan->mode; fb.ctl = ctl; fb.header = header; fb.ghist = ghist; fb.buf = buf;
+        fb.tiles_per_row = tiles_per_row<T>((uint64_t)N, FB_THREADS * FB_UNROLL);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(di.sm_count * di.fallback_blocks_per_sm[dtype_index<T>()]));
+        cfg.blockDim = dim3(FB_THREADS);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        CUDA_TRY(cudaLaunchKernelEx(&cfg, fallback_kernel<T>, fb));
+        ++g_launches;
+    }
+
+    {   // refine: order the buffer of every row
+        RefineParams<T> rp;
+        rp.ctl = ctl; rp.buf = buf; rp.capacity = (uint32_t)capacity; rp.k = (uint32_t)k;
+        uint32_t sort_cap = 32;
+        while (sort_cap < (uint32_t)k) sort_cap <<= 1;
+        // small buffers are sorted whole, skipping the select
+        while (sort_cap < 2048 && sort_cap < (uint32_t)capacity) sort_cap <<= 1;
+        rp.sort_cap = sort_cap;
+        const size_t room = (REFINE_SMEM_MAX - (size_t)sort_cap * 8) / 8;
+        rp.stage_cap = (uint32_t)std::min<size_t>((size_t)capacity, room);
+        if (rp.stage_cap <= sort_cap) rp.stage_cap = 0;
+        rp.out_vals = out_vals; rp.out_idx = out_idx; rp.use_pdl = 1;
+        unsigned threads = 128;
+        while (threads < 1024 && threads * 8 < (unsigned)capacity) threads <<= 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)rows);
+        cfg.blockDim = dim3(threads);
+        cfg.dynamicSmemBytes = ((size_t)sort_cap + rp.stage_cap) * 8;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        CUDA_TRY(cudaLaunchKernelEx(&cfg, refine_kernel<T>, rp));
+        ++g_launches;
+    }
+    return PROFK_OK;
+}
+
+template <typename T>
+int topk_auto(const T* in, int64_t rows, int64_t N, int64_t k, double eps, double recall, uint64_t seed, void* stream,
+              T* out_vals, int64_t* out_idx) {
+    profk_plan_t plan;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        const auto key = std::make_tuple(N, k, eps, recall);
+        auto it = g_plan_cache.find(key);
+        if (it == g_plan_cache.end()) {
+            const int rc = profk_plan(N, k, eps, recall, &plan);
+            if (rc != PROFK_OK) return rc;
+            if (g_plan_cache.size() > 4096) g_plan_cache.clear();
+            g_plan_cache[key] = plan;
+        } else {
+            plan = it->second;
+        }
+    }
+    return topk_planned<T>(in, rows, N, k, &plan, seed, stream, out_vals, out_idx);
+}
+
+template <typename T>
+int filter_only(const T* in, int64_t rows, int64_t N, const T* tau, int64_t capacity, uint64_t* buf_keys, uint32_t* counts,
+                void* stream) {
+    if (!in || !tau || !buf_keys || !counts) return PROFK_EINVAL;
+    if (rows < 1 || N < 1 || N > N_MAX || capacity < 1 || capacity > N_MAX) return PROFK_EINVAL;
+    if ((uintptr_t)in % sizeof(T) || (uintptr_t)tau % sizeof(T) || (uintptr_t)buf_keys % 8 || (uintptr_t)counts % 4)
+        return PROFK_EINVAL;
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    DeviceInfo di;
+    const int rc = ensure_device_info<T>(dev, &di);
+    if (rc != PROFK_OK) return rc;
+    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, counts, 1, false, static_cast<cudaStream_t>(stream));
+}
+
+template <typename T>
+int sample_threshold(const T* in, int64_t rows, int64_t N, int64_t m, int64_t r, uint64_t seed, T* tau, uint32_t* sample_idx,
+                     void* stream) {
+    if (!in || !tau) return PROFK_EINVAL;
+    if (rows < 1 || N < 1 || N > N_MAX || m < 1 || m > std::min<int64_t>(N, M_MAX) || r < 1 || r > m) return PROFK_EINVAL;
+    if ((uintptr_t)in % sizeof(T) || (uintptr_t)tau % sizeof(T) || (uintptr_t)sample_idx % 4) return PROFK_EINVAL;
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    DeviceInfo di;
+    const int rc = ensure_device_info<T>(dev, &di);
+    if (rc != PROFK_OK) return rc;
+    return launch_sample_select<T>(in, rows, N, m, r, seed, tau, nullptr, nullptr, 0, sample_idx, static_cast<cudaStream_t>(stream));
+}
+
+}  // namespace
+
+// --------------------------------------------------------------------------------------- C ABI
+extern "C" {
+
+int profk_workspace_bytes(int64_t rows, int64_t capacity, int64_t k, size_t* bytes) {
+    if (!bytes || rows < 1 || capacity < 1 || k < 1 || capacity < k || capacity > N_MAX || rows * capacity >= (1LL << 40))
+        return PROFK_EINVAL;
+    *bytes = ws_layout(rows, capacity).total;
+    return PROFK_OK;
+}
+
+int profk_set_workspace(void* dev_ptr, size_t bytes) {
+    if ((dev_ptr == nullptr) != (bytes == 0)) return PROFK_EINVAL;
+    if ((uintptr_t)dev_ptr % 256) return PROFK_EINVAL;
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(g_mutex);
+    g_workspace[dev] = Workspace{dev_ptr, bytes};
+    return PROFK_OK;
+}
+
+int profk_topk_f32(const float* in, int64_t rows, int64_t N, int64_t k, double eps, double recall, uint64_t seed,
+                   void* stream, float* out_vals, int64_t* out_idx) {
+    return topk_auto<float>(in, rows, N, k, eps, recall, seed, stream, out_vals, out_idx);
+}
+
+int profk_topk_bf16(const void* in, int64_t rows, int64_t N, int64_t k, double eps, double recall, uint64_t seed,
+                    void* stream, void* out_vals, int64_t* out_idx) {
+    return topk_auto<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(in), rows, N, k, eps, recall, seed, stream,
+                                    static_cast<__nv_bfloat16*>(out_vals), out_idx);
+}
+
+int profk_topk_planned_f32(const float* in, int64_t rows, int64_t N, int64_t k, const profk_plan_t* plan, uint64_t seed,
+                           void* stream, float* out_vals, int64_t* out_idx) {
+    return topk_planned<float>(in, rows, N, k, plan, seed, stream, out_vals, out_idx);
+}
+
+int profk_topk_planned_bf16(const void* in, int64_t rows, int64_t N, int64_t k, const profk_plan_t* plan, uint64_t seed,
+                            void* stream, void* out_vals, int64_t* out_idx) {
+    return topk_planned<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(in), rows, N, k, plan, seed, stream,
+                                       static_cast<__nv_bfloat16*>(out_vals), out_idx);
+}
+
+int profk_filter_f32(const float* in, int64_t rows, int64_t N, const float* tau, int64_t capacity, uint64_t* buf_keys,
+                     uint32_t* counts, void* stream) {
+    return filter_only<float>(in, rows, N, tau, capacity, buf_keys, counts, stream);
+}
+
+int profk_filter_bf16(const void* in, int64_t rows, int64_t N, const void* tau, int64_t capacity, uint64_t* buf_keys,
+                      uint32_t* counts, void* stream) {
+    return filter_only<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(in), rows, N, static_cast<const __nv_bfloat16*>(tau),
+                                      capacity, buf_keys, counts, stream);
+}
+
+int profk_sample_threshold_f32(const float* in, int64_t rows, int64_t N, int64_t m, int64_t r, uint64_t seed, float* tau,
+                               uint32_t* sample_idx, void* stream) {
+    return sample_threshold<float>(in, rows, N, m, r, seed, tau, sample_idx, stream);
+}
+
+int profk_sample_threshold_bf16(const void* in, int64_t rows, int64_t N, int64_t m, int64_t r, uint64_t seed, void* tau,
+                                uint32_t* sample_idx, void* stream) {
+    return sample_threshold<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(in), rows, N, m, r, seed,
+                                           static_cast<__nv_bfloat16*>(tau), sample_idx, stream);
+}
+
+int profk_read_stats(void* stream, int64_t rows, profk_row_stats_t* out) {
+    if (!out || rows < 1) return PROFK_EINVAL;
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    Workspace ws;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        ws = g_workspace[dev];
+    }
+    const WsLayout lay = ws_layout(rows, 1);
+    if (!ws.ptr || ws.bytes < lay.off_ctl + (size_t)rows * sizeof(RowCtl)) return PROFK_EWORKSPACE;
+    std::vector<RowCtl> host((size_t)rows);
+    WsHeader hdr;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char* base = static_cast<unsigned char*>(ws.ptr);
+    CUDA_TRY(cudaMemcpyAsync(host.data(), base + lay.off_ctl, (size_t)rows * sizeof(RowCtl), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaMemcpyAsync(&hdr, base + lay.off_header, sizeof(WsHeader), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    for (int64_t r = 0; r < rows; ++r) {
+        out[r].tau_bits = host[r].tau_bits;
+        out[r].survivors = host[r].count;
+        out[r].capacity = host[r].capacity;
+        out[r].status = host[r].status | (hdr.error ? 0x80000000u : 0u);
+    }
+    return PROFK_OK;
+}
+
+int profk_last_launch_count(void) { return g_launches; }
+
+const char* profk_strerror(int code) {
+    switch (code) {
+        case PROFK_OK: return "ok";
+        case PROFK_EINVAL: return "invalid argument";
+        case PROFK_EWORKSPACE: return "workspace missing or too small";
+        case PROFK_ECUDA: return "CUDA runtime error";
+        case PROFK_ETIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,246 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_12573_b200 as profk
+from oracle import philox as o_philox
+from oracle import plan as o_plan
+from oracle import stages as o_stages
+from oracle import topk as o_topk
+from paper_2608_12573_b200 import _build, workloads
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    _build.build()
+    profk.lib()
+    torch.cuda.set_device(0)
+
+
+def bits(a: np.ndarray) -> np.ndarray:
+    return a.view(np.uint32) if a.dtype == np.float32 else a.view(np.uint16)
+
+
+def gpu_topk(x: torch.Tensor, k: int, **kw):
+    v, i = profk.topk(x.cuda(), k, **kw)
+    torch.cuda.synchronize()
+    return workloads.as_numpy(v), i.cpu().numpy()
+
+
+def assert_exact(x: torch.Tensor, k: int, v: np.ndarray, i: np.ndarray):
+    xn = workloads.as_numpy(x)
+    ov, oi = o_topk.topk(xn, k)
+    assert np.array_equal(i, oi), "indices differ from the oracle"
+    assert np.array_equal(bits(v), bits(ov)), "values differ from the oracle"
+
+
+# ----------------------------------------------------------------------------- whole call
+def test_config1_uniform_2p20_k64():
+    x = workloads.uniform(1 << 20, seed=0)
+    v, i = gpu_topk(x, 64, eps=1e-3, seed=0)
+    assert_exact(x, 64, v, i)
+    tau_bits, R, cap, status = profk.read_stats(1)[0]
+    pl = o_plan.plan_guarded(1 << 20, 64, 1e-3)
+    res = o_stages.run_row(workloads.as_numpy(x), 64, pl.m, pl.r, pl.capacity, pl.k_accept, seed=0)
+    assert cap == pl.capacity
+    assert tau_bits == int(np.asarray([res.tau]).view(np.uint32)[0])        # same sample, same threshold
+    assert status == res.status
+    assert R == res.survivors or (res.survivors > cap and R > cap)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_result_does_not_depend_on_the_seed(seed):
+    x = workloads.normal(1, 1 << 18, seed=77)[0]
+    v, i = gpu_topk(x, 100, eps=1e-3, seed=seed)
+    assert_exact(x, 100, v, i)
+
+
+@pytest.mark.parametrize("n,k", [(1, 1), (2, 2), (5, 3), (33, 33), (1000, 1), (4097, 17), (65537, 256), (262145, 1000),
+                                 (1_000_003, 77), (3_000_001, 2999)])
+def test_ragged_sizes(n, k):
+    x = workloads.normal(1, n, seed=n)[0]
+    v, i = gpu_topk(x, k, eps=1e-3, seed=1)
+    assert_exact(x, k, v, i)
+
+
+def test_unaligned_base_pointer_and_odd_row_stride():
+    big = workloads.normal(1, 3 * 100_003 + 8, seed=5)[0].cuda()
+    for off in (1, 2, 3):
+        x = big[off: off + 3 * 100_003].view(3, 100_003)                     # rows start at odd element offsets
+        v, i = profk.topk(x, 50, eps=1e-3, seed=2)
+        torch.cuda.synchronize()
+        assert_exact(x.cpu(), 50, v.cpu().numpy(), i.cpu().numpy())
+    xb = big.to(torch.bfloat16)
+    for off in (1, 3, 7):
+        x = xb[off: off + 3 * 100_003].view(3, 100_003)
+        v, i = profk.topk(x, 50, eps=1e-3, seed=2)
+        torch.cuda.synchronize()
+        assert_exact(x.cpu(), 50, workloads.as_numpy(v), i.cpu().numpy())
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_batched_rows(dtype):
+    x = workloads.normal(24, 1 << 17, seed=2, dtype=dtype)
+    v, i = gpu_topk(x, 32, eps=1e-3, seed=9)
+    assert_exact(x, 32, v, i)
+    stats = profk.read_stats(24)
+    pl = o_plan.plan_guarded(1 << 17, 32, 1e-3)
+    xn = workloads.as_numpy(x)
+    for r in (0, 7, 23):
+        res = o_stages.run_row(xn[r], 32, pl.m, pl.r, pl.capacity, pl.k_accept, seed=9, row=r)
+        want_tau = int(np.asarray([res.tau]).view(np.uint32 if dtype == torch.float32 else np.uint16)[0])
+        assert stats[r][0] == want_tau and stats[r][3] == res.status
+        assert stats[r][1] == res.survivors or (res.survivors > pl.capacity and stats[r][1] > pl.capacity)
+
+
+# ----------------------------------------------------------------------------- forced failures
+def _forced(x, k, plan):
+    v, i = profk.topk(x.cuda(), k, plan_override=plan, seed=3)
+    torch.cuda.synchronize()
+    rows = 1 if x.dim() == 1 else x.shape[0]
+    return workloads.as_numpy(v), i.cpu().numpy(), profk.read_stats(rows)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_forced_overflow_recall_failure_and_direct_mode(dtype):
+    x = workloads.normal(5, 200_000, seed=11, dtype=dtype)
+    k = 64
+    # capacity == k: every row overflows
+    v, i, st = _forced(x, k, profk.Plan(m=4096, r=40, capacity=k, k_accept=k, mode=0))
+    assert_exact(x, k, v, i)
+    assert all(s[3] == profk.ROW_OVERFLOW for s in st)
+    # threshold = sample maximum: (almost) nothing survives
+    v, i, st = _forced(x, k, profk.Plan(m=65536, r=1, capacity=4096, k_accept=k, mode=0))
+    assert_exact(x, k, v, i)
+    assert all(s[3] == profk.ROW_RECALL and s[1] < k for s in st)
+    # direct exact selection
+    v, i, st = _forced(x, k, profk.Plan(m=0, r=0, capacity=k, k_accept=k, mode=1))
+    assert_exact(x, k, v, i)
+    assert all(s[3] == profk.ROW_DIRECT for s in st)
+
+
+def test_mixed_rows_some_fail():
+    # rows 0 and 2 hold many copies of their maximum, so their buffers overflow; the others do not
+    x = workloads.normal(4, 150_000, seed=12)
+    x[0, ::3] = 9.0
+    x[2, 1::2] = 7.5
+    v, i, st = _forced(x, 40, profk.Plan(m=2048, r=4, capacity=2000, k_accept=40, mode=0))
+    assert_exact(x, 40, v, i)
+    assert [s[3] for s in st] == [profk.ROW_OVERFLOW, profk.ROW_OK, profk.ROW_OVERFLOW, profk.ROW_OK]
+
+
+def test_k_equals_n_and_plan_direct_mode():
+    x = workloads.normal(1, 5000, seed=13)[0]
+    v, i = gpu_topk(x, 5000)
+    assert_exact(x, 5000, v, i)
+    x = workloads.normal(3, 40_000, seed=14)                                 # N <= 2 S: plan says mode 1
+    assert profk.plan(40_000, 10).mode == 1
+    v, i = gpu_topk(x, 10)
+    assert_exact(x, 10, v, i)
+
+
+# ----------------------------------------------------------------------------- ties and special values
+def test_ties_and_degenerate_inputs():
+    n = 300_000
+    for name in ("few_values", "spikes"):
+        recipe, seed = workloads.ADVERSARIAL[name]
+        x = recipe(n, seed)
+        for k in (1, 64, 1000):
+            v, i = gpu_topk(x, k, eps=1e-3, seed=4)
+            assert_exact(x, k, v, i)
+    x = torch.zeros(n)
+    v, i = gpu_topk(x, 100)
+    assert np.array_equal(i, np.arange(100))                                 # all equal: lowest indices win
+    x = workloads.sorted_uniform(n, 6)
+    v, i = gpu_topk(x, 500, eps=1e-3)
+    assert_exact(x, 500, v, i)
+    v, i = gpu_topk(torch.flip(x, [0]), 500, eps=1e-3)
+    assert_exact(torch.flip(x, [0]), 500, v, i)
+
+
+def test_nan_inf_and_signed_zero_follow_the_total_order():
+    x = workloads.normal(1, 100_000, seed=15)[0]
+    x[5] = float("nan"); x[77] = float("inf"); x[78] = float("inf"); x[99] = -float("inf")
+    x[1000:1010] = 0.0; x[2000:2010] = -0.0
+    for k in (1, 3, 5000, 8192):
+        v, i = gpu_topk(x, k)
+        assert_exact(x, k, v, i)
+    xb = x.to(torch.bfloat16)
+    v, i = gpu_topk(xb, 1000)
+    assert_exact(xb, 1000, v, i)
+
+
+# ----------------------------------------------------------------------------- stages on their own
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_sample_indices_and_threshold_match_the_oracle(dtype):
+    n, m, r = 1_000_003, 5000, 7
+    x = workloads.normal(3, n, seed=16, dtype=dtype)
+    tau, sidx = profk.sample_threshold(x.cuda(), m, r, seed=0xABCDEF0123, want_indices=True)
+    torch.cuda.synchronize()
+    xn = workloads.as_numpy(x)
+    for row in range(3):
+        want_idx = o_philox.sample_indices(n, m, 0xABCDEF0123, row)
+        assert np.array_equal(sidx[row].cpu().numpy().astype(np.int64) & 0xFFFFFFFF, want_idx)
+        want_tau = o_stages.threshold(xn[row], want_idx, r)
+        assert bits(workloads.as_numpy(tau[row:row + 1]))[0] == bits(np.asarray([want_tau]))[0]
+    # large sample spread over an 8-CTA cluster, deep rank
+    tau = profk.sample_threshold(x[:1].cuda(), 131072, 9000, seed=5)
+    torch.cuda.synchronize()
+    want = o_stages.threshold(xn[0], o_philox.sample_indices(n, 131072, 5, 0), 9000)
+    assert bits(workloads.as_numpy(tau))[0] == bits(np.asarray([want]))[0]
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_filter_keeps_exactly_the_survivor_set(dtype):
+    n = 777_777
+    x = workloads.normal(2, n, seed=17, dtype=dtype)
+    xn = workloads.as_numpy(x)
+    tau = torch.tensor([2.5, 3.0]).to(dtype)
+    buf, counts = profk.filter_pass(x.cuda(), tau.cuda(), capacity=20_000)
+    torch.cuda.synchronize()
+    for row in range(2):
+        want = o_stages.survivor_set(xn[row], workloads.as_numpy(tau)[row])
+        c = int(counts[row])
+        assert c == want.size
+        rec = buf[row, :c].cpu().numpy().view(np.uint64)
+        got_idx = np.sort((rec & np.uint64(0xFFFFFFFF)).astype(np.int64))
+        assert np.array_equal(got_idx, want)                                  # same set, any order
+        keys = (~(rec >> np.uint64(32))).astype(np.uint32)
+        okeys = o_topk.order_key(xn[row])
+        okeys32 = okeys.astype(np.uint32) if dtype == torch.float32 else (okeys.astype(np.uint32) << 16)
+        order = np.argsort(rec & np.uint64(0xFFFFFFFF))
+        assert np.array_equal(keys[order], okeys32[want])
+    # overflow: the counter only has to exceed the capacity
+    buf, counts = profk.filter_pass(x.cuda(), torch.tensor([-10.0, -10.0]).to(dtype).cuda(), capacity=1000)
+    torch.cuda.synchronize()
+    assert int(counts[0]) > 1000 and int(counts[1]) > 1000
+
+
+# ----------------------------------------------------------------------------- relaxed recall
+def test_relaxed_recall_returns_a_padded_prefix():
+    x = workloads.normal(1, 1 << 20, seed=18)[0]
+    k = 512
+    ov, oi = o_topk.topk_row(workloads.as_numpy(x), k)
+    short = 0
+    for seed in range(12):
+        # a plan whose threshold is often too high for k but fine for k_accept
+        pl = profk.Plan(m=8192, r=3, capacity=4096, k_accept=128, mode=0)
+        v, i = profk.topk(x.cuda(), k, plan_override=pl, seed=seed)
+        torch.cuda.synchronize()
+        v, i = v.cpu().numpy(), i.cpu().numpy()
+        _, R, _, status = profk.read_stats(1)[0]
+        n_real = min(k, R) if status == profk.ROW_OK else k
+        assert np.array_equal(i[:n_real], oi[:n_real]) and np.array_equal(bits(v[:n_real]), bits(ov[:n_real]))
+        assert np.all(i[n_real:] == -1) and np.all(np.isneginf(v[n_real:]))
+        short += n_real < k
+    assert short > 0, "no seed exercised the short-buffer branch"
+    pl = profk.plan(1 << 20, k, 1e-2, recall=0.95)
+    v, i = gpu_topk(x, k, eps=1e-2, recall=0.95, seed=1)
+    _, R, _, status = profk.read_stats(1)[0]
+    n_real = min(k, R) if status == profk.ROW_OK else k
+    assert n_real >= pl.k_accept
+    assert np.array_equal(i[:n_real], oi[:n_real])
