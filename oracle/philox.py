@@ -9,8 +9,10 @@ path implements a second time on its own:
   * stratum j contributes exactly one index, lo_j + floor(u_j (hi_j - lo_j) / 2^64),
     where u_j is a 64-bit word from the counter-based generator Philox4x32-10
     (Salmon, Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3",
-    SC'11) with key = (seed low word, seed high word) and
-    counter = (j, row low word, row high word, 0);  u_j = word0 + 2^32 word1.
+    SC'11) with key = (seed low word, seed high word).  One generator block of
+    four words serves two strata: block b has counter (b, row low word, row high
+    word, 0); stratum 2b takes u = word0 + 2^32 word1, stratum 2b+1 takes
+    u = word2 + 2^32 word3.
 
 Indices are distinct by construction and every element of a stratum is equally
 likely.  The random numbers are a function of (seed, row, j) only, so the two
@@ -71,8 +73,11 @@ def sample_indices(N: int, S: int, seed: int, row: int = 0) -> np.ndarray:
         raise ValueError("need 1 <= S <= N")
     lo, hi = stratum_bounds(N, S)
     j = np.arange(S, dtype=np.uint64)
-    w0, w1, _, _ = philox4x32_10(j, row & 0xFFFFFFFF, (row >> 32) & 0xFFFFFFFF, 0,
-                                 seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)
+    b0, b1, b2, b3 = philox4x32_10(j >> np.uint64(1), row & 0xFFFFFFFF, (row >> 32) & 0xFFFFFFFF, 0,
+                                   seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)
+    odd = (j & np.uint64(1)).astype(bool)
+    w0 = np.where(odd, b2, b0)
+    w1 = np.where(odd, b3, b1)
     width = (hi - lo).astype(np.uint64)                   # < 2^32 always (N < 2^32)
     # floor(u * width / 2^64) with u = w0 + 2^32 w1, in 64-bit pieces:
     #   u * width = w1*width * 2^32 + w0*width

@@ -82,9 +82,24 @@ def _check(code: int, what: str) -> None:
         raise ProfkError(f"{what}: {lib().profk_strerror(code).decode()} ({code})")
 
 
+_plan_cache: dict = {}
+
+
 def plan(N: int, k: int, eps: float = 1e-3, recall: float = 1.0, s_min: int | None = None,
          s_max: int | None = None, cost_ratio: float | None = None) -> Plan:
     """`profk_plan` / `profk_plan_ex`: the parameters (S, t, M) for one row of length N."""
+    key = (N, k, eps, recall, s_min, s_max, cost_ratio)
+    hit = _plan_cache.get(key)
+    if hit is not None:
+        return hit
+    res = _plan_uncached(N, k, eps, recall, s_min, s_max, cost_ratio)
+    if len(_plan_cache) > 4096:
+        _plan_cache.clear()
+    _plan_cache[key] = res
+    return res
+
+
+def _plan_uncached(N, k, eps, recall, s_min, s_max, cost_ratio) -> Plan:
     out = _PlanStruct()
     if s_min is None and s_max is None and cost_ratio is None:
         code = lib().profk_plan(ctypes.c_int64(N), ctypes.c_int64(k), ctypes.c_double(eps),
@@ -107,22 +122,30 @@ def workspace_bytes(rows: int, capacity: int, k: int) -> int:
 
 
 _workspaces: dict = {}     # device index -> torch tensor kept alive while registered
+_workspace_ok: set = set()  # (device, rows, capacity, k) shapes known to fit the registered workspace
 
 
 def ensure_workspace(rows: int, capacity: int, k: int, device) -> None:
     """Allocate (through torch) and register a workspace large enough for the shape."""
     import torch
 
-    need = workspace_bytes(rows, capacity, k)
     dev = torch.device(device)
     idx = dev.index if dev.index is not None else torch.cuda.current_device()
+    if (idx, rows, capacity, k) in _workspace_ok:
+        return
+    need = workspace_bytes(rows, capacity, k)
     cur = _workspaces.get(idx)
-    if cur is None or cur.numel() < need:
+    if cur is not None and cur.numel() >= need:
+        _workspace_ok.add((idx, rows, capacity, k))
+        return
+    if True:
         with torch.cuda.device(idx):
             buf = torch.empty(max(need, 1 << 20), dtype=torch.uint8, device=dev)
             _check(lib().profk_set_workspace(ctypes.c_void_p(buf.data_ptr()), ctypes.c_size_t(buf.numel())),
                    "profk_set_workspace")
         _workspaces[idx] = buf
+        _workspace_ok.clear()
+        _workspace_ok.add((idx, rows, capacity, k))
 
 
 def _stream_ptr():

@@ -22,7 +22,7 @@ def nvcc_command(extra: list[str] | None = None) -> list[str]:
     cmd = [nvcc, "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
            "-o", LIB_PATH] + [os.path.join(CSRC, s) for s in SOURCES]
-    return cmd + (extra or [])
+    return cmd + (extra or []) + os.environ.get("PROFK_NVCC_FLAGS", "").split()
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

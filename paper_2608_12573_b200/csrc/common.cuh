@@ -21,14 +21,23 @@ __device__ __forceinline__ uint32_t bits32_from_key(uint32_t k) {
     return (k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k;
 }
 
+// Bit pattern of a float through an opaque move: the compiler must not rewrite the integer
+// key arithmetic below as floating-point sign / abs operations, which would replace a NaN's
+// payload by the canonical NaN and so change its key.
+__device__ __forceinline__ uint32_t float_bits_exact(float v) {
+    uint32_t b;
+    asm("mov.b32 %0, %1;" : "=r"(b) : "f"(v));
+    return b;
+}
+
 template <typename T> struct Elem;
 
 template <> struct Elem<float> {
     using vec_t = float4;                       // 128-bit vector
     static constexpr int VEC = 4;               // elements per vector
     static constexpr uint32_t NEG_INF_BITS = 0xFF800000u;
-    static __device__ __forceinline__ uint32_t bits(float v) { return __float_as_uint(v); }
-    static __device__ __forceinline__ uint32_t key(float v) { return key_from_bits32(__float_as_uint(v)); }
+    static __device__ __forceinline__ uint32_t bits(float v) { return float_bits_exact(v); }
+    static __device__ __forceinline__ uint32_t key(float v) { return key_from_bits32(float_bits_exact(v)); }
     static __device__ __forceinline__ float from_key(uint32_t k) { return __uint_as_float(bits32_from_key(k)); }
     static __device__ __forceinline__ float from_bits(uint32_t b) { return __uint_as_float(b); }
     static __device__ __forceinline__ float as_float(float v) { return v; }
@@ -59,6 +68,17 @@ __device__ __forceinline__ uint64_t make_record(uint32_t key, uint32_t idx) {
 }
 __device__ __forceinline__ uint32_t record_key(uint64_t rec) { return ~(uint32_t)(rec >> 32); }
 __device__ __forceinline__ uint32_t record_idx(uint64_t rec) { return (uint32_t)rec; }
+
+// Coarse histogram of the survivors, filled by the filter and read by the refine step:
+// bin 0 holds the largest keys.  hi_key is (an estimate of) the largest key, shift scales
+// the distance below it to COARSE_BINS bins; keys above hi_key land in bin 0, keys far
+// below it in the last bin.
+constexpr int COARSE_BITS = 12;
+constexpr uint32_t COARSE_BINS = 1u << COARSE_BITS;
+__device__ __forceinline__ uint32_t coarse_bin(uint32_t key, uint32_t hi_key, uint32_t shift) {
+    const uint32_t d = key >= hi_key ? 0u : (hi_key - key) >> shift;
+    return d < COARSE_BINS ? d : COARSE_BINS - 1;
+}
 
 // ---------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon et al., SC'11): ten rounds, key bumped by the Weyl constants between rounds.
@@ -105,6 +125,22 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
 }
 
 __device__ __forceinline__ unsigned lane_id() { return threadIdx.x & 31u; }
+
+// Optional phase stamps for tuning (SM cycle counter of CTA 0); compiled out by default.
+#ifdef PROFK_TRACE
+__device__ long long g_profk_trace[4][32];
+#define PROFK_STAMP(kernel, slot)                                                   \
+    do {                                                                            \
+        if (threadIdx.x == 0 && blockIdx.x == 0) {                                  \
+            g_profk_trace[kernel][slot] = clock64();                                \
+            unsigned long long gt;                                                  \
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));                  \
+            g_profk_trace[kernel + 2][slot] = (long long)gt;                        \
+        }                                                                           \
+    } while (0)
+#else
+#define PROFK_STAMP(kernel, slot) do { } while (0)
+#endif
 
 // Programmatic dependent launch: wait for the preceding kernel's memory to be visible /
 // allow the following kernel to start its prologue.

@@ -1,9 +1,9 @@
 // Count check and exact replacement (Section 3, "Refinement": "if fewer than k candidates
 // are collected, or if the buffer overflows ..., falls back to an exact top-k computation
-// on the full input").  The decision is taken on the device: this kernel reads the
-// per-row survivor counters, and for every row that failed it selects the exact top-k of
-// the whole row into the row's candidate buffer, so that the refine kernel that follows
-// orders the buffer the same way for every row.
+// on the full input").  The decision is taken on the device: the refine kernel checks every
+// row's survivor count and leaves the rows that failed to this kernel, which returns at once
+// when there are none.  For each failed row it selects the exact top-k of the whole row into
+// the row's candidate buffer, orders it and writes the row's output.
 //
 // The exact selection is a most-significant-digit radix select over 64-bit candidate
 // records (value key, then index), 11 bits per pass, run by the whole grid with a grid
@@ -11,32 +11,33 @@
 // co-resident; every wait is bounded and reports through the workspace header.
 #pragma once
 
+#include "refine.cuh"
 #include "rowscan.cuh"
 #include "sample_select.cuh"
 
 namespace profk {
 
-constexpr int FB_THREADS = 512;
+constexpr int FB_THREADS = 1024;
 constexpr int FB_UNROLL = 4;
 constexpr int FB_BINS = 2048;
 constexpr int FB_PASSES = 6;                // 5 x 11 bits + 9 bits = 64
 constexpr uint32_t SPIN_LIMIT = 1u << 24;   // polls (each ~100 ns apart) before a wait gives up
 
-enum : uint32_t { ROW_OK = 0, ROW_RECALL = 1, ROW_OVERFLOW = 2, ROW_DIRECT = 3, ROW_TIMEOUT_BIT = 0x80000000u };
 
 template <typename T> struct FallbackParams {
     const T* in;
     uint64_t N;
     uint64_t rows;
     uint32_t k;
-    uint32_t k_accept;
     uint32_t capacity;
-    int mode;                 // 1 = every row takes the exact path
     RowCtl* ctl;
     WsHeader* header;
     uint32_t* ghist;          // FB_PASSES x FB_BINS global histogram
     uint64_t* buf;            // rows x capacity records
     uint64_t tiles_per_row;
+    int use_pdl;              // 1 = launched as a programmatic dependent of the refine kernel
+    T* out_vals;              // rows x k
+    int64_t* out_idx;         // rows x k
 };
 
 // Sense-free generation barrier over all CTAs of a co-resident grid.  Returns false when
@@ -105,25 +106,18 @@ __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackPara
 
     const unsigned tid = threadIdx.x, lane = lane_id(), warp = tid >> 5;
     pdl_launch_dependents();
+    if (p.use_pdl) pdl_wait();
+
+    // The count check was taken by the refine kernel (or, in direct mode, every row was marked by
+    // the initialisation kernel): in the common case no row failed and this kernel is one load long.
+    if (__ldcg(&p.header->n_failed) == 0) return;
 
     uint32_t gen = *((volatile uint32_t*)&p.header->bar_gen);   // read before this CTA's first arrival
 
     for (uint64_t chunk = 0; chunk < p.rows; chunk += FB_THREADS) {
-        // ---- count check for FB_THREADS rows at a time; every CTA takes the same decisions ----
+        // ---- FB_THREADS rows at a time; every CTA reads the same status words ----
         const uint64_t r = chunk + tid;
-        bool failed = false;
-        if (r < p.rows) {
-            const uint32_t R = p.ctl[r].count;
-            uint32_t status = ROW_OK;
-            if (p.mode == 1) status = ROW_DIRECT;
-            else if (R > p.capacity) status = ROW_OVERFLOW;
-            else if (R < p.k_accept) status = ROW_RECALL;
-            failed = status != ROW_OK;
-            if (blockIdx.x == 0) {
-                p.ctl[r].status = status;
-                p.ctl[r].n_final = failed ? p.k : R;
-            }
-        }
+        const bool failed = r < p.rows && __ldcg(&p.ctl[r].status) != ROW_OK;
         const unsigned m = __ballot_sync(FULL_MASK, failed);
         if (lane == 0) flag_masks[warp] = m;
         __syncthreads();
@@ -205,6 +199,18 @@ __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackPara
                         if (take && pos < p.capacity) dst[pos] = rec;
                     }
                 });
+
+                // ---- order the k records and write the row's output (first CTA; the others move on
+                //      and meet it again at the next row's barrier) ----
+                if (!grid_barrier(p.header, gen)) return;
+                if (blockIdx.x == 0) {
+                    extern __shared__ __align__(16) unsigned char fb_smem[];
+                    uint64_t* sortbuf = reinterpret_cast<uint64_t*>(fb_smem);
+                    for (uint32_t i = tid; i < p.k; i += FB_THREADS) sortbuf[i] = __ldcg(&dst[i]);
+                    __syncthreads();
+                    sort_and_write<T>(sortbuf, p.k, p.k, p.k, row, p.out_vals, p.out_idx);
+                    __syncthreads();
+                }
             }
         }
         __syncthreads();   // flag_masks is rewritten by the next chunk

@@ -4,10 +4,26 @@
 // The kernel is bound by HBM bandwidth: one 128-bit load per VEC elements, one compare
 // per element, and nothing else on the common path.  Survivors are rare (1e-3 .. 1e-5 of
 // the elements), so the append is a warp-cooperative slow path taken only when some lane
-// of the warp saw a survivor: a warp prefix sum and one global atomic per warp.
+// of the warp saw a survivor: a warp prefix sum, one global atomic per warp, and one
+// histogram increment per survivor for the refine step.
 #pragma once
 
 #include "rowscan.cuh"
+#include "sample_select.cuh"
+
+// Launch shape of the filter kernel (tuned on B200; overridable at build time for experiments).
+#ifndef PROFK_FILTER_THREADS
+#define PROFK_FILTER_THREADS 512
+#endif
+#ifndef PROFK_FILTER_UNROLL
+#define PROFK_FILTER_UNROLL 4
+#endif
+#ifndef PROFK_FILTER_MINBLOCKS_F32
+#define PROFK_FILTER_MINBLOCKS_F32 3
+#endif
+#ifndef PROFK_FILTER_MINBLOCKS_BF16
+#define PROFK_FILTER_MINBLOCKS_BF16 2
+#endif
 
 namespace profk {
 
@@ -23,6 +39,8 @@ template <typename T> struct FilterParams {
     uint64_t tiles_per_row;
     uint64_t total_tiles;
     int use_pdl;             // 1 = launched as a programmatic dependent of the threshold kernel
+    const RowCtl* ctl;       // per-row histogram parameters (needed only with `coarse`)
+    uint32_t* coarse;        // rows x COARSE_BINS survivor histogram (null = none)
 };
 
 // not (x < tau) for every lane of a vector, OR-ed: does the vector hold any survivor?
@@ -39,30 +57,29 @@ __device__ __forceinline__ bool vec_any_pass(const uint4& v, __nv_bfloat16 tau) 
 }
 
 template <typename T, int THREADS, int UNROLL>
-__global__ void __launch_bounds__(THREADS) filter_kernel(const FilterParams<T> p) {
+__global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOCKS_F32 : PROFK_FILTER_MINBLOCKS_BF16) filter_kernel(const FilterParams<T> p) {
     using V = typename Elem<T>::vec_t;
     constexpr int VEC = Elem<T>::VEC;
     constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
 
     const unsigned lane = lane_id();
-
-    uint64_t tile = blockIdx.x;
-    if (tile >= p.total_tiles) return;
+    uint32_t tile = blockIdx.x;                  // the grid never exceeds the number of tiles (< 2^32)
+    const uint32_t total_tiles = (uint32_t)p.total_tiles, tiles_per_row = (uint32_t)p.tiles_per_row;
 
     // Decode the first tile and issue its loads before waiting on the threshold kernel:
     // the input does not depend on it.
-    uint64_t row = tile / p.tiles_per_row;
-    uint64_t trow = tile - row * p.tiles_per_row;
+    uint32_t row = tile / tiles_per_row;
+    uint32_t trow = tile - row * tiles_per_row;
     RowView<T> rv = row_view(p.in, p.N, row);
     V v[UNROLL];
     bool inside[UNROLL];
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u)
-        v[u] = load_row_vector(rv, p.N, trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x, &inside[u]);
+        v[u] = load_row_vector(rv, p.N, (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x, &inside[u]);
 
     if (p.use_pdl) pdl_wait();
 
-    uint64_t skip_row = ~0ull;    // row whose buffer this warp has seen overflow: nothing more to append
+    uint32_t skip_row = 0xFFFFFFFFu;    // row whose buffer this warp has seen overflow: nothing more to append
     while (true) {
         const T tau = p.tau[row];
         bool hit = false;
@@ -78,7 +95,7 @@ __global__ void __launch_bounds__(THREADS) filter_kernel(const FilterParams<T> p
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 mine[u] = 0;
-                const uint64_t q = trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
+                const uint64_t q = (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
                 const int64_t i0 = (int64_t)(q * VEC) - (int64_t)rv.mis;
 #pragma unroll
                 for (int l = 0; l < VEC; ++l) {
@@ -96,41 +113,52 @@ __global__ void __launch_bounds__(THREADS) filter_kernel(const FilterParams<T> p
                 if (lane >= (unsigned)d) incl += nb;
             }
             const unsigned total = __shfl_sync(FULL_MASK, incl, 31);
-            unsigned base = 0;
-            if (lane == 0 && total) base = atomicAdd(p.counts + row * p.count_stride, total);
-            base = __shfl_sync(FULL_MASK, base, 0);
-            unsigned pos = base + incl - cnt;
-            uint64_t* dst = p.buf + row * (uint64_t)p.capacity;
+            if (total) {
+                // the histogram parameters travel while the counter atomic is in flight
+                uint32_t hi_key = 0, bin_shift = 0;
+                uint32_t* hist = nullptr;
+                if (p.coarse) {
+                    hi_key = p.ctl[row].hi_key;
+                    bin_shift = p.ctl[row].bin_shift;
+                    hist = p.coarse + (uint64_t)row * COARSE_BINS;
+                }
+                unsigned base = 0;
+                if (lane == 0) base = atomicAdd(p.counts + (uint64_t)row * p.count_stride, total);
+                base = __shfl_sync(FULL_MASK, base, 0);
+                unsigned pos = base + incl - cnt;
+                uint64_t* dst = p.buf + (uint64_t)row * p.capacity;
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u) {
-                if (mine[u]) {
-                    const uint64_t q = trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
-                    const int64_t i0 = (int64_t)(q * VEC) - (int64_t)rv.mis;
+                for (int u = 0; u < UNROLL; ++u) {
+                    if (mine[u]) {
+                        const uint64_t q = (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
+                        const int64_t i0 = (int64_t)(q * VEC) - (int64_t)rv.mis;
 #pragma unroll
-                    for (int l = 0; l < VEC; ++l) {
-                        if (mine[u] & (1u << l)) {
-                            if (pos < p.capacity)
-                                dst[pos] = make_record(Elem<T>::key(vec_elem(v[u], l)), (uint32_t)(i0 + l));
-                            ++pos;
+                        for (int l = 0; l < VEC; ++l) {
+                            if (mine[u] & (1u << l)) {
+                                const uint32_t key = Elem<T>::key(vec_elem(v[u], l));
+                                if (pos < p.capacity) dst[pos] = make_record(key, (uint32_t)(i0 + l));
+                                if (hist) atomicAdd(&hist[coarse_bin(key, hi_key, bin_shift)], 1u);
+                                ++pos;
+                            }
                         }
                     }
                 }
+                if ((uint64_t)base + total > p.capacity) skip_row = row;   // overflow: the exact path redoes this row
             }
-            if ((uint64_t)base + total > p.capacity) skip_row = row;   // overflow: the exact path will redo this row
         }
 
         // Next tile of this CTA; tiles of a row already known to overflow are not even loaded.
-        uint64_t nrow;
+        uint32_t nrow;
         do {
+            if (total_tiles - tile <= gridDim.x) return;
             tile += gridDim.x;
-            if (tile >= p.total_tiles) return;
-            nrow = tile / p.tiles_per_row;
+            nrow = tile / tiles_per_row;
         } while (nrow == skip_row);
-        trow = tile - nrow * p.tiles_per_row;
+        trow = tile - nrow * tiles_per_row;
         if (nrow != row) { row = nrow; rv = row_view(p.in, p.N, row); }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u)
-            v[u] = load_row_vector(rv, p.N, trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x, &inside[u]);
+            v[u] = load_row_vector(rv, p.N, (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x, &inside[u]);
     }
 }
 

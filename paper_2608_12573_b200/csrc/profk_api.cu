@@ -1,8 +1,9 @@
 // C ABI of the library (see profk.h): argument checks, workspace layout and the launch
-// sequence  threshold -> filter -> count check / exact replacement -> refine.
+// sequence  threshold -> filter -> count check + refine -> exact replacement of failed rows.
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cstdio>
 #include <cstring>
 #include <map>
@@ -20,19 +21,21 @@ using namespace profk;
 
 namespace {
 
-constexpr int FILTER_THREADS = 512;
-constexpr int FILTER_UNROLL = 4;
+constexpr int FILTER_THREADS = PROFK_FILTER_THREADS;
+constexpr int FILTER_UNROLL = PROFK_FILTER_UNROLL;
 constexpr uint32_t SORT_CAP_MAX = 8192;          // largest k the single-CTA refine orders in shared memory
 constexpr size_t REFINE_SMEM_MAX = 200 * 1024;   // dynamic shared memory the refine kernel may ask for
 constexpr int64_t N_MAX = 4278190080LL;          // 2^32 - 2^24
 constexpr int64_t M_MAX = 262144;                // largest sample the cluster select holds (8 CTAs x 32768 keys)
 
 thread_local int g_launches = 0;
+std::atomic<int> g_coop_pdl{-1};                 // -1 untried, 1 accepted, 0 refused by the runtime
 
 struct DeviceInfo {
     int sm_count = 0;
     int filter_blocks_per_sm[2] = {0, 0};     // by dtype
     int fallback_blocks_per_sm[2] = {0, 0};
+    int max_cluster[2] = {8, 8};              // 16 when the device can co-schedule 16 CTAs of the threshold kernel
     bool ready = false;
 };
 
@@ -46,7 +49,7 @@ std::map<std::tuple<int64_t, int64_t, double, double>, profk_plan_t> g_plan_cach
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-    size_t off_header, off_ghist, off_ctl, off_tau, off_buf, total;
+    size_t off_header, off_ghist, off_ctl, off_tau, off_coarse, off_buf, total;
 };
 
 WsLayout ws_layout(int64_t rows, int64_t capacity) {
@@ -55,7 +58,8 @@ WsLayout ws_layout(int64_t rows, int64_t capacity) {
     l.off_ghist = sizeof(WsHeader);
     l.off_ctl = align_up(l.off_ghist + (size_t)FB_PASSES * FB_BINS * sizeof(uint32_t), 256);
     l.off_tau = align_up(l.off_ctl + (size_t)rows * sizeof(RowCtl), 256);
-    l.off_buf = align_up(l.off_tau + (size_t)rows * 4, 256);
+    l.off_coarse = align_up(l.off_tau + (size_t)rows * 4, 256);
+    l.off_buf = align_up(l.off_coarse + (size_t)rows * COARSE_BINS * sizeof(uint32_t), 256);
     l.total = align_up(l.off_buf + (size_t)rows * (size_t)capacity * sizeof(uint64_t), 256);
     return l;
 }
@@ -85,36 +89,53 @@ template <typename T> int ensure_device_info(int dev, DeviceInfo* out) {
         di.fallback_blocks_per_sm[d] = std::max(nb, 1);
         CUDA_TRY(cudaFuncSetAttribute(sample_select_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
         CUDA_TRY(cudaFuncSetAttribute(refine_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFINE_SMEM_MAX));
+        CUDA_TRY(cudaFuncSetAttribute(fallback_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SORT_CAP_MAX * 8)));
+        // Clusters of 16 are beyond the portable size: allowed only where one actually fits.
+        if (cudaFuncSetAttribute(sample_select_kernel<T>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(16); cfg.blockDim = dim3(SEL_THREADS); cfg.dynamicSmemBytes = 16384 * sizeof(uint32_t);
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 16; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr; cfg.numAttrs = 1;
+            int nclusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&nclusters, sample_select_kernel<T>, &cfg) == cudaSuccess && nclusters >= 1)
+                di.max_cluster[d] = 16;
+        }
+        (void)cudaGetLastError();
     }
     *out = di;
     return PROFK_OK;
 }
 
-__global__ void init_ctl_kernel(RowCtl* ctl, uint64_t rows, WsHeader* header, uint32_t capacity) {
+// Direct mode has no threshold / filter kernels: mark every row for exact selection.
+__global__ void init_ctl_kernel(RowCtl* ctl, uint64_t rows, WsHeader* header, uint32_t capacity, uint32_t k) {
     const uint64_t r = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (r < rows) {
         RowCtl* c = ctl + r;
-        c->tau_bits = 0; c->count = 0; c->collect = 0; c->status = 0; c->n_final = 0; c->capacity = capacity;
+        c->tau_bits = 0; c->count = 0; c->collect = 0; c->status = ROW_DIRECT; c->n_final = k; c->capacity = capacity;
     }
-    if (r == 0) { header->bar_count = 0; header->error = 0; }
+    if (r == 0) { header->bar_count = 0; header->error = 0; header->done = 0; header->n_failed = (uint32_t)rows; }
 }
 
 // Cluster size for the threshold kernel: spread one row's gather over several SMs when
 // there are few rows; never more keys per CTA than its shared memory holds.
-int pick_cluster(int64_t rows, int64_t m) {
-    int c = rows <= 18 ? 8 : rows <= 37 ? 4 : rows <= 74 ? 2 : 1;
-    while (c < 8 && (m + c - 1) / c > 32768) c *= 2;
+int pick_cluster(int64_t rows, int64_t m, int max_cluster) {
+    int c = rows <= 9 ? 16 : rows <= 18 ? 8 : rows <= 37 ? 4 : rows <= 74 ? 2 : 1;
+    if (c > max_cluster) c = max_cluster;
+    while (c < 8 && (m + c - 1) / c > 32766) c *= 2;
     return c;
 }
 
 template <typename T>
-int launch_sample_select(const T* in, int64_t rows, int64_t N, int64_t m, int64_t r, uint64_t seed, T* tau, RowCtl* ctl,
-                         WsHeader* header, uint32_t capacity, uint32_t* sample_idx, cudaStream_t st) {
-    const int csize = pick_cluster(rows, m);
+int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, int64_t m, int64_t r, uint64_t seed, T* tau, RowCtl* ctl,
+                         WsHeader* header, uint32_t capacity, uint32_t* coarse, uint32_t* sample_idx, cudaStream_t st) {
+    const int csize = pick_cluster(rows, m, di.max_cluster[dtype_index<T>()]);
     SelectParams<T> sp;
     sp.in = in; sp.N = (uint64_t)N; sp.S = (uint32_t)m; sp.t = (uint32_t)r; sp.seed = seed;
-    sp.per_cta = (uint32_t)((m + csize - 1) / csize);
-    sp.tau = tau; sp.ctl = ctl; sp.header = header; sp.capacity = capacity; sp.sample_idx = sample_idx;
+    sp.per_cta = (uint32_t)(((m + csize - 1) / csize + 1) & ~1LL);      // even: samples are drawn in pairs
+    sp.q = (uint64_t)(N / m); sp.rem = (uint32_t)(N % m); sp.inv_s = 1.0f / (float)m;
+    sp.tau = tau; sp.ctl = ctl; sp.header = header; sp.capacity = capacity; sp.coarse = coarse; sp.sample_idx = sample_idx;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(rows * csize));
     cfg.blockDim = dim3(SEL_THREADS);
@@ -131,13 +152,15 @@ int launch_sample_select(const T* in, int64_t rows, int64_t N, int64_t m, int64_
 
 template <typename T>
 int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, const T* tau, int64_t capacity, uint64_t* buf,
-                  uint32_t* counts, uint32_t count_stride, bool pdl, cudaStream_t st) {
+                  uint32_t* counts, uint32_t count_stride, bool pdl, const RowCtl* ctl, uint32_t* coarse, cudaStream_t st) {
     FilterParams<T> fp;
     fp.in = in; fp.N = (uint64_t)N; fp.rows = (uint64_t)rows; fp.tau = tau; fp.capacity = (uint32_t)capacity;
     fp.buf = buf; fp.counts = counts; fp.count_stride = count_stride;
     fp.tiles_per_row = tiles_per_row<T>((uint64_t)N, FILTER_THREADS * FILTER_UNROLL);
     fp.total_tiles = fp.tiles_per_row * (uint64_t)rows;
+    if (fp.total_tiles >= (1ull << 32)) return PROFK_EINVAL;      // rows * N beyond 2^45 elements
     fp.use_pdl = pdl ? 1 : 0;
+    fp.ctl = ctl; fp.coarse = coarse;
     const uint64_t max_grid = (uint64_t)di.sm_count * di.filter_blocks_per_sm[dtype_index<T>()];
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)std::min<uint64_t>(fp.total_tiles, max_grid));
@@ -187,62 +210,87 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     uint32_t* ghist = reinterpret_cast<uint32_t*>(base + lay.off_ghist);
     RowCtl* ctl = reinterpret_cast<RowCtl*>(base + lay.off_ctl);
     T* tau = reinterpret_cast<T*>(base + lay.off_tau);
+    uint32_t* coarse = reinterpret_cast<uint32_t*>(base + lay.off_coarse);
     uint64_t* buf = reinterpret_cast<uint64_t*>(base + lay.off_buf);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
+    uint32_t sort_cap = 32;
+    while (sort_cap < (uint32_t)k) sort_cap <<= 1;
+
     if (plan->mode == 0) {
-        rc = launch_sample_select<T>(in, rows, N, plan->m, plan->r, seed, tau, ctl, header, (uint32_t)capacity, nullptr, st);
+        rc = launch_sample_select<T>(di, in, rows, N, plan->m, plan->r, seed, tau, ctl, header, (uint32_t)capacity, coarse, nullptr, st);
         if (rc != PROFK_OK) return rc;
-        rc = launch_filter<T>(di, in, rows, N, tau, capacity, buf, &ctl[0].count, sizeof(RowCtl) / 4, true, st);
+        rc = launch_filter<T>(di, in, rows, N, tau, capacity, buf, &ctl[0].count, sizeof(RowCtl) / 4, true, ctl, coarse, st);
         if (rc != PROFK_OK) return rc;
-    } else {
-        init_ctl_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(ctl, (uint64_t)rows, header, (uint32_t)capacity);
-        CUDA_TRY(cudaGetLastError());
-        ++g_launches;
-    }
 
-    {   // count check + exact replacement of failed rows (cooperative: all CTAs co-resident)
-        FallbackParams<T> fb;
-        fb.in = in; fb.N = (uint64_t)N; fb.rows = (uint64_t)rows; fb.k = (uint32_t)k;
-        fb.k_accept = (uint32_t)(plan->mode == 0 ? plan->k_accept : k);
-        fb.capacity = (uint32_t)capacity; fb.mode = plan->mode; fb.ctl = ctl; fb.header = header; fb.ghist = ghist; fb.buf = buf;
-        fb.tiles_per_row = tiles_per_row<T>((uint64_t)N, FB_THREADS * FB_UNROLL);
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)(di.sm_count * di.fallback_blocks_per_sm[dtype_index<T>()]));
-        cfg.blockDim = dim3(FB_THREADS);
-        cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeCooperative;
-        attr[0].val.cooperative = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        CUDA_TRY(cudaLaunchKernelEx(&cfg, fallback_kernel<T>, fb));
-        ++g_launches;
-    }
-
-    {   // refine: order the buffer of every row
+        // refine: count check, then order the buffer of every row that passed it
         RefineParams<T> rp;
-        rp.ctl = ctl; rp.buf = buf; rp.capacity = (uint32_t)capacity; rp.k = (uint32_t)k;
-        uint32_t sort_cap = 32;
-        while (sort_cap < (uint32_t)k) sort_cap <<= 1;
-        // small buffers are sorted whole, skipping the select
-        while (sort_cap < 2048 && sort_cap < (uint32_t)capacity) sort_cap <<= 1;
-        rp.sort_cap = sort_cap;
-        const size_t room = (REFINE_SMEM_MAX - (size_t)sort_cap * 8) / 8;
+        rp.ctl = ctl; rp.header = header; rp.buf = buf; rp.capacity = (uint32_t)capacity; rp.k = (uint32_t)k;
+        rp.k_accept = (uint32_t)plan->k_accept;
+        uint32_t rsort = sort_cap;
+        while (rsort < 2048 && rsort < (uint32_t)capacity) rsort <<= 1;     // small buffers are sorted whole
+        rp.sort_cap = rsort;
+        const size_t room = (REFINE_SMEM_MAX - (size_t)rsort * 8) / 8;
         rp.stage_cap = (uint32_t)std::min<size_t>((size_t)capacity, room);
-        if (rp.stage_cap <= sort_cap) rp.stage_cap = 0;
-        rp.out_vals = out_vals; rp.out_idx = out_idx; rp.use_pdl = 1;
+        if (rp.stage_cap <= rsort) rp.stage_cap = 0;
+        rp.out_vals = out_vals; rp.out_idx = out_idx; rp.use_pdl = 1; rp.coarse = coarse;
         unsigned threads = 128;
         while (threads < 1024 && threads * 8 < (unsigned)capacity) threads <<= 1;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)rows);
         cfg.blockDim = dim3(threads);
-        cfg.dynamicSmemBytes = ((size_t)sort_cap + rp.stage_cap) * 8;
+        cfg.dynamicSmemBytes = ((size_t)rsort + rp.stage_cap) * 8;
         cfg.stream = st;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr; cfg.numAttrs = 1;
         CUDA_TRY(cudaLaunchKernelEx(&cfg, refine_kernel<T>, rp));
+        ++g_launches;
+    } else {
+        init_ctl_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(ctl, (uint64_t)rows, header, (uint32_t)capacity, (uint32_t)k);
+        CUDA_TRY(cudaGetLastError());
+        ++g_launches;
+    }
+
+    {   // exact selection, ordering and output of the rows that failed the check (cooperative: all CTAs co-resident)
+        FallbackParams<T> fb;
+        fb.in = in; fb.N = (uint64_t)N; fb.rows = (uint64_t)rows; fb.k = (uint32_t)k;
+        fb.capacity = (uint32_t)capacity; fb.ctl = ctl; fb.header = header; fb.ghist = ghist; fb.buf = buf;
+        fb.tiles_per_row = tiles_per_row<T>((uint64_t)N, FB_THREADS * FB_UNROLL);
+        fb.use_pdl = 0;
+        fb.out_vals = out_vals; fb.out_idx = out_idx;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)di.sm_count);       // one CTA per SM: cheap to launch when no row failed
+        cfg.blockDim = dim3(FB_THREADS);
+        cfg.dynamicSmemBytes = (size_t)sort_cap * 8;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        // A cooperative launch that is also a programmatic dependent hides its launch latency behind
+        // the refine kernel; if the runtime refuses the combination, launch it as a plain cooperative kernel.
+        int pdl_state = g_coop_pdl.load();
+        bool launched = false;
+        if (plan->mode == 0 && pdl_state != 0) {
+            cfg.numAttrs = 2;
+            fb.use_pdl = 1;
+            if (cudaLaunchKernelEx(&cfg, fallback_kernel<T>, fb) == cudaSuccess) {
+                launched = true;
+                g_coop_pdl.store(1);
+            } else {
+                (void)cudaGetLastError();
+                g_coop_pdl.store(0);
+            }
+        }
+        if (!launched) {
+            cfg.numAttrs = 1;
+            fb.use_pdl = 0;
+            CUDA_TRY(cudaLaunchKernelEx(&cfg, fallback_kernel<T>, fb));
+        }
         ++g_launches;
     }
     return PROFK_OK;
@@ -280,7 +328,8 @@ int filter_only(const T* in, int64_t rows, int64_t N, const T* tau, int64_t capa
     DeviceInfo di;
     const int rc = ensure_device_info<T>(dev, &di);
     if (rc != PROFK_OK) return rc;
-    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, counts, 1, false, static_cast<cudaStream_t>(stream));
+    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, counts, 1, false, nullptr, nullptr,
+                            static_cast<cudaStream_t>(stream));
 }
 
 template <typename T>
@@ -294,7 +343,7 @@ int sample_threshold(const T* in, int64_t rows, int64_t N, int64_t m, int64_t r,
     DeviceInfo di;
     const int rc = ensure_device_info<T>(dev, &di);
     if (rc != PROFK_OK) return rc;
-    return launch_sample_select<T>(in, rows, N, m, r, seed, tau, nullptr, nullptr, 0, sample_idx, static_cast<cudaStream_t>(stream));
+    return launch_sample_select<T>(di, in, rows, N, m, r, seed, tau, nullptr, nullptr, 0, nullptr, sample_idx, static_cast<cudaStream_t>(stream));
 }
 
 }  // namespace
@@ -391,6 +440,14 @@ int profk_read_stats(void* stream, int64_t rows, profk_row_stats_t* out) {
 }
 
 int profk_last_launch_count(void) { return g_launches; }
+
+#ifdef PROFK_TRACE
+int profk_debug_read_trace(long long* out /* [host] 4 x 32 */) {
+    CUDA_TRY(cudaDeviceSynchronize());
+    CUDA_TRY(cudaMemcpyFromSymbol(out, g_profk_trace, sizeof(long long) * 4 * 32));
+    return PROFK_OK;
+}
+#endif
 
 const char* profk_strerror(int code) {
     switch (code) {

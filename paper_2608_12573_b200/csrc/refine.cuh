@@ -1,29 +1,40 @@
-// Stage 4 (Section 3, "Refinement"): exact top-k of the candidate buffer, written out in
-// the order "value descending, index ascending".
+// Stage 4 (Section 3, "Refinement"): the count check and the exact top-k of the candidate
+// buffer, written out in the order "value descending, index ascending".
 //
 // Candidate records are 64-bit integers whose ascending order is exactly that order, so
-// refinement is "the k smallest records, sorted".  One CTA per row: the records are staged
-// in shared memory when they fit, a most-significant-digit radix select (11 bits per pass,
-// starting at the first bit in which the records differ) cuts them down to k, and a
-// bitonic sort in shared memory orders the k winners.
+// refinement is "the k smallest records, sorted".  One CTA per row.  The CTA first takes the
+// paper's check -- fewer than k candidates, or more than the buffer holds, means the row is
+// left to the exact-selection kernel that follows.  Otherwise: the filter kernel has already
+// counted the survivors into a coarse 4096-bin histogram, so one scan of that histogram finds
+// the bin holding the k-th best record; a single pass over the buffer keeps the records of
+// better bins (placed by prefix sums, no atomics) and ranks the few records of the boundary
+// bin.  When the histogram cannot be used (ties pile up in one bin) a most-significant-digit
+// radix select over the records does the same job.  A bitonic sort orders the k winners.
 #pragma once
 
 #include "sample_select.cuh"
 
 namespace profk {
 
-constexpr int RF_BINS = 2048;
+constexpr int RF_BITS = 12;                 // digit width of the general select
+constexpr int RF_BINS = 1 << RF_BITS;
+constexpr uint32_t RF_EDGE_CAP = 1024;      // boundary bins up to this size are ranked directly
+
+enum : uint32_t { ROW_OK = 0, ROW_RECALL = 1, ROW_OVERFLOW = 2, ROW_DIRECT = 3 };
 
 template <typename T> struct RefineParams {
-    const RowCtl* ctl;
+    RowCtl* ctl;
+    WsHeader* header;
     const uint64_t* buf;     // rows x capacity records
     uint32_t capacity;
     uint32_t k;
+    uint32_t k_accept;
     uint32_t stage_cap;      // records that fit the shared-memory staging area
     uint32_t sort_cap;       // power of two >= k: size of the shared-memory sort area
     T* out_vals;             // rows x k
     int64_t* out_idx;        // rows x k
     int use_pdl;
+    const uint32_t* coarse;  // rows x COARSE_BINS survivor histogram written by the filter (null = none)
 };
 
 __device__ __forceinline__ uint64_t shr64(uint64_t x, int s) { return s >= 64 ? 0ull : (x >> s); }
@@ -69,112 +80,293 @@ __device__ __forceinline__ void bitonic_sort_shared(uint64_t* a, uint32_t P) {
     }
 }
 
+// Shared state of one select.
+struct SelectShared {
+    uint32_t hist[RF_BINS];
+    uint64_t edge[RF_EDGE_CAP];      // records of the boundary bin
+    uint32_t warp_sums[32];
+    uint32_t digit, before, cnt, fill, n_edge, total;
+    unsigned long long or_bits, limit;
+};
+
+// Records read from memory (shared or global): every thread visits whole-warp rounds.
+struct MemRecords {
+    const uint64_t* recs;
+    uint32_t n;
+    template <typename F> __device__ __forceinline__ void for_each(F&& f) const {
+        const uint32_t n_round = (n + 31u) & ~31u;
+        for (uint32_t i = threadIdx.x; i < n_round; i += blockDim.x) f(i < n ? recs[i] : 0ull, i < n);
+    }
+};
+
+// General select: finds limit = the need-th smallest record (records are distinct) by radix
+// passes and compacts the records <= limit into sortbuf.  sh.or_bits = OR over (record XOR
+// first); sh.fill and sh.n_edge must be zero.  All threads call it.
+template <typename Src>
+__device__ __forceinline__ void select_smallest(const Src& src, uint64_t first, uint32_t need, uint64_t* sortbuf,
+                                                uint32_t sort_cap, SelectShared& sh) {
+    const unsigned tid = threadIdx.x, nthr = blockDim.x, lane = lane_id();
+    const int top = 64 - __clzll((long long)sh.or_bits);       // bits >= top are common to all records
+    uint64_t prefix = shr64(first, top);
+    uint64_t limit = ~0ull;
+    for (int done = 0; done < top;) {
+        const int shift = top - done - RF_BITS > 0 ? top - done - RF_BITS : 0;
+        const int width = top - done - shift;
+        const uint32_t nbins = 1u << width;
+        for (uint32_t i = tid; i < nbins; i += nthr) sh.hist[i] = 0;
+        __syncthreads();
+        src.for_each([&](uint64_t rec, bool valid) {
+            if (valid && shr64(rec, shift + width) == prefix) atomicAdd(&sh.hist[(uint32_t)(rec >> shift) & (nbins - 1)], 1u);
+        });
+        __syncthreads();
+        const uint32_t per = (RF_BINS + nthr - 1) / nthr;
+        uint32_t sum = 0;
+        for (uint32_t j = 0; j < per; ++j) {
+            const uint32_t bin = tid * per + j;
+            sum += bin < nbins ? sh.hist[bin] : 0;
+        }
+        uint32_t before = block_scan_any(sum, sh.warp_sums) - sum;
+        for (uint32_t j = 0; j < per; ++j) {
+            const uint32_t bin = tid * per + j;
+            const uint32_t c = bin < nbins ? sh.hist[bin] : 0;
+            if (before < need && need <= before + c) { sh.digit = bin; sh.before = before; sh.cnt = c; }
+            before += c;
+        }
+        __syncthreads();
+        prefix = (prefix << width) | sh.digit;
+        need -= sh.before;
+        const uint32_t in_bin = sh.cnt;
+        done += width;
+        __syncthreads();
+        if (in_bin == need || done >= top) { limit = ((prefix + 1) << shift) - 1; break; }
+        if (in_bin <= RF_EDGE_CAP) {
+            // collect the boundary bin and rank its records: the need-th smallest is the limit
+            src.for_each([&](uint64_t rec, bool valid) {
+                if (valid && shr64(rec, shift) == prefix) {
+                    const uint32_t pos = atomicAdd(&sh.n_edge, 1u);
+                    if (pos < RF_EDGE_CAP) sh.edge[pos] = rec;
+                }
+            });
+            __syncthreads();
+            for (uint32_t i = tid; i < in_bin; i += nthr) {
+                const uint64_t mine = sh.edge[i];
+                uint32_t rank = 0;
+                for (uint32_t j = 0; j < in_bin; ++j) rank += sh.edge[j] < mine;
+                if (rank == need - 1) sh.limit = mine;
+            }
+            __syncthreads();
+            limit = sh.limit;
+            break;
+        }
+    }
+    // compact the winners (one shared-memory atomic per warp and visit)
+    src.for_each([&](uint64_t rec, bool valid) {
+        const bool take = valid && rec <= limit;
+        const unsigned bal = __ballot_sync(FULL_MASK, take);
+        if (bal) {
+            uint32_t base = 0;
+            if (lane == 0) base = atomicAdd(&sh.fill, (uint32_t)__popc(bal));
+            base = __shfl_sync(FULL_MASK, base, 0);
+            const uint32_t pos = base + __popc(bal & ((1u << lane) - 1u));
+            if (take && pos < sort_cap) sortbuf[pos] = rec;
+        }
+    });
+    __syncthreads();
+}
+
+// Ascending bitonic sort of P records (P a power of two, 32 <= P <= 1024), one per thread of
+// the first P threads.  Exchanges at distance < 32 are warp shuffles; only the longer ones
+// go through shared memory (scratch holds P records) with a named barrier over those P
+// threads, so the rest of the CTA does not take part.
+__device__ __forceinline__ uint64_t bitonic_sort_first_threads(uint64_t v, uint32_t P, uint64_t* scratch) {
+    const unsigned tid = threadIdx.x;
+    for (uint32_t size = 2; size <= P; size <<= 1) {
+        const bool ascending = (tid & size) == 0;
+        for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
+            uint64_t other;
+            if (stride >= 32) {
+                scratch[tid] = v;
+                asm volatile("bar.sync 1, %0;" ::"r"(P) : "memory");
+                other = scratch[tid ^ stride];
+                asm volatile("bar.sync 1, %0;" ::"r"(P) : "memory");
+            } else {
+                other = __shfl_xor_sync(FULL_MASK, v, stride);
+            }
+            const bool lower = (tid & stride) == 0;
+            const bool keep_min = lower == ascending;
+            v = (keep_min == (other < v)) ? other : v;
+        }
+    }
+    return v;
+}
+
 template <typename T>
-__global__ void refine_kernel(const RefineParams<T> p) {
+__device__ __forceinline__ void write_output(T* out_vals, int64_t* out_idx, uint32_t k, uint64_t row, uint32_t j, uint64_t rec) {
+    out_vals[row * (uint64_t)k + j] = Elem<T>::from_key(record_key(rec));
+    out_idx[row * (uint64_t)k + j] = (int64_t)record_idx(rec);
+}
+
+// Orders the m records in sortbuf (all threads have passed a barrier since they were written)
+// and writes the first kk of them, then the padding of relaxed mode, as row `row` of the output.
+template <typename T>
+__device__ __forceinline__ void sort_and_write(uint64_t* sortbuf, uint32_t m, uint32_t kk, uint32_t k, uint64_t row,
+                                               T* out_vals, int64_t* out_idx) {
+    const unsigned tid = threadIdx.x, nthr = blockDim.x;
+    for (uint32_t j = kk + tid; j < k; j += nthr) {       // relaxed mode: padding after a short buffer
+        out_vals[row * (uint64_t)k + j] = Elem<T>::from_bits(Elem<T>::NEG_INF_BITS);
+        out_idx[row * (uint64_t)k + j] = -1;
+    }
+    if (m <= nthr) {
+        uint32_t P = 32;
+        while (P < m) P <<= 1;
+        const uint64_t v0 = tid < m ? sortbuf[tid] : ~0ull;
+        __syncthreads();                                    // sortbuf doubles as the exchange scratch
+        if (tid < P) {
+            const uint64_t v = bitonic_sort_first_threads(v0, P, sortbuf);
+            if (tid < kk) write_output(out_vals, out_idx, k, row, tid, v);
+        }
+    } else {
+        uint32_t P = 1;
+        while (P < m) P <<= 1;
+        for (uint32_t i = m + tid; i < P; i += nthr) sortbuf[i] = ~0ull;
+        __syncthreads();
+        bitonic_sort_shared(sortbuf, P);
+        for (uint32_t j = tid; j < kk; j += nthr) write_output(out_vals, out_idx, k, row, j, sortbuf[j]);
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(1024) refine_kernel(const RefineParams<T> p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint64_t* sortbuf = reinterpret_cast<uint64_t*>(smem_raw);                 // sort_cap records
     uint64_t* staged = sortbuf + p.sort_cap;                                   // stage_cap records
-    __shared__ uint32_t hist[RF_BINS];
-    __shared__ uint32_t warp_sums[32];
-    __shared__ uint32_t s_digit, s_before, s_cnt, s_fill;
-    __shared__ unsigned long long s_or;
+    __shared__ SelectShared sh;
 
-    const unsigned tid = threadIdx.x, nthr = blockDim.x;
+    const unsigned tid = threadIdx.x, nthr = blockDim.x, lane = lane_id();
     const uint64_t row = blockIdx.x;
+    if (tid == 0) { sh.or_bits = 0ull; sh.fill = 0; sh.n_edge = 0; }
+    __syncthreads();
+    pdl_launch_dependents();                 // the exact-selection kernel may be staged behind this one
     if (p.use_pdl) pdl_wait();
+    PROFK_STAMP(1, 0);
 
-    uint32_t n = p.ctl[row].n_final;
-    if (n > p.capacity) n = p.capacity;
+    // ---- the count check of stage 4 ----
+    const RowCtl ctl = p.ctl[row];
+    const uint32_t R = ctl.count;
+    const uint32_t status = R > p.capacity ? ROW_OVERFLOW : R < p.k_accept ? ROW_RECALL : ROW_OK;
+    if (tid == 0) {
+        p.ctl[row].status = status;
+        p.ctl[row].n_final = status ? p.k : R;
+        if (status) atomicAdd(&p.header->n_failed, 1u);
+    }
+    if (status != ROW_OK) return;            // the exact-selection kernel takes this row
+
+    const uint32_t n = R;
     const uint32_t kk = n < p.k ? n : p.k;          // real outputs; the rest is padding (relaxed mode)
     const uint64_t* src = p.buf + row * (uint64_t)p.capacity;
 
-    const bool use_stage = n <= p.stage_cap && n > p.sort_cap;
-    if (use_stage) {
-        for (uint32_t i = tid; i < n; i += nthr) staged[i] = src[i];
+    uint32_t m;   // records in sortbuf that remain to be ordered
+    if (n <= p.sort_cap) {
+        for (uint32_t i = tid; i < n; i += nthr) sortbuf[i] = src[i];
+        m = n;
         __syncthreads();
-    }
-    const uint64_t* recs = use_stage ? staged : src;
-
-    uint32_t m;   // records to sort
-    if (n > p.sort_cap) {
-        // ---- radix select: limit = the kk-th smallest record ----
-        if (tid == 0) { s_or = 0ull; s_fill = 0; }
-        __syncthreads();
-        const uint64_t first = recs[0];
-        uint64_t diff = 0;
-        for (uint32_t i = tid; i < n; i += nthr) diff |= recs[i] ^ first;
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) diff |= __shfl_xor_sync(FULL_MASK, diff, d);
-        if (lane_id() == 0 && diff) atomicOr(&s_or, (unsigned long long)diff);
-        __syncthreads();
-        const int top = 64 - __clzll((long long)s_or);      // bits >= top are common to all records (s_or != 0: n >= 2)
-        uint64_t prefix = shr64(first, top);
-        uint32_t need = kk;
-        uint64_t limit = ~0ull;
-        for (int done = 0; done < top;) {
-            const int shift = top - done - 11 > 0 ? top - done - 11 : 0;
-            const int width = top - done - shift;
-            const uint32_t nbins = 1u << width;
-            for (uint32_t i = tid; i < nbins; i += nthr) hist[i] = 0;
-            __syncthreads();
-            for (uint32_t i = tid; i < n; i += nthr) {
-                const uint64_t rec = recs[i];
-                if (shr64(rec, shift + width) == prefix) atomicAdd(&hist[(uint32_t)(rec >> shift) & (nbins - 1)], 1u);
-            }
-            __syncthreads();
-            const uint32_t per = (RF_BINS + nthr - 1) / nthr;
+    } else {
+        bool resolved = false;
+        if (p.coarse != nullptr) {
+            // ---- scan the coarse histogram (bin 0 = largest keys) for the bin of the kk-th best record ----
+            const uint32_t* hist = p.coarse + row * COARSE_BINS;
+            const uint32_t per = (COARSE_BINS + nthr - 1) / nthr;
             uint32_t sum = 0;
             for (uint32_t j = 0; j < per; ++j) {
                 const uint32_t bin = tid * per + j;
-                sum += bin < nbins ? hist[bin] : 0;
+                sum += bin < COARSE_BINS ? __ldcg(&hist[bin]) : 0;
             }
-            uint32_t before = block_scan_any(sum, warp_sums) - sum;
+            uint32_t before = block_scan_any(sum, sh.warp_sums) - sum;
             for (uint32_t j = 0; j < per; ++j) {
                 const uint32_t bin = tid * per + j;
-                const uint32_t c = bin < nbins ? hist[bin] : 0;
-                if (before < need && need <= before + c) { s_digit = bin; s_before = before; s_cnt = c; }
+                const uint32_t c = bin < COARSE_BINS ? __ldcg(&hist[bin]) : 0;
+                if (before < kk && kk <= before + c) { sh.digit = bin; sh.before = before; sh.cnt = c; }
                 before += c;
             }
             __syncthreads();
-            prefix = (prefix << width) | s_digit;
-            need -= s_before;
-            const bool whole_bin = s_cnt == need;
-            done += width;
-            __syncthreads();
-            if (whole_bin || done >= top) { limit = ((prefix + 1) << shift) - 1; break; }
-        }
-        // ---- compact the kk winners into the sort area ----
-        for (uint32_t i = tid; i < n; i += nthr) {
-            const uint64_t rec = recs[i];
-            if (rec <= limit) {
-                const uint32_t pos = atomicAdd(&s_fill, 1u);
-                if (pos < p.sort_cap) sortbuf[pos] = rec;
+            const uint32_t edge_bin = sh.digit, need = kk - sh.before, in_bin = sh.cnt;
+            PROFK_STAMP(1, 1);
+            if (in_bin <= RF_EDGE_CAP) {
+                // ---- one pass over the records: those of better bins are winners, those of the boundary
+                //      bin go to the edge list; both are placed by a block-wide prefix sum ----
+                uint32_t run_w = 0, run_e = 0;
+                for (uint32_t base = 0; base < n; base += 8 * nthr) {
+                    uint64_t r[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const uint32_t i = base + u * nthr + tid;
+                        r[u] = i < n ? src[i] : 0ull;
+                    }
+                    uint32_t wmask = 0, emask = 0;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const uint32_t i = base + u * nthr + tid;
+                        const uint32_t bin = coarse_bin(record_key(r[u]), ctl.hi_key, ctl.bin_shift);
+                        if (i < n && bin < edge_bin) wmask |= 1u << u;
+                        if (i < n && bin == edge_bin) emask |= 1u << u;
+                    }
+                    const uint32_t cw = __popc(wmask), ce = __popc(emask);
+                    const uint32_t incl = block_scan_any(cw | (ce << 16), sh.warp_sums);   // two 16-bit counters
+                    if (tid == nthr - 1) sh.total = incl;
+                    uint32_t pw = run_w + (incl & 0xFFFFu) - cw, pe = run_e + (incl >> 16) - ce;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        if (wmask & (1u << u)) { if (pw < p.sort_cap) sortbuf[pw] = r[u]; ++pw; }
+                        if (emask & (1u << u)) { if (pe < RF_EDGE_CAP) sh.edge[pe] = r[u]; ++pe; }
+                    }
+                    __syncthreads();
+                    run_w += sh.total & 0xFFFFu;
+                    run_e += sh.total >> 16;
+                    __syncthreads();
+                }
+                PROFK_STAMP(1, 2);
+                // ---- rank the boundary bin; its `need` best records complete the winners ----
+                for (uint32_t i = tid; i < in_bin; i += nthr) {
+                    const uint64_t mine = sh.edge[i];
+                    uint32_t rank = 0;
+                    for (uint32_t j = 0; j < in_bin; ++j) rank += sh.edge[j] < mine;
+                    if (rank < need && run_w + rank < p.sort_cap) sortbuf[run_w + rank] = mine;
+                }
+                __syncthreads();
+                resolved = true;
             }
         }
-        m = kk;
-    } else {
-        for (uint32_t i = tid; i < n; i += nthr) sortbuf[i] = src[i];
-        m = n;
-    }
-
-    uint32_t P = 1;
-    while (P < m) P <<= 1;
-    for (uint32_t i = m + tid; i < P; i += nthr) sortbuf[i] = ~0ull;
-    __syncthreads();
-    bitonic_sort_shared(sortbuf, P);
-
-    T* ov = p.out_vals + row * (uint64_t)p.k;
-    int64_t* oi = p.out_idx + row * (uint64_t)p.k;
-    for (uint32_t j = tid; j < p.k; j += nthr) {
-        if (j < kk) {
-            const uint64_t rec = sortbuf[j];
-            ov[j] = Elem<T>::from_key(record_key(rec));
-            oi[j] = (int64_t)record_idx(rec);
-        } else {
-            ov[j] = Elem<T>::from_bits(Elem<T>::NEG_INF_BITS);
-            oi[j] = -1;
+        if (!resolved) {
+            // ---- general select (no usable histogram, or too many ties in the boundary bin) ----
+            const bool use_stage = n <= p.stage_cap;
+            const uint64_t first = src[0];
+            uint64_t diff = 0;
+            for (uint32_t base = 0; base < n; base += 8 * nthr) {
+                uint64_t r[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const uint32_t i = base + u * nthr + tid;
+                    r[u] = i < n ? src[i] : first;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const uint32_t i = base + u * nthr + tid;
+                    diff |= r[u] ^ first;
+                    if (use_stage && i < n) staged[i] = r[u];
+                }
+            }
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) diff |= __shfl_xor_sync(FULL_MASK, diff, d);
+            if (lane == 0 && diff) atomicOr(&sh.or_bits, (unsigned long long)diff);
+            __syncthreads();
+            MemRecords mem{use_stage ? staged : src, n};
+            select_smallest(mem, first, kk, sortbuf, p.sort_cap, sh);
         }
+        m = kk;
     }
+    PROFK_STAMP(1, 3);
+    sort_and_write<T>(sortbuf, m, kk, p.k, row, p.out_vals, p.out_idx);
+    PROFK_STAMP(1, 4);
 }
 
 }  // namespace profk

@@ -2,12 +2,21 @@
 // Philox samples of a row and select the t-th largest as the threshold tau.
 //
 // One thread-block cluster handles one row.  Each CTA of the cluster gathers its share of
-// the samples into shared memory as order keys; the t-th largest key is found by a radix
-// select whose per-digit histograms are summed across the cluster through distributed
-// shared memory (hardware cluster barriers only -- no spinning on global memory).
+// the samples into shared memory as order keys.  The t-th largest key is then found by
+//   * a short cut for small ranks (t <= 128): every CTA derives a lower bound L on the
+//     answer from the maxima of 128 groups of its keys (the t-th largest group maximum has
+//     at least t keys at or above it), sends only its keys >= L to the first CTA through
+//     distributed shared memory (remote atomics and stores), and the first CTA ranks those
+//     few candidates directly;
+//   * otherwise (deep ranks, or so many ties that the candidates do not fit) a radix select
+//     whose per-digit histograms are summed across the cluster through distributed shared
+//     memory.
+// Only hardware cluster barriers are used -- no spinning on global memory.
 #pragma once
 
 #include <cooperative_groups.h>
+
+#include <utility>
 
 #include "common.cuh"
 
@@ -16,7 +25,9 @@ namespace profk {
 namespace cg = cooperative_groups;
 
 constexpr int SEL_THREADS = 1024;
-constexpr int SEL_BINS = 2048;       // 11-bit digits
+constexpr int SEL_BINS = 2048;        // 11-bit digits
+constexpr int SEL_GROUPS = 128;       // groups of 8 lanes whose maxima bound the answer from below
+constexpr uint32_t SEL_CAND_CAP = 1024;
 
 // Per-row control block in the workspace.
 struct RowCtl {
@@ -26,7 +37,8 @@ struct RowCtl {
     uint32_t status;     // PROFK_ROW_* (| 0x80000000 on a timeout)
     uint32_t n_final;    // records the refine step has to order
     uint32_t capacity;
-    uint32_t pad[2];
+    uint32_t hi_key;     // coarse histogram: largest sampled key ...
+    uint32_t bin_shift;  // ... and the shift that maps [tau, hi_key] onto COARSE_BINS bins
 };
 static_assert(sizeof(RowCtl) == 32, "RowCtl is 32 bytes");
 
@@ -35,7 +47,9 @@ struct WsHeader {
     uint32_t bar_count;
     uint32_t bar_gen;
     uint32_t error;      // non-zero = a bounded wait gave up
-    uint32_t pad[61];
+    uint32_t done;       // CTAs of the filter kernel that have finished (ticket for its last CTA)
+    uint32_t n_failed;   // rows whose count check failed (written by the filter's last CTA)
+    uint32_t pad[59];
 };
 static_assert(sizeof(WsHeader) == 256, "WsHeader is 256 bytes");
 
@@ -45,15 +59,51 @@ template <typename T> struct SelectParams {
     uint32_t S;            // sample size
     uint32_t t;            // rank, 1-based, t-th largest
     uint64_t seed;
-    uint32_t per_cta;      // samples per CTA of the cluster = ceil(S / cluster size)
+    uint32_t per_cta;      // samples per CTA of the cluster (even)
+    uint64_t q;            // N / S
+    uint32_t rem;          // N % S
+    float inv_s;           // 1 / S
     T* tau;                // rows thresholds out
     RowCtl* ctl;           // may be null (stand-alone use)
     WsHeader* header;      // may be null
     uint32_t capacity;
+    uint32_t* coarse;      // may be null; rows x COARSE_BINS survivor histogram, zeroed here
     uint32_t* sample_idx;  // may be null; rows x S
 };
 
-// Block-wide inclusive scan of one value per thread (blockDim.x == SEL_THREADS).
+// Writes tau and the parameters of the coarse survivor histogram for one row.
+template <typename T>
+__device__ __forceinline__ void publish_threshold(const SelectParams<T>& p, uint64_t row, uint32_t tau_key, uint32_t max_key) {
+    const T tau = Elem<T>::from_key(tau_key);
+    p.tau[row] = tau;
+    if (p.ctl) {
+        RowCtl* c = p.ctl + row;
+        c->tau_bits = Elem<T>::bits(tau);
+        // The largest sampled key sits near rank N/S of the row, so the histogram reaches three
+        // sample spans above it; whatever lies higher still shares bin 0.
+        const uint64_t span = (uint64_t)max_key - tau_key;            // max_key >= tau_key
+        const uint64_t top = (uint64_t)max_key + 3 * span;
+        const uint32_t hi_key = top > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)top;
+        c->hi_key = hi_key;
+        const uint32_t range = hi_key - tau_key;
+        const int bits = 32 - __clz(range);                           // range < 2^bits
+        c->bin_shift = bits > COARSE_BITS ? (uint32_t)(bits - COARSE_BITS) : 0u;
+    }
+}
+
+// floor(j * N / S) = j * (N / S) + floor(j * (N % S) / S).  The second quotient is below S
+// (< 2^18), so a float estimate is within one of it and an integer check repairs it.
+__device__ __forceinline__ uint64_t stratum_start(uint64_t j, uint64_t q, uint32_t rem, uint32_t S, float inv_s) {
+    if (rem == 0) return j * q;
+    const uint64_t x = j * (uint64_t)rem;
+    int64_t e = (int64_t)((float)x * inv_s);
+    int64_t r = (int64_t)x - e * (int64_t)S;
+    while (r < 0) { --e; r += S; }
+    while (r >= (int64_t)S) { ++e; r -= S; }
+    return j * q + (uint64_t)e;
+}
+
+// Block-wide inclusive scan of one value per thread (blockDim.x == SEL_THREADS or fewer warps).
 __device__ __forceinline__ uint32_t block_inclusive_scan(uint32_t v, uint32_t* warp_sums) {
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
 #pragma unroll
@@ -82,84 +132,219 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw);          // per_cta keys
     __shared__ uint32_t hist[2][SEL_BINS];                           // this CTA's histogram, double-buffered
+    __shared__ uint32_t cand[SEL_CAND_CAP];                          // candidates (filled in the first CTA only)
+    __shared__ uint32_t gmax[SEL_GROUPS];
     __shared__ uint32_t warp_sums[32];
-    __shared__ uint32_t s_digit, s_before;
+    __shared__ uint32_t s_digit, s_before, s_ncand, s_lower;
 
     cg::cluster_group cluster = cg::this_cluster();
     const unsigned csize = cluster.num_blocks();
     const unsigned crank = cluster.block_rank();
     const uint64_t row = blockIdx.x / csize;
-    const unsigned tid = threadIdx.x;
+    const unsigned tid = threadIdx.x, lane = lane_id();
 
     pdl_launch_dependents();   // the filter kernel may start its prologue now
+    PROFK_STAMP(0, 0);
+
+    if (tid == 0) { s_ncand = 0; s_lower = 0; }
+    __syncthreads();
+    // Split barrier: "my candidate counter is zero".  Peers wait for it only after their gather,
+    // by which time every CTA has long arrived.
+    auto zeroed = cluster.barrier_arrive();
 
     // ---- stage 1: gather this CTA's share of the sample -------------------------------
+    // Samples come in pairs: one Philox block (four words) serves samples 2p and 2p+1.
     const uint32_t j0 = crank * p.per_cta;
     const uint32_t j1 = min(p.S, j0 + p.per_cta);
     const uint32_t n_local = j1 > j0 ? j1 - j0 : 0;
+    const uint32_t n_round = (n_local + 31u) & ~31u;                 // whole warps take part in ballots
     const T* rowp = p.in + row * p.N;
-    for (uint32_t i = tid; i < n_local; i += SEL_THREADS) {
-        const uint32_t idx = sample_index(p.N, p.S, j0 + i, row, p.seed);
-        keys[i] = Elem<T>::key(rowp[idx]);
-        if (p.sample_idx) p.sample_idx[row * p.S + j0 + i] = idx;
+    uint32_t my_max = 0;
+    constexpr int PB = 2;                                            // pairs per batch: 4 loads in flight per thread
+    for (uint32_t pp0 = 0; 2 * pp0 < n_local; pp0 += PB * SEL_THREADS) {
+        uint32_t idx[2 * PB];
+        bool ok[2 * PB];
+#pragma unroll
+        for (int b = 0; b < PB; ++b) {
+            const uint32_t pp = pp0 + b * SEL_THREADS + tid;
+            const uint64_t j = (uint64_t)j0 + 2ull * pp;             // even sample of the pair
+            ok[2 * b] = j < j1;
+            ok[2 * b + 1] = j + 1 < j1;
+            idx[2 * b] = idx[2 * b + 1] = 0;
+            if (ok[2 * b]) {
+                const Philox4 r = philox4x32_10((uint32_t)(j >> 1), (uint32_t)row, (uint32_t)(row >> 32), 0u,
+                                                (uint32_t)p.seed, (uint32_t)(p.seed >> 32));
+                const uint64_t b0 = stratum_start(j, p.q, p.rem, p.S, p.inv_s);
+                const uint64_t b1 = stratum_start(j + 1, p.q, p.rem, p.S, p.inv_s);
+                idx[2 * b] = (uint32_t)(b0 + __umul64hi(((uint64_t)r.y << 32) | r.x, b1 - b0));
+                if (ok[2 * b + 1]) {
+                    const uint64_t b2 = stratum_start(j + 2, p.q, p.rem, p.S, p.inv_s);
+                    idx[2 * b + 1] = (uint32_t)(b1 + __umul64hi(((uint64_t)r.w << 32) | r.z, b2 - b1));
+                }
+            }
+        }
+        T val[2 * PB];
+#pragma unroll
+        for (int s = 0; s < 2 * PB; ++s)
+            if (ok[s]) val[s] = rowp[idx[s]];
+#pragma unroll
+        for (int s = 0; s < 2 * PB; ++s) {
+            if (ok[s]) {
+                const uint32_t pp = pp0 + (s >> 1) * SEL_THREADS + tid;
+                const uint32_t local = 2 * pp + (s & 1);
+                const uint32_t k = Elem<T>::key(val[s]);
+                keys[local] = k;
+                my_max = max(my_max, k);
+                if (p.sample_idx) p.sample_idx[row * p.S + j0 + local] = idx[s];
+            }
+        }
+    }
+    if (p.coarse) {   // the CTAs of the cluster share the zeroing of the row's histogram
+        uint32_t* h = p.coarse + row * COARSE_BINS;
+        for (uint32_t b = crank * SEL_THREADS + tid; b < COARSE_BINS; b += csize * SEL_THREADS) h[b] = 0;
     }
     if (crank == 0 && tid == 0) {
         if (p.ctl) {
             RowCtl* c = p.ctl + row;
             c->count = 0; c->collect = 0; c->status = 0; c->n_final = 0; c->capacity = p.capacity;
         }
-        if (p.header && row == 0) { p.header->bar_count = 0; p.header->error = 0; }
+        if (p.header && row == 0) { p.header->bar_count = 0; p.header->error = 0; p.header->done = 0; p.header->n_failed = 0; }
     }
+    PROFK_STAMP(0, 1);
 
-    // ---- stage 2: radix select of the t-th largest key over the cluster ----------------
-    constexpr int NPASS = sizeof(T) == 4 ? 3 : 2;
-    const int shifts[3] = {21, sizeof(T) == 4 ? 10 : 16, 0};
-    const int widths[3] = {11, sizeof(T) == 4 ? 11 : 5, 10};
+    bool done = false;
 
-    uint32_t prefix = 0;        // selected high bits so far (right-aligned)
-    uint32_t need = p.t;        // rank among the keys that match the prefix, from the top
-    int consumed = 0;           // number of high bits fixed
-#pragma unroll
-    for (int pass = 0; pass < NPASS; ++pass) {
-        const int shift = shifts[pass], width = widths[pass];
-        const uint32_t nbins = 1u << width;
-        uint32_t* h = hist[pass & 1];
-        for (uint32_t b = tid; b < nbins; b += SEL_THREADS) h[b] = 0;
+    // ---- stage 2, short cut for small ranks -------------------------------------------
+    if (p.t <= SEL_GROUPS) {
+        // maxima of the 128 groups of 8 consecutive lanes
+        uint32_t g = my_max;
+        g = max(g, __shfl_xor_sync(FULL_MASK, g, 1));
+        g = max(g, __shfl_xor_sync(FULL_MASK, g, 2));
+        g = max(g, __shfl_xor_sync(FULL_MASK, g, 4));
+        if ((tid & 7u) == 0) gmax[tid >> 3] = g;
         __syncthreads();
-        for (uint32_t i = tid; i < n_local; i += SEL_THREADS) {
-            const uint32_t k = keys[i];
-            if (consumed == 0 || (k >> (32 - consumed)) == prefix) atomicAdd(&h[(k >> shift) & (nbins - 1)], 1u);
+        {   // rank of group tid/8 among the 128 maxima, the eight lanes of the group sharing the loop
+            const unsigned grp = tid >> 3, part = tid & 7u;
+            const uint32_t mine = gmax[grp];
+            uint32_t rank = 0;
+#pragma unroll
+            for (int jj = 0; jj < SEL_GROUPS / 8; ++jj) {
+                const unsigned j = part * (SEL_GROUPS / 8) + jj;
+                const uint32_t o = gmax[j];
+                rank += (o > mine) || (o == mine && j < grp);
+            }
+            rank += __shfl_xor_sync(FULL_MASK, rank, 1);
+            rank += __shfl_xor_sync(FULL_MASK, rank, 2);
+            rank += __shfl_xor_sync(FULL_MASK, rank, 4);
+            if (part == 0 && rank == p.t - 1) s_lower = mine;     // at least t keys of this CTA are >= mine
         }
-        cluster.sync();   // every CTA's histogram of this pass is complete
-
-        // Sum the histograms of all CTAs; thread t owns the two bins 2t, 2t+1 counted from the top.
-        uint32_t c0 = 0, c1 = 0;
-        const uint32_t rb0 = 2 * tid, rb1 = 2 * tid + 1;            // reversed bin numbers
-        if (rb0 < nbins) {
-            for (unsigned c = 0; c < csize; ++c) {
-                const uint32_t* ph = cluster.map_shared_rank(h, c);
-                c0 += ph[nbins - 1 - rb0];
-                c1 += ph[nbins - 1 - rb1];
+        __syncthreads();
+        const uint32_t lower = s_lower;
+        PROFK_STAMP(0, 2);
+        // every CTA sends its keys >= lower to the first CTA: one remote atomic per warp that has any
+        uint32_t* cand0 = cluster.map_shared_rank(cand, 0);
+        uint32_t* ncand0 = cluster.map_shared_rank(&s_ncand, 0);
+        cluster.barrier_wait(std::move(zeroed));
+        for (uint32_t i = tid; i < n_round; i += SEL_THREADS) {
+            const uint32_t k = i < n_local ? keys[i] : 0;
+            const bool take = i < n_local && k >= lower;
+            const unsigned bal = __ballot_sync(FULL_MASK, take);
+            if (bal) {
+                uint32_t base = 0;
+                if (lane == 0) base = atomicAdd(ncand0, (uint32_t)__popc(bal));
+                base = __shfl_sync(FULL_MASK, base, 0);
+                const uint32_t slot = base + __popc(bal & ((1u << lane) - 1u));
+                if (take && slot < SEL_CAND_CAP) cand0[slot] = k;
             }
         }
-        const uint32_t incl = block_inclusive_scan(c0 + c1, warp_sums);   // keys in reversed bins <= rb1
-        const uint32_t before0 = incl - c0 - c1, before1 = incl - c1;
-        if (before0 < need && need <= before0 + c0) { s_digit = nbins - 1 - rb0; s_before = before0; }
-        else if (before1 < need && need <= before1 + c1) { s_digit = nbins - 1 - rb1; s_before = before1; }
-        __syncthreads();
-        prefix = (prefix << width) | s_digit;
-        need -= s_before;
-        consumed += width;
-        __syncthreads();   // s_digit / s_before are rewritten in the next pass
+        PROFK_STAMP(0, 3);
+        cluster.sync();                               // all candidates have arrived
+        PROFK_STAMP(0, 4);
+        const uint32_t ncand = *ncand0;
+        auto seen = cluster.barrier_arrive();         // "I have read the count": the first CTA may leave after its peers did
+        if (ncand <= SEL_CAND_CAP) {
+            if (crank == 0) {
+                // rank the candidates, eight lanes per candidate sharing the comparison loop
+                const unsigned part = tid & 7u;
+                for (uint32_t c0 = 0; c0 < ncand; c0 += SEL_THREADS / 8) {
+                    const uint32_t c = c0 + (tid >> 3);
+                    const uint32_t mine = c < ncand ? cand[c] : 0;
+                    uint32_t rank = 0;
+                    for (uint32_t j = part; j < ncand; j += 8) {
+                        const uint32_t o = cand[j];
+                        rank += (o > mine) || (o == mine && j < c);
+                    }
+                    rank += __shfl_xor_sync(FULL_MASK, rank, 1);
+                    rank += __shfl_xor_sync(FULL_MASK, rank, 2);
+                    rank += __shfl_xor_sync(FULL_MASK, rank, 4);
+                    if (part == 0 && c < ncand && rank == 0) s_lower = mine;      // the largest sampled key
+                    if (part == 0 && c < ncand && rank == p.t - 1) s_digit = mine; // the t-th largest: tau
+                }
+            }
+            if (crank == 0) {
+                __syncthreads();
+                if (tid == 0) publish_threshold(p, row, s_digit, s_lower);
+            }
+            done = true;
+            PROFK_STAMP(0, 5);
+            cluster.barrier_wait(std::move(seen));
+        } else {
+            cluster.barrier_wait(std::move(seen));
+        }
+    } else {
+        cluster.barrier_wait(std::move(zeroed));
     }
-    const uint32_t tau_key = prefix << (32 - consumed);
 
-    if (crank == 0 && tid == 0) {
-        const T tau = Elem<T>::from_key(tau_key);
-        p.tau[row] = tau;
-        if (p.ctl) p.ctl[row].tau_bits = Elem<T>::bits(tau);
+    // ---- stage 2, general case: radix select over the cluster --------------------------
+    if (!done) {
+        constexpr int NPASS = sizeof(T) == 4 ? 3 : 2;
+        const int shifts[3] = {21, sizeof(T) == 4 ? 10 : 16, 0};
+        const int widths[3] = {11, sizeof(T) == 4 ? 11 : 5, 10};
+        uint32_t prefix = 0;        // selected high bits so far (right-aligned)
+        uint32_t need = p.t;        // rank among the keys that match the prefix, from the top
+        int consumed = 0;           // number of high bits fixed
+#pragma unroll
+        for (int pass = 0; pass < NPASS; ++pass) {
+            const int shift = shifts[pass], width = widths[pass];
+            const uint32_t nbins = 1u << width;
+            uint32_t* h = hist[pass & 1];
+            for (uint32_t b = tid; b < nbins; b += SEL_THREADS) h[b] = 0;
+            __syncthreads();
+            for (uint32_t i = tid; i < n_round; i += SEL_THREADS) {
+                const uint32_t k = i < n_local ? keys[i] : 0;
+                const bool in_class = i < n_local && (consumed == 0 || (k >> (32 - consumed)) == prefix);
+                const uint32_t digit = in_class ? (k >> shift) & (nbins - 1) : 0xFFFFFFFFu;
+                const unsigned peers = __match_any_sync(FULL_MASK, digit);
+                if (in_class && lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&h[digit], __popc(peers));
+            }
+            cluster.sync();   // every CTA's histogram of this pass is complete
+
+            // Sum the histograms of all CTAs; thread t owns the two bins 2t, 2t+1 counted from the top.
+            uint32_t c0 = 0, c1 = 0;
+            const uint32_t rb0 = 2 * tid, rb1 = 2 * tid + 1;            // reversed bin numbers
+            if (rb0 < nbins) {
+#pragma unroll 4
+                for (unsigned c = 0; c < csize; ++c) {
+                    const uint32_t* ph = cluster.map_shared_rank(h, c);
+                    c0 += ph[nbins - 1 - rb0];
+                    c1 += ph[nbins - 1 - rb1];
+                }
+            }
+            const uint32_t incl = block_inclusive_scan(c0 + c1, warp_sums);   // keys in reversed bins <= rb1
+            const uint32_t before0 = incl - c0 - c1, before1 = incl - c1;
+            if (before0 < need && need <= before0 + c0) { s_digit = nbins - 1 - rb0; s_before = before0; }
+            else if (before1 < need && need <= before1 + c1) { s_digit = nbins - 1 - rb1; s_before = before1; }
+            __syncthreads();
+            prefix = (prefix << width) | s_digit;
+            need -= s_before;
+            consumed += width;
+            __syncthreads();   // s_digit / s_before are rewritten in the next pass
+        }
+        const uint32_t tau_key = prefix << (32 - consumed);
+        if (crank == 0 && tid == 0) publish_threshold(p, row, tau_key, 0xFFFFFFFFu);   // no cheap maximum on this path
+        cluster.sync();   // no CTA leaves while a peer may still read its histogram
     }
-    cluster.sync();   // no CTA leaves while a peer may still read its histogram
+    PROFK_STAMP(0, 6);
 }
 
 }  // namespace profk
