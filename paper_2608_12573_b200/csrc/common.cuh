@@ -69,17 +69,6 @@ __device__ __forceinline__ uint64_t make_record(uint32_t key, uint32_t idx) {
 __device__ __forceinline__ uint32_t record_key(uint64_t rec) { return ~(uint32_t)(rec >> 32); }
 __device__ __forceinline__ uint32_t record_idx(uint64_t rec) { return (uint32_t)rec; }
 
-// Coarse histogram of the survivors, filled by the filter and read by the refine step:
-// bin 0 holds the largest keys.  hi_key is (an estimate of) the largest key, shift scales
-// the distance below it to COARSE_BINS bins; keys above hi_key land in bin 0, keys far
-// below it in the last bin.
-constexpr int COARSE_BITS = 12;
-constexpr uint32_t COARSE_BINS = 1u << COARSE_BITS;
-__device__ __forceinline__ uint32_t coarse_bin(uint32_t key, uint32_t hi_key, uint32_t shift) {
-    const uint32_t d = key >= hi_key ? 0u : (hi_key - key) >> shift;
-    return d < COARSE_BINS ? d : COARSE_BINS - 1;
-}
-
 // ---------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon et al., SC'11): ten rounds, key bumped by the Weyl constants between rounds.
 struct Philox4 { uint32_t x, y, z, w; };

@@ -4,12 +4,10 @@
 // The kernel is bound by HBM bandwidth: one 128-bit load per VEC elements, one compare
 // per element, and nothing else on the common path.  Survivors are rare (1e-3 .. 1e-5 of
 // the elements), so the append is a warp-cooperative slow path taken only when some lane
-// of the warp saw a survivor: a warp prefix sum, one global atomic per warp, and one
-// histogram increment per survivor for the refine step.
+// of the warp saw a survivor: a warp prefix sum and one global atomic per warp.
 #pragma once
 
 #include "rowscan.cuh"
-#include "sample_select.cuh"
 
 // Launch shape of the filter kernel (tuned on B200; overridable at build time for experiments).
 #ifndef PROFK_FILTER_THREADS
@@ -39,8 +37,6 @@ template <typename T> struct FilterParams {
     uint64_t tiles_per_row;
     uint64_t total_tiles;
     int use_pdl;             // 1 = launched as a programmatic dependent of the threshold kernel
-    const RowCtl* ctl;       // per-row histogram parameters (needed only with `coarse`)
-    uint32_t* coarse;        // rows x COARSE_BINS survivor histogram (null = none)
 };
 
 // not (x < tau) for every lane of a vector, OR-ed: does the vector hold any survivor?
@@ -114,14 +110,6 @@ __global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOC
             }
             const unsigned total = __shfl_sync(FULL_MASK, incl, 31);
             if (total) {
-                // the histogram parameters travel while the counter atomic is in flight
-                uint32_t hi_key = 0, bin_shift = 0;
-                uint32_t* hist = nullptr;
-                if (p.coarse) {
-                    hi_key = p.ctl[row].hi_key;
-                    bin_shift = p.ctl[row].bin_shift;
-                    hist = p.coarse + (uint64_t)row * COARSE_BINS;
-                }
                 unsigned base = 0;
                 if (lane == 0) base = atomicAdd(p.counts + (uint64_t)row * p.count_stride, total);
                 base = __shfl_sync(FULL_MASK, base, 0);
@@ -135,9 +123,8 @@ __global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOC
 #pragma unroll
                         for (int l = 0; l < VEC; ++l) {
                             if (mine[u] & (1u << l)) {
-                                const uint32_t key = Elem<T>::key(vec_elem(v[u], l));
-                                if (pos < p.capacity) dst[pos] = make_record(key, (uint32_t)(i0 + l));
-                                if (hist) atomicAdd(&hist[coarse_bin(key, hi_key, bin_shift)], 1u);
+                                if (pos < p.capacity)
+                                    dst[pos] = make_record(Elem<T>::key(vec_elem(v[u], l)), (uint32_t)(i0 + l));
                                 ++pos;
                             }
                         }

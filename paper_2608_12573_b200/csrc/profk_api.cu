@@ -24,7 +24,7 @@ namespace {
 constexpr int FILTER_THREADS = PROFK_FILTER_THREADS;
 constexpr int FILTER_UNROLL = PROFK_FILTER_UNROLL;
 constexpr uint32_t SORT_CAP_MAX = 8192;          // largest k the single-CTA refine orders in shared memory
-constexpr size_t REFINE_SMEM_MAX = 200 * 1024;   // dynamic shared memory the refine kernel may ask for
+constexpr size_t REFINE_SMEM_MAX = 160 * 1024;   // dynamic shared memory the refine kernel may ask for (it has ~41 KB static)
 constexpr int64_t N_MAX = 4278190080LL;          // 2^32 - 2^24
 constexpr int64_t M_MAX = 262144;                // largest sample the cluster select holds (8 CTAs x 32768 keys)
 
@@ -49,7 +49,7 @@ std::map<std::tuple<int64_t, int64_t, double, double>, profk_plan_t> g_plan_cach
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-    size_t off_header, off_ghist, off_ctl, off_tau, off_coarse, off_buf, total;
+    size_t off_header, off_ghist, off_ctl, off_tau, off_buf, total;
 };
 
 WsLayout ws_layout(int64_t rows, int64_t capacity) {
@@ -58,8 +58,7 @@ WsLayout ws_layout(int64_t rows, int64_t capacity) {
     l.off_ghist = sizeof(WsHeader);
     l.off_ctl = align_up(l.off_ghist + (size_t)FB_PASSES * FB_BINS * sizeof(uint32_t), 256);
     l.off_tau = align_up(l.off_ctl + (size_t)rows * sizeof(RowCtl), 256);
-    l.off_coarse = align_up(l.off_tau + (size_t)rows * 4, 256);
-    l.off_buf = align_up(l.off_coarse + (size_t)rows * COARSE_BINS * sizeof(uint32_t), 256);
+    l.off_buf = align_up(l.off_tau + (size_t)rows * 4, 256);
     l.total = align_up(l.off_buf + (size_t)rows * (size_t)capacity * sizeof(uint64_t), 256);
     return l;
 }
@@ -129,13 +128,13 @@ int pick_cluster(int64_t rows, int64_t m, int max_cluster) {
 
 template <typename T>
 int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, int64_t m, int64_t r, uint64_t seed, T* tau, RowCtl* ctl,
-                         WsHeader* header, uint32_t capacity, uint32_t* coarse, uint32_t* sample_idx, cudaStream_t st) {
+                         WsHeader* header, uint32_t capacity, uint32_t* sample_idx, cudaStream_t st) {
     const int csize = pick_cluster(rows, m, di.max_cluster[dtype_index<T>()]);
     SelectParams<T> sp;
     sp.in = in; sp.N = (uint64_t)N; sp.S = (uint32_t)m; sp.t = (uint32_t)r; sp.seed = seed;
     sp.per_cta = (uint32_t)(((m + csize - 1) / csize + 1) & ~1LL);      // even: samples are drawn in pairs
     sp.q = (uint64_t)(N / m); sp.rem = (uint32_t)(N % m); sp.inv_s = 1.0f / (float)m;
-    sp.tau = tau; sp.ctl = ctl; sp.header = header; sp.capacity = capacity; sp.coarse = coarse; sp.sample_idx = sample_idx;
+    sp.tau = tau; sp.ctl = ctl; sp.header = header; sp.capacity = capacity; sp.sample_idx = sample_idx;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(rows * csize));
     cfg.blockDim = dim3(SEL_THREADS);
@@ -152,7 +151,7 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
 
 template <typename T>
 int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, const T* tau, int64_t capacity, uint64_t* buf,
-                  uint32_t* counts, uint32_t count_stride, bool pdl, const RowCtl* ctl, uint32_t* coarse, cudaStream_t st) {
+                  uint32_t* counts, uint32_t count_stride, bool pdl, cudaStream_t st) {
     FilterParams<T> fp;
     fp.in = in; fp.N = (uint64_t)N; fp.rows = (uint64_t)rows; fp.tau = tau; fp.capacity = (uint32_t)capacity;
     fp.buf = buf; fp.counts = counts; fp.count_stride = count_stride;
@@ -160,7 +159,6 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     fp.total_tiles = fp.tiles_per_row * (uint64_t)rows;
     if (fp.total_tiles >= (1ull << 32)) return PROFK_EINVAL;      // rows * N beyond 2^45 elements
     fp.use_pdl = pdl ? 1 : 0;
-    fp.ctl = ctl; fp.coarse = coarse;
     const uint64_t max_grid = (uint64_t)di.sm_count * di.filter_blocks_per_sm[dtype_index<T>()];
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)std::min<uint64_t>(fp.total_tiles, max_grid));
@@ -210,7 +208,6 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     uint32_t* ghist = reinterpret_cast<uint32_t*>(base + lay.off_ghist);
     RowCtl* ctl = reinterpret_cast<RowCtl*>(base + lay.off_ctl);
     T* tau = reinterpret_cast<T*>(base + lay.off_tau);
-    uint32_t* coarse = reinterpret_cast<uint32_t*>(base + lay.off_coarse);
     uint64_t* buf = reinterpret_cast<uint64_t*>(base + lay.off_buf);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
@@ -218,28 +215,24 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     while (sort_cap < (uint32_t)k) sort_cap <<= 1;
 
     if (plan->mode == 0) {
-        rc = launch_sample_select<T>(di, in, rows, N, plan->m, plan->r, seed, tau, ctl, header, (uint32_t)capacity, coarse, nullptr, st);
+        rc = launch_sample_select<T>(di, in, rows, N, plan->m, plan->r, seed, tau, ctl, header, (uint32_t)capacity, nullptr, st);
         if (rc != PROFK_OK) return rc;
-        rc = launch_filter<T>(di, in, rows, N, tau, capacity, buf, &ctl[0].count, sizeof(RowCtl) / 4, true, ctl, coarse, st);
+        rc = launch_filter<T>(di, in, rows, N, tau, capacity, buf, &ctl[0].count, sizeof(RowCtl) / 4, true, st);
         if (rc != PROFK_OK) return rc;
 
         // refine: count check, then order the buffer of every row that passed it
         RefineParams<T> rp;
         rp.ctl = ctl; rp.header = header; rp.buf = buf; rp.capacity = (uint32_t)capacity; rp.k = (uint32_t)k;
         rp.k_accept = (uint32_t)plan->k_accept;
-        uint32_t rsort = sort_cap;
-        while (rsort < 2048 && rsort < (uint32_t)capacity) rsort <<= 1;     // small buffers are sorted whole
-        rp.sort_cap = rsort;
-        const size_t room = (REFINE_SMEM_MAX - (size_t)rsort * 8) / 8;
-        rp.stage_cap = (uint32_t)std::min<size_t>((size_t)capacity, room);
-        if (rp.stage_cap <= rsort) rp.stage_cap = 0;
-        rp.out_vals = out_vals; rp.out_idx = out_idx; rp.use_pdl = 1; rp.coarse = coarse;
+        rp.sort_cap = sort_cap;
+        rp.stage_cap = 0;            // the general select (crowded bins only) reads the buffer in place
+        rp.out_vals = out_vals; rp.out_idx = out_idx; rp.use_pdl = 1;
         unsigned threads = 128;
         while (threads < 1024 && threads * 8 < (unsigned)capacity) threads <<= 1;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)rows);
         cfg.blockDim = dim3(threads);
-        cfg.dynamicSmemBytes = ((size_t)rsort + rp.stage_cap) * 8;
+        cfg.dynamicSmemBytes = ((size_t)sort_cap + RF_EDGE_CAP + rp.stage_cap) * 8;
         cfg.stream = st;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -328,8 +321,7 @@ int filter_only(const T* in, int64_t rows, int64_t N, const T* tau, int64_t capa
     DeviceInfo di;
     const int rc = ensure_device_info<T>(dev, &di);
     if (rc != PROFK_OK) return rc;
-    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, counts, 1, false, nullptr, nullptr,
-                            static_cast<cudaStream_t>(stream));
+    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, counts, 1, false, static_cast<cudaStream_t>(stream));
 }
 
 template <typename T>
@@ -343,7 +335,7 @@ int sample_threshold(const T* in, int64_t rows, int64_t N, int64_t m, int64_t r,
     DeviceInfo di;
     const int rc = ensure_device_info<T>(dev, &di);
     if (rc != PROFK_OK) return rc;
-    return launch_sample_select<T>(di, in, rows, N, m, r, seed, tau, nullptr, nullptr, 0, nullptr, sample_idx, static_cast<cudaStream_t>(stream));
+    return launch_sample_select<T>(di, in, rows, N, m, r, seed, tau, nullptr, nullptr, 0, sample_idx, static_cast<cudaStream_t>(stream));
 }
 
 }  // namespace

@@ -4,12 +4,13 @@
 // Candidate records are 64-bit integers whose ascending order is exactly that order, so
 // refinement is "the k smallest records, sorted".  One CTA per row.  The CTA first takes the
 // paper's check -- fewer than k candidates, or more than the buffer holds, means the row is
-// left to the exact-selection kernel that follows.  Otherwise: the filter kernel has already
-// counted the survivors into a coarse 4096-bin histogram, so one scan of that histogram finds
-// the bin holding the k-th best record; a single pass over the buffer keeps the records of
-// better bins (placed by prefix sums, no atomics) and ranks the few records of the boundary
-// bin.  When the histogram cannot be used (ties pile up in one bin) a most-significant-digit
-// radix select over the records does the same job.  A bitonic sort orders the k winners.
+// left to the exact-selection kernel that follows.  Otherwise the records (held in registers
+// when they fit) are binned by their key's distance above tau into 4096 bins; a scan of the
+// bin counts gives every bin its first output position and finds the bin that holds the k-th
+// best record; the records of that bin and of all better bins are grouped by bin in shared
+// memory, and each of them finds its final position by ranking itself inside its (small) bin.
+// No sort is needed.  When a bin is too crowded for that (many equal values) a
+// most-significant-digit radix select plus a bitonic sort does the same job.
 #pragma once
 
 #include "sample_select.cuh"
@@ -29,12 +30,11 @@ template <typename T> struct RefineParams {
     uint32_t capacity;
     uint32_t k;
     uint32_t k_accept;
-    uint32_t stage_cap;      // records that fit the shared-memory staging area
-    uint32_t sort_cap;       // power of two >= k: size of the shared-memory sort area
+    uint32_t stage_cap;      // records the general select may stage in shared memory (0 = read them from the buffer)
+    uint32_t sort_cap;       // power of two >= k: records the sort area holds (the area has RF_EDGE_CAP more)
     T* out_vals;             // rows x k
     int64_t* out_idx;        // rows x k
     int use_pdl;
-    const uint32_t* coarse;  // rows x COARSE_BINS survivor histogram written by the filter (null = none)
 };
 
 __device__ __forceinline__ uint64_t shr64(uint64_t x, int s) { return s >= 64 ? 0ull : (x >> s); }
@@ -82,10 +82,11 @@ __device__ __forceinline__ void bitonic_sort_shared(uint64_t* a, uint32_t P) {
 
 // Shared state of one select.
 struct SelectShared {
-    uint32_t hist[RF_BINS];
-    uint64_t edge[RF_EDGE_CAP];      // records of the boundary bin
+    uint32_t hist[RF_BINS];          // bin counts, then running cursors
+    uint32_t start[RF_BINS];         // first position of every bin
+    uint64_t edge[RF_EDGE_CAP];      // records of the boundary bin (general select only)
     uint32_t warp_sums[32];
-    uint32_t digit, before, cnt, fill, n_edge, total;
+    uint32_t digit, before, cnt, fill, n_edge, crowded, dmax;
     unsigned long long or_bits, limit;
 };
 
@@ -207,15 +208,11 @@ __device__ __forceinline__ void write_output(T* out_vals, int64_t* out_idx, uint
 }
 
 // Orders the m records in sortbuf (all threads have passed a barrier since they were written)
-// and writes the first kk of them, then the padding of relaxed mode, as row `row` of the output.
+// and writes the first kk of them as row `row` of the output.
 template <typename T>
 __device__ __forceinline__ void sort_and_write(uint64_t* sortbuf, uint32_t m, uint32_t kk, uint32_t k, uint64_t row,
                                                T* out_vals, int64_t* out_idx) {
     const unsigned tid = threadIdx.x, nthr = blockDim.x;
-    for (uint32_t j = kk + tid; j < k; j += nthr) {       // relaxed mode: padding after a short buffer
-        out_vals[row * (uint64_t)k + j] = Elem<T>::from_bits(Elem<T>::NEG_INF_BITS);
-        out_idx[row * (uint64_t)k + j] = -1;
-    }
     if (m <= nthr) {
         uint32_t P = 32;
         while (P < m) P <<= 1;
@@ -238,13 +235,14 @@ __device__ __forceinline__ void sort_and_write(uint64_t* sortbuf, uint32_t m, ui
 template <typename T>
 __global__ void __launch_bounds__(1024) refine_kernel(const RefineParams<T> p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    uint64_t* sortbuf = reinterpret_cast<uint64_t*>(smem_raw);                 // sort_cap records
-    uint64_t* staged = sortbuf + p.sort_cap;                                   // stage_cap records
+    uint64_t* sortbuf = reinterpret_cast<uint64_t*>(smem_raw);                 // sort_cap + RF_EDGE_CAP records
+    uint64_t* staged = sortbuf + p.sort_cap + RF_EDGE_CAP;                     // stage_cap records
     __shared__ SelectShared sh;
 
     const unsigned tid = threadIdx.x, nthr = blockDim.x, lane = lane_id();
     const uint64_t row = blockIdx.x;
-    if (tid == 0) { sh.or_bits = 0ull; sh.fill = 0; sh.n_edge = 0; }
+    if (tid == 0) { sh.or_bits = 0ull; sh.fill = 0; sh.n_edge = 0; sh.crowded = 0; sh.dmax = 0; }
+    for (uint32_t i = tid; i < RF_BINS; i += nthr) sh.hist[i] = 0;
     __syncthreads();
     pdl_launch_dependents();                 // the exact-selection kernel may be staged behind this one
     if (p.use_pdl) pdl_wait();
@@ -264,109 +262,133 @@ __global__ void __launch_bounds__(1024) refine_kernel(const RefineParams<T> p) {
     const uint32_t n = R;
     const uint32_t kk = n < p.k ? n : p.k;          // real outputs; the rest is padding (relaxed mode)
     const uint64_t* src = p.buf + row * (uint64_t)p.capacity;
+    for (uint32_t j = kk + tid; j < p.k; j += nthr) {       // relaxed mode: padding after a short buffer
+        p.out_vals[row * (uint64_t)p.k + j] = Elem<T>::from_bits(Elem<T>::NEG_INF_BITS);
+        p.out_idx[row * (uint64_t)p.k + j] = -1;
+    }
 
-    uint32_t m;   // records in sortbuf that remain to be ordered
+    // ---- bin the records by the distance of their key above tau (bin 0 = largest keys) ----
+    const uint32_t tau_key = Elem<T>::key(Elem<T>::from_bits(ctl.tau_bits));
+    const uint32_t nbatch = (n + 8 * nthr - 1) / (8 * nthr);   // one batch = 8 records per thread, kept in registers
+    uint64_t r[8];
+    auto load_batch = [&](uint32_t b) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t i = (b * 8 + u) * nthr + tid;
+            r[u] = i < n ? src[i] : ~0ull;
+        }
+    };
+    auto valid = [&](uint32_t b, int u) { return (b * 8 + u) * nthr + tid < n; };
+    auto dist = [&](uint64_t rec) { const uint32_t key = record_key(rec); return key > tau_key ? key - tau_key : 0u; };
+
+    uint32_t dmax = 0;
+    for (uint32_t b = 0; b < nbatch; ++b) {
+        load_batch(b);
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (valid(b, u)) dmax = max(dmax, dist(r[u]));
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) dmax = max(dmax, __shfl_xor_sync(FULL_MASK, dmax, d));
+    if (lane == 0) sh.warp_sums[tid >> 5] = dmax;
+    __syncthreads();
+    if (tid < 32) {
+        uint32_t w = tid < (nthr >> 5) ? sh.warp_sums[tid] : 0;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) w = max(w, __shfl_xor_sync(FULL_MASK, w, d));
+        if (tid == 0) sh.dmax = w;
+    }
+    __syncthreads();
+    const int dbits = 32 - __clz(sh.dmax);                             // dmax < 2^dbits
+    const int shift = dbits > RF_BITS ? dbits - RF_BITS : 0;
+    auto bin_of = [&](uint64_t rec) { return (uint32_t)(RF_BINS - 1) - (dist(rec) >> shift); };
+    PROFK_STAMP(1, 1);
+
+    for (uint32_t b = 0; b < nbatch; ++b) {
+        if (nbatch > 1) load_batch(b);
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (valid(b, u)) atomicAdd(&sh.hist[bin_of(r[u])], 1u);
+    }
+    __syncthreads();
+
+    // ---- scan the bin counts: first position of every bin, and the bin of the kk-th best record ----
+    {
+        const uint32_t per = (RF_BINS + nthr - 1) / nthr;
+        uint32_t sum = 0;
+        for (uint32_t j = 0; j < per; ++j) {
+            const uint32_t bin = tid * per + j;
+            sum += bin < RF_BINS ? sh.hist[bin] : 0;
+        }
+        uint32_t before = block_scan_any(sum, sh.warp_sums) - sum;
+        for (uint32_t j = 0; j < per; ++j) {
+            const uint32_t bin = tid * per + j;
+            if (bin < RF_BINS) {
+                const uint32_t c = sh.hist[bin];
+                if (before < kk && kk <= before + c) { sh.digit = bin; sh.before = before; sh.cnt = c; }
+                if (before < kk && c > RF_EDGE_CAP) sh.crowded = 1;         // a bin that matters is too full to rank
+                sh.start[bin] = before;
+                sh.hist[bin] = before;                                      // becomes the bin's write cursor
+                before += c;
+            }
+        }
+    }
+    __syncthreads();
+    PROFK_STAMP(1, 2);
+
+    if (!sh.crowded) {
+        // ---- group the records of the boundary bin and of all better bins by bin ----
+        const uint32_t edge_bin = sh.digit;
+        const uint32_t n_grouped = sh.before + sh.cnt;                      // < kk + RF_EDGE_CAP
+        for (uint32_t b = 0; b < nbatch; ++b) {
+            if (nbatch > 1) load_batch(b);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                if (valid(b, u)) {
+                    const uint32_t bin = bin_of(r[u]);
+                    if (bin <= edge_bin) sortbuf[atomicAdd(&sh.hist[bin], 1u)] = r[u];
+                }
+            }
+        }
+        __syncthreads();
+        PROFK_STAMP(1, 3);
+        // ---- every grouped record ranks itself inside its bin: that is its place in the output ----
+        for (uint32_t s = tid; s < n_grouped; s += nthr) {
+            const uint64_t mine = sortbuf[s];
+            const uint32_t bin = bin_of(mine);
+            const uint32_t first = sh.start[bin], last = sh.hist[bin];
+            uint32_t pos = first;
+            for (uint32_t j = first; j < last; ++j) pos += sortbuf[j] < mine;
+            if (pos < kk) write_output(p.out_vals, p.out_idx, p.k, row, pos, mine);
+        }
+        PROFK_STAMP(1, 4);
+        return;
+    }
+
+    // ---- crowded bins (many equal values): general select, then sort ----
+    uint32_t m;
     if (n <= p.sort_cap) {
         for (uint32_t i = tid; i < n; i += nthr) sortbuf[i] = src[i];
         m = n;
         __syncthreads();
     } else {
-        bool resolved = false;
-        if (p.coarse != nullptr) {
-            // ---- scan the coarse histogram (bin 0 = largest keys) for the bin of the kk-th best record ----
-            const uint32_t* hist = p.coarse + row * COARSE_BINS;
-            const uint32_t per = (COARSE_BINS + nthr - 1) / nthr;
-            uint32_t sum = 0;
-            for (uint32_t j = 0; j < per; ++j) {
-                const uint32_t bin = tid * per + j;
-                sum += bin < COARSE_BINS ? __ldcg(&hist[bin]) : 0;
-            }
-            uint32_t before = block_scan_any(sum, sh.warp_sums) - sum;
-            for (uint32_t j = 0; j < per; ++j) {
-                const uint32_t bin = tid * per + j;
-                const uint32_t c = bin < COARSE_BINS ? __ldcg(&hist[bin]) : 0;
-                if (before < kk && kk <= before + c) { sh.digit = bin; sh.before = before; sh.cnt = c; }
-                before += c;
-            }
-            __syncthreads();
-            const uint32_t edge_bin = sh.digit, need = kk - sh.before, in_bin = sh.cnt;
-            PROFK_STAMP(1, 1);
-            if (in_bin <= RF_EDGE_CAP) {
-                // ---- one pass over the records: those of better bins are winners, those of the boundary
-                //      bin go to the edge list; both are placed by a block-wide prefix sum ----
-                uint32_t run_w = 0, run_e = 0;
-                for (uint32_t base = 0; base < n; base += 8 * nthr) {
-                    uint64_t r[8];
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const uint32_t i = base + u * nthr + tid;
-                        r[u] = i < n ? src[i] : 0ull;
-                    }
-                    uint32_t wmask = 0, emask = 0;
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const uint32_t i = base + u * nthr + tid;
-                        const uint32_t bin = coarse_bin(record_key(r[u]), ctl.hi_key, ctl.bin_shift);
-                        if (i < n && bin < edge_bin) wmask |= 1u << u;
-                        if (i < n && bin == edge_bin) emask |= 1u << u;
-                    }
-                    const uint32_t cw = __popc(wmask), ce = __popc(emask);
-                    const uint32_t incl = block_scan_any(cw | (ce << 16), sh.warp_sums);   // two 16-bit counters
-                    if (tid == nthr - 1) sh.total = incl;
-                    uint32_t pw = run_w + (incl & 0xFFFFu) - cw, pe = run_e + (incl >> 16) - ce;
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        if (wmask & (1u << u)) { if (pw < p.sort_cap) sortbuf[pw] = r[u]; ++pw; }
-                        if (emask & (1u << u)) { if (pe < RF_EDGE_CAP) sh.edge[pe] = r[u]; ++pe; }
-                    }
-                    __syncthreads();
-                    run_w += sh.total & 0xFFFFu;
-                    run_e += sh.total >> 16;
-                    __syncthreads();
-                }
-                PROFK_STAMP(1, 2);
-                // ---- rank the boundary bin; its `need` best records complete the winners ----
-                for (uint32_t i = tid; i < in_bin; i += nthr) {
-                    const uint64_t mine = sh.edge[i];
-                    uint32_t rank = 0;
-                    for (uint32_t j = 0; j < in_bin; ++j) rank += sh.edge[j] < mine;
-                    if (rank < need && run_w + rank < p.sort_cap) sortbuf[run_w + rank] = mine;
-                }
-                __syncthreads();
-                resolved = true;
-            }
+        const bool use_stage = n <= p.stage_cap;
+        const uint64_t first = src[0];
+        uint64_t diff = 0;
+        for (uint32_t i = tid; i < n; i += nthr) {
+            const uint64_t rec = src[i];
+            diff |= rec ^ first;
+            if (use_stage) staged[i] = rec;
         }
-        if (!resolved) {
-            // ---- general select (no usable histogram, or too many ties in the boundary bin) ----
-            const bool use_stage = n <= p.stage_cap;
-            const uint64_t first = src[0];
-            uint64_t diff = 0;
-            for (uint32_t base = 0; base < n; base += 8 * nthr) {
-                uint64_t r[8];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const uint32_t i = base + u * nthr + tid;
-                    r[u] = i < n ? src[i] : first;
-                }
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const uint32_t i = base + u * nthr + tid;
-                    diff |= r[u] ^ first;
-                    if (use_stage && i < n) staged[i] = r[u];
-                }
-            }
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) diff |= __shfl_xor_sync(FULL_MASK, diff, d);
-            if (lane == 0 && diff) atomicOr(&sh.or_bits, (unsigned long long)diff);
-            __syncthreads();
-            MemRecords mem{use_stage ? staged : src, n};
-            select_smallest(mem, first, kk, sortbuf, p.sort_cap, sh);
-        }
+        for (int d = 16; d > 0; d >>= 1) diff |= __shfl_xor_sync(FULL_MASK, diff, d);
+        if (lane == 0 && diff) atomicOr(&sh.or_bits, (unsigned long long)diff);
+        __syncthreads();
+        MemRecords mem{use_stage ? staged : src, n};
+        select_smallest(mem, first, kk, sortbuf, p.sort_cap, sh);
         m = kk;
     }
-    PROFK_STAMP(1, 3);
     sort_and_write<T>(sortbuf, m, kk, p.k, row, p.out_vals, p.out_idx);
-    PROFK_STAMP(1, 4);
 }
 
 }  // namespace profk

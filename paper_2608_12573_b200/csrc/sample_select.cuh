@@ -37,8 +37,7 @@ struct RowCtl {
     uint32_t status;     // PROFK_ROW_* (| 0x80000000 on a timeout)
     uint32_t n_final;    // records the refine step has to order
     uint32_t capacity;
-    uint32_t hi_key;     // coarse histogram: largest sampled key ...
-    uint32_t bin_shift;  // ... and the shift that maps [tau, hi_key] onto COARSE_BINS bins
+    uint32_t pad[2];
 };
 static_assert(sizeof(RowCtl) == 32, "RowCtl is 32 bytes");
 
@@ -67,28 +66,15 @@ template <typename T> struct SelectParams {
     RowCtl* ctl;           // may be null (stand-alone use)
     WsHeader* header;      // may be null
     uint32_t capacity;
-    uint32_t* coarse;      // may be null; rows x COARSE_BINS survivor histogram, zeroed here
     uint32_t* sample_idx;  // may be null; rows x S
 };
 
-// Writes tau and the parameters of the coarse survivor histogram for one row.
+// Writes tau for one row.
 template <typename T>
-__device__ __forceinline__ void publish_threshold(const SelectParams<T>& p, uint64_t row, uint32_t tau_key, uint32_t max_key) {
+__device__ __forceinline__ void publish_threshold(const SelectParams<T>& p, uint64_t row, uint32_t tau_key) {
     const T tau = Elem<T>::from_key(tau_key);
     p.tau[row] = tau;
-    if (p.ctl) {
-        RowCtl* c = p.ctl + row;
-        c->tau_bits = Elem<T>::bits(tau);
-        // The largest sampled key sits near rank N/S of the row, so the histogram reaches three
-        // sample spans above it; whatever lies higher still shares bin 0.
-        const uint64_t span = (uint64_t)max_key - tau_key;            // max_key >= tau_key
-        const uint64_t top = (uint64_t)max_key + 3 * span;
-        const uint32_t hi_key = top > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)top;
-        c->hi_key = hi_key;
-        const uint32_t range = hi_key - tau_key;
-        const int bits = 32 - __clz(range);                           // range < 2^bits
-        c->bin_shift = bits > COARSE_BITS ? (uint32_t)(bits - COARSE_BITS) : 0u;
-    }
+    if (p.ctl) p.ctl[row].tau_bits = Elem<T>::bits(tau);
 }
 
 // floor(j * N / S) = j * (N / S) + floor(j * (N % S) / S).  The second quotient is below S
@@ -199,10 +185,6 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
             }
         }
     }
-    if (p.coarse) {   // the CTAs of the cluster share the zeroing of the row's histogram
-        uint32_t* h = p.coarse + row * COARSE_BINS;
-        for (uint32_t b = crank * SEL_THREADS + tid; b < COARSE_BINS; b += csize * SEL_THREADS) h[b] = 0;
-    }
     if (crank == 0 && tid == 0) {
         if (p.ctl) {
             RowCtl* c = p.ctl + row;
@@ -277,13 +259,8 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
                     rank += __shfl_xor_sync(FULL_MASK, rank, 1);
                     rank += __shfl_xor_sync(FULL_MASK, rank, 2);
                     rank += __shfl_xor_sync(FULL_MASK, rank, 4);
-                    if (part == 0 && c < ncand && rank == 0) s_lower = mine;      // the largest sampled key
-                    if (part == 0 && c < ncand && rank == p.t - 1) s_digit = mine; // the t-th largest: tau
+                    if (part == 0 && c < ncand && rank == p.t - 1) publish_threshold(p, row, mine);   // the t-th largest: tau
                 }
-            }
-            if (crank == 0) {
-                __syncthreads();
-                if (tid == 0) publish_threshold(p, row, s_digit, s_lower);
             }
             done = true;
             PROFK_STAMP(0, 5);
@@ -341,7 +318,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
             __syncthreads();   // s_digit / s_before are rewritten in the next pass
         }
         const uint32_t tau_key = prefix << (32 - consumed);
-        if (crank == 0 && tid == 0) publish_threshold(p, row, tau_key, 0xFFFFFFFFu);   // no cheap maximum on this path
+        if (crank == 0 && tid == 0) publish_threshold(p, row, tau_key);
         cluster.sync();   // no CTA leaves while a peer may still read its histogram
     }
     PROFK_STAMP(0, 6);
