@@ -33,7 +33,9 @@ template <typename T> struct FallbackParams {
     RowCtl* ctl;
     WsHeader* header;
     uint32_t* ghist;          // FB_PASSES x FB_BINS global histogram
-    uint64_t* buf;            // rows x capacity records
+    uint64_t* buf;            // row r's records start at buf + r * buf_stride
+    uint64_t buf_stride;
+    int sort_rows;            // 1 = order and write the repaired rows here; 0 = a later kernel does (large k)
     uint64_t tiles_per_row;
     int use_pdl;              // 1 = launched as a programmatic dependent of the refine kernel
     T* out_vals;              // rows x k
@@ -185,7 +187,7 @@ __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackPara
                 }
 
                 // ---- collect the k records <= limit into the row's buffer ----
-                uint64_t* dst = p.buf + row * (uint64_t)p.capacity;
+                uint64_t* dst = p.buf + row * p.buf_stride;
                 uint32_t* counter = &p.ctl[row].collect;
                 const unsigned lt_mask = (1u << lane) - 1u;
                 for_each_record(p, row, [&](uint64_t rec, bool valid) {
@@ -203,7 +205,7 @@ __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackPara
                 // ---- order the k records and write the row's output (first CTA; the others move on
                 //      and meet it again at the next row's barrier) ----
                 if (!grid_barrier(p.header, gen)) return;
-                if (blockIdx.x == 0) {
+                if (p.sort_rows && blockIdx.x == 0) {
                     extern __shared__ __align__(16) unsigned char fb_smem[];
                     uint64_t* sortbuf = reinterpret_cast<uint64_t*>(fb_smem);
                     for (uint32_t i = tid; i < p.k; i += FB_THREADS) sortbuf[i] = __ldcg(&dst[i]);

@@ -31,7 +31,8 @@ template <typename T> struct FilterParams {
     uint64_t rows;
     const T* tau;            // rows thresholds
     uint32_t capacity;       // records per row buffer
-    uint64_t* buf;           // rows x capacity records
+    uint64_t* buf;           // row r's records start at buf + r * buf_stride
+    uint64_t buf_stride;
     uint32_t* counts;        // per-row survivor counter (stride in 32-bit words)
     uint32_t count_stride;
     uint64_t tiles_per_row;
@@ -114,7 +115,7 @@ __global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOC
                 if (lane == 0) base = atomicAdd(p.counts + (uint64_t)row * p.count_stride, total);
                 base = __shfl_sync(FULL_MASK, base, 0);
                 unsigned pos = base + incl - cnt;
-                uint64_t* dst = p.buf + (uint64_t)row * p.capacity;
+                uint64_t* dst = p.buf + (uint64_t)row * p.buf_stride;
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u) {
                     if (mine[u]) {

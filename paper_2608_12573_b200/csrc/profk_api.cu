@@ -15,6 +15,7 @@
 #include "filter.cuh"
 #include "profk.h"
 #include "refine.cuh"
+#include "refine_large.cuh"
 #include "sample_select.cuh"
 
 using namespace profk;
@@ -36,6 +37,7 @@ struct DeviceInfo {
     int filter_blocks_per_sm[2] = {0, 0};     // by dtype
     int fallback_blocks_per_sm[2] = {0, 0};
     int max_cluster[2] = {8, 8};              // 16 when the device can co-schedule 16 CTAs of the threshold kernel
+    int large_cluster[2] = {8, 8};            // same for the cluster sort (128 KB of shared memory per CTA)
     bool ready = false;
 };
 
@@ -52,14 +54,23 @@ struct WsLayout {
     size_t off_header, off_ghist, off_ctl, off_tau, off_buf, total;
 };
 
-WsLayout ws_layout(int64_t rows, int64_t capacity) {
+// Records reserved per row: the capacity itself, or -- when k is too large for the single-CTA
+// refine -- the power of two the cluster sort pads the row to.
+uint64_t row_stride_for(int64_t capacity, int64_t k) {
+    if (k <= (int64_t)SORT_CAP_MAX) return (uint64_t)capacity;
+    uint64_t p = BT_TILE;
+    while (p < (uint64_t)capacity) p <<= 1;
+    return p;
+}
+
+WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k) {
     WsLayout l;
     l.off_header = 0;
     l.off_ghist = sizeof(WsHeader);
     l.off_ctl = align_up(l.off_ghist + (size_t)FB_PASSES * FB_BINS * sizeof(uint32_t), 256);
     l.off_tau = align_up(l.off_ctl + (size_t)rows * sizeof(RowCtl), 256);
     l.off_buf = align_up(l.off_tau + (size_t)rows * 4, 256);
-    l.total = align_up(l.off_buf + (size_t)rows * (size_t)capacity * sizeof(uint64_t), 256);
+    l.total = align_up(l.off_buf + (size_t)rows * (size_t)row_stride_for(capacity, k) * sizeof(uint64_t), 256);
     return l;
 }
 
@@ -100,6 +111,19 @@ template <typename T> int ensure_device_info(int dev, DeviceInfo* out) {
             int nclusters = 0;
             if (cudaOccupancyMaxActiveClusters(&nclusters, sample_select_kernel<T>, &cfg) == cudaSuccess && nclusters >= 1)
                 di.max_cluster[d] = 16;
+        }
+        (void)cudaGetLastError();
+        CUDA_TRY(cudaFuncSetAttribute(refine_large_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(BT_TILE * 8)));
+        if (cudaFuncSetAttribute(refine_large_kernel<T>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(16); cfg.blockDim = dim3(BT_THREADS); cfg.dynamicSmemBytes = BT_TILE * 8;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 16; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr; cfg.numAttrs = 1;
+            int nclusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&nclusters, refine_large_kernel<T>, &cfg) == cudaSuccess && nclusters >= 1)
+                di.large_cluster[d] = 16;
         }
         (void)cudaGetLastError();
     }
@@ -151,10 +175,11 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
 
 template <typename T>
 int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, const T* tau, int64_t capacity, uint64_t* buf,
+                  uint64_t buf_stride,
                   uint32_t* counts, uint32_t count_stride, bool pdl, cudaStream_t st) {
     FilterParams<T> fp;
     fp.in = in; fp.N = (uint64_t)N; fp.rows = (uint64_t)rows; fp.tau = tau; fp.capacity = (uint32_t)capacity;
-    fp.buf = buf; fp.counts = counts; fp.count_stride = count_stride;
+    fp.buf = buf; fp.buf_stride = buf_stride; fp.counts = counts; fp.count_stride = count_stride;
     fp.tiles_per_row = tiles_per_row<T>((uint64_t)N, FILTER_THREADS * FILTER_UNROLL);
     fp.total_tiles = fp.tiles_per_row * (uint64_t)rows;
     if (fp.total_tiles >= (1ull << 32)) return PROFK_EINVAL;      // rows * N beyond 2^45 elements
@@ -175,6 +200,31 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
 }
 
 template <typename T>
+int launch_refine_large(const DeviceInfo& di, RowCtl* ctl, WsHeader* header, uint64_t* buf, uint64_t row_stride, int64_t rows,
+                        int64_t capacity, int64_t k, int64_t k_accept, int phase, T* out_vals, int64_t* out_idx, cudaStream_t st) {
+    LargeParams<T> lp;
+    lp.ctl = ctl; lp.header = header; lp.buf = buf; lp.row_stride = row_stride; lp.capacity = (uint32_t)capacity;
+    lp.k = (uint32_t)k; lp.k_accept = (uint32_t)k_accept; lp.phase = phase; lp.out_vals = out_vals; lp.out_idx = out_idx;
+    lp.use_pdl = 1;
+    int csize = di.large_cluster[dtype_index<T>()];
+    while (csize > 1 && (uint64_t)csize * BT_TILE > row_stride) csize /= 2;     // no more CTAs than tiles
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(rows * csize));
+    cfg.blockDim = dim3(BT_THREADS);
+    cfg.dynamicSmemBytes = (size_t)BT_TILE * 8;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 2;
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, refine_large_kernel<T>, lp));
+    ++g_launches;
+    return PROFK_OK;
+}
+
+template <typename T>
 int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_plan_t* plan, uint64_t seed, void* stream,
                  T* out_vals, int64_t* out_idx) {
     g_launches = 0;
@@ -188,7 +238,6 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         if (plan->m < 1 || plan->m > std::min<int64_t>(N, M_MAX) || plan->r < 1 || plan->r > plan->m) return PROFK_EINVAL;
         if (plan->k_accept < 1 || plan->k_accept > k) return PROFK_EINVAL;
     }
-    if (k > SORT_CAP_MAX) return PROFK_EINVAL;   // larger selections need the multi-CTA sort
 
     int dev = 0;
     CUDA_TRY(cudaGetDevice(&dev));
@@ -201,8 +250,10 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         std::lock_guard<std::mutex> lock(g_mutex);
         ws = g_workspace[dev];
     }
-    const WsLayout lay = ws_layout(rows, capacity);
+    const WsLayout lay = ws_layout(rows, capacity, k);
     if (!ws.ptr || ws.bytes < lay.total) return PROFK_EWORKSPACE;
+    const uint64_t row_stride = row_stride_for(capacity, k);
+    const bool large = k > (int64_t)SORT_CAP_MAX;
     unsigned char* base = static_cast<unsigned char*>(ws.ptr);
     WsHeader* header = reinterpret_cast<WsHeader*>(base + lay.off_header);
     uint32_t* ghist = reinterpret_cast<uint32_t*>(base + lay.off_ghist);
@@ -212,17 +263,21 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
     uint32_t sort_cap = 32;
-    while (sort_cap < (uint32_t)k) sort_cap <<= 1;
+    while (sort_cap < (uint32_t)k && sort_cap < SORT_CAP_MAX) sort_cap <<= 1;
 
     if (plan->mode == 0) {
         rc = launch_sample_select<T>(di, in, rows, N, plan->m, plan->r, seed, tau, ctl, header, (uint32_t)capacity, nullptr, st);
         if (rc != PROFK_OK) return rc;
-        rc = launch_filter<T>(di, in, rows, N, tau, capacity, buf, &ctl[0].count, sizeof(RowCtl) / 4, true, st);
+        rc = launch_filter<T>(di, in, rows, N, tau, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, st);
         if (rc != PROFK_OK) return rc;
 
+        if (large) {
+            rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, rows, capacity, k, plan->k_accept, 0, out_vals, out_idx, st);
+            if (rc != PROFK_OK) return rc;
+        } else {
         // refine: count check, then order the buffer of every row that passed it
         RefineParams<T> rp;
-        rp.ctl = ctl; rp.header = header; rp.buf = buf; rp.capacity = (uint32_t)capacity; rp.k = (uint32_t)k;
+        rp.ctl = ctl; rp.header = header; rp.buf = buf; rp.buf_stride = row_stride; rp.capacity = (uint32_t)capacity; rp.k = (uint32_t)k;
         rp.k_accept = (uint32_t)plan->k_accept;
         rp.sort_cap = sort_cap;
         rp.stage_cap = 0;            // the general select (crowded bins only) reads the buffer in place
@@ -240,6 +295,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         cfg.attrs = attr; cfg.numAttrs = 1;
         CUDA_TRY(cudaLaunchKernelEx(&cfg, refine_kernel<T>, rp));
         ++g_launches;
+        }
     } else {
         init_ctl_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(ctl, (uint64_t)rows, header, (uint32_t)capacity, (uint32_t)k);
         CUDA_TRY(cudaGetLastError());
@@ -250,13 +306,14 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         FallbackParams<T> fb;
         fb.in = in; fb.N = (uint64_t)N; fb.rows = (uint64_t)rows; fb.k = (uint32_t)k;
         fb.capacity = (uint32_t)capacity; fb.ctl = ctl; fb.header = header; fb.ghist = ghist; fb.buf = buf;
+        fb.buf_stride = row_stride; fb.sort_rows = large ? 0 : 1;
         fb.tiles_per_row = tiles_per_row<T>((uint64_t)N, FB_THREADS * FB_UNROLL);
         fb.use_pdl = 0;
         fb.out_vals = out_vals; fb.out_idx = out_idx;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)di.sm_count);       // one CTA per SM: cheap to launch when no row failed
         cfg.blockDim = dim3(FB_THREADS);
-        cfg.dynamicSmemBytes = (size_t)sort_cap * 8;
+        cfg.dynamicSmemBytes = large ? 0 : (size_t)sort_cap * 8;
         cfg.stream = st;
         cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeCooperative;
@@ -285,6 +342,10 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
             CUDA_TRY(cudaLaunchKernelEx(&cfg, fallback_kernel<T>, fb));
         }
         ++g_launches;
+    }
+    if (large) {   // the rows the exact selection repaired still have to be ordered and written
+        rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, rows, capacity, k, k, 1, out_vals, out_idx, st);
+        if (rc != PROFK_OK) return rc;
     }
     return PROFK_OK;
 }
@@ -321,7 +382,7 @@ int filter_only(const T* in, int64_t rows, int64_t N, const T* tau, int64_t capa
     DeviceInfo di;
     const int rc = ensure_device_info<T>(dev, &di);
     if (rc != PROFK_OK) return rc;
-    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, counts, 1, false, static_cast<cudaStream_t>(stream));
+    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, (uint64_t)capacity, counts, 1, false, static_cast<cudaStream_t>(stream));
 }
 
 template <typename T>
@@ -346,7 +407,7 @@ extern "C" {
 int profk_workspace_bytes(int64_t rows, int64_t capacity, int64_t k, size_t* bytes) {
     if (!bytes || rows < 1 || capacity < 1 || k < 1 || capacity < k || capacity > N_MAX || rows * capacity >= (1LL << 40))
         return PROFK_EINVAL;
-    *bytes = ws_layout(rows, capacity).total;
+    *bytes = ws_layout(rows, capacity, k).total;
     return PROFK_OK;
 }
 
@@ -413,7 +474,7 @@ int profk_read_stats(void* stream, int64_t rows, profk_row_stats_t* out) {
         std::lock_guard<std::mutex> lock(g_mutex);
         ws = g_workspace[dev];
     }
-    const WsLayout lay = ws_layout(rows, 1);
+    const WsLayout lay = ws_layout(rows, 1, 1);
     if (!ws.ptr || ws.bytes < lay.off_ctl + (size_t)rows * sizeof(RowCtl)) return PROFK_EWORKSPACE;
     std::vector<RowCtl> host((size_t)rows);
     WsHeader hdr;

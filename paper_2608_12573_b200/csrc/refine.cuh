@@ -26,7 +26,8 @@ enum : uint32_t { ROW_OK = 0, ROW_RECALL = 1, ROW_OVERFLOW = 2, ROW_DIRECT = 3 }
 template <typename T> struct RefineParams {
     RowCtl* ctl;
     WsHeader* header;
-    const uint64_t* buf;     // rows x capacity records
+    const uint64_t* buf;     // row r's records start at buf + r * buf_stride
+    uint64_t buf_stride;
     uint32_t capacity;
     uint32_t k;
     uint32_t k_accept;
@@ -261,7 +262,7 @@ __global__ void __launch_bounds__(1024) refine_kernel(const RefineParams<T> p) {
 
     const uint32_t n = R;
     const uint32_t kk = n < p.k ? n : p.k;          // real outputs; the rest is padding (relaxed mode)
-    const uint64_t* src = p.buf + row * (uint64_t)p.capacity;
+    const uint64_t* src = p.buf + row * p.buf_stride;
     for (uint32_t j = kk + tid; j < p.k; j += nthr) {       // relaxed mode: padding after a short buffer
         p.out_vals[row * (uint64_t)p.k + j] = Elem<T>::from_bits(Elem<T>::NEG_INF_BITS);
         p.out_idx[row * (uint64_t)p.k + j] = -1;

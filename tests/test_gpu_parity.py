@@ -166,12 +166,42 @@ def test_nan_inf_and_signed_zero_follow_the_total_order():
     x = workloads.normal(1, 100_000, seed=15)[0]
     x[5] = float("nan"); x[77] = float("inf"); x[78] = float("inf"); x[99] = -float("inf")
     x[1000:1010] = 0.0; x[2000:2010] = -0.0
-    for k in (1, 3, 5000, 8192):
+    for k in (1, 3, 5000, 8192, 50_000, 100_000):
         v, i = gpu_topk(x, k)
         assert_exact(x, k, v, i)
     xb = x.to(torch.bfloat16)
     v, i = gpu_topk(xb, 1000)
     assert_exact(xb, 1000, v, i)
+
+
+# ----------------------------------------------------------------------------- large selections
+def test_large_k_uses_the_cluster_sort():
+    x = workloads.normal(1, 1 << 22, seed=21)[0]
+    for k in (8193, 20_000, 100_000):
+        v, i = gpu_topk(x, k, eps=1e-3, seed=2)
+        assert_exact(x, k, v, i)
+    xb = workloads.relu_gaussian(1 << 22, seed=3)                      # bf16, thousands of copies of each value
+    for k in (10_000, 65_536):
+        v, i = gpu_topk(xb, k, eps=1e-3, seed=5)
+        assert_exact(xb, k, v, i)
+
+
+def test_large_k_batched_forced_failures_and_direct_mode():
+    x = workloads.normal(3, 300_000, seed=22)
+    k = 10_000
+    v, i = gpu_topk(x, k, eps=1e-3, seed=1)
+    assert_exact(x, k, v, i)
+    v, i, st = _forced(x, k, profk.Plan(m=8192, r=400, capacity=k, k_accept=k, mode=0))      # every row overflows
+    assert_exact(x, k, v, i)
+    assert all(s[3] == profk.ROW_OVERFLOW for s in st)
+    v, i, st = _forced(x, k, profk.Plan(m=8192, r=100, capacity=60_000, k_accept=k, mode=0))  # too few survivors
+    assert_exact(x, k, v, i)
+    assert all(s[3] == profk.ROW_RECALL for s in st)
+    v, i, st = _forced(x, k, profk.Plan(m=0, r=0, capacity=k, k_accept=k, mode=1))
+    assert_exact(x, k, v, i)
+    y = workloads.normal(1, 70_000, seed=23)[0]
+    v, i = gpu_topk(y, 70_000)                                          # k = N
+    assert_exact(y, 70_000, v, i)
 
 
 # ----------------------------------------------------------------------------- stages on their own
