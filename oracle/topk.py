@@ -80,8 +80,22 @@ def topk_brute(x: np.ndarray, k: int) -> tuple[np.ndarray, np.ndarray]:
     return x[idx].copy(), idx
 
 
-def verify_topk(x: np.ndarray, k: int, vals: np.ndarray, idx: np.ndarray) -> list[str]:
+def _first_positions(keys: np.ndarray, value, count: int, chunk: int = 1 << 24) -> np.ndarray:
+    """The `count` lowest positions where keys == value (scanned chunk by chunk to bound memory)."""
+    found: list[np.ndarray] = []
+    have = 0
+    for start in range(0, keys.shape[0], chunk):
+        if have >= count:
+            break
+        hit = np.flatnonzero(keys[start:start + chunk] == value) + start
+        found.append(hit[:count - have])
+        have += found[-1].size
+    return np.concatenate(found) if found else np.empty(0, dtype=np.int64)
+
+
+def verify_topk(x: np.ndarray, k: int, vals: np.ndarray, idx: np.ndarray, keys: np.ndarray | None = None) -> list[str]:
     """Check a claimed top-k of one row against the definition in O(N).
+    (`keys` = order_key(x), if the caller already has it.)
 
     The claimed answer equals the unique correct one iff all of these hold:
       1. idx are k distinct in-range indices and vals[j] is bitwise x[idx[j]];
@@ -104,7 +118,8 @@ def verify_topk(x: np.ndarray, k: int, vals: np.ndarray, idx: np.ndarray) -> lis
     bits = np.uint32 if x.dtype == np.float32 else np.uint16
     if not np.array_equal(x[idx].view(bits), np.ascontiguousarray(vals).view(bits)):
         bad.append("value != x[index]")
-    keys = order_key(x)
+    if keys is None:
+        keys = order_key(x)
     lk = keys[idx].astype(np.int64)
     dk = np.diff(lk)
     di = np.diff(idx.astype(np.int64))
@@ -116,7 +131,7 @@ def verify_topk(x: np.ndarray, k: int, vals: np.ndarray, idx: np.ndarray) -> lis
     if above_all != above_listed:
         bad.append("missing a larger element")
     n_tie = k - above_listed
-    ties_expected = np.flatnonzero(keys == kth)[:n_tie]
+    ties_expected = _first_positions(keys, kth, n_tie)
     ties_listed = np.sort(idx[lk == int(kth)])
     if not np.array_equal(ties_expected, ties_listed):
         bad.append("ties are not the lowest indices")

@@ -1,0 +1,105 @@
+"""The five benchmark configurations at full size, in the launch configuration the benchmark times.
+
+Small enough for a full sort: compared element by element with the oracle's sort.  Too large
+for that (2^29, 2^30): every output row is checked with the oracle's O(N) checker, which accepts
+exactly the unique correct answer (see tests/test_oracle_topk.py for its pins).
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_12573_b200 as profk
+from oracle import plan as o_plan
+from oracle import topk as o_topk
+from paper_2608_12573_b200 import _build, workloads
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    _build.build()
+    profk.lib()
+    torch.cuda.set_device(0)
+
+
+def bits(a):
+    return a.view(np.uint32) if a.dtype == np.float32 else a.view(np.uint16)
+
+
+def run(xd, k, **kw):
+    v, i = profk.topk(xd, k, **kw)
+    torch.cuda.synchronize()
+    return workloads.as_numpy(v), i.cpu().numpy()
+
+
+def test_config2_single_row_2p26():
+    x = workloads.normal(1, 1 << 26, seed=1)[0]
+    xn = workloads.as_numpy(x)
+    ov, oi = o_topk.topk_row(xn, 4096)                      # one full sort serves every k (prefix property)
+    xd = x.cuda()
+    fallbacks = 0
+    for k in (16, 256, 4096):
+        for eps in (1e-2, 1e-4):
+            for seed in (0, 1, 2):
+                v, i = run(xd, k, eps=eps, seed=seed)
+                assert np.array_equal(i, oi[:k]) and np.array_equal(bits(v), bits(ov[:k])), (k, eps, seed)
+                st = profk.read_stats(1)[0]
+                assert st[2] == o_plan.plan_guarded(1 << 26, k, eps).capacity
+                fallbacks += st[3] != profk.ROW_OK
+    assert fallbacks <= 2
+    # relaxed recall 0.95: a prefix of the exact answer, at least k_accept long, then padding
+    for k in (16, 256, 4096):
+        pl = o_plan.plan_guarded(1 << 26, k, 1e-2, recall=0.95)
+        v, i = run(xd, k, eps=1e-2, recall=0.95, seed=3)
+        _, R, _, status = profk.read_stats(1)[0]
+        n_real = min(k, R) if status == profk.ROW_OK else k
+        assert n_real >= pl.k_accept
+        assert np.array_equal(i[:n_real], oi[:n_real]) and np.array_equal(bits(v[:n_real]), bits(ov[:n_real]))
+        assert np.all(i[n_real:] == -1) and np.all(np.isneginf(v[n_real:]))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_config3_batched_512_rows(dtype):
+    x = workloads.normal(512, 1 << 20, seed=2, dtype=dtype)
+    xn = workloads.as_numpy(x)
+    v, i = run(x.cuda(), 32, eps=1e-3, seed=0)
+    for r in range(512):                                     # every row through the checker
+        assert o_topk.verify_topk(xn[r], 32, v[r], i[r]) == [], r
+    for r in (0, 1, 255, 511):                               # a few rows through the full sort as well
+        ov, oi = o_topk.topk_row(xn[r], 32)
+        assert np.array_equal(i[r], oi) and np.array_equal(bits(v[r]), bits(ov))
+    st = profk.read_stats(512)
+    assert sum(s[3] != profk.ROW_OK for s in st) <= 8        # eps = 1e-3 per row: a handful at most
+
+
+def test_config4_flattened_batchtopk_2p29_bf16():
+    n, k = 1 << 29, 32 * 4096
+    x = workloads.relu_gaussian(n, seed=3)                   # 4096 tokens x 131072 latents, flattened
+    xn = workloads.as_numpy(x)
+    keys = o_topk.order_key(xn)
+    xd = x.cuda()
+    del x
+    for seed in (0, 1):
+        v, i = run(xd, k, eps=1e-3, seed=seed)
+        assert o_topk.verify_topk(xn, k, v, i, keys=keys) == []
+    st = profk.read_stats(1)[0]
+    assert st[2] == o_plan.plan_guarded(n, k, 1e-3).capacity
+
+
+@pytest.mark.parametrize("name", ["cauchy", "pareto", "sorted", "few_values", "spikes"])
+def test_config5_adversarial_2p30(name):
+    n = 1 << 30
+    recipe, seed = workloads.ADVERSARIAL[name]
+    xd = recipe(n, seed, device="cuda")                      # drawn on the GPU (seeded): minutes faster than the host
+    xn = xd.cpu().numpy()
+    keys = o_topk.order_key(xn)
+    for k in (1, 64, 1024, 65536):
+        v, i = run(xd, k, eps=1e-3, seed=k)
+        assert o_topk.verify_topk(xn, k, v, i, keys=keys) == [], (name, k)
+        st = profk.read_stats(1)[0]
+        if name in ("few_values", "spikes") and not (name == "spikes" and k <= 64):
+            assert st[3] == profk.ROW_OVERFLOW               # ties flood the buffer: the exact path answers
+    del xd
+    torch.cuda.empty_cache()
