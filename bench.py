@@ -34,11 +34,20 @@ CONFIGS = {
     "cfg2_relaxed": (1, 1 << 26, "f32", "normal", 1, 4096, 1e-2, 0.95),
     "cfg3_f32": (512, 1 << 20, "f32", "normal", 2, 32, 1e-3, 1.0),
     "cfg3_bf16": (512, 1 << 20, "bf16", "normal", 2, 32, 1e-3, 1.0),
+    "cfg4": (1, 1 << 29, "bf16", "relu_gaussian", 3, 32 * 4096, 1e-3, 1.0),
+    "cfg5_cauchy_k64": (1, 1 << 30, "f32", "cauchy", 4, 64, 1e-3, 1.0),
+    "cfg5_cauchy_k65536": (1, 1 << 30, "f32", "cauchy", 4, 65536, 1e-3, 1.0),
+    "cfg5_pareto_k1": (1, 1 << 30, "f32", "pareto", 5, 1, 1e-3, 1.0),
+    "cfg5_pareto_k1024": (1, 1 << 30, "f32", "pareto", 5, 1024, 1e-3, 1.0),
+    "cfg5_sorted_k1024": (1, 1 << 30, "f32", "sorted", 6, 1024, 1e-3, 1.0),
+    "cfg5_few_values_k64": (1, 1 << 30, "f32", "few_values", 7, 64, 1e-3, 1.0),
+    "cfg5_spikes_k64": (1, 1 << 30, "f32", "spikes", 8, 64, 1e-3, 1.0),
+    "cfg5_spikes_k1024": (1, 1 << 30, "f32", "spikes", 8, 1024, 1e-3, 1.0),
 }
 
 # DRAM bytes (read + write) of one filter launch at cfg2, from the ncu capture summarised in
-# profiles/filter_kernel_f32_2p26.md; None until a capture exists.
-FILTER_TRAFFIC_BYTES = {"cfg2": None}
+# profiles/filter_kernel_f32_2p26.md (dram__bytes_read.sum + dram__bytes_write.sum).
+FILTER_TRAFFIC_BYTES = {"cfg2": 272.34e6}
 
 L2_BYTES = 126 * 1024 * 1024
 
@@ -51,16 +60,23 @@ def measured_peak_gbs():
     return 6650.0, "fallback"
 
 
-def make_input(cfg, seed_offset=0):
+def make_input(cfg, seed_offset=0, device="cpu"):
+    """One batch of the workload (rows x N).  Inputs of 2^29 elements and more are drawn on the GPU."""
     import torch
 
     from paper_2608_12573_b200 import workloads
 
     rows, n, dt, recipe, seed, *_ = cfg
     dtype = torch.float32 if dt == "f32" else torch.bfloat16
+    seed = seed + seed_offset
     if recipe == "uniform":
-        return workloads.uniform(n, seed + seed_offset).view(1, n)
-    return workloads.normal(rows, n, seed + seed_offset, dtype=dtype)
+        return workloads.uniform(n, seed, device).view(1, n)
+    if recipe == "normal":
+        return workloads.normal(rows, n, seed, dtype=dtype, device=device)
+    if recipe == "relu_gaussian":
+        return workloads.relu_gaussian(n, seed, dtype=dtype, device=device).view(1, n)
+    fn, _ = workloads.ADVERSARIAL[recipe]
+    return fn(n, seed, device=device).view(1, n)
 
 
 class ClockSampler:
@@ -117,7 +133,7 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def time_oracle(cfg, sample_elems: int, steps: int, warmup: int):
+def time_oracle(cfg, sample_elems: int, steps: int, warmup: int, x=None):
     """The CPU oracle as it stands (full stable sort per row), on a bounded sample of the workload."""
     import numpy as np
 
@@ -125,7 +141,8 @@ def time_oracle(cfg, sample_elems: int, steps: int, warmup: int):
     from paper_2608_12573_b200 import workloads
 
     rows, n, dt, recipe, seed, k, eps, recall = cfg
-    x = make_input(cfg)
+    if x is None:
+        x = make_input(cfg) if rows * n < (1 << 29) else make_input((rows, sample_elems) + tuple(cfg[2:]))
     xn = workloads.as_numpy(x)
     per_row = min(n, sample_elems)
     n_rows = max(1, min(rows, sample_elems // per_row))
@@ -210,8 +227,13 @@ def main():
 
     # Inputs: enough distinct copies that no step finds its input in L2 (126 MB).
     copies = max(2, min(8, -(-3 * L2_BYTES // in_bytes)))
-    host_inputs = [make_input(cfg, seed_offset=1000 * c + 7919 * rank).pin_memory() for c in range(copies)]
-    dev_inputs = [h.to(dev) for h in host_inputs]
+    big = rows * n >= (1 << 29)
+    if big:        # drawn on the device (seeded); one pinned host copy serves the end-to-end leg
+        dev_inputs = [make_input(cfg, seed_offset=1000 * c + 7919 * rank, device=str(dev)) for c in range(copies)]
+        host_inputs = [dev_inputs[0].cpu().pin_memory()]
+    else:
+        host_inputs = [make_input(cfg, seed_offset=1000 * c + 7919 * rank).pin_memory() for c in range(copies)]
+        dev_inputs = [h.to(dev) for h in host_inputs]
     pl = profk.plan(n, k, eps, recall)
     profk.ensure_workspace(rows, pl.capacity, k, dev)
     out_vals = torch.empty((rows, k), dtype=dev_inputs[0].dtype, device=dev)
@@ -256,7 +278,7 @@ def main():
     value = world * rows * n / (ms_per_step * 1e-3)
 
     # fallback rate observed over a separate run of seeds (statistics read-back synchronises, so not timed)
-    n_seeds = 200 if rows == 1 else max(1, 200 // rows)
+    n_seeds = (40 if big else 200) if rows == 1 else max(1, 200 // rows)
     for s in range(n_seeds):
         profk.topk(dev_inputs[s % copies], k, eps=eps, recall=recall, seed=10_000 + s, out=(out_vals, out_idx))
         fallbacks += sum(1 for st in profk.read_stats(rows) if (st[3] & 0xFF) in (profk.ROW_RECALL, profk.ROW_OVERFLOW))
@@ -266,7 +288,7 @@ def main():
     stage = torch.empty_like(dev_inputs[0])
 
     def e2e_step(i):
-        stage.copy_(host_inputs[i % copies], non_blocking=True)
+        stage.copy_(host_inputs[i % len(host_inputs)], non_blocking=True)
         profk.topk(stage, k, eps=eps, recall=recall, seed=i, out=(out_vals, out_idx))
         host_vals.copy_(out_vals, non_blocking=True)
         host_idx.copy_(out_idx, non_blocking=True)
@@ -313,19 +335,21 @@ def main():
         for i in range(warmup):
             filt(i)
         torch.cuda.synchronize()
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        # `steps` launches back to back, each with its own zeroed counter, bracketed by one pair of events:
+        # the average is the kernel's duration plus the ~1 us gap between queued launches.
+        many = torch.zeros(steps * rows, dtype=torch.int32, device=dev)
+        fe0, fe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        fe0.record()
         for i in range(steps):
-            counts.zero_()
-            evs[i][0].record()
             code = fn(ctypes.c_void_p(dev_inputs[i % copies].data_ptr()), ctypes.c_int64(rows), ctypes.c_int64(n),
                       ctypes.c_void_p(taus.data_ptr()), ctypes.c_int64(pl.capacity), ctypes.c_void_p(buf.data_ptr()),
-                      ctypes.c_void_p(counts.data_ptr()), stream)
-            evs[i][1].record()
+                      ctypes.c_void_p(many.data_ptr() + 4 * i * rows), stream)
+        fe1.record()
         torch.cuda.synchronize()
-        filt_ms = sum(a.elapsed_time(b) for a, b in evs) / steps
+        filt_ms = fe0.elapsed_time(fe1) / steps
+        survivors = float(many[:rows].sum().item())
     clocks = sampler.stop()
     if taus is not None:
-        survivors = float(counts.sum().item())
         algo_bytes = in_bytes + survivors * 8            # read every element once + one 8-byte record per survivor
         peak, peak_kind = measured_peak_gbs()
         achieved = algo_bytes / (filt_ms * 1e-3) / 1e9
@@ -348,7 +372,7 @@ def main():
     cpu_baseline = None
     if not args.no_cpu_baseline:
         cpu_sample = 1 << 25
-        v, dt_s, sample = time_oracle(cfg, cpu_sample, 1, 0)
+        v, dt_s, sample = time_oracle(cfg, cpu_sample, 1, 0, x=host_inputs[0])
         cpu_baseline = {"value": v, "unit": "elements/s", "cores": 1, "kind": "oracle", "sample": sample,
                         "seconds": dt_s}
 

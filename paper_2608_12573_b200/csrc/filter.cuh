@@ -4,7 +4,11 @@
 // The kernel is bound by HBM bandwidth: one 128-bit load per VEC elements, one compare
 // per element, and nothing else on the common path.  Survivors are rare (1e-3 .. 1e-5 of
 // the elements), so the append is a warp-cooperative slow path taken only when some lane
-// of the warp saw a survivor: a warp prefix sum and one global atomic per warp.
+// of the warp saw a survivor.  Survivors are first collected in a small per-warp stage in
+// shared memory and appended to the row buffer 32 or more at a time, so the round trip of
+// the global counter atomic is paid once per flush, not once per tile with a survivor; the
+// slow path is a separate function so that its registers do not limit the occupancy of the
+// streaming loop.
 #pragma once
 
 #include "rowscan.cuh"
@@ -53,13 +57,187 @@ __device__ __forceinline__ bool vec_any_pass(const uint4& v, __nv_bfloat16 tau) 
     return (a & b & c & d) != 0xFFFFFFFFu;    // some lane is not below tau
 }
 
+constexpr uint32_t STAGE_CAP = 64;       // records a warp collects in shared memory ...
+constexpr uint32_t STAGE_FLUSH = 32;     // ... and the fill at which it appends them to the row buffer
+
+// Per-warp staging state, kept in shared memory so that the streaming loop carries none of it.
+struct WarpStage {
+    uint64_t rec[STAGE_CAP];
+    uint32_t fill;        // records waiting
+    uint32_t row;         // the row they belong to
+};
+
+// Appends a warp's staged records to their row's buffer: one global atomic and a few coalesced
+// stores per STAGE_FLUSH survivors.  Returns the row if its buffer has overflowed, else ~0.
+template <typename T>
+__device__ __noinline__ uint32_t flush_stage(const FilterParams<T>& p, WarpStage* st) {
+    const unsigned lane = lane_id();
+    const uint32_t fill = st->fill, row = st->row;
+    unsigned base = 0;
+    if (lane == 0) base = atomicAdd(p.counts + (uint64_t)row * p.count_stride, fill);
+    base = __shfl_sync(FULL_MASK, base, 0);
+    uint64_t* dst = p.buf + (uint64_t)row * p.buf_stride;
+    for (uint32_t i = lane; i < fill; i += 32)
+        if (base + i < p.capacity) dst[base + i] = st->rec[i];
+    __syncwarp();
+    if (lane == 0) st->fill = 0;
+    __syncwarp();
+    return (uint64_t)base + fill > p.capacity ? row : 0xFFFFFFFFu;
+}
+
+// The slow path of one warp and one tile: exact per-element test, records into the warp's stage
+// (or straight into the buffer when the tile is full of survivors).  Kept out of line so that its
+// registers do not weigh on the streaming loop.  Returns a row whose buffer has overflowed, or ~0.
 template <typename T, int THREADS, int UNROLL>
-__global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOCKS_F32 : PROFK_FILTER_MINBLOCKS_BF16) filter_kernel(const FilterParams<T> p) {
+__device__ __noinline__ uint32_t filter_slow_path(const FilterParams<T>& p, WarpStage* st,
+                                                  typename Elem<T>::vec_t v0, typename Elem<T>::vec_t v1,
+                                                  typename Elem<T>::vec_t v2, typename Elem<T>::vec_t v3,
+                                                  uint32_t inside_mask, uint32_t row, uint32_t trow, uint32_t mis, T tau) {
     using V = typename Elem<T>::vec_t;
     constexpr int VEC = Elem<T>::VEC;
     constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
-
+    static_assert(UNROLL == 4, "the slow path takes four vectors");
+    const V v[4] = {v0, v1, v2, v3};
     const unsigned lane = lane_id();
+    const float tau_f = Elem<T>::as_float(tau);
+    unsigned mine[UNROLL];          // per vector: bit l set = element l survives
+    unsigned cnt = 0;
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+        mine[u] = 0;
+        const uint64_t q = (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
+        const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
+#pragma unroll
+        for (int l = 0; l < VEC; ++l) {
+            const int64_t i = i0 + l;
+            const bool ok = ((inside_mask >> u) & 1u) && i >= 0 && i < (int64_t)p.N &&
+                            !(Elem<T>::as_float(vec_elem(v[u], l)) < tau_f);
+            if (ok) mine[u] |= 1u << l;
+        }
+        cnt += __popc(mine[u]);
+    }
+    unsigned incl = cnt;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const unsigned nb = __shfl_up_sync(FULL_MASK, incl, d);
+        if (lane >= (unsigned)d) incl += nb;
+    }
+    const unsigned total = __shfl_sync(FULL_MASK, incl, 31);
+    if (total == 0) return 0xFFFFFFFFu;
+
+    uint32_t overflowed = 0xFFFFFFFFu;
+    uint32_t fill = st->fill;
+    if (fill && (st->row != row || fill + total > STAGE_CAP)) {
+        overflowed = flush_stage(p, st);
+        fill = 0;
+    }
+    uint64_t* out;
+    unsigned pos, limit;
+    const bool to_stage = total <= STAGE_CAP;
+    if (to_stage) {                           // the usual case
+        out = st->rec; pos = fill + incl - cnt; limit = STAGE_CAP;
+    } else {                                  // a tile full of survivors: straight to the buffer
+        unsigned base = 0;
+        if (lane == 0) base = atomicAdd(p.counts + (uint64_t)row * p.count_stride, total);
+        base = __shfl_sync(FULL_MASK, base, 0);
+        out = p.buf + (uint64_t)row * p.buf_stride; pos = base + incl - cnt; limit = p.capacity;
+        if ((uint64_t)base + total > p.capacity) overflowed = row;
+    }
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+        if (mine[u]) {
+            const uint64_t q = (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
+            const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
+#pragma unroll
+            for (int l = 0; l < VEC; ++l) {
+                if (mine[u] & (1u << l)) {
+                    if (pos < limit) out[pos] = make_record(Elem<T>::key(vec_elem(v[u], l)), (uint32_t)(i0 + l));
+                    ++pos;
+                }
+            }
+        }
+    }
+    if (to_stage) {
+        __syncwarp();
+        if (lane == 0) { st->fill = fill + total; st->row = row; }
+        __syncwarp();
+        if (fill + total >= STAGE_FLUSH) {
+            const uint32_t o = flush_stage(p, st);
+            if (o != 0xFFFFFFFFu) overflowed = o;
+        }
+    }
+    return overflowed;
+}
+
+// The slow path without staging (sparse survivors): one global atomic per warp and tile, records
+// written straight to the row buffer.  Returns the row if its buffer has overflowed, else ~0.
+template <typename T, int THREADS, int UNROLL>
+__device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T>& p, const typename Elem<T>::vec_t (&v)[UNROLL],
+                                                            const bool (&inside)[UNROLL], uint32_t row, uint32_t trow,
+                                                            uint32_t mis, T tau) {
+    constexpr int VEC = Elem<T>::VEC;
+    constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
+    const unsigned lane = lane_id();
+    const float tau_f = Elem<T>::as_float(tau);
+    unsigned mine[UNROLL];          // per vector: bit l set = element l survives
+    unsigned cnt = 0;
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+        mine[u] = 0;
+        const uint64_t q = (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
+        const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
+#pragma unroll
+        for (int l = 0; l < VEC; ++l) {
+            const int64_t i = i0 + l;
+            const bool ok = inside[u] && i >= 0 && i < (int64_t)p.N && !(Elem<T>::as_float(vec_elem(v[u], l)) < tau_f);
+            if (ok) mine[u] |= 1u << l;
+        }
+        cnt += __popc(mine[u]);
+    }
+    unsigned incl = cnt;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const unsigned nb = __shfl_up_sync(FULL_MASK, incl, d);
+        if (lane >= (unsigned)d) incl += nb;
+    }
+    const unsigned total = __shfl_sync(FULL_MASK, incl, 31);
+    if (total == 0) return 0xFFFFFFFFu;
+    unsigned base = 0;
+    if (lane == 0) base = atomicAdd(p.counts + (uint64_t)row * p.count_stride, total);
+    base = __shfl_sync(FULL_MASK, base, 0);
+    unsigned pos = base + incl - cnt;
+    uint64_t* dst = p.buf + (uint64_t)row * p.buf_stride;
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+        if (mine[u]) {
+            const uint64_t q = (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
+            const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
+#pragma unroll
+            for (int l = 0; l < VEC; ++l) {
+                if (mine[u] & (1u << l)) {
+                    if (pos < p.capacity) dst[pos] = make_record(Elem<T>::key(vec_elem(v[u], l)), (uint32_t)(i0 + l));
+                    ++pos;
+                }
+            }
+        }
+    }
+    return (uint64_t)base + total > p.capacity ? row : 0xFFFFFFFFu;
+}
+
+// STAGED = collect survivors in per-warp shared-memory stages (dense survivors, one row at a time);
+// otherwise append them directly (sparse survivors or many short rows).
+template <typename T, int THREADS, int UNROLL, bool STAGED>
+__global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOCKS_F32 : PROFK_FILTER_MINBLOCKS_BF16) filter_kernel(const __grid_constant__ FilterParams<T> p) {
+    using V = typename Elem<T>::vec_t;
+    constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
+    __shared__ WarpStage stages[STAGED ? THREADS / 32 : 1];
+
+    WarpStage* st = &stages[STAGED ? threadIdx.x >> 5 : 0];
+    if (STAGED) {
+        if (lane_id() == 0) { st->fill = 0; st->row = 0; }
+        __syncwarp();
+    }
+
     uint32_t tile = blockIdx.x;                  // the grid never exceeds the number of tiles (< 2^32)
     const uint32_t total_tiles = (uint32_t)p.total_tiles, tiles_per_row = (uint32_t)p.tiles_per_row;
 
@@ -84,70 +262,34 @@ __global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOC
         for (int u = 0; u < UNROLL; ++u) hit |= (inside[u] && vec_any_pass(v[u], tau));
 
         if (__any_sync(FULL_MASK, hit) && row != skip_row) {
-            // Slow path: exact per-element test; a warp-wide prefix sum of the per-lane
-            // survivor counts places every lane's records behind one atomic per warp.
-            const float tau_f = Elem<T>::as_float(tau);
-            unsigned mine[UNROLL];          // per vector: bit l set = element l survives
-            unsigned cnt = 0;
+            uint32_t o;
+            if (STAGED) {
+                uint32_t inside_mask = 0;
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u) {
-                mine[u] = 0;
-                const uint64_t q = (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
-                const int64_t i0 = (int64_t)(q * VEC) - (int64_t)rv.mis;
-#pragma unroll
-                for (int l = 0; l < VEC; ++l) {
-                    const int64_t i = i0 + l;
-                    const bool ok = inside[u] && i >= 0 && i < (int64_t)p.N &&
-                                    !(Elem<T>::as_float(vec_elem(v[u], l)) < tau_f);
-                    if (ok) mine[u] |= 1u << l;
-                }
-                cnt += __popc(mine[u]);
+                for (int u = 0; u < UNROLL; ++u) inside_mask |= inside[u] ? 1u << u : 0u;
+                o = filter_slow_path<T, THREADS, UNROLL>(p, st, v[0], v[1], v[2], v[3], inside_mask, row, trow, rv.mis, tau);
+            } else {
+                o = filter_slow_path_direct<T, THREADS, UNROLL>(p, v, inside, row, trow, rv.mis, tau);
             }
-            unsigned incl = cnt;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const unsigned nb = __shfl_up_sync(FULL_MASK, incl, d);
-                if (lane >= (unsigned)d) incl += nb;
-            }
-            const unsigned total = __shfl_sync(FULL_MASK, incl, 31);
-            if (total) {
-                unsigned base = 0;
-                if (lane == 0) base = atomicAdd(p.counts + (uint64_t)row * p.count_stride, total);
-                base = __shfl_sync(FULL_MASK, base, 0);
-                unsigned pos = base + incl - cnt;
-                uint64_t* dst = p.buf + (uint64_t)row * p.buf_stride;
-#pragma unroll
-                for (int u = 0; u < UNROLL; ++u) {
-                    if (mine[u]) {
-                        const uint64_t q = (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
-                        const int64_t i0 = (int64_t)(q * VEC) - (int64_t)rv.mis;
-#pragma unroll
-                        for (int l = 0; l < VEC; ++l) {
-                            if (mine[u] & (1u << l)) {
-                                if (pos < p.capacity)
-                                    dst[pos] = make_record(Elem<T>::key(vec_elem(v[u], l)), (uint32_t)(i0 + l));
-                                ++pos;
-                            }
-                        }
-                    }
-                }
-                if ((uint64_t)base + total > p.capacity) skip_row = row;   // overflow: the exact path redoes this row
-            }
+            if (o != 0xFFFFFFFFu) skip_row = o;
         }
 
         // Next tile of this CTA; tiles of a row already known to overflow are not even loaded.
         uint32_t nrow;
+        bool more = true;
         do {
-            if (total_tiles - tile <= gridDim.x) return;
+            if (total_tiles - tile <= gridDim.x) { more = false; break; }
             tile += gridDim.x;
             nrow = tile / tiles_per_row;
         } while (nrow == skip_row);
+        if (!more) break;
         trow = tile - nrow * tiles_per_row;
         if (nrow != row) { row = nrow; rv = row_view(p.in, p.N, row); }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u)
             v[u] = load_row_vector(rv, p.N, (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x, &inside[u]);
     }
+    if (STAGED && st->fill) flush_stage(p, st);
 }
 
 }  // namespace profk

@@ -35,6 +35,7 @@ std::atomic<int> g_coop_pdl{-1};                 // -1 untried, 1 accepted, 0 re
 struct DeviceInfo {
     int sm_count = 0;
     int filter_blocks_per_sm[2] = {0, 0};     // by dtype
+    int filter_staged_blocks_per_sm[2] = {0, 0};
     int fallback_blocks_per_sm[2] = {0, 0};
     int max_cluster[2] = {8, 8};              // 16 when the device can co-schedule 16 CTAs of the threshold kernel
     int large_cluster[2] = {8, 8};            // same for the cluster sort (128 KB of shared memory per CTA)
@@ -92,9 +93,12 @@ template <typename T> int ensure_device_info(int dev, DeviceInfo* out) {
     const int d = dtype_index<T>();
     if (di.filter_blocks_per_sm[d] == 0) {
         int nb = 0;
-        CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL>,
+        CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false>,
                                                                  FILTER_THREADS, 0));
         di.filter_blocks_per_sm[d] = std::max(nb, 1);
+        CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, true>,
+                                                                 FILTER_THREADS, 0));
+        di.filter_staged_blocks_per_sm[d] = std::max(nb, 1);
         CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fallback_kernel<T>, FB_THREADS, 0));
         di.fallback_blocks_per_sm[d] = std::max(nb, 1);
         CUDA_TRY(cudaFuncSetAttribute(sample_select_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
@@ -175,8 +179,7 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
 
 template <typename T>
 int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, const T* tau, int64_t capacity, uint64_t* buf,
-                  uint64_t buf_stride,
-                  uint32_t* counts, uint32_t count_stride, bool pdl, cudaStream_t st) {
+                  uint64_t buf_stride, uint32_t* counts, uint32_t count_stride, bool pdl, bool staged, cudaStream_t st) {
     FilterParams<T> fp;
     fp.in = in; fp.N = (uint64_t)N; fp.rows = (uint64_t)rows; fp.tau = tau; fp.capacity = (uint32_t)capacity;
     fp.buf = buf; fp.buf_stride = buf_stride; fp.counts = counts; fp.count_stride = count_stride;
@@ -184,7 +187,8 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     fp.total_tiles = fp.tiles_per_row * (uint64_t)rows;
     if (fp.total_tiles >= (1ull << 32)) return PROFK_EINVAL;      // rows * N beyond 2^45 elements
     fp.use_pdl = pdl ? 1 : 0;
-    const uint64_t max_grid = (uint64_t)di.sm_count * di.filter_blocks_per_sm[dtype_index<T>()];
+    const uint64_t max_grid = (uint64_t)di.sm_count *
+        (staged ? di.filter_staged_blocks_per_sm[dtype_index<T>()] : di.filter_blocks_per_sm[dtype_index<T>()]);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)std::min<uint64_t>(fp.total_tiles, max_grid));
     cfg.blockDim = dim3(FILTER_THREADS);
@@ -194,7 +198,8 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL>, fp));
+    if (staged) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, true>, fp));
+    else CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false>, fp));
     ++g_launches;
     return PROFK_OK;
 }
@@ -265,10 +270,15 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     uint32_t sort_cap = 32;
     while (sort_cap < (uint32_t)k && sort_cap < SORT_CAP_MAX) sort_cap <<= 1;
 
+    // Survivors are staged per warp when a warp's tile is expected to hold a good fraction of one
+    // (expected survivors per element ~ r / m); sparse survivors are appended directly.
+    const double per_warp_tile = (double)plan->r / (double)std::max<int64_t>(plan->m, 1) * 32.0 * FILTER_UNROLL * Elem<T>::VEC;
+    const bool staged = plan->mode == 0 && rows == 1 && per_warp_tile > 0.2;
+
     if (plan->mode == 0) {
         rc = launch_sample_select<T>(di, in, rows, N, plan->m, plan->r, seed, tau, ctl, header, (uint32_t)capacity, nullptr, st);
         if (rc != PROFK_OK) return rc;
-        rc = launch_filter<T>(di, in, rows, N, tau, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, st);
+        rc = launch_filter<T>(di, in, rows, N, tau, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, st);
         if (rc != PROFK_OK) return rc;
 
         if (large) {
@@ -382,7 +392,7 @@ int filter_only(const T* in, int64_t rows, int64_t N, const T* tau, int64_t capa
     DeviceInfo di;
     const int rc = ensure_device_info<T>(dev, &di);
     if (rc != PROFK_OK) return rc;
-    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, (uint64_t)capacity, counts, 1, false, static_cast<cudaStream_t>(stream));
+    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, (uint64_t)capacity, counts, 1, false, false, static_cast<cudaStream_t>(stream));
 }
 
 template <typename T>
