@@ -170,8 +170,9 @@ int profk_topk_planned_bf16(const void* in, int64_t rows, int64_t N, int64_t k, 
  *   counts     [device] rows uint32, must be zero on entry; on return the
  *              number of survivors (exact if <= capacity, else some value > capacity)
  * A candidate record packs the complemented order key of the value in the high
- * 32 bits (bf16: key in bits 63..48) and the index in the low 32 bits, so that
- * ascending records are "value descending, index ascending".  Records are
+ * 32 bits (bf16: the 16-bit key in bits 47..32, bits 63..48 all ones) and the
+ * index in the low 32 bits, so that ascending records are "value descending,
+ * index ascending".  Records are
  * appended in no particular order.  Needs no workspace.
  */
 int profk_filter_f32(const float* in, int64_t rows, int64_t N, const float* tau, int64_t capacity,

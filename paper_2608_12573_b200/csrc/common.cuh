@@ -12,8 +12,9 @@ constexpr unsigned FULL_MASK = 0xFFFFFFFFu;
 
 // ---------------------------------------------------------------------------------------
 // Order keys.  key(x) is an unsigned integer whose order is the total order
-// -NaN < -inf < ... < -0 < +0 < ... < +inf < +NaN of the bit patterns.  Both element types
-// use a 32-bit key; a bf16 key occupies the upper 16 bits (lower 16 bits zero).
+// -NaN < -inf < ... < -0 < +0 < ... < +inf < +NaN of the bit patterns.  Keys travel in 32-bit
+// words; a bf16 key is the 16-bit key of its pattern in the lower half (KEY_BITS = 16), so that
+// in a candidate record it sits directly above the index.
 __device__ __forceinline__ uint32_t key_from_bits32(uint32_t b) {
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
@@ -35,6 +36,7 @@ template <typename T> struct Elem;
 template <> struct Elem<float> {
     using vec_t = float4;                       // 128-bit vector
     static constexpr int VEC = 4;               // elements per vector
+    static constexpr int KEY_BITS = 32;
     static constexpr uint32_t NEG_INF_BITS = 0xFF800000u;
     static __device__ __forceinline__ uint32_t bits(float v) { return float_bits_exact(v); }
     static __device__ __forceinline__ uint32_t key(float v) { return key_from_bits32(float_bits_exact(v)); }
@@ -46,13 +48,14 @@ template <> struct Elem<float> {
 template <> struct Elem<__nv_bfloat16> {
     using vec_t = uint4;                        // 8 bf16 in 128 bits
     static constexpr int VEC = 8;
+    static constexpr int KEY_BITS = 16;
     static constexpr uint32_t NEG_INF_BITS = 0xFF80u;
     static __device__ __forceinline__ uint32_t bits(__nv_bfloat16 v) { return (uint32_t)__bfloat16_as_ushort(v); }
     static __device__ __forceinline__ uint32_t key(__nv_bfloat16 v) {
-        return key_from_bits32((uint32_t)__bfloat16_as_ushort(v) << 16) & 0xFFFF0000u;
+        return key_from_bits32((uint32_t)__bfloat16_as_ushort(v) << 16) >> 16;
     }
     static __device__ __forceinline__ __nv_bfloat16 from_key(uint32_t k) {
-        const uint32_t k16 = k >> 16;
+        const uint32_t k16 = k & 0xFFFFu;
         const uint32_t b = (k16 & 0x8000u) ? (k16 & 0x7FFFu) : (~k16 & 0xFFFFu);
         return __ushort_as_bfloat16((unsigned short)b);
     }

@@ -52,16 +52,16 @@ std::map<std::tuple<int64_t, int64_t, double, double>, profk_plan_t> g_plan_cach
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-    size_t off_header, off_ghist, off_ctl, off_tau, off_buf, total;
+    size_t off_header, off_ghist, off_ctl, off_tau, off_bins, off_buf, total;
 };
 
 // Records reserved per row: the capacity itself, or -- when k is too large for the single-CTA
-// refine -- the power of two the cluster sort pads the row to.
+// refine -- twice the power of two the cluster sort pads the row to (records, then scratch).
 uint64_t row_stride_for(int64_t capacity, int64_t k) {
     if (k <= (int64_t)SORT_CAP_MAX) return (uint64_t)capacity;
     uint64_t p = BT_TILE;
     while (p < (uint64_t)capacity) p <<= 1;
-    return p;
+    return 2 * p;
 }
 
 WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k) {
@@ -70,7 +70,9 @@ WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k) {
     l.off_ghist = sizeof(WsHeader);
     l.off_ctl = align_up(l.off_ghist + (size_t)FB_PASSES * FB_BINS * sizeof(uint32_t), 256);
     l.off_tau = align_up(l.off_ctl + (size_t)rows * sizeof(RowCtl), 256);
-    l.off_buf = align_up(l.off_tau + (size_t)rows * 4, 256);
+    l.off_bins = align_up(l.off_tau + (size_t)rows * 4, 256);
+    const size_t bins_bytes = k > (int64_t)SORT_CAP_MAX ? (size_t)rows * (LG_BINS + 8) * sizeof(uint32_t) : 0;
+    l.off_buf = align_up(l.off_bins + bins_bytes, 256);
     l.total = align_up(l.off_buf + (size_t)rows * (size_t)row_stride_for(capacity, k) * sizeof(uint64_t), 256);
     return l;
 }
@@ -205,10 +207,11 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
 }
 
 template <typename T>
-int launch_refine_large(const DeviceInfo& di, RowCtl* ctl, WsHeader* header, uint64_t* buf, uint64_t row_stride, int64_t rows,
+int launch_refine_large(const DeviceInfo& di, RowCtl* ctl, WsHeader* header, uint64_t* buf, uint64_t row_pitch, uint32_t* bins, int64_t rows,
                         int64_t capacity, int64_t k, int64_t k_accept, int phase, T* out_vals, int64_t* out_idx, cudaStream_t st) {
     LargeParams<T> lp;
-    lp.ctl = ctl; lp.header = header; lp.buf = buf; lp.row_stride = row_stride; lp.capacity = (uint32_t)capacity;
+    const uint64_t row_stride = row_pitch / 2;
+    lp.ctl = ctl; lp.header = header; lp.buf = buf; lp.row_stride = row_stride; lp.bins = bins; lp.capacity = (uint32_t)capacity;
     lp.k = (uint32_t)k; lp.k_accept = (uint32_t)k_accept; lp.phase = phase; lp.out_vals = out_vals; lp.out_idx = out_idx;
     lp.use_pdl = 1;
     int csize = di.large_cluster[dtype_index<T>()];
@@ -265,6 +268,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     RowCtl* ctl = reinterpret_cast<RowCtl*>(base + lay.off_ctl);
     T* tau = reinterpret_cast<T*>(base + lay.off_tau);
     uint64_t* buf = reinterpret_cast<uint64_t*>(base + lay.off_buf);
+    uint32_t* bins = reinterpret_cast<uint32_t*>(base + lay.off_bins);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
     uint32_t sort_cap = 32;
@@ -282,7 +286,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         if (rc != PROFK_OK) return rc;
 
         if (large) {
-            rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, rows, capacity, k, plan->k_accept, 0, out_vals, out_idx, st);
+            rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, rows, capacity, k, plan->k_accept, 0, out_vals, out_idx, st);
             if (rc != PROFK_OK) return rc;
         } else {
         // refine: count check, then order the buffer of every row that passed it
@@ -354,7 +358,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         ++g_launches;
     }
     if (large) {   // the rows the exact selection repaired still have to be ordered and written
-        rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, rows, capacity, k, k, 1, out_vals, out_idx, st);
+        rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, rows, capacity, k, k, 1, out_vals, out_idx, st);
         if (rc != PROFK_OK) return rc;
     }
     return PROFK_OK;

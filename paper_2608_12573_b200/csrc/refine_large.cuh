@@ -1,14 +1,18 @@
 // Stage 4 for large selections (k beyond what one CTA orders in shared memory; the flattened
 // BatchTopK case of Section 5, "Application", selects K = B k = 131,072 values): the count
-// check, then a full ascending sort of the row's candidate records -- which is "value
-// descending, index ascending" -- by one thread-block cluster, and the first k are the answer.
+// check, then the k smallest candidate records in ascending order -- which is "value
+// descending, index ascending" -- by one thread-block cluster.
 //
-// The sort is a bitonic network over P = 2^j records in the row's buffer (padded with all-ones
-// records).  Exchanges at distance below one tile (16384 records = 128 KB) run in shared
-// memory, tile by tile; the few longer ones run on the buffer in global memory, separated by
-// hardware cluster barriers.  A bitonic network does the same work whatever the data, so
-// heavy ties (bf16 inputs hold thousands of copies of each value near the threshold) cost
-// nothing extra.
+// Main path: the records are binned on the top 18 bits of their distance above the smallest
+// record (262144 bins in global memory; because a record holds the value key above the index,
+// equal values are spread over bins by index), a cluster-wide scan turns the counts into
+// first positions, the records are scattered into a second buffer grouped by bin, and every
+// record of a bin that reaches into the first k positions ranks itself inside its bin -- a
+// handful of comparisons -- to find its place in the output.
+// Reserve path, taken when a bin is too crowded for that (an outlier stretches the range):
+// a bitonic network over P = 2^j records in the row's buffer, exchanges below one tile
+// (16384 records = 128 KB) in shared memory, the longer ones on the buffer in global memory.
+// Both paths use hardware cluster barriers only.
 #pragma once
 
 #include <cooperative_groups.h>
@@ -19,12 +23,16 @@ namespace profk {
 
 constexpr uint32_t BT_TILE = 16384;          // records per shared-memory tile
 constexpr int BT_THREADS = 1024;
+constexpr int LG_BITS = 18;                  // digit width of the binning
+constexpr uint32_t LG_BINS = 1u << LG_BITS;
+constexpr uint32_t LG_CROWDED = 1024;        // a bin this full (among those that matter) sends the row to the reserve path
 
 template <typename T> struct LargeParams {
     RowCtl* ctl;
     WsHeader* header;
-    uint64_t* buf;           // rows x row_stride records; row_stride is a power of two >= capacity, >= BT_TILE
-    uint64_t row_stride;
+    uint64_t* buf;           // row r: records at buf + r * 2 * row_stride, then row_stride records of scratch;
+    uint64_t row_stride;     //        row_stride is a power of two >= capacity, >= BT_TILE
+    uint32_t* bins;          // rows x (LG_BINS + 8) words: bin counts / positions, then flags
     uint32_t capacity;
     uint32_t k;
     uint32_t k_accept;
@@ -88,14 +96,121 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         n = p.k;                             // the exact selection left exactly k records
     }
     const uint32_t kk = n < p.k ? n : p.k;
-    uint64_t* G = p.buf + row * p.row_stride;
-    uint64_t P = BT_TILE;
-    while (P < n) P <<= 1;
+    uint64_t* G = p.buf + row * 2 * p.row_stride;
+    uint64_t* G2 = G + p.row_stride;
+    uint32_t* bins = p.bins + row * (uint64_t)(LG_BINS + 8);
+    uint32_t* flags = bins + LG_BINS;                                // [0] = some bin that matters is crowded
 
     for (uint64_t j = kk + gid; j < p.k; j += gthreads) {            // relaxed mode: padding after a short buffer
         p.out_vals[row * (uint64_t)p.k + j] = Elem<T>::from_bits(Elem<T>::NEG_INF_BITS);
         p.out_idx[row * (uint64_t)p.k + j] = -1;
     }
+
+    // ================= main path: bin, scan, scatter, rank inside bins =================
+    __shared__ unsigned long long s_min[32], s_max[32], s_cta_min, s_cta_max;
+    __shared__ uint32_t s_warp[32], s_cta_total;
+    {
+        // smallest and largest record of the row; clear the bins meanwhile
+        for (uint64_t b = gid; b < LG_BINS + 8; b += gthreads) bins[b] = 0;
+        unsigned long long lo = ~0ull, hi = 0ull;
+        for (uint64_t i = gid; i < n; i += gthreads) {
+            const unsigned long long rec = __ldcg(&G[i]);
+            lo = rec < lo ? rec : lo;
+            hi = rec > hi ? rec : hi;
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            const unsigned long long l2 = __shfl_xor_sync(FULL_MASK, lo, d), h2 = __shfl_xor_sync(FULL_MASK, hi, d);
+            lo = l2 < lo ? l2 : lo;
+            hi = h2 > hi ? h2 : hi;
+        }
+        if ((tid & 31) == 0) { s_min[tid >> 5] = lo; s_max[tid >> 5] = hi; }
+        __syncthreads();
+        if (tid < 32) {
+            lo = s_min[tid]; hi = s_max[tid];
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+                const unsigned long long l2 = __shfl_xor_sync(FULL_MASK, lo, d), h2 = __shfl_xor_sync(FULL_MASK, hi, d);
+                lo = l2 < lo ? l2 : lo;
+                hi = h2 > hi ? h2 : hi;
+            }
+            if (tid == 0) { s_cta_min = lo; s_cta_max = hi; }
+        }
+        cluster.sync();
+        unsigned long long rmin = ~0ull, rmax = 0ull;
+        for (unsigned c = 0; c < csize; ++c) {
+            const unsigned long long l2 = *cluster.map_shared_rank(&s_cta_min, c), h2 = *cluster.map_shared_rank(&s_cta_max, c);
+            rmin = l2 < rmin ? l2 : rmin;
+            rmax = h2 > rmax ? h2 : rmax;
+        }
+        const int rbits = 64 - __clzll((long long)(rmax - rmin));    // range < 2^rbits
+        const int shift = rbits > LG_BITS ? rbits - LG_BITS : 0;
+        auto bin_of = [&](unsigned long long rec) { return (uint32_t)((rec - rmin) >> shift); };
+
+        // histogram (global atomics spread over 65536 addresses)
+        for (uint64_t i = gid; i < n; i += gthreads) atomicAdd(&bins[bin_of(__ldcg(&G[i]))], 1u);
+        cluster.sync();
+
+        // scan: CTA c owns bins [c, c+1) * LG_BINS / csize; counts become end positions
+        const uint32_t per_cta = LG_BINS / csize, per_thr = per_cta / BT_THREADS;      // csize <= 16: per_thr >= 4
+        const uint32_t b0 = crank * per_cta + tid * per_thr;
+        uint32_t sum = 0;
+        for (uint32_t j = 0; j < per_thr; ++j) sum += __ldcg(&bins[b0 + j]);
+        uint32_t incl = sum;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t v = __shfl_up_sync(FULL_MASK, incl, d);
+            if ((tid & 31) >= (unsigned)d) incl += v;
+        }
+        if ((tid & 31) == 31) s_warp[tid >> 5] = incl;
+        __syncthreads();
+        if (tid < 32) {
+            uint32_t w = s_warp[tid];
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t v = __shfl_up_sync(FULL_MASK, w, d);
+                if (tid >= (unsigned)d) w += v;
+            }
+            s_warp[tid] = w;
+            if (tid == 31) s_cta_total = w;
+        }
+        cluster.sync();
+        uint32_t before = incl - sum + ((tid >> 5) ? s_warp[(tid >> 5) - 1] : 0);
+        for (unsigned c = 0; c < crank; ++c) before += *cluster.map_shared_rank(&s_cta_total, c);
+        for (uint32_t j = 0; j < per_thr; ++j) {
+            const uint32_t c = __ldcg(&bins[b0 + j]);
+            if (before < kk && c > LG_CROWDED) atomicOr(&flags[0], 1u);
+            bins[b0 + j] = before;                                   // first position; the scatter advances it to the end
+            before += c;
+        }
+        cluster.sync();
+
+        if (__ldcg(&flags[0]) == 0) {
+            // scatter into the second buffer, grouped by bin
+            for (uint64_t i = gid; i < n; i += gthreads) {
+                const unsigned long long rec = __ldcg(&G[i]);
+                G2[atomicAdd(&bins[bin_of(rec)], 1u)] = rec;
+            }
+            cluster.sync();
+            // rank inside the bin: bin b now occupies [end of bin b-1, bins[b])
+            for (uint64_t g = gid; g < n; g += gthreads) {
+                const unsigned long long rec = __ldcg(&G2[g]);
+                const uint32_t b = bin_of(rec);
+                const uint32_t first = b ? __ldcg(&bins[b - 1]) : 0u;
+                if (first >= kk) continue;
+                const uint32_t last = __ldcg(&bins[b]);
+                uint32_t pos = first;
+                for (uint32_t j = first; j < last; ++j) pos += __ldcg(&G2[j]) < rec;
+                if (pos < kk) write_output(p.out_vals, p.out_idx, p.k, row, pos, rec);
+            }
+            cluster.sync();              // peers may still be reading this CTA's shared memory above
+            return;
+        }
+    }
+
+    // ================= reserve path: bitonic network =================
+    uint64_t P = BT_TILE;
+    while (P < n) P <<= 1;
 
     // ---- sort every tile (sizes 2 .. BT_TILE); positions beyond n hold all-ones padding ----
     const uint64_t tiles = P / BT_TILE;

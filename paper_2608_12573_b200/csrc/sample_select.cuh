@@ -275,7 +275,8 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
     // ---- stage 2, general case: radix select over the cluster --------------------------
     if (!done) {
         constexpr int NPASS = sizeof(T) == 4 ? 3 : 2;
-        const int shifts[3] = {21, sizeof(T) == 4 ? 10 : 16, 0};
+        constexpr int KB = Elem<T>::KEY_BITS;
+        const int shifts[3] = {KB - 11, sizeof(T) == 4 ? 10 : 0, 0};
         const int widths[3] = {11, sizeof(T) == 4 ? 11 : 5, 10};
         uint32_t prefix = 0;        // selected high bits so far (right-aligned)
         uint32_t need = p.t;        // rank among the keys that match the prefix, from the top
@@ -289,7 +290,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
             __syncthreads();
             for (uint32_t i = tid; i < n_round; i += SEL_THREADS) {
                 const uint32_t k = i < n_local ? keys[i] : 0;
-                const bool in_class = i < n_local && (consumed == 0 || (k >> (32 - consumed)) == prefix);
+                const bool in_class = i < n_local && (consumed == 0 || (k >> (KB - consumed)) == prefix);
                 const uint32_t digit = in_class ? (k >> shift) & (nbins - 1) : 0xFFFFFFFFu;
                 const unsigned peers = __match_any_sync(FULL_MASK, digit);
                 if (in_class && lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&h[digit], __popc(peers));
@@ -317,7 +318,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
             consumed += width;
             __syncthreads();   // s_digit / s_before are rewritten in the next pass
         }
-        const uint32_t tau_key = prefix << (32 - consumed);
+        const uint32_t tau_key = prefix << (KB - consumed);
         if (crank == 0 && tid == 0) publish_threshold(p, row, tau_key);
         cluster.sync();   // no CTA leaves while a peer may still read its histogram
     }

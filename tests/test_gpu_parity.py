@@ -241,7 +241,7 @@ def test_filter_keeps_exactly_the_survivor_set(dtype):
         assert np.array_equal(got_idx, want)                                  # same set, any order
         keys = (~(rec >> np.uint64(32))).astype(np.uint32)
         okeys = o_topk.order_key(xn[row])
-        okeys32 = okeys.astype(np.uint32) if dtype == torch.float32 else (okeys.astype(np.uint32) << 16)
+        okeys32 = okeys.astype(np.uint32)                                    # a bf16 key sits in the low 16 bits
         order = np.argsort(rec & np.uint64(0xFFFFFFFF))
         assert np.array_equal(keys[order], okeys32[want])
     # overflow: the counter only has to exceed the capacity
