@@ -105,14 +105,15 @@ __device__ __noinline__ uint32_t filter_slow_path(const FilterParams<T>& p, Warp
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) {
         mine[u] = 0;
-        const uint64_t q = (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
-        const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
+        if (((inside_mask >> u) & 1u) && vec_any_pass(v[u], tau)) {      // most vectors hold no survivor
+            const uint64_t q = (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
+            const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
 #pragma unroll
-        for (int l = 0; l < VEC; ++l) {
-            const int64_t i = i0 + l;
-            const bool ok = ((inside_mask >> u) & 1u) && i >= 0 && i < (int64_t)p.N &&
-                            !(Elem<T>::as_float(vec_elem(v[u], l)) < tau_f);
-            if (ok) mine[u] |= 1u << l;
+            for (int l = 0; l < VEC; ++l) {
+                const int64_t i = i0 + l;
+                const bool ok = i >= 0 && i < (int64_t)p.N && !(Elem<T>::as_float(vec_elem(v[u], l)) < tau_f);
+                if (ok) mine[u] |= 1u << l;
+            }
         }
         cnt += __popc(mine[u]);
     }
@@ -184,13 +185,15 @@ __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) {
         mine[u] = 0;
-        const uint64_t q = (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
-        const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
+        if (inside[u] && vec_any_pass(v[u], tau)) {                      // most vectors hold no survivor
+            const uint64_t q = (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
+            const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
 #pragma unroll
-        for (int l = 0; l < VEC; ++l) {
-            const int64_t i = i0 + l;
-            const bool ok = inside[u] && i >= 0 && i < (int64_t)p.N && !(Elem<T>::as_float(vec_elem(v[u], l)) < tau_f);
-            if (ok) mine[u] |= 1u << l;
+            for (int l = 0; l < VEC; ++l) {
+                const int64_t i = i0 + l;
+                const bool ok = i >= 0 && i < (int64_t)p.N && !(Elem<T>::as_float(vec_elem(v[u], l)) < tau_f);
+                if (ok) mine[u] |= 1u << l;
+            }
         }
         cnt += __popc(mine[u]);
     }

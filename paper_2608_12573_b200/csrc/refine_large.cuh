@@ -113,10 +113,17 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         // smallest and largest record of the row; clear the bins meanwhile
         for (uint64_t b = gid; b < LG_BINS + 8; b += gthreads) bins[b] = 0;
         unsigned long long lo = ~0ull, hi = 0ull;
-        for (uint64_t i = gid; i < n; i += gthreads) {
-            const unsigned long long rec = __ldcg(&G[i]);
-            lo = rec < lo ? rec : lo;
-            hi = rec > hi ? rec : hi;
+        for (uint64_t i0 = gid; i0 < n; i0 += 4 * gthreads) {           // four loads in flight per thread
+            unsigned long long rec[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) rec[u] = i0 + u * gthreads < n ? __ldcg(&G[i0 + u * gthreads]) : ~0ull;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (i0 + u * gthreads < n) {
+                    lo = rec[u] < lo ? rec[u] : lo;
+                    hi = rec[u] > hi ? rec[u] : hi;
+                }
+            }
         }
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) {
@@ -148,7 +155,14 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         auto bin_of = [&](unsigned long long rec) { return (uint32_t)((rec - rmin) >> shift); };
 
         // histogram (global atomics spread over 65536 addresses)
-        for (uint64_t i = gid; i < n; i += gthreads) atomicAdd(&bins[bin_of(__ldcg(&G[i]))], 1u);
+        for (uint64_t i0 = gid; i0 < n; i0 += 4 * gthreads) {
+            unsigned long long rec[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) rec[u] = i0 + u * gthreads < n ? __ldcg(&G[i0 + u * gthreads]) : 0ull;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (i0 + u * gthreads < n) atomicAdd(&bins[bin_of(rec[u])], 1u);
+        }
         cluster.sync();
 
         // scan: CTA c owns bins [c, c+1) * LG_BINS / csize; counts become end positions
@@ -187,21 +201,40 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
 
         if (__ldcg(&flags[0]) == 0) {
             // scatter into the second buffer, grouped by bin
-            for (uint64_t i = gid; i < n; i += gthreads) {
-                const unsigned long long rec = __ldcg(&G[i]);
-                G2[atomicAdd(&bins[bin_of(rec)], 1u)] = rec;
+            for (uint64_t i0 = gid; i0 < n; i0 += 4 * gthreads) {
+                unsigned long long rec[4];
+                uint32_t pos[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) rec[u] = i0 + u * gthreads < n ? __ldcg(&G[i0 + u * gthreads]) : 0ull;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) pos[u] = i0 + u * gthreads < n ? atomicAdd(&bins[bin_of(rec[u])], 1u) : 0u;
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (i0 + u * gthreads < n) G2[pos[u]] = rec[u];
             }
             cluster.sync();
             // rank inside the bin: bin b now occupies [end of bin b-1, bins[b])
-            for (uint64_t g = gid; g < n; g += gthreads) {
-                const unsigned long long rec = __ldcg(&G2[g]);
-                const uint32_t b = bin_of(rec);
-                const uint32_t first = b ? __ldcg(&bins[b - 1]) : 0u;
-                if (first >= kk) continue;
-                const uint32_t last = __ldcg(&bins[b]);
-                uint32_t pos = first;
-                for (uint32_t j = first; j < last; ++j) pos += __ldcg(&G2[j]) < rec;
-                if (pos < kk) write_output(p.out_vals, p.out_idx, p.k, row, pos, rec);
+            // (only positions below the end of the bin that holds position kk-1 matter; they are a prefix)
+            for (uint64_t g0 = gid; g0 < n; g0 += 4 * gthreads) {
+                unsigned long long rec[4];
+                uint32_t first[4], last[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) rec[u] = g0 + u * gthreads < n ? __ldcg(&G2[g0 + u * gthreads]) : rmin;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t b = bin_of(rec[u]);
+                    first[u] = b ? __ldcg(&bins[b - 1]) : 0u;
+                    last[u] = __ldcg(&bins[b]);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (g0 + u * gthreads < n && first[u] < kk) {
+                        uint32_t pos = first[u];
+                        for (uint32_t j = first[u]; j < last[u]; ++j) pos += __ldcg(&G2[j]) < rec[u];
+                        if (pos < kk) write_output(p.out_vals, p.out_idx, p.k, row, pos, rec[u]);
+                    }
+                }
+                if (g0 >= kk + LG_CROWDED) break;           // grouped positions beyond every bin that matters
             }
             cluster.sync();              // peers may still be reading this CTA's shared memory above
             return;
