@@ -46,7 +46,8 @@ typedef enum profk_status {
     PROFK_EINVAL = -1,     /* bad argument (range, null pointer, alignment) */
     PROFK_EWORKSPACE = -2, /* no workspace registered on this device, or it is too small */
     PROFK_ECUDA = -3,      /* a CUDA runtime call or launch reported an error */
-    PROFK_ETIMEOUT = -4    /* (statistics only) a bounded device-side wait gave up */
+    PROFK_ETIMEOUT = -4,   /* (statistics only) a bounded device-side wait gave up */
+    PROFK_ETOOLARGE = -5   /* profk_topk_noalloc_f32 only: the shape needs more than the built-in scratch */
 } profk_status_t;
 
 typedef enum profk_dtype { PROFK_F32 = 0, PROFK_BF16 = 1 } profk_dtype_t;
@@ -189,6 +190,32 @@ int profk_sample_threshold_f32(const float* in, int64_t rows, int64_t N, int64_t
                                float* tau, uint32_t* sample_idx, void* stream);
 int profk_sample_threshold_bf16(const void* in, int64_t rows, int64_t N, int64_t m, int64_t r, uint64_t seed,
                                 void* tau, uint32_t* sample_idx, void* stream);
+
+/*
+ * (This entry point has no counterpart in the paper; it exists for callers that must not
+ * allocate.)  Same result as profk_topk_f32, but no workspace has to be registered and no
+ * call made here allocates or frees anything, on the host side of CUDA or on the device:
+ * the scratch is a 16 MiB array that is part of the library itself.  It is meant for code
+ * that runs where an allocation is forbidden or would deadlock -- a callback of a memory
+ * pool that is itself inside an allocation, a real-time or plug-in context that was handed
+ * its buffers up front, a host that has already given all device memory to another
+ * allocator -- and still needs a top-k of buffers it already owns.
+ *   - Limit: the workspace the shape needs (profk_workspace_bytes for rows, the plan's
+ *     capacity and k) must fit 16 MiB; roughly rows * capacity <= 2,000,000 records, e.g.
+ *     one row of any length up to the library limit with small k, or 512 rows of 2^20
+ *     elements with k = 32.  Anything larger returns PROFK_ETOOLARGE and does nothing.
+ *   - Every GPU that loads the library holds the 16 MiB until the process exits.
+ *   - The first call on each device looks up the array's device address (it keeps the
+ *     result); make that first call outside any stream capture.
+ *   - All calls share the one array, and it keeps whatever the last call left in it.  Each
+ *     call re-initialises the parts that must start at zero, so calls issued one after the
+ *     other on a stream are fine; two calls that overlap on the GPU (different streams,
+ *     different threads) race on it and give wrong answers.
+ *   - profk_read_stats does not see this call (it reads the registered workspace).
+ * Arguments, layout and the other errors are those of profk_topk_f32.
+ */
+int profk_topk_noalloc_f32(const float* in, int64_t rows, int64_t N, int64_t k, double eps, double recall,
+                           uint64_t seed, void* stream, float* out_vals, int64_t* out_idx);
 
 /*
  * Copies the statistics of the last call that used the registered workspace to

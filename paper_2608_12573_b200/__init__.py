@@ -19,7 +19,7 @@ EXPORTS = [
     "profk_plan", "profk_plan_ex", "profk_workspace_bytes", "profk_set_workspace",
     "profk_topk_f32", "profk_topk_bf16", "profk_topk_planned_f32", "profk_topk_planned_bf16",
     "profk_filter_f32", "profk_filter_bf16", "profk_sample_threshold_f32", "profk_sample_threshold_bf16",
-    "profk_read_stats", "profk_last_launch_count", "profk_strerror",
+    "profk_read_stats", "profk_last_launch_count", "profk_strerror", "profk_topk_noalloc_f32",
 ]
 
 ROW_OK, ROW_RECALL, ROW_OVERFLOW, ROW_DIRECT = 0, 1, 2, 3
@@ -210,6 +210,31 @@ def topk(x, k: int, eps: float = 1e-3, recall: float = 1.0, seed: int = 0, plan_
     if one_d:
         return vals[0], idx[0]
     return vals, idx
+
+
+def topk_noalloc(x, k: int, eps: float = 1e-3, recall: float = 1.0, seed: int = 0, out=None):
+    """`profk_topk_noalloc_f32`: top-k with the library's built-in scratch, for callers that must not
+    allocate.  The output tensors are the caller's (`out=(values, indices)`); when `out` is omitted this
+    convenience wrapper allocates them through torch, which the C entry point itself never does.
+    float32 only; shapes whose workspace exceeds 16 MiB raise ProfkError."""
+    import torch
+
+    one_d = x.dim() == 1
+    x2 = _rows_view(x)
+    if x2.dtype != torch.float32:
+        raise ProfkError("topk_noalloc: float32 only")
+    rows, n = x2.shape
+    if out is None:
+        out = (torch.empty((rows, k), dtype=x2.dtype, device=x2.device),
+               torch.empty((rows, k), dtype=torch.int64, device=x2.device))
+    vals, idx = out
+    with torch.cuda.device(x2.device):
+        code = lib().profk_topk_noalloc_f32(ctypes.c_void_p(x2.data_ptr()), ctypes.c_int64(rows), ctypes.c_int64(n),
+                                            ctypes.c_int64(k), ctypes.c_double(eps), ctypes.c_double(recall),
+                                            ctypes.c_uint64(seed), _stream_ptr(), ctypes.c_void_p(vals.data_ptr()),
+                                            ctypes.c_void_p(idx.data_ptr()))
+    _check(code, "profk_topk_noalloc_f32")
+    return (vals[0], idx[0]) if one_d else (vals, idx)
 
 
 def filter_pass(x, tau, capacity: int):

@@ -30,6 +30,8 @@ constexpr int64_t N_MAX = 4278190080LL;          // 2^32 - 2^24
 constexpr int64_t M_MAX = 262144;                // largest sample the cluster select holds (8 CTAs x 32768 keys)
 
 thread_local int g_launches = 0;
+thread_local void* g_ws_override_ptr = nullptr;   // set by the allocation-free entry point for the duration of its call
+thread_local size_t g_ws_override_bytes = 0;
 std::atomic<int> g_coop_pdl{-1};                 // -1 untried, 1 accepted, 0 refused by the runtime
 
 struct DeviceInfo {
@@ -254,7 +256,9 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     if (rc != PROFK_OK) return rc;
 
     Workspace ws;
-    {
+    if (g_ws_override_ptr) {
+        ws = Workspace{g_ws_override_ptr, g_ws_override_bytes};
+    } else {
         std::lock_guard<std::mutex> lock(g_mutex);
         ws = g_workspace[dev];
     }
@@ -479,6 +483,45 @@ int profk_sample_threshold_bf16(const void* in, int64_t rows, int64_t N, int64_t
                                            static_cast<__nv_bfloat16*>(tau), sample_idx, stream);
 }
 
+// ---- allocation-free entry point -------------------------------------------------------------
+// Scratch for profk_topk_noalloc_f32: part of the library image, so every GPU that loads the
+// library holds these 16 MiB until the process exits, whether or not the entry point is used.
+constexpr size_t NOALLOC_SCRATCH_BYTES = (size_t)16 << 20;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_SCRATCH_BYTES];
+
+int profk_topk_noalloc_f32(const float* in, int64_t rows, int64_t N, int64_t k, double eps, double recall, uint64_t seed,
+                           void* stream, float* out_vals, int64_t* out_idx) {
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    // In host code `g_noalloc_scratch` is only a handle of the symbol, not a device address: the
+    // address on the current device comes from the runtime, once per device, and is cached.
+    static std::mutex ptr_mutex;
+    static std::map<int, void*> ptr_by_device;
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(ptr_mutex);
+        auto it = ptr_by_device.find(dev);
+        if (it == ptr_by_device.end()) {
+            void* p = nullptr;
+            CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+            if (!p) return PROFK_ECUDA;
+            it = ptr_by_device.emplace(dev, p).first;
+        }
+        scratch = it->second;
+    }
+    profk_plan_t plan;
+    const int prc = profk_plan(N, k, eps, recall, &plan);
+    if (prc != PROFK_OK) return prc;
+    if (rows < 1 || rows * plan.capacity >= (1LL << 40)) return PROFK_EINVAL;
+    if (ws_layout(rows, plan.capacity, k).total > NOALLOC_SCRATCH_BYTES) return PROFK_ETOOLARGE;
+    g_ws_override_ptr = scratch;
+    g_ws_override_bytes = NOALLOC_SCRATCH_BYTES;
+    const int rc = topk_planned<float>(in, rows, N, k, &plan, seed, stream, out_vals, out_idx);
+    g_ws_override_ptr = nullptr;
+    g_ws_override_bytes = 0;
+    return rc;
+}
+
 int profk_read_stats(void* stream, int64_t rows, profk_row_stats_t* out) {
     if (!out || rows < 1) return PROFK_EINVAL;
     int dev = 0;
@@ -523,6 +566,7 @@ const char* profk_strerror(int code) {
         case PROFK_EWORKSPACE: return "workspace missing or too small";
         case PROFK_ECUDA: return "CUDA runtime error";
         case PROFK_ETIMEOUT: return "device-side wait timed out";
+        case PROFK_ETOOLARGE: return "problem too large for the built-in scratch of the allocation-free entry point";
         default: return "unknown status";
     }
 }
