@@ -203,7 +203,7 @@ def main():
     import torch
 
     import paper_2608_12573_b200 as profk
-    from paper_2608_12573_b200 import _build
+    from paper_2608_12573_b200 import _build, sharding
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -229,10 +229,10 @@ def main():
     copies = max(2, min(8, -(-3 * L2_BYTES // in_bytes)))
     big = rows * n >= (1 << 29)
     if big:        # drawn on the device (seeded); one pinned host copy serves the end-to-end leg
-        dev_inputs = [make_input(cfg, seed_offset=1000 * c + 7919 * rank, device=str(dev)) for c in range(copies)]
+        dev_inputs = [make_input(cfg, seed_offset=1000 * c + sharding.rank_seed_offset(rank), device=str(dev)) for c in range(copies)]
         host_inputs = [dev_inputs[0].cpu().pin_memory()]
     else:
-        host_inputs = [make_input(cfg, seed_offset=1000 * c + 7919 * rank).pin_memory() for c in range(copies)]
+        host_inputs = [make_input(cfg, seed_offset=1000 * c + sharding.rank_seed_offset(rank)).pin_memory() for c in range(copies)]
         dev_inputs = [h.to(dev) for h in host_inputs]
     pl = profk.plan(n, k, eps, recall)
     profk.ensure_workspace(rows, pl.capacity, k, dev)
@@ -270,12 +270,9 @@ def main():
         if rank == 0:
             print(json.dumps({"hot_path_only": True, "ms_per_step": ms_total / steps, "launches_per_step": launches_per_step}))
         return
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
+    ms_total = sharding.max_over_ranks(ms_total, dev)
     ms_per_step = ms_total / steps
-    value = world * rows * n / (ms_per_step * 1e-3)
+    value = sharding.whole_job_rate(rows * n, world, ms_per_step)
 
     # fallback rate observed over a separate run of seeds (statistics read-back synchronises, so not timed)
     n_seeds = (40 if big else 200) if rows == 1 else max(1, 200 // rows)
@@ -302,11 +299,8 @@ def main():
         e2e_step(i)
     ev1.record()
     barrier()
-    t = torch.tensor([ev0.elapsed_time(ev1)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t.item()) / e2e_steps
-    e2e_value = world * rows * n / (e2e_ms * 1e-3)
+    e2e_ms = sharding.max_over_ranks(ev0.elapsed_time(ev1), dev) / e2e_steps
+    e2e_value = sharding.whole_job_rate(rows * n, world, e2e_ms)
 
     if rank != 0:
         if world > 1:
