@@ -42,6 +42,8 @@ template <typename T> struct FilterParams {
     uint64_t tiles_per_row;
     uint64_t total_tiles;
     int use_pdl;             // 1 = launched as a programmatic dependent of the threshold kernel
+    uint32_t* tile_counter;  // zeroed counter that hands out the tiles from dyn_start on (null = fixed stride throughout)
+    uint32_t dyn_start;      // first tile handed out dynamically (a multiple of the grid size)
 };
 
 // not (x < tau) for every lane of a vector, OR-ed: does the vector hold any survivor?
@@ -92,10 +94,9 @@ template <typename T, int THREADS, int UNROLL>
 __device__ __noinline__ uint32_t filter_slow_path(const FilterParams<T>& p, WarpStage* st,
                                                   typename Elem<T>::vec_t v0, typename Elem<T>::vec_t v1,
                                                   typename Elem<T>::vec_t v2, typename Elem<T>::vec_t v3,
-                                                  uint32_t inside_mask, uint32_t row, uint32_t trow, uint32_t mis, T tau) {
+                                                  uint32_t inside_mask, uint32_t row, uint64_t qbase, uint32_t mis, T tau) {
     using V = typename Elem<T>::vec_t;
     constexpr int VEC = Elem<T>::VEC;
-    constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
     static_assert(UNROLL == 4, "the slow path takes four vectors");
     const V v[4] = {v0, v1, v2, v3};
     const unsigned lane = lane_id();
@@ -106,7 +107,7 @@ __device__ __noinline__ uint32_t filter_slow_path(const FilterParams<T>& p, Warp
     for (int u = 0; u < UNROLL; ++u) {
         mine[u] = 0;
         if (((inside_mask >> u) & 1u) && vec_any_pass(v[u], tau)) {      // most vectors hold no survivor
-            const uint64_t q = (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
+            const uint64_t q = qbase + (uint64_t)u * THREADS + threadIdx.x;
             const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
 #pragma unroll
             for (int l = 0; l < VEC; ++l) {
@@ -147,7 +148,7 @@ __device__ __noinline__ uint32_t filter_slow_path(const FilterParams<T>& p, Warp
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) {
         if (mine[u]) {
-            const uint64_t q = (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
+            const uint64_t q = qbase + (uint64_t)u * THREADS + threadIdx.x;
             const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
 #pragma unroll
             for (int l = 0; l < VEC; ++l) {
@@ -174,10 +175,9 @@ __device__ __noinline__ uint32_t filter_slow_path(const FilterParams<T>& p, Warp
 // written straight to the row buffer.  Returns the row if its buffer has overflowed, else ~0.
 template <typename T, int THREADS, int UNROLL>
 __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T>& p, const typename Elem<T>::vec_t (&v)[UNROLL],
-                                                            const bool (&inside)[UNROLL], uint32_t row, uint32_t trow,
+                                                            const bool (&inside)[UNROLL], uint32_t row, uint64_t qbase,
                                                             uint32_t mis, T tau) {
     constexpr int VEC = Elem<T>::VEC;
-    constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
     const unsigned lane = lane_id();
     const float tau_f = Elem<T>::as_float(tau);
     unsigned mine[UNROLL];          // per vector: bit l set = element l survives
@@ -186,7 +186,7 @@ __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T
     for (int u = 0; u < UNROLL; ++u) {
         mine[u] = 0;
         if (inside[u] && vec_any_pass(v[u], tau)) {                      // most vectors hold no survivor
-            const uint64_t q = (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
+            const uint64_t q = qbase + (uint64_t)u * THREADS + threadIdx.x;
             const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
 #pragma unroll
             for (int l = 0; l < VEC; ++l) {
@@ -213,7 +213,7 @@ __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) {
         if (mine[u]) {
-            const uint64_t q = (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x;
+            const uint64_t q = qbase + (uint64_t)u * THREADS + threadIdx.x;
             const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
 #pragma unroll
             for (int l = 0; l < VEC; ++l) {
@@ -229,37 +229,59 @@ __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T
 
 // STAGED = collect survivors in per-warp shared-memory stages (dense survivors, one row at a time);
 // otherwise append them directly (sparse survivors or many short rows).
+//
+// Work distribution: a tile is TILE_VECTORS consecutive vectors of one row (32 KB), loaded by the
+// whole CTA at once (every warp-level load is one contiguous 512-byte run, the CTA's loads one 32 KB
+// run).  A CTA takes tiles blockIdx.x, + gridDim.x, ... with its warps running freely; the last few
+// tiles of the launch (from dyn_start on) come from a global counter instead, so that SMs that saw
+// less bandwidth take fewer of them and all CTAs finish together.  The counter is read one tile
+// ahead, so its round trip hides behind the loads; only this tail needs a CTA barrier per tile.
 template <typename T, int THREADS, int UNROLL, bool STAGED>
 __global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOCKS_F32 : PROFK_FILTER_MINBLOCKS_BF16) filter_kernel(const __grid_constant__ FilterParams<T> p) {
     using V = typename Elem<T>::vec_t;
     constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
     __shared__ WarpStage stages[STAGED ? THREADS / 32 : 1];
+    __shared__ uint32_t s_next[2];
 
+    const unsigned lane = lane_id();
     WarpStage* st = &stages[STAGED ? threadIdx.x >> 5 : 0];
     if (STAGED) {
-        if (lane_id() == 0) { st->fill = 0; st->row = 0; }
+        if (lane == 0) { st->fill = 0; st->row = 0; }
         __syncwarp();
     }
 
-    uint32_t tile = blockIdx.x;                  // the grid never exceeds the number of tiles (< 2^32)
     const uint32_t total_tiles = (uint32_t)p.total_tiles, tiles_per_row = (uint32_t)p.tiles_per_row;
+    uint32_t tile = blockIdx.x;                  // the grid never exceeds the number of tiles (< 2^32)
 
     // Decode the first tile and issue its loads before waiting on the threshold kernel:
     // the input does not depend on it.
     uint32_t row = tile / tiles_per_row;
-    uint32_t trow = tile - row * tiles_per_row;
+    uint64_t qbase = (uint64_t)(tile - row * tiles_per_row) * TILE_VECTORS;
     RowView<T> rv = row_view(p.in, p.N, row);
     V v[UNROLL];
     bool inside[UNROLL];
 #pragma unroll
-    for (int u = 0; u < UNROLL; ++u)
-        v[u] = load_row_vector(rv, p.N, (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x, &inside[u]);
+    for (int u = 0; u < UNROLL; ++u) v[u] = load_row_vector(rv, p.N, qbase + (uint64_t)u * THREADS + threadIdx.x, &inside[u]);
 
+    PROFK_STAMP(0, 10);
     if (p.use_pdl) pdl_wait();
+    pdl_launch_dependents();            // the refine kernel may be staged behind this one
+    PROFK_STAMP(0, 11);
 
     uint32_t skip_row = 0xFFFFFFFFu;    // row whose buffer this warp has seen overflow: nothing more to append
+    uint32_t parity = 0;
+    T tau = p.tau[row];
     while (true) {
-        const T tau = p.tau[row];
+        // Tiles below dyn_start follow the fixed stride and the warps run freely; the last few tiles of
+        // the launch are handed out by the counter.  Thread 0 asks for the next one now; the answer is
+        // needed only after this tile.
+        const bool dynamic = p.tile_counter != nullptr && tile + gridDim.x >= p.dyn_start;
+        uint32_t upcoming = 0;
+        if (dynamic && threadIdx.x == 0) {
+            const uint32_t t = p.dyn_start + atomicAdd(p.tile_counter, 1u);
+            upcoming = t < total_tiles ? t : total_tiles;
+        }
+
         bool hit = false;
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) hit |= (inside[u] && vec_any_pass(v[u], tau));
@@ -270,29 +292,43 @@ __global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOC
                 uint32_t inside_mask = 0;
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u) inside_mask |= inside[u] ? 1u << u : 0u;
-                o = filter_slow_path<T, THREADS, UNROLL>(p, st, v[0], v[1], v[2], v[3], inside_mask, row, trow, rv.mis, tau);
+                o = filter_slow_path<T, THREADS, UNROLL>(p, st, v[0], v[1], v[2], v[3], inside_mask, row, qbase, rv.mis, tau);
             } else {
-                o = filter_slow_path_direct<T, THREADS, UNROLL>(p, v, inside, row, trow, rv.mis, tau);
+                o = filter_slow_path_direct<T, THREADS, UNROLL>(p, v, inside, row, qbase, rv.mis, tau);
             }
             if (o != 0xFFFFFFFFu) skip_row = o;
         }
 
-        // Next tile of this CTA; tiles of a row already known to overflow are not even loaded.
-        uint32_t nrow;
-        bool more = true;
-        do {
-            if (total_tiles - tile <= gridDim.x) { more = false; break; }
-            tile += gridDim.x;
-            nrow = tile / tiles_per_row;
-        } while (nrow == skip_row);
-        if (!more) break;
-        trow = tile - nrow * tiles_per_row;
-        if (nrow != row) { row = nrow; rv = row_view(p.in, p.N, row); }
+        if (dynamic) {
+            if (threadIdx.x == 0) s_next[parity] = upcoming;
+            __syncthreads();
+            tile = s_next[parity];
+            parity ^= 1u;
+        } else {
+            tile = total_tiles - tile <= gridDim.x ? total_tiles : tile + gridDim.x;
+        }
+        if (tile >= total_tiles) break;
+        const uint32_t nrow = tile / tiles_per_row;
+        qbase = (uint64_t)(tile - nrow * tiles_per_row) * TILE_VECTORS;
+        if (nrow != row) { row = nrow; rv = row_view(p.in, p.N, row); tau = p.tau[row]; }
+        if (row == skip_row) {                   // this warp knows the row has overflowed: nothing to load
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u)
-            v[u] = load_row_vector(rv, p.N, (uint64_t)trow * TILE_VECTORS + (uint64_t)u * THREADS + threadIdx.x, &inside[u]);
+            for (int u = 0; u < UNROLL; ++u) inside[u] = false;
+            continue;
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) v[u] = load_row_vector(rv, p.N, qbase + (uint64_t)u * THREADS + threadIdx.x, &inside[u]);
     }
     if (STAGED && st->fill) flush_stage(p, st);
+    PROFK_STAMP(0, 12);
+#ifdef PROFK_TRACE
+    if (threadIdx.x == 0) {
+        unsigned long long gt;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
+        atomicMax((unsigned long long*)&g_profk_trace[2][13], gt);      // latest CTA end
+        atomicMin((unsigned long long*)&g_profk_trace[2][14], gt);      // earliest CTA end
+    }
+#endif
 }
 
 }  // namespace profk

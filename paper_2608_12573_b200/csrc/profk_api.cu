@@ -22,6 +22,9 @@ using namespace profk;
 
 namespace {
 
+#ifndef PROFK_DYNAMIC_ROUNDS
+#define PROFK_DYNAMIC_ROUNDS 2      // tiles per CTA (on average) that the filter hands out dynamically at the end
+#endif
 constexpr int FILTER_THREADS = PROFK_FILTER_THREADS;
 constexpr int FILTER_UNROLL = PROFK_FILTER_UNROLL;
 constexpr uint32_t SORT_CAP_MAX = 8192;          // largest k the single-CTA refine orders in shared memory
@@ -183,7 +186,7 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
 
 template <typename T>
 int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, const T* tau, int64_t capacity, uint64_t* buf,
-                  uint64_t buf_stride, uint32_t* counts, uint32_t count_stride, bool pdl, bool staged, cudaStream_t st) {
+                  uint64_t buf_stride, uint32_t* counts, uint32_t count_stride, bool pdl, bool staged, uint32_t* tile_counter, cudaStream_t st) {
     FilterParams<T> fp;
     fp.in = in; fp.N = (uint64_t)N; fp.rows = (uint64_t)rows; fp.tau = tau; fp.capacity = (uint32_t)capacity;
     fp.buf = buf; fp.buf_stride = buf_stride; fp.counts = counts; fp.count_stride = count_stride;
@@ -191,10 +194,15 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     fp.total_tiles = fp.tiles_per_row * (uint64_t)rows;
     if (fp.total_tiles >= (1ull << 32)) return PROFK_EINVAL;      // rows * N beyond 2^45 elements
     fp.use_pdl = pdl ? 1 : 0;
+    fp.tile_counter = tile_counter;
     const uint64_t max_grid = (uint64_t)di.sm_count *
         (staged ? di.filter_staged_blocks_per_sm[dtype_index<T>()] : di.filter_blocks_per_sm[dtype_index<T>()]);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)std::min<uint64_t>(fp.total_tiles, max_grid));
+    // all but the last ~PROFK_DYNAMIC_ROUNDS tiles per CTA follow the fixed stride
+    const uint64_t rounds = fp.total_tiles / cfg.gridDim.x;
+    fp.dyn_start = (uint32_t)((rounds > PROFK_DYNAMIC_ROUNDS ? rounds - PROFK_DYNAMIC_ROUNDS : 0) * cfg.gridDim.x);
+    if (rounds <= PROFK_DYNAMIC_ROUNDS) fp.tile_counter = nullptr;
     cfg.blockDim = dim3(FILTER_THREADS);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = st;
@@ -286,7 +294,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     if (plan->mode == 0) {
         rc = launch_sample_select<T>(di, in, rows, N, plan->m, plan->r, seed, tau, ctl, header, (uint32_t)capacity, nullptr, st);
         if (rc != PROFK_OK) return rc;
-        rc = launch_filter<T>(di, in, rows, N, tau, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, st);
+        rc = launch_filter<T>(di, in, rows, N, tau, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, &header->tile_counter, st);
         if (rc != PROFK_OK) return rc;
 
         if (large) {
@@ -400,7 +408,7 @@ int filter_only(const T* in, int64_t rows, int64_t N, const T* tau, int64_t capa
     DeviceInfo di;
     const int rc = ensure_device_info<T>(dev, &di);
     if (rc != PROFK_OK) return rc;
-    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, (uint64_t)capacity, counts, 1, false, false, static_cast<cudaStream_t>(stream));
+    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, (uint64_t)capacity, counts, 1, false, false, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 template <typename T>

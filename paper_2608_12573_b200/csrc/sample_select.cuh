@@ -47,8 +47,9 @@ struct WsHeader {
     uint32_t bar_gen;
     uint32_t error;      // non-zero = a bounded wait gave up
     uint32_t done;       // CTAs of the filter kernel that have finished (ticket for its last CTA)
-    uint32_t n_failed;   // rows whose count check failed (written by the filter's last CTA)
-    uint32_t pad[59];
+    uint32_t n_failed;   // rows whose count check failed
+    uint32_t tile_counter;  // hands out the filter kernel's tiles
+    uint32_t pad[58];
 };
 static_assert(sizeof(WsHeader) == 256, "WsHeader is 256 bytes");
 
@@ -131,6 +132,9 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
 
     pdl_launch_dependents();   // the filter kernel may start its prologue now
     PROFK_STAMP(0, 0);
+#ifdef PROFK_TRACE
+    if (threadIdx.x == 0 && blockIdx.x == 0) { g_profk_trace[2][13] = 0; g_profk_trace[2][14] = 0x7FFFFFFFFFFFFFFFll; }
+#endif
 
     if (tid == 0) { s_ncand = 0; s_lower = 0; }
     __syncthreads();
@@ -190,7 +194,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
             RowCtl* c = p.ctl + row;
             c->count = 0; c->collect = 0; c->status = 0; c->n_final = 0; c->capacity = p.capacity;
         }
-        if (p.header && row == 0) { p.header->bar_count = 0; p.header->error = 0; p.header->done = 0; p.header->n_failed = 0; }
+        if (p.header && row == 0) { p.header->bar_count = 0; p.header->error = 0; p.header->done = 0; p.header->n_failed = 0; p.header->tile_counter = 0; }
     }
     PROFK_STAMP(0, 1);
 
