@@ -5,7 +5,7 @@
 // refinement is "the k smallest records, sorted".  One CTA per row.  The CTA first takes the
 // paper's check -- fewer than k candidates, or more than the buffer holds, means the row is
 // left to the exact-selection kernel that follows.  Otherwise the records (held in registers
-// when they fit) are binned by their key's distance above tau into 4096 bins; a scan of the
+// when they fit) are binned by their key's distance above tau into 4096 logarithmic bins; a scan of the
 // bin counts gives every bin its first output position and finds the bin that holds the k-th
 // best record; the records of that bin and of all better bins are grouped by bin in shared
 // memory, and each of them finds its final position by ranking itself inside its (small) bin.
@@ -83,11 +83,11 @@ __device__ __forceinline__ void bitonic_sort_shared(uint64_t* a, uint32_t P) {
 
 // Shared state of one select.
 struct SelectShared {
-    uint32_t hist[RF_BINS];          // bin counts, then running cursors
-    uint32_t start[RF_BINS];         // first position of every bin
+    alignas(16) uint32_t hist[RF_BINS];   // bin counts, then running cursors
+    alignas(16) uint32_t start[RF_BINS];  // first position of every bin
     uint64_t edge[RF_EDGE_CAP];      // records of the boundary bin (general select only)
     uint32_t warp_sums[32];
-    uint32_t digit, before, cnt, fill, n_edge, crowded, dmax;
+    uint32_t digit, before, cnt, fill, n_edge, crowded;
     unsigned long long or_bits, limit;
 };
 
@@ -242,12 +242,22 @@ __global__ void __launch_bounds__(1024) refine_kernel(const RefineParams<T> p) {
 
     const unsigned tid = threadIdx.x, nthr = blockDim.x, lane = lane_id();
     const uint64_t row = blockIdx.x;
-    if (tid == 0) { sh.or_bits = 0ull; sh.fill = 0; sh.n_edge = 0; sh.crowded = 0; sh.dmax = 0; }
+    if (tid == 0) { sh.or_bits = 0ull; sh.fill = 0; sh.n_edge = 0; sh.crowded = 0; }
     for (uint32_t i = tid; i < RF_BINS; i += nthr) sh.hist[i] = 0;
     __syncthreads();
     pdl_launch_dependents();                 // the exact-selection kernel may be staged behind this one
     if (p.use_pdl) pdl_wait();
     PROFK_STAMP(1, 0);
+
+    // The first batch of records (8 per thread, kept in registers) is requested at once, together with
+    // the row's control block: which of them are real is known when the survivor count arrives.
+    const uint64_t* src = p.buf + row * p.buf_stride;
+    uint64_t r[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const uint32_t i = u * nthr + tid;
+        r[u] = i < p.capacity ? src[i] : ~0ull;
+    }
 
     // ---- the count check of stage 4 ----
     const RowCtl ctl = p.ctl[row];
@@ -262,16 +272,17 @@ __global__ void __launch_bounds__(1024) refine_kernel(const RefineParams<T> p) {
 
     const uint32_t n = R;
     const uint32_t kk = n < p.k ? n : p.k;          // real outputs; the rest is padding (relaxed mode)
-    const uint64_t* src = p.buf + row * p.buf_stride;
     for (uint32_t j = kk + tid; j < p.k; j += nthr) {       // relaxed mode: padding after a short buffer
         p.out_vals[row * (uint64_t)p.k + j] = Elem<T>::from_bits(Elem<T>::NEG_INF_BITS);
         p.out_idx[row * (uint64_t)p.k + j] = -1;
     }
 
-    // ---- bin the records by the distance of their key above tau (bin 0 = largest keys) ----
+    // ---- bin the records by the distance d of their key above tau, on a logarithmic scale: the bin is
+    //      the exponent and the top seven mantissa bits of d as a float (monotone in d, 32 x 128 = 4096
+    //      bins, fine where the records are dense -- just above tau -- and coarse where they are rare).
+    //      Bin 0 holds the largest keys. ----
     const uint32_t tau_key = Elem<T>::key(Elem<T>::from_bits(ctl.tau_bits));
-    const uint32_t nbatch = (n + 8 * nthr - 1) / (8 * nthr);   // one batch = 8 records per thread, kept in registers
-    uint64_t r[8];
+    const uint32_t nbatch = (n + 8 * nthr - 1) / (8 * nthr);   // one batch = 8 records per thread
     auto load_batch = [&](uint32_t b) {
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
@@ -280,33 +291,17 @@ __global__ void __launch_bounds__(1024) refine_kernel(const RefineParams<T> p) {
         }
     };
     auto valid = [&](uint32_t b, int u) { return (b * 8 + u) * nthr + tid < n; };
-    auto dist = [&](uint64_t rec) { const uint32_t key = record_key(rec); return key > tau_key ? key - tau_key : 0u; };
-
-    uint32_t dmax = 0;
-    for (uint32_t b = 0; b < nbatch; ++b) {
-        load_batch(b);
-#pragma unroll
-        for (int u = 0; u < 8; ++u)
-            if (valid(b, u)) dmax = max(dmax, dist(r[u]));
-    }
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) dmax = max(dmax, __shfl_xor_sync(FULL_MASK, dmax, d));
-    if (lane == 0) sh.warp_sums[tid >> 5] = dmax;
-    __syncthreads();
-    if (tid < 32) {
-        uint32_t w = tid < (nthr >> 5) ? sh.warp_sums[tid] : 0;
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) w = max(w, __shfl_xor_sync(FULL_MASK, w, d));
-        if (tid == 0) sh.dmax = w;
-    }
-    __syncthreads();
-    const int dbits = 32 - __clz(sh.dmax);                             // dmax < 2^dbits
-    const int shift = dbits > RF_BITS ? dbits - RF_BITS : 0;
-    auto bin_of = [&](uint64_t rec) { return (uint32_t)(RF_BINS - 1) - (dist(rec) >> shift); };
+    auto bin_of = [&](uint64_t rec) {
+        const uint32_t key = record_key(rec);
+        const uint32_t d = key > tau_key ? key - tau_key : 0u;
+        const uint32_t f = __float_as_uint((float)d);           // 0 for d = 0, exponent >= 127 otherwise
+        const uint32_t level = f > (127u << 23) ? (f >> 16) - (127u << 7) : 0u;     // 0 .. 4095
+        return (uint32_t)(RF_BINS - 1) - level;
+    };
     PROFK_STAMP(1, 1);
 
     for (uint32_t b = 0; b < nbatch; ++b) {
-        if (nbatch > 1) load_batch(b);
+        if (b > 0) load_batch(b);
 #pragma unroll
         for (int u = 0; u < 8; ++u)
             if (valid(b, u)) atomicAdd(&sh.hist[bin_of(r[u])], 1u);
@@ -314,7 +309,36 @@ __global__ void __launch_bounds__(1024) refine_kernel(const RefineParams<T> p) {
     __syncthreads();
 
     // ---- scan the bin counts: first position of every bin, and the bin of the kk-th best record ----
-    {
+    if (nthr * 4 == RF_BINS) {
+        // four bins per thread, read and written as one 16-byte vector; two barriers in all
+        const uint4 c = reinterpret_cast<const uint4*>(sh.hist)[tid];
+        const uint32_t sum = c.x + c.y + c.z + c.w;
+        uint32_t incl = sum;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t v = __shfl_up_sync(FULL_MASK, incl, d);
+            if (lane >= (unsigned)d) incl += v;
+        }
+        if (lane == 31) sh.warp_sums[tid >> 5] = incl;
+        __syncthreads();
+        uint32_t w = sh.warp_sums[lane];                       // every warp scans the 32 warp totals itself
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t v = __shfl_up_sync(FULL_MASK, w, d);
+            if (lane >= (unsigned)d) w += v;
+        }
+        const uint32_t warp_before = __shfl_sync(FULL_MASK, w, (tid >> 5) ? (tid >> 5) - 1 : 0);
+        const uint32_t b0 = incl - sum + ((tid >> 5) ? warp_before : 0u);
+        const uint32_t b1 = b0 + c.x, b2 = b1 + c.y, b3 = b2 + c.z;
+        const uint32_t before[4] = {b0, b1, b2, b3}, cnt[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (before[j] < kk && kk <= before[j] + cnt[j]) { sh.digit = tid * 4 + j; sh.before = before[j]; sh.cnt = cnt[j]; }
+            if (before[j] < kk && cnt[j] > RF_EDGE_CAP) sh.crowded = 1;
+        }
+        reinterpret_cast<uint4*>(sh.start)[tid] = make_uint4(b0, b1, b2, b3);
+        reinterpret_cast<uint4*>(sh.hist)[tid] = make_uint4(b0, b1, b2, b3);     // the bins' write cursors
+    } else {
         const uint32_t per = (RF_BINS + nthr - 1) / nthr;
         uint32_t sum = 0;
         for (uint32_t j = 0; j < per; ++j) {
