@@ -1,14 +1,16 @@
-// Count check and exact replacement (Section 3, "Refinement": "if fewer than k candidates
-// are collected, or if the buffer overflows ..., falls back to an exact top-k computation
-// on the full input").  The decision is taken on the device: the refine kernel checks every
-// row's survivor count and leaves the rows that failed to this kernel, which returns at once
-// when there are none.  For each failed row it selects the exact top-k of the whole row into
-// the row's candidate buffer, orders it and writes the row's output.
+// Exact replacement of failed rows by the whole grid (Section 3, "Refinement": "if fewer than k
+// candidates are collected, or if the buffer overflows ..., falls back to an exact top-k
+// computation on the full input"), for the calls whose refine kernel does not do it itself:
+// many rows, where one cluster per row would be mostly idle CTAs, and large selections.  The
+// decision is taken on the device: the refine kernel checks every row's survivor count and
+// leaves the rows that failed to this kernel, which returns at once when there are none.  For
+// each failed row it selects the exact top-k of the whole row into the row's candidate buffer
+// and, for selections small enough, orders it and writes the row's output.
 //
-// The exact selection is a most-significant-digit radix select over 64-bit candidate
-// records (value key, then index), 11 bits per pass, run by the whole grid with a grid
-// barrier after each pass.  The kernel is launched cooperatively so that all CTAs are
-// co-resident; every wait is bounded and reports through the workspace header.
+// The exact selection is a most-significant-digit radix select over 64-bit candidate records
+// (value key, then index), 11 bits per pass, run by the whole grid with a grid barrier after
+// each pass.  The kernel is launched cooperatively so that all CTAs are co-resident; every
+// wait is bounded and reports through the workspace header.
 #pragma once
 
 #include "refine.cuh"

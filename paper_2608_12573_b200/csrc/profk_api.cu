@@ -28,6 +28,9 @@ namespace {
 constexpr int FILTER_THREADS = PROFK_FILTER_THREADS;
 constexpr int FILTER_UNROLL = PROFK_FILTER_UNROLL;
 constexpr uint32_t SORT_CAP_MAX = 8192;          // largest k the single-CTA refine orders in shared memory
+constexpr int64_t XS_MAX_ROWS = 18;              // most rows for which the refine kernel itself replaces failed rows
+constexpr unsigned XS_MAX_SEGMENTS = 32;         // most (row, segment) pairs of that exact selection
+constexpr unsigned REFINE_CLUSTER_THREADS = 512;   // fewest threads of a refine CTA that may have to read whole rows
 constexpr size_t REFINE_SMEM_MAX = 160 * 1024;   // dynamic shared memory the refine kernel may ask for (it has ~41 KB static)
 constexpr int64_t N_MAX = 4278190080LL;          // 2^32 - 2^24
 constexpr int64_t M_MAX = 262144;                // largest sample the cluster select holds (8 CTAs x 32768 keys)
@@ -44,6 +47,7 @@ struct DeviceInfo {
     int fallback_blocks_per_sm[2] = {0, 0};
     int max_cluster[2] = {8, 8};              // 16 when the device can co-schedule 16 CTAs of the threshold kernel
     int large_cluster[2] = {8, 8};            // same for the cluster sort (128 KB of shared memory per CTA)
+    int refine_cluster[2] = {8, 8};           // same for the refine kernel at its largest footprint
     bool ready = false;
 };
 
@@ -57,7 +61,7 @@ std::map<std::tuple<int64_t, int64_t, double, double>, profk_plan_t> g_plan_cach
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-    size_t off_header, off_ghist, off_ctl, off_tau, off_bins, off_buf, total;
+    size_t off_header, off_ghist, off_ctl, off_tau, off_bins, off_xs_counters, off_xs_records, off_buf, total;
 };
 
 // Records reserved per row: the capacity itself, or -- when k is too large for the single-CTA
@@ -77,7 +81,12 @@ WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k) {
     l.off_tau = align_up(l.off_ctl + (size_t)rows * sizeof(RowCtl), 256);
     l.off_bins = align_up(l.off_tau + (size_t)rows * 4, 256);
     const size_t bins_bytes = k > (int64_t)SORT_CAP_MAX ? (size_t)rows * (LG_BINS + 8) * sizeof(uint32_t) : 0;
-    l.off_buf = align_up(l.off_bins + bins_bytes, 256);
+    // scratch of the in-refine exact selection (few rows, k within the single-CTA refine): up to
+    // XS_MAX_SEGMENTS segments in all, each with a counter and k + XS_EDGE records
+    const bool xs = rows <= XS_MAX_ROWS && k <= (int64_t)SORT_CAP_MAX;
+    l.off_xs_counters = align_up(l.off_bins + bins_bytes, 256);
+    l.off_xs_records = align_up(l.off_xs_counters + (xs ? XS_MAX_SEGMENTS * sizeof(uint32_t) : 0), 256);
+    l.off_buf = align_up(l.off_xs_records + (xs ? (size_t)XS_MAX_SEGMENTS * (size_t)(k + XS_EDGE) * sizeof(uint64_t) : 0), 256);
     l.total = align_up(l.off_buf + (size_t)rows * (size_t)row_stride_for(capacity, k) * sizeof(uint64_t), 256);
     return l;
 }
@@ -109,7 +118,8 @@ template <typename T> int ensure_device_info(int dev, DeviceInfo* out) {
         CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fallback_kernel<T>, FB_THREADS, 0));
         di.fallback_blocks_per_sm[d] = std::max(nb, 1);
         CUDA_TRY(cudaFuncSetAttribute(sample_select_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
-        CUDA_TRY(cudaFuncSetAttribute(refine_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFINE_SMEM_MAX));
+        CUDA_TRY(cudaFuncSetAttribute(refine_kernel<T, 48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFINE_SMEM_MAX));
+        CUDA_TRY(cudaFuncSetAttribute(refine_kernel<T, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFINE_SMEM_MAX));
         CUDA_TRY(cudaFuncSetAttribute(fallback_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SORT_CAP_MAX * 8)));
         // Clusters of 16 are beyond the portable size: allowed only where one actually fits.
         if (cudaFuncSetAttribute(sample_select_kernel<T>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
@@ -122,6 +132,19 @@ template <typename T> int ensure_device_info(int dev, DeviceInfo* out) {
             int nclusters = 0;
             if (cudaOccupancyMaxActiveClusters(&nclusters, sample_select_kernel<T>, &cfg) == cudaSuccess && nclusters >= 1)
                 di.max_cluster[d] = 16;
+        }
+        (void)cudaGetLastError();
+        if (cudaFuncSetAttribute(refine_kernel<T, 48>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+            cudaFuncSetAttribute(refine_kernel<T, 64>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(16); cfg.blockDim = dim3(1024); cfg.dynamicSmemBytes = REFINE_SMEM_MAX;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 16; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr; cfg.numAttrs = 1;
+            int nclusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&nclusters, refine_kernel<T, 64>, &cfg) == cudaSuccess && nclusters >= 1)
+                di.refine_cluster[d] = 16;
         }
         (void)cudaGetLastError();
         CUDA_TRY(cudaFuncSetAttribute(refine_large_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(BT_TILE * 8)));
@@ -178,7 +201,9 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
+    // Without a cluster dimension a kernel runs as implicit clusters of one CTA, which is what a
+    // one-CTA cluster is -- and a plain grid of many CTAs launches much faster than as many clusters.
+    cfg.attrs = attr; cfg.numAttrs = csize > 1 ? 1 : 0;
     CUDA_TRY(cudaLaunchKernelEx(&cfg, sample_select_kernel<T>, sp));
     ++g_launches;
     return PROFK_OK;
@@ -242,6 +267,71 @@ int launch_refine_large(const DeviceInfo& di, RowCtl* ctl, WsHeader* header, uin
     return PROFK_OK;
 }
 
+// Who replaces a row that fails the count check.  With few rows each row gets a cluster of CTAs in
+// the refine kernel, large enough to read a whole row at a good rate, and the call ends with that
+// kernel.  With many rows a cluster per row would be mostly idle CTAs, and a single CTA is too slow a
+// reader when failures are not rare (many rows, loose eps): the rows are left to a grid-wide
+// cooperative kernel that follows, whose launch is a few microseconds in a call that is long anyway.
+template <typename T> int refine_cluster_size(const DeviceInfo& di, int64_t rows, int64_t N) {
+    int csize = rows <= 9 ? 16 : rows <= XS_MAX_ROWS ? 8 : 1;
+    csize = std::min(csize, di.refine_cluster[dtype_index<T>()]);
+    const int64_t tile_elems = (int64_t)1024 * XS_UNROLL * Elem<T>::VEC;      // the largest tile a CTA may have
+    while (csize > 1 && (int64_t)csize * tile_elems > N) csize /= 2;       // no more CTAs than tiles of the row
+    return csize;
+}
+
+// Count check + refine, one cluster of `csize` CTAs per row (see refine_cluster_size).
+template <typename T>
+int launch_refine(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, RowCtl* ctl, WsHeader* header, uint64_t* buf,
+                  uint64_t row_stride, int64_t capacity, int64_t k, int64_t k_accept, bool direct, int csize, uint64_t* xs_records,
+                  uint32_t* xs_counters, T* out_vals, int64_t* out_idx, cudaStream_t st) {
+    uint32_t sort_cap = 32;
+    while (sort_cap < (uint32_t)k && sort_cap < SORT_CAP_MAX) sort_cap <<= 1;
+    RefineParams<T> rp;
+    rp.in = in; rp.N = (uint64_t)N;
+    rp.ctl = ctl; rp.header = header; rp.buf = buf; rp.buf_stride = row_stride; rp.capacity = (uint32_t)capacity; rp.k = (uint32_t)k;
+    rp.k_accept = (uint32_t)k_accept;
+    rp.sort_cap = sort_cap;
+    rp.stage_cap = 0;            // the general select (crowded bins only) reads the buffer in place
+    rp.out_vals = out_vals; rp.out_idx = out_idx;
+    rp.use_pdl = direct ? 0 : 1;
+    rp.direct = direct ? 1 : 0;
+    rp.cluster_size = (uint32_t)csize;
+    unsigned threads = csize > 1 ? REFINE_CLUSTER_THREADS : 128;      // a cluster may have to read whole rows
+    while (threads < 1024 && threads * 8 < (unsigned)capacity) threads <<= 1;
+    // A failed row is cut into segments, one cluster each, so that all SMs read it: as many clusters per
+    // row as the SMs hold at once, but no more than the row has tiles for.
+    int64_t nseg = 1;
+    if (csize > 1) {
+        const int64_t tiles = (int64_t)tiles_per_row<T>((uint64_t)N, threads * XS_UNROLL);
+        nseg = std::max<int64_t>(1, std::min<int64_t>({di.sm_count / (rows * csize), tiles / csize, (int64_t)XS_MAX_SEGMENTS / rows}));
+    }
+    rp.clusters_per_row = (uint32_t)nseg;
+    rp.xs_records = xs_records; rp.xs_counters = xs_counters;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(rows * nseg * csize));
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = ((size_t)sort_cap + RF_EDGE_CAP + rp.stage_cap) * 8;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    unsigned na = 0;
+    if (csize > 1) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = (unsigned)csize; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    if (!direct) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    cfg.attrs = attr; cfg.numAttrs = na;
+    if (threads <= 512) CUDA_TRY(cudaLaunchKernelEx(&cfg, refine_kernel<T, 48>, rp));
+    else CUDA_TRY(cudaLaunchKernelEx(&cfg, refine_kernel<T, 64>, rp));
+    ++g_launches;
+    return PROFK_OK;
+}
+
 template <typename T>
 int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_plan_t* plan, uint64_t seed, void* stream,
                  T* out_vals, int64_t* out_idx) {
@@ -281,15 +371,19 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     T* tau = reinterpret_cast<T*>(base + lay.off_tau);
     uint64_t* buf = reinterpret_cast<uint64_t*>(base + lay.off_buf);
     uint32_t* bins = reinterpret_cast<uint32_t*>(base + lay.off_bins);
+    uint32_t* xs_counters = reinterpret_cast<uint32_t*>(base + lay.off_xs_counters);
+    uint64_t* xs_records = reinterpret_cast<uint64_t*>(base + lay.off_xs_records);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-
-    uint32_t sort_cap = 32;
-    while (sort_cap < (uint32_t)k && sort_cap < SORT_CAP_MAX) sort_cap <<= 1;
 
     // Survivors are staged per warp when a warp's tile is expected to hold a good fraction of one
     // (expected survivors per element ~ r / m); sparse survivors are appended directly.
     const double per_warp_tile = (double)plan->r / (double)std::max<int64_t>(plan->m, 1) * 32.0 * FILTER_UNROLL * Elem<T>::VEC;
     const bool staged = plan->mode == 0 && rows == 1 && per_warp_tile > 0.1;
+
+    const int csize = (large || rows > XS_MAX_ROWS) ? 1 : refine_cluster_size<T>(di, rows, N);
+    const bool exact_in_refine = csize > 1;
+    uint32_t fb_sort_cap = 32;
+    while (fb_sort_cap < (uint32_t)k && fb_sort_cap < SORT_CAP_MAX) fb_sort_cap <<= 1;
 
     if (plan->mode == 0) {
         rc = launch_sample_select<T>(di, in, rows, N, plan->m, plan->r, seed, tau, ctl, header, (uint32_t)capacity, nullptr, st);
@@ -299,36 +393,23 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
 
         if (large) {
             rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, rows, capacity, k, plan->k_accept, 0, out_vals, out_idx, st);
-            if (rc != PROFK_OK) return rc;
         } else {
-        // refine: count check, then order the buffer of every row that passed it
-        RefineParams<T> rp;
-        rp.ctl = ctl; rp.header = header; rp.buf = buf; rp.buf_stride = row_stride; rp.capacity = (uint32_t)capacity; rp.k = (uint32_t)k;
-        rp.k_accept = (uint32_t)plan->k_accept;
-        rp.sort_cap = sort_cap;
-        rp.stage_cap = 0;            // the general select (crowded bins only) reads the buffer in place
-        rp.out_vals = out_vals; rp.out_idx = out_idx; rp.use_pdl = 1;
-        unsigned threads = 128;
-        while (threads < 1024 && threads * 8 < (unsigned)capacity) threads <<= 1;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)rows);
-        cfg.blockDim = dim3(threads);
-        cfg.dynamicSmemBytes = ((size_t)sort_cap + RF_EDGE_CAP + rp.stage_cap) * 8;
-        cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        CUDA_TRY(cudaLaunchKernelEx(&cfg, refine_kernel<T>, rp));
-        ++g_launches;
+            // count check and refine; with clusters, also the exact selection of the rows that fail the check
+            rc = launch_refine<T>(di, in, rows, N, ctl, header, buf, row_stride, capacity, k, plan->k_accept, false, csize, xs_records, xs_counters, out_vals, out_idx, st);
         }
+        if (rc != PROFK_OK) return rc;
     } else {
         init_ctl_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(ctl, (uint64_t)rows, header, (uint32_t)capacity, (uint32_t)k);
         CUDA_TRY(cudaGetLastError());
         ++g_launches;
+        if (exact_in_refine)
+            return launch_refine<T>(di, in, rows, N, ctl, header, buf, row_stride, capacity, k, k, true, csize, xs_records, xs_counters, out_vals, out_idx, st);
     }
 
-    {   // exact selection, ordering and output of the rows that failed the check (cooperative: all CTAs co-resident)
+    if (!exact_in_refine) {
+        // Exact selection of the rows that failed the check (or, in direct mode, of all rows) by a grid-wide
+        // cooperative kernel: all CTAs co-resident.  For large selections it runs between the two phases
+        // of the cluster refine.
         FallbackParams<T> fb;
         fb.in = in; fb.N = (uint64_t)N; fb.rows = (uint64_t)rows; fb.k = (uint32_t)k;
         fb.capacity = (uint32_t)capacity; fb.ctl = ctl; fb.header = header; fb.ghist = ghist; fb.buf = buf;
@@ -337,9 +418,9 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         fb.use_pdl = 0;
         fb.out_vals = out_vals; fb.out_idx = out_idx;
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)di.sm_count);       // one CTA per SM: cheap to launch when no row failed
+        cfg.gridDim = dim3((unsigned)di.sm_count);
         cfg.blockDim = dim3(FB_THREADS);
-        cfg.dynamicSmemBytes = large ? 0 : (size_t)sort_cap * 8;
+        cfg.dynamicSmemBytes = large ? 0 : (size_t)fb_sort_cap * 8;
         cfg.stream = st;
         cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeCooperative;
@@ -348,7 +429,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         // A cooperative launch that is also a programmatic dependent hides its launch latency behind
-        // the refine kernel; if the runtime refuses the combination, launch it as a plain cooperative kernel.
+        // the kernel before it; if the runtime refuses the combination, launch it as a plain cooperative kernel.
         int pdl_state = g_coop_pdl.load();
         bool launched = false;
         if (plan->mode == 0 && pdl_state != 0) {

@@ -2,28 +2,30 @@
 // buffer, written out in the order "value descending, index ascending".
 //
 // Candidate records are 64-bit integers whose ascending order is exactly that order, so
-// refinement is "the k smallest records, sorted".  One CTA per row.  The CTA first takes the
-// paper's check -- fewer than k candidates, or more than the buffer holds, means the row is
-// left to the exact-selection kernel that follows.  Otherwise the records (held in registers
-// when they fit) are binned by their key's distance above tau into 4096 logarithmic bins; a scan of the
-// bin counts gives every bin its first output position and finds the bin that holds the k-th
-// best record; the records of that bin and of all better bins are grouped by bin in shared
-// memory, and each of them finds its final position by ranking itself inside its (small) bin.
-// No sort is needed.  When a bin is too crowded for that (many equal values) a
+// refinement is "the k smallest records, sorted".  One thread-block cluster per row; its first
+// CTA does the refinement proper.  Every CTA first takes the paper's check -- fewer than k
+// candidates, or more than the buffer holds, means the row is replaced by an exact top-k of the
+// full input, which the whole cluster computes (exact_select.cuh); when the check passes, as it
+// almost always does, the other CTAs leave at once.  The first CTA then bins the records (held
+// in registers when they fit) by their key's distance above tau into 4096 logarithmic bins; a
+// scan of the bin counts gives every bin its first output position and finds the bin that holds
+// the k-th best record; the records of that bin and of all better bins are grouped by bin in
+// shared memory, and each of them finds its final position by ranking itself inside its (small)
+// bin.  No sort is needed.  When a bin is too crowded for that (many equal values) a
 // most-significant-digit radix select plus a bitonic sort does the same job.
+//
+// In direct mode (a row too short for sampling to pay) there is no threshold and no buffer to
+// refine: every row goes straight to the exact selection.
 #pragma once
 
-#include "sample_select.cuh"
+#include "exact_select.cuh"
+#include "select_sort.cuh"
 
 namespace profk {
 
-constexpr int RF_BITS = 12;                 // digit width of the general select
-constexpr int RF_BINS = 1 << RF_BITS;
-constexpr uint32_t RF_EDGE_CAP = 1024;      // boundary bins up to this size are ranked directly
-
-enum : uint32_t { ROW_OK = 0, ROW_RECALL = 1, ROW_OVERFLOW = 2, ROW_DIRECT = 3 };
-
 template <typename T> struct RefineParams {
+    const T* in;             // rows x N input (read only by the exact selection)
+    uint64_t N;
     RowCtl* ctl;
     WsHeader* header;
     const uint64_t* buf;     // row r's records start at buf + r * buf_stride
@@ -36,216 +38,96 @@ template <typename T> struct RefineParams {
     T* out_vals;             // rows x k
     int64_t* out_idx;        // rows x k
     int use_pdl;
+    int direct;              // 1 = no threshold / filter ran: every row is selected exactly
+    uint32_t cluster_size;   // CTAs per cluster; 1 = launched without a cluster dimension, and rows that fail the
+                             // check are left to the exact-selection kernel that follows
+    uint32_t clusters_per_row;   // segments a failed row is cut into for its exact selection, one cluster each
+    uint64_t* xs_records;    // rows x clusters_per_row x (k + XS_EDGE) records selected from the segments
+    uint32_t* xs_counters;   // rows x clusters_per_row append counters
 };
 
-__device__ __forceinline__ uint64_t shr64(uint64_t x, int s) { return s >= 64 ? 0ull : (x >> s); }
-
-// Block-wide inclusive scan for any block size that is a multiple of 32 (<= 1024).
-__device__ __forceinline__ uint32_t block_scan_any(uint32_t v, uint32_t* warp_sums) {
-    const unsigned lane = lane_id(), warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t n = __shfl_up_sync(FULL_MASK, v, d);
-        if (lane >= (unsigned)d) v += n;
-    }
-    if (lane == 31) warp_sums[warp] = v;
-    __syncthreads();
-    if (warp == 0) {
-        uint32_t w = lane < nwarps ? warp_sums[lane] : 0;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t n = __shfl_up_sync(FULL_MASK, w, d);
-            if (lane >= (unsigned)d) w += n;
-        }
-        warp_sums[lane] = w;
-    }
-    __syncthreads();
-    if (warp > 0) v += warp_sums[warp - 1];
-    __syncthreads();   // warp_sums may be reused right away
-    return v;
-}
-
-// Ascending bitonic sort of P = 2^j records in shared memory by the whole CTA.
-__device__ __forceinline__ void bitonic_sort_shared(uint64_t* a, uint32_t P) {
-    for (uint32_t size = 2; size <= P; size <<= 1) {
-        for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
-            for (uint32_t i = threadIdx.x; i < (P >> 1); i += blockDim.x) {
-                const uint32_t lo = 2 * i - (i & (stride - 1));
-                const uint32_t hi = lo + stride;
-                const bool ascending = (lo & size) == 0;
-                const uint64_t x = a[lo], y = a[hi];
-                if ((x > y) == ascending) { a[lo] = y; a[hi] = x; }
-            }
-            __syncthreads();
-        }
-    }
-}
-
-// Shared state of one select.
-struct SelectShared {
-    alignas(16) uint32_t hist[RF_BINS];   // bin counts, then running cursors
-    alignas(16) uint32_t start[RF_BINS];  // first position of every bin
-    uint64_t edge[RF_EDGE_CAP];      // records of the boundary bin (general select only)
-    uint32_t warp_sums[32];
-    uint32_t digit, before, cnt, fill, n_edge, crowded;
-    unsigned long long or_bits, limit;
-};
-
-// Records read from memory (shared or global): every thread visits whole-warp rounds.
-struct MemRecords {
+// Records selected from the segments of a row, read through L2 (other clusters wrote them); unused
+// slots hold all-ones.
+struct SegmentRecords {
     const uint64_t* recs;
     uint32_t n;
     template <typename F> __device__ __forceinline__ void for_each(F&& f) const {
         const uint32_t n_round = (n + 31u) & ~31u;
-        for (uint32_t i = threadIdx.x; i < n_round; i += blockDim.x) f(i < n ? recs[i] : 0ull, i < n);
+        for (uint32_t i = threadIdx.x; i < n_round; i += blockDim.x) {
+            const uint64_t rec = i < n ? __ldcg(&recs[i]) : ~0ull;
+            f(rec, rec != ~0ull);
+        }
     }
 };
 
-// General select: finds limit = the need-th smallest record (records are distinct) by radix
-// passes and compacts the records <= limit into sortbuf.  sh.or_bits = OR over (record XOR
-// first); sh.fill and sh.n_edge must be zero.  All threads call it.
-template <typename Src>
-__device__ __forceinline__ void select_smallest(const Src& src, uint64_t first, uint32_t need, uint64_t* sortbuf,
-                                                uint32_t sort_cap, SelectShared& sh) {
+// The exact top-k of the full row, for a row that failed the count check (Section 3, "Refinement").
+// Cluster `seg` of the row's clusters selects the k smallest records (and a few more) of its segment of
+// the row; the cluster that finishes last merges: the k smallest of all segments' records, ordered, are
+// the row's output.  The ticket is the row's `collect` word, zero on entry and zero again on exit.
+template <typename T>
+__device__ __noinline__ void exact_row(const RefineParams<T>& p, uint64_t row, unsigned seg, unsigned crank, uint64_t* sortbuf,
+                                          SelectShared& sh) {
     const unsigned tid = threadIdx.x, nthr = blockDim.x, lane = lane_id();
-    const int top = 64 - __clzll((long long)sh.or_bits);       // bits >= top are common to all records
-    uint64_t prefix = shr64(first, top);
-    uint64_t limit = ~0ull;
-    for (int done = 0; done < top;) {
-        const int shift = top - done - RF_BITS > 0 ? top - done - RF_BITS : 0;
-        const int width = top - done - shift;
-        const uint32_t nbins = 1u << width;
-        for (uint32_t i = tid; i < nbins; i += nthr) sh.hist[i] = 0;
-        __syncthreads();
-        src.for_each([&](uint64_t rec, bool valid) {
-            if (valid && shr64(rec, shift + width) == prefix) atomicAdd(&sh.hist[(uint32_t)(rec >> shift) & (nbins - 1)], 1u);
-        });
-        __syncthreads();
-        const uint32_t per = (RF_BINS + nthr - 1) / nthr;
-        uint32_t sum = 0;
-        for (uint32_t j = 0; j < per; ++j) {
-            const uint32_t bin = tid * per + j;
-            sum += bin < nbins ? sh.hist[bin] : 0;
-        }
-        uint32_t before = block_scan_any(sum, sh.warp_sums) - sum;
-        for (uint32_t j = 0; j < per; ++j) {
-            const uint32_t bin = tid * per + j;
-            const uint32_t c = bin < nbins ? sh.hist[bin] : 0;
-            if (before < need && need <= before + c) { sh.digit = bin; sh.before = before; sh.cnt = c; }
-            before += c;
-        }
-        __syncthreads();
-        prefix = (prefix << width) | sh.digit;
-        need -= sh.before;
-        const uint32_t in_bin = sh.cnt;
-        done += width;
-        __syncthreads();
-        if (in_bin == need || done >= top) { limit = ((prefix + 1) << shift) - 1; break; }
-        if (in_bin <= RF_EDGE_CAP) {
-            // collect the boundary bin and rank its records: the need-th smallest is the limit
-            src.for_each([&](uint64_t rec, bool valid) {
-                if (valid && shr64(rec, shift) == prefix) {
-                    const uint32_t pos = atomicAdd(&sh.n_edge, 1u);
-                    if (pos < RF_EDGE_CAP) sh.edge[pos] = rec;
-                }
-            });
-            __syncthreads();
-            for (uint32_t i = tid; i < in_bin; i += nthr) {
-                const uint64_t mine = sh.edge[i];
-                uint32_t rank = 0;
-                for (uint32_t j = 0; j < in_bin; ++j) rank += sh.edge[j] < mine;
-                if (rank == need - 1) sh.limit = mine;
-            }
-            __syncthreads();
-            limit = sh.limit;
-            break;
-        }
+    const unsigned csize = p.cluster_size, nseg = p.clusters_per_row;
+    const uint64_t tiles = tiles_per_row<T>(p.N, nthr * XS_UNROLL);
+    const uint64_t seg_lo = tiles * seg / nseg, seg_hi = tiles * (seg + 1) / nseg;
+    const uint32_t slots = p.k + XS_EDGE;                // per segment: a superset of its k smallest records
+    const uint64_t* recs = p.xs_records + (row * nseg) * (uint64_t)slots;
+    exact_select_cluster<T>(p.in, p.N, row, p.k, seg_lo, seg_hi, p.xs_records + (row * nseg + seg) * (uint64_t)slots,
+                            p.xs_counters + row * nseg + seg, sh, csize, crank);
+    if (crank != 0) return;
+
+    // every thread of this cluster has fenced its records; the last cluster to get here sees them all
+    if (tid == 0) {
+        const uint32_t ticket = atomicAdd(&p.ctl[row].collect, 1u);
+        const bool last = ticket == nseg - 1;
+        if (last) { p.ctl[row].collect = 0; __threadfence(); }
+        sh.cnt = last ? 1u : 0u;
+        sh.or_bits = 0ull; sh.fill = 0; sh.n_edge = 0;
     }
-    // compact the winners (one shared-memory atomic per warp and visit)
-    src.for_each([&](uint64_t rec, bool valid) {
-        const bool take = valid && rec <= limit;
-        const unsigned bal = __ballot_sync(FULL_MASK, take);
-        if (bal) {
-            uint32_t base = 0;
-            if (lane == 0) base = atomicAdd(&sh.fill, (uint32_t)__popc(bal));
-            base = __shfl_sync(FULL_MASK, base, 0);
-            const uint32_t pos = base + __popc(bal & ((1u << lane) - 1u));
-            if (take && pos < sort_cap) sortbuf[pos] = rec;
-        }
-    });
     __syncthreads();
-}
+    if (sh.cnt == 0) return;
+    __syncthreads();                         // sh.cnt is rewritten by the select below
 
-// Ascending bitonic sort of P records (P a power of two, 32 <= P <= 1024), one per thread of
-// the first P threads.  Exchanges at distance < 32 are warp shuffles; only the longer ones
-// go through shared memory (scratch holds P records) with a named barrier over those P
-// threads, so the rest of the CTA does not take part.
-__device__ __forceinline__ uint64_t bitonic_sort_first_threads(uint64_t v, uint32_t P, uint64_t* scratch) {
-    const unsigned tid = threadIdx.x;
-    for (uint32_t size = 2; size <= P; size <<= 1) {
-        const bool ascending = (tid & size) == 0;
-        for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
-            uint64_t other;
-            if (stride >= 32) {
-                scratch[tid] = v;
-                asm volatile("bar.sync 1, %0;" ::"r"(P) : "memory");
-                other = scratch[tid ^ stride];
-                asm volatile("bar.sync 1, %0;" ::"r"(P) : "memory");
-            } else {
-                other = __shfl_xor_sync(FULL_MASK, v, stride);
-            }
-            const bool lower = (tid & stride) == 0;
-            const bool keep_min = lower == ascending;
-            v = (keep_min == (other < v)) ? other : v;
-        }
+    const uint32_t n = nseg * slots;
+    const uint64_t first = __ldcg(&recs[0]);             // segment 0 is never empty
+    uint64_t diff = 0;
+    for (uint32_t i = tid; i < n; i += nthr) {
+        const uint64_t rec = __ldcg(&recs[i]);
+        if (rec != ~0ull) diff |= rec ^ first;
     }
-    return v;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) diff |= __shfl_xor_sync(FULL_MASK, diff, d);
+    if (lane == 0 && diff) atomicOr(&sh.or_bits, (unsigned long long)diff);
+    __syncthreads();
+    select_smallest(SegmentRecords{recs, n}, first, p.k, sortbuf, p.sort_cap, sh);
+    sort_and_write<T>(sortbuf, p.k, p.k, p.k, row, p.out_vals, p.out_idx);
 }
 
-template <typename T>
-__device__ __forceinline__ void write_output(T* out_vals, int64_t* out_idx, uint32_t k, uint64_t row, uint32_t j, uint64_t rec) {
-    out_vals[row * (uint64_t)k + j] = Elem<T>::from_key(record_key(rec));
-    out_idx[row * (uint64_t)k + j] = (int64_t)record_idx(rec);
-}
-
-// Orders the m records in sortbuf (all threads have passed a barrier since they were written)
-// and writes the first kk of them as row `row` of the output.
-template <typename T>
-__device__ __forceinline__ void sort_and_write(uint64_t* sortbuf, uint32_t m, uint32_t kk, uint32_t k, uint64_t row,
-                                               T* out_vals, int64_t* out_idx) {
-    const unsigned tid = threadIdx.x, nthr = blockDim.x;
-    if (m <= nthr) {
-        uint32_t P = 32;
-        while (P < m) P <<= 1;
-        const uint64_t v0 = tid < m ? sortbuf[tid] : ~0ull;
-        __syncthreads();                                    // sortbuf doubles as the exchange scratch
-        if (tid < P) {
-            const uint64_t v = bitonic_sort_first_threads(v0, P, sortbuf);
-            if (tid < kk) write_output(out_vals, out_idx, k, row, tid, v);
-        }
-    } else {
-        uint32_t P = 1;
-        while (P < m) P <<= 1;
-        for (uint32_t i = m + tid; i < P; i += nthr) sortbuf[i] = ~0ull;
-        __syncthreads();
-        bitonic_sort_shared(sortbuf, P);
-        for (uint32_t j = tid; j < kk; j += nthr) write_output(out_vals, out_idx, k, row, j, sortbuf[j]);
-    }
-}
-
-template <typename T>
-__global__ void __launch_bounds__(1024) refine_kernel(const RefineParams<T> p) {
+// Two builds of the kernel.  With up to 512 threads a refine CTA has to start beside the last CTAs
+// of the filter kernel on an SM, and 48 registers per thread is what fits there; the (rare) exact
+// selection then runs with spills.  A CTA of 1024 threads does not fit there anyway and gets the
+// registers the exact selection wants.
+template <typename T, int MAXREG>
+__global__ void __maxnreg__(MAXREG) refine_kernel(const __grid_constant__ RefineParams<T> p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint64_t* sortbuf = reinterpret_cast<uint64_t*>(smem_raw);                 // sort_cap + RF_EDGE_CAP records
     uint64_t* staged = sortbuf + p.sort_cap + RF_EDGE_CAP;                     // stage_cap records
     __shared__ SelectShared sh;
 
+    // CTAs of a row are consecutive: clusters_per_row clusters (along x) of cluster_size CTAs.
+    const unsigned csize = p.cluster_size, nseg = p.clusters_per_row;
+    const unsigned cta_in_row = blockIdx.x % (csize * nseg);
+    const unsigned seg = cta_in_row / csize, crank = cta_in_row % csize;
+    const bool refiner = cta_in_row == 0;            // the CTA that refines the row's buffer
     const unsigned tid = threadIdx.x, nthr = blockDim.x, lane = lane_id();
-    const uint64_t row = blockIdx.x;
-    if (tid == 0) { sh.or_bits = 0ull; sh.fill = 0; sh.n_edge = 0; sh.crowded = 0; }
-    for (uint32_t i = tid; i < RF_BINS; i += nthr) sh.hist[i] = 0;
-    __syncthreads();
-    pdl_launch_dependents();                 // the exact-selection kernel may be staged behind this one
+    const uint64_t row = blockIdx.x / (csize * nseg);
+    if (refiner) {
+        if (tid == 0) { sh.or_bits = 0ull; sh.fill = 0; sh.n_edge = 0; sh.crowded = 0; }
+        for (uint32_t i = tid; i < RF_BINS; i += nthr) sh.hist[i] = 0;
+        __syncthreads();
+    }
+    pdl_launch_dependents();
     if (p.use_pdl) pdl_wait();
     PROFK_STAMP(1, 0);
 
@@ -253,22 +135,36 @@ __global__ void __launch_bounds__(1024) refine_kernel(const RefineParams<T> p) {
     // the row's control block: which of them are real is known when the survivor count arrives.
     const uint64_t* src = p.buf + row * p.buf_stride;
     uint64_t r[8];
+    if (refiner && !p.direct) {
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-        const uint32_t i = u * nthr + tid;
-        r[u] = i < p.capacity ? src[i] : ~0ull;
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t i = u * nthr + tid;
+            r[u] = i < p.capacity ? src[i] : ~0ull;
+        }
     }
 
     // ---- the count check of stage 4 ----
-    const RowCtl ctl = p.ctl[row];
-    const uint32_t R = ctl.count;
-    const uint32_t status = R > p.capacity ? ROW_OVERFLOW : R < p.k_accept ? ROW_RECALL : ROW_OK;
-    if (tid == 0) {
-        p.ctl[row].status = status;
-        p.ctl[row].n_final = status ? p.k : R;
-        if (status) atomicAdd(&p.header->n_failed, 1u);
+    RowCtl ctl;
+    uint32_t status;
+    if (p.direct) {                          // the row's control block was set up by the initialisation kernel
+        ctl.tau_bits = 0; ctl.count = 0;
+        status = ROW_DIRECT;
+    } else {
+        ctl = p.ctl[row];
+        status = ctl.count > p.capacity ? ROW_OVERFLOW : ctl.count < p.k_accept ? ROW_RECALL : ROW_OK;
+        if (refiner && tid == 0) {
+            p.ctl[row].status = status;
+            p.ctl[row].n_final = status ? p.k : ctl.count;
+            if (status) atomicAdd(&p.header->n_failed, 1u);
+        }
     }
-    if (status != ROW_OK) return;            // the exact-selection kernel takes this row
+    if (status != ROW_OK) {
+        if (csize == 1) return;              // the exact-selection kernel that follows takes this row
+        exact_row<T>(p, row, seg, crank, sortbuf, sh);
+        return;
+    }
+    if (!refiner) return;
+    const uint32_t R = ctl.count;
 
     const uint32_t n = R;
     const uint32_t kk = n < p.k ? n : p.k;          // real outputs; the rest is padding (relaxed mode)
