@@ -198,12 +198,16 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
     cfg.blockDim = dim3(SEL_THREADS);
     cfg.dynamicSmemBytes = (size_t)sp.per_cta * sizeof(uint32_t);
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    // Without a cluster dimension a kernel runs as implicit clusters of one CTA, which is what a
-    // one-CTA cluster is -- and a plain grid of many CTAs launches much faster than as many clusters.
-    cfg.attrs = attr; cfg.numAttrs = csize > 1 ? 1 : 0;
+    // The kernel may be staged behind whatever runs before it on the stream (it waits for that work
+    // before it touches the input or the workspace): its launch and the computation of the sample
+    // positions then overlap that work's tail.  Without a cluster dimension a kernel runs as implicit
+    // clusters of one CTA, which is what a one-CTA cluster is.
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)csize; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = csize > 1 ? 2 : 1;
     CUDA_TRY(cudaLaunchKernelEx(&cfg, sample_select_kernel<T>, sp));
     ++g_launches;
     return PROFK_OK;

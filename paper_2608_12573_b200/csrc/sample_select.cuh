@@ -173,6 +173,16 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
                 }
             }
         }
+        // The sample positions do not depend on the data: only now does the kernel need the work queued
+        // before it on the stream (whatever produced the input, or the previous call on this workspace).
+        // (Their cache lines and address translations are requested meanwhile: a prefetch has no effect
+        // on memory, and L2 is where a later write by that work lands too.)
+        if (pp0 == 0) {
+#pragma unroll
+            for (int s = 0; s < 2 * PB; ++s)
+                if (ok[s]) asm volatile("prefetch.global.L2 [%0];" ::"l"(rowp + idx[s]));
+            pdl_wait();
+        }
         T val[2 * PB];
 #pragma unroll
         for (int s = 0; s < 2 * PB; ++s)
@@ -189,6 +199,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
             }
         }
     }
+    pdl_wait();                  // CTAs without a share of the sample have not waited yet
     if (crank == 0 && tid == 0) {
         if (p.ctl) {
             RowCtl* c = p.ctl + row;
