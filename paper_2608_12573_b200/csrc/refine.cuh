@@ -66,7 +66,7 @@ struct SegmentRecords {
 // the row's output.  The ticket is the row's `collect` word, zero on entry and zero again on exit.
 template <typename T>
 __device__ __noinline__ void exact_row(const RefineParams<T>& p, uint64_t row, unsigned seg, unsigned crank, uint64_t* sortbuf,
-                                          SelectShared& sh) {
+                                       SelectShared& sh, bool overflowed, uint32_t tau_key) {
     const unsigned tid = threadIdx.x, nthr = blockDim.x, lane = lane_id();
     const unsigned csize = p.cluster_size, nseg = p.clusters_per_row;
     const uint64_t tiles = tiles_per_row<T>(p.N, nthr * XS_UNROLL);
@@ -74,7 +74,7 @@ __device__ __noinline__ void exact_row(const RefineParams<T>& p, uint64_t row, u
     const uint32_t slots = p.k + XS_EDGE;                // per segment: a superset of its k smallest records
     const uint64_t* recs = p.xs_records + (row * nseg) * (uint64_t)slots;
     exact_select_cluster<T>(p.in, p.N, row, p.k, seg_lo, seg_hi, p.xs_records + (row * nseg + seg) * (uint64_t)slots,
-                            p.xs_counters + row * nseg + seg, sh, csize, crank);
+                            p.xs_counters + row * nseg + seg, sh, csize, crank, overflowed, tau_key);
     if (crank != 0) return;
 
     // every thread of this cluster has fenced its records; the last cluster to get here sees them all
@@ -160,7 +160,7 @@ __global__ void __maxnreg__(MAXREG) refine_kernel(const __grid_constant__ Refine
     }
     if (status != ROW_OK) {
         if (csize == 1) return;              // the exact-selection kernel that follows takes this row
-        exact_row<T>(p, row, seg, crank, sortbuf, sh);
+        exact_row<T>(p, row, seg, crank, sortbuf, sh, status == ROW_OVERFLOW, Elem<T>::key(Elem<T>::from_bits(ctl.tau_bits)));
         return;
     }
     if (!refiner) return;
