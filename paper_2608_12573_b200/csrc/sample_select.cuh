@@ -28,6 +28,7 @@ constexpr int SEL_THREADS = 1024;
 constexpr int SEL_BINS = 2048;        // 11-bit digits
 constexpr int SEL_GROUPS = 128;       // groups of 8 lanes whose maxima bound the answer from below
 constexpr uint32_t SEL_CAND_CAP = 1024;
+constexpr uint32_t SEL_SPREAD_MIN = 128;    // more candidates than this are ranked by all CTAs of the cluster
 
 // Per-row control block in the workspace.
 struct RowCtl {
@@ -258,29 +259,43 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
         cluster.sync();                               // all candidates have arrived
         PROFK_STAMP(0, 4);
         const uint32_t ncand = *ncand0;
-        auto seen = cluster.barrier_arrive();         // "I have read the count": the first CTA may leave after its peers did
         if (ncand <= SEL_CAND_CAP) {
-            if (crank == 0) {
-                // rank the candidates, eight lanes per candidate sharing the comparison loop
-                const unsigned part = tid & 7u;
-                for (uint32_t c0 = 0; c0 < ncand; c0 += SEL_THREADS / 8) {
-                    const uint32_t c = c0 + (tid >> 3);
-                    const uint32_t mine = c < ncand ? cand[c] : 0;
-                    uint32_t rank = 0;
-                    for (uint32_t j = part; j < ncand; j += 8) {
-                        const uint32_t o = cand[j];
-                        rank += (o > mine) || (o == mine && j < c);
-                    }
-                    rank += __shfl_xor_sync(FULL_MASK, rank, 1);
-                    rank += __shfl_xor_sync(FULL_MASK, rank, 2);
-                    rank += __shfl_xor_sync(FULL_MASK, rank, 4);
-                    if (part == 0 && c < ncand && rank == p.t - 1) publish_threshold(p, row, mine);   // the t-th largest: tau
+            // Every CTA takes a copy of the candidates and looks at its share of them (candidate c goes to
+            // CTA c mod csize): the t-th largest key is the candidate with fewer than t candidates above
+            // it and at least t at or above it.  Eight lanes share one candidate's comparisons.  Equal
+            // candidates all qualify and publish the same value.
+            // A handful of candidates (small ranks) is not worth the copies: the first CTA looks at all.
+            const bool spread = ncand > SEL_SPREAD_MIN;
+            if (spread && crank != 0)
+                for (uint32_t i = tid; i < ncand; i += SEL_THREADS) cand[i] = cand0[i];
+            auto seen = cluster.barrier_arrive();     // "I have read the first CTA's memory": it may leave after its peers did
+            if (spread) __syncthreads();
+            PROFK_STAMP(0, 7);
+            const unsigned part = tid & 7u;
+            const uint32_t c_first = spread ? (tid >> 3) * csize + crank : crank == 0 ? (tid >> 3) : ncand;
+            const uint32_t c_step = (SEL_THREADS / 8) * (spread ? csize : 1u);
+            for (uint32_t c = c_first; c < ncand; c += c_step) {      // whole groups of eight lanes together
+                const uint32_t mine = cand[c];
+                uint32_t above = 0, at_or_above = 0;
+                for (uint32_t j = part; j < ncand; j += 8) {
+                    const uint32_t o = cand[j];
+                    above += o > mine;
+                    at_or_above += o >= mine;
                 }
+                const unsigned group = 0xFFu << (lane & 24u);
+                above += __shfl_xor_sync(group, above, 1);
+                above += __shfl_xor_sync(group, above, 2);
+                above += __shfl_xor_sync(group, above, 4);
+                at_or_above += __shfl_xor_sync(group, at_or_above, 1);
+                at_or_above += __shfl_xor_sync(group, at_or_above, 2);
+                at_or_above += __shfl_xor_sync(group, at_or_above, 4);
+                if (part == 0 && above < p.t && p.t <= at_or_above) publish_threshold(p, row, mine);   // tau
             }
             done = true;
             PROFK_STAMP(0, 5);
             cluster.barrier_wait(std::move(seen));
         } else {
+            auto seen = cluster.barrier_arrive();
             cluster.barrier_wait(std::move(seen));
         }
     } else {
