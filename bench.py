@@ -194,8 +194,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--hot-path-only", action="store_true",
                     help="run only warm-up + timed steps of the hot path (for profiler captures) and exit")
+    ap.add_argument("--rows", type=int, default=0,
+                    help="override the configuration's number of rows (a smaller case of the same kernels for a profiler capture)")
     args = ap.parse_args()
     cfg = CONFIGS[args.config]
+    if args.rows > 0:
+        cfg = (args.rows,) + cfg[1:]
     if args.impl == "reference":
         run_reference(args, cfg, args.config)
         return
