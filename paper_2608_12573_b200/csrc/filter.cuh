@@ -59,6 +59,84 @@ __device__ __forceinline__ bool vec_any_pass(const uint4& v, __nv_bfloat16 tau) 
     return (a & b & c & d) != 0xFFFFFFFFu;    // some lane is not below tau
 }
 
+// Bit l set = element l of the vector is not below tau (the same test as vec_any_pass, per element).
+__device__ __forceinline__ unsigned vec_pass_mask(const float4& v, float tau) {
+    return (unsigned)!(v.x < tau) | ((unsigned)!(v.y < tau) << 1) | ((unsigned)!(v.z < tau) << 2) | ((unsigned)!(v.w < tau) << 3);
+}
+__device__ __forceinline__ unsigned vec_pass_mask(const uint4& v, __nv_bfloat16 tau) {
+    const __nv_bfloat162 t2 = __halves2bfloat162(tau, tau);
+    const unsigned w[4] = {v.x, v.y, v.z, v.w};
+    unsigned m = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const unsigned below = __hlt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&w[j]), t2);   // 0xFFFF per half that is < tau
+        m |= ((~below & 1u) | ((~below >> 15) & 2u)) << (2 * j);
+    }
+    return m;
+}
+
+// Survivors of one thread's vectors of a tile: bit u * VEC + l set = element l of vector u is inside the row
+// and not below tau.  Vectors without a survivor (nearly all) cost one packed test.
+template <typename T, int THREADS, int UNROLL>
+__device__ __forceinline__ uint32_t survivor_mask(const typename Elem<T>::vec_t (&v)[UNROLL], uint32_t inside_mask, uint64_t N,
+                                                  uint64_t qbase, uint32_t mis, T tau) {
+    constexpr int VEC = Elem<T>::VEC;
+    static_assert(VEC * UNROLL <= 32, "one bit per element of the thread's share of a tile");
+    uint32_t mine = 0;
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+        if (((inside_mask >> u) & 1u) && vec_any_pass(v[u], tau)) {
+            unsigned m = vec_pass_mask(v[u], tau);
+            const uint64_t q = qbase + (uint64_t)u * THREADS + threadIdx.x;
+            const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
+            if (i0 < 0 || i0 + VEC > (int64_t)N) {          // a vector across an end of the row: drop the lanes outside
+#pragma unroll
+                for (int l = 0; l < VEC; ++l)
+                    if (i0 + l < 0 || i0 + l >= (int64_t)N) m &= ~(1u << l);
+            }
+            mine |= m << (u * VEC);
+        }
+    }
+    return mine;
+}
+
+// Exclusive prefix of cnt over the lanes of the warp, and the warp's total.  Survivors are rare: usually no
+// lane has more than one, and a vote does it; otherwise a shuffle scan.
+__device__ __forceinline__ unsigned warp_exclusive_count(unsigned cnt, unsigned lane, unsigned* total) {
+    const unsigned has = __ballot_sync(FULL_MASK, cnt != 0);
+    if (!__any_sync(FULL_MASK, cnt > 1)) {
+        *total = __popc(has);
+        return __popc(has & ((1u << lane) - 1u));
+    }
+    unsigned incl = cnt;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const unsigned nb = __shfl_up_sync(FULL_MASK, incl, d);
+        if (lane >= (unsigned)d) incl += nb;
+    }
+    *total = __shfl_sync(FULL_MASK, incl, 31);
+    return incl - cnt;
+}
+
+// Writes one thread's survivors as records to out[pos], out[pos + 1], ... (positions >= limit are dropped).
+// Survivors are few: a loop over the set bits, each picking its element out of the registers.
+template <typename T, int THREADS, int UNROLL>
+__device__ __forceinline__ void emit_survivors(const typename Elem<T>::vec_t (&v)[UNROLL], uint32_t mine, uint64_t qbase,
+                                               uint32_t mis, uint64_t* out, unsigned pos, unsigned limit) {
+    constexpr int VEC = Elem<T>::VEC;
+    static_assert(UNROLL == 4, "four vectors per thread and tile");
+    while (mine) {
+        const int b = __ffs(mine) - 1;
+        mine &= mine - 1;
+        const int u = b / VEC, l = b % VEC;
+        const T x = u == 0 ? vec_elem(v[0], l) : u == 1 ? vec_elem(v[1], l) : u == 2 ? vec_elem(v[2], l) : vec_elem(v[3], l);
+        const uint64_t q = qbase + (uint64_t)u * THREADS + threadIdx.x;
+        const uint32_t i = (uint32_t)((int64_t)(q * VEC) - (int64_t)mis) + (uint32_t)l;
+        if (pos < limit) out[pos] = make_record(Elem<T>::key(x), i);
+        ++pos;
+    }
+}
+
 constexpr uint32_t STAGE_CAP = 64;       // records a warp collects in shared memory ...
 constexpr uint32_t STAGE_FLUSH = 32;     // ... and the fill at which it appends them to the row buffer
 
@@ -100,31 +178,43 @@ __device__ __noinline__ uint32_t filter_slow_path(const FilterParams<T>& p, Warp
     static_assert(UNROLL == 4, "the slow path takes four vectors");
     const V v[4] = {v0, v1, v2, v3};
     const unsigned lane = lane_id();
-    const float tau_f = Elem<T>::as_float(tau);
-    unsigned mine[UNROLL];          // per vector: bit l set = element l survives
-    unsigned cnt = 0;
+    // Per element: a survivor mask, the warp's prefix of the counts, then the records.  With four elements
+    // per vector the straight-line form (every element tested and written under a predicate) is the cheaper
+    // one, also in registers; with eight it is a loop over the set bits of the mask.
+    constexpr bool STRAIGHT = VEC <= 4;
+    unsigned mine_u[UNROLL];        // STRAIGHT: per vector, bit l set = element l survives
+    uint32_t mine = 0;              // otherwise: bit u * VEC + l
+    unsigned cnt = 0, total, before;
+    if constexpr (STRAIGHT) {
+        const float tau_f = Elem<T>::as_float(tau);
 #pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-        mine[u] = 0;
-        if (((inside_mask >> u) & 1u) && vec_any_pass(v[u], tau)) {      // most vectors hold no survivor
-            const uint64_t q = qbase + (uint64_t)u * THREADS + threadIdx.x;
-            const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
+        for (int u = 0; u < UNROLL; ++u) {
+            mine_u[u] = 0;
+            if (((inside_mask >> u) & 1u) && vec_any_pass(v[u], tau)) {      // most vectors hold no survivor
+                const uint64_t q = qbase + (uint64_t)u * THREADS + threadIdx.x;
+                const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
 #pragma unroll
-            for (int l = 0; l < VEC; ++l) {
-                const int64_t i = i0 + l;
-                const bool ok = i >= 0 && i < (int64_t)p.N && !(Elem<T>::as_float(vec_elem(v[u], l)) < tau_f);
-                if (ok) mine[u] |= 1u << l;
+                for (int l = 0; l < VEC; ++l) {
+                    const int64_t i = i0 + l;
+                    const bool ok = i >= 0 && i < (int64_t)p.N && !(Elem<T>::as_float(vec_elem(v[u], l)) < tau_f);
+                    if (ok) mine_u[u] |= 1u << l;
+                }
             }
+            cnt += __popc(mine_u[u]);
         }
-        cnt += __popc(mine[u]);
-    }
-    unsigned incl = cnt;
+        unsigned incl = cnt;
 #pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const unsigned nb = __shfl_up_sync(FULL_MASK, incl, d);
-        if (lane >= (unsigned)d) incl += nb;
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned nb = __shfl_up_sync(FULL_MASK, incl, d);
+            if (lane >= (unsigned)d) incl += nb;
+        }
+        total = __shfl_sync(FULL_MASK, incl, 31);
+        before = incl - cnt;
+    } else {
+        mine = survivor_mask<T, THREADS, UNROLL>(v, inside_mask, p.N, qbase, mis, tau);
+        cnt = __popc(mine);
+        before = warp_exclusive_count(cnt, lane, &total);
     }
-    const unsigned total = __shfl_sync(FULL_MASK, incl, 31);
     if (total == 0) return 0xFFFFFFFFu;
 
     uint32_t overflowed = 0xFFFFFFFFu;
@@ -137,27 +227,31 @@ __device__ __noinline__ uint32_t filter_slow_path(const FilterParams<T>& p, Warp
     unsigned pos, limit;
     const bool to_stage = total <= STAGE_CAP;
     if (to_stage) {                           // the usual case
-        out = st->rec; pos = fill + incl - cnt; limit = STAGE_CAP;
+        out = st->rec; pos = fill + before; limit = STAGE_CAP;
     } else {                                  // a tile full of survivors: straight to the buffer
         unsigned base = 0;
         if (lane == 0) base = atomicAdd(p.counts + (uint64_t)row * p.count_stride, total);
         base = __shfl_sync(FULL_MASK, base, 0);
-        out = p.buf + (uint64_t)row * p.buf_stride; pos = base + incl - cnt; limit = p.capacity;
+        out = p.buf + (uint64_t)row * p.buf_stride; pos = base + before; limit = p.capacity;
         if ((uint64_t)base + total > p.capacity) overflowed = row;
     }
+    if constexpr (STRAIGHT) {
 #pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-        if (mine[u]) {
-            const uint64_t q = qbase + (uint64_t)u * THREADS + threadIdx.x;
-            const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
+        for (int u = 0; u < UNROLL; ++u) {
+            if (mine_u[u]) {
+                const uint64_t q = qbase + (uint64_t)u * THREADS + threadIdx.x;
+                const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
 #pragma unroll
-            for (int l = 0; l < VEC; ++l) {
-                if (mine[u] & (1u << l)) {
-                    if (pos < limit) out[pos] = make_record(Elem<T>::key(vec_elem(v[u], l)), (uint32_t)(i0 + l));
-                    ++pos;
+                for (int l = 0; l < VEC; ++l) {
+                    if (mine_u[u] & (1u << l)) {
+                        if (pos < limit) out[pos] = make_record(Elem<T>::key(vec_elem(v[u], l)), (uint32_t)(i0 + l));
+                        ++pos;
+                    }
                 }
             }
         }
+    } else {
+        if (cnt) emit_survivors<T, THREADS, UNROLL>(v, mine, qbase, mis, out, pos, limit);
     }
     if (to_stage) {
         __syncwarp();
@@ -177,53 +271,19 @@ template <typename T, int THREADS, int UNROLL>
 __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T>& p, const typename Elem<T>::vec_t (&v)[UNROLL],
                                                             const bool (&inside)[UNROLL], uint32_t row, uint64_t qbase,
                                                             uint32_t mis, T tau) {
-    constexpr int VEC = Elem<T>::VEC;
     const unsigned lane = lane_id();
-    const float tau_f = Elem<T>::as_float(tau);
-    unsigned mine[UNROLL];          // per vector: bit l set = element l survives
-    unsigned cnt = 0;
+    uint32_t inside_mask = 0;
 #pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-        mine[u] = 0;
-        if (inside[u] && vec_any_pass(v[u], tau)) {                      // most vectors hold no survivor
-            const uint64_t q = qbase + (uint64_t)u * THREADS + threadIdx.x;
-            const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
-#pragma unroll
-            for (int l = 0; l < VEC; ++l) {
-                const int64_t i = i0 + l;
-                const bool ok = i >= 0 && i < (int64_t)p.N && !(Elem<T>::as_float(vec_elem(v[u], l)) < tau_f);
-                if (ok) mine[u] |= 1u << l;
-            }
-        }
-        cnt += __popc(mine[u]);
-    }
-    unsigned incl = cnt;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const unsigned nb = __shfl_up_sync(FULL_MASK, incl, d);
-        if (lane >= (unsigned)d) incl += nb;
-    }
-    const unsigned total = __shfl_sync(FULL_MASK, incl, 31);
+    for (int u = 0; u < UNROLL; ++u) inside_mask |= inside[u] ? 1u << u : 0u;
+    const uint32_t mine = survivor_mask<T, THREADS, UNROLL>(v, inside_mask, p.N, qbase, mis, tau);
+    const unsigned cnt = __popc(mine);
+    unsigned total;
+    const unsigned before = warp_exclusive_count(cnt, lane, &total);
     if (total == 0) return 0xFFFFFFFFu;
     unsigned base = 0;
     if (lane == 0) base = atomicAdd(p.counts + (uint64_t)row * p.count_stride, total);
     base = __shfl_sync(FULL_MASK, base, 0);
-    unsigned pos = base + incl - cnt;
-    uint64_t* dst = p.buf + (uint64_t)row * p.buf_stride;
-#pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-        if (mine[u]) {
-            const uint64_t q = qbase + (uint64_t)u * THREADS + threadIdx.x;
-            const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
-#pragma unroll
-            for (int l = 0; l < VEC; ++l) {
-                if (mine[u] & (1u << l)) {
-                    if (pos < p.capacity) dst[pos] = make_record(Elem<T>::key(vec_elem(v[u], l)), (uint32_t)(i0 + l));
-                    ++pos;
-                }
-            }
-        }
-    }
+    if (cnt) emit_survivors<T, THREADS, UNROLL>(v, mine, qbase, mis, p.buf + (uint64_t)row * p.buf_stride, base + before, p.capacity);
     return (uint64_t)base + total > p.capacity ? row : 0xFFFFFFFFu;
 }
 
