@@ -464,6 +464,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
 template <typename T>
 int topk_auto(const T* in, int64_t rows, int64_t N, int64_t k, double eps, double recall, uint64_t seed, void* stream,
               T* out_vals, int64_t* out_idx) {
+    g_launches = 0;
     profk_plan_t plan;
     {
         std::lock_guard<std::mutex> lock(g_mutex);
