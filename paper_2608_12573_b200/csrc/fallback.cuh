@@ -13,6 +13,7 @@
 // wait is bounded and reports through the workspace header.
 #pragma once
 
+#include "grid_barrier.cuh"
 #include "refine.cuh"
 #include "rowscan.cuh"
 #include "sample_select.cuh"
@@ -23,7 +24,6 @@ constexpr int FB_THREADS = 1024;
 constexpr int FB_UNROLL = 4;
 constexpr int FB_BINS = 2048;
 constexpr int FB_PASSES = 6;                // 5 x 11 bits + 9 bits = 64
-constexpr uint32_t SPIN_LIMIT = 1u << 24;   // polls (each ~100 ns apart) before a wait gives up
 
 
 template <typename T> struct FallbackParams {
@@ -43,35 +43,6 @@ template <typename T> struct FallbackParams {
     T* out_vals;              // rows x k
     int64_t* out_idx;         // rows x k
 };
-
-// Sense-free generation barrier over all CTAs of a co-resident grid.  Returns false when
-// the wait gave up (or an earlier one did); the caller then leaves the kernel.
-__device__ __forceinline__ bool grid_barrier(WsHeader* h, uint32_t& gen) {
-    __shared__ uint32_t s_ok;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        uint32_t ok = 1;
-        __threadfence();
-        const uint32_t arrived = atomicAdd(&h->bar_count, 1u);
-        if (arrived == gridDim.x - 1) {
-            atomicExch(&h->bar_count, 0u);
-            __threadfence();
-            atomicAdd(&h->bar_gen, 1u);
-        } else {
-            uint32_t polls = 0;
-            while (*((volatile uint32_t*)&h->bar_gen) == gen) {
-                __nanosleep(64);
-                if (++polls > SPIN_LIMIT) { atomicExch(&h->error, 1u); ok = 0; break; }
-            }
-        }
-        __threadfence();
-        if (*((volatile uint32_t*)&h->error) != 0) ok = 0;
-        s_ok = ok;
-    }
-    __syncthreads();
-    gen += 1;
-    return s_ok != 0;
-}
 
 // Visits every element of `row` that falls to this CTA (tiles blockIdx.x, +gridDim.x, ...):
 // f(record, valid) is called by all 32 lanes of each warp together.

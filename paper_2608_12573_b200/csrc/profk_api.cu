@@ -28,6 +28,7 @@ namespace {
 constexpr int FILTER_THREADS = PROFK_FILTER_THREADS;
 constexpr int FILTER_UNROLL = PROFK_FILTER_UNROLL;
 constexpr uint32_t SORT_CAP_MAX = 8192;          // largest k the single-CTA refine orders in shared memory
+constexpr int LARGE_MAX_CTAS = 1024;             // CTAs of the large refine (its per-CTA slots live in the 48 KB histogram area)
 constexpr int64_t XS_MAX_ROWS = 18;              // most rows for which the refine kernel itself replaces failed rows
 constexpr unsigned XS_MAX_SEGMENTS = 32;         // most (row, segment) pairs of that exact selection
 constexpr unsigned REFINE_CLUSTER_THREADS = 512;   // fewest threads of a refine CTA that may have to read whole rows
@@ -46,7 +47,6 @@ struct DeviceInfo {
     int filter_staged_blocks_per_sm[2] = {0, 0};
     int fallback_blocks_per_sm[2] = {0, 0};
     int max_cluster[2] = {8, 8};              // 16 when the device can co-schedule 16 CTAs of the threshold kernel
-    int large_cluster[2] = {8, 8};            // same for the cluster sort (128 KB of shared memory per CTA)
     int refine_cluster[2] = {8, 8};           // same for the refine kernel at its largest footprint
     bool ready = false;
 };
@@ -148,17 +148,6 @@ template <typename T> int ensure_device_info(int dev, DeviceInfo* out) {
         }
         (void)cudaGetLastError();
         CUDA_TRY(cudaFuncSetAttribute(refine_large_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(BT_TILE * 8)));
-        if (cudaFuncSetAttribute(refine_large_kernel<T>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
-            cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(16); cfg.blockDim = dim3(BT_THREADS); cfg.dynamicSmemBytes = BT_TILE * 8;
-            cudaLaunchAttribute attr[1];
-            attr[0].id = cudaLaunchAttributeClusterDimension;
-            attr[0].val.clusterDim.x = 16; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-            cfg.attrs = attr; cfg.numAttrs = 1;
-            int nclusters = 0;
-            if (cudaOccupancyMaxActiveClusters(&nclusters, refine_large_kernel<T>, &cfg) == cudaSuccess && nclusters >= 1)
-                di.large_cluster[d] = 16;
-        }
         (void)cudaGetLastError();
     }
     *out = di;
@@ -245,30 +234,51 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     return PROFK_OK;
 }
 
+// Cooperative launch (all CTAs co-resident: the kernel uses grid barriers), staged behind the kernel before it
+// when the runtime accepts a cooperative launch that is also a programmatic dependent.  `set_pdl` tells the
+// kernel's parameters which way it went.
+template <typename Kernel, typename Params, typename SetPdl>
+int launch_cooperative(cudaLaunchConfig_t cfg, Kernel kernel, Params params, bool after_kernel, SetPdl set_pdl) {
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    if (after_kernel && g_coop_pdl.load() != 0) {
+        cfg.numAttrs = 2;
+        set_pdl(params, 1);
+        if (cudaLaunchKernelEx(&cfg, kernel, params) == cudaSuccess) {
+            g_coop_pdl.store(1);
+            ++g_launches;
+            return PROFK_OK;
+        }
+        (void)cudaGetLastError();
+        g_coop_pdl.store(0);
+    }
+    cfg.numAttrs = 1;
+    set_pdl(params, 0);
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, params));
+    ++g_launches;
+    return PROFK_OK;
+}
+
+// Count check + ordering for large selections: the whole grid, one CTA per SM, one row after the other.
 template <typename T>
-int launch_refine_large(const DeviceInfo& di, RowCtl* ctl, WsHeader* header, uint64_t* buf, uint64_t row_pitch, uint32_t* bins, int64_t rows,
-                        int64_t capacity, int64_t k, int64_t k_accept, int phase, T* out_vals, int64_t* out_idx, cudaStream_t st) {
+int launch_refine_large(const DeviceInfo& di, RowCtl* ctl, WsHeader* header, uint64_t* buf, uint64_t row_pitch, uint32_t* bins,
+                        unsigned long long* slots, int64_t rows, int64_t capacity, int64_t k, int64_t k_accept, int phase, T* out_vals,
+                        int64_t* out_idx, cudaStream_t st) {
     LargeParams<T> lp;
-    const uint64_t row_stride = row_pitch / 2;
-    lp.ctl = ctl; lp.header = header; lp.buf = buf; lp.row_stride = row_stride; lp.bins = bins; lp.capacity = (uint32_t)capacity;
+    lp.ctl = ctl; lp.header = header; lp.buf = buf; lp.row_stride = row_pitch / 2; lp.bins = bins; lp.slots = slots;
+    lp.rows = (uint64_t)rows; lp.capacity = (uint32_t)capacity;
     lp.k = (uint32_t)k; lp.k_accept = (uint32_t)k_accept; lp.phase = phase; lp.out_vals = out_vals; lp.out_idx = out_idx;
-    lp.use_pdl = 1;
-    int csize = di.large_cluster[dtype_index<T>()];
-    while (csize > 1 && (uint64_t)csize * BT_TILE > row_stride) csize /= 2;     // no more CTAs than tiles
+    lp.use_pdl = 0;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(rows * csize));
+    cfg.gridDim = dim3((unsigned)std::min(di.sm_count, LARGE_MAX_CTAS));
     cfg.blockDim = dim3(BT_THREADS);
     cfg.dynamicSmemBytes = (size_t)BT_TILE * 8;
     cfg.stream = st;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = 2;
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, refine_large_kernel<T>, lp));
-    ++g_launches;
-    return PROFK_OK;
+    return launch_cooperative(cfg, refine_large_kernel<T>, lp, true, [](LargeParams<T>& q, int v) { q.use_pdl = v; });
 }
 
 // Who replaces a row that fails the count check.  With few rows each row gets a cluster of CTAs in
@@ -396,7 +406,8 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         if (rc != PROFK_OK) return rc;
 
         if (large) {
-            rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, rows, capacity, k, plan->k_accept, 0, out_vals, out_idx, st);
+            rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, reinterpret_cast<unsigned long long*>(ghist), rows, capacity, k, plan->k_accept, 0,
+                                        out_vals, out_idx, st);
         } else {
             // count check and refine; with clusters, also the exact selection of the rows that fail the check
             rc = launch_refine<T>(di, in, rows, N, ctl, header, buf, row_stride, capacity, k, plan->k_accept, false, csize, xs_records, xs_counters, out_vals, out_idx, st);
@@ -426,36 +437,12 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         cfg.blockDim = dim3(FB_THREADS);
         cfg.dynamicSmemBytes = large ? 0 : (size_t)fb_sort_cap * 8;
         cfg.stream = st;
-        cudaLaunchAttribute attr[2];
-        attr[0].id = cudaLaunchAttributeCooperative;
-        attr[0].val.cooperative = 1;
-        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[1].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        // A cooperative launch that is also a programmatic dependent hides its launch latency behind
-        // the kernel before it; if the runtime refuses the combination, launch it as a plain cooperative kernel.
-        int pdl_state = g_coop_pdl.load();
-        bool launched = false;
-        if (plan->mode == 0 && pdl_state != 0) {
-            cfg.numAttrs = 2;
-            fb.use_pdl = 1;
-            if (cudaLaunchKernelEx(&cfg, fallback_kernel<T>, fb) == cudaSuccess) {
-                launched = true;
-                g_coop_pdl.store(1);
-            } else {
-                (void)cudaGetLastError();
-                g_coop_pdl.store(0);
-            }
-        }
-        if (!launched) {
-            cfg.numAttrs = 1;
-            fb.use_pdl = 0;
-            CUDA_TRY(cudaLaunchKernelEx(&cfg, fallback_kernel<T>, fb));
-        }
-        ++g_launches;
+        rc = launch_cooperative(cfg, fallback_kernel<T>, fb, plan->mode == 0, [](FallbackParams<T>& q, int v) { q.use_pdl = v; });
+        if (rc != PROFK_OK) return rc;
     }
     if (large) {   // the rows the exact selection repaired still have to be ordered and written
-        rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, rows, capacity, k, k, 1, out_vals, out_idx, st);
+        rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, reinterpret_cast<unsigned long long*>(ghist), rows, capacity, k, k, 1, out_vals,
+                                    out_idx, st);
         if (rc != PROFK_OK) return rc;
     }
     return PROFK_OK;

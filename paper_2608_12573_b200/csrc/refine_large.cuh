@@ -1,7 +1,8 @@
 // Stage 4 for large selections (k beyond what one CTA orders in shared memory; the flattened
 // BatchTopK case of Section 5, "Application", selects K = B k = 131,072 values): the count
 // check, then the k smallest candidate records in ascending order -- which is "value
-// descending, index ascending" -- by one thread-block cluster.
+// descending, index ascending" -- by the whole grid, launched cooperatively (one CTA per SM, all
+// co-resident), one row after the other.
 //
 // Main path: the records are binned on the top 18 bits of their distance above the smallest
 // record (262144 bins in global memory; because a record holds the value key above the index,
@@ -12,11 +13,11 @@
 // Reserve path, taken when a bin is too crowded for that (an outlier stretches the range):
 // a bitonic network over P = 2^j records in the row's buffer, exchanges below one tile
 // (16384 records = 128 KB) in shared memory, the longer ones on the buffer in global memory.
-// Both paths use hardware cluster barriers only.
+// The steps of both paths are separated by grid barriers whose waits are bounded: a wait that gives
+// up sets the workspace's error flag and the kernel returns.
 #pragma once
 
-#include <cooperative_groups.h>
-
+#include "grid_barrier.cuh"
 #include "refine.cuh"
 
 namespace profk {
@@ -33,6 +34,8 @@ template <typename T> struct LargeParams {
     uint64_t* buf;           // row r: records at buf + r * 2 * row_stride, then row_stride records of scratch;
     uint64_t row_stride;     //        row_stride is a power of two >= capacity, >= BT_TILE
     uint32_t* bins;          // rows x (LG_BINS + 8) words: bin counts / positions, then flags
+    unsigned long long* slots;   // 2 words per CTA of the grid, then one per CTA: per-CTA minima / maxima and scan totals
+    uint64_t rows;
     uint32_t capacity;
     uint32_t k;
     uint32_t k_accept;
@@ -65,65 +68,61 @@ template <typename T>
 __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const LargeParams<T> p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint64_t* tile = reinterpret_cast<uint64_t*>(smem_raw);          // BT_TILE records
+    __shared__ unsigned long long s_min[32], s_max[32];
+    __shared__ uint32_t s_warp[32];
 
-    namespace cg = cooperative_groups;
-    cg::cluster_group cluster = cg::this_cluster();
-    const unsigned csize = cluster.num_blocks();
-    const unsigned crank = cluster.block_rank();
-    const uint64_t row = blockIdx.x / csize;
+    const unsigned nctas = gridDim.x, cta = blockIdx.x;
     const unsigned tid = threadIdx.x;
-    const uint64_t gid = (uint64_t)crank * BT_THREADS + tid;         // thread index inside the cluster
-    const uint64_t gthreads = (uint64_t)csize * BT_THREADS;
+    const uint64_t gid = (uint64_t)cta * BT_THREADS + tid;           // thread index inside the grid
+    const uint64_t gthreads = (uint64_t)nctas * BT_THREADS;
+    unsigned long long* slot_min = p.slots;
+    unsigned long long* slot_max = p.slots + nctas;
+    unsigned long long* slot_total = p.slots + 2 * nctas;
+    // The scan is shared by a power-of-two number of CTAs (at most 256, so that a thread owns a whole bin).
+    unsigned scan_ctas = 1;
+    while (scan_ctas * 2 <= nctas && scan_ctas < 256) scan_ctas *= 2;
 
     pdl_launch_dependents();
     if (p.use_pdl) pdl_wait();
+    uint32_t gen = *((volatile uint32_t*)&p.header->bar_gen);        // read before this CTA's first arrival
 
-    // ---- which rows this launch handles (the decision is the same in every CTA of the cluster) ----
-    const RowCtl ctl = p.ctl[row];
-    uint32_t n;
-    if (p.phase == 0) {
-        const uint32_t R = ctl.count;
-        const uint32_t status = R > p.capacity ? ROW_OVERFLOW : R < p.k_accept ? ROW_RECALL : ROW_OK;
-        if (crank == 0 && tid == 0) {
-            p.ctl[row].status = status;
-            p.ctl[row].n_final = status ? p.k : R;
-            if (status) atomicAdd(&p.header->n_failed, 1u);
+    for (uint64_t row = 0; row < p.rows; ++row) {
+        // ---- is this row for this launch?  (the decision is the same in every CTA) ----
+        const RowCtl ctl = p.ctl[row];
+        uint32_t n;
+        if (p.phase == 0) {
+            const uint32_t R = ctl.count;
+            const uint32_t status = R > p.capacity ? ROW_OVERFLOW : R < p.k_accept ? ROW_RECALL : ROW_OK;
+            if (cta == 0 && tid == 0) {
+                p.ctl[row].status = status;
+                p.ctl[row].n_final = status ? p.k : R;
+                if (status) atomicAdd(&p.header->n_failed, 1u);
+            }
+            if (status != ROW_OK) continue;      // the exact-selection kernel and the second phase take this row
+            n = R;
+        } else {
+            if (ctl.status == ROW_OK) continue;  // already written by the first phase
+            n = p.k;                             // the exact selection left exactly k records
         }
-        if (status != ROW_OK) return;        // the exact-selection kernel and the second phase take this row
-        n = R;
-    } else {
-        if (ctl.status == ROW_OK) return;    // already written by the first phase
-        n = p.k;                             // the exact selection left exactly k records
-    }
-    const uint32_t kk = n < p.k ? n : p.k;
-    uint64_t* G = p.buf + row * 2 * p.row_stride;
-    uint64_t* G2 = G + p.row_stride;
-    uint32_t* bins = p.bins + row * (uint64_t)(LG_BINS + 8);
-    uint32_t* flags = bins + LG_BINS;                                // [0] = some bin that matters is crowded
+        const uint32_t kk = n < p.k ? n : p.k;
+        uint64_t* G = p.buf + row * 2 * p.row_stride;
+        uint64_t* G2 = G + p.row_stride;
+        uint32_t* bins = p.bins + row * (uint64_t)(LG_BINS + 8);
+        uint32_t* flags = bins + LG_BINS;                                // [0] = some bin that matters is crowded
 
-    for (uint64_t j = kk + gid; j < p.k; j += gthreads) {            // relaxed mode: padding after a short buffer
-        p.out_vals[row * (uint64_t)p.k + j] = Elem<T>::from_bits(Elem<T>::NEG_INF_BITS);
-        p.out_idx[row * (uint64_t)p.k + j] = -1;
-    }
+        for (uint64_t j = kk + gid; j < p.k; j += gthreads) {            // relaxed mode: padding after a short buffer
+            p.out_vals[row * (uint64_t)p.k + j] = Elem<T>::from_bits(Elem<T>::NEG_INF_BITS);
+            p.out_idx[row * (uint64_t)p.k + j] = -1;
+        }
 
-    // ================= main path: bin, scan, scatter, rank inside bins =================
-    __shared__ unsigned long long s_min[32], s_max[32], s_cta_min, s_cta_max;
-    __shared__ uint32_t s_warp[32], s_cta_total;
-    {
+        // ================= main path: bin, scan, scatter, rank inside bins =================
         // smallest and largest record of the row; clear the bins meanwhile
         for (uint64_t b = gid; b < LG_BINS + 8; b += gthreads) bins[b] = 0;
         unsigned long long lo = ~0ull, hi = 0ull;
-        for (uint64_t i0 = gid; i0 < n; i0 += 4 * gthreads) {           // four loads in flight per thread
-            unsigned long long rec[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) rec[u] = i0 + u * gthreads < n ? __ldcg(&G[i0 + u * gthreads]) : ~0ull;
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (i0 + u * gthreads < n) {
-                    lo = rec[u] < lo ? rec[u] : lo;
-                    hi = rec[u] > hi ? rec[u] : hi;
-                }
-            }
+        for (uint64_t i = gid; i < n; i += gthreads) {
+            const unsigned long long rec = __ldcg(&G[i]);
+            lo = rec < lo ? rec : lo;
+            hi = rec > hi ? rec : hi;
         }
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) {
@@ -141,12 +140,18 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
                 lo = l2 < lo ? l2 : lo;
                 hi = h2 > hi ? h2 : hi;
             }
-            if (tid == 0) { s_cta_min = lo; s_cta_max = hi; }
+            if (tid == 0) { slot_min[cta] = lo; slot_max[cta] = hi; }
         }
-        cluster.sync();
+        if (!grid_barrier(p.header, gen)) return;
         unsigned long long rmin = ~0ull, rmax = 0ull;
-        for (unsigned c = 0; c < csize; ++c) {
-            const unsigned long long l2 = *cluster.map_shared_rank(&s_cta_min, c), h2 = *cluster.map_shared_rank(&s_cta_max, c);
+        for (unsigned c = tid & 31; c < nctas; c += 32) {
+            const unsigned long long l2 = __ldcg(&slot_min[c]), h2 = __ldcg(&slot_max[c]);
+            rmin = l2 < rmin ? l2 : rmin;
+            rmax = h2 > rmax ? h2 : rmax;
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            const unsigned long long l2 = __shfl_xor_sync(FULL_MASK, rmin, d), h2 = __shfl_xor_sync(FULL_MASK, rmax, d);
             rmin = l2 < rmin ? l2 : rmin;
             rmax = h2 > rmax ? h2 : rmax;
         }
@@ -154,133 +159,116 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         const int shift = rbits > LG_BITS ? rbits - LG_BITS : 0;
         auto bin_of = [&](unsigned long long rec) { return (uint32_t)((rec - rmin) >> shift); };
 
-        // histogram (global atomics spread over 65536 addresses)
-        for (uint64_t i0 = gid; i0 < n; i0 += 4 * gthreads) {
-            unsigned long long rec[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) rec[u] = i0 + u * gthreads < n ? __ldcg(&G[i0 + u * gthreads]) : 0ull;
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (i0 + u * gthreads < n) atomicAdd(&bins[bin_of(rec[u])], 1u);
-        }
-        cluster.sync();
+        // histogram (global atomics spread over the bins)
+        for (uint64_t i = gid; i < n; i += gthreads) atomicAdd(&bins[bin_of(__ldcg(&G[i]))], 1u);
+        if (!grid_barrier(p.header, gen)) return;
 
-        // scan: CTA c owns bins [c, c+1) * LG_BINS / csize; counts become end positions
-        const uint32_t per_cta = LG_BINS / csize, per_thr = per_cta / BT_THREADS;      // csize <= 16: per_thr >= 4
-        const uint32_t b0 = crank * per_cta + tid * per_thr;
-        uint32_t sum = 0;
-        for (uint32_t j = 0; j < per_thr; ++j) sum += __ldcg(&bins[b0 + j]);
-        uint32_t incl = sum;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t v = __shfl_up_sync(FULL_MASK, incl, d);
-            if ((tid & 31) >= (unsigned)d) incl += v;
-        }
-        if ((tid & 31) == 31) s_warp[tid >> 5] = incl;
-        __syncthreads();
-        if (tid < 32) {
-            uint32_t w = s_warp[tid];
+        // scan: CTA c < scan_ctas owns bins [c, c+1) * LG_BINS / scan_ctas; counts become first positions
+        const uint32_t per_cta = LG_BINS / scan_ctas, per_thr = per_cta / BT_THREADS;
+        const uint32_t b0 = cta * per_cta + tid * per_thr;
+        uint32_t sum = 0, incl = 0;
+        if (cta < scan_ctas) {
+            for (uint32_t j = 0; j < per_thr; ++j) sum += __ldcg(&bins[b0 + j]);
+            incl = sum;
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t v = __shfl_up_sync(FULL_MASK, w, d);
-                if (tid >= (unsigned)d) w += v;
+                const uint32_t v = __shfl_up_sync(FULL_MASK, incl, d);
+                if ((tid & 31) >= (unsigned)d) incl += v;
             }
-            s_warp[tid] = w;
-            if (tid == 31) s_cta_total = w;
+            if ((tid & 31) == 31) s_warp[tid >> 5] = incl;
+            __syncthreads();
+            if (tid < 32) {
+                uint32_t w = s_warp[tid];
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const uint32_t v = __shfl_up_sync(FULL_MASK, w, d);
+                    if (tid >= (unsigned)d) w += v;
+                }
+                s_warp[tid] = w;
+                if (tid == 31) slot_total[cta] = w;
+            }
         }
-        cluster.sync();
-        uint32_t before = incl - sum + ((tid >> 5) ? s_warp[(tid >> 5) - 1] : 0);
-        for (unsigned c = 0; c < crank; ++c) before += *cluster.map_shared_rank(&s_cta_total, c);
-        for (uint32_t j = 0; j < per_thr; ++j) {
-            const uint32_t c = __ldcg(&bins[b0 + j]);
-            if (before < kk && c > LG_CROWDED) atomicOr(&flags[0], 1u);
-            bins[b0 + j] = before;                                   // first position; the scatter advances it to the end
-            before += c;
+        if (!grid_barrier(p.header, gen)) return;
+        if (cta < scan_ctas) {
+            uint32_t before = incl - sum + ((tid >> 5) ? s_warp[(tid >> 5) - 1] : 0);
+            uint32_t ahead = 0;                                      // records in the bins of the CTAs before this one
+            for (unsigned c = tid & 31; c < cta; c += 32) ahead += (uint32_t)__ldcg(&slot_total[c]);
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) ahead += __shfl_xor_sync(FULL_MASK, ahead, d);
+            before += ahead;
+            for (uint32_t j = 0; j < per_thr; ++j) {
+                const uint32_t c = __ldcg(&bins[b0 + j]);
+                if (before < kk && c > LG_CROWDED) atomicOr(&flags[0], 1u);
+                bins[b0 + j] = before;                               // first position; the scatter advances it to the end
+                before += c;
+            }
         }
-        cluster.sync();
+        if (!grid_barrier(p.header, gen)) return;
 
         if (__ldcg(&flags[0]) == 0) {
             // scatter into the second buffer, grouped by bin
-            for (uint64_t i0 = gid; i0 < n; i0 += 4 * gthreads) {
-                unsigned long long rec[4];
-                uint32_t pos[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) rec[u] = i0 + u * gthreads < n ? __ldcg(&G[i0 + u * gthreads]) : 0ull;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) pos[u] = i0 + u * gthreads < n ? atomicAdd(&bins[bin_of(rec[u])], 1u) : 0u;
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (i0 + u * gthreads < n) G2[pos[u]] = rec[u];
+            for (uint64_t i = gid; i < n; i += gthreads) {
+                const unsigned long long rec = __ldcg(&G[i]);
+                G2[atomicAdd(&bins[bin_of(rec)], 1u)] = rec;
             }
-            cluster.sync();
+            if (!grid_barrier(p.header, gen)) return;
             // rank inside the bin: bin b now occupies [end of bin b-1, bins[b])
             // (only positions below the end of the bin that holds position kk-1 matter; they are a prefix)
-            for (uint64_t g0 = gid; g0 < n; g0 += 4 * gthreads) {
-                unsigned long long rec[4];
-                uint32_t first[4], last[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) rec[u] = g0 + u * gthreads < n ? __ldcg(&G2[g0 + u * gthreads]) : rmin;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const uint32_t b = bin_of(rec[u]);
-                    first[u] = b ? __ldcg(&bins[b - 1]) : 0u;
-                    last[u] = __ldcg(&bins[b]);
+            const uint64_t g_end = (uint64_t)kk + LG_CROWDED < n ? (uint64_t)kk + LG_CROWDED : n;
+            for (uint64_t g = gid; g < g_end; g += gthreads) {
+                const unsigned long long rec = __ldcg(&G2[g]);
+                const uint32_t b = bin_of(rec);
+                const uint32_t first = b ? __ldcg(&bins[b - 1]) : 0u, last = __ldcg(&bins[b]);
+                if (first < kk) {
+                    uint32_t pos = first;
+                    for (uint32_t j = first; j < last; ++j) pos += __ldcg(&G2[j]) < rec;
+                    if (pos < kk) write_output(p.out_vals, p.out_idx, p.k, row, pos, rec);
                 }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    if (g0 + u * gthreads < n && first[u] < kk) {
-                        uint32_t pos = first[u];
-                        for (uint32_t j = first[u]; j < last[u]; ++j) pos += __ldcg(&G2[j]) < rec[u];
-                        if (pos < kk) write_output(p.out_vals, p.out_idx, p.k, row, pos, rec[u]);
-                    }
-                }
-                if (g0 >= kk + LG_CROWDED) break;           // grouped positions beyond every bin that matters
             }
-            cluster.sync();              // peers may still be reading this CTA's shared memory above
-            return;
+            continue;                    // next row: its first barrier also orders this row's reads before any reuse
         }
-    }
 
-    // ================= reserve path: bitonic network =================
-    uint64_t P = BT_TILE;
-    while (P < n) P <<= 1;
+        // ================= reserve path: bitonic network =================
+        uint64_t P = BT_TILE;
+        while (P < n) P <<= 1;
 
-    // ---- sort every tile (sizes 2 .. BT_TILE); positions beyond n hold all-ones padding ----
-    const uint64_t tiles = P / BT_TILE;
-    for (uint64_t t = crank; t < tiles; t += csize) {
-        const uint64_t base = t * BT_TILE;
-        for (uint32_t i = tid; i < BT_TILE; i += BT_THREADS) tile[i] = base + i < n ? __ldcg(&G[base + i]) : ~0ull;
-        __syncthreads();
-        bitonic_tile_steps(tile, base, 2, BT_TILE);
-        for (uint32_t i = tid; i < BT_TILE; i += BT_THREADS) G[base + i] = tile[i];
-        __syncthreads();
-    }
-    cluster.sync();
-
-    // ---- merge: exchanges at distance >= BT_TILE on the buffer, the rest tile by tile ----
-    for (uint64_t size = 2ull * BT_TILE; size <= P; size <<= 1) {
-        for (uint64_t stride = size / 2; stride >= BT_TILE; stride >>= 1) {
-            for (uint64_t q = gid; q < P / 2; q += gthreads) {
-                const uint64_t lo = 2 * q - (q & (stride - 1));
-                const uint64_t hi = lo + stride;
-                const bool ascending = (lo & size) == 0;
-                const uint64_t x = __ldcg(&G[lo]), y = __ldcg(&G[hi]);
-                if ((x > y) == ascending) { G[lo] = y; G[hi] = x; }
-            }
-            cluster.sync();
-        }
-        for (uint64_t t = crank; t < tiles; t += csize) {
+        // ---- sort every tile (sizes 2 .. BT_TILE); positions beyond n hold all-ones padding ----
+        const uint64_t tiles = P / BT_TILE;
+        for (uint64_t t = cta; t < tiles; t += nctas) {
             const uint64_t base = t * BT_TILE;
-            for (uint32_t i = tid; i < BT_TILE; i += BT_THREADS) tile[i] = __ldcg(&G[base + i]);
+            for (uint32_t i = tid; i < BT_TILE; i += BT_THREADS) tile[i] = base + i < n ? __ldcg(&G[base + i]) : ~0ull;
             __syncthreads();
-            bitonic_tile_steps(tile, base, size, size);
+            bitonic_tile_steps(tile, base, 2, BT_TILE);
             for (uint32_t i = tid; i < BT_TILE; i += BT_THREADS) G[base + i] = tile[i];
             __syncthreads();
         }
-        cluster.sync();
-    }
+        if (!grid_barrier(p.header, gen)) return;
 
-    for (uint64_t j = gid; j < kk; j += gthreads) write_output(p.out_vals, p.out_idx, p.k, row, (uint32_t)j, __ldcg(&G[j]));
+        // ---- merge: exchanges at distance >= BT_TILE on the buffer, the rest tile by tile ----
+        for (uint64_t size = 2ull * BT_TILE; size <= P; size <<= 1) {
+            for (uint64_t stride = size / 2; stride >= BT_TILE; stride >>= 1) {
+                for (uint64_t q = gid; q < P / 2; q += gthreads) {
+                    const uint64_t lo2 = 2 * q - (q & (stride - 1));
+                    const uint64_t hi2 = lo2 + stride;
+                    const bool ascending = (lo2 & size) == 0;
+                    const uint64_t x = __ldcg(&G[lo2]), y = __ldcg(&G[hi2]);
+                    if ((x > y) == ascending) { G[lo2] = y; G[hi2] = x; }
+                }
+                if (!grid_barrier(p.header, gen)) return;
+            }
+            for (uint64_t t = cta; t < tiles; t += nctas) {
+                const uint64_t base = t * BT_TILE;
+                for (uint32_t i = tid; i < BT_TILE; i += BT_THREADS) tile[i] = __ldcg(&G[base + i]);
+                __syncthreads();
+                bitonic_tile_steps(tile, base, size, size);
+                for (uint32_t i = tid; i < BT_TILE; i += BT_THREADS) G[base + i] = tile[i];
+                __syncthreads();
+            }
+            if (!grid_barrier(p.header, gen)) return;
+        }
+
+        for (uint64_t j = gid; j < kk; j += gthreads) write_output(p.out_vals, p.out_idx, p.k, row, (uint32_t)j, __ldcg(&G[j]));
+    }
 }
 
 }  // namespace profk
