@@ -28,6 +28,7 @@ namespace {
 constexpr int FILTER_THREADS = PROFK_FILTER_THREADS;
 constexpr int FILTER_UNROLL = PROFK_FILTER_UNROLL;
 constexpr uint32_t SORT_CAP_MAX = 8192;          // largest k the single-CTA refine orders in shared memory
+constexpr int64_t GATHER_MAX_ROWS = 4;           // most rows for which the sample may be gathered by a kernel of its own
 constexpr int LARGE_MAX_CTAS = 1024;             // CTAs of the large refine (its per-CTA slots live in the 48 KB histogram area)
 constexpr int64_t XS_MAX_ROWS = 18;              // most rows for which the refine kernel itself replaces failed rows
 constexpr unsigned XS_MAX_SEGMENTS = 32;         // most (row, segment) pairs of that exact selection
@@ -61,7 +62,7 @@ std::map<std::tuple<int64_t, int64_t, double, double>, profk_plan_t> g_plan_cach
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-    size_t off_header, off_ghist, off_ctl, off_tau, off_bins, off_xs_counters, off_xs_records, off_buf, total;
+    size_t off_header, off_ghist, off_ctl, off_tau, off_bins, off_xs_counters, off_xs_records, off_keys, off_buf, total;
 };
 
 // Records reserved per row: the capacity itself, or -- when k is too large for the single-CTA
@@ -86,7 +87,9 @@ WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k) {
     const bool xs = rows <= XS_MAX_ROWS && k <= (int64_t)SORT_CAP_MAX;
     l.off_xs_counters = align_up(l.off_bins + bins_bytes, 256);
     l.off_xs_records = align_up(l.off_xs_counters + (xs ? XS_MAX_SEGMENTS * sizeof(uint32_t) : 0), 256);
-    l.off_buf = align_up(l.off_xs_records + (xs ? (size_t)XS_MAX_SEGMENTS * (size_t)(k + XS_EDGE) * sizeof(uint64_t) : 0), 256);
+    // keys of the sample when a kernel of its own gathers them (few rows only)
+    l.off_keys = align_up(l.off_xs_records + (xs ? (size_t)XS_MAX_SEGMENTS * (size_t)(k + XS_EDGE) * sizeof(uint64_t) : 0), 256);
+    l.off_buf = align_up(l.off_keys + (rows <= GATHER_MAX_ROWS ? (size_t)rows * (size_t)M_MAX * sizeof(uint32_t) : 0), 256);
     l.total = align_up(l.off_buf + (size_t)rows * (size_t)row_stride_for(capacity, k) * sizeof(uint64_t), 256);
     return l;
 }
@@ -175,9 +178,30 @@ int pick_cluster(int64_t rows, int64_t m, int max_cluster) {
 
 template <typename T>
 int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, int64_t m, int64_t r, uint64_t seed, T* tau, RowCtl* ctl,
-                         WsHeader* header, uint32_t capacity, uint32_t* sample_idx, cudaStream_t st) {
+                         WsHeader* header, uint32_t capacity, uint32_t* sample_idx, uint32_t* keys_scratch, cudaStream_t st) {
     const int csize = pick_cluster(rows, m, di.max_cluster[dtype_index<T>()]);
+    // A large sample, or a sample of a very long row (every element on a page of its own), is gathered by a
+    // kernel over all SMs first; the cluster then only selects.
+    const bool spread_gather = keys_scratch != nullptr && rows <= GATHER_MAX_ROWS &&
+                               (m > 65536 || (int64_t)N * (int64_t)sizeof(T) >= (512LL << 20));
+    if (spread_gather) {
+        GatherParams<T> gp;
+        gp.in = in; gp.N = (uint64_t)N; gp.rows = (uint64_t)rows; gp.S = (uint32_t)m; gp.seed = seed;
+        gp.q = (uint64_t)(N / m); gp.rem = (uint32_t)(N % m); gp.inv_s = 1.0f / (float)m; gp.keys_out = keys_scratch;
+        const int64_t pairs = rows * ((m + 1) / 2);
+        cudaLaunchConfig_t gcfg = {};
+        gcfg.gridDim = dim3((unsigned)((pairs + GATHER_THREADS - 1) / GATHER_THREADS));
+        gcfg.blockDim = dim3(GATHER_THREADS);
+        gcfg.stream = st;
+        cudaLaunchAttribute gattr[1];
+        gattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        gattr[0].val.programmaticStreamSerializationAllowed = 1;
+        gcfg.attrs = gattr; gcfg.numAttrs = 1;
+        CUDA_TRY(cudaLaunchKernelEx(&gcfg, gather_kernel<T>, gp));
+        ++g_launches;
+    }
     SelectParams<T> sp;
+    sp.keys_in = spread_gather ? keys_scratch : nullptr;
     sp.in = in; sp.N = (uint64_t)N; sp.S = (uint32_t)m; sp.t = (uint32_t)r; sp.seed = seed;
     sp.per_cta = (uint32_t)(((m + csize - 1) / csize + 1) & ~1LL);      // even: samples are drawn in pairs
     sp.q = (uint64_t)(N / m); sp.rem = (uint32_t)(N % m); sp.inv_s = 1.0f / (float)m;
@@ -387,6 +411,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     uint32_t* bins = reinterpret_cast<uint32_t*>(base + lay.off_bins);
     uint32_t* xs_counters = reinterpret_cast<uint32_t*>(base + lay.off_xs_counters);
     uint64_t* xs_records = reinterpret_cast<uint64_t*>(base + lay.off_xs_records);
+    uint32_t* keys_scratch = reinterpret_cast<uint32_t*>(base + lay.off_keys);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
     // Survivors are staged per warp when a warp's tile is expected to hold a good fraction of one
@@ -400,7 +425,8 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     while (fb_sort_cap < (uint32_t)k && fb_sort_cap < SORT_CAP_MAX) fb_sort_cap <<= 1;
 
     if (plan->mode == 0) {
-        rc = launch_sample_select<T>(di, in, rows, N, plan->m, plan->r, seed, tau, ctl, header, (uint32_t)capacity, nullptr, st);
+        rc = launch_sample_select<T>(di, in, rows, N, plan->m, plan->r, seed, tau, ctl, header, (uint32_t)capacity, nullptr,
+                                     rows <= GATHER_MAX_ROWS ? keys_scratch : nullptr, st);
         if (rc != PROFK_OK) return rc;
         rc = launch_filter<T>(di, in, rows, N, tau, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, &header->tile_counter, st);
         if (rc != PROFK_OK) return rc;
@@ -495,7 +521,7 @@ int sample_threshold(const T* in, int64_t rows, int64_t N, int64_t m, int64_t r,
     DeviceInfo di;
     const int rc = ensure_device_info<T>(dev, &di);
     if (rc != PROFK_OK) return rc;
-    return launch_sample_select<T>(di, in, rows, N, m, r, seed, tau, nullptr, nullptr, 0, sample_idx, static_cast<cudaStream_t>(stream));
+    return launch_sample_select<T>(di, in, rows, N, m, r, seed, tau, nullptr, nullptr, 0, sample_idx, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 }  // namespace

@@ -27,7 +27,7 @@ namespace cg = cooperative_groups;
 constexpr int SEL_THREADS = 1024;
 constexpr int SEL_BINS = 2048;        // 11-bit digits
 constexpr int SEL_GROUPS = 128;       // groups of 8 lanes whose maxima bound the answer from below
-constexpr uint32_t SEL_CAND_CAP = 1024;
+constexpr uint32_t SEL_CAND_CAP = 4096;
 constexpr uint32_t SEL_SPREAD_MIN = 128;    // more candidates than this are ranked by all CTAs of the cluster
 
 // Per-row control block in the workspace.
@@ -69,6 +69,7 @@ template <typename T> struct SelectParams {
     WsHeader* header;      // may be null
     uint32_t capacity;
     uint32_t* sample_idx;  // may be null; rows x S
+    const uint32_t* keys_in;   // null, or rows x S keys of the sample gathered by gather_kernel before this one
 };
 
 // Writes tau for one row.
@@ -115,6 +116,57 @@ __device__ __forceinline__ uint32_t block_inclusive_scan(uint32_t v, uint32_t* w
     return v;
 }
 
+// Stage 1 on its own, over the whole GPU: the keys of the sampled elements of every row, in sample order.
+// One thread per pair of samples.  For a long row every sample lies on a page of its own, and the address
+// translations of a large sample take a 16-CTA cluster tens of microseconds; spread over all SMs they take a few.
+constexpr int GATHER_THREADS = 256;
+
+template <typename T> struct GatherParams {
+    const T* in;
+    uint64_t N;
+    uint64_t rows;
+    uint32_t S;
+    uint64_t seed;
+    uint64_t q;            // N / S
+    uint32_t rem;          // N % S
+    float inv_s;           // 1 / S
+    uint32_t* keys_out;    // rows x S
+};
+
+template <typename T>
+__global__ void __launch_bounds__(GATHER_THREADS) gather_kernel(const GatherParams<T> p) {
+    pdl_launch_dependents();
+    const uint64_t pairs = ((uint64_t)p.S + 1) / 2;
+    const uint64_t g = (uint64_t)blockIdx.x * GATHER_THREADS + threadIdx.x;
+    const bool active = g < p.rows * pairs;
+    const uint64_t row = active ? g / pairs : 0;
+    const uint64_t j = active ? 2 * (g % pairs) : 0;                 // even sample of the pair
+    const bool second = active && j + 1 < p.S;
+    const T* rowp = p.in + row * p.N;
+    uint32_t idx0 = 0, idx1 = 0;
+    if (active) {
+        const Philox4 r = philox4x32_10((uint32_t)(j >> 1), (uint32_t)row, (uint32_t)(row >> 32), 0u,
+                                        (uint32_t)p.seed, (uint32_t)(p.seed >> 32));
+        const uint64_t b0 = stratum_start(j, p.q, p.rem, p.S, p.inv_s);
+        const uint64_t b1 = stratum_start(j + 1, p.q, p.rem, p.S, p.inv_s);
+        idx0 = (uint32_t)(b0 + __umul64hi(((uint64_t)r.y << 32) | r.x, b1 - b0));
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(rowp + idx0));
+        if (second) {
+            const uint64_t b2 = stratum_start(j + 2, p.q, p.rem, p.S, p.inv_s);
+            idx1 = (uint32_t)(b1 + __umul64hi(((uint64_t)r.w << 32) | r.z, b2 - b1));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(rowp + idx1));
+        }
+    }
+    pdl_wait();                  // the positions needed nothing; the values need the work queued before this kernel
+    if (active) {
+        const T v0 = rowp[idx0];
+        const T v1 = second ? rowp[idx1] : v0;
+        uint32_t* out = p.keys_out + row * p.S + j;
+        out[0] = Elem<T>::key(v0);
+        if (second) out[1] = Elem<T>::key(v1);
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const SelectParams<T> p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -152,7 +204,17 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
     const T* rowp = p.in + row * p.N;
     uint32_t my_max = 0;
     constexpr int PB = 2;                                            // pairs per batch: 4 loads in flight per thread
-    for (uint32_t pp0 = 0; 2 * pp0 < n_local; pp0 += PB * SEL_THREADS) {
+    if (p.keys_in) {
+        // the sample was gathered by the kernel before this one: take this CTA's share of its keys
+        pdl_wait();
+        const uint32_t* src = p.keys_in + row * p.S + j0;
+        for (uint32_t i = tid; i < n_local; i += SEL_THREADS) {
+            const uint32_t k = __ldcg(&src[i]);
+            keys[i] = k;
+            my_max = max(my_max, k);
+        }
+    }
+    for (uint32_t pp0 = 0; !p.keys_in && 2 * pp0 < n_local; pp0 += PB * SEL_THREADS) {
         uint32_t idx[2 * PB];
         bool ok[2 * PB];
 #pragma unroll
