@@ -269,12 +269,8 @@ __device__ __noinline__ uint32_t filter_slow_path(const FilterParams<T>& p, Warp
 // written straight to the row buffer.  Returns the row if its buffer has overflowed, else ~0.
 template <typename T, int THREADS, int UNROLL>
 __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T>& p, const typename Elem<T>::vec_t (&v)[UNROLL],
-                                                            const bool (&inside)[UNROLL], uint32_t row, uint64_t qbase,
-                                                            uint32_t mis, T tau) {
+                                                            uint32_t inside_mask, uint32_t row, uint64_t qbase, uint32_t mis, T tau) {
     const unsigned lane = lane_id();
-    uint32_t inside_mask = 0;
-#pragma unroll
-    for (int u = 0; u < UNROLL; ++u) inside_mask |= inside[u] ? 1u << u : 0u;
     const uint32_t mine = survivor_mask<T, THREADS, UNROLL>(v, inside_mask, p.N, qbase, mis, tau);
     const unsigned cnt = __popc(mine);
     unsigned total;
@@ -310,18 +306,42 @@ __global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOC
         __syncwarp();
     }
 
+    constexpr int VEC = Elem<T>::VEC;
+    constexpr uint32_t ALL_INSIDE = (1u << UNROLL) - 1u;
     const uint32_t total_tiles = (uint32_t)p.total_tiles, tiles_per_row = (uint32_t)p.tiles_per_row;
+    const bool one_row = tiles_per_row == total_tiles;
     uint32_t tile = blockIdx.x;                  // the grid never exceeds the number of tiles (< 2^32)
 
-    // Decode the first tile and issue its loads before waiting on the threshold kernel:
-    // the input does not depend on it.
-    uint32_t row = tile / tiles_per_row;
-    uint64_t qbase = (uint64_t)(tile - row * tiles_per_row) * TILE_VECTORS;
-    RowView<T> rv = row_view(p.in, p.N, row);
+    uint32_t row = 0;
+    uint64_t qbase;                              // first vector of the tile inside its row
+    RowView<T> rv;
     V v[UNROLL];
-    bool inside[UNROLL];
+    uint32_t inside_mask;                        // bit u: vector u holds at least one element of the row
+    // Row and position of `tile`, and its loads.  A tile that lies wholly inside its row -- all but the first
+    // and the last of a row -- is four plain 128-bit loads off one pointer; the others take the checked path.
+    auto decode_and_load = [&](bool first_time) {
+        uint32_t nrow = 0, tin = tile;
+        if (!one_row) { nrow = tile / tiles_per_row; tin = tile - nrow * tiles_per_row; }
+        qbase = (uint64_t)tin * TILE_VECTORS;
+        if (first_time || nrow != row) { row = nrow; rv = row_view(p.in, p.N, row); }
+        if (qbase * VEC >= rv.mis && (qbase + TILE_VECTORS) * VEC <= p.N + rv.mis) {
+            const V* ptr = reinterpret_cast<const V*>(rv.aligned_base) + qbase + threadIdx.x;
 #pragma unroll
-    for (int u = 0; u < UNROLL; ++u) v[u] = load_row_vector(rv, p.N, qbase + (uint64_t)u * THREADS + threadIdx.x, &inside[u]);
+            for (int u = 0; u < UNROLL; ++u) v[u] = ld_stream(ptr + u * THREADS);
+            inside_mask = ALL_INSIDE;
+        } else {
+            inside_mask = 0;
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                bool in;
+                v[u] = load_row_vector(rv, p.N, qbase + (uint64_t)u * THREADS + threadIdx.x, &in);
+                inside_mask |= in ? 1u << u : 0u;
+            }
+        }
+    };
+
+    // The first tile's loads are issued before waiting on the threshold kernel: the input does not depend on it.
+    decode_and_load(true);
 
     PROFK_STAMP(0, 10);
     if (p.use_pdl) pdl_wait();
@@ -330,6 +350,7 @@ __global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOC
 
     uint32_t skip_row = 0xFFFFFFFFu;    // row whose buffer this warp has seen overflow: nothing more to append
     uint32_t parity = 0;
+    uint32_t tau_row = row;
     T tau = p.tau[row];
     while (true) {
         // Tiles below dyn_start follow the fixed stride and the warps run freely; the last few tiles of
@@ -343,19 +364,18 @@ __global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOC
         }
 
         bool hit = false;
+        if (inside_mask == ALL_INSIDE) {
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) hit |= (inside[u] && vec_any_pass(v[u], tau));
+            for (int u = 0; u < UNROLL; ++u) hit |= vec_any_pass(v[u], tau);
+        } else {
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) hit |= (((inside_mask >> u) & 1u) && vec_any_pass(v[u], tau));
+        }
 
         if (__any_sync(FULL_MASK, hit) && row != skip_row) {
             uint32_t o;
-            if (STAGED) {
-                uint32_t inside_mask = 0;
-#pragma unroll
-                for (int u = 0; u < UNROLL; ++u) inside_mask |= inside[u] ? 1u << u : 0u;
-                o = filter_slow_path<T, THREADS, UNROLL>(p, st, v[0], v[1], v[2], v[3], inside_mask, row, qbase, rv.mis, tau);
-            } else {
-                o = filter_slow_path_direct<T, THREADS, UNROLL>(p, v, inside, row, qbase, rv.mis, tau);
-            }
+            if (STAGED) o = filter_slow_path<T, THREADS, UNROLL>(p, st, v[0], v[1], v[2], v[3], inside_mask, row, qbase, rv.mis, tau);
+            else o = filter_slow_path_direct<T, THREADS, UNROLL>(p, v, inside_mask, row, qbase, rv.mis, tau);
             if (o != 0xFFFFFFFFu) skip_row = o;
         }
 
@@ -368,16 +388,12 @@ __global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOC
             tile = total_tiles - tile <= gridDim.x ? total_tiles : tile + gridDim.x;
         }
         if (tile >= total_tiles) break;
-        const uint32_t nrow = tile / tiles_per_row;
-        qbase = (uint64_t)(tile - nrow * tiles_per_row) * TILE_VECTORS;
-        if (nrow != row) { row = nrow; rv = row_view(p.in, p.N, row); tau = p.tau[row]; }
-        if (row == skip_row) {                   // this warp knows the row has overflowed: nothing to load
-#pragma unroll
-            for (int u = 0; u < UNROLL; ++u) inside[u] = false;
-            continue;
+        if (skip_row != 0xFFFFFFFFu && (one_row ? 0u : tile / tiles_per_row) == skip_row) {
+            inside_mask = 0;            // this warp knows the row has overflowed: nothing to load (it stays in the
+            continue;                   // loop: the hand-out of the last tiles is a matter for the whole CTA)
         }
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u) v[u] = load_row_vector(rv, p.N, qbase + (uint64_t)u * THREADS + threadIdx.x, &inside[u]);
+        decode_and_load(false);
+        if (row != tau_row) { tau_row = row; tau = p.tau[row]; }
     }
     if (STAGED && st->fill) flush_stage(p, st);
     PROFK_STAMP(0, 12);

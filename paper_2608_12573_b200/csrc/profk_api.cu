@@ -417,7 +417,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     // Survivors are staged per warp when a warp's tile is expected to hold a good fraction of one
     // (expected survivors per element ~ r / m); sparse survivors are appended directly.
     const double per_warp_tile = (double)plan->r / (double)std::max<int64_t>(plan->m, 1) * 32.0 * FILTER_UNROLL * Elem<T>::VEC;
-    const bool staged = plan->mode == 0 && rows == 1 && per_warp_tile > 0.1;
+    const bool staged = plan->mode == 0 && rows == 1 && per_warp_tile > 0.25;
 
     const int csize = (large || rows > XS_MAX_ROWS) ? 1 : refine_cluster_size<T>(di, rows, N);
     const bool exact_in_refine = csize > 1;
