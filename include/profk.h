@@ -91,8 +91,16 @@ typedef struct profk_plan {
     double p_overflow;
 } profk_plan_t;
 
-/* Tuning inputs of Algorithm 1; profk_plan uses the paper's defaults
- * s_min = 32768, s_max = 131072, cost_ratio (tau_B / tau_A) = 1. */
+/* Tuning inputs of Algorithm 1.  The paper's values (Section 4) are
+ * s_min = 32768, s_max = 131072, cost_ratio (tau_B / tau_A) = 1; profk_plan_ex
+ * takes them when `tuning` is NULL.  profk_plan and the profk_topk_* entry
+ * points use profk_default_tuning(N): the same, except that the floor on the
+ * sample size follows the row length for short rows,
+ *     s_min = min(32768, max(1024, N / 512)),
+ * because on this GPU a sample of 32768 elements touches every 128-byte line of
+ * a row of 2^20 elements (the sample pass would read the whole row) and rows of
+ * 2^16 elements would not be filtered at all.  Any choice keeps the failure
+ * budget: rank and capacity are derived from the bounds for the S in use. */
 typedef struct profk_tuning {
     int64_t s_min;
     int64_t s_max;
@@ -116,6 +124,7 @@ typedef struct profk_row_stats {
  * Returns PROFK_EINVAL on a bad argument.  profk_plan_ex takes the tuning
  * inputs explicitly (NULL = defaults).
  */
+int profk_default_tuning(int64_t N, profk_tuning_t* tuning /* [host] out */);
 int profk_plan(int64_t N, int64_t k, double eps, double recall, profk_plan_t* out);
 int profk_plan_ex(int64_t N, int64_t k, double eps, double recall, const profk_tuning_t* tuning,
                   profk_plan_t* out);

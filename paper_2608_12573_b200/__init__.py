@@ -16,7 +16,7 @@ _LIB = None
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libprofk.so")
 
 EXPORTS = [
-    "profk_plan", "profk_plan_ex", "profk_workspace_bytes", "profk_set_workspace",
+    "profk_plan", "profk_plan_ex", "profk_default_tuning", "profk_workspace_bytes", "profk_set_workspace",
     "profk_topk_f32", "profk_topk_bf16", "profk_topk_planned_f32", "profk_topk_planned_bf16",
     "profk_filter_f32", "profk_filter_bf16", "profk_sample_threshold_f32", "profk_sample_threshold_bf16",
     "profk_read_stats", "profk_last_launch_count", "profk_strerror", "profk_topk_noalloc_f32",
@@ -85,9 +85,22 @@ def _check(code: int, what: str) -> None:
 _plan_cache: dict = {}
 
 
+PAPER_TUNING = dict(s_min=32768, s_max=131072, cost_ratio=1.0)     # Section 4's values of the tuning inputs
+
+
+def default_tuning(N: int) -> dict:
+    """`profk_default_tuning`: the tuning inputs `plan` uses when none are given (the paper's, with the
+    floor on the sample size following the row length for short rows)."""
+    t = _TuningStruct(0, 0, 0.0)
+    _check(lib().profk_default_tuning(ctypes.c_int64(N), ctypes.byref(t)), "profk_default_tuning")
+    return dict(s_min=int(t.s_min), s_max=int(t.s_max), cost_ratio=float(t.cost_ratio))
+
+
 def plan(N: int, k: int, eps: float = 1e-3, recall: float = 1.0, s_min: int | None = None,
          s_max: int | None = None, cost_ratio: float | None = None) -> Plan:
-    """`profk_plan` / `profk_plan_ex`: the parameters (S, t, M) for one row of length N."""
+    """`profk_plan` / `profk_plan_ex`: the parameters (S, t, M) for one row of length N.  Without tuning
+    inputs: the library's defaults (`default_tuning`); `plan(N, k, eps, recall, **PAPER_TUNING)` gives the
+    paper's."""
     key = (N, k, eps, recall, s_min, s_max, cost_ratio)
     hit = _plan_cache.get(key)
     if hit is not None:

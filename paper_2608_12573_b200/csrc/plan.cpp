@@ -153,6 +153,24 @@ extern "C" int profk_plan_ex(int64_t N, int64_t k, double eps, double recall, co
     return PROFK_OK;
 }
 
+// The library's own choice of the tuning inputs.  Section 4's floor S_min = 32768 is kept for long rows.
+// For a short row it is lowered to N / 512 (not below 1024): on this GPU DRAM delivers 128 bytes per sampled
+// element, so 32768 samples of a 2^20-element row read the whole row once before the filtering scan reads
+// it again, and 2^16-element rows would not be filtered at all (N <= 2 S).  The guarded rank and capacity
+// keep the failure budget for any S.
+extern "C" int profk_default_tuning(int64_t N, profk_tuning_t* tuning) {
+    if (!tuning || N < 1) return PROFK_EINVAL;
+    int64_t s_min = N / 512;
+    if (s_min < 1024) s_min = 1024;
+    if (s_min > 32768) s_min = 32768;
+    tuning->s_min = s_min;
+    tuning->s_max = 131072;
+    tuning->cost_ratio = 1.0;
+    return PROFK_OK;
+}
+
 extern "C" int profk_plan(int64_t N, int64_t k, double eps, double recall, profk_plan_t* out) {
-    return profk_plan_ex(N, k, eps, recall, nullptr, out);
+    profk_tuning_t tuning;
+    if (profk_default_tuning(N, &tuning) != PROFK_OK) return PROFK_EINVAL;
+    return profk_plan_ex(N, k, eps, recall, &tuning, out);
 }

@@ -46,12 +46,12 @@ def test_config2_single_row_2p26():
                 v, i = run(xd, k, eps=eps, seed=seed)
                 assert np.array_equal(i, oi[:k]) and np.array_equal(bits(v), bits(ov[:k])), (k, eps, seed)
                 st = profk.read_stats(1)[0]
-                assert st[2] == o_plan.plan_guarded(1 << 26, k, eps).capacity
+                assert st[2] == o_plan.plan_guarded(1 << 26, k, eps, **profk.default_tuning(1 << 26)).capacity
                 fallbacks += st[3] != profk.ROW_OK
     assert fallbacks <= 2
     # relaxed recall 0.95: a prefix of the exact answer, at least k_accept long, then padding
     for k in (16, 256, 4096):
-        pl = o_plan.plan_guarded(1 << 26, k, 1e-2, recall=0.95)
+        pl = o_plan.plan_guarded(1 << 26, k, 1e-2, recall=0.95, **profk.default_tuning(1 << 26))
         v, i = run(xd, k, eps=1e-2, recall=0.95, seed=3)
         _, R, _, status = profk.read_stats(1)[0]
         n_real = min(k, R) if status == profk.ROW_OK else k
@@ -85,7 +85,7 @@ def test_config4_flattened_batchtopk_2p29_bf16():
         v, i = run(xd, k, eps=1e-3, seed=seed)
         assert o_topk.verify_topk(xn, k, v, i, keys=keys) == []
     st = profk.read_stats(1)[0]
-    assert st[2] == o_plan.plan_guarded(n, k, 1e-3).capacity
+    assert st[2] == o_plan.plan_guarded(n, k, 1e-3, **profk.default_tuning(n)).capacity
 
 
 @pytest.mark.parametrize("name", ["cauchy", "pareto", "sorted", "few_values", "spikes"])

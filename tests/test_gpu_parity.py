@@ -44,7 +44,7 @@ def test_config1_uniform_2p20_k64():
     v, i = gpu_topk(x, 64, eps=1e-3, seed=0)
     assert_exact(x, 64, v, i)
     tau_bits, R, cap, status = profk.read_stats(1)[0]
-    pl = o_plan.plan_guarded(1 << 20, 64, 1e-3)
+    pl = o_plan.plan_guarded(1 << 20, 64, 1e-3, **profk.default_tuning(1 << 20))     # the oracle's plan on the library's tuning inputs
     res = o_stages.run_row(workloads.as_numpy(x), 64, pl.m, pl.r, pl.capacity, pl.k_accept, seed=0)
     assert cap == pl.capacity
     assert tau_bits == int(np.asarray([res.tau]).view(np.uint32)[0])        # same sample, same threshold
@@ -88,7 +88,7 @@ def test_batched_rows(dtype):
     v, i = gpu_topk(x, 32, eps=1e-3, seed=9)
     assert_exact(x, 32, v, i)
     stats = profk.read_stats(24)
-    pl = o_plan.plan_guarded(1 << 17, 32, 1e-3)
+    pl = o_plan.plan_guarded(1 << 17, 32, 1e-3, **profk.default_tuning(1 << 17))
     xn = workloads.as_numpy(x)
     for r in (0, 7, 23):
         res = o_stages.run_row(xn[r], 32, pl.m, pl.r, pl.capacity, pl.k_accept, seed=9, row=r)
@@ -137,10 +137,14 @@ def test_k_equals_n_and_plan_direct_mode():
     x = workloads.normal(1, 5000, seed=13)[0]
     v, i = gpu_topk(x, 5000)
     assert_exact(x, 5000, v, i)
-    x = workloads.normal(3, 40_000, seed=14)                                 # N <= 2 S: plan says mode 1
-    assert profk.plan(40_000, 10).mode == 1
+    x = workloads.normal(3, 2_000, seed=14)                                  # N <= 2 S: plan says mode 1
+    assert profk.plan(2_000, 10).mode == 1
     v, i = gpu_topk(x, 10)
     assert_exact(x, 10, v, i)
+    x = workloads.normal(3, 40_000, seed=14)                                 # k so large that the buffer would hold half the row
+    assert profk.plan(40_000, 15_000).mode == 1
+    v, i = gpu_topk(x, 15_000)
+    assert_exact(x, 15_000, v, i)
 
 
 # ----------------------------------------------------------------------------- ties and special values

@@ -42,9 +42,16 @@ SHAPES = [(2 ** 20, 64, 1e-3, 1.0), (2 ** 26, 16, 1e-2, 1.0), (2 ** 26, 16, 1e-4
 
 
 @pytest.mark.parametrize("N,k,eps,recall", SHAPES)
-def test_host_plan_equals_oracle_plan(lib, N, k, eps, recall):
-    got = profk.plan(N, k, eps, recall)
-    want = oracle_plan.plan_guarded(N, k, eps, recall)
+@pytest.mark.parametrize("tuning", ["paper", "library"])
+def test_host_plan_equals_oracle_plan(lib, N, k, eps, recall, tuning):
+    if tuning == "paper":        # Section 4's S_min = 32768, S_max = 2^17, cost ratio 1: the oracle's defaults
+        got = profk.plan(N, k, eps, recall, **profk.PAPER_TUNING)
+        want = oracle_plan.plan_guarded(N, k, eps, recall)
+    else:                        # the library's own floor for short rows, handed to the oracle as a tuning input
+        s_min = min(32768, max(1024, N // 512))
+        assert profk.default_tuning(N) == dict(s_min=s_min, s_max=131072, cost_ratio=1.0)
+        got = profk.plan(N, k, eps, recall)
+        want = oracle_plan.plan_guarded(N, k, eps, recall, s_min=s_min)
     assert (got.m, got.r, got.capacity, got.k_accept, got.mode) == (want.m, want.r, want.capacity, want.k_accept, want.mode)
     assert got.z == pytest.approx(want.z, rel=1e-12)
     assert got.alpha == want.alpha
