@@ -42,7 +42,15 @@ template <typename T> struct FallbackParams {
     int use_pdl;              // 1 = launched as a programmatic dependent of the refine kernel
     T* out_vals;              // rows x k
     int64_t* out_idx;         // rows x k
+    // Many failed rows at once (a batch in direct mode, a batch of tie-flooded rows) are dealt out one per CTA
+    // instead: each CTA runs the exact selection of exact_select.cuh on its own.  Null = always row by row.
+    uint64_t* cta_records;    // gridDim.x x (k + XS_EDGE) records of scratch
+    uint32_t* cta_counters;   // gridDim.x counters
+    uint32_t sort_cap;        // power of two >= k: records the dynamic shared memory holds
 };
+
+static_assert(FB_BINS <= RF_BINS, "the grid-wide selection's histogram lives in SelectShared::hist");
+constexpr uint32_t FB_PARALLEL_MIN = 8;     // from this many failed rows on, one CTA per row beats the grid per row
 
 // Visits every element of `row` that falls to this CTA (tiles blockIdx.x, +gridDim.x, ...):
 // f(record, valid) is called by all 32 lanes of each warp together.
@@ -74,8 +82,9 @@ __device__ __forceinline__ void for_each_record(const FallbackParams<T>& p, uint
 
 template <typename T>
 __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackParams<T> p) {
-    __shared__ uint32_t sh_hist[FB_BINS];
-    __shared__ uint32_t warp_sums[32];
+    __shared__ SelectShared sh;                 // the per-CTA selection's state; its arrays also serve the grid-wide one
+    uint32_t* sh_hist = sh.hist;                // FB_BINS <= RF_BINS words
+    uint32_t* warp_sums = sh.warp_sums;
     __shared__ uint32_t flag_masks[FB_THREADS / 32];
     __shared__ uint32_t s_digit, s_before, s_cnt;
 
@@ -85,7 +94,27 @@ __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackPara
 
     // The count check was taken by the refine kernel (or, in direct mode, every row was marked by
     // the initialisation kernel): in the common case no row failed and this kernel is one load long.
-    if (__ldcg(&p.header->n_failed) == 0) return;
+    const uint32_t n_failed = __ldcg(&p.header->n_failed);
+    if (n_failed == 0) return;
+
+    if (p.cta_records && n_failed >= FB_PARALLEL_MIN) {
+        // ---- many rows: each CTA takes failed rows of its own (no grid barrier is reached) ----
+        extern __shared__ __align__(16) unsigned char fb_smem[];
+        uint64_t* sortbuf = reinterpret_cast<uint64_t*>(fb_smem);
+        const uint32_t slots = p.k + XS_EDGE;
+        uint64_t* recs = p.cta_records + (uint64_t)blockIdx.x * slots;
+        const uint64_t tiles = tiles_per_row<T>(p.N, FB_THREADS * XS_UNROLL);
+        for (uint64_t row = blockIdx.x; row < p.rows; row += gridDim.x) {
+            const uint32_t status = __ldcg(&p.ctl[row].status);
+            if (status == ROW_OK) continue;
+            const uint32_t tau_key = Elem<T>::key(Elem<T>::from_bits(__ldcg(&p.ctl[row].tau_bits)));
+            exact_select_cluster<T>(p.in, p.N, row, p.k, 0, tiles, recs, p.cta_counters + blockIdx.x, sh, 1u, 0u,
+                                    status == ROW_OVERFLOW, tau_key);
+            finish_from_segments<T>(recs, slots, p.k, p.sort_cap, sortbuf, sh, row, p.out_vals, p.out_idx);
+            __syncthreads();
+        }
+        return;
+    }
 
     uint32_t gen = *((volatile uint32_t*)&p.header->bar_gen);   // read before this CTA's first arrival
 

@@ -28,6 +28,7 @@ namespace {
 constexpr int FILTER_THREADS = PROFK_FILTER_THREADS;
 constexpr int FILTER_UNROLL = PROFK_FILTER_UNROLL;
 constexpr uint32_t SORT_CAP_MAX = 8192;          // largest k the single-CTA refine orders in shared memory
+constexpr unsigned FB_MAX_CTAS = 256;             // most CTAs of the grid-wide exact selection (its per-CTA scratch is sized for them)
 constexpr int64_t GATHER_MAX_ROWS = 4;           // most rows for which the sample may be gathered by a kernel of its own
 constexpr int LARGE_MAX_CTAS = 1024;             // CTAs of the large refine (its per-CTA slots live in the 48 KB histogram area)
 constexpr int64_t XS_MAX_ROWS = 18;              // most rows for which the refine kernel itself replaces failed rows
@@ -62,7 +63,7 @@ std::map<std::tuple<int64_t, int64_t, double, double>, profk_plan_t> g_plan_cach
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-    size_t off_header, off_ghist, off_ctl, off_tau, off_bins, off_xs_counters, off_xs_records, off_keys, off_buf, total;
+    size_t off_header, off_ghist, off_ctl, off_tau, off_bins, off_xs_counters, off_xs_records, off_keys, off_fb_counters, off_fb_records, off_buf, total;
 };
 
 // Records reserved per row: the capacity itself, or -- when k is too large for the single-CTA
@@ -89,7 +90,11 @@ WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k) {
     l.off_xs_records = align_up(l.off_xs_counters + (xs ? XS_MAX_SEGMENTS * sizeof(uint32_t) : 0), 256);
     // keys of the sample when a kernel of its own gathers them (few rows only)
     l.off_keys = align_up(l.off_xs_records + (xs ? (size_t)XS_MAX_SEGMENTS * (size_t)(k + XS_EDGE) * sizeof(uint64_t) : 0), 256);
-    l.off_buf = align_up(l.off_keys + (rows <= GATHER_MAX_ROWS ? (size_t)rows * (size_t)M_MAX * sizeof(uint32_t) : 0), 256);
+    // scratch of the grid-wide exact selection when it deals failed rows out one per CTA (many rows only)
+    const bool fbp = rows > XS_MAX_ROWS && k <= (int64_t)SORT_CAP_MAX;
+    l.off_fb_counters = align_up(l.off_keys + (rows <= GATHER_MAX_ROWS ? (size_t)rows * (size_t)M_MAX * sizeof(uint32_t) : 0), 256);
+    l.off_fb_records = align_up(l.off_fb_counters + (fbp ? FB_MAX_CTAS * sizeof(uint32_t) : 0), 256);
+    l.off_buf = align_up(l.off_fb_records + (fbp ? (size_t)FB_MAX_CTAS * (size_t)(k + XS_EDGE) * sizeof(uint64_t) : 0), 256);
     l.total = align_up(l.off_buf + (size_t)rows * (size_t)row_stride_for(capacity, k) * sizeof(uint64_t), 256);
     return l;
 }
@@ -458,8 +463,12 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         fb.tiles_per_row = tiles_per_row<T>((uint64_t)N, FB_THREADS * FB_UNROLL);
         fb.use_pdl = 0;
         fb.out_vals = out_vals; fb.out_idx = out_idx;
+        const bool fbp = rows > XS_MAX_ROWS && !large;
+        fb.cta_records = fbp ? reinterpret_cast<uint64_t*>(base + lay.off_fb_records) : nullptr;
+        fb.cta_counters = fbp ? reinterpret_cast<uint32_t*>(base + lay.off_fb_counters) : nullptr;
+        fb.sort_cap = fb_sort_cap;
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)di.sm_count);
+        cfg.gridDim = dim3(std::min<unsigned>((unsigned)di.sm_count, FB_MAX_CTAS));
         cfg.blockDim = dim3(FB_THREADS);
         cfg.dynamicSmemBytes = large ? 0 : (size_t)fb_sort_cap * 8;
         cfg.stream = st;

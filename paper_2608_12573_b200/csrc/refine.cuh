@@ -60,6 +60,30 @@ struct SegmentRecords {
     }
 };
 
+// The k smallest of the n records at `recs` (slots that hold all-ones are empty; at least k are not, and
+// recs[0] is one of them), ordered, as row `row` of the output.  One CTA; the records were written by other
+// CTAs, fenced, and are read through L2.
+template <typename T>
+__device__ __forceinline__ void finish_from_segments(const uint64_t* recs, uint32_t n, uint32_t k, uint32_t sort_cap,
+                                                     uint64_t* sortbuf, SelectShared& sh, uint64_t row, T* out_vals,
+                                                     int64_t* out_idx) {
+    const unsigned tid = threadIdx.x, nthr = blockDim.x, lane = lane_id();
+    if (tid == 0) { sh.or_bits = 0ull; sh.fill = 0; sh.n_edge = 0; }
+    __syncthreads();
+    const uint64_t first = __ldcg(&recs[0]);
+    uint64_t diff = 0;
+    for (uint32_t i = tid; i < n; i += nthr) {
+        const uint64_t rec = __ldcg(&recs[i]);
+        if (rec != ~0ull) diff |= rec ^ first;
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) diff |= __shfl_xor_sync(FULL_MASK, diff, d);
+    if (lane == 0 && diff) atomicOr(&sh.or_bits, (unsigned long long)diff);
+    __syncthreads();
+    select_smallest(SegmentRecords{recs, n}, first, k, sortbuf, sort_cap, sh);
+    sort_and_write<T>(sortbuf, k, k, k, row, out_vals, out_idx);
+}
+
 // The exact top-k of the full row, for a row that failed the count check (Section 3, "Refinement").
 // Cluster `seg` of the row's clusters selects the k smallest records (and a few more) of its segment of
 // the row; the cluster that finishes last merges: the k smallest of all segments' records, ordered, are
@@ -67,7 +91,7 @@ struct SegmentRecords {
 template <typename T>
 __device__ __noinline__ void exact_row(const RefineParams<T>& p, uint64_t row, unsigned seg, unsigned crank, uint64_t* sortbuf,
                                        SelectShared& sh, bool overflowed, uint32_t tau_key) {
-    const unsigned tid = threadIdx.x, nthr = blockDim.x, lane = lane_id();
+    const unsigned tid = threadIdx.x, nthr = blockDim.x;
     const unsigned csize = p.cluster_size, nseg = p.clusters_per_row;
     const uint64_t tiles = tiles_per_row<T>(p.N, nthr * XS_UNROLL);
     const uint64_t seg_lo = tiles * seg / nseg, seg_hi = tiles * (seg + 1) / nseg;
@@ -83,25 +107,12 @@ __device__ __noinline__ void exact_row(const RefineParams<T>& p, uint64_t row, u
         const bool last = ticket == nseg - 1;
         if (last) { p.ctl[row].collect = 0; __threadfence(); }
         sh.cnt = last ? 1u : 0u;
-        sh.or_bits = 0ull; sh.fill = 0; sh.n_edge = 0;
     }
     __syncthreads();
     if (sh.cnt == 0) return;
     __syncthreads();                         // sh.cnt is rewritten by the select below
 
-    const uint32_t n = nseg * slots;
-    const uint64_t first = __ldcg(&recs[0]);             // segment 0 is never empty
-    uint64_t diff = 0;
-    for (uint32_t i = tid; i < n; i += nthr) {
-        const uint64_t rec = __ldcg(&recs[i]);
-        if (rec != ~0ull) diff |= rec ^ first;
-    }
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) diff |= __shfl_xor_sync(FULL_MASK, diff, d);
-    if (lane == 0 && diff) atomicOr(&sh.or_bits, (unsigned long long)diff);
-    __syncthreads();
-    select_smallest(SegmentRecords{recs, n}, first, p.k, sortbuf, p.sort_cap, sh);
-    sort_and_write<T>(sortbuf, p.k, p.k, p.k, row, p.out_vals, p.out_idx);
+    finish_from_segments<T>(recs, nseg * slots, p.k, p.sort_cap, sortbuf, sh, row, p.out_vals, p.out_idx);
 }
 
 // Two builds of the kernel.  With up to 512 threads a refine CTA has to start beside the last CTAs

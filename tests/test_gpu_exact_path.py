@@ -128,6 +128,27 @@ def test_direct_mode_with_clusters(dtype):
         assert_exact(x, k, v, i)
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_direct_mode_and_failures_of_many_rows(dtype):
+    # many rows at once: the grid-wide kernel deals them out one per CTA
+    x = workloads.normal(300, 70_001, seed=27, dtype=dtype)
+    for k in (5, 2000):
+        v, i, st = forced(x.cuda(), k, profk.Plan(m=0, r=0, capacity=k, k_accept=k, mode=1))
+        assert all(s[3] == profk.ROW_DIRECT for s in st)
+        assert_exact(x, k, v, i)
+    v, i, st = forced(x.cuda(), 100, overflow_plan(100))
+    assert all(s[3] == profk.ROW_OVERFLOW for s in st)
+    assert_exact(x, 100, v, i)
+    x = torch.zeros((200, 50_000), dtype=dtype)                  # every row a flood of ties: lowest indices win
+    v, i, st = forced(x.cuda(), 64, overflow_plan(64))
+    assert np.array_equal(i, np.tile(np.arange(64), (200, 1)))
+    # the library's own plan for short rows of this kind
+    x = workloads.normal(2048, 1 << 16, seed=28, dtype=dtype)
+    v, i = profk.topk(x.cuda(), 8)
+    torch.cuda.synchronize()
+    assert_exact(x, 8, workloads.as_numpy(v), i.cpu().numpy())
+
+
 def test_special_values_in_the_exact_path():
     x = workloads.normal(1, 1_000_000, seed=26)[0]
     x[5] = float("nan"); x[77] = float("inf"); x[99_999] = float("inf"); x[123_456] = -float("inf")
