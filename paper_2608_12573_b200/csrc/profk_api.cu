@@ -125,12 +125,12 @@ template <typename T> int ensure_device_info(int dev, DeviceInfo* out) {
         di.filter_staged_blocks_per_sm[d] = std::max(nb, 1);
         CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fallback_kernel<T>, FB_THREADS, 0));
         di.fallback_blocks_per_sm[d] = std::max(nb, 1);
-        CUDA_TRY(cudaFuncSetAttribute(sample_select_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
+        CUDA_TRY(cudaFuncSetAttribute(sample_select_kernel<T, SEL_THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
         CUDA_TRY(cudaFuncSetAttribute(refine_kernel<T, 48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFINE_SMEM_MAX));
         CUDA_TRY(cudaFuncSetAttribute(refine_kernel<T, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFINE_SMEM_MAX));
         CUDA_TRY(cudaFuncSetAttribute(fallback_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SORT_CAP_MAX * 8)));
         // Clusters of 16 are beyond the portable size: allowed only where one actually fits.
-        if (cudaFuncSetAttribute(sample_select_kernel<T>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+        if (cudaFuncSetAttribute(sample_select_kernel<T, SEL_THREADS>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3(16); cfg.blockDim = dim3(SEL_THREADS); cfg.dynamicSmemBytes = 16384 * sizeof(uint32_t);
             cudaLaunchAttribute attr[1];
@@ -138,7 +138,7 @@ template <typename T> int ensure_device_info(int dev, DeviceInfo* out) {
             attr[0].val.clusterDim.x = 16; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
             cfg.attrs = attr; cfg.numAttrs = 1;
             int nclusters = 0;
-            if (cudaOccupancyMaxActiveClusters(&nclusters, sample_select_kernel<T>, &cfg) == cudaSuccess && nclusters >= 1)
+            if (cudaOccupancyMaxActiveClusters(&nclusters, sample_select_kernel<T, SEL_THREADS>, &cfg) == cudaSuccess && nclusters >= 1)
                 di.max_cluster[d] = 16;
         }
         (void)cudaGetLastError();
@@ -226,7 +226,13 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
     attr[1].id = cudaLaunchAttributeClusterDimension;
     attr[1].val.clusterDim.x = (unsigned)csize; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = csize > 1 ? 2 : 1;
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, sample_select_kernel<T>, sp));
+    // Batches of rows with small samples: one small CTA per row, four to an SM.
+    if (csize == 1 && m <= (int64_t)SEL_CAND_CAP && r <= SEL_SMALL_THREADS / 8 && !sp.keys_in) {
+        cfg.blockDim = dim3(SEL_SMALL_THREADS);
+        CUDA_TRY(cudaLaunchKernelEx(&cfg, sample_select_kernel<T, SEL_SMALL_THREADS>, sp));
+    } else {
+        CUDA_TRY(cudaLaunchKernelEx(&cfg, sample_select_kernel<T, SEL_THREADS>, sp));
+    }
     ++g_launches;
     return PROFK_OK;
 }

@@ -25,6 +25,7 @@ namespace profk {
 namespace cg = cooperative_groups;
 
 constexpr int SEL_THREADS = 1024;
+constexpr int SEL_SMALL_THREADS = 256;  // CTA size of the variant for batches of rows with small samples
 constexpr int SEL_BINS = 2048;        // 11-bit digits
 constexpr int SEL_GROUPS = 128;       // groups of 8 lanes whose maxima bound the answer from below
 constexpr uint32_t SEL_CAND_CAP = 4096;
@@ -167,13 +168,18 @@ __global__ void __launch_bounds__(GATHER_THREADS) gather_kernel(const GatherPara
     }
 }
 
-template <typename T>
-__global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const SelectParams<T> p) {
+// THREADS = THREADS is the general kernel.  THREADS = SEL_SMALL_THREADS is for batches of rows with small
+// samples (one CTA per row, at most SEL_CAND_CAP samples, rank at most THREADS / 8): four such CTAs share an
+// SM, so four times as many rows are in flight in a kernel that is all latency; it has no radix path, because
+// with so few samples all of them fit among the candidates.
+template <typename T, int THREADS>
+__global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sample_select_kernel(const SelectParams<T> p) {
+    constexpr int GROUPS = THREADS / 8;          // groups of 8 lanes whose maxima bound the answer from below
+    constexpr bool GENERAL = THREADS == SEL_THREADS;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw);          // per_cta keys
-    __shared__ uint32_t hist[2][SEL_BINS];                           // this CTA's histogram, double-buffered
     __shared__ uint32_t cand[SEL_CAND_CAP];                          // candidates (filled in the first CTA only)
-    __shared__ uint32_t gmax[SEL_GROUPS];
+    __shared__ uint32_t gmax[GROUPS];
     __shared__ uint32_t warp_sums[32];
     __shared__ uint32_t s_digit, s_before, s_ncand, s_lower;
 
@@ -208,18 +214,18 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
         // the sample was gathered by the kernel before this one: take this CTA's share of its keys
         pdl_wait();
         const uint32_t* src = p.keys_in + row * p.S + j0;
-        for (uint32_t i = tid; i < n_local; i += SEL_THREADS) {
+        for (uint32_t i = tid; i < n_local; i += THREADS) {
             const uint32_t k = __ldcg(&src[i]);
             keys[i] = k;
             my_max = max(my_max, k);
         }
     }
-    for (uint32_t pp0 = 0; !p.keys_in && 2 * pp0 < n_local; pp0 += PB * SEL_THREADS) {
+    for (uint32_t pp0 = 0; !p.keys_in && 2 * pp0 < n_local; pp0 += PB * THREADS) {
         uint32_t idx[2 * PB];
         bool ok[2 * PB];
 #pragma unroll
         for (int b = 0; b < PB; ++b) {
-            const uint32_t pp = pp0 + b * SEL_THREADS + tid;
+            const uint32_t pp = pp0 + b * THREADS + tid;
             const uint64_t j = (uint64_t)j0 + 2ull * pp;             // even sample of the pair
             ok[2 * b] = j < j1;
             ok[2 * b + 1] = j + 1 < j1;
@@ -253,7 +259,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
 #pragma unroll
         for (int s = 0; s < 2 * PB; ++s) {
             if (ok[s]) {
-                const uint32_t pp = pp0 + (s >> 1) * SEL_THREADS + tid;
+                const uint32_t pp = pp0 + (s >> 1) * THREADS + tid;
                 const uint32_t local = 2 * pp + (s & 1);
                 const uint32_t k = Elem<T>::key(val[s]);
                 keys[local] = k;
@@ -275,8 +281,10 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
     bool done = false;
 
     // ---- stage 2, short cut for small ranks -------------------------------------------
-    if (p.t <= SEL_GROUPS) {
-        // maxima of the 128 groups of 8 consecutive lanes
+    const bool bounded = p.t <= (uint32_t)GROUPS;
+    if (bounded || !GENERAL) {
+        if (bounded) {
+        // maxima of the groups of 8 consecutive lanes
         uint32_t g = my_max;
         g = max(g, __shfl_xor_sync(FULL_MASK, g, 1));
         g = max(g, __shfl_xor_sync(FULL_MASK, g, 2));
@@ -288,8 +296,8 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
             const uint32_t mine = gmax[grp];
             uint32_t rank = 0;
 #pragma unroll
-            for (int jj = 0; jj < SEL_GROUPS / 8; ++jj) {
-                const unsigned j = part * (SEL_GROUPS / 8) + jj;
+            for (int jj = 0; jj < GROUPS / 8; ++jj) {
+                const unsigned j = part * (GROUPS / 8) + jj;
                 const uint32_t o = gmax[j];
                 rank += (o > mine) || (o == mine && j < grp);
             }
@@ -298,6 +306,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
             rank += __shfl_xor_sync(FULL_MASK, rank, 4);
             if (part == 0 && rank == p.t - 1) s_lower = mine;     // at least t keys of this CTA are >= mine
         }
+        }                                   // (not bounded: the bound stays 0 and every key is a candidate)
         __syncthreads();
         const uint32_t lower = s_lower;
         PROFK_STAMP(0, 2);
@@ -305,7 +314,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
         uint32_t* cand0 = cluster.map_shared_rank(cand, 0);
         uint32_t* ncand0 = cluster.map_shared_rank(&s_ncand, 0);
         cluster.barrier_wait(std::move(zeroed));
-        for (uint32_t i = tid; i < n_round; i += SEL_THREADS) {
+        for (uint32_t i = tid; i < n_round; i += THREADS) {
             const uint32_t k = i < n_local ? keys[i] : 0;
             const bool take = i < n_local && k >= lower;
             const unsigned bal = __ballot_sync(FULL_MASK, take);
@@ -329,13 +338,13 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
             // A handful of candidates (small ranks) is not worth the copies: the first CTA looks at all.
             const bool spread = ncand > SEL_SPREAD_MIN;
             if (spread && crank != 0)
-                for (uint32_t i = tid; i < ncand; i += SEL_THREADS) cand[i] = cand0[i];
+                for (uint32_t i = tid; i < ncand; i += THREADS) cand[i] = cand0[i];
             auto seen = cluster.barrier_arrive();     // "I have read the first CTA's memory": it may leave after its peers did
             if (spread) __syncthreads();
             PROFK_STAMP(0, 7);
             const unsigned part = tid & 7u;
             const uint32_t c_first = spread ? (tid >> 3) * csize + crank : crank == 0 ? (tid >> 3) : ncand;
-            const uint32_t c_step = (SEL_THREADS / 8) * (spread ? csize : 1u);
+            const uint32_t c_step = (THREADS / 8) * (spread ? csize : 1u);
             for (uint32_t c = c_first; c < ncand; c += c_step) {      // whole groups of eight lanes together
                 const uint32_t mine = cand[c];
                 uint32_t above = 0, at_or_above = 0;
@@ -365,7 +374,9 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
     }
 
     // ---- stage 2, general case: radix select over the cluster --------------------------
+    if constexpr (GENERAL) {
     if (!done) {
+        __shared__ uint32_t hist[2][SEL_BINS];                       // this CTA's histogram, double-buffered
         constexpr int NPASS = sizeof(T) == 4 ? 3 : 2;
         constexpr int KB = Elem<T>::KEY_BITS;
         const int shifts[3] = {KB - 11, sizeof(T) == 4 ? 10 : 0, 0};
@@ -378,9 +389,9 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
             const int shift = shifts[pass], width = widths[pass];
             const uint32_t nbins = 1u << width;
             uint32_t* h = hist[pass & 1];
-            for (uint32_t b = tid; b < nbins; b += SEL_THREADS) h[b] = 0;
+            for (uint32_t b = tid; b < nbins; b += THREADS) h[b] = 0;
             __syncthreads();
-            for (uint32_t i = tid; i < n_round; i += SEL_THREADS) {
+            for (uint32_t i = tid; i < n_round; i += THREADS) {
                 const uint32_t k = i < n_local ? keys[i] : 0;
                 const bool in_class = i < n_local && (consumed == 0 || (k >> (KB - consumed)) == prefix);
                 const uint32_t digit = in_class ? (k >> shift) & (nbins - 1) : 0xFFFFFFFFu;
@@ -413,6 +424,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) sample_select_kernel(const Sel
         const uint32_t tau_key = prefix << (KB - consumed);
         if (crank == 0 && tid == 0) publish_threshold(p, row, tau_key);
         cluster.sync();   // no CTA leaves while a peer may still read its histogram
+    }
     }
     PROFK_STAMP(0, 6);
 }
