@@ -30,6 +30,10 @@
  *     -NaN < -inf < ... < -0 < +0 < ... < +inf < +NaN of their bit patterns.
  *   - Limits: 1 <= k <= N <= 2^32 - 2^24 per row, rows >= 1, rows * capacity < 2^40.
  *   - Two calls that use the same workspace must not overlap on the device.
+ *   - The kernels of a call are enqueued as programmatic dependents of one
+ *     another and of whatever precedes the call on the stream: each waits for
+ *     the work before it (griddepcontrol.wait) before it reads the input or
+ *     touches the workspace, so ordinary stream order is all a caller relies on.
  */
 #ifndef PROFK_H
 #define PROFK_H
@@ -122,7 +126,8 @@ typedef struct profk_row_stats {
  *   recall    1.0 = exact mode; rho in (0,1) = relaxed mode (accept ceil(rho k) survivors)
  *   out       [host] receives the plan
  * Returns PROFK_EINVAL on a bad argument.  profk_plan_ex takes the tuning
- * inputs explicitly (NULL = defaults).
+ * inputs explicitly (NULL = the paper's constants); profk_default_tuning
+ * writes the ones profk_plan uses for a row of length N.
  */
 int profk_default_tuning(int64_t N, profk_tuning_t* tuning /* [host] out */);
 int profk_plan(int64_t N, int64_t k, double eps, double recall, profk_plan_t* out);
