@@ -26,8 +26,8 @@
 #ifndef PROFK_FILTER_MINBLOCKS_BF16
 #define PROFK_FILTER_MINBLOCKS_BF16 3            // the direct-append variant fits 40 registers without spills
 #endif
-#ifndef PROFK_FILTER_MINBLOCKS_BF16_STAGED
-#define PROFK_FILTER_MINBLOCKS_BF16_STAGED 2     // the staged variant does not: it spills at 40 and loses more than it gains
+#ifndef PROFK_FILTER_MINBLOCKS_STAGED
+#define PROFK_FILTER_MINBLOCKS_STAGED 2          // the staged variants do not: they spill at 40 and lose more than they gain
 #endif
 
 namespace profk {
@@ -296,7 +296,7 @@ __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T
 // less bandwidth take fewer of them and all CTAs finish together.  The counter is read one tile
 // ahead, so its round trip hides behind the loads; only this tail needs a CTA barrier per tile.
 template <typename T, int THREADS, int UNROLL, bool STAGED>
-__global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOCKS_F32 : STAGED ? PROFK_FILTER_MINBLOCKS_BF16_STAGED : PROFK_FILTER_MINBLOCKS_BF16) filter_kernel(const __grid_constant__ FilterParams<T> p) {
+__global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGED : sizeof(T) == 4 ? PROFK_FILTER_MINBLOCKS_F32 : PROFK_FILTER_MINBLOCKS_BF16) filter_kernel(const __grid_constant__ FilterParams<T> p) {
     using V = typename Elem<T>::vec_t;
     constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
     __shared__ WarpStage stages[STAGED ? THREADS / 32 : 1];
