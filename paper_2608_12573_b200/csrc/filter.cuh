@@ -47,7 +47,16 @@ template <typename T> struct FilterParams {
     int use_pdl;             // 1 = launched as a programmatic dependent of the threshold kernel
     uint32_t* tile_counter;  // zeroed counter that hands out the tiles from dyn_start on (null = fixed stride throughout)
     uint32_t dyn_start;      // first tile handed out dynamically (a multiple of the grid size)
+    // Partitioned append (the PARTS build of the kernel only).  With very many survivors the single counter of a
+    // row becomes the bottleneck -- atomics on one address retire about 2 ns apart, 164 K of them are a quarter of
+    // a 2^30-element scan -- so the row's buffer is cut into FILTER_PARTS equal parts, each with a counter in a
+    // cache line of its own, and a CTA appends to part blockIdx.x mod FILTER_PARTS.
+    uint32_t part_cap;       // records per part
+    uint32_t* part_counts;   // row r, part j: part_counts[(r * FILTER_PARTS + j) * FILTER_PART_STRIDE] (zeroed)
 };
+
+constexpr uint32_t FILTER_PARTS = 8;
+constexpr uint32_t FILTER_PART_STRIDE = 64;     // words between two counters: 256 bytes
 
 // not (x < tau) for every lane of a vector, OR-ed: does the vector hold any survivor?
 __device__ __forceinline__ bool vec_any_pass(const float4& v, float tau) {
@@ -270,7 +279,7 @@ __device__ __noinline__ uint32_t filter_slow_path(const FilterParams<T>& p, Warp
 
 // The slow path without staging (sparse survivors): one global atomic per warp and tile, records
 // written straight to the row buffer.  Returns the row if its buffer has overflowed, else ~0.
-template <typename T, int THREADS, int UNROLL>
+template <typename T, int THREADS, int UNROLL, bool PARTS>
 __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T>& p, const typename Elem<T>::vec_t (&v)[UNROLL],
                                                             uint32_t inside_mask, uint32_t row, uint64_t qbase, uint32_t mis, T tau) {
     const unsigned lane = lane_id();
@@ -279,11 +288,20 @@ __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T
     unsigned total;
     const unsigned before = warp_exclusive_count(cnt, lane, &total);
     if (total == 0) return 0xFFFFFFFFu;
+    uint32_t* counter = p.counts + (uint64_t)row * p.count_stride;
+    uint64_t* dst = p.buf + (uint64_t)row * p.buf_stride;
+    uint32_t cap = p.capacity;
+    if (PARTS) {
+        const uint32_t part = blockIdx.x % FILTER_PARTS;
+        counter = p.part_counts + ((uint64_t)row * FILTER_PARTS + part) * FILTER_PART_STRIDE;
+        dst += (uint64_t)part * p.part_cap;
+        cap = p.part_cap;
+    }
     unsigned base = 0;
-    if (lane == 0) base = atomicAdd(p.counts + (uint64_t)row * p.count_stride, total);
+    if (lane == 0) base = atomicAdd(counter, total);
     base = __shfl_sync(FULL_MASK, base, 0);
-    if (cnt) emit_survivors<T, THREADS, UNROLL>(v, mine, qbase, mis, p.buf + (uint64_t)row * p.buf_stride, base + before, p.capacity);
-    return (uint64_t)base + total > p.capacity ? row : 0xFFFFFFFFu;
+    if (cnt) emit_survivors<T, THREADS, UNROLL>(v, mine, qbase, mis, dst, base + before, cap);
+    return (uint64_t)base + total > cap ? row : 0xFFFFFFFFu;
 }
 
 // STAGED = collect survivors in per-warp shared-memory stages (dense survivors, one row at a time);
@@ -295,7 +313,7 @@ __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T
 // tiles of the launch (from dyn_start on) come from a global counter instead, so that SMs that saw
 // less bandwidth take fewer of them and all CTAs finish together.  The counter is read one tile
 // ahead, so its round trip hides behind the loads; only this tail needs a CTA barrier per tile.
-template <typename T, int THREADS, int UNROLL, bool STAGED>
+template <typename T, int THREADS, int UNROLL, bool STAGED, bool PARTS = false>
 __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGED : sizeof(T) == 4 ? PROFK_FILTER_MINBLOCKS_F32 : PROFK_FILTER_MINBLOCKS_BF16) filter_kernel(const __grid_constant__ FilterParams<T> p) {
     using V = typename Elem<T>::vec_t;
     constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
@@ -378,7 +396,7 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
         if (__any_sync(FULL_MASK, hit) && row != skip_row) {
             uint32_t o;
             if (STAGED) o = filter_slow_path<T, THREADS, UNROLL>(p, st, v[0], v[1], v[2], v[3], inside_mask, row, qbase, rv.mis, tau);
-            else o = filter_slow_path_direct<T, THREADS, UNROLL>(p, v, inside_mask, row, qbase, rv.mis, tau);
+            else o = filter_slow_path_direct<T, THREADS, UNROLL, PARTS>(p, v, inside_mask, row, qbase, rv.mis, tau);
             if (o != 0xFFFFFFFFu) skip_row = o;
         }
 

@@ -63,7 +63,7 @@ std::map<std::tuple<int64_t, int64_t, double, double>, profk_plan_t> g_plan_cach
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-    size_t off_header, off_ghist, off_ctl, off_tau, off_bins, off_xs_counters, off_xs_records, off_keys, off_fb_counters, off_fb_records, off_buf, total;
+    size_t off_header, off_ghist, off_ctl, off_tau, off_bins, off_xs_counters, off_xs_records, off_keys, off_fb_counters, off_fb_records, off_parts, off_buf, total;
 };
 
 // Records reserved per row: the capacity itself, or -- when k is too large for the single-CTA
@@ -94,7 +94,9 @@ WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k) {
     const bool fbp = rows > XS_MAX_ROWS && k <= (int64_t)SORT_CAP_MAX;
     l.off_fb_counters = align_up(l.off_keys + (rows <= GATHER_MAX_ROWS ? (size_t)rows * (size_t)M_MAX * sizeof(uint32_t) : 0), 256);
     l.off_fb_records = align_up(l.off_fb_counters + (fbp ? FB_MAX_CTAS * sizeof(uint32_t) : 0), 256);
-    l.off_buf = align_up(l.off_fb_records + (fbp ? (size_t)FB_MAX_CTAS * (size_t)(k + XS_EDGE) * sizeof(uint64_t) : 0), 256);
+    // counters of the partitioned append (large selections only), each in a 256-byte line of its own
+    l.off_parts = align_up(l.off_fb_records + (fbp ? (size_t)FB_MAX_CTAS * (size_t)(k + XS_EDGE) * sizeof(uint64_t) : 0), 256);
+    l.off_buf = align_up(l.off_parts + (k > (int64_t)SORT_CAP_MAX ? (size_t)rows * FILTER_PARTS * FILTER_PART_STRIDE * sizeof(uint32_t) : 0), 256);
     l.total = align_up(l.off_buf + (size_t)rows * (size_t)row_stride_for(capacity, k) * sizeof(uint64_t), 256);
     return l;
 }
@@ -183,7 +185,8 @@ int pick_cluster(int64_t rows, int64_t m, int max_cluster) {
 
 template <typename T>
 int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, int64_t m, int64_t r, uint64_t seed, T* tau, RowCtl* ctl,
-                         WsHeader* header, uint32_t capacity, uint32_t* sample_idx, uint32_t* keys_scratch, cudaStream_t st) {
+                         WsHeader* header, uint32_t capacity, uint32_t* sample_idx, uint32_t* keys_scratch, uint32_t* part_counts,
+                         cudaStream_t st) {
     const int csize = pick_cluster(rows, m, di.max_cluster[dtype_index<T>()]);
     // A large sample, or a sample of a very long row (every element on a page of its own), is gathered by a
     // kernel over all SMs first; the cluster then only selects.
@@ -207,6 +210,7 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
     }
     SelectParams<T> sp;
     sp.keys_in = spread_gather ? keys_scratch : nullptr;
+    sp.part_counts = part_counts;
     sp.in = in; sp.N = (uint64_t)N; sp.S = (uint32_t)m; sp.t = (uint32_t)r; sp.seed = seed;
     sp.per_cta = (uint32_t)(((m + csize - 1) / csize + 1) & ~1LL);      // even: samples are drawn in pairs
     sp.q = (uint64_t)(N / m); sp.rem = (uint32_t)(N % m); sp.inv_s = 1.0f / (float)m;
@@ -239,7 +243,8 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
 
 template <typename T>
 int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, const T* tau, int64_t capacity, uint64_t* buf,
-                  uint64_t buf_stride, uint32_t* counts, uint32_t count_stride, bool pdl, bool staged, uint32_t* tile_counter, cudaStream_t st) {
+                  uint64_t buf_stride, uint32_t* counts, uint32_t count_stride, bool pdl, bool staged, uint32_t* tile_counter, bool parts,
+                  uint32_t part_cap, uint32_t* part_counts, cudaStream_t st) {
     FilterParams<T> fp;
     fp.in = in; fp.N = (uint64_t)N; fp.rows = (uint64_t)rows; fp.tau = tau; fp.capacity = (uint32_t)capacity;
     fp.buf = buf; fp.buf_stride = buf_stride; fp.counts = counts; fp.count_stride = count_stride;
@@ -248,6 +253,7 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     if (fp.total_tiles >= (1ull << 32)) return PROFK_EINVAL;      // rows * N beyond 2^45 elements
     fp.use_pdl = pdl ? 1 : 0;
     fp.tile_counter = tile_counter;
+    fp.part_cap = part_cap; fp.part_counts = part_counts;
     const uint64_t max_grid = (uint64_t)di.sm_count *
         (staged ? di.filter_staged_blocks_per_sm[dtype_index<T>()] : di.filter_blocks_per_sm[dtype_index<T>()]);
     cudaLaunchConfig_t cfg = {};
@@ -264,6 +270,7 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
     if (staged) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, true>, fp));
+    else if (parts) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false, true>, fp));
     else CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false>, fp));
     ++g_launches;
     return PROFK_OK;
@@ -301,10 +308,11 @@ int launch_cooperative(cudaLaunchConfig_t cfg, Kernel kernel, Params params, boo
 // Count check + ordering for large selections: the whole grid, one CTA per SM, one row after the other.
 template <typename T>
 int launch_refine_large(const DeviceInfo& di, RowCtl* ctl, WsHeader* header, uint64_t* buf, uint64_t row_pitch, uint32_t* bins,
-                        unsigned long long* slots, int64_t rows, int64_t capacity, int64_t k, int64_t k_accept, int phase, T* out_vals,
-                        int64_t* out_idx, cudaStream_t st) {
+                        unsigned long long* slots, bool parts, uint32_t part_cap, const uint32_t* part_counts, int64_t rows,
+                        int64_t capacity, int64_t k, int64_t k_accept, int phase, T* out_vals, int64_t* out_idx, cudaStream_t st) {
     LargeParams<T> lp;
     lp.ctl = ctl; lp.header = header; lp.buf = buf; lp.row_stride = row_pitch / 2; lp.bins = bins; lp.slots = slots;
+    lp.parts = (phase == 0 && parts) ? FILTER_PARTS : 1u; lp.part_cap = part_cap; lp.part_counts = part_counts;
     lp.rows = (uint64_t)rows; lp.capacity = (uint32_t)capacity;
     lp.k = (uint32_t)k; lp.k_accept = (uint32_t)k_accept; lp.phase = phase; lp.out_vals = out_vals; lp.out_idx = out_idx;
     lp.use_pdl = 0;
@@ -430,6 +438,12 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     const double per_warp_tile = (double)plan->r / (double)std::max<int64_t>(plan->m, 1) * 32.0 * FILTER_UNROLL * Elem<T>::VEC;
     const bool staged = plan->mode == 0 && rows == 1 && per_warp_tile > 0.25;
 
+    // Large selections keep so many survivors that a row's single append counter would hold the scan up:
+    // the direct variant then appends to FILTER_PARTS parts of the buffer, each with a counter of its own.
+    const bool parts = large && !staged && plan->mode == 0;
+    const uint32_t part_cap = (uint32_t)(row_stride / 2 / FILTER_PARTS);
+    uint32_t* part_counts = reinterpret_cast<uint32_t*>(base + lay.off_parts);
+
     const int csize = (large || rows > XS_MAX_ROWS) ? 1 : refine_cluster_size<T>(di, rows, N);
     const bool exact_in_refine = csize > 1;
     uint32_t fb_sort_cap = 32;
@@ -437,13 +451,15 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
 
     if (plan->mode == 0) {
         rc = launch_sample_select<T>(di, in, rows, N, plan->m, plan->r, seed, tau, ctl, header, (uint32_t)capacity, nullptr,
-                                     rows <= GATHER_MAX_ROWS ? keys_scratch : nullptr, st);
+                                     rows <= GATHER_MAX_ROWS ? keys_scratch : nullptr, parts ? part_counts : nullptr, st);
         if (rc != PROFK_OK) return rc;
-        rc = launch_filter<T>(di, in, rows, N, tau, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, &header->tile_counter, st);
+        rc = launch_filter<T>(di, in, rows, N, tau, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, &header->tile_counter,
+                              parts, part_cap, part_counts, st);
         if (rc != PROFK_OK) return rc;
 
         if (large) {
-            rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, reinterpret_cast<unsigned long long*>(ghist), rows, capacity, k, plan->k_accept, 0,
+            rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, reinterpret_cast<unsigned long long*>(ghist), parts, part_cap, part_counts, rows,
+                                        capacity, k, plan->k_accept, 0,
                                         out_vals, out_idx, st);
         } else {
             // count check and refine; with clusters, also the exact selection of the rows that fail the check
@@ -482,7 +498,8 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         if (rc != PROFK_OK) return rc;
     }
     if (large) {   // the rows the exact selection repaired still have to be ordered and written
-        rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, reinterpret_cast<unsigned long long*>(ghist), rows, capacity, k, k, 1, out_vals,
+        rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, reinterpret_cast<unsigned long long*>(ghist), false, part_cap, part_counts, rows,
+                                    capacity, k, k, 1, out_vals,
                                     out_idx, st);
         if (rc != PROFK_OK) return rc;
     }
@@ -522,7 +539,8 @@ int filter_only(const T* in, int64_t rows, int64_t N, const T* tau, int64_t capa
     DeviceInfo di;
     const int rc = ensure_device_info<T>(dev, &di);
     if (rc != PROFK_OK) return rc;
-    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, (uint64_t)capacity, counts, 1, false, false, nullptr, static_cast<cudaStream_t>(stream));
+    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, (uint64_t)capacity, counts, 1, false, false, nullptr, false, 0u, nullptr,
+                            static_cast<cudaStream_t>(stream));
 }
 
 template <typename T>
@@ -536,7 +554,8 @@ int sample_threshold(const T* in, int64_t rows, int64_t N, int64_t m, int64_t r,
     DeviceInfo di;
     const int rc = ensure_device_info<T>(dev, &di);
     if (rc != PROFK_OK) return rc;
-    return launch_sample_select<T>(di, in, rows, N, m, r, seed, tau, nullptr, nullptr, 0, sample_idx, nullptr, static_cast<cudaStream_t>(stream));
+    return launch_sample_select<T>(di, in, rows, N, m, r, seed, tau, nullptr, nullptr, 0, sample_idx, nullptr, nullptr,
+                                   static_cast<cudaStream_t>(stream));
 }
 
 }  // namespace

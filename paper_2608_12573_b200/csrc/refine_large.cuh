@@ -35,6 +35,9 @@ template <typename T> struct LargeParams {
     uint64_t row_stride;     //        row_stride is a power of two >= capacity, >= BT_TILE
     uint32_t* bins;          // rows x (LG_BINS + 8) words: bin counts / positions, then flags
     unsigned long long* slots;   // 2 words per CTA of the grid, then one per CTA: per-CTA minima / maxima and scan totals
+    uint32_t parts;          // 1, or 8: the filter appended to that many parts of the row's buffer (first phase only)
+    uint32_t part_cap;       // records per part
+    const uint32_t* part_counts;   // row r, part j: part_counts[(r * 8 + j) * 64]
     uint64_t rows;
     uint32_t capacity;
     uint32_t k;
@@ -90,10 +93,27 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         // ---- is this row for this launch?  (the decision is the same in every CTA) ----
         const RowCtl ctl = p.ctl[row];
         uint32_t n;
+        uint32_t nparts = 1, pcount[8] = {0, 0, 0, 0, 0, 0, 0, 0};      // the records are pcount[j] at G + j * part_cap
         if (p.phase == 0) {
-            const uint32_t R = ctl.count;
-            const uint32_t status = R > p.capacity ? ROW_OVERFLOW : R < p.k_accept ? ROW_RECALL : ROW_OK;
+            uint32_t R = ctl.count;
+            bool part_full = false;
+            if (p.parts > 1) {                   // partitioned append: the row's count is the sum of its parts'
+                nparts = 8;
+                uint64_t sum = 0;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint32_t c = p.part_counts[(row * 8 + j) * 64];
+                    part_full |= c > p.part_cap;
+                    pcount[j] = c < p.part_cap ? c : p.part_cap;
+                    sum += c;
+                }
+                R = sum > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)sum;
+            } else {
+                pcount[0] = R;
+            }
+            const uint32_t status = (R > p.capacity || part_full) ? ROW_OVERFLOW : R < p.k_accept ? ROW_RECALL : ROW_OK;
             if (cta == 0 && tid == 0) {
+                if (p.parts > 1) p.ctl[row].count = part_full && R <= p.capacity ? p.capacity + 1 : R;   // what the statistics report
                 p.ctl[row].status = status;
                 p.ctl[row].n_final = status ? p.k : R;
                 if (status) atomicAdd(&p.header->n_failed, 1u);
@@ -103,12 +123,20 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         } else {
             if (ctl.status == ROW_OK) continue;  // already written by the first phase
             n = p.k;                             // the exact selection left exactly k records
+            pcount[0] = n;
         }
         const uint32_t kk = n < p.k ? n : p.k;
         uint64_t* G = p.buf + row * 2 * p.row_stride;
         uint64_t* G2 = G + p.row_stride;
         uint32_t* bins = p.bins + row * (uint64_t)(LG_BINS + 8);
         uint32_t* flags = bins + LG_BINS;                                // [0] = some bin that matters is crowded
+        // every record of the row once, spread over the grid's threads
+        auto for_each_record = [&](auto&& f) {
+            for (uint32_t j = 0; j < nparts; ++j) {
+                const uint64_t* part = G + (uint64_t)j * p.part_cap;
+                for (uint64_t i = gid; i < pcount[j]; i += gthreads) f((unsigned long long)__ldcg(&part[i]));
+            }
+        };
 
         for (uint64_t j = kk + gid; j < p.k; j += gthreads) {            // relaxed mode: padding after a short buffer
             p.out_vals[row * (uint64_t)p.k + j] = Elem<T>::from_bits(Elem<T>::NEG_INF_BITS);
@@ -119,11 +147,10 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         // smallest and largest record of the row; clear the bins meanwhile
         for (uint64_t b = gid; b < LG_BINS + 8; b += gthreads) bins[b] = 0;
         unsigned long long lo = ~0ull, hi = 0ull;
-        for (uint64_t i = gid; i < n; i += gthreads) {
-            const unsigned long long rec = __ldcg(&G[i]);
+        for_each_record([&](unsigned long long rec) {
             lo = rec < lo ? rec : lo;
             hi = rec > hi ? rec : hi;
-        }
+        });
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) {
             const unsigned long long l2 = __shfl_xor_sync(FULL_MASK, lo, d), h2 = __shfl_xor_sync(FULL_MASK, hi, d);
@@ -160,7 +187,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         auto bin_of = [&](unsigned long long rec) { return (uint32_t)((rec - rmin) >> shift); };
 
         // histogram (global atomics spread over the bins)
-        for (uint64_t i = gid; i < n; i += gthreads) atomicAdd(&bins[bin_of(__ldcg(&G[i]))], 1u);
+        for_each_record([&](unsigned long long rec) { atomicAdd(&bins[bin_of(rec)], 1u); });
         if (!grid_barrier(p.header, gen)) return;
 
         // scan: CTA c < scan_ctas owns bins [c, c+1) * LG_BINS / scan_ctas; counts become first positions
@@ -207,10 +234,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
 
         if (__ldcg(&flags[0]) == 0) {
             // scatter into the second buffer, grouped by bin
-            for (uint64_t i = gid; i < n; i += gthreads) {
-                const unsigned long long rec = __ldcg(&G[i]);
-                G2[atomicAdd(&bins[bin_of(rec)], 1u)] = rec;
-            }
+            for_each_record([&](unsigned long long rec) { G2[atomicAdd(&bins[bin_of(rec)], 1u)] = rec; });
             if (!grid_barrier(p.header, gen)) return;
             // rank inside the bin: bin b now occupies [end of bin b-1, bins[b])
             // (only positions below the end of the bin that holds position kk-1 matter; they are a prefix)
@@ -229,6 +253,17 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         }
 
         // ================= reserve path: bitonic network =================
+        if (nparts > 1) {                        // it wants the records in one run: through the second buffer and back
+            uint64_t first = 0;
+            for (uint32_t j = 0; j < nparts; ++j) {
+                const uint64_t* part = G + (uint64_t)j * p.part_cap;
+                for (uint64_t i = gid; i < pcount[j]; i += gthreads) G2[first + i] = __ldcg(&part[i]);
+                first += pcount[j];
+            }
+            if (!grid_barrier(p.header, gen)) return;
+            for (uint64_t i = gid; i < n; i += gthreads) G[i] = __ldcg(&G2[i]);
+            if (!grid_barrier(p.header, gen)) return;
+        }
         uint64_t P = BT_TILE;
         while (P < n) P <<= 1;
 
