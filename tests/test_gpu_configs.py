@@ -103,3 +103,41 @@ def test_config5_adversarial_2p30(name):
             assert st[3] == profk.ROW_OVERFLOW               # ties flood the buffer: the exact path answers
     del xd
     torch.cuda.empty_cache()
+
+
+def test_longest_row_the_library_accepts():
+    """N = 2^32 - 2^24 (17 GB of fp32): the answer is planted, so it is known without a sort -- the background is
+    U[0,1), the k winners are distinct values above 1 at positions that include both ends of the row and both
+    sides of 2^31 and 2^32 - 2^25, where 32-bit index arithmetic would first go wrong."""
+    n = (1 << 32) - (1 << 24)
+    k = 300
+    free, _ = torch.cuda.mem_get_info()
+    if free < n * 4 + (2 << 30):
+        pytest.skip("not enough free device memory for a 17 GB row")
+    g = torch.Generator(device="cuda").manual_seed(41)
+    x = torch.empty(n, dtype=torch.float32, device="cuda")
+    step = 1 << 28
+    for lo in range(0, n, step):                                 # drawn in pieces: no second 17 GB temporary
+        hi = min(n, lo + step)
+        x[lo:hi].uniform_(0.0, 1.0, generator=g)
+    rng = np.random.default_rng(42)
+    special = np.array([0, 1, (1 << 31) - 1, 1 << 31, (1 << 31) + 1, (1 << 32) - (1 << 25) - 1, (1 << 32) - (1 << 25),
+                        n - 2, n - 1], dtype=np.int64)
+    others = rng.choice(n, size=k - len(special), replace=False).astype(np.int64)
+    pos = np.unique(np.concatenate([special, others]))
+    assert len(pos) == k
+    rng.shuffle(pos)
+    vals = (2.0 + np.arange(k, dtype=np.float64) * 2.0 ** -10).astype(np.float32)     # distinct, exactly representable
+    x[torch.from_numpy(pos).cuda()] = torch.from_numpy(vals).cuda()
+    for seed in (0, 1):
+        v, i = run(x, k, eps=1e-3, seed=seed)
+        order = np.argsort(-vals, kind="stable")
+        assert np.array_equal(i, pos[order]), "indices differ from the planted answer"
+        assert np.array_equal(bits(v), bits(vals[order])), "values differ from the planted answer"
+    st = profk.read_stats(1)[0]
+    assert st[3] == profk.ROW_OK and k <= st[1] <= st[2]
+    # and the exact replacement at this length: a buffer of k slots overflows at once
+    v, i = profk.topk(x, k, plan_override=profk.Plan(m=32768, r=3000, capacity=k, k_accept=k, mode=0), seed=2)
+    torch.cuda.synchronize()
+    assert profk.read_stats(1)[0][3] == profk.ROW_OVERFLOW
+    assert np.array_equal(i.cpu().numpy(), pos[order]) and np.array_equal(bits(workloads.as_numpy(v)), bits(vals[order]))

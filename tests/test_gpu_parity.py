@@ -278,3 +278,24 @@ def test_relaxed_recall_returns_a_padded_prefix():
     n_real = min(k, R) if status == profk.ROW_OK else k
     assert n_real >= pl.k_accept
     assert np.array_equal(i[:n_real], oi[:n_real])
+
+
+# ----------------------------------------------------------------------------- stream order
+def test_input_produced_on_the_stream_just_before_the_call():
+    # The first kernel of a call may be staged behind the work before it on the stream and must wait for that work
+    # before it reads the input: here the input is overwritten by a kernel queued right before every call, on a
+    # side stream, with no synchronisation in between.
+    n, k = 1 << 22, 100
+    side = torch.cuda.Stream()
+    x = torch.empty(n, device="cuda")
+    g = torch.Generator(device="cuda").manual_seed(7)
+    outs, snaps = [], []
+    with torch.cuda.stream(side):
+        for it in range(6):
+            x.normal_(generator=g)                   # producer kernel
+            v, i = profk.topk(x, k, seed=it)         # consumer, same stream
+            outs.append((v.clone(), i.clone()))
+            snaps.append(x.clone())                  # what the consumer must have seen
+    side.synchronize()
+    for (v, i), snap in zip(outs, snaps):
+        assert_exact(snap.cpu(), k, workloads.as_numpy(v), i.cpu().numpy())
