@@ -34,6 +34,8 @@
  *     another and of whatever precedes the call on the stream: each waits for
  *     the work before it (griddepcontrol.wait) before it reads the input or
  *     touches the workspace, so ordinary stream order is all a caller relies on.
+ *     A call can be captured into a CUDA graph once its shape has been used
+ *     outside a capture (the first use sets kernel attributes).
  */
 #ifndef PROFK_H
 #define PROFK_H

@@ -299,3 +299,25 @@ def test_input_produced_on_the_stream_just_before_the_call():
     side.synchronize()
     for (v, i), snap in zip(outs, snaps):
         assert_exact(snap.cpu(), k, workloads.as_numpy(v), i.cpu().numpy())
+
+
+def test_call_captured_in_a_cuda_graph():
+    # All launches of a call (cluster launches, programmatic dependents, the cooperative kernels of the many-row
+    # and large-k paths) can be captured once and replayed on new data.
+    for rows, n, k in [(1, 1 << 22, 128), (64, 1 << 16, 16), (1, 1 << 22, 20000)]:
+        x = torch.empty((rows, n), device="cuda")
+        out = (torch.empty((rows, k), device="cuda"), torch.empty((rows, k), dtype=torch.int64, device="cuda"))
+        g = torch.Generator(device="cuda").manual_seed(rows + k)
+        x.normal_(generator=g)
+        profk.topk(x, k, out=out)                    # first use of the shape (workspace, attributes) outside the capture
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                profk.topk(x, k, out=out, seed=3)
+        for _ in range(2):
+            x.normal_(generator=g)
+            graph.replay()
+            torch.cuda.synchronize()
+            assert_exact(x.cpu(), k, workloads.as_numpy(out[0]), out[1].cpu().numpy())
