@@ -47,7 +47,6 @@ struct DeviceInfo {
     int sm_count = 0;
     int filter_blocks_per_sm[2] = {0, 0};     // by dtype
     int filter_staged_blocks_per_sm[2] = {0, 0};
-    int fallback_blocks_per_sm[2] = {0, 0};
     int max_cluster[2] = {8, 8};              // 16 when the device can co-schedule 16 CTAs of the threshold kernel
     int refine_cluster[2] = {8, 8};           // same for the refine kernel at its largest footprint
     bool ready = false;
@@ -125,8 +124,6 @@ template <typename T> int ensure_device_info(int dev, DeviceInfo* out) {
         CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, true>,
                                                                  FILTER_THREADS, 0));
         di.filter_staged_blocks_per_sm[d] = std::max(nb, 1);
-        CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fallback_kernel<T>, FB_THREADS, 0));
-        di.fallback_blocks_per_sm[d] = std::max(nb, 1);
         CUDA_TRY(cudaFuncSetAttribute(sample_select_kernel<T, SEL_THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
         CUDA_TRY(cudaFuncSetAttribute(refine_kernel<T, 48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFINE_SMEM_MAX));
         CUDA_TRY(cudaFuncSetAttribute(refine_kernel<T, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFINE_SMEM_MAX));
