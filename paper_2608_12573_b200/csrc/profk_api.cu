@@ -27,7 +27,7 @@ namespace {
 #endif
 constexpr int FILTER_THREADS = PROFK_FILTER_THREADS;
 constexpr int FILTER_UNROLL = PROFK_FILTER_UNROLL;
-constexpr uint32_t SORT_CAP_MAX = 8192;          // largest k the single-CTA refine orders in shared memory
+constexpr uint32_t SORT_CAP_MAX = 16384;         // largest k the single-CTA refine orders in shared memory
 constexpr unsigned FB_MAX_CTAS = 256;             // most CTAs of the grid-wide exact selection (its per-CTA scratch is sized for them)
 constexpr int64_t GATHER_MAX_ROWS = 4;           // most rows for which the sample may be gathered by a kernel of its own
 constexpr int LARGE_MAX_CTAS = 1024;             // CTAs of the large refine (its per-CTA slots live in the 48 KB histogram area)
