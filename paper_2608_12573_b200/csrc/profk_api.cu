@@ -168,7 +168,10 @@ __global__ void init_ctl_kernel(RowCtl* ctl, uint64_t rows, WsHeader* header, ui
         RowCtl* c = ctl + r;
         c->tau_bits = 0; c->count = 0; c->collect = 0; c->status = ROW_DIRECT; c->n_final = k; c->capacity = capacity;
     }
-    if (r == 0) { header->bar_count = 0; header->error = 0; header->done = 0; header->n_failed = (uint32_t)rows; }
+    if (r == 0) {
+        header->bar_count = 0; header->error = 0; header->done = 0; header->n_failed = (uint32_t)rows;
+        for (int g = 0; g < 8; ++g) header->group_bar[g][0] = 0;
+    }
 }
 
 // Cluster size for the threshold kernel: spread one row's gather over several SMs when
@@ -314,7 +317,11 @@ int launch_refine_large(const DeviceInfo& di, RowCtl* ctl, WsHeader* header, uin
     lp.k = (uint32_t)k; lp.k_accept = (uint32_t)k_accept; lp.phase = phase; lp.out_vals = out_vals; lp.out_idx = out_idx;
     lp.use_pdl = 0;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)std::min(di.sm_count, LARGE_MAX_CTAS));
+    // Several rows: the grid splits into groups of CTAs that take rows side by side (a row alone keeps all SMs).
+    const unsigned groups = (unsigned)std::min<int64_t>(rows, 8);
+    const unsigned ctas = (unsigned)std::min(di.sm_count, LARGE_MAX_CTAS);
+    lp.groups = groups;
+    cfg.gridDim = dim3(ctas / groups * groups);
     cfg.blockDim = dim3(BT_THREADS);
     cfg.dynamicSmemBytes = (size_t)BT_TILE * 8;
     cfg.stream = st;

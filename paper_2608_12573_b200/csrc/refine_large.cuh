@@ -35,6 +35,7 @@ template <typename T> struct LargeParams {
     uint64_t row_stride;     //        row_stride is a power of two >= capacity, >= BT_TILE
     uint32_t* bins;          // rows x (LG_BINS + 8) words: bin counts / positions, then flags
     unsigned long long* slots;   // 2 words per CTA of the grid, then one per CTA: per-CTA minima / maxima and scan totals
+    uint32_t groups;         // CTA groups the grid is cut into (<= 8; gridDim.x is a multiple of it)
     uint32_t parts;          // 1, or 8: the filter appended to that many parts of the row's buffer (first phase only)
     uint32_t part_cap;       // records per part
     const uint32_t* part_counts;   // row r, part j: part_counts[(r * 8 + j) * 64]
@@ -74,22 +75,27 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
     __shared__ unsigned long long s_min[32], s_max[32];
     __shared__ uint32_t s_warp[32];
 
-    const unsigned nctas = gridDim.x, cta = blockIdx.x;
+    // The grid works as p.groups groups of CTAs (one for a single row); a group takes rows group, group + groups, ...
+    // one after the other, all its CTAs on one row, with a barrier of its own.
+    const unsigned nctas = gridDim.x / p.groups, group = blockIdx.x / nctas, cta = blockIdx.x % nctas;
     const unsigned tid = threadIdx.x;
-    const uint64_t gid = (uint64_t)cta * BT_THREADS + tid;           // thread index inside the grid
+    const uint64_t gid = (uint64_t)cta * BT_THREADS + tid;           // thread index inside the group
     const uint64_t gthreads = (uint64_t)nctas * BT_THREADS;
-    unsigned long long* slot_min = p.slots;
-    unsigned long long* slot_max = p.slots + nctas;
-    unsigned long long* slot_total = p.slots + 2 * nctas;
+    unsigned long long* slot_min = p.slots + group * nctas;
+    unsigned long long* slot_max = p.slots + gridDim.x + group * nctas;
+    unsigned long long* slot_total = p.slots + 2 * gridDim.x + group * nctas;
+    uint32_t* bar_count = &p.header->group_bar[group][0];
+    uint32_t* bar_gen = &p.header->group_bar[group][1];
+    auto barrier = [&](uint32_t& g) { return cta_group_barrier(bar_count, bar_gen, &p.header->error, nctas, g); };
     // The scan is shared by a power-of-two number of CTAs (at most 256, so that a thread owns a whole bin).
     unsigned scan_ctas = 1;
     while (scan_ctas * 2 <= nctas && scan_ctas < 256) scan_ctas *= 2;
 
     pdl_launch_dependents();
     if (p.use_pdl) pdl_wait();
-    uint32_t gen = *((volatile uint32_t*)&p.header->bar_gen);        // read before this CTA's first arrival
+    uint32_t gen = *((volatile uint32_t*)bar_gen);                   // read before this CTA's first arrival
 
-    for (uint64_t row = 0; row < p.rows; ++row) {
+    for (uint64_t row = group; row < p.rows; row += p.groups) {
         // ---- is this row for this launch?  (the decision is the same in every CTA) ----
         const RowCtl ctl = p.ctl[row];
         uint32_t n;
@@ -169,7 +175,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
             }
             if (tid == 0) { slot_min[cta] = lo; slot_max[cta] = hi; }
         }
-        if (!grid_barrier(p.header, gen)) return;
+        if (!barrier(gen)) return;
         unsigned long long rmin = ~0ull, rmax = 0ull;
         for (unsigned c = tid & 31; c < nctas; c += 32) {
             const unsigned long long l2 = __ldcg(&slot_min[c]), h2 = __ldcg(&slot_max[c]);
@@ -188,7 +194,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
 
         // histogram (global atomics spread over the bins)
         for_each_record([&](unsigned long long rec) { atomicAdd(&bins[bin_of(rec)], 1u); });
-        if (!grid_barrier(p.header, gen)) return;
+        if (!barrier(gen)) return;
 
         // scan: CTA c < scan_ctas owns bins [c, c+1) * LG_BINS / scan_ctas; counts become first positions
         const uint32_t per_cta = LG_BINS / scan_ctas, per_thr = per_cta / BT_THREADS;
@@ -215,7 +221,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
                 if (tid == 31) slot_total[cta] = w;
             }
         }
-        if (!grid_barrier(p.header, gen)) return;
+        if (!barrier(gen)) return;
         if (cta < scan_ctas) {
             uint32_t before = incl - sum + ((tid >> 5) ? s_warp[(tid >> 5) - 1] : 0);
             uint32_t ahead = 0;                                      // records in the bins of the CTAs before this one
@@ -230,12 +236,12 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
                 before += c;
             }
         }
-        if (!grid_barrier(p.header, gen)) return;
+        if (!barrier(gen)) return;
 
         if (__ldcg(&flags[0]) == 0) {
             // scatter into the second buffer, grouped by bin
             for_each_record([&](unsigned long long rec) { G2[atomicAdd(&bins[bin_of(rec)], 1u)] = rec; });
-            if (!grid_barrier(p.header, gen)) return;
+            if (!barrier(gen)) return;
             // rank inside the bin: bin b now occupies [end of bin b-1, bins[b])
             // (only positions below the end of the bin that holds position kk-1 matter; they are a prefix)
             const uint64_t g_end = (uint64_t)kk + LG_CROWDED < n ? (uint64_t)kk + LG_CROWDED : n;
@@ -260,9 +266,9 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
                 for (uint64_t i = gid; i < pcount[j]; i += gthreads) G2[first + i] = __ldcg(&part[i]);
                 first += pcount[j];
             }
-            if (!grid_barrier(p.header, gen)) return;
+            if (!barrier(gen)) return;
             for (uint64_t i = gid; i < n; i += gthreads) G[i] = __ldcg(&G2[i]);
-            if (!grid_barrier(p.header, gen)) return;
+            if (!barrier(gen)) return;
         }
         uint64_t P = BT_TILE;
         while (P < n) P <<= 1;
@@ -277,7 +283,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
             for (uint32_t i = tid; i < BT_TILE; i += BT_THREADS) G[base + i] = tile[i];
             __syncthreads();
         }
-        if (!grid_barrier(p.header, gen)) return;
+        if (!barrier(gen)) return;
 
         // ---- merge: exchanges at distance >= BT_TILE on the buffer, the rest tile by tile ----
         for (uint64_t size = 2ull * BT_TILE; size <= P; size <<= 1) {
@@ -289,7 +295,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
                     const uint64_t x = __ldcg(&G[lo2]), y = __ldcg(&G[hi2]);
                     if ((x > y) == ascending) { G[lo2] = y; G[hi2] = x; }
                 }
-                if (!grid_barrier(p.header, gen)) return;
+                if (!barrier(gen)) return;
             }
             for (uint64_t t = cta; t < tiles; t += nctas) {
                 const uint64_t base = t * BT_TILE;
@@ -299,7 +305,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
                 for (uint32_t i = tid; i < BT_TILE; i += BT_THREADS) G[base + i] = tile[i];
                 __syncthreads();
             }
-            if (!grid_barrier(p.header, gen)) return;
+            if (!barrier(gen)) return;
         }
 
         for (uint64_t j = gid; j < kk; j += gthreads) write_output(p.out_vals, p.out_idx, p.k, row, (uint32_t)j, __ldcg(&G[j]));

@@ -51,7 +51,8 @@ struct WsHeader {
     uint32_t done;       // CTAs of the filter kernel that have finished (ticket for its last CTA)
     uint32_t n_failed;   // rows whose count check failed
     uint32_t tile_counter;  // hands out the filter kernel's tiles
-    uint32_t pad[58];
+    uint32_t group_bar[8][2];   // barriers of the CTA groups of the large-k refine: {arrivals, generation}
+    uint32_t pad[42];
 };
 static_assert(sizeof(WsHeader) == 256, "WsHeader is 256 bytes");
 
@@ -277,7 +278,10 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
             if (p.part_counts)
                 for (int j = 0; j < 8; ++j) p.part_counts[(row * 8 + j) * 64] = 0;
         }
-        if (p.header && row == 0) { p.header->bar_count = 0; p.header->error = 0; p.header->done = 0; p.header->n_failed = 0; p.header->tile_counter = 0; }
+        if (p.header && row == 0) {
+            p.header->bar_count = 0; p.header->error = 0; p.header->done = 0; p.header->n_failed = 0; p.header->tile_counter = 0;
+            for (int g = 0; g < 8; ++g) p.header->group_bar[g][0] = 0;
+        }
     }
     PROFK_STAMP(0, 1);
 
