@@ -86,8 +86,9 @@ __device__ __forceinline__ uint64_t xs_elements_in_tiles(uint64_t N, uint32_t mi
 }
 
 // Writes a superset of the k smallest records (all records, if there are at most k) among the
-// elements of row `row` that lie in tiles [seg_lo, seg_hi) to dst[0 .. k + XS_EDGE), in any order:
-// fewer than k + XS_EDGE records, the unused slots filled with all-ones (no record has that value).
+// elements of row `row` that lie in tiles [seg_lo, seg_hi) to dst[0 .. k + edge), in any order: at most
+// k + edge - 1 records (exactly the k smallest when edge is 0), the unused slots filled with all-ones (no
+// record has that value).
 // Returns after a cluster barrier: on return the records are in global memory.
 // Called by all threads of all CTAs of the cluster (CTA `crank` of `csize`); *collect is a counter
 // for this call alone.
@@ -103,7 +104,8 @@ __device__ __forceinline__ uint64_t xs_elements_in_tiles(uint64_t N, uint32_t mi
 template <typename T>
 __device__ __noinline__ void exact_select_cluster(const T* in, uint64_t N, uint64_t row, uint32_t k, uint64_t seg_lo,
                                                   uint64_t seg_hi, uint64_t* dst, uint32_t* collect, SelectShared& sh,
-                                                  unsigned csize, unsigned crank, bool use_tau, uint32_t tau_key) {
+                                                  unsigned csize, unsigned crank, bool use_tau, uint32_t tau_key,
+                                                  uint32_t edge = XS_EDGE) {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
     constexpr int VEC = Elem<T>::VEC;
@@ -114,7 +116,7 @@ __device__ __noinline__ void exact_select_cluster(const T* in, uint64_t N, uint6
     const uint64_t tile_elems = (uint64_t)nthr * XS_UNROLL * VEC;
     const int idx_bits = N > 1 ? 64 - __clzll((long long)(N - 1)) : 1;      // bits an index occupies
     const uint64_t n_seg = xs_elements_in_tiles(N, rv.mis, tile_elems, seg_lo, seg_hi);
-    const uint32_t slots = k + XS_EDGE;
+    const uint32_t slots = k + edge;
     if (crank == 0 && tid == 0) *collect = 0;          // ordered before the appends by the barriers below
     for (uint32_t i = crank * nthr + tid; i < slots; i += csize * nthr) dst[i] = ~0ull;      // so are these
 
@@ -267,7 +269,7 @@ __device__ __noinline__ void exact_select_cluster(const T* in, uint64_t N, uint6
                 none_chosen = false;
                 lo_sel = lo;
                 need -= before;
-                if (in_bin - need < XS_EDGE || lo == 0) {
+                if (in_bin - need < edge || in_bin == need || lo == 0) {
                     limit = limit_of_class(lo);
                     found = true;
                 } else {
@@ -320,7 +322,7 @@ __device__ __noinline__ void exact_select_cluster(const T* in, uint64_t N, uint6
         sync_all();                         // peers have read this CTA's histogram; sh.digit may be rewritten
 
         // Stop when at most XS_EDGE - 1 records beyond the k-th would be taken along.
-        if (in_bin - need < XS_EDGE || (!key_phase && lo == 0)) {
+        if (in_bin - need < edge || in_bin == need || (!key_phase && lo == 0)) {
             limit = limit_of_class(lo);
             found = true;
         } else if (key_phase && lo == 0) {  // the key is known and widely shared: go on with the index

@@ -47,6 +47,7 @@ template <typename T> struct FallbackParams {
     uint64_t* cta_records;    // gridDim.x x (k + XS_EDGE) records of scratch
     uint32_t* cta_counters;   // gridDim.x counters
     uint32_t sort_cap;        // power of two >= k: records the dynamic shared memory holds
+    int parallel;             // 1 = the one-row-per-CTA mode may be used (its scratch is there, or none is needed)
 };
 
 static_assert(FB_BINS <= RF_BINS, "the grid-wide selection's histogram lives in SelectShared::hist");
@@ -97,7 +98,7 @@ __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackPara
     const uint32_t n_failed = __ldcg(&p.header->n_failed);
     if (n_failed == 0) return;
 
-    if (p.cta_records && n_failed >= FB_PARALLEL_MIN) {
+    if (p.parallel && n_failed >= FB_PARALLEL_MIN) {
         // ---- many rows: each CTA takes failed rows of its own (no grid barrier is reached) ----
         extern __shared__ __align__(16) unsigned char fb_smem[];
         uint64_t* sortbuf = reinterpret_cast<uint64_t*>(fb_smem);
@@ -108,9 +109,15 @@ __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackPara
             const uint32_t status = __ldcg(&p.ctl[row].status);
             if (status == ROW_OK) continue;
             const uint32_t tau_key = Elem<T>::key(Elem<T>::from_bits(__ldcg(&p.ctl[row].tau_bits)));
-            exact_select_cluster<T>(p.in, p.N, row, p.k, 0, tiles, recs, p.cta_counters + blockIdx.x, sh, 1u, 0u,
-                                    status == ROW_OVERFLOW, tau_key);
-            finish_from_segments<T>(recs, slots, p.k, p.sort_cap, sortbuf, sh, row, p.out_vals, p.out_idx);
+            if (p.sort_rows) {
+                exact_select_cluster<T>(p.in, p.N, row, p.k, 0, tiles, recs, p.cta_counters + blockIdx.x, sh, 1u, 0u,
+                                        status == ROW_OVERFLOW, tau_key);
+                finish_from_segments<T>(recs, slots, p.k, p.sort_cap, sortbuf, sh, row, p.out_vals, p.out_idx);
+            } else {
+                // large selections: exactly the k best records into the row's buffer, for the kernel that orders them
+                exact_select_cluster<T>(p.in, p.N, row, p.k, 0, tiles, p.buf + row * p.buf_stride, &p.ctl[row].collect, sh, 1u, 0u,
+                                        status == ROW_OVERFLOW, tau_key, 0u);
+            }
             __syncthreads();
         }
         return;

@@ -170,7 +170,7 @@ __global__ void init_ctl_kernel(RowCtl* ctl, uint64_t rows, WsHeader* header, ui
     }
     if (r == 0) {
         header->bar_count = 0; header->error = 0; header->done = 0; header->n_failed = (uint32_t)rows;
-        for (int g = 0; g < 8; ++g) header->group_bar[g][0] = 0;
+        for (int g = 0; g < WS_GROUPS; ++g) header->group_bar[g][0] = 0;
     }
 }
 
@@ -318,7 +318,7 @@ int launch_refine_large(const DeviceInfo& di, RowCtl* ctl, WsHeader* header, uin
     lp.use_pdl = 0;
     cudaLaunchConfig_t cfg = {};
     // Several rows: the grid splits into groups of CTAs that take rows side by side (a row alone keeps all SMs).
-    const unsigned groups = (unsigned)std::min<int64_t>(rows, 8);
+    const unsigned groups = (unsigned)std::min<int64_t>(rows, WS_GROUPS);
     const unsigned ctas = (unsigned)std::min(di.sm_count, LARGE_MAX_CTAS);
     lp.groups = groups;
     cfg.gridDim = dim3(ctas / groups * groups);
@@ -493,6 +493,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         fb.cta_records = fbp ? reinterpret_cast<uint64_t*>(base + lay.off_fb_records) : nullptr;
         fb.cta_counters = fbp ? reinterpret_cast<uint32_t*>(base + lay.off_fb_counters) : nullptr;
         fb.sort_cap = fb_sort_cap;
+        fb.parallel = (fbp || large) ? 1 : 0;      // large selections write into the rows' own buffers
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(std::min<unsigned>((unsigned)di.sm_count, FB_MAX_CTAS));
         cfg.blockDim = dim3(FB_THREADS);

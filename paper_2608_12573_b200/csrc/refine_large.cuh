@@ -35,7 +35,7 @@ template <typename T> struct LargeParams {
     uint64_t row_stride;     //        row_stride is a power of two >= capacity, >= BT_TILE
     uint32_t* bins;          // rows x (LG_BINS + 8) words: bin counts / positions, then flags
     unsigned long long* slots;   // 2 words per CTA of the grid, then one per CTA: per-CTA minima / maxima and scan totals
-    uint32_t groups;         // CTA groups the grid is cut into (<= 8; gridDim.x is a multiple of it)
+    uint32_t groups;         // CTA groups the grid is cut into (<= WS_GROUPS; gridDim.x is a multiple of it)
     uint32_t parts;          // 1, or 8: the filter appended to that many parts of the row's buffer (first phase only)
     uint32_t part_cap;       // records per part
     const uint32_t* part_counts;   // row r, part j: part_counts[(r * 8 + j) * 64]

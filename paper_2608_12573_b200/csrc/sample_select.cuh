@@ -43,6 +43,8 @@ struct RowCtl {
 };
 static_assert(sizeof(RowCtl) == 32, "RowCtl is 32 bytes");
 
+constexpr int WS_GROUPS = 32;            // most CTA groups of the large-k refine
+
 // Header of the workspace: state of the grid barrier used by the exact-selection kernel.
 struct WsHeader {
     uint32_t bar_count;
@@ -51,10 +53,10 @@ struct WsHeader {
     uint32_t done;       // CTAs of the filter kernel that have finished (ticket for its last CTA)
     uint32_t n_failed;   // rows whose count check failed
     uint32_t tile_counter;  // hands out the filter kernel's tiles
-    uint32_t group_bar[8][2];   // barriers of the CTA groups of the large-k refine: {arrivals, generation}
-    uint32_t pad[42];
+    uint32_t pad[58];
+    uint32_t group_bar[WS_GROUPS][2];   // barriers of the CTA groups of the large-k refine: {arrivals, generation}
 };
-static_assert(sizeof(WsHeader) == 256, "WsHeader is 256 bytes");
+static_assert(sizeof(WsHeader) == 512, "WsHeader is 512 bytes");
 
 template <typename T> struct SelectParams {
     const T* in;
@@ -280,7 +282,7 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
         }
         if (p.header && row == 0) {
             p.header->bar_count = 0; p.header->error = 0; p.header->done = 0; p.header->n_failed = 0; p.header->tile_counter = 0;
-            for (int g = 0; g < 8; ++g) p.header->group_bar[g][0] = 0;
+            for (int g = 0; g < WS_GROUPS; ++g) p.header->group_bar[g][0] = 0;
         }
     }
     PROFK_STAMP(0, 1);
