@@ -16,6 +16,14 @@ no top-k member is lost); in relaxed mode the acceptance test is
 k_accept <= R <= M and a short buffer is returned as it is, followed by padding
 (value -inf, index -1).
 
+Tie-proof variant (`composite=True`; not in the paper, whose analysis assumes distinct
+ranks): the threshold is the t-th sample as a RECORD under (value descending, index
+ascending) -- its value tau and its index tau_idx -- and the filter drops the elements
+that have exactly tau's value (the same order key) and an index above tau_idx.  Records
+are distinct, so R is the rank of the threshold record among all records of the row and
+Lemma 1's law holds for any input, ties included; on rows without ties at tau nothing
+changes.
+
 Status codes mirror the library's per-row statistics.
 
 Pins (tests/test_oracle_stages.py): whenever k <= R <= M the refined answer
@@ -75,16 +83,38 @@ def survivor_set(x: np.ndarray, tau) -> np.ndarray:
     return np.flatnonzero(~(xf < tf))
 
 
+def threshold_record(x: np.ndarray, sample_idx: np.ndarray, t: int):
+    """Stage 2 on records: the t-th sample under (value descending, index ascending), as (value, index)."""
+    sampled = x[sample_idx]
+    order = np.lexsort((sample_idx, ~topk.order_key(sampled)))      # last key is the primary one
+    j = order[t - 1]
+    return sampled[j], int(sample_idx[j])
+
+
+def survivor_set_record(x: np.ndarray, tau, tau_idx: int) -> np.ndarray:
+    """Indices kept by the tie-proof stage 3, ascending: not (x_i < tau), minus the elements with tau's own
+    order key and an index above tau_idx."""
+    xf = _as_float(x)
+    tf = _as_float(np.asarray([tau], dtype=x.dtype))[0]
+    same = topk.order_key(x) == topk.order_key(np.asarray([tau], dtype=x.dtype))[0]
+    late = np.arange(x.shape[0]) > tau_idx
+    return np.flatnonzero(~(xf < tf) & ~(same & late))
+
+
 def run_row(x: np.ndarray, k: int, m: int, r: int, capacity: int, k_accept: int,
-            seed: int, row: int = 0, mode: int = 0) -> StageResult:
+            seed: int, row: int = 0, mode: int = 0, composite: bool = False) -> StageResult:
     """All four stages on one row with an explicit plan (m, r, capacity, k_accept)."""
     n = x.shape[0]
     if mode == 1:
         vals, idx = topk.topk_row(x, k)
         return StageResult(np.empty(0, np.int64), None, 0, STATUS_DIRECT, vals, idx)
     s_idx = philox.sample_indices(n, m, seed, row)                  # stage 1
-    tau = threshold(x, s_idx, r)                                     # stage 2
-    kept = survivor_set(x, tau)                                      # stage 3
+    if composite:
+        tau, tau_idx = threshold_record(x, s_idx, r)                 # stage 2, on records
+        kept = survivor_set_record(x, tau, tau_idx)                  # stage 3, tie-proof
+    else:
+        tau = threshold(x, s_idx, r)                                 # stage 2
+        kept = survivor_set(x, tau)                                  # stage 3
     R = int(kept.size)
     if R > capacity:                                                 # stage 4, failure branches
         vals, idx = topk.topk_row(x, k)

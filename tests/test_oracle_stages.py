@@ -71,3 +71,69 @@ def test_bf16_rows_and_nan_are_kept():
     g = f.copy(); g[17] = np.nan
     tau = np.float32(1.0)
     assert 17 in stages.survivor_set(g, tau)                                       # not (NaN < tau)
+
+
+# ----------------------------------------------------------------------------- tie-proof variant (records)
+def _records_desc(x):
+    """All (value, index) records of the row in the order (value descending, index ascending), by brute force."""
+    return sorted(range(len(x)), key=lambda i: (-float(x[i]), i))
+
+
+def test_record_threshold_on_distinct_values_changes_nothing():
+    x = np.random.default_rng(3).permutation(4000).astype(np.float32)
+    s_idx = philox.sample_indices(4000, 64, seed=2)
+    tau, tau_idx = stages.threshold_record(x, s_idx, 5)
+    assert tau == stages.threshold(x, s_idx, 5) and x[tau_idx] == tau and tau_idx in set(s_idx.tolist())
+    assert np.array_equal(stages.survivor_set_record(x, tau, tau_idx), stages.survivor_set(x, tau))
+    for seed in range(10):
+        a = stages.run_row(x, 20, 64, 3, 600, 20, seed=seed)
+        b = stages.run_row(x, 20, 64, 3, 600, 20, seed=seed, composite=True)
+        assert (a.status, a.survivors) == (b.status, b.survivors) and np.array_equal(a.idx, b.idx)
+
+
+def test_record_threshold_with_ties_is_the_rank_of_the_threshold_record():
+    rng = np.random.default_rng(4)
+    x = rng.integers(0, 4, size=600).astype(np.float32)                # four values, 150 copies each
+    order = _records_desc(x)
+    for seed in range(8):
+        s_idx = philox.sample_indices(600, 40, seed=seed)
+        for t in (1, 3, 10, 40):
+            tau, tau_idx = stages.threshold_record(x, s_idx, t)
+            # brute force: the t-th sampled record in the full order of records
+            sampled_in_order = [i for i in order if i in set(s_idx.tolist())]
+            assert tau_idx == sampled_in_order[t - 1] and tau == x[tau_idx]
+            kept = stages.survivor_set_record(x, tau, tau_idx)
+            rank = order.index(tau_idx) + 1                             # Lemma 1's R for distinct records
+            assert kept.size == rank and set(kept.tolist()) == set(order[:rank])
+            # the literal filter keeps every copy of tau: at least as many, usually far more
+            assert stages.count_survivors(x, tau) >= rank
+
+
+def test_record_filter_on_a_constant_row_follows_the_rank_law():
+    # All elements equal: the literal filter keeps the whole row (R = N, certain overflow); on records the row is
+    # as good as sorted by index, R = tau_idx + 1, and its mean is Lemma 1's t (N + 1) / (S + 1).
+    n, S, t = 20_000, 200, 7
+    x = np.full(n, 2.5, dtype=np.float32)
+    Rs = []
+    for seed in range(300):
+        s_idx = philox.sample_indices(n, S, seed=seed)
+        tau, tau_idx = stages.threshold_record(x, s_idx, t)
+        assert tau_idx == np.sort(s_idx)[t - 1]
+        R = stages.survivor_set_record(x, tau, tau_idx).size
+        assert R == tau_idx + 1
+        Rs.append(R)
+        assert stages.count_survivors(x, tau) == n
+    # (stratified sampling: the t-th smallest index lies in stratum t - 1, uniformly: mean (t - 1/2) N / S + 1/2)
+    assert abs(np.mean(Rs) - ((t - 0.5) * n / S + 0.5)) < 3 * (n / S) / np.sqrt(12 * 300)
+    res = stages.run_row(x, k=50, m=S, r=t, capacity=2000, k_accept=50, seed=1, composite=True)
+    assert res.status == stages.STATUS_OK and np.array_equal(res.idx, np.arange(50))
+    assert stages.run_row(x, k=50, m=S, r=t, capacity=2000, k_accept=50, seed=1).status == stages.STATUS_OVERFLOW
+
+
+def test_record_filter_keeps_the_topk_whenever_enough_survive():
+    rng = np.random.default_rng(5)
+    for seed in range(30):
+        x = rng.integers(0, 8, size=3000).astype(np.float32)           # heavy ties
+        res = stages.run_row(x, k=25, m=128, r=4, capacity=500, k_accept=25, seed=seed, composite=True)
+        v, i = topk.topk_row(x, 25)
+        assert np.array_equal(res.idx, i) and np.array_equal(res.vals, v)
