@@ -9,10 +9,15 @@ Section 3 of the paper, "The Prof-K algorithm":
   4. Refinement: exact top-k of the buffer; if fewer than k candidates were kept,
      or the buffer overflowed, exact top-k of the whole row instead.
 
-Readings: "descending order" is the total order of `topk.order_key`; the filter
-predicate is "not (x_i < tau)" in floating point, which equals x_i >= tau on
-inputs without NaN and keeps NaN otherwise (a superset of the key-order set, so
-no top-k member is lost); in relaxed mode the acceptance test is
+Readings: "descending order" is the total order of `topk.order_key`, and the
+filter's "x_i >= tau" is read in that same order (key(x_i) >= key(tau)), so the
+kept elements are exactly the R largest of the row and the count check
+k <= R <= M says what it is meant to say.  On ordinary values this is the
+floating-point comparison; it differs only where the two orders do (-0.0 ranks
+below +0.0; a NaN with the sign bit set ranks lowest and one without it highest,
+whereas floating point calls the zeros equal and a NaN unordered -- counting a
+lowest-ranked NaN among the survivors would let the check pass without the
+top-k in the buffer).  In relaxed mode the acceptance test is
 k_accept <= R <= M and a short buffer is returned as it is, followed by padding
 (value -inf, index -1).
 
@@ -55,13 +60,6 @@ class StageResult:
     idx: np.ndarray             # k indices, int64, -1 = padding
 
 
-def _as_float(x: np.ndarray) -> np.ndarray:
-    """Numeric view for the comparison: bf16 bit patterns widen exactly to float32."""
-    if x.dtype == np.uint16:
-        return (x.astype(np.uint32) << np.uint32(16)).view(np.float32)
-    return x
-
-
 def threshold(x: np.ndarray, sample_idx: np.ndarray, t: int):
     """Stage 2: the t-th largest sampled value (ties in value are the same value)."""
     sampled = x[sample_idx]
@@ -69,18 +67,18 @@ def threshold(x: np.ndarray, sample_idx: np.ndarray, t: int):
     return sampled[order[t - 1]]
 
 
+def _key_of(x: np.ndarray, tau):
+    return topk.order_key(np.asarray([tau], dtype=x.dtype))[0]
+
+
 def count_survivors(x: np.ndarray, tau) -> int:
-    """Stage 3's R = |{i : x_i >= tau}| with the predicate not (x_i < tau)."""
-    xf = _as_float(x)
-    tf = _as_float(np.asarray([tau], dtype=x.dtype))[0]
-    return int(np.count_nonzero(~(xf < tf)))
+    """Stage 3's R = |{i : x_i >= tau}|, the comparison taken in the total order."""
+    return int(np.count_nonzero(topk.order_key(x) >= _key_of(x, tau)))
 
 
 def survivor_set(x: np.ndarray, tau) -> np.ndarray:
     """Indices kept by stage 3, ascending."""
-    xf = _as_float(x)
-    tf = _as_float(np.asarray([tau], dtype=x.dtype))[0]
-    return np.flatnonzero(~(xf < tf))
+    return np.flatnonzero(topk.order_key(x) >= _key_of(x, tau))
 
 
 def threshold_record(x: np.ndarray, sample_idx: np.ndarray, t: int):
@@ -92,13 +90,10 @@ def threshold_record(x: np.ndarray, sample_idx: np.ndarray, t: int):
 
 
 def survivor_set_record(x: np.ndarray, tau, tau_idx: int) -> np.ndarray:
-    """Indices kept by the tie-proof stage 3, ascending: not (x_i < tau), minus the elements with tau's own
-    order key and an index above tau_idx."""
-    xf = _as_float(x)
-    tf = _as_float(np.asarray([tau], dtype=x.dtype))[0]
-    same = topk.order_key(x) == topk.order_key(np.asarray([tau], dtype=x.dtype))[0]
-    late = np.arange(x.shape[0]) > tau_idx
-    return np.flatnonzero(~(xf < tf) & ~(same & late))
+    """Indices kept by the tie-proof stage 3, ascending: the elements above tau, and those equal to tau (the same
+    order key) with an index up to tau_idx."""
+    keys, tk = topk.order_key(x), _key_of(x, tau)
+    return np.flatnonzero((keys > tk) | ((keys == tk) & (np.arange(x.shape[0]) <= tau_idx)))
 
 
 def run_row(x: np.ndarray, k: int, m: int, r: int, capacity: int, k_accept: int,

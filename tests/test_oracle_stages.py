@@ -137,3 +137,37 @@ def test_record_filter_keeps_the_topk_whenever_enough_survive():
         res = stages.run_row(x, k=25, m=128, r=4, capacity=500, k_accept=25, seed=seed, composite=True)
         v, i = topk.topk_row(x, 25)
         assert np.array_equal(res.idx, i) and np.array_equal(res.vals, v)
+
+
+# ----------------------------------------------------------------------------- the filter's comparison on special values
+def _f32(bits_list):
+    return np.array(bits_list, dtype=np.uint32).view(np.float32)
+
+
+def test_filter_comparison_is_the_total_order_on_zeros_and_nans():
+    NEG_NAN, POS_NAN = 0xFFC00000, 0x7FC00000
+    x = _f32([NEG_NAN, NEG_NAN, NEG_NAN, 0x3F800000, 0x3F000000, 0x3E4CCCCD, 0x00000000, 0x80000000, POS_NAN])
+    #          -nan     -nan     -nan     1.0         0.5         0.2         +0.0        -0.0        +nan
+    one, zero, neg_zero = x[3], x[6], x[7]
+    # floating point would call the three sign-bit NaNs "not below 1.0"; in the total order they rank lowest
+    assert stages.survivor_set(x, one).tolist() == [3, 8] and stages.count_survivors(x, one) == 2
+    assert stages.survivor_set(x, zero).tolist() == [3, 4, 5, 6, 8]          # -0.0 ranks below +0.0
+    assert stages.survivor_set(x, neg_zero).tolist() == [3, 4, 5, 6, 7, 8]
+    # whatever the threshold, the kept elements are the R largest of the row: the buffer's top-k is the row's
+    for tau in x:
+        kept = stages.survivor_set(x, tau)
+        R = kept.size
+        _, want = topk.topk_row(x, R)
+        assert sorted(kept.tolist()) == sorted(want.tolist())
+    # a run through all four stages on a row with sign-bit NaNs: the count check passes and the answer is exact
+    rng = np.random.default_rng(9)
+    y = rng.standard_normal(5000).astype(np.float32)
+    y[::7] = _f32([NEG_NAN])[0]
+    v, i = topk.topk_row(y, 10)
+    statuses = set()
+    for seed in range(20):
+        # threshold = the sample maximum: fewer than ten elements rank at or above it, though 715 NaNs are "not below" it
+        res = stages.run_row(y, k=10, m=64, r=1, capacity=2000, k_accept=10, seed=seed)
+        assert np.array_equal(res.idx, i)
+        statuses.add(res.status)
+    assert stages.STATUS_RECALL in statuses
