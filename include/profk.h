@@ -66,6 +66,20 @@ enum {
     PROFK_ROW_DIRECT = 3    /* plan mode 1: exact selection without sampling or filtering  */
 };
 
+/* How the filter of stage 3 treats copies of the threshold value (profk_plan_t.tie_rule).
+ *   PROFK_TIES_KEEP_ALL  Section 3 as printed: tau is the t-th largest sampled value and every x_i >= tau
+ *                        is kept.  The analysis of Section 4 assumes distinct values; on a row with very
+ *                        many copies of tau all of them survive and the buffer overflows.
+ *   PROFK_TIES_BY_INDEX  tau is the t-th sampled element under (value descending, index ascending), a value
+ *                        and an index, and of the elements whose bit pattern equals tau's only those with an
+ *                        index <= tau's are kept.  Elements then have distinct ranks, the rank law of Lemma 1
+ *                        holds for any input, and R is the rank of the threshold element.  On a row with no
+ *                        second copy of tau both rules keep the same elements.  profk_plan's choice. */
+enum {
+    PROFK_TIES_KEEP_ALL = 0,
+    PROFK_TIES_BY_INDEX = 1
+};
+
 /*
  * The parameters (S, t, M) of Section 4 / Algorithm 1, as this library chooses them.
  *   m         sample size S: Algorithm 1 steps 1-4 (Eq. optimal_S with log2 k,
@@ -79,6 +93,7 @@ enum {
  *   k_accept  k in exact mode (recall == 1), ceil(recall * k) in relaxed mode.
  *   mode      0 = sample / filter / refine; 1 = direct exact selection, chosen
  *             when 2 * capacity >= N or N <= 2 * m (the filter would not pay).
+ *   tie_rule  PROFK_TIES_*; profk_plan and profk_plan_ex set PROFK_TIES_BY_INDEX.
  *   z, alpha  Algorithm 1's z = 2 Phi^{-1}(1 - eps/2) and alpha = k / N.
  *   p_recall_fail, p_overflow   the two bounds for the returned (m, r, capacity).
  * Both bounds are binomial tail bounds valid for the stratified sampler the
@@ -90,7 +105,7 @@ typedef struct profk_plan {
     int64_t capacity;
     int64_t k_accept;
     int32_t mode;
-    int32_t reserved;
+    int32_t tie_rule;
     double z;
     double alpha;
     double p_recall_fail;
@@ -116,7 +131,8 @@ typedef struct profk_tuning {
 /* What happened to one row (read back with profk_read_stats). */
 typedef struct profk_row_stats {
     uint32_t tau_bits;   /* threshold tau: fp32 bit pattern, or bf16 pattern in the low 16 bits */
-    uint32_t survivors;  /* R = |{i : x_i >= tau}|; exact when <= capacity, otherwise only "> capacity" */
+    uint32_t survivors;  /* R, the elements the filter kept (|{i : x_i >= tau}| less the dropped copies of tau);
+                            exact when <= capacity, otherwise only "> capacity" */
     uint32_t capacity;   /* M used for the row */
     uint32_t status;     /* PROFK_ROW_*; bit 31 set = a device-side wait timed out (result invalid) */
 } profk_row_stats_t;

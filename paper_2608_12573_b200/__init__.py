@@ -23,6 +23,7 @@ EXPORTS = [
 ]
 
 ROW_OK, ROW_RECALL, ROW_OVERFLOW, ROW_DIRECT = 0, 1, 2, 3
+TIES_KEEP_ALL, TIES_BY_INDEX = 0, 1      # profk_plan_t.tie_rule: the filter as printed / the threshold as a (value, index) record
 
 
 class ProfkError(RuntimeError):
@@ -31,7 +32,7 @@ class ProfkError(RuntimeError):
 
 class _PlanStruct(ctypes.Structure):
     _fields_ = [("m", ctypes.c_int64), ("r", ctypes.c_int64), ("capacity", ctypes.c_int64),
-                ("k_accept", ctypes.c_int64), ("mode", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("k_accept", ctypes.c_int64), ("mode", ctypes.c_int32), ("tie_rule", ctypes.c_int32),
                 ("z", ctypes.c_double), ("alpha", ctypes.c_double),
                 ("p_recall_fail", ctypes.c_double), ("p_overflow", ctypes.c_double)]
 
@@ -56,9 +57,10 @@ class Plan:
     alpha: float = 0.0
     p_recall_fail: float = 0.0
     p_overflow: float = 0.0
+    tie_rule: int = TIES_BY_INDEX
 
     def _struct(self) -> _PlanStruct:
-        return _PlanStruct(self.m, self.r, self.capacity, self.k_accept, self.mode, 0,
+        return _PlanStruct(self.m, self.r, self.capacity, self.k_accept, self.mode, self.tie_rule,
                            self.z, self.alpha, self.p_recall_fail, self.p_overflow)
 
 
@@ -124,7 +126,7 @@ def _plan_uncached(N, k, eps, recall, s_min, s_max, cost_ratio) -> Plan:
                                    ctypes.c_double(recall), ctypes.byref(tun), ctypes.byref(out))
     _check(code, "profk_plan")
     return Plan(out.m, out.r, out.capacity, out.k_accept, out.mode, out.z, out.alpha,
-                out.p_recall_fail, out.p_overflow)
+                out.p_recall_fail, out.p_overflow, out.tie_rule)
 
 
 def workspace_bytes(rows: int, capacity: int, k: int) -> int:

@@ -53,23 +53,12 @@ template <typename T> struct FilterParams {
     // cache line of its own, and a CTA appends to part blockIdx.x mod FILTER_PARTS.
     uint32_t part_cap;       // records per part
     uint32_t* part_counts;   // row r, part j: part_counts[(r * FILTER_PARTS + j) * FILTER_PART_STRIDE] (zeroed)
+    // Threshold records written by the threshold kernel (null = take `tau`, a value alone): row r's is {bits of tau,
+    // bits of the value that follows tau in the total order, tau_idx, 0}.  Of the elements with exactly tau's bit
+    // pattern only those with an index <= tau_idx are kept (0xFFFFFFFF: all of them), so that a flood of copies of tau
+    // does not fill the buffer.
+    const uint4* thr;
 };
-
-constexpr uint32_t FILTER_PARTS = 8;
-constexpr uint32_t FILTER_PART_STRIDE = 64;     // words between two counters: 256 bytes
-
-// not (x < tau) for every lane of a vector, OR-ed: does the vector hold any survivor?
-__device__ __forceinline__ bool vec_any_pass(const float4& v, float tau) {
-    return !(v.x < tau) | !(v.y < tau) | !(v.z < tau) | !(v.w < tau);
-}
-__device__ __forceinline__ bool vec_any_pass(const uint4& v, __nv_bfloat16 tau) {
-    const __nv_bfloat162 t2 = __halves2bfloat162(tau, tau);
-    const unsigned a = __hlt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&v.x), t2);
-    const unsigned b = __hlt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&v.y), t2);
-    const unsigned c = __hlt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&v.z), t2);
-    const unsigned d = __hlt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&v.w), t2);
-    return (a & b & c & d) != 0xFFFFFFFFu;    // some lane is not below tau
-}
 
 // Bit l set = element l of the vector is not below tau (the same test as vec_any_pass, per element).
 __device__ __forceinline__ unsigned vec_pass_mask(const float4& v, float tau) {
@@ -87,26 +76,89 @@ __device__ __forceinline__ unsigned vec_pass_mask(const uint4& v, __nv_bfloat16 
     return m;
 }
 
+// Does the vector hold an element that floating point calls equal to tau, or unordered with it (a NaN on either
+// side)?  Those are the elements on which the float test and the total order of the keys can differ: a copy of tau,
+// a zero of the other sign, a NaN.  One "equal or unordered" comparison per element.
+__device__ __forceinline__ bool vec_any_equal_or_unordered(const float4& v, float tau) {
+    unsigned r;
+    asm("{\n\t.reg .pred a, b, c, d;\n\t"
+        "setp.equ.f32 a, %1, %5;\n\tsetp.equ.f32 b, %2, %5;\n\tsetp.equ.f32 c, %3, %5;\n\tsetp.equ.f32 d, %4, %5;\n\t"
+        "or.pred a, a, b;\n\tor.pred c, c, d;\n\tor.pred a, a, c;\n\tselp.u32 %0, 1, 0, a;\n\t}"
+        : "=r"(r) : "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "f"(tau));
+    return r != 0;
+}
+__device__ __forceinline__ bool vec_any_equal_or_unordered(const uint4& v, __nv_bfloat16 tau) {
+    const __nv_bfloat162 t2 = __halves2bfloat162(tau, tau);
+    return (__hequ2_mask(*reinterpret_cast<const __nv_bfloat162*>(&v.x), t2) | __hequ2_mask(*reinterpret_cast<const __nv_bfloat162*>(&v.y), t2) |
+            __hequ2_mask(*reinterpret_cast<const __nv_bfloat162*>(&v.z), t2) | __hequ2_mask(*reinterpret_cast<const __nv_bfloat162*>(&v.w), t2)) != 0;
+}
+
+// Index up to which copies of tau are kept in `row` (read on the slow paths only).
+template <typename T>
+__device__ __forceinline__ uint32_t tie_limit(const FilterParams<T>& p, uint32_t row) {
+    return p.thr ? reinterpret_cast<const uint32_t*>(p.thr + row)[2] : 0xFFFFFFFFu;
+}
+
+// The exact test, in the total order of the keys, for the elements of a vector that passed the float test
+// "not (x < tau)" (mask m; element l has index i0 + l): kept are the elements above tau and the copies of tau at
+// or before the threshold record.  The float test lets through a few more: -0.0 for tau = +0.0, NaNs with the sign
+// bit set (they rank lowest), copies of tau beyond the record.  An element that floating point puts strictly above
+// tau is above it in the total order too, so only vectors with an element equal to tau or unordered with it -- rare
+// -- are looked at, and the record's index is read only when a copy of tau turns up.
+template <typename T>
+__device__ __noinline__ unsigned confirm_each(const FilterParams<T>& p, uint32_t row, typename Elem<T>::vec_t v, unsigned m, int64_t i0, T tau) {
+    unsigned keep = m;
+    const uint32_t tau_key = Elem<T>::key(tau);
+    while (m) {
+        const int l = __ffs(m) - 1;
+        m &= m - 1;
+        const uint32_t key = Elem<T>::key(vec_elem(v, l));
+        if (key < tau_key || (key == tau_key && i0 + l > (int64_t)tie_limit(p, row))) keep &= ~(1u << l);
+    }
+    return keep;
+}
+template <typename T>
+__device__ __forceinline__ unsigned confirm_survivors(const FilterParams<T>& p, uint32_t row, const typename Elem<T>::vec_t& v,
+                                                      unsigned m, int64_t i0, T tau) {
+    return vec_any_equal_or_unordered(v, tau) ? confirm_each<T>(p, row, v, m, i0, tau) : m;
+}
+
+constexpr uint32_t FILTER_PARTS = 8;
+constexpr uint32_t FILTER_PART_STRIDE = 64;     // words between two counters: 256 bytes
+
+// not (x < tau) for every lane of a vector, OR-ed: does the vector hold any survivor?
+__device__ __forceinline__ bool vec_any_pass(const float4& v, float tau) {
+    return !(v.x < tau) | !(v.y < tau) | !(v.z < tau) | !(v.w < tau);
+}
+__device__ __forceinline__ bool vec_any_pass(const uint4& v, __nv_bfloat16 tau) {
+    const __nv_bfloat162 t2 = __halves2bfloat162(tau, tau);
+    const unsigned a = __hlt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&v.x), t2);
+    const unsigned b = __hlt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&v.y), t2);
+    const unsigned c = __hlt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&v.z), t2);
+    const unsigned d = __hlt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&v.w), t2);
+    return (a & b & c & d) != 0xFFFFFFFFu;    // some lane is not below tau
+}
+
 // Survivors of one thread's vectors of a tile: bit u * VEC + l set = element l of vector u is inside the row
-// and not below tau.  Vectors without a survivor (nearly all) cost one packed test.
+// and kept.  Vectors without an element that is not below tau (nearly all) cost one packed test.
 template <typename T, int THREADS, int UNROLL>
 __device__ __forceinline__ uint32_t survivor_mask(const typename Elem<T>::vec_t (&v)[UNROLL], uint32_t inside_mask, uint64_t N,
-                                                  uint64_t qbase, uint32_t mis, T tau) {
+                                                  uint64_t qbase, uint32_t mis, T tau, const FilterParams<T>& p, uint32_t row) {
     constexpr int VEC = Elem<T>::VEC;
     static_assert(VEC * UNROLL <= 32, "one bit per element of the thread's share of a tile");
     uint32_t mine = 0;
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) {
         if (((inside_mask >> u) & 1u) && vec_any_pass(v[u], tau)) {
-            unsigned m = vec_pass_mask(v[u], tau);
             const uint64_t q = qbase + (uint64_t)u * THREADS + threadIdx.x;
             const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
+            unsigned m = vec_pass_mask(v[u], tau);
             if (i0 < 0 || i0 + VEC > (int64_t)N) {          // a vector across an end of the row: drop the lanes outside
 #pragma unroll
                 for (int l = 0; l < VEC; ++l)
                     if (i0 + l < 0 || i0 + l >= (int64_t)N) m &= ~(1u << l);
             }
-            mine |= m << (u * VEC);
+            mine |= confirm_survivors<T>(p, row, v[u], m, i0, tau) << (u * VEC);
         }
     }
     return mine;
@@ -211,6 +263,7 @@ __device__ __noinline__ uint32_t filter_slow_path(const FilterParams<T>& p, Warp
                     const bool ok = i >= 0 && i < (int64_t)p.N && !(Elem<T>::as_float(vec_elem(v[u], l)) < tau_f);
                     if (ok) mine_u[u] |= 1u << l;
                 }
+                mine_u[u] = confirm_survivors<T>(p, row, v[u], mine_u[u], i0, tau);
             }
             cnt += __popc(mine_u[u]);
         }
@@ -223,7 +276,7 @@ __device__ __noinline__ uint32_t filter_slow_path(const FilterParams<T>& p, Warp
         total = __shfl_sync(FULL_MASK, incl, 31);
         before = incl - cnt;
     } else {
-        mine = survivor_mask<T, THREADS, UNROLL>(v, inside_mask, p.N, qbase, mis, tau);
+        mine = survivor_mask<T, THREADS, UNROLL>(v, inside_mask, p.N, qbase, mis, tau, p, row);
         cnt = __popc(mine);
         before = warp_exclusive_count(cnt, lane, &total);
     }
@@ -283,7 +336,7 @@ template <typename T, int THREADS, int UNROLL, bool PARTS>
 __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T>& p, const typename Elem<T>::vec_t (&v)[UNROLL],
                                                             uint32_t inside_mask, uint32_t row, uint64_t qbase, uint32_t mis, T tau) {
     const unsigned lane = lane_id();
-    const uint32_t mine = survivor_mask<T, THREADS, UNROLL>(v, inside_mask, p.N, qbase, mis, tau);
+    const uint32_t mine = survivor_mask<T, THREADS, UNROLL>(v, inside_mask, p.N, qbase, mis, tau, p, row);
     const unsigned cnt = __popc(mine);
     unsigned total;
     const unsigned before = warp_exclusive_count(cnt, lane, &total);
@@ -372,8 +425,29 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
     uint32_t skip_row = 0xFFFFFFFFu;    // row whose buffer this warp has seen overflow: nothing more to append
     uint32_t parity = 0;
     uint32_t tau_row = row;
-    T tau = p.tau[row];
+    // The row's threshold, and what the streaming test compares with: tau itself up to the tile that holds the
+    // threshold record, the next value in the total order in the tiles after it -- there no copy of tau is
+    // kept, and a row that is one flood of copies of tau stays on the fast path.  (Single rows only: in a batch a
+    // CTA changes row at almost every tile, and the extra work at each change cost 2 % on rows without ties.)
+    T tau_lo, tau_hi;
+    uint32_t tie_tile;
+    auto load_threshold = [&]() {
+        if (p.thr && one_row) {
+            const uint4 t = p.thr[row];
+            tau_lo = Elem<T>::from_bits(t.x);
+            tau_hi = Elem<T>::from_bits(t.y);
+            tie_tile = t.z == 0xFFFFFFFFu ? 0xFFFFFFFFu : (uint32_t)(((uint64_t)t.z + rv.mis) / ((uint64_t)TILE_VECTORS * VEC));
+        } else if (p.thr) {
+            tau_lo = tau_hi = Elem<T>::from_bits(reinterpret_cast<const uint32_t*>(p.thr + row)[0]);
+            tie_tile = 0xFFFFFFFFu;
+        } else {
+            tau_lo = tau_hi = p.tau[row];
+            tie_tile = 0xFFFFFFFFu;
+        }
+    };
+    load_threshold();
     while (true) {
+        const T tau = (uint32_t)(qbase / TILE_VECTORS) > tie_tile ? tau_hi : tau_lo;
         // Tiles below dyn_start follow the fixed stride and the warps run freely; the last few tiles of
         // the launch are handed out by the counter.  Thread 0 asks for the next one now; the answer is
         // needed only after this tile.
@@ -395,8 +469,8 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
 
         if (__any_sync(FULL_MASK, hit) && row != skip_row) {
             uint32_t o;
-            if (STAGED) o = filter_slow_path<T, THREADS, UNROLL>(p, st, v[0], v[1], v[2], v[3], inside_mask, row, qbase, rv.mis, tau);
-            else o = filter_slow_path_direct<T, THREADS, UNROLL, PARTS>(p, v, inside_mask, row, qbase, rv.mis, tau);
+            if (STAGED) o = filter_slow_path<T, THREADS, UNROLL>(p, st, v[0], v[1], v[2], v[3], inside_mask, row, qbase, rv.mis, tau_lo);
+            else o = filter_slow_path_direct<T, THREADS, UNROLL, PARTS>(p, v, inside_mask, row, qbase, rv.mis, tau_lo);
             if (o != 0xFFFFFFFFu) skip_row = o;
         }
 
@@ -414,7 +488,7 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
             continue;                   // loop: the hand-out of the last tiles is a matter for the whole CTA)
         }
         decode_and_load(false);
-        if (row != tau_row) { tau_row = row; tau = p.tau[row]; }
+        if (row != tau_row) { tau_row = row; load_threshold(); }
     }
     if (STAGED && st->fill) flush_stage(p, st);
     PROFK_STAMP(0, 12);

@@ -146,6 +146,7 @@ extern "C" int profk_plan_ex(int64_t N, int64_t k, double eps, double recall, co
     out->capacity = capacity;
     out->k_accept = k_acc;
     out->mode = (2 * capacity >= N || N <= 2 * S) ? 1 : 0;
+    out->tie_rule = PROFK_TIES_BY_INDEX;
     out->z = z;
     out->alpha = alpha;
     out->p_recall_fail = recall_fail_bound(N, S, t, k_acc);

@@ -80,7 +80,7 @@ WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k) {
     l.off_ghist = sizeof(WsHeader);
     l.off_ctl = align_up(l.off_ghist + (size_t)FB_PASSES * FB_BINS * sizeof(uint32_t), 256);
     l.off_tau = align_up(l.off_ctl + (size_t)rows * sizeof(RowCtl), 256);
-    l.off_bins = align_up(l.off_tau + (size_t)rows * 4, 256);
+    l.off_bins = align_up(l.off_tau + (size_t)rows * sizeof(uint4), 256);
     const size_t bins_bytes = k > (int64_t)SORT_CAP_MAX ? (size_t)rows * (LG_BINS + 8) * sizeof(uint32_t) : 0;
     // scratch of the in-refine exact selection (few rows, k within the single-CTA refine): up to
     // XS_MAX_SEGMENTS segments in all, each with a counter and k + XS_EDGE records
@@ -186,7 +186,7 @@ int pick_cluster(int64_t rows, int64_t m, int max_cluster) {
 template <typename T>
 int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, int64_t m, int64_t r, uint64_t seed, T* tau, RowCtl* ctl,
                          WsHeader* header, uint32_t capacity, uint32_t* sample_idx, uint32_t* keys_scratch, uint32_t* part_counts,
-                         cudaStream_t st) {
+                         bool by_record, uint4* thr, cudaStream_t st) {
     const int csize = pick_cluster(rows, m, di.max_cluster[dtype_index<T>()]);
     // A large sample, or a sample of a very long row (every element on a page of its own), is gathered by a
     // kernel over all SMs first; the cluster then only selects.
@@ -211,6 +211,8 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
     SelectParams<T> sp;
     sp.keys_in = spread_gather ? keys_scratch : nullptr;
     sp.part_counts = part_counts;
+    sp.by_record = by_record ? 1 : 0;
+    sp.thr = thr;
     sp.in = in; sp.N = (uint64_t)N; sp.S = (uint32_t)m; sp.t = (uint32_t)r; sp.seed = seed;
     sp.per_cta = (uint32_t)(((m + csize - 1) / csize + 1) & ~1LL);      // even: samples are drawn in pairs
     sp.q = (uint64_t)(N / m); sp.rem = (uint32_t)(N % m); sp.inv_s = 1.0f / (float)m;
@@ -244,8 +246,9 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
 template <typename T>
 int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, const T* tau, int64_t capacity, uint64_t* buf,
                   uint64_t buf_stride, uint32_t* counts, uint32_t count_stride, bool pdl, bool staged, uint32_t* tile_counter, bool parts,
-                  uint32_t part_cap, uint32_t* part_counts, cudaStream_t st) {
+                  uint32_t part_cap, uint32_t* part_counts, const uint4* thr, cudaStream_t st) {
     FilterParams<T> fp;
+    fp.thr = thr;
     fp.in = in; fp.N = (uint64_t)N; fp.rows = (uint64_t)rows; fp.tau = tau; fp.capacity = (uint32_t)capacity;
     fp.buf = buf; fp.buf_stride = buf_stride; fp.counts = counts; fp.count_stride = count_stride;
     fp.tiles_per_row = tiles_per_row<T>((uint64_t)N, FILTER_THREADS * FILTER_UNROLL);
@@ -403,6 +406,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     const int64_t capacity = plan->capacity;
     if (capacity < k || capacity > N || rows * capacity >= (1LL << 40)) return PROFK_EINVAL;
     if (plan->mode != 0 && plan->mode != 1) return PROFK_EINVAL;
+    if (plan->tie_rule != PROFK_TIES_KEEP_ALL && plan->tie_rule != PROFK_TIES_BY_INDEX) return PROFK_EINVAL;
     if (plan->mode == 0) {
         if (plan->m < 1 || plan->m > std::min<int64_t>(N, M_MAX) || plan->r < 1 || plan->r > plan->m) return PROFK_EINVAL;
         if (plan->k_accept < 1 || plan->k_accept > k) return PROFK_EINVAL;
@@ -429,7 +433,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     WsHeader* header = reinterpret_cast<WsHeader*>(base + lay.off_header);
     uint32_t* ghist = reinterpret_cast<uint32_t*>(base + lay.off_ghist);
     RowCtl* ctl = reinterpret_cast<RowCtl*>(base + lay.off_ctl);
-    T* tau = reinterpret_cast<T*>(base + lay.off_tau);
+    uint4* thr = reinterpret_cast<uint4*>(base + lay.off_tau);
     uint64_t* buf = reinterpret_cast<uint64_t*>(base + lay.off_buf);
     uint32_t* bins = reinterpret_cast<uint32_t*>(base + lay.off_bins);
     uint32_t* xs_counters = reinterpret_cast<uint32_t*>(base + lay.off_xs_counters);
@@ -454,11 +458,11 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     while (fb_sort_cap < (uint32_t)k && fb_sort_cap < SORT_CAP_MAX) fb_sort_cap <<= 1;
 
     if (plan->mode == 0) {
-        rc = launch_sample_select<T>(di, in, rows, N, plan->m, plan->r, seed, tau, ctl, header, (uint32_t)capacity, nullptr,
-                                     rows <= GATHER_MAX_ROWS ? keys_scratch : nullptr, parts ? part_counts : nullptr, st);
+        rc = launch_sample_select<T>(di, in, rows, N, plan->m, plan->r, seed, nullptr, ctl, header, (uint32_t)capacity, nullptr,
+                                     rows <= GATHER_MAX_ROWS ? keys_scratch : nullptr, parts ? part_counts : nullptr, plan->tie_rule == PROFK_TIES_BY_INDEX, thr, st);
         if (rc != PROFK_OK) return rc;
-        rc = launch_filter<T>(di, in, rows, N, tau, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, &header->tile_counter,
-                              parts, part_cap, part_counts, st);
+        rc = launch_filter<T>(di, in, rows, N, nullptr, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, &header->tile_counter,
+                              parts, part_cap, part_counts, thr, st);
         if (rc != PROFK_OK) return rc;
 
         if (large) {
@@ -544,7 +548,7 @@ int filter_only(const T* in, int64_t rows, int64_t N, const T* tau, int64_t capa
     DeviceInfo di;
     const int rc = ensure_device_info<T>(dev, &di);
     if (rc != PROFK_OK) return rc;
-    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, (uint64_t)capacity, counts, 1, false, false, nullptr, false, 0u, nullptr,
+    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, (uint64_t)capacity, counts, 1, false, false, nullptr, false, 0u, nullptr, nullptr,
                             static_cast<cudaStream_t>(stream));
 }
 
@@ -559,7 +563,7 @@ int sample_threshold(const T* in, int64_t rows, int64_t N, int64_t m, int64_t r,
     DeviceInfo di;
     const int rc = ensure_device_info<T>(dev, &di);
     if (rc != PROFK_OK) return rc;
-    return launch_sample_select<T>(di, in, rows, N, m, r, seed, tau, nullptr, nullptr, 0, sample_idx, nullptr, nullptr,
+    return launch_sample_select<T>(di, in, rows, N, m, r, seed, tau, nullptr, nullptr, 0, sample_idx, nullptr, nullptr, false, nullptr,
                                    static_cast<cudaStream_t>(stream));
 }
 

@@ -39,7 +39,8 @@ struct RowCtl {
     uint32_t status;     // PROFK_ROW_* (| 0x80000000 on a timeout)
     uint32_t n_final;    // records the refine step has to order
     uint32_t capacity;
-    uint32_t pad[2];
+    uint32_t tau_idx;    // index of the threshold record; 0xFFFFFFFF = the threshold is the value alone
+    uint32_t pad;
 };
 static_assert(sizeof(RowCtl) == 32, "RowCtl is 32 bytes");
 
@@ -68,22 +69,17 @@ template <typename T> struct SelectParams {
     uint64_t q;            // N / S
     uint32_t rem;          // N % S
     float inv_s;           // 1 / S
-    T* tau;                // rows thresholds out
+    T* tau;                // rows thresholds out (may be null when thr is given)
+    uint4* thr;            // null, or rows threshold records for the filter: {bits of tau, bits of the next value in the total
+                           // order, index of the threshold record (0xFFFFFFFF = the threshold is the value alone), 0}
     RowCtl* ctl;           // may be null (stand-alone use)
     WsHeader* header;      // may be null
     uint32_t capacity;
     uint32_t* sample_idx;  // may be null; rows x S
     const uint32_t* keys_in;   // null, or rows x S keys of the sample gathered by gather_kernel before this one
     uint32_t* part_counts;     // null, or the counters of the partitioned append (8 per row, 64 words apart) to reset with the row's
+    int by_record;             // 1 = the threshold is the t-th sampled record (value descending, index ascending), 0 = its value
 };
-
-// Writes tau for one row.
-template <typename T>
-__device__ __forceinline__ void publish_threshold(const SelectParams<T>& p, uint64_t row, uint32_t tau_key) {
-    const T tau = Elem<T>::from_key(tau_key);
-    p.tau[row] = tau;
-    if (p.ctl) p.ctl[row].tau_bits = Elem<T>::bits(tau);
-}
 
 // floor(j * N / S) = j * (N / S) + floor(j * (N % S) / S).  The second quotient is below S
 // (< 2^18), so a float estimate is within one of it and an integer check repairs it.
@@ -95,6 +91,32 @@ __device__ __forceinline__ uint64_t stratum_start(uint64_t j, uint64_t q, uint32
     while (r < 0) { --e; r += S; }
     while (r >= (int64_t)S) { ++e; r -= S; }
     return j * q + (uint64_t)e;
+}
+
+// Writes tau for one row: the key of the threshold and the number j of the sample that holds it.  Samples are
+// stratified, so among samples "smaller index" and "smaller sample number" are the same order; the element
+// index of sample j is drawn again here by the one thread that publishes.
+template <typename T>
+__device__ __forceinline__ void publish_threshold(const SelectParams<T>& p, uint64_t row, uint32_t tau_key, uint32_t j) {
+    const T tau = Elem<T>::from_key(tau_key);
+    if (p.tau) p.tau[row] = tau;
+    if (p.ctl) {
+        p.ctl[row].tau_bits = Elem<T>::bits(tau);
+        uint32_t idx = 0xFFFFFFFFu;
+        if (p.by_record) {
+            const Philox4 r = philox4x32_10(j >> 1, (uint32_t)row, (uint32_t)(row >> 32), 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32));
+            const uint64_t b0 = stratum_start(j, p.q, p.rem, p.S, p.inv_s);
+            const uint64_t b1 = stratum_start((uint64_t)j + 1, p.q, p.rem, p.S, p.inv_s);
+            const uint64_t u = (j & 1u) ? (((uint64_t)r.w << 32) | r.z) : (((uint64_t)r.y << 32) | r.x);
+            idx = (uint32_t)(b0 + __umul64hi(u, b1 - b0));
+        }
+        p.ctl[row].tau_idx = idx;
+        if (p.thr) {
+            const uint32_t top = Elem<T>::KEY_BITS == 32 ? 0xFFFFFFFFu : 0xFFFFu;
+            const uint32_t next_key = tau_key == top ? tau_key : tau_key + 1u;
+            p.thr[row] = make_uint4(Elem<T>::bits(tau), Elem<T>::bits(Elem<T>::from_key(next_key)), idx, 0u);
+        }
+    }
 }
 
 // Block-wide inclusive scan of one value per thread (blockDim.x == SEL_THREADS or fewer warps).
@@ -182,7 +204,9 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
     constexpr bool GENERAL = THREADS == SEL_THREADS;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw);          // per_cta keys
-    __shared__ uint32_t cand[SEL_CAND_CAP];                          // candidates (filled in the first CTA only)
+    // Candidates (filled in the first CTA only), as records (key << 32) | ~(sample number): distinct, and their
+    // descending order is (value descending, index ascending).  The radix path reuses the space for its histograms.
+    __shared__ uint64_t cand[SEL_CAND_CAP];
     __shared__ uint32_t gmax[GROUPS];
     __shared__ uint32_t warp_sums[32];
     __shared__ uint32_t s_digit, s_before, s_ncand, s_lower;
@@ -320,7 +344,7 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
         const uint32_t lower = s_lower;
         PROFK_STAMP(0, 2);
         // every CTA sends its keys >= lower to the first CTA: one remote atomic per warp that has any
-        uint32_t* cand0 = cluster.map_shared_rank(cand, 0);
+        uint64_t* cand0 = cluster.map_shared_rank(cand, 0);
         uint32_t* ncand0 = cluster.map_shared_rank(&s_ncand, 0);
         cluster.barrier_wait(std::move(zeroed));
         for (uint32_t i = tid; i < n_round; i += THREADS) {
@@ -332,7 +356,7 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
                 if (lane == 0) base = atomicAdd(ncand0, (uint32_t)__popc(bal));
                 base = __shfl_sync(FULL_MASK, base, 0);
                 const uint32_t slot = base + __popc(bal & ((1u << lane) - 1u));
-                if (take && slot < SEL_CAND_CAP) cand0[slot] = k;
+                if (take && slot < SEL_CAND_CAP) cand0[slot] = ((uint64_t)k << 32) | (uint64_t)(0xFFFFFFFFu - (j0 + i));
             }
         }
         PROFK_STAMP(0, 3);
@@ -341,9 +365,8 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
         const uint32_t ncand = *ncand0;
         if (ncand <= SEL_CAND_CAP) {
             // Every CTA takes a copy of the candidates and looks at its share of them (candidate c goes to
-            // CTA c mod csize): the t-th largest key is the candidate with fewer than t candidates above
-            // it and at least t at or above it.  Eight lanes share one candidate's comparisons.  Equal
-            // candidates all qualify and publish the same value.
+            // CTA c mod csize): the t-th largest record is the one candidate with exactly t - 1 candidates
+            // above it.  Eight lanes share one candidate's comparisons.
             // A handful of candidates (small ranks) is not worth the copies: the first CTA looks at all.
             const bool spread = ncand > SEL_SPREAD_MIN;
             if (spread && crank != 0)
@@ -355,21 +378,15 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
             const uint32_t c_first = spread ? (tid >> 3) * csize + crank : crank == 0 ? (tid >> 3) : ncand;
             const uint32_t c_step = (THREADS / 8) * (spread ? csize : 1u);
             for (uint32_t c = c_first; c < ncand; c += c_step) {      // whole groups of eight lanes together
-                const uint32_t mine = cand[c];
-                uint32_t above = 0, at_or_above = 0;
-                for (uint32_t j = part; j < ncand; j += 8) {
-                    const uint32_t o = cand[j];
-                    above += o > mine;
-                    at_or_above += o >= mine;
-                }
+                const uint64_t mine = cand[c];
+                uint32_t above = 0;
+                for (uint32_t j = part; j < ncand; j += 8) above += cand[j] > mine;
                 const unsigned group = 0xFFu << (lane & 24u);
                 above += __shfl_xor_sync(group, above, 1);
                 above += __shfl_xor_sync(group, above, 2);
                 above += __shfl_xor_sync(group, above, 4);
-                at_or_above += __shfl_xor_sync(group, at_or_above, 1);
-                at_or_above += __shfl_xor_sync(group, at_or_above, 2);
-                at_or_above += __shfl_xor_sync(group, at_or_above, 4);
-                if (part == 0 && above < p.t && p.t <= at_or_above) publish_threshold(p, row, mine);   // tau
+                if (part == 0 && above == p.t - 1)                                                      // tau
+                    publish_threshold(p, row, (uint32_t)(mine >> 32), 0xFFFFFFFFu - (uint32_t)mine);
             }
             done = true;
             PROFK_STAMP(0, 5);
@@ -385,7 +402,8 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
     // ---- stage 2, general case: radix select over the cluster --------------------------
     if constexpr (GENERAL) {
     if (!done) {
-        __shared__ uint32_t hist[2][SEL_BINS];                       // this CTA's histogram, double-buffered
+        static_assert(sizeof(cand) >= 2 * SEL_BINS * sizeof(uint32_t), "the histograms fit in the candidates' space");
+        uint32_t (*hist)[SEL_BINS] = reinterpret_cast<uint32_t (*)[SEL_BINS]>(cand);   // this CTA's histogram, double-buffered
         constexpr int NPASS = sizeof(T) == 4 ? 3 : 2;
         constexpr int KB = Elem<T>::KEY_BITS;
         const int shifts[3] = {KB - 11, sizeof(T) == 4 ? 10 : 0, 0};
@@ -431,8 +449,32 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
             __syncthreads();   // s_digit / s_before are rewritten in the next pass
         }
         const uint32_t tau_key = prefix << (KB - consumed);
-        if (crank == 0 && tid == 0) publish_threshold(p, row, tau_key);
-        cluster.sync();   // no CTA leaves while a peer may still read its histogram
+        // Of the samples with exactly this key the threshold record is the need-th in sample order.  CTAs hold
+        // consecutive runs of the sample: count the equal keys per CTA, find the CTA that holds the need-th,
+        // and there the position by scans over runs of THREADS keys.
+        uint32_t eq = 0;
+        for (uint32_t i = tid; i < n_local; i += THREADS) eq += keys[i] == tau_key;
+        eq = block_inclusive_scan(eq, warp_sums);
+        if (tid == THREADS - 1) s_ncand = eq;           // (the candidates' counter is free by now)
+        cluster.sync();
+        uint32_t before = 0;
+        for (unsigned c = 0; c < crank; ++c) before += *cluster.map_shared_rank(&s_ncand, c);
+        const uint32_t mine_eq = s_ncand;
+        if (before < need && need <= before + mine_eq) {             // uniform over the CTA
+            uint32_t left = need - before;                           // 1-based among this CTA's equal keys
+            for (uint32_t c0 = 0; c0 < n_local; c0 += THREADS) {
+                const uint32_t i = c0 + tid;
+                const uint32_t flag = i < n_local && keys[i] == tau_key;
+                __syncthreads();                                     // warp_sums of the scan before
+                const uint32_t incl = block_inclusive_scan(flag, warp_sums);
+                if (flag && incl == left) publish_threshold(p, row, tau_key, j0 + i);
+                __syncthreads();
+                const uint32_t in_run = warp_sums[31];
+                if (in_run >= left) break;
+                left -= in_run;
+            }
+        }
+        cluster.sync();   // no CTA leaves while a peer may still read its histogram or its count
     }
     }
     PROFK_STAMP(0, 6);

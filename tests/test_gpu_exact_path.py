@@ -114,7 +114,7 @@ def test_row_counts_around_the_switch_to_the_grid_kernel(rows):
     assert all(s[3] == profk.ROW_OVERFLOW for s in st)
     assert_exact(x, 50, v, i)
     # mixed: only the tie-heavy row fails
-    v, i, st = forced(x.cuda(), 50, profk.Plan(m=2048, r=4, capacity=2000, k_accept=50, mode=0))
+    v, i, st = forced(x.cuda(), 50, profk.Plan(m=2048, r=4, capacity=2000, k_accept=50, mode=0, tie_rule=profk.TIES_KEEP_ALL))
     assert st[rows // 2][3] == profk.ROW_OVERFLOW
     assert_exact(x, 50, v, i)
 

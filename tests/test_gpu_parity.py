@@ -38,18 +38,28 @@ def assert_exact(x: torch.Tensor, k: int, v: np.ndarray, i: np.ndarray):
     assert np.array_equal(bits(v), bits(ov)), "values differ from the oracle"
 
 
+def assert_stats_match(x: torch.Tensor, k: int, pl, seed: int, stats, rows=None):
+    """Threshold, survivor count and outcome of the count check, row by row, against the oracle's run of the four
+    stages under the same plan, seed and tie rule."""
+    xn = workloads.as_numpy(x)
+    xn = xn[None, :] if xn.ndim == 1 else xn
+    for r in (range(xn.shape[0]) if rows is None else rows):
+        res = o_stages.run_row(xn[r], k, pl.m, pl.r, pl.capacity, pl.k_accept, seed=seed, row=r,
+                               composite=getattr(pl, "tie_rule", profk.TIES_BY_INDEX) == profk.TIES_BY_INDEX)
+        tau_bits, R, cap, status = stats[r]
+        assert cap == pl.capacity
+        assert tau_bits == int(bits(np.asarray([res.tau]))[0]), f"row {r}: threshold differs"     # same sample, same threshold
+        assert status == res.status, f"row {r}: status {status}, oracle {res.status}"
+        assert R == res.survivors or (res.survivors > cap and R > cap), f"row {r}: R = {R}, oracle {res.survivors}"
+
+
 # ----------------------------------------------------------------------------- whole call
 def test_config1_uniform_2p20_k64():
     x = workloads.uniform(1 << 20, seed=0)
     v, i = gpu_topk(x, 64, eps=1e-3, seed=0)
     assert_exact(x, 64, v, i)
-    tau_bits, R, cap, status = profk.read_stats(1)[0]
     pl = o_plan.plan_guarded(1 << 20, 64, 1e-3, **profk.default_tuning(1 << 20))     # the oracle's plan on the library's tuning inputs
-    res = o_stages.run_row(workloads.as_numpy(x), 64, pl.m, pl.r, pl.capacity, pl.k_accept, seed=0)
-    assert cap == pl.capacity
-    assert tau_bits == int(np.asarray([res.tau]).view(np.uint32)[0])        # same sample, same threshold
-    assert status == res.status
-    assert R == res.survivors or (res.survivors > cap and R > cap)
+    assert_stats_match(x, 64, pl, 0, profk.read_stats(1))
 
 
 @pytest.mark.parametrize("seed", range(6))
@@ -89,12 +99,13 @@ def test_batched_rows(dtype):
     assert_exact(x, 32, v, i)
     stats = profk.read_stats(24)
     pl = o_plan.plan_guarded(1 << 17, 32, 1e-3, **profk.default_tuning(1 << 17))
-    xn = workloads.as_numpy(x)
-    for r in (0, 7, 23):
-        res = o_stages.run_row(xn[r], 32, pl.m, pl.r, pl.capacity, pl.k_accept, seed=9, row=r)
-        want_tau = int(np.asarray([res.tau]).view(np.uint32 if dtype == torch.float32 else np.uint16)[0])
-        assert stats[r][0] == want_tau and stats[r][3] == res.status
-        assert stats[r][1] == res.survivors or (res.survivors > pl.capacity and stats[r][1] > pl.capacity)
+    assert_stats_match(x, 32, pl, 9, stats)                  # (bf16 rows hold many copies of their threshold)
+    # the same rows with the filter as printed: every copy of the threshold value survives
+    literal = profk.Plan(m=pl.m, r=pl.r, capacity=pl.capacity, k_accept=pl.k_accept, mode=0, tie_rule=profk.TIES_KEEP_ALL)
+    v, i = profk.topk(x.cuda(), 32, plan_override=literal, seed=9)
+    torch.cuda.synchronize()
+    assert_exact(x, 32, workloads.as_numpy(v), i.cpu().numpy())
+    assert_stats_match(x, 32, literal, 9, profk.read_stats(24))
 
 
 # ----------------------------------------------------------------------------- forced failures
@@ -124,13 +135,46 @@ def test_forced_overflow_recall_failure_and_direct_mode(dtype):
 
 
 def test_mixed_rows_some_fail():
-    # rows 0 and 2 hold many copies of their maximum, so their buffers overflow; the others do not
+    # rows 0 and 2 hold many copies of their maximum: with the filter as printed their buffers overflow, the others do not
     x = workloads.normal(4, 150_000, seed=12)
     x[0, ::3] = 9.0
     x[2, 1::2] = 7.5
-    v, i, st = _forced(x, 40, profk.Plan(m=2048, r=4, capacity=2000, k_accept=40, mode=0))
+    pl = profk.Plan(m=2048, r=4, capacity=2000, k_accept=40, mode=0, tie_rule=profk.TIES_KEEP_ALL)
+    v, i, st = _forced(x, 40, pl)
     assert_exact(x, 40, v, i)
     assert [s[3] for s in st] == [profk.ROW_OVERFLOW, profk.ROW_OK, profk.ROW_OVERFLOW, profk.ROW_OK]
+    assert_stats_match(x, 40, pl, 3, st)
+    # with the threshold as a record only the copies up to the threshold's index survive: no row fails
+    pl = profk.Plan(m=2048, r=4, capacity=2000, k_accept=40, mode=0)
+    v, i, st = _forced(x, 40, pl)
+    assert_exact(x, 40, v, i)
+    assert_stats_match(x, 40, pl, 3, st)
+    assert [s[3] for s in st] == [profk.ROW_OK] * 4
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_threshold_record_on_rows_full_of_copies(dtype):
+    # constant rows, rows of a few values, a row whose copies of the threshold straddle tile and row ends, under
+    # both tie rules and for ranks that take the candidate ranking (small t) and the radix path (deep t)
+    n = 400_003
+    g = torch.Generator().manual_seed(31)
+    x = torch.stack([torch.full((n,), 1.25), torch.randint(0, 3, (n,), generator=g).float(),
+                     torch.relu(torch.randn(n, generator=g) - 1.0), torch.zeros(n),
+                     torch.randint(0, 200, (n,), generator=g).float() / 8]).to(dtype)
+    x[3, -5:] = 1.0
+    for m, r, cap in ((4096, 6, 3000), (4096, 200, 40_000), (32768, 3000, 60_000), (1024, 1024, n // 2)):
+        for rule in (profk.TIES_BY_INDEX, profk.TIES_KEEP_ALL):
+            pl = profk.Plan(m=m, r=r, capacity=cap, k_accept=50, mode=0, tie_rule=rule)
+            v, i, st = _forced(x, 50, pl)
+            assert_exact(x, 50, v, i)
+            assert_stats_match(x, 50, pl, 3, st)
+    # one long row: the sample is gathered by its own kernel and selected by a 16-CTA cluster
+    y = torch.randint(0, 4, (6_000_000,), generator=g).float().to(dtype)
+    for m, r in ((131072, 40), (131072, 5000), (16384, 128)):
+        pl = profk.Plan(m=m, r=r, capacity=600_000, k_accept=100, mode=0)
+        v, i, st = _forced(y, 100, pl)
+        assert_exact(y, 100, v, i)
+        assert_stats_match(y, 100, pl, 3, st)
 
 
 def test_k_equals_n_and_plan_direct_mode():
@@ -176,6 +220,26 @@ def test_nan_inf_and_signed_zero_follow_the_total_order():
     xb = x.to(torch.bfloat16)
     v, i = gpu_topk(xb, 1000)
     assert_exact(xb, 1000, v, i)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_survivors_are_counted_in_the_total_order(dtype):
+    # NaNs with the sign bit set rank lowest and -0.0 ranks below +0.0: floating point would count them as
+    # "not below" a threshold they do not reach, and the count check would pass on a buffer without the top-k
+    x = workloads.normal(3, 200_000, seed=19).to(dtype)
+    raw = x.view(torch.int32 if dtype == torch.float32 else torch.int16)
+    neg_nan = -(1 << 22) if dtype == torch.float32 else -(1 << 6)            # 0xFFC00000 / 0xFFC0
+    raw[0, ::7] = neg_nan
+    x[1] = torch.relu(x[1])
+    x[1, ::5] = -0.0                                                          # floods of +0.0 and of -0.0
+    raw[2, ::3] = neg_nan
+    x[2, 1::3] = float("nan")
+    for m, r, cap in ((64, 1, 50_000), (4096, 3000, 190_000), (4096, 2000, 150_000), (2048, 40, 100_000)):
+        for rule in (profk.TIES_BY_INDEX, profk.TIES_KEEP_ALL):
+            pl = profk.Plan(m=m, r=r, capacity=cap, k_accept=10, mode=0, tie_rule=rule)
+            v, i, st = _forced(x, 10, pl)
+            assert_exact(x, 10, v, i)
+            assert_stats_match(x, 10, pl, 3, st)
 
 
 # ----------------------------------------------------------------------------- large selections
