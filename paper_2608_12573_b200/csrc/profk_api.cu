@@ -125,6 +125,8 @@ template <typename T> int ensure_device_info(int dev, DeviceInfo* out) {
                                                                  FILTER_THREADS, 0));
         di.filter_staged_blocks_per_sm[d] = std::max(nb, 1);
         CUDA_TRY(cudaFuncSetAttribute(sample_select_kernel<T, SEL_THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
+        // (the small build holds 33 KB of static shared memory: with 4096 keys it passes the 48 KB that need no opt-in)
+        CUDA_TRY(cudaFuncSetAttribute(sample_select_kernel<T, SEL_SMALL_THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * 1024));
         CUDA_TRY(cudaFuncSetAttribute(refine_kernel<T, 48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFINE_SMEM_MAX));
         CUDA_TRY(cudaFuncSetAttribute(refine_kernel<T, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFINE_SMEM_MAX));
         CUDA_TRY(cudaFuncSetAttribute(fallback_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SORT_CAP_MAX * 8)));

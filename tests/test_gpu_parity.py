@@ -223,6 +223,17 @@ def test_nan_inf_and_signed_zero_follow_the_total_order():
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_batch_with_the_largest_sample_of_the_small_threshold_kernel(dtype):
+    # 80 rows, one 256-thread CTA each, 4096 samples: every sample is a candidate's worth of shared memory
+    x = workloads.normal(80, 100_000, seed=33, dtype=dtype)
+    for r in (1, 20, 32):
+        pl = profk.Plan(m=4096, r=r, capacity=8000, k_accept=16, mode=0)
+        v, i, st = _forced(x, 16, pl)
+        assert_exact(x, 16, v, i)
+        assert_stats_match(x, 16, pl, 3, st, rows=(0, 41, 79))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_survivors_are_counted_in_the_total_order(dtype):
     # NaNs with the sign bit set rank lowest and -0.0 ranks below +0.0: floating point would count them as
     # "not below" a threshold they do not reach, and the count check would pass on a buffer without the top-k
