@@ -197,7 +197,10 @@ int profk_topk_planned_bf16(const void* in, int64_t rows, int64_t N, int64_t k, 
 
 /*
  * Stage 3 alone (the filtering scan of Section 3): for every row append the
- * elements with x_i >= tau[row] to the row's buffer and count them.
+ * elements with x_i >= tau[row] to the row's buffer and count them.  The
+ * comparison is taken in the total order of the values (-NaN < -inf < ... <
+ * -0 < +0 < ... < +inf < +NaN, by bit pattern), the order the sample is
+ * sorted in; the threshold is a value alone (tie rule PROFK_TIES_KEEP_ALL).
  *   tau        [device] rows thresholds of the element type
  *   buf_keys   [device] rows x capacity uint64 candidate records (see below)
  *   counts     [device] rows uint32, must be zero on entry; on return the

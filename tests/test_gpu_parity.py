@@ -222,6 +222,26 @@ def test_nan_inf_and_signed_zero_follow_the_total_order():
     assert_exact(xb, 1000, v, i)
 
 
+def test_failure_rate_on_rows_full_of_ties_stays_within_the_budget():
+    # 256 rows x 8 seeds of a ReLU-Gaussian in bf16 (half the row is one value, the rest repeats by the hundred) and of a
+    # four-valued row: the library's plan at eps = 1e-2, counted over 2048 row-calls each
+    eps, k, n = 1e-2, 64, 1 << 18
+    g = torch.Generator().manual_seed(35)
+    inputs = {"relu bf16": torch.relu(torch.randn((256, n), generator=g)).to(torch.bfloat16),
+              "four values": torch.randint(0, 4, (256, n), generator=g).to(torch.float32)}
+    for name, x in inputs.items():
+        xd = x.cuda()
+        ov, oi = o_topk.topk(workloads.as_numpy(x), k)
+        failed = 0
+        for seed in range(8):
+            v, i = profk.topk(xd, k, eps=eps, seed=seed)
+            torch.cuda.synchronize()
+            assert np.array_equal(i.cpu().numpy(), oi) and np.array_equal(bits(workloads.as_numpy(v)), bits(ov)), (name, seed)
+            failed += sum(1 for st in profk.read_stats(256) if st[3] != profk.ROW_OK)
+        calls = 8 * 256
+        assert failed <= calls * eps + 4 * np.sqrt(calls * eps), (name, failed)
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_batch_with_the_largest_sample_of_the_small_threshold_kernel(dtype):
     # 80 rows, one 256-thread CTA each, 4096 samples: every sample is a candidate's worth of shared memory

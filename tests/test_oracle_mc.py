@@ -47,3 +47,25 @@ def test_failure_rates_at_the_benchmark_shapes(N, k, eps):
     S, t, M = plan.plan_paper(N, k, eps)
     ga, gb = mc.failure_rate_exchangeable(N, S, t, k, M, 20_000, rng)
     assert ga + gb > eps
+
+
+def test_record_threshold_keeps_the_budget_on_rows_full_of_ties():
+    """The four stages run on rows whose values repeat thousands of times: with the threshold taken as a
+    (value, index) record the count check fails no more often than the budget allows, as on distinct values;
+    with the filter as printed the copies of tau overflow the buffer on every run."""
+    from oracle import stages
+    rng = np.random.default_rng(4)
+    N, k, eps = 1 << 15, 16, 5e-2
+    p = plan.plan_guarded(N, k, eps, s_min=1024, s_max=1024)
+    rows = {"constant": np.full(N, 3.0, dtype=np.float32),
+            "four values": rng.integers(0, 4, size=N).astype(np.float32),
+            "relu": np.maximum(rng.standard_normal(N), 0.0).astype(np.float32)}
+    trials = 400
+    for name, x in rows.items():
+        by_record = sum(stages.run_row(x, k, p.m, p.r, p.capacity, p.k_accept, seed=s, composite=True).status != stages.STATUS_OK
+                        for s in range(trials))
+        assert by_record <= trials * eps + 3 * np.sqrt(trials * eps), name
+        if name != "relu":                                           # (relu: the top of the row is distinct values)
+            literal = sum(stages.run_row(x, k, p.m, p.r, p.capacity, p.k_accept, seed=s).status == stages.STATUS_OVERFLOW
+                          for s in range(40))
+            assert literal == 40, name
