@@ -238,7 +238,7 @@ def main():
     else:
         host_inputs = [make_input(cfg, seed_offset=1000 * c + sharding.rank_seed_offset(rank)).pin_memory() for c in range(copies)]
         dev_inputs = [h.to(dev) for h in host_inputs]
-    pl = profk.plan(n, k, eps, recall)
+    pl = profk.plan(n, k, eps, recall, rows=rows)
     profk.ensure_workspace(rows, pl.capacity, k, dev)
     out_vals = torch.empty((rows, k), dtype=dev_inputs[0].dtype, device=dev)
     out_idx = torch.empty((rows, k), dtype=torch.int64, device=dev)

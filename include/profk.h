@@ -114,14 +114,23 @@ typedef struct profk_plan {
 
 /* Tuning inputs of Algorithm 1.  The paper's values (Section 4) are
  * s_min = 32768, s_max = 131072, cost_ratio (tau_B / tau_A) = 1; profk_plan_ex
- * takes them when `tuning` is NULL.  profk_plan and the profk_topk_* entry
- * points use profk_default_tuning(N): the same, except that the floor on the
- * sample size follows the row length for short rows,
- *     s_min = min(32768, max(1024, N / 512)),
- * because on this GPU a sample of 32768 elements touches every 128-byte line of
- * a row of 2^20 elements (the sample pass would read the whole row) and rows of
- * 2^16 elements would not be filtered at all.  Any choice keeps the failure
- * budget: rank and capacity are derived from the bounds for the S in use. */
+ * takes them when `tuning` is NULL.  profk_plan_batch and the profk_topk_*
+ * entry points use profk_default_tuning_batch(rows, N), tuned on B200:
+ *   - the floor on the sample size follows the row length for short rows,
+ *         s_min = min(32768, max(1024, N / 512)),
+ *     because on this GPU a sample of 32768 elements touches every 128-byte
+ *     line of a row of 2^20 elements (the sample pass would read the whole
+ *     row) and rows of 2^16 elements would not be filtered at all;
+ *   - the cost ratio grows with the row length, N / 2^22 clamped to [1, 16]
+ *     for up to PROFK_ALL_SM_GATHER_ROWS rows (their sample is gathered by a
+ *     kernel over all SMs, cheap at any size, while every survivor costs a
+ *     trip through the filter's slow path and a record in the refine step),
+ *     clamped to [1, 4] for larger batches.
+ * profk_default_tuning(N) and profk_plan(N, ...) are the one-row forms.  Any
+ * choice keeps the failure budget: rank and capacity are derived from the
+ * bounds for the S in use. */
+#define PROFK_ALL_SM_GATHER_ROWS 4
+
 typedef struct profk_tuning {
     int64_t s_min;
     int64_t s_max;
@@ -148,7 +157,9 @@ typedef struct profk_row_stats {
  * writes the ones profk_plan uses for a row of length N.
  */
 int profk_default_tuning(int64_t N, profk_tuning_t* tuning /* [host] out */);
+int profk_default_tuning_batch(int64_t rows, int64_t N, profk_tuning_t* tuning /* [host] out */);
 int profk_plan(int64_t N, int64_t k, double eps, double recall, profk_plan_t* out);
+int profk_plan_batch(int64_t rows, int64_t N, int64_t k, double eps, double recall, profk_plan_t* out);
 int profk_plan_ex(int64_t N, int64_t k, double eps, double recall, const profk_tuning_t* tuning,
                   profk_plan_t* out);
 

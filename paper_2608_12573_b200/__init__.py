@@ -16,7 +16,7 @@ _LIB = None
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libprofk.so")
 
 EXPORTS = [
-    "profk_plan", "profk_plan_ex", "profk_default_tuning", "profk_workspace_bytes", "profk_set_workspace",
+    "profk_plan", "profk_plan_batch", "profk_plan_ex", "profk_default_tuning", "profk_default_tuning_batch", "profk_workspace_bytes", "profk_set_workspace",
     "profk_topk_f32", "profk_topk_bf16", "profk_topk_planned_f32", "profk_topk_planned_bf16",
     "profk_filter_f32", "profk_filter_bf16", "profk_sample_threshold_f32", "profk_sample_threshold_bf16",
     "profk_read_stats", "profk_last_launch_count", "profk_strerror", "profk_topk_noalloc_f32",
@@ -90,35 +90,35 @@ _plan_cache: dict = {}
 PAPER_TUNING = dict(s_min=32768, s_max=131072, cost_ratio=1.0)     # Section 4's values of the tuning inputs
 
 
-def default_tuning(N: int) -> dict:
-    """`profk_default_tuning`: the tuning inputs `plan` uses when none are given (the paper's, with the
-    floor on the sample size following the row length for short rows)."""
+def default_tuning(N: int, rows: int = 1) -> dict:
+    """`profk_default_tuning_batch`: the tuning inputs `plan` uses when none are given (the paper's, with the
+    floor on the sample size following the row length for short rows and the cost ratio growing with it)."""
     t = _TuningStruct(0, 0, 0.0)
-    _check(lib().profk_default_tuning(ctypes.c_int64(N), ctypes.byref(t)), "profk_default_tuning")
+    _check(lib().profk_default_tuning_batch(ctypes.c_int64(rows), ctypes.c_int64(N), ctypes.byref(t)), "profk_default_tuning_batch")
     return dict(s_min=int(t.s_min), s_max=int(t.s_max), cost_ratio=float(t.cost_ratio))
 
 
 def plan(N: int, k: int, eps: float = 1e-3, recall: float = 1.0, s_min: int | None = None,
-         s_max: int | None = None, cost_ratio: float | None = None) -> Plan:
-    """`profk_plan` / `profk_plan_ex`: the parameters (S, t, M) for one row of length N.  Without tuning
-    inputs: the library's defaults (`default_tuning`); `plan(N, k, eps, recall, **PAPER_TUNING)` gives the
-    paper's."""
-    key = (N, k, eps, recall, s_min, s_max, cost_ratio)
+         s_max: int | None = None, cost_ratio: float | None = None, rows: int = 1) -> Plan:
+    """`profk_plan_batch` / `profk_plan_ex`: the parameters (S, t, M) for rows of length N.  Without tuning
+    inputs: the library's defaults for a call with `rows` rows (`default_tuning`);
+    `plan(N, k, eps, recall, **PAPER_TUNING)` gives the paper's."""
+    key = (N, k, eps, recall, s_min, s_max, cost_ratio, rows)
     hit = _plan_cache.get(key)
     if hit is not None:
         return hit
-    res = _plan_uncached(N, k, eps, recall, s_min, s_max, cost_ratio)
+    res = _plan_uncached(N, k, eps, recall, s_min, s_max, cost_ratio, rows)
     if len(_plan_cache) > 4096:
         _plan_cache.clear()
     _plan_cache[key] = res
     return res
 
 
-def _plan_uncached(N, k, eps, recall, s_min, s_max, cost_ratio) -> Plan:
+def _plan_uncached(N, k, eps, recall, s_min, s_max, cost_ratio, rows) -> Plan:
     out = _PlanStruct()
     if s_min is None and s_max is None and cost_ratio is None:
-        code = lib().profk_plan(ctypes.c_int64(N), ctypes.c_int64(k), ctypes.c_double(eps),
-                                ctypes.c_double(recall), ctypes.byref(out))
+        code = lib().profk_plan_batch(ctypes.c_int64(rows), ctypes.c_int64(N), ctypes.c_int64(k), ctypes.c_double(eps),
+                                      ctypes.c_double(recall), ctypes.byref(out))
     else:
         tun = _TuningStruct(32768 if s_min is None else s_min, 131072 if s_max is None else s_max,
                             1.0 if cost_ratio is None else cost_ratio)
@@ -201,7 +201,7 @@ def topk(x, k: int, eps: float = 1e-3, recall: float = 1.0, seed: int = 0, plan_
     one_d = x.dim() == 1
     x2 = _rows_view(x)
     rows, n = x2.shape
-    pl = plan_override if plan_override is not None else plan(n, k, eps, recall)
+    pl = plan_override if plan_override is not None else plan(n, k, eps, recall, rows=rows)
     ensure_workspace(rows, pl.capacity, k, x2.device)
     if out is None:
         vals = torch.empty((rows, k), dtype=x2.dtype, device=x2.device)

@@ -159,19 +159,39 @@ extern "C" int profk_plan_ex(int64_t N, int64_t k, double eps, double recall, co
 // element, so 32768 samples of a 2^20-element row read the whole row once before the filtering scan reads
 // it again, and 2^16-element rows would not be filtered at all (N <= 2 S).  The guarded rank and capacity
 // keep the failure budget for any S.
-extern "C" int profk_default_tuning(int64_t N, profk_tuning_t* tuning) {
-    if (!tuning || N < 1) return PROFK_EINVAL;
+//
+// The cost ratio tau_B / tau_A of Eq. (cost_model) -- what a unit of buffer work costs against a sampled
+// element -- is 1 in the paper and grows here with the row length, N / 2^22 clamped to [1, 16] for up to
+// PROFK_ALL_SM_GATHER_ROWS rows and to [1, 4] for larger batches: the sample of a long row is gathered by a
+// kernel over all SMs in a few microseconds whatever its size, while every survivor costs a trip through the
+// filter's slow path and a record in the refine step.  Measured on B200: 2^26, k = 256, eps = 1e-4: 51.3 -> 49.0 us;
+// k = 4096: 63.6 -> 60.0; 2^30 Cauchy, k = 64: 631 -> 610; four rows of 2^26, k = 256: 187 -> 167; rows of 2^22 and
+// shorter are planned as before.  S_max stays Section 4's 131072: with 262144 the selection of a deep rank among
+// so many keys cost the flattened BatchTopK shape (2^29, K = 131072) 16 us and gained the others 1-2.
+extern "C" int profk_default_tuning_batch(int64_t rows, int64_t N, profk_tuning_t* tuning) {
+    if (!tuning || N < 1 || rows < 1) return PROFK_EINVAL;
     int64_t s_min = N / 512;
     if (s_min < 1024) s_min = 1024;
     if (s_min > 32768) s_min = 32768;
+    const bool all_sm_gather = rows <= PROFK_ALL_SM_GATHER_ROWS;
+    double ratio = (double)N / 4194304.0;
+    const double ratio_max = all_sm_gather ? 16.0 : 4.0;
+    if (ratio < 1.0) ratio = 1.0;
+    if (ratio > ratio_max) ratio = ratio_max;
     tuning->s_min = s_min;
     tuning->s_max = 131072;
-    tuning->cost_ratio = 1.0;
+    tuning->cost_ratio = ratio;
     return PROFK_OK;
 }
 
-extern "C" int profk_plan(int64_t N, int64_t k, double eps, double recall, profk_plan_t* out) {
+extern "C" int profk_default_tuning(int64_t N, profk_tuning_t* tuning) { return profk_default_tuning_batch(1, N, tuning); }
+
+extern "C" int profk_plan_batch(int64_t rows, int64_t N, int64_t k, double eps, double recall, profk_plan_t* out) {
     profk_tuning_t tuning;
-    if (profk_default_tuning(N, &tuning) != PROFK_OK) return PROFK_EINVAL;
+    if (profk_default_tuning_batch(rows, N, &tuning) != PROFK_OK) return PROFK_EINVAL;
     return profk_plan_ex(N, k, eps, recall, &tuning, out);
+}
+
+extern "C" int profk_plan(int64_t N, int64_t k, double eps, double recall, profk_plan_t* out) {
+    return profk_plan_batch(1, N, k, eps, recall, out);
 }

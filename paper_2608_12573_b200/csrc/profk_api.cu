@@ -29,7 +29,7 @@ constexpr int FILTER_THREADS = PROFK_FILTER_THREADS;
 constexpr int FILTER_UNROLL = PROFK_FILTER_UNROLL;
 constexpr uint32_t SORT_CAP_MAX = 16384;         // largest k the single-CTA refine orders in shared memory
 constexpr unsigned FB_MAX_CTAS = 256;             // most CTAs of the grid-wide exact selection (its per-CTA scratch is sized for them)
-constexpr int64_t GATHER_MAX_ROWS = 4;           // most rows for which the sample may be gathered by a kernel of its own
+constexpr int64_t GATHER_MAX_ROWS = PROFK_ALL_SM_GATHER_ROWS;   // most rows for which the sample may be gathered by a kernel of its own
 constexpr int LARGE_MAX_CTAS = 1024;             // CTAs of the large refine (its per-CTA slots live in the 48 KB histogram area)
 constexpr int64_t XS_MAX_ROWS = 18;              // most rows for which the refine kernel itself replaces failed rows
 constexpr unsigned XS_MAX_SEGMENTS = 32;         // most (row, segment) pairs of that exact selection
@@ -57,7 +57,7 @@ struct Workspace { void* ptr = nullptr; size_t bytes = 0; };
 std::mutex g_mutex;
 std::map<int, DeviceInfo> g_devinfo;
 std::map<int, Workspace> g_workspace;
-std::map<std::tuple<int64_t, int64_t, double, double>, profk_plan_t> g_plan_cache;
+std::map<std::tuple<int64_t, int64_t, int64_t, double, double>, profk_plan_t> g_plan_cache;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -524,10 +524,11 @@ int topk_auto(const T* in, int64_t rows, int64_t N, int64_t k, double eps, doubl
     profk_plan_t plan;
     {
         std::lock_guard<std::mutex> lock(g_mutex);
-        const auto key = std::make_tuple(N, k, eps, recall);
+        const int64_t plan_rows = rows <= GATHER_MAX_ROWS ? 1 : GATHER_MAX_ROWS + 1;     // the two classes the tuning knows
+        const auto key = std::make_tuple(plan_rows, N, k, eps, recall);
         auto it = g_plan_cache.find(key);
         if (it == g_plan_cache.end()) {
-            const int rc = profk_plan(N, k, eps, recall, &plan);
+            const int rc = profk_plan_batch(plan_rows, N, k, eps, recall, &plan);
             if (rc != PROFK_OK) return rc;
             if (g_plan_cache.size() > 4096) g_plan_cache.clear();
             g_plan_cache[key] = plan;
@@ -662,9 +663,10 @@ int profk_topk_noalloc_f32(const float* in, int64_t rows, int64_t N, int64_t k, 
         scratch = it->second;
     }
     profk_plan_t plan;
-    const int prc = profk_plan(N, k, eps, recall, &plan);
+    if (rows < 1) return PROFK_EINVAL;
+    const int prc = profk_plan_batch(rows, N, k, eps, recall, &plan);
     if (prc != PROFK_OK) return prc;
-    if (rows < 1 || rows * plan.capacity >= (1LL << 40)) return PROFK_EINVAL;
+    if ( rows * plan.capacity >= (1LL << 40)) return PROFK_EINVAL;
     if (ws_layout(rows, plan.capacity, k).total > NOALLOC_SCRATCH_BYTES) return PROFK_ETOOLARGE;
     g_ws_override_ptr = scratch;
     g_ws_override_bytes = NOALLOC_SCRATCH_BYTES;

@@ -42,16 +42,19 @@ SHAPES = [(2 ** 20, 64, 1e-3, 1.0), (2 ** 26, 16, 1e-2, 1.0), (2 ** 26, 16, 1e-4
 
 
 @pytest.mark.parametrize("N,k,eps,recall", SHAPES)
-@pytest.mark.parametrize("tuning", ["paper", "library"])
+@pytest.mark.parametrize("tuning", ["paper", "library", "library, batch"])
 def test_host_plan_equals_oracle_plan(lib, N, k, eps, recall, tuning):
     if tuning == "paper":        # Section 4's S_min = 32768, S_max = 2^17, cost ratio 1: the oracle's defaults
         got = profk.plan(N, k, eps, recall, **profk.PAPER_TUNING)
         want = oracle_plan.plan_guarded(N, k, eps, recall)
-    else:                        # the library's own floor for short rows, handed to the oracle as a tuning input
+    else:                        # the library's own tuning inputs (a floor that follows short rows, a cost ratio that grows
+        rows = 1 if tuning == "library" else 5      # with long ones), handed to the oracle as tuning inputs
         s_min = min(32768, max(1024, N // 512))
-        assert profk.default_tuning(N) == dict(s_min=s_min, s_max=131072, cost_ratio=1.0)
-        got = profk.plan(N, k, eps, recall)
-        want = oracle_plan.plan_guarded(N, k, eps, recall, s_min=s_min)
+        ratio = min(max(N / 2 ** 22, 1.0), 16.0 if rows <= 4 else 4.0)
+        s_max = 131072
+        assert profk.default_tuning(N, rows=rows) == dict(s_min=s_min, s_max=s_max, cost_ratio=ratio)
+        got = profk.plan(N, k, eps, recall, rows=rows)
+        want = oracle_plan.plan_guarded(N, k, eps, recall, s_min=s_min, s_max=s_max, cost_ratio=ratio)
     assert (got.m, got.r, got.capacity, got.k_accept, got.mode) == (want.m, want.r, want.capacity, want.k_accept, want.mode)
     assert got.z == pytest.approx(want.z, rel=1e-12)
     assert got.alpha == want.alpha

@@ -36,7 +36,7 @@ def test_noalloc_entry_matches_the_ordinary_one_twice_in_a_row():
     for rows, n, k in shapes:
         xs = [workloads.normal(rows, n, seed=40 + r).cuda() for r in range(2)]      # two different inputs, two calls in a row
         # reference: the existing entry point, with a registered workspace
-        pl = profk.plan(n, k, 1e-3)
+        pl = profk.plan(n, k, 1e-3, rows=rows)
         profk.ensure_workspace(rows, pl.capacity, k, xs[0].device)
         want = []
         for r, x in enumerate(xs):
