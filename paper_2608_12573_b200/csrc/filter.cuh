@@ -58,7 +58,13 @@ template <typename T> struct FilterParams {
     // pattern only those with an index <= tau_idx are kept (0xFFFFFFFF: all of them), so that a flood of copies of tau
     // does not fill the buffer.
     const uint4* thr;
+    // Tiles (0 or FILTER_PREFETCH) a CTA copies into its shared memory while it waits for the threshold kernel, beyond
+    // the one it holds in registers: the input does not depend on the threshold, and HBM is idle meanwhile.
+    uint32_t prefetch_tiles;
 };
+
+constexpr uint32_t FILTER_PREFETCH = 2;
+constexpr uint32_t PREFETCH_SPIN_LIMIT = 1u << 22;
 
 // Bit l set = element l of the vector is not below tau (the same test as vec_any_pass, per element).
 __device__ __forceinline__ unsigned vec_pass_mask(const float4& v, float tau) {
@@ -372,6 +378,8 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
     constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
     __shared__ WarpStage stages[STAGED ? THREADS / 32 : 1];
     __shared__ uint32_t s_next[2];
+    __shared__ __align__(8) uint64_t pf_bar;                         // counts the bytes of the prefetched tiles
+    extern __shared__ __align__(128) unsigned char pf_smem[];        // p.prefetch_tiles tiles of 32 KB (or nothing)
 
     const unsigned lane = lane_id();
     WarpStage* st = &stages[STAGED ? threadIdx.x >> 5 : 0];
@@ -393,12 +401,20 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
     uint32_t inside_mask;                        // bit u: vector u holds at least one element of the row
     // Row and position of `tile`, and its loads.  A tile that lies wholly inside its row -- all but the first
     // and the last of a row -- is four plain 128-bit loads off one pointer; the others take the checked path.
+    uint32_t pf_left = 0;                        // tiles still waiting in shared memory (single rows only)
     auto decode_and_load = [&](bool first_time) {
         uint32_t nrow = 0, tin = tile;
         if (!one_row) { nrow = tile / tiles_per_row; tin = tile - nrow * tiles_per_row; }
         qbase = (uint64_t)tin * TILE_VECTORS;
         if (first_time || nrow != row) { row = nrow; rv = row_view(p.in, p.N, row); }
-        if (qbase * VEC >= rv.mis && (qbase + TILE_VECTORS) * VEC <= p.N + rv.mis) {
+        if (pf_left) {
+            // one of the tiles copied into shared memory before the wait for the threshold kernel
+            const V* src = reinterpret_cast<const V*>(pf_smem) + (size_t)(p.prefetch_tiles - pf_left) * TILE_VECTORS + threadIdx.x;
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) v[u] = src[u * THREADS];
+            inside_mask = ALL_INSIDE;
+            --pf_left;
+        } else if (qbase * VEC >= rv.mis && (qbase + TILE_VECTORS) * VEC <= p.N + rv.mis) {
             const V* ptr = reinterpret_cast<const V*>(rv.aligned_base) + qbase + threadIdx.x;
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) v[u] = ld_stream(ptr + u * THREADS);
@@ -417,10 +433,51 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
     // The first tile's loads are issued before waiting on the threshold kernel: the input does not depend on it.
     decode_and_load(true);
 
+    // So are bulk copies of the CTA's next tiles into shared memory, when the launch asked for them (a single row,
+    // tiles that lie wholly inside it and are dealt by the fixed stride): one thread issues them, an mbarrier counts
+    // their bytes, and everybody waits on it -- with a limit -- when the first of them is due.
+    bool pf_ok = false;
+    if (p.prefetch_tiles) {
+        const uint64_t last = (uint64_t)tile + (uint64_t)p.prefetch_tiles * gridDim.x;          // last tile to copy
+        pf_ok = one_row && last < p.dyn_start && (uint64_t)tile * TILE_VECTORS * VEC >= rv.mis &&
+                (last + 1) * TILE_VECTORS * VEC <= p.N + rv.mis;
+        if (pf_ok) {
+            const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&pf_bar);
+            if (threadIdx.x == 0) {
+                asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
+                asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(p.prefetch_tiles * TILE_VECTORS * 16u) : "memory");
+                for (uint32_t j = 0; j < p.prefetch_tiles; ++j) {
+                    const V* src = reinterpret_cast<const V*>(rv.aligned_base) + ((uint64_t)tile + (uint64_t)(j + 1) * gridDim.x) * TILE_VECTORS;
+                    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(pf_smem + (size_t)j * TILE_VECTORS * 16u);
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(dst), "l"(src), "r"(TILE_VECTORS * 16u), "r"(bar) : "memory");
+                }
+            }
+            __syncthreads();            // the barrier is initialised before anyone may wait on it
+        }
+    }
+
     PROFK_STAMP(0, 10);
     if (p.use_pdl) pdl_wait();
     pdl_launch_dependents();            // the refine kernel may be staged behind this one
     PROFK_STAMP(0, 11);
+    // The copies were issued microseconds ago; should they not have landed within the limit, the tiles are read with
+    // plain loads instead and the copies are waited for once more before the CTA leaves.
+    auto prefetch_landed = [&]() {
+        const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&pf_bar);
+        for (uint32_t spin = 0; spin < PREFETCH_SPIN_LIMIT; ++spin) {
+            uint32_t done;
+            asm volatile("{\n\t.reg .pred q;\n\tmbarrier.try_wait.parity.shared::cta.b64 q, [%1], 0;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+                         : "=r"(done) : "r"(bar) : "memory");
+            if (done) return true;
+        }
+        return false;
+    };
+    bool pf_pending = false;
+    if (pf_ok) {
+        if (prefetch_landed()) pf_left = p.prefetch_tiles; else pf_pending = true;
+    }
 
     uint32_t skip_row = 0xFFFFFFFFu;    // row whose buffer this warp has seen overflow: nothing more to append
     uint32_t parity = 0;
@@ -491,6 +548,7 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
         if (row != tau_row) { tau_row = row; load_threshold(); }
     }
     if (STAGED && st->fill) flush_stage(p, st);
+    if (pf_pending) prefetch_landed();
     PROFK_STAMP(0, 12);
 #ifdef PROFK_TRACE
     if (threadIdx.x == 0) {
