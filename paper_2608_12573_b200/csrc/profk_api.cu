@@ -125,8 +125,9 @@ template <typename T> int ensure_device_info(int dev, DeviceInfo* out) {
                                                                  FILTER_THREADS, 0));
         di.filter_staged_blocks_per_sm[d] = std::max(nb, 1);
         CUDA_TRY(cudaFuncSetAttribute(sample_select_kernel<T, SEL_THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
-        CUDA_TRY(cudaFuncSetAttribute(filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)(FILTER_PREFETCH * FILTER_THREADS * FILTER_UNROLL * 16u)));
+        const int prefetch_bytes = (int)(FILTER_PREFETCH * FILTER_THREADS * FILTER_UNROLL * 16u);
+        CUDA_TRY(cudaFuncSetAttribute(filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, prefetch_bytes));
+        CUDA_TRY(cudaFuncSetAttribute(filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, prefetch_bytes));
         // (the small build holds 33 KB of static shared memory: with 4096 keys it passes the 48 KB that need no opt-in)
         CUDA_TRY(cudaFuncSetAttribute(sample_select_kernel<T, SEL_SMALL_THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * 1024));
         CUDA_TRY(cudaFuncSetAttribute(refine_kernel<T, 48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFINE_SMEM_MAX));
@@ -271,7 +272,8 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     if (rounds <= PROFK_DYNAMIC_ROUNDS) fp.tile_counter = nullptr;
     cfg.blockDim = dim3(FILTER_THREADS);
     // A single row scanned behind the threshold kernel: each CTA copies its next tiles into shared memory while it waits.
-    const bool prefetch = pdl && !staged && !parts && rows == 1 && fp.dyn_start >= (FILTER_PREFETCH + 1) * cfg.gridDim.x;
+    // (Not the staged build: its two CTAs per SM spill already, and the copies cost the 2^29 bf16 row 3 us.)
+    const bool prefetch = pdl && !staged && rows == 1 && fp.dyn_start >= (FILTER_PREFETCH + 1) * cfg.gridDim.x;
     fp.prefetch_tiles = prefetch ? FILTER_PREFETCH : 0u;
     cfg.dynamicSmemBytes = prefetch ? FILTER_PREFETCH * FILTER_THREADS * FILTER_UNROLL * 16u : 0;
     cfg.stream = st;
