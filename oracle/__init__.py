@@ -2,7 +2,7 @@
 
 Everything in this package is a plain, slow, CPU-only restatement of what the
 GPU path has to compute, written from the paper so that a reader can check it
-against the paper by eye.  It exists to judge the CUDA library; it is not a
+against the paper by eye.  It exists to check the CUDA library; it is not a
 fallback for it.  Only the tests, the smoke check and the CPU-baseline leg of
 the benchmark may import it.  It shares no code with the CUDA sources: the
 order-preserving key transform, the parameter formulas, the binomial / hyper-
