@@ -29,6 +29,8 @@ constexpr int FILTER_THREADS = PROFK_FILTER_THREADS;
 constexpr int FILTER_UNROLL = PROFK_FILTER_UNROLL;
 constexpr uint32_t SORT_CAP_MAX = 16384;         // largest k the single-CTA refine orders in shared memory
 constexpr unsigned FB_MAX_CTAS = 256;             // most CTAs of the grid-wide exact selection (its per-CTA scratch is sized for them)
+// Samples above this size are gathered by a kernel over all SMs (65536: 2^26, k = 16, S = 40529 took 49.7 us, not 47.0).
+constexpr int64_t GATHER_MIN_SAMPLE = 32768;
 constexpr int64_t GATHER_MAX_ROWS = PROFK_ALL_SM_GATHER_ROWS;   // most rows for which the sample may be gathered by a kernel of its own
 constexpr int LARGE_MAX_CTAS = 1024;             // CTAs of the large refine (its per-CTA slots live in the 48 KB histogram area)
 constexpr int64_t XS_MAX_ROWS = 18;              // most rows for which the refine kernel itself replaces failed rows
@@ -196,7 +198,7 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
     // A large sample, or a sample of a very long row (every element on a page of its own), is gathered by a
     // kernel over all SMs first; the cluster then only selects.
     const bool spread_gather = keys_scratch != nullptr && rows <= GATHER_MAX_ROWS &&
-                               (m > 65536 || (int64_t)N * (int64_t)sizeof(T) >= (512LL << 20));
+                               (m > GATHER_MIN_SAMPLE || (int64_t)N * (int64_t)sizeof(T) >= (512LL << 20));
     if (spread_gather) {
         GatherParams<T> gp;
         gp.in = in; gp.N = (uint64_t)N; gp.rows = (uint64_t)rows; gp.S = (uint32_t)m; gp.seed = seed;
