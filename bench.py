@@ -35,6 +35,9 @@ CONFIGS = {
     "cfg3_f32": (512, 1 << 20, "f32", "normal", 2, 32, 1e-3, 1.0),
     "cfg3_bf16": (512, 1 << 20, "bf16", "normal", 2, 32, 1e-3, 1.0),
     "cfg4": (1, 1 << 29, "bf16", "relu_gaussian", 3, 32 * 4096, 1e-3, 1.0),
+    # the shape of Section 5's sparse-autoencoder measurement: N = 50,331,648 flattened activations, K = 131,072
+    "cfg4_sae_f32": (1, 50331648, "f32", "relu_gaussian", 3, 131072, 1e-3, 1.0),
+    "cfg4_sae_bf16": (1, 50331648, "bf16", "relu_gaussian", 3, 131072, 1e-3, 1.0),
     "cfg5_cauchy_k64": (1, 1 << 30, "f32", "cauchy", 4, 64, 1e-3, 1.0),
     "cfg5_cauchy_k65536": (1, 1 << 30, "f32", "cauchy", 4, 65536, 1e-3, 1.0),
     "cfg5_pareto_k1": (1, 1 << 30, "f32", "pareto", 5, 1, 1e-3, 1.0),

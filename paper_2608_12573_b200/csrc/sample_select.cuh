@@ -7,8 +7,9 @@
 //     answer from the maxima of 128 groups of its keys (the t-th largest group maximum has
 //     at least t keys at or above it), sends only its keys >= L to the first CTA through
 //     distributed shared memory (remote atomics and stores), and the first CTA ranks those
-//     few candidates directly;
-//   * otherwise (deep ranks, or so many ties that the candidates do not fit) a radix select
+//     few candidates directly; for ranks up to 128 per CTA of the cluster the bound is the smallest over the
+//     CTAs of their ceil(t / csize)-th largest group maxima, and the candidates are ranked by the whole cluster;
+//   * otherwise (deeper ranks, or so many ties that the candidates do not fit) a radix select
 //     whose per-digit histograms are summed across the cluster through distributed shared
 //     memory.
 // Only hardware cluster barriers are used -- no spinning on global memory.
@@ -209,7 +210,7 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
     __shared__ uint64_t cand[SEL_CAND_CAP];
     __shared__ uint32_t gmax[GROUPS];
     __shared__ uint32_t warp_sums[32];
-    __shared__ uint32_t s_digit, s_before, s_ncand, s_lower;
+    __shared__ uint32_t s_digit, s_before, s_ncand, s_lower, s_lmin;
 
     cg::cluster_group cluster = cg::this_cluster();
     const unsigned csize = cluster.num_blocks();
@@ -223,7 +224,7 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
     if (threadIdx.x == 0 && blockIdx.x == 0) { g_profk_trace[2][13] = 0; g_profk_trace[2][14] = 0x7FFFFFFFFFFFFFFFll; }
 #endif
 
-    if (tid == 0) { s_ncand = 0; s_lower = 0; }
+    if (tid == 0) { s_ncand = 0; s_lower = 0; s_lmin = 0xFFFFFFFFu; }
     __syncthreads();
     // Split barrier: "my candidate counter is zero".  Peers wait for it only after their gather,
     // by which time every CTA has long arrived.
@@ -314,9 +315,14 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
     bool done = false;
 
     // ---- stage 2, short cut for small ranks -------------------------------------------
+    // Deeper ranks, up to GROUPS per CTA of the cluster: every CTA takes the ceil(t / csize)-th largest of its group
+    // maxima -- it has that many keys at or above it -- and the smallest of these bounds over the cluster has
+    // csize * ceil(t / csize) >= t keys at or above it: one more exchange through the first CTA's shared memory.
     const bool bounded = p.t <= (uint32_t)GROUPS;
-    if (bounded || !GENERAL) {
-        if (bounded) {
+    const uint32_t cta_rank = bounded ? p.t : (p.t + csize - 1) / csize;
+    const bool wide = GENERAL && !bounded && csize > 1 && cta_rank <= (uint32_t)GROUPS;
+    if (bounded || wide || !GENERAL) {
+        if (bounded || wide) {
         // maxima of the groups of 8 consecutive lanes
         uint32_t g = my_max;
         g = max(g, __shfl_xor_sync(FULL_MASK, g, 1));
@@ -337,16 +343,22 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
             rank += __shfl_xor_sync(FULL_MASK, rank, 1);
             rank += __shfl_xor_sync(FULL_MASK, rank, 2);
             rank += __shfl_xor_sync(FULL_MASK, rank, 4);
-            if (part == 0 && rank == p.t - 1) s_lower = mine;     // at least t keys of this CTA are >= mine
+            if (part == 0 && rank == cta_rank - 1) s_lower = mine;     // at least cta_rank keys of this CTA are >= mine
         }
         }                                   // (not bounded: the bound stays 0 and every key is a candidate)
         __syncthreads();
-        const uint32_t lower = s_lower;
+        uint32_t lower = s_lower;
         PROFK_STAMP(0, 2);
         // every CTA sends its keys >= lower to the first CTA: one remote atomic per warp that has any
         uint64_t* cand0 = cluster.map_shared_rank(cand, 0);
         uint32_t* ncand0 = cluster.map_shared_rank(&s_ncand, 0);
         cluster.barrier_wait(std::move(zeroed));
+        if (wide) {
+            uint32_t* lmin0 = cluster.map_shared_rank(&s_lmin, 0);
+            if (tid == 0) atomicMin(lmin0, lower);
+            cluster.sync();
+            lower = *lmin0;
+        }
         for (uint32_t i = tid; i < n_round; i += THREADS) {
             const uint32_t k = i < n_local ? keys[i] : 0;
             const bool take = i < n_local && k >= lower;

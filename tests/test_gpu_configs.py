@@ -88,6 +88,21 @@ def test_config4_flattened_batchtopk_2p29_bf16():
     assert st[2] == o_plan.plan_guarded(n, k, 1e-3, **profk.default_tuning(n)).capacity
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_flattened_batchtopk_at_the_papers_sae_shape(dtype):
+    # Section 5's measurement shape: N = 50,331,648 flattened activations, K = 131,072; small enough for the full sort
+    n, k = 50_331_648, 131_072
+    x = workloads.relu_gaussian(n, seed=3, dtype=dtype)
+    xn = workloads.as_numpy(x)
+    ov, oi = o_topk.topk_row(xn, k)
+    xd = x.cuda()
+    for seed in (0, 1):
+        v, i = run(xd, k, eps=1e-3, seed=seed)
+        assert np.array_equal(i, oi) and np.array_equal(bits(v), bits(ov)), seed
+    st = profk.read_stats(1)[0]
+    assert st[2] == o_plan.plan_guarded(n, k, 1e-3, **profk.default_tuning(n)).capacity
+
+
 @pytest.mark.parametrize("name", ["cauchy", "pareto", "sorted", "few_values", "spikes"])
 def test_config5_adversarial_2p30(name):
     n = 1 << 30

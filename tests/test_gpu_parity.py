@@ -316,6 +316,12 @@ def test_sample_indices_and_threshold_match_the_oracle(dtype):
         assert np.array_equal(sidx[row].cpu().numpy().astype(np.int64) & 0xFFFFFFFF, want_idx)
         want_tau = o_stages.threshold(xn[row], want_idx, r)
         assert bits(workloads.as_numpy(tau[row:row + 1]))[0] == bits(np.asarray([want_tau]))[0]
+    # ranks beyond 128 that the cluster still bounds from its group maxima (up to 128 per CTA)
+    for m2, r2 in ((131072, 405), (131072, 2048), (40000, 129), (65536, 1500)):
+        tau = profk.sample_threshold(x[:1].cuda(), m2, r2, seed=6)
+        torch.cuda.synchronize()
+        want = o_stages.threshold(xn[0], o_philox.sample_indices(n, m2, 6, 0), r2)
+        assert bits(workloads.as_numpy(tau))[0] == bits(np.asarray([want]))[0], (m2, r2)
     # large sample spread over an 8-CTA cluster, deep rank
     tau = profk.sample_threshold(x[:1].cuda(), 131072, 9000, seed=5)
     torch.cuda.synchronize()
