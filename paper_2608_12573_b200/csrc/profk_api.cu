@@ -455,7 +455,10 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     // Survivors are staged per warp when a warp's tile is expected to hold a good fraction of one
     // (expected survivors per element ~ r / m); sparse survivors are appended directly.
     const double per_warp_tile = (double)plan->r / (double)std::max<int64_t>(plan->m, 1) * 32.0 * FILTER_UNROLL * Elem<T>::VEC;
-    const bool staged = plan->mode == 0 && rows == 1 && per_warp_tile > 0.25;
+        // (The direct append has three CTAs per SM, eight counters for large selections and the prefetch behind the threshold
+    // kernel; it holds up to about two survivors per warp-tile: 2^29 bf16, K = 131072 at 0.4: 248 -> 237 us; 50 M fp32,
+    // K = 131072 at 1.6: 124 -> 114; 50 M bf16 at 3.2 stays staged, 120 against 127.)
+    const bool staged = plan->mode == 0 && rows == 1 && per_warp_tile > 2.0;
 
     // Large selections keep so many survivors that a row's single append counter would hold the scan up:
     // the direct variant then appends to FILTER_PARTS parts of the buffer, each with a counter of its own.
