@@ -137,10 +137,21 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         uint32_t* bins = p.bins + row * (uint64_t)(LG_BINS + 8);
         uint32_t* flags = bins + LG_BINS;                                // [0] = some bin that matters is crowded
         // every record of the row once, spread over the grid's threads
+        // (The parts are walked as one run of sum(pcount) positions: part by part, a part of 20 K records would
+        // keep one thread in seven of the grid busy and cost a memory round trip of its own, eight per pass.)
+        uint32_t pend[8];                                                // pend[j] = records in parts 0..j
+        {
+            uint32_t acc = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { acc += pcount[j]; pend[j] = acc; }
+        }
         auto for_each_record = [&](auto&& f) {
-            for (uint32_t j = 0; j < nparts; ++j) {
-                const uint64_t* part = G + (uint64_t)j * p.part_cap;
-                for (uint64_t i = gid; i < pcount[j]; i += gthreads) f((unsigned long long)__ldcg(&part[i]));
+            for (uint64_t i = gid; i < pend[7]; i += gthreads) {
+                uint32_t j = 0, before = 0;
+#pragma unroll
+                for (int q = 0; q < 7; ++q)
+                    if (i >= pend[q]) { j = q + 1; before = pend[q]; }
+                f((unsigned long long)__ldcg(G + (uint64_t)j * p.part_cap + (i - before)));
             }
         };
 
