@@ -10,6 +10,13 @@ namespace profk {
 
 constexpr unsigned FULL_MASK = 0xFFFFFFFFu;
 
+// Partitioned append of the filter (large selections): parts of a row's buffer, each with a counter of its own.
+#ifndef PROFK_FILTER_PARTS
+#define PROFK_FILTER_PARTS 8
+#endif
+constexpr uint32_t FILTER_PARTS = PROFK_FILTER_PARTS;
+constexpr uint32_t FILTER_PART_STRIDE = 64;     // words between two counters: 256 bytes
+
 // ---------------------------------------------------------------------------------------
 // Order keys.  key(x) is an unsigned integer whose order is the total order
 // -NaN < -inf < ... < -0 < +0 < ... < +inf < +NaN of the bit patterns.  Keys travel in 32-bit

@@ -129,8 +129,6 @@ __device__ __forceinline__ unsigned confirm_survivors(const FilterParams<T>& p, 
     return vec_any_equal_or_unordered(v, tau) ? confirm_each<T>(p, row, v, m, i0, tau) : m;
 }
 
-constexpr uint32_t FILTER_PARTS = 8;
-constexpr uint32_t FILTER_PART_STRIDE = 64;     // words between two counters: 256 bytes
 
 // not (x < tau) for every lane of a vector, OR-ed: does the vector hold any survivor?
 __device__ __forceinline__ bool vec_any_pass(const float4& v, float tau) {

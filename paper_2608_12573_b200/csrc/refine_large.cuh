@@ -36,7 +36,7 @@ template <typename T> struct LargeParams {
     uint32_t* bins;          // rows x (LG_BINS + 8) words: bin counts / positions, then flags
     unsigned long long* slots;   // 2 words per CTA of the grid, then one per CTA: per-CTA minima / maxima and scan totals
     uint32_t groups;         // CTA groups the grid is cut into (<= WS_GROUPS; gridDim.x is a multiple of it)
-    uint32_t parts;          // 1, or 8: the filter appended to that many parts of the row's buffer (first phase only)
+    uint32_t parts;          // 1, or FILTER_PARTS: the filter appended to that many parts of the row's buffer (first phase only)
     uint32_t part_cap;       // records per part
     const uint32_t* part_counts;   // row r, part j: part_counts[(r * 8 + j) * 64]
     uint64_t rows;
@@ -99,16 +99,16 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         // ---- is this row for this launch?  (the decision is the same in every CTA) ----
         const RowCtl ctl = p.ctl[row];
         uint32_t n;
-        uint32_t nparts = 1, pcount[8] = {0, 0, 0, 0, 0, 0, 0, 0};      // the records are pcount[j] at G + j * part_cap
+        uint32_t nparts = 1, pcount[FILTER_PARTS] = {};      // the records are pcount[j] at G + j * part_cap
         if (p.phase == 0) {
             uint32_t R = ctl.count;
             bool part_full = false;
             if (p.parts > 1) {                   // partitioned append: the row's count is the sum of its parts'
-                nparts = 8;
+                nparts = FILTER_PARTS;
                 uint64_t sum = 0;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const uint32_t c = p.part_counts[(row * 8 + j) * 64];
+                for (int j = 0; j < (int)FILTER_PARTS; ++j) {
+                    const uint32_t c = p.part_counts[(row * FILTER_PARTS + j) * FILTER_PART_STRIDE];
                     part_full |= c > p.part_cap;
                     pcount[j] = c < p.part_cap ? c : p.part_cap;
                     sum += c;
@@ -139,17 +139,17 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         // every record of the row once, spread over the grid's threads
         // (The parts are walked as one run of sum(pcount) positions: part by part, a part of 20 K records would
         // keep one thread in seven of the grid busy and cost a memory round trip of its own, eight per pass.)
-        uint32_t pend[8];                                                // pend[j] = records in parts 0..j
+        uint32_t pend[FILTER_PARTS];                                                // pend[j] = records in parts 0..j
         {
             uint32_t acc = 0;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) { acc += pcount[j]; pend[j] = acc; }
+            for (int j = 0; j < (int)FILTER_PARTS; ++j) { acc += pcount[j]; pend[j] = acc; }
         }
         auto for_each_record = [&](auto&& f) {
-            for (uint64_t i = gid; i < pend[7]; i += gthreads) {
+            for (uint64_t i = gid; i < pend[FILTER_PARTS - 1]; i += gthreads) {
                 uint32_t j = 0, before = 0;
 #pragma unroll
-                for (int q = 0; q < 7; ++q)
+                for (int q = 0; q < (int)FILTER_PARTS - 1; ++q)
                     if (i >= pend[q]) { j = q + 1; before = pend[q]; }
                 f((unsigned long long)__ldcg(G + (uint64_t)j * p.part_cap + (i - before)));
             }

@@ -78,7 +78,7 @@ template <typename T> struct SelectParams {
     uint32_t capacity;
     uint32_t* sample_idx;  // may be null; rows x S
     const uint32_t* keys_in;   // null, or rows x S keys of the sample gathered by gather_kernel before this one
-    uint32_t* part_counts;     // null, or the counters of the partitioned append (8 per row, 64 words apart) to reset with the row's
+    uint32_t* part_counts;     // null, or the counters of the partitioned append (FILTER_PARTS per row, FILTER_PART_STRIDE words apart) to reset with the row's
     int by_record;             // 1 = the threshold is the t-th sampled record (value descending, index ascending), 0 = its value
 };
 
@@ -303,7 +303,7 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
             RowCtl* c = p.ctl + row;
             c->count = 0; c->collect = 0; c->status = 0; c->n_final = 0; c->capacity = p.capacity;
             if (p.part_counts)
-                for (int j = 0; j < 8; ++j) p.part_counts[(row * 8 + j) * 64] = 0;
+                for (int j = 0; j < (int)FILTER_PARTS; ++j) p.part_counts[(row * FILTER_PARTS + j) * FILTER_PART_STRIDE] = 0;
         }
         if (p.header && row == 0) {
             p.header->bar_count = 0; p.header->error = 0; p.header->done = 0; p.header->n_failed = 0; p.header->tile_counter = 0;
