@@ -378,7 +378,7 @@ def main():
 
     cpu_baseline = None
     if not args.no_cpu_baseline:
-        cpu_sample = 1 << 25
+        cpu_sample = 1 << 26          # about ten seconds of the oracle on one core
         v, dt_s, sample = time_oracle(cfg, cpu_sample, 1, 0, x=host_inputs[0])
         cpu_baseline = {"value": v, "unit": "elements/s", "cores": 1, "kind": "oracle", "sample": sample,
                         "seconds": dt_s}
