@@ -28,6 +28,15 @@ namespace {
 constexpr int FILTER_THREADS = PROFK_FILTER_THREADS;
 constexpr int FILTER_UNROLL = PROFK_FILTER_UNROLL;
 constexpr uint32_t SORT_CAP_MAX = 16384;         // largest k the single-CTA refine orders in shared memory
+// Selections the whole grid refines (refine_large_kernel) instead of one CTA per row: beyond the single-CTA limit, and
+// from 8193 on when there are at most LARGE_FEW_ROWS rows -- one CTA takes 100-280 us over 12000-16384 records of a
+// long row (bf16, whose equal keys send the selection through the index digits, worst), the grid 80-100; with many
+// rows the CTAs work side by side and win.
+constexpr int64_t LARGE_FEW_ROWS = 4;
+constexpr int64_t LARGE_FEW_K = 8192;
+inline bool large_selection(int64_t rows, int64_t k) {
+    return k > (int64_t)SORT_CAP_MAX || (rows <= LARGE_FEW_ROWS && k > LARGE_FEW_K);
+}
 constexpr unsigned FB_MAX_CTAS = 256;             // most CTAs of the grid-wide exact selection (its per-CTA scratch is sized for them)
 // Samples above this size are gathered by a kernel over all SMs (65536: 2^26, k = 16, S = 40529 took 49.7 us, not 47.0).
 constexpr int64_t GATHER_MIN_SAMPLE = 32768;
@@ -69,8 +78,8 @@ struct WsLayout {
 
 // Records reserved per row: the capacity itself, or -- when k is too large for the single-CTA
 // refine -- twice the power of two the cluster sort pads the row to (records, then scratch).
-uint64_t row_stride_for(int64_t capacity, int64_t k) {
-    if (k <= (int64_t)SORT_CAP_MAX) return (uint64_t)capacity;
+uint64_t row_stride_for(int64_t rows, int64_t capacity, int64_t k) {
+    if (!large_selection(rows, k)) return (uint64_t)capacity;
     uint64_t p = BT_TILE;
     while (p < (uint64_t)capacity) p <<= 1;
     return 2 * p;
@@ -83,22 +92,23 @@ WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k) {
     l.off_ctl = align_up(l.off_ghist + (size_t)FB_PASSES * FB_BINS * sizeof(uint32_t), 256);
     l.off_tau = align_up(l.off_ctl + (size_t)rows * sizeof(RowCtl), 256);
     l.off_bins = align_up(l.off_tau + (size_t)rows * sizeof(uint4), 256);
-    const size_t bins_bytes = k > (int64_t)SORT_CAP_MAX ? (size_t)rows * (LG_BINS + 8) * sizeof(uint32_t) : 0;
+    const bool large = large_selection(rows, k);
+    const size_t bins_bytes = large ? (size_t)rows * (LG_BINS + 8) * sizeof(uint32_t) : 0;
     // scratch of the in-refine exact selection (few rows, k within the single-CTA refine): up to
     // XS_MAX_SEGMENTS segments in all, each with a counter and k + XS_EDGE records
-    const bool xs = rows <= XS_MAX_ROWS && k <= (int64_t)SORT_CAP_MAX;
+    const bool xs = rows <= XS_MAX_ROWS && !large;
     l.off_xs_counters = align_up(l.off_bins + bins_bytes, 256);
     l.off_xs_records = align_up(l.off_xs_counters + (xs ? XS_MAX_SEGMENTS * sizeof(uint32_t) : 0), 256);
     // keys of the sample when a kernel of its own gathers them (few rows only)
     l.off_keys = align_up(l.off_xs_records + (xs ? (size_t)XS_MAX_SEGMENTS * (size_t)(k + XS_EDGE) * sizeof(uint64_t) : 0), 256);
     // scratch of the grid-wide exact selection when it deals failed rows out one per CTA (many rows only)
-    const bool fbp = rows > XS_MAX_ROWS && k <= (int64_t)SORT_CAP_MAX;
+    const bool fbp = rows > XS_MAX_ROWS && !large;
     l.off_fb_counters = align_up(l.off_keys + (rows <= GATHER_MAX_ROWS ? (size_t)rows * (size_t)M_MAX * sizeof(uint32_t) : 0), 256);
     l.off_fb_records = align_up(l.off_fb_counters + (fbp ? FB_MAX_CTAS * sizeof(uint32_t) : 0), 256);
     // counters of the partitioned append (large selections only), each in a 256-byte line of its own
     l.off_parts = align_up(l.off_fb_records + (fbp ? (size_t)FB_MAX_CTAS * (size_t)(k + XS_EDGE) * sizeof(uint64_t) : 0), 256);
-    l.off_buf = align_up(l.off_parts + (k > (int64_t)SORT_CAP_MAX ? (size_t)rows * FILTER_PARTS * FILTER_PART_STRIDE * sizeof(uint32_t) : 0), 256);
-    l.total = align_up(l.off_buf + (size_t)rows * (size_t)row_stride_for(capacity, k) * sizeof(uint64_t), 256);
+    l.off_buf = align_up(l.off_parts + (large ? (size_t)rows * FILTER_PARTS * FILTER_PART_STRIDE * sizeof(uint32_t) : 0), 256);
+    l.total = align_up(l.off_buf + (size_t)rows * (size_t)row_stride_for(rows, capacity, k) * sizeof(uint64_t), 256);
     return l;
 }
 
@@ -438,8 +448,8 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     }
     const WsLayout lay = ws_layout(rows, capacity, k);
     if (!ws.ptr || ws.bytes < lay.total) return PROFK_EWORKSPACE;
-    const uint64_t row_stride = row_stride_for(capacity, k);
-    const bool large = k > (int64_t)SORT_CAP_MAX;
+    const uint64_t row_stride = row_stride_for(rows, capacity, k);
+    const bool large = large_selection(rows, k);
     unsigned char* base = static_cast<unsigned char*>(ws.ptr);
     WsHeader* header = reinterpret_cast<WsHeader*>(base + lay.off_header);
     uint32_t* ghist = reinterpret_cast<uint32_t*>(base + lay.off_ghist);
