@@ -30,6 +30,10 @@ constexpr int SEL_SMALL_THREADS = 256;  // CTA size of the variant for batches o
 constexpr int SEL_BINS = 2048;        // 11-bit digits
 constexpr int SEL_GROUPS = 128;       // groups of 8 lanes whose maxima bound the answer from below
 constexpr uint32_t SEL_CAND_CAP = 4096;
+#ifndef PROFK_SEL_WIDE_MIN
+#define PROFK_SEL_WIDE_MIN 16
+#endif
+constexpr uint32_t SEL_WIDE_MIN = PROFK_SEL_WIDE_MIN;   // smallest rank for which a cluster exchanges its CTAs' bounds
 constexpr uint32_t SEL_SPREAD_MIN = 128;    // more candidates than this are ranked by all CTAs of the cluster
 
 // Per-row control block in the workspace.
@@ -318,7 +322,9 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
     // Deeper ranks, up to GROUPS per CTA of the cluster: every CTA takes the ceil(t / csize)-th largest of its group
     // maxima -- it has that many keys at or above it -- and the smallest of these bounds over the cluster has
     // csize * ceil(t / csize) >= t keys at or above it: one more exchange through the first CTA's shared memory.
-    const bool bounded = p.t <= (uint32_t)GROUPS;
+    // (A cluster uses the cluster-wide bound from rank SEL_WIDE_MIN on: with a bound of its own every CTA sends two to
+    // three times t keys, and towards t = 128 sixteen CTAs overflow the room for candidates and fall into the radix select.)
+    const bool bounded = p.t <= (uint32_t)GROUPS && (csize == 1 || p.t < SEL_WIDE_MIN);
     const uint32_t cta_rank = bounded ? p.t : (p.t + csize - 1) / csize;
     const bool wide = GENERAL && !bounded && csize > 1 && cta_rank <= (uint32_t)GROUPS;
     if (bounded || wide || !GENERAL) {
