@@ -329,6 +329,21 @@ def test_sample_indices_and_threshold_match_the_oracle(dtype):
     assert bits(workloads.as_numpy(tau))[0] == bits(np.asarray([want]))[0]
 
 
+@pytest.mark.parametrize("rows", [12, 20, 40, 80])
+def test_threshold_of_mid_ranks_in_clusters_of_every_size(rows):
+    # 8-, 4-, 2- and 1-CTA clusters per row; ranks on both sides of the switch to the cluster-wide bound, and beyond 128
+    n = 300_007
+    x = workloads.normal(rows, n, seed=36)
+    xn = workloads.as_numpy(x)
+    for m, r in ((8192, 15), (8192, 16), (8192, 100), (20000, 128), (20000, 300)):
+        tau = profk.sample_threshold(x.cuda(), m, r, seed=11)
+        torch.cuda.synchronize()
+        got = bits(workloads.as_numpy(tau))
+        for row in (0, rows // 2, rows - 1):
+            want = o_stages.threshold(xn[row], o_philox.sample_indices(n, m, 11, row), r)
+            assert got[row] == bits(np.asarray([want]))[0], (m, r, row)
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_filter_keeps_exactly_the_survivor_set(dtype):
     n = 777_777
