@@ -23,6 +23,8 @@ stages    the four stages (sample, threshold, filter, refine/fallback) run
           literally on a NumPy array.                     (Section 3)
 mc        Monte Carlo estimates of the two failure events.
 
-Parity pins: see each module's header.  `plan.plan_guarded` in relaxed-recall
-mode (recall < 1) is **parity unpinned**: the paper gives no formula for it.
+Parity pins: see each module's header.  For `plan.plan_guarded` in relaxed-recall
+mode (recall < 1) the paper prints no formula; that mode is pinned by Lemma 1's
+exact tail for the accepted count, minimality of the rank and a Monte Carlo of
+the two failure events (tests/test_oracle_plan.py, tests/test_oracle_mc.py).
 """

@@ -23,12 +23,15 @@ eps/2 + eps/2) but replaces two things that do not meet that contract:
     of Eq. (M) and the smallest M whose overflow bound is at most eps/2; both
     bounds are the binomial bounds of `rank_law` for the stratified sampler.
 
-Readings of points the paper leaves open (all listed again in the design notes):
+Readings of points the paper leaves open:
 `log k` in Eq. (cost_model) / Eq. (optimal_S) is log2 (Algorithm 1 says so); the
 rounding of S* is half away from zero; S is also capped at N; relaxed recall
 rho < 1 means "accept k_rho = ceil(rho k) survivors", i.e. the recall bound is
-taken for k_rho instead of k -- the paper gives no formula for that mode, so
-that part is PARITY UNPINNED; when the buffer would hold half the input or the
+taken for k_rho instead of k while the capacity still follows k (the buffer has
+to hold the k requested outputs) -- the paper gives no formula for that mode,
+so it is pinned by what the mathematics fixes: Lemma 1's exact tail
+Pr(R < k_rho) <= eps/2, minimality of the rank, and a Monte Carlo of both
+failure events with k_rho as the accepted count; when the buffer would hold half the input or the
 sample would be half the input the filter is pointless and the plan says
 mode = 1 (direct exact selection).
 

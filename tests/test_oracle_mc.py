@@ -49,6 +49,25 @@ def test_failure_rates_at_the_benchmark_shapes(N, k, eps):
     assert ga + gb > eps
 
 
+@pytest.mark.parametrize("N,k,eps,recall", [(1 << 26, 4096, 1e-2, 0.5), (1 << 26, 4096, 1e-2, 0.9), (1 << 26, 4096, 1e-2, 0.95)])
+def test_relaxed_plan_meets_the_budget_for_the_accepted_count_and_no_lower_rank_does(N, k, eps, recall):
+    """Relaxed recall by simulation: the failure events are R < k_rho and R > M.  The plan keeps their total
+    within eps, and its rank is minimal -- at one rank less the simulated recall failure alone exceeds eps/2."""
+    rng = np.random.default_rng(5)
+    trials = 400_000
+    p = plan.plan_guarded(N, k, eps, recall=recall)
+    assert p.k_accept == int(np.ceil(recall * k)) and p.r > 1
+    fa, fb = mc.failure_rate_exchangeable(N, p.m, p.r, p.k_accept, p.capacity, trials, rng)
+    sigma = np.sqrt(eps / trials)
+    assert fa + fb <= eps + 4 * sigma
+    assert fa == pytest.approx(rank_law.p_recall_fail_srs(N, p.m, p.r, p.k_accept), abs=4 * sigma)
+    ga, _ = mc.failure_rate_exchangeable(N, p.m, p.r - 1, p.k_accept, p.capacity, trials, rng)
+    assert ga > eps / 2 + 4 * sigma
+    # against the full k the same rank would be over budget: the plan really is the one for k_rho
+    ha, _ = mc.failure_rate_exchangeable(N, p.m, p.r, k, p.capacity, trials, rng)
+    assert ha > eps / 2 + 4 * sigma if recall < 0.95 else ha > fa
+
+
 def test_record_threshold_keeps_the_budget_on_rows_full_of_ties():
     """The four stages run on rows whose values repeat thousands of times: with the threshold taken as a
     (value, index) record the count check fails no more often than the budget allows, as on distinct values;

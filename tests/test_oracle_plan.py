@@ -125,6 +125,44 @@ def test_guarded_plan_contract(N, k, eps):
     assert t_gauss - 1 <= p.r <= t_gauss + 6
 
 
+RELAXED_SHAPES = [(2 ** 26, 4096, 1e-2, 0.5), (2 ** 26, 4096, 1e-2, 0.9), (2 ** 26, 4096, 1e-2, 0.95), (2 ** 26, 256, 1e-4, 0.5),
+                  (2 ** 20, 64, 1e-3, 0.9), (2 ** 18, 64, 1e-2, 0.9), (2 ** 29, 131072, 1e-3, 0.95), (1_000_003, 77, 1e-3, 0.9)]
+
+
+@pytest.mark.parametrize("N,k,eps,recall", RELAXED_SHAPES)
+def test_guarded_plan_contract_in_relaxed_mode(N, k, eps, recall):
+    """Relaxed recall (the abstract's "recovering 95% of the true top-k"): the paper gives no formula, the
+    mathematics does.  With k_rho = ceil(rho k) accepted survivors Theorem 1's budget reads
+    Pr(R < k_rho) <= eps/2 and Pr(R > M) <= eps/2, the rank is the smallest that meets the first, and the
+    buffer still has to hold the k requested outputs, so the capacity follows k, not k_rho."""
+    p = plan.plan_guarded(N, k, eps, recall=recall)
+    exact = plan.plan_guarded(N, k, eps)
+    k_rho = math.ceil(recall * k)
+    assert p.k_accept == k_rho < k and p.m == exact.m
+    # the recall half of the budget, for k_rho: the plan's own bound and Lemma 1's exact tail
+    assert p.p_recall_fail <= eps / 2
+    assert p.p_recall_fail == rank_law.p_recall_fail_bound(N, p.m, p.r, k_rho)
+    assert rank_law.p_recall_fail_srs(N, p.m, p.r, k_rho) <= eps / 2
+    # minimality: one rank less breaks the bound for k_rho (a plan that took the rank for k would sit above it)
+    if p.r > 1:
+        assert rank_law.p_recall_fail_bound(N, p.m, p.r - 1, k_rho) > eps / 2
+    assert p.r <= exact.r
+    # the overflow half of the budget, and a capacity derived from k: never below Eq. (M) for k, and minimal above it
+    assert p.p_overflow <= eps / 2 and rank_law.p_overflow_srs(N, p.m, p.r, p.capacity) <= eps / 2
+    m_paper = math.ceil(plan.eq_M(N, k, p.m, p.z))
+    assert p.capacity >= m_paper >= k
+    if p.capacity > m_paper:
+        assert rank_law.p_overflow_bound(N, p.m, p.r, p.capacity - 1) > eps / 2
+    # a lower rank keeps fewer elements: the capacity does not grow
+    assert p.capacity <= exact.capacity
+
+
+def test_relaxed_rank_differs_from_the_exact_one_where_the_pins_can_see_it():
+    # (shapes on which taking the rank for k instead of k_rho, or the reverse, changes the plan)
+    for N, k, eps, recall in RELAXED_SHAPES[:4]:
+        assert plan.plan_guarded(N, k, eps, recall=recall).r < plan.plan_guarded(N, k, eps).r
+
+
 def test_guarded_capacity_approaches_the_closed_form_in_the_gaussian_regime():
     ratios = []
     for k in (2 ** 12, 2 ** 15, 2 ** 18, 2 ** 21):                                 # alpha S = 8 .. 4096 at S = 2^17
