@@ -30,10 +30,17 @@
  *     -NaN < -inf < ... < -0 < +0 < ... < +inf < +NaN of their bit patterns.
  *   - Limits: 1 <= k <= N <= 2^32 - 2^24 per row, rows >= 1, rows * capacity < 2^40.
  *   - Two calls that use the same workspace must not overlap on the device.
- *   - The kernels of a call are enqueued as programmatic dependents of one
- *     another and of whatever precedes the call on the stream: each waits for
- *     the work before it (griddepcontrol.wait) before it reads the input or
- *     touches the workspace, so ordinary stream order is all a caller relies on.
+ *   - Ordinary stream order is all a caller relies on.  The kernels of a call
+ *     are enqueued as programmatic dependents of one another and of whatever
+ *     precedes the call on the stream.  The call's first kernel computes its
+ *     sample positions early but waits for the work before it
+ *     (griddepcontrol.wait) before it reads the input or touches the workspace,
+ *     and only after that wait does it release the kernels behind it.  The
+ *     filtering scan does read tiles of the input before its own wait -- by then
+ *     the first kernel's wait has returned, so whatever wrote the input has
+ *     finished and its writes are visible, also when that producer itself
+ *     released its dependents early (a GEMM epilogue with programmatic launch,
+ *     or this library's own last kernel when one call's output feeds the next).
  *     A call can be captured into a CUDA graph once its shape has been used
  *     outside a capture (the first use sets kernel attributes).
  */
@@ -52,7 +59,7 @@ typedef enum profk_status {
     PROFK_EINVAL = -1,     /* bad argument (range, null pointer, alignment) */
     PROFK_EWORKSPACE = -2, /* no workspace registered on this device, or it is too small */
     PROFK_ECUDA = -3,      /* a CUDA runtime call or launch reported an error */
-    PROFK_ETIMEOUT = -4,   /* (statistics only) a bounded device-side wait gave up */
+    PROFK_ETIMEOUT = -4,   /* profk_read_stats: a bounded device-side wait gave up during the call (result invalid) */
     PROFK_ETOOLARGE = -5   /* profk_topk_noalloc_f32 only: the shape needs more than the built-in scratch */
 } profk_status_t;
 
@@ -239,9 +246,9 @@ int profk_sample_threshold_bf16(const void* in, int64_t rows, int64_t N, int64_t
 
 /*
  * (This entry point has no counterpart in the paper; it exists for callers that must not
- * allocate.)  Same result as profk_topk_f32, but no workspace has to be registered and no
- * call made here allocates or frees anything, on the host side of CUDA or on the device:
- * the scratch is a 16 MiB array that is part of the library itself.  It is meant for code
+ * allocate.)  Same result as profk_topk_f32, but no workspace has to be registered and the
+ * entry point calls no allocator, neither cudaMalloc / cudaFree nor an allocating library
+ * routine: the scratch is a 16 MiB array that is part of the library itself.  It is meant for code
  * that runs where an allocation is forbidden or would deadlock -- a callback of a memory
  * pool that is itself inside an allocation, a real-time or plug-in context that was handed
  * its buffers up front, a host that has already given all device memory to another
@@ -251,8 +258,13 @@ int profk_sample_threshold_bf16(const void* in, int64_t rows, int64_t N, int64_t
  *     one row of any length up to the library limit with small k, or 512 rows of 2^20
  *     elements with k = 32.  Anything larger returns PROFK_ETOOLARGE and does nothing.
  *   - Every GPU that loads the library holds the 16 MiB until the process exits.
- *   - The first call on each device looks up the array's device address (it keeps the
- *     result); make that first call outside any stream capture.
+ *   - The first call on each device is a set-up call: it looks up the array's device address
+ *     (and keeps it), and like any first use of this library on a device it may make the driver
+ *     load the library's code and the array onto the device, sets kernel attributes and fills a
+ *     small host-side table.  Make that first call before the region in which nothing may be
+ *     allocated, and outside any stream capture; in a process whose device memory is already
+ *     exhausted it can fail with PROFK_ECUDA.  Calls after it allocate nothing, on the host side
+ *     of CUDA or on the device; the plan of the last 16 shapes is kept in a fixed table.
  *   - All calls share the one array, and it keeps whatever the last call left in it.  Each
  *     call re-initialises the parts that must start at zero, so calls issued one after the
  *     other on a stream are fine; two calls that overlap on the GPU (different streams,
@@ -265,12 +277,24 @@ int profk_topk_noalloc_f32(const float* in, int64_t rows, int64_t N, int64_t k, 
 
 /*
  * Copies the statistics of the last call that used the registered workspace to
- * the host and waits for `stream`.  out: [host] rows entries.
+ * the host and waits for `stream`.  out: [host] rows entries.  Every wait inside
+ * the kernels is bounded (the grid barriers of the exact-selection and large-k
+ * kernels); when one gave up, the kernels returned early, the call's outputs are
+ * invalid, every status word has bit 31 set and the return value is
+ * PROFK_ETIMEOUT (the entries are filled in all the same).  The next call on the
+ * workspace clears the flag.
  */
 int profk_read_stats(void* stream, int64_t rows, profk_row_stats_t* out);
 
 /* Number of kernels the last profk_topk* call on this thread enqueued. */
 int profk_last_launch_count(void);
+
+/*
+ * Diagnostic: how many polls a CTA of the filtering scan spends on the tiles it copied into shared memory while
+ * the threshold was being computed before it reads them with plain loads instead (negative = the default, 2^22;
+ * 0 = never use the copies).  Results do not depend on it.  Process-wide.
+ */
+int profk_debug_set_prefetch_wait_polls(int64_t polls);
 
 /* Static text for a status code. */
 const char* profk_strerror(int code);

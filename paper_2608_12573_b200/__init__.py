@@ -20,6 +20,7 @@ EXPORTS = [
     "profk_topk_f32", "profk_topk_bf16", "profk_topk_planned_f32", "profk_topk_planned_bf16",
     "profk_filter_f32", "profk_filter_bf16", "profk_sample_threshold_f32", "profk_sample_threshold_bf16",
     "profk_read_stats", "profk_last_launch_count", "profk_strerror", "profk_topk_noalloc_f32",
+    "profk_debug_set_prefetch_wait_polls",
 ]
 
 ROW_OK, ROW_RECALL, ROW_OVERFLOW, ROW_DIRECT = 0, 1, 2, 3
@@ -153,14 +154,13 @@ def ensure_workspace(rows: int, capacity: int, k: int, device) -> None:
     if cur is not None and cur.numel() >= need:
         _workspace_ok.add((idx, rows, capacity, k))
         return
-    if True:
-        with torch.cuda.device(idx):
-            buf = torch.empty(max(need, 1 << 20), dtype=torch.uint8, device=dev)
-            _check(lib().profk_set_workspace(ctypes.c_void_p(buf.data_ptr()), ctypes.c_size_t(buf.numel())),
-                   "profk_set_workspace")
-        _workspaces[idx] = buf
-        _workspace_ok.clear()
-        _workspace_ok.add((idx, rows, capacity, k))
+    with torch.cuda.device(idx):
+        buf = torch.empty(max(need, 1 << 20), dtype=torch.uint8, device=dev)
+        _check(lib().profk_set_workspace(ctypes.c_void_p(buf.data_ptr()), ctypes.c_size_t(buf.numel())),
+               "profk_set_workspace")
+    _workspaces[idx] = buf
+    _workspace_ok.clear()
+    _workspace_ok.add((idx, rows, capacity, k))
 
 
 def _stream_ptr():

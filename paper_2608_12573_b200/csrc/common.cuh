@@ -97,16 +97,6 @@ __device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint3
     return Philox4{c0, c1, c2, c3};
 }
 
-// Index of stratum j's sample: one uniform draw from [floor(jN/S), floor((j+1)N/S)).
-__device__ __forceinline__ uint32_t sample_index(uint64_t N, uint64_t S, uint64_t j, uint64_t row, uint64_t seed) {
-    const uint64_t lo = j * N / S;
-    const uint64_t hi = (j + 1) * N / S;
-    const Philox4 p = philox4x32_10((uint32_t)j, (uint32_t)row, (uint32_t)(row >> 32), 0u,
-                                    (uint32_t)seed, (uint32_t)(seed >> 32));
-    const uint64_t u = ((uint64_t)p.y << 32) | (uint64_t)p.x;
-    return (uint32_t)(lo + __umul64hi(u, hi - lo));
-}
-
 // ---------------------------------------------------------------------------------------
 // Streaming loads: the input is read exactly once, so keep it out of L1.
 
@@ -124,22 +114,6 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
 }
 
 __device__ __forceinline__ unsigned lane_id() { return threadIdx.x & 31u; }
-
-// Optional phase stamps for tuning (SM cycle counter of CTA 0); compiled out by default.
-#ifdef PROFK_TRACE
-__device__ long long g_profk_trace[4][32];
-#define PROFK_STAMP(kernel, slot)                                                   \
-    do {                                                                            \
-        if (threadIdx.x == 0 && blockIdx.x == 0) {                                  \
-            g_profk_trace[kernel][slot] = clock64();                                \
-            unsigned long long gt;                                                  \
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));                  \
-            g_profk_trace[kernel + 2][slot] = (long long)gt;                        \
-        }                                                                           \
-    } while (0)
-#else
-#define PROFK_STAMP(kernel, slot) do { } while (0)
-#endif
 
 // Programmatic dependent launch: wait for the preceding kernel's memory to be visible /
 // allow the following kernel to start its prologue.

@@ -61,6 +61,10 @@ template <typename T> struct FilterParams {
     // Tiles (0 or FILTER_PREFETCH) a CTA copies into its shared memory while it waits for the threshold kernel, beyond
     // the one it holds in registers: the input does not depend on the threshold, and HBM is idle meanwhile.
     uint32_t prefetch_tiles;
+    // Polls of the mbarrier that counts those copies before the CTA gives up on them and reads the tiles with plain
+    // loads (PREFETCH_SPIN_LIMIT; a test sets 0 to take that branch).  The wait before the CTA leaves always has the
+    // full limit: shared memory must not be handed on while a copy into it is in flight.
+    uint32_t prefetch_spin_limit;
 };
 
 constexpr uint32_t FILTER_PREFETCH = 2;
@@ -455,16 +459,13 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
             __syncthreads();            // the barrier is initialised before anyone may wait on it
         }
     }
-
-    PROFK_STAMP(0, 10);
     if (p.use_pdl) pdl_wait();
     pdl_launch_dependents();            // the refine kernel may be staged behind this one
-    PROFK_STAMP(0, 11);
     // The copies were issued microseconds ago; should they not have landed within the limit, the tiles are read with
     // plain loads instead and the copies are waited for once more before the CTA leaves.
-    auto prefetch_landed = [&]() {
+    auto prefetch_landed = [&](uint32_t limit) {
         const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&pf_bar);
-        for (uint32_t spin = 0; spin < PREFETCH_SPIN_LIMIT; ++spin) {
+        for (uint32_t spin = 0; spin < limit; ++spin) {
             uint32_t done;
             asm volatile("{\n\t.reg .pred q;\n\tmbarrier.try_wait.parity.shared::cta.b64 q, [%1], 0;\n\tselp.u32 %0, 1, 0, q;\n\t}"
                          : "=r"(done) : "r"(bar) : "memory");
@@ -474,7 +475,7 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
     };
     bool pf_pending = false;
     if (pf_ok) {
-        if (prefetch_landed()) pf_left = p.prefetch_tiles; else pf_pending = true;
+        if (prefetch_landed(p.prefetch_spin_limit)) pf_left = p.prefetch_tiles; else pf_pending = true;
     }
 
     uint32_t skip_row = 0xFFFFFFFFu;    // row whose buffer this warp has seen overflow: nothing more to append
@@ -546,16 +547,7 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
         if (row != tau_row) { tau_row = row; load_threshold(); }
     }
     if (STAGED && st->fill) flush_stage(p, st);
-    if (pf_pending) prefetch_landed();
-    PROFK_STAMP(0, 12);
-#ifdef PROFK_TRACE
-    if (threadIdx.x == 0) {
-        unsigned long long gt;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
-        atomicMax((unsigned long long*)&g_profk_trace[2][13], gt);      // latest CTA end
-        atomicMin((unsigned long long*)&g_profk_trace[2][14], gt);      // earliest CTA end
-    }
-#endif
+    if (pf_pending) prefetch_landed(PREFETCH_SPIN_LIMIT);
 }
 
 }  // namespace profk

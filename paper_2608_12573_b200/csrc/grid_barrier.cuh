@@ -10,9 +10,9 @@ constexpr uint32_t SPIN_LIMIT = 1u << 24;   // polls (each ~100 ns apart) before
 // Sense-free generation barrier over `members` co-resident CTAs that share the words *count (zero before
 // the first use, and again after every completed barrier) and *generation (any value).  `gen` is the caller's
 // copy of the generation, read before its first arrival.  Returns false when the wait gave up (or an earlier
-// one did, anywhere in the grid); the caller then leaves the kernel.
+// one did, anywhere in the grid); the caller then leaves the kernel.  `limit` is the number of polls a wait may take.
 __device__ __forceinline__ bool cta_group_barrier(uint32_t* count, uint32_t* generation, uint32_t* error, uint32_t members,
-                                                  uint32_t& gen) {
+                                                  uint32_t& gen, uint32_t limit = SPIN_LIMIT) {
     __shared__ uint32_t s_ok;
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -27,7 +27,7 @@ __device__ __forceinline__ bool cta_group_barrier(uint32_t* count, uint32_t* gen
             uint32_t polls = 0;
             while (*((volatile uint32_t*)generation) == gen) {
                 __nanosleep(64);
-                if (++polls > SPIN_LIMIT) { atomicExch(error, 1u); ok = 0; break; }
+                if (++polls > limit) { atomicExch(error, 1u); ok = 0; break; }
             }
         }
         __threadfence();

@@ -52,6 +52,7 @@ constexpr int64_t M_MAX = 262144;                // largest sample the cluster s
 thread_local int g_launches = 0;
 thread_local void* g_ws_override_ptr = nullptr;   // set by the allocation-free entry point for the duration of its call
 thread_local size_t g_ws_override_bytes = 0;
+std::atomic<uint32_t> g_prefetch_spin_limit{PREFETCH_SPIN_LIMIT};   // see profk_debug_set_prefetch_wait_polls
 std::atomic<int> g_coop_pdl{-1};                 // -1 untried, 1 accepted, 0 refused by the runtime
 
 struct DeviceInfo {
@@ -287,6 +288,7 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     // (Not the staged build: its two CTAs per SM spill already, and the copies cost the 2^29 bf16 row 3 us.)
     const bool prefetch = pdl && !staged && rows == 1 && fp.dyn_start >= (FILTER_PREFETCH + 1) * cfg.gridDim.x;
     fp.prefetch_tiles = prefetch ? FILTER_PREFETCH : 0u;
+    fp.prefetch_spin_limit = g_prefetch_spin_limit.load();
     cfg.dynamicSmemBytes = prefetch ? FILTER_PREFETCH * FILTER_THREADS * FILTER_UNROLL * 16u : 0;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -669,26 +671,43 @@ int profk_topk_noalloc_f32(const float* in, int64_t rows, int64_t N, int64_t k, 
     int dev = 0;
     CUDA_TRY(cudaGetDevice(&dev));
     // In host code `g_noalloc_scratch` is only a handle of the symbol, not a device address: the
-    // address on the current device comes from the runtime, once per device, and is cached.
-    static std::mutex ptr_mutex;
-    static std::map<int, void*> ptr_by_device;
+    // address on the current device comes from the runtime, once per device, and is kept.  Both
+    // tables below have a fixed size, so that nothing here allocates on the host either.
+    constexpr int MAX_DEVICES = 64;
+    constexpr int PLAN_SLOTS = 16;
+    struct PlanSlot { int64_t rows_class, N, k; double eps, recall; profk_plan_t plan; bool used; };
+    static std::mutex table_mutex;
+    static void* ptr_by_device[MAX_DEVICES] = {};
+    static PlanSlot plans[PLAN_SLOTS] = {};
+    static int next_slot = 0;
+    if (dev < 0 || dev >= MAX_DEVICES) return PROFK_EINVAL;
+    if (rows < 1) return PROFK_EINVAL;
     void* scratch = nullptr;
+    profk_plan_t plan;
     {
-        std::lock_guard<std::mutex> lock(ptr_mutex);
-        auto it = ptr_by_device.find(dev);
-        if (it == ptr_by_device.end()) {
+        std::lock_guard<std::mutex> lock(table_mutex);
+        if (!ptr_by_device[dev]) {
             void* p = nullptr;
             CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
             if (!p) return PROFK_ECUDA;
-            it = ptr_by_device.emplace(dev, p).first;
+            ptr_by_device[dev] = p;
         }
-        scratch = it->second;
+        scratch = ptr_by_device[dev];
+        // the plan costs some host time (tail sums, bisections): kept for the last few shapes
+        const int64_t rows_class = rows <= GATHER_MAX_ROWS ? 1 : GATHER_MAX_ROWS + 1;     // the two classes the tuning knows
+        const PlanSlot* hit = nullptr;
+        for (const PlanSlot& ps : plans)
+            if (ps.used && ps.rows_class == rows_class && ps.N == N && ps.k == k && ps.eps == eps && ps.recall == recall) hit = &ps;
+        if (hit) {
+            plan = hit->plan;
+        } else {
+            const int prc = profk_plan_batch(rows_class, N, k, eps, recall, &plan);
+            if (prc != PROFK_OK) return prc;
+            plans[next_slot] = PlanSlot{rows_class, N, k, eps, recall, plan, true};
+            next_slot = (next_slot + 1) % PLAN_SLOTS;
+        }
     }
-    profk_plan_t plan;
-    if (rows < 1) return PROFK_EINVAL;
-    const int prc = profk_plan_batch(rows, N, k, eps, recall, &plan);
-    if (prc != PROFK_OK) return prc;
-    if ( rows * plan.capacity >= (1LL << 40)) return PROFK_EINVAL;
+    if (rows * plan.capacity >= (1LL << 40)) return PROFK_EINVAL;
     if (ws_layout(rows, plan.capacity, k).total > NOALLOC_SCRATCH_BYTES) return PROFK_ETOOLARGE;
     g_ws_override_ptr = scratch;
     g_ws_override_bytes = NOALLOC_SCRATCH_BYTES;
@@ -722,18 +741,15 @@ int profk_read_stats(void* stream, int64_t rows, profk_row_stats_t* out) {
         out[r].capacity = host[r].capacity;
         out[r].status = host[r].status | (hdr.error ? 0x80000000u : 0u);
     }
-    return PROFK_OK;
+    return hdr.error ? PROFK_ETIMEOUT : PROFK_OK;
 }
 
 int profk_last_launch_count(void) { return g_launches; }
 
-#ifdef PROFK_TRACE
-int profk_debug_read_trace(long long* out /* [host] 4 x 32 */) {
-    CUDA_TRY(cudaDeviceSynchronize());
-    CUDA_TRY(cudaMemcpyFromSymbol(out, g_profk_trace, sizeof(long long) * 4 * 32));
+int profk_debug_set_prefetch_wait_polls(int64_t polls) {
+    g_prefetch_spin_limit.store(polls < 0 ? PREFETCH_SPIN_LIMIT : (uint32_t)std::min<int64_t>(polls, PREFETCH_SPIN_LIMIT));
     return PROFK_OK;
 }
-#endif
 
 const char* profk_strerror(int code) {
     switch (code) {

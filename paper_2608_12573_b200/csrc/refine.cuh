@@ -140,7 +140,6 @@ __global__ void __maxnreg__(MAXREG) refine_kernel(const __grid_constant__ Refine
     }
     pdl_launch_dependents();
     if (p.use_pdl) pdl_wait();
-    PROFK_STAMP(1, 0);
 
     // The first batch of records (8 per thread, kept in registers) is requested at once, together with
     // the row's control block: which of them are real is known when the survivor count arrives.
@@ -205,7 +204,6 @@ __global__ void __maxnreg__(MAXREG) refine_kernel(const __grid_constant__ Refine
         const uint32_t level = f > (127u << 23) ? (f >> 16) - (127u << 7) : 0u;     // 0 .. 4095
         return (uint32_t)(RF_BINS - 1) - level;
     };
-    PROFK_STAMP(1, 1);
 
     for (uint32_t b = 0; b < nbatch; ++b) {
         if (b > 0) load_batch(b);
@@ -266,7 +264,6 @@ __global__ void __maxnreg__(MAXREG) refine_kernel(const __grid_constant__ Refine
         }
     }
     __syncthreads();
-    PROFK_STAMP(1, 2);
 
     if (!sh.crowded) {
         // ---- group the records of the boundary bin and of all better bins by bin ----
@@ -283,7 +280,6 @@ __global__ void __maxnreg__(MAXREG) refine_kernel(const __grid_constant__ Refine
             }
         }
         __syncthreads();
-        PROFK_STAMP(1, 3);
         // ---- every grouped record ranks itself inside its bin: that is its place in the output ----
         for (uint32_t s = tid; s < n_grouped; s += nthr) {
             const uint64_t mine = sortbuf[s];
@@ -293,7 +289,6 @@ __global__ void __maxnreg__(MAXREG) refine_kernel(const __grid_constant__ Refine
             for (uint32_t j = first; j < last; ++j) pos += sortbuf[j] < mine;
             if (pos < kk) write_output(p.out_vals, p.out_idx, p.k, row, pos, mine);
         }
-        PROFK_STAMP(1, 4);
         return;
     }
 

@@ -167,7 +167,6 @@ template <typename T> struct GatherParams {
 
 template <typename T>
 __global__ void __launch_bounds__(GATHER_THREADS) gather_kernel(const GatherParams<T> p) {
-    pdl_launch_dependents();
     const uint64_t pairs = ((uint64_t)p.S + 1) / 2;
     const uint64_t g = (uint64_t)blockIdx.x * GATHER_THREADS + threadIdx.x;
     const bool active = g < p.rows * pairs;
@@ -190,6 +189,9 @@ __global__ void __launch_bounds__(GATHER_THREADS) gather_kernel(const GatherPara
         }
     }
     pdl_wait();                  // the positions needed nothing; the values need the work queued before this kernel
+    // Dependents are released only now, after the wait: the kernels behind this one read the input before their
+    // own wait (which covers this kernel alone), so they must not start before whatever wrote the input has finished.
+    pdl_launch_dependents();
     if (active) {
         const T v0 = rowp[idx0];
         const T v1 = second ? rowp[idx1] : v0;
@@ -221,12 +223,6 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
     const unsigned crank = cluster.block_rank();
     const uint64_t row = blockIdx.x / csize;
     const unsigned tid = threadIdx.x, lane = lane_id();
-
-    pdl_launch_dependents();   // the filter kernel may start its prologue now
-    PROFK_STAMP(0, 0);
-#ifdef PROFK_TRACE
-    if (threadIdx.x == 0 && blockIdx.x == 0) { g_profk_trace[2][13] = 0; g_profk_trace[2][14] = 0x7FFFFFFFFFFFFFFFll; }
-#endif
 
     if (tid == 0) { s_ncand = 0; s_lower = 0; s_lmin = 0xFFFFFFFFu; }
     __syncthreads();
@@ -302,6 +298,11 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
         }
     }
     pdl_wait();                  // CTAs without a share of the sample have not waited yet
+    // The filter kernel may start its prologue now -- and not earlier.  It reads tiles of the input before its own
+    // wait, which covers this kernel only; this kernel's wait has just returned, so whatever produced the input has
+    // finished, even a producer that released its own dependents early.  The filter's prologue still overlaps the
+    // whole selection below.
+    pdl_launch_dependents();
     if (crank == 0 && tid == 0) {
         if (p.ctl) {
             RowCtl* c = p.ctl + row;
@@ -314,7 +315,6 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
             for (int g = 0; g < WS_GROUPS; ++g) p.header->group_bar[g][0] = 0;
         }
     }
-    PROFK_STAMP(0, 1);
 
     bool done = false;
 
@@ -354,7 +354,6 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
         }                                   // (not bounded: the bound stays 0 and every key is a candidate)
         __syncthreads();
         uint32_t lower = s_lower;
-        PROFK_STAMP(0, 2);
         // every CTA sends its keys >= lower to the first CTA: one remote atomic per warp that has any
         uint64_t* cand0 = cluster.map_shared_rank(cand, 0);
         uint32_t* ncand0 = cluster.map_shared_rank(&s_ncand, 0);
@@ -377,9 +376,7 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
                 if (take && slot < SEL_CAND_CAP) cand0[slot] = ((uint64_t)k << 32) | (uint64_t)(0xFFFFFFFFu - (j0 + i));
             }
         }
-        PROFK_STAMP(0, 3);
         cluster.sync();                               // all candidates have arrived
-        PROFK_STAMP(0, 4);
         const uint32_t ncand = *ncand0;
         if (ncand <= SEL_CAND_CAP) {
             // Every CTA takes a copy of the candidates and looks at its share of them (candidate c goes to
@@ -391,7 +388,6 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
                 for (uint32_t i = tid; i < ncand; i += THREADS) cand[i] = cand0[i];
             auto seen = cluster.barrier_arrive();     // "I have read the first CTA's memory": it may leave after its peers did
             if (spread) __syncthreads();
-            PROFK_STAMP(0, 7);
             const unsigned part = tid & 7u;
             const uint32_t c_first = spread ? (tid >> 3) * csize + crank : crank == 0 ? (tid >> 3) : ncand;
             const uint32_t c_step = (THREADS / 8) * (spread ? csize : 1u);
@@ -407,7 +403,6 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
                     publish_threshold(p, row, (uint32_t)(mine >> 32), 0xFFFFFFFFu - (uint32_t)mine);
             }
             done = true;
-            PROFK_STAMP(0, 5);
             cluster.barrier_wait(std::move(seen));
         } else {
             auto seen = cluster.barrier_arrive();
@@ -495,7 +490,6 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
         cluster.sync();   // no CTA leaves while a peer may still read its histogram or its count
     }
     }
-    PROFK_STAMP(0, 6);
 }
 
 }  // namespace profk

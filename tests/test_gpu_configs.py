@@ -60,6 +60,37 @@ def test_config2_single_row_2p26():
         assert np.all(i[n_real:] == -1) and np.all(np.isneginf(v[n_real:]))
 
 
+def test_relaxed_recall_statistics_over_a_thousand_rows():
+    """Relaxed mode, measured: 256 rows x 4 seeds = 1024 row-calls with rho = 0.5, eps = 1e-2.  Every output row is a
+    prefix of the oracle's answer followed by padding, at least ceil(rho k) long; the share of rows whose filter kept
+    fewer than ceil(rho k) candidates (they are repaired, and counted here) stays within eps/2 + 4 sigma, and the share
+    of rows that failed either check within eps + 4 sigma: recall >= rho in at least 1 - eps of the rows."""
+    rows, n, k, rho, eps = 256, 1 << 18, 512, 0.5, 1e-2
+    x = workloads.normal(rows, n, seed=21)
+    xn = workloads.as_numpy(x)
+    ov, oi = o_topk.topk(xn, k)
+    pl = o_plan.plan_guarded(n, k, eps, recall=rho, **profk.default_tuning(n, rows=rows))
+    assert pl.k_accept == 256 and pl.mode == 0 and pl.r < o_plan.plan_guarded(n, k, eps, **profk.default_tuning(n, rows=rows)).r
+    xd = x.cuda()
+    short = recall_failed = failed = total = 0
+    for seed in range(4):
+        v, i = run(xd, k, eps=eps, recall=rho, seed=100 + seed)
+        for r, (_, R, cap, status) in enumerate(profk.read_stats(rows)):
+            assert cap == pl.capacity
+            n_real = min(k, R) if status == profk.ROW_OK else k
+            assert n_real >= pl.k_accept, (seed, r)
+            assert np.array_equal(i[r, :n_real], oi[r, :n_real]) and np.array_equal(bits(v[r, :n_real]), bits(ov[r, :n_real])), (seed, r)
+            assert np.all(i[r, n_real:] == -1) and np.all(np.isneginf(v[r, n_real:])), (seed, r)
+            short += n_real < k
+            recall_failed += status == profk.ROW_RECALL
+            failed += status != profk.ROW_OK
+            total += 1
+    assert total == 1024
+    assert recall_failed / total <= eps / 2 + 4 * np.sqrt(eps / 2 / total)
+    assert failed / total <= eps + 4 * np.sqrt(eps / total)
+    assert short > 100                                        # the mode is exercised: about one row in five returns fewer than k
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_config3_batched_512_rows(dtype):
     x = workloads.normal(512, 1 << 20, seed=2, dtype=dtype)

@@ -5,15 +5,21 @@ the first failure has already run every other test.
 they need a top-k -- code inside an allocator callback, a plug-in that was handed all its buffers up
 front, a process whose device memory already belongs to another pool.  Its scratch is a fixed array
 inside the library, so the test checks three things through the C ABI: that it returns exactly what
-the ordinary entry point returns, that it still does so on a second call in a row (the array then
-holds the first call's leftovers), and that it refuses shapes that do not fit instead of overrunning.
+the ordinary entry point returns (and what the CPU oracle's full sort returns), that it still does so
+on a second call in a row (the array then holds the first call's leftovers), and that it refuses
+shapes that do not fit instead of overrunning.  The shapes reach every layout the scratch can take:
+a few rows (the refine kernel's clusters and their exact-selection scratch), a batch of more than 18
+rows (the per-CTA scratch of the grid-wide exact selection), and a selection beyond 8192 (bins,
+partitioned append counters and a doubled row pitch).
 """
 import ctypes
 
+import numpy as np
 import pytest
 import torch
 
 import paper_2608_12573_b200 as profk
+from oracle import topk as o_topk
 from paper_2608_12573_b200 import _build, workloads
 
 pytestmark = pytest.mark.gpu
@@ -32,7 +38,7 @@ def test_noalloc_entry_matches_the_ordinary_one_twice_in_a_row():
     _build.build()
     lib = profk.lib()
     torch.cuda.set_device(0)
-    shapes = [(1, 1 << 22, 100), (6, 300_001, 17)]
+    shapes = [(1, 1 << 22, 100), (6, 300_001, 17), (64, 1 << 18, 32), (1, 1 << 22, 10_000), (2, 1 << 20, 9_000)]
     for rows, n, k in shapes:
         xs = [workloads.normal(rows, n, seed=40 + r).cuda() for r in range(2)]      # two different inputs, two calls in a row
         # reference: the existing entry point, with a registered workspace
@@ -51,9 +57,12 @@ def test_noalloc_entry_matches_the_ordinary_one_twice_in_a_row():
         for r, x in enumerate(xs):
             assert _call(lib.profk_topk_noalloc_f32, x, k, 1e-3, 7 + r, got[r][0], got[r][1]) == 0
         torch.cuda.synchronize()
-        for (wv, wi), (gv, gi) in zip(want, got):
+        for x, (wv, wi), (gv, gi) in zip(xs, want, got):
             assert torch.equal(wi, gi)                                              # integer work: bit-exact
             assert torch.equal(wv.view(torch.int32), gv.view(torch.int32))          # values bit for bit as well
+            ov, oi = o_topk.topk(x.cpu().numpy(), k)                                # and both equal the oracle's full sort
+            assert np.array_equal(gi.cpu().numpy(), oi)
+            assert np.array_equal(gv.cpu().numpy().view(np.uint32), ov.view(np.uint32))
 
 
 def test_noalloc_entry_refuses_what_does_not_fit():
