@@ -286,6 +286,25 @@ def measure_extra_config(profk, torch, name, dev, peak):
            "filter_ms_per_launch": filt["ms_per_launch"] if filt else None,
            "filter_GBps": filt["GBps"] if filt else None,
            "filter_frac_of_measured_peak": (filt["GBps"] / peak) if filt and filt["GBps"] else None}
+    if name.startswith("cfg4"):
+        # The same selection through the BatchTopK consumer entry point (Section 5, "Application"): the kept set
+        # without ordering -- as unordered (value, index) pairs, with the bit mask, and as a dense array.
+        forms = {"pairs": dict(want_pairs=True), "pairs_and_mask": dict(want_pairs=True, want_mask=True),
+                 "dense": dict(want_pairs=False, want_dense=True)}
+        res["batchtopk_ms_per_call"] = {}
+        for form, kw in forms.items():
+            for i in range(3):
+                profk.batchtopk(inputs[i % copies], k, eps=eps, seed=i, **kw)
+            torch.cuda.synchronize()
+            e0.record()
+            for i in range(calls):
+                profk.batchtopk(inputs[i % copies], k, eps=eps, seed=5 + i, **kw)
+            e1.record()
+            torch.cuda.synchronize()
+            res["batchtopk_ms_per_call"][form] = e0.elapsed_time(e1) / calls
+        res["batchtopk_launches_per_call"] = profk.last_launch_count()
+        res["batchtopk_note"] = ("outputs are allocated through torch inside the timed loop (caching allocator); the dense form also "
+                                 "writes N elements of zeros")
     if k > 8192 and rows <= 4:
         res["filter_note"] = ("the stand-alone filter launch appends to one counter per row; inside the call a selection this large "
                               "appends to eight (or stages per warp), so the call's own filter pass is faster than this figure")

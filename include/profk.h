@@ -214,6 +214,38 @@ int profk_topk_planned_bf16(const void* in, int64_t rows, int64_t N, int64_t k, 
                             uint64_t seed, void* stream, void* out_vals, int64_t* out_idx);
 
 /*
+ * Flattened BatchTopK (Section 5, "Application: BatchTopK sparse autoencoders"): the B x d_dict matrix of
+ * pre-activations is read as ONE row of N = B * d_dict elements, its K = B * k largest entries are kept and every
+ * other entry becomes zero.  Stages 1-3 and the count check of Section 3 run as in profk_topk_*; stage 4 only finds
+ * the K-th best candidate and emits the kept set -- nothing is sorted, because the consumer of a BatchTopK does not
+ * need an order.  The kept set is exactly the set profk_topk_* would return for (1 row, N, K): ties at the K-th value
+ * go to the lowest indices, also when the count check fails and the exact selection of the whole row replaces the
+ * buffer.  Exact mode only.  The set comes in up to three forms; pass NULL for a form that is not wanted (at least one
+ * is; sel_vals and sel_idx go together):
+ *   sel_vals, sel_idx  [device] K values and K int64 indices of the kept entries, in no particular order (the order
+ *                      may differ from call to call; compare as a set)
+ *   mask               [device] ceil(N / 32) uint32 words; bit (i % 32) of word i / 32 is set iff entry i is kept
+ *   dense              [device] N elements: entry i holds in[i] (bit for bit) if it is kept, else +0.0.  May be `in`
+ *                      itself (in place): the input is then overwritten once the kernels have finished reading it.
+ * All outputs are written entirely by the call (mask and dense are zeroed first); none is read.
+ *   in     [device] N elements;  eps, seed, stream as for profk_topk_*
+ * The workspace must hold profk_batchtopk_workspace_bytes(capacity, K) bytes, capacity from profk_plan(N, K, eps, 1)
+ * (a little more than profk_workspace_bytes(1, capacity, K) when K <= 8192).  profk_read_stats(stream, 1, ..) reports
+ * the row as after profk_topk_*.  The _planned forms take (S, t, M) explicitly (k_accept must equal K): the test hook
+ * that forces overflow, recall failure and direct mode.
+ * Errors: PROFK_EINVAL, PROFK_EWORKSPACE, PROFK_ECUDA.
+ */
+int profk_batchtopk_workspace_bytes(int64_t capacity, int64_t K, size_t* bytes /* [host] */);
+int profk_batchtopk_f32(const float* in, int64_t N, int64_t K, double eps, uint64_t seed, void* stream,
+                        float* sel_vals, int64_t* sel_idx, uint32_t* mask, float* dense);
+int profk_batchtopk_bf16(const void* in, int64_t N, int64_t K, double eps, uint64_t seed, void* stream,
+                         void* sel_vals, int64_t* sel_idx, uint32_t* mask, void* dense);
+int profk_batchtopk_planned_f32(const float* in, int64_t N, int64_t K, const profk_plan_t* plan, uint64_t seed, void* stream,
+                                float* sel_vals, int64_t* sel_idx, uint32_t* mask, float* dense);
+int profk_batchtopk_planned_bf16(const void* in, int64_t N, int64_t K, const profk_plan_t* plan, uint64_t seed, void* stream,
+                                 void* sel_vals, int64_t* sel_idx, uint32_t* mask, void* dense);
+
+/*
  * Stage 3 alone (the filtering scan of Section 3): for every row append the
  * elements with x_i >= tau[row] to the row's buffer and count them.  The
  * comparison is taken in the total order of the values (-NaN < -inf < ... <

@@ -12,10 +12,16 @@ On inputs without NaN and without -0.0 this is plain numeric order.
 
 bfloat16 has no NumPy dtype: a bf16 array is passed as its uint16 bit patterns.
 
+The flattened BatchTopK of Section 5 ("Application: BatchTopK sparse
+autoencoders") keeps the K largest entries of the flattened activation matrix
+and sets the rest to zero: `kept_mask`, `kept_dense` and `pack_mask` state that
+result in the three forms the library emits, all derived from `topk_row`.
+
 Pins (tests/test_oracle_topk.py): brute force on tiny inputs with ties, the
 special case k = N (a stable descending sort), the prefix property in k, and
 the checker `verify_topk` accepting the true answer and rejecting every single
-corruption tried.
+corruption tried; for the BatchTopK forms, brute force on tiny tied inputs, a
+hand example, the defining properties of the kept set and NumPy's `packbits`.
 """
 from __future__ import annotations
 
@@ -62,6 +68,35 @@ def topk(x: np.ndarray, k: int) -> tuple[np.ndarray, np.ndarray]:
     for r in range(x.shape[0]):
         vals[r], idx[r] = topk_row(x[r], k)
     return vals, idx
+
+
+def kept_mask(x: np.ndarray, k: int) -> np.ndarray:
+    """BatchTopK's kept set as a boolean mask over the flattened input: entry i is True iff i is among the
+    top-k of the flattened array (ties at the k-th value go to the lowest indices)."""
+    flat = x.reshape(-1)
+    _, idx = topk_row(flat, k)
+    mask = np.zeros(flat.shape[0], dtype=bool)
+    mask[idx] = True
+    return mask
+
+
+def kept_dense(x: np.ndarray, k: int) -> np.ndarray:
+    """BatchTopK's result as a dense array: the kept entries bit for bit at their positions, +0.0 elsewhere
+    (the all-zero bit pattern in either element type).  Same shape as x."""
+    flat = x.reshape(-1)
+    mask = kept_mask(flat, k)
+    out = np.zeros_like(flat)
+    out[mask] = flat[mask]
+    return out.reshape(x.shape)
+
+
+def pack_mask(mask: np.ndarray) -> np.ndarray:
+    """Boolean mask -> uint32 words, bit (i % 32) of word (i // 32) = mask[i]; the last word is zero-padded."""
+    n = mask.shape[0]
+    words = np.zeros((n + 31) // 32, dtype=np.uint32)
+    pos = np.flatnonzero(mask)
+    np.bitwise_or.at(words, pos // 32, (np.uint32(1) << (pos % 32).astype(np.uint32)))
+    return words
 
 
 def topk_brute(x: np.ndarray, k: int) -> tuple[np.ndarray, np.ndarray]:

@@ -21,6 +21,8 @@ EXPORTS = [
     "profk_filter_f32", "profk_filter_bf16", "profk_sample_threshold_f32", "profk_sample_threshold_bf16",
     "profk_read_stats", "profk_last_launch_count", "profk_strerror", "profk_topk_noalloc_f32",
     "profk_debug_set_prefetch_wait_polls",
+    "profk_batchtopk_workspace_bytes", "profk_batchtopk_f32", "profk_batchtopk_bf16", "profk_batchtopk_planned_f32",
+    "profk_batchtopk_planned_bf16",
 ]
 
 ROW_OK, ROW_RECALL, ROW_OVERFLOW, ROW_DIRECT = 0, 1, 2, 3
@@ -225,6 +227,75 @@ def topk(x, k: int, eps: float = 1e-3, recall: float = 1.0, seed: int = 0, plan_
     if one_d:
         return vals[0], idx[0]
     return vals, idx
+
+
+def batchtopk_workspace_bytes(capacity: int, k: int) -> int:
+    n = ctypes.c_size_t()
+    _check(lib().profk_batchtopk_workspace_bytes(ctypes.c_int64(capacity), ctypes.c_int64(k), ctypes.byref(n)),
+           "profk_batchtopk_workspace_bytes")
+    return int(n.value)
+
+
+def _ensure_bytes(need: int, device) -> None:
+    """Register a workspace of at least `need` bytes on `device` (allocated through torch)."""
+    import torch
+
+    dev = torch.device(device)
+    idx = dev.index if dev.index is not None else torch.cuda.current_device()
+    cur = _workspaces.get(idx)
+    if cur is not None and cur.numel() >= need:
+        return
+    with torch.cuda.device(idx):
+        buf = torch.empty(max(need, 1 << 20), dtype=torch.uint8, device=dev)
+        _check(lib().profk_set_workspace(ctypes.c_void_p(buf.data_ptr()), ctypes.c_size_t(buf.numel())),
+               "profk_set_workspace")
+    _workspaces[idx] = buf
+    _workspace_ok.clear()
+
+
+def batchtopk(x, k: int, eps: float = 1e-3, seed: int = 0, want_pairs: bool = True, want_mask: bool = False,
+              want_dense: bool = False, in_place: bool = False, plan_override: Plan | None = None):
+    """`profk_batchtopk_*` on the current stream: the K largest entries of the flattened tensor `x` as a set.
+
+    Returns a dict with the forms asked for: "values", "indices" (K each, in no particular order), "mask"
+    (int32 words, bit i % 32 of word i // 32), "dense" (a tensor shaped like `x`; `in_place=True` overwrites
+    `x` itself and returns it).  Nothing is synchronised."""
+    import torch
+
+    if not x.is_cuda or not x.is_contiguous():
+        raise ProfkError("input must be a contiguous CUDA tensor")
+    flat = x.view(-1)
+    n = flat.numel()
+    pl = plan_override if plan_override is not None else plan(n, k, eps, 1.0)
+    _ensure_bytes(batchtopk_workspace_bytes(pl.capacity, k), flat.device)
+    out = {}
+    vals = idx = mask = dense = None
+    if want_pairs:
+        vals = torch.empty(k, dtype=flat.dtype, device=flat.device)
+        idx = torch.empty(k, dtype=torch.int64, device=flat.device)
+        out["values"], out["indices"] = vals, idx
+    if want_mask:
+        mask = torch.empty((n + 31) // 32, dtype=torch.int32, device=flat.device)
+        out["mask"] = mask
+    if want_dense or in_place:
+        dense = flat if in_place else torch.empty_like(flat)
+        out["dense"] = dense.view(x.shape)
+
+    def ptr(t):
+        return ctypes.c_void_p(t.data_ptr() if t is not None else None)
+
+    sfx = _suffix(flat)
+    with torch.cuda.device(flat.device):
+        if plan_override is None:
+            code = getattr(lib(), f"profk_batchtopk_{sfx}")(ptr(flat), ctypes.c_int64(n), ctypes.c_int64(k), ctypes.c_double(eps),
+                                                          ctypes.c_uint64(seed), _stream_ptr(), ptr(vals), ptr(idx), ptr(mask), ptr(dense))
+        else:
+            st = pl._struct()
+            code = getattr(lib(), f"profk_batchtopk_planned_{sfx}")(ptr(flat), ctypes.c_int64(n), ctypes.c_int64(k), ctypes.byref(st),
+                                                                  ctypes.c_uint64(seed), _stream_ptr(), ptr(vals), ptr(idx), ptr(mask),
+                                                                  ptr(dense))
+    _check(code, "profk_batchtopk")
+    return out
 
 
 def topk_noalloc(x, k: int, eps: float = 1e-3, recall: float = 1.0, seed: int = 0, out=None):

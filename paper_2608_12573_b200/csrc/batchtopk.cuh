@@ -1,0 +1,306 @@
+// Flattened BatchTopK (Section 5, "Application: BatchTopK sparse autoencoders"): the B x d_dict pre-activations are
+// one row of N = B * d_dict elements, the K = B * k largest are kept and all others become zero.  The consumer wants
+// the kept SET -- as a list of (value, index) pairs in any order, as a bit mask, or scattered into a dense array of
+// zeros -- not an ordered list, so after the filtering scan nothing has to be sorted: it is enough to find the K-th
+// best candidate record and to emit every record up to it.
+//
+// One cooperative kernel (one CTA per SM, all co-resident, bounded grid barriers) does stage 4 in that form:
+//   * the count check of Section 3, "Refinement"; a row that fails it is replaced on the spot by the exact selection
+//     of the whole row (grid_exact_select_row), which leaves exactly K records -- all of them kept;
+//   * otherwise a histogram select over the R candidate records.  A record r is at distance D = T - r below the
+//     largest record the filter can have kept (T = tau's key with an all-ones index), larger D = better record.
+//     Level 0 bins D on a logarithmic scale (6 bits of exponent, 12 of mantissa: 2^18 bins in global memory, fine
+//     where records are dense); the bin that holds the K-th best record is found by a two-step scan (128 segment
+//     totals, then the one segment); if that bin is crowded (many equal values: its records differ only in the index)
+//     the next levels bin its D range linearly, 18 bits at a time, until at most BK_EDGE records are left in the
+//     boundary class;
+//   * the emit pass: every record of a better class is kept; the boundary class is copied to a short list and ranked
+//     there, its best `need` records are kept as well.  Kept records are appended to the pair list (one atomic per CTA
+//     and pass), set their bit in the mask and are written to the dense array, which the kernel has zeroed before.
+#pragma once
+
+#include "fallback.cuh"
+
+namespace profk {
+
+constexpr int BK_THREADS = FB_THREADS;          // the exact selection it may call is written for this CTA size
+constexpr int BK_BITS = 18;
+constexpr uint32_t BK_BINS = 1u << BK_BITS;
+constexpr uint32_t BK_FLAGS = 8;                // words after the bins: [0] pairs appended, [1] records in the boundary list
+constexpr uint32_t BK_EDGE = 1024;              // a boundary class up to this size is ranked directly
+constexpr uint32_t BK_SEGMENTS = 128;           // the scan cuts the bins into this many segments ...
+constexpr uint32_t BK_SEG_BINS = BK_BINS / BK_SEGMENTS;      // ... of 2048 bins, two per thread
+static_assert(BK_SEG_BINS == 2 * BK_THREADS, "a CTA scans one segment with two bins per thread");
+constexpr int BK_MAX_LEVELS = 6;                // 12 + 18 * 3 > 64 bits: more levels than any input needs
+
+template <typename T> struct BatchTopkParams {
+    FallbackParams<T> fb;        // the row (rows == 1), K, capacity, control block, header, histogram area, buffer
+    uint32_t* bins;              // BK_BINS + BK_FLAGS words
+    uint32_t* seg_totals;        // BK_SEGMENTS words
+    uint64_t* edge;              // BK_EDGE records: the boundary class
+    uint32_t parts;              // 1, or FILTER_PARTS: the filter appended to that many parts of the buffer
+    uint32_t part_cap;
+    const uint32_t* part_counts;
+    T* sel_vals;                 // K values of the kept elements, any order (null = not wanted); with sel_idx
+    int64_t* sel_idx;            // K indices, same order
+    uint32_t* mask;              // ceil(N / 32) words, bit i & 31 of word i >> 5 = element i is kept (null = not wanted)
+    T* dense;                    // N elements: the kept values at their positions, zero elsewhere; may be the input itself
+    int use_pdl;
+    int direct;                  // 1 = no threshold / filter ran: the row is selected exactly
+};
+
+// Bin of the logarithmic level: exponent e = floor(log2 D) in the top 6 bits, the 12 bits after the leading one below.
+// Monotone in D.  D = 0 shares bin 0 with D = 1.
+__device__ __forceinline__ uint32_t bk_log_bin(uint64_t D) {
+    if (D < 2) return 0;
+    const int e = 63 - __clzll((long long)D);
+    const uint64_t frac = D ^ (1ull << e);
+    const uint32_t m = e >= 12 ? (uint32_t)(frac >> (e - 12)) : (uint32_t)(frac << (12 - e));
+    return ((uint32_t)e << 12) | m;
+}
+// The D range of a bin of the logarithmic level: [lo, lo + 2^w).
+__device__ __forceinline__ void bk_log_bin_range(uint32_t bin, uint64_t* lo, int* w) {
+    if (bin == 0) { *lo = 0; *w = 1; return; }
+    const int e = (int)(bin >> 12);
+    const uint64_t m = bin & 4095u;
+    if (e >= 12) { *lo = (1ull << e) | (m << (e - 12)); *w = e - 12; }
+    else { *lo = (1ull << e) + (m >> (12 - e)); *w = 0; }
+}
+
+// Zeroes n elements at p (aligned to the element size only) with 16-byte stores where the address allows.
+template <typename E>
+__device__ __forceinline__ void bk_zero_fill(E* p, uint64_t n, uint64_t gid, uint64_t gthreads) {
+    const uintptr_t a = (uintptr_t)p;
+    const uint64_t head_bytes = (16 - (a & 15)) & 15;
+    uint64_t head = head_bytes / sizeof(E);
+    if (head > n) head = n;
+    const uint64_t body = (n - head) * sizeof(E) / 16;                   // whole 16-byte vectors
+    const uint64_t tail0 = head + body * (16 / sizeof(E));
+    for (uint64_t i = gid; i < head; i += gthreads) p[i] = E{};
+    uint4* v = reinterpret_cast<uint4*>(p + head);
+    for (uint64_t i = gid; i < body; i += gthreads) v[i] = make_uint4(0u, 0u, 0u, 0u);
+    for (uint64_t i = tail0 + gid; i < n; i += gthreads) p[i] = E{};
+}
+
+template <typename T>
+__global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const BatchTopkParams<T> p) {
+    __shared__ SelectShared sh;                  // hist / start / warp_sums serve the scans here and the exact selection
+    __shared__ uint32_t s_seg, s_seg_before, s_bin, s_bin_before, s_bin_count, s_base;
+    __shared__ uint32_t s_warp_count[BK_THREADS / 32];
+
+    const unsigned tid = threadIdx.x, lane = lane_id(), warp = tid >> 5;
+    const unsigned nctas = gridDim.x, cta = blockIdx.x;
+    const uint64_t gid = (uint64_t)cta * BK_THREADS + tid, gthreads = (uint64_t)nctas * BK_THREADS;
+    const FallbackParams<T>& fb = p.fb;
+    uint32_t* flags = p.bins + BK_BINS;
+
+    // Prologue, before the wait for the filter kernel: the workspace's bins and flags (nobody else uses them).
+    for (uint64_t b = gid; b < BK_BINS + BK_FLAGS; b += gthreads) p.bins[b] = 0;
+    pdl_launch_dependents();
+    if (p.use_pdl) pdl_wait();
+    uint32_t gen = *((volatile uint32_t*)&fb.header->bar_gen);          // read before this CTA's first arrival
+
+    // ---- the count check of stage 4 (the same in every CTA) ----
+    const uint32_t K = fb.k;
+    uint32_t pcount[FILTER_PARTS] = {};           // the records are pcount[j] at buf + j * part_cap
+    uint32_t status;
+    if (p.direct) {
+        status = ROW_DIRECT;
+    } else {
+        uint32_t R = __ldcg(&fb.ctl[0].count);
+        bool part_full = false;
+        if (p.parts > 1) {                        // partitioned append: the row's count is the sum of its parts'
+            uint64_t sum = 0;
+#pragma unroll
+            for (int j = 0; j < (int)FILTER_PARTS; ++j) {
+                const uint32_t c = __ldcg(&p.part_counts[j * FILTER_PART_STRIDE]);
+                part_full |= c > p.part_cap;
+                pcount[j] = c < p.part_cap ? c : p.part_cap;
+                sum += c;
+            }
+            R = sum > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)sum;
+        } else {
+            pcount[0] = R;
+        }
+        status = (R > fb.capacity || part_full) ? ROW_OVERFLOW : R < K ? ROW_RECALL : ROW_OK;
+        if (cta == 0 && tid == 0) {
+            if (p.parts > 1) fb.ctl[0].count = part_full && R <= fb.capacity ? fb.capacity + 1 : R;     // what the statistics report
+            fb.ctl[0].status = status;
+            fb.ctl[0].n_final = K;
+            if (status) atomicAdd(&fb.header->n_failed, 1u);
+        }
+    }
+    bool keep_all = false;                        // every record in the buffer is kept (it holds exactly K)
+    if (status != ROW_OK) {
+        // The exact replacement (Section 3, "Refinement"): the K best records of the whole row, into the buffer.
+        if (!grid_exact_select_row<T>(fb, 0, gen, sh.hist, sh.warp_sums)) return;
+#pragma unroll
+        for (int j = 0; j < (int)FILTER_PARTS; ++j) pcount[j] = 0;
+        pcount[0] = K;
+        keep_all = true;
+    }
+    uint32_t pend[FILTER_PARTS];                  // pend[j] = records in parts 0..j
+    {
+        uint32_t acc = 0;
+#pragma unroll
+        for (int j = 0; j < (int)FILTER_PARTS; ++j) { acc += pcount[j]; pend[j] = acc; }
+    }
+    const uint32_t total = pend[FILTER_PARTS - 1];
+    const uint32_t iters = (uint32_t)((total + gthreads - 1) / gthreads);        // the same for every thread
+    auto record_at = [&](uint64_t i) {
+        uint32_t j = 0, before = 0;
+#pragma unroll
+        for (int q = 0; q < (int)FILTER_PARTS - 1; ++q)
+            if (i >= pend[q]) { j = q + 1; before = pend[q]; }
+        return (uint64_t)__ldcg(fb.buf + (uint64_t)j * p.part_cap + (i - before));
+    };
+
+    // The dense result and the mask start from zero.  (After the exact selection, which reads the input: the dense
+    // array may be the input itself.)  The barriers below order these stores before the emit pass.
+    if (p.mask) bk_zero_fill(p.mask, (fb.N + 31) / 32, gid, gthreads);
+    if (p.dense) bk_zero_fill(p.dense, fb.N, gid, gthreads);
+
+    // ---- the class of the K-th best record ----
+    // D = top - record >= 0 for every record the filter kept (their keys are >= tau's); larger D = better record.
+    const uint32_t tau_key = Elem<T>::key(Elem<T>::from_bits(__ldcg(&fb.ctl[0].tau_bits)));
+    const uint64_t top = make_record(tau_key, 0xFFFFFFFFu);
+    uint64_t cls_lo = 0;          // the boundary class is cls_lo <= D < cls_lo + 2^cls_w ...
+    int cls_w = 64;               // ... (64: every D)
+    uint32_t need = K;            // ... and its `need` best records are kept, with every record of a better class
+    bool whole = keep_all;        // the whole boundary class is kept: nothing to rank
+    if (keep_all) need = 0;
+    if (!grid_barrier(fb.header, gen)) return;                            // bins are zero, in every CTA's view
+    for (int level = 0; !whole && level < BK_MAX_LEVELS; ++level) {
+        const int sh_bits = cls_w > BK_BITS ? cls_w - BK_BITS : 0;       // linear levels: D's bits below the bin
+        auto bin_of = [&](uint64_t D, bool* in_class) {
+            if (level == 0) { *in_class = true; return bk_log_bin(D); }
+            *in_class = D >= cls_lo && ((D - cls_lo) >> cls_w) == 0;
+            return (uint32_t)((D - cls_lo) >> sh_bits) & (BK_BINS - 1);
+        };
+        // histogram, best records in the lowest bins
+        for (uint64_t i = gid; i < total; i += gthreads) {
+            bool in_class;
+            const uint32_t b = bin_of(top - record_at(i), &in_class);
+            if (in_class) atomicAdd(&p.bins[BK_BINS - 1 - b], 1u);
+        }
+        if (!grid_barrier(fb.header, gen)) return;
+        // totals of the segments
+        for (uint32_t s = cta; s < BK_SEGMENTS; s += nctas) {
+            const uint2 c = __ldcg(reinterpret_cast<const uint2*>(p.bins + s * BK_SEG_BINS) + tid);
+            const uint32_t incl = block_inclusive_scan(c.x + c.y, sh.warp_sums);
+            if (tid == BK_THREADS - 1) p.seg_totals[s] = incl;
+            __syncthreads();
+        }
+        if (!grid_barrier(fb.header, gen)) return;
+        // every CTA: the segment, then the bin, of the need-th best record of the class
+        if (warp == 0) {
+            uint32_t t[BK_SEGMENTS / 32], sum = 0;
+#pragma unroll
+            for (int j = 0; j < (int)(BK_SEGMENTS / 32); ++j) { t[j] = __ldcg(&p.seg_totals[lane * (BK_SEGMENTS / 32) + j]); sum += t[j]; }
+            uint32_t incl = sum;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t v = __shfl_up_sync(FULL_MASK, incl, d);
+                if (lane >= (unsigned)d) incl += v;
+            }
+            uint32_t before = incl - sum;
+#pragma unroll
+            for (int j = 0; j < (int)(BK_SEGMENTS / 32); ++j) {
+                if (before < need && need <= before + t[j]) { s_seg = lane * (BK_SEGMENTS / 32) + j; s_seg_before = before; }
+                before += t[j];
+            }
+        }
+        __syncthreads();
+        {
+            const uint32_t seg = s_seg, seg_before = s_seg_before;
+            const uint2 c = __ldcg(reinterpret_cast<const uint2*>(p.bins + seg * BK_SEG_BINS) + tid);
+            const uint32_t incl = block_inclusive_scan(c.x + c.y, sh.warp_sums);
+            const uint32_t b0 = seg_before + incl - c.x - c.y, b1 = b0 + c.x;
+            if (b0 < need && need <= b0 + c.x) { s_bin = seg * BK_SEG_BINS + 2 * tid; s_bin_before = b0; s_bin_count = c.x; }
+            else if (b1 < need && need <= b1 + c.y) { s_bin = seg * BK_SEG_BINS + 2 * tid + 1; s_bin_before = b1; s_bin_count = c.y; }
+            __syncthreads();
+        }
+        const uint32_t bin = BK_BINS - 1 - s_bin, in_bin = s_bin_count;
+        need -= s_bin_before;
+        if (level == 0) bk_log_bin_range(bin, &cls_lo, &cls_w);
+        else { cls_lo += (uint64_t)bin << sh_bits; cls_w = sh_bits; }
+        __syncthreads();                           // the shared words are rewritten by the next level
+        if (in_bin == need) { whole = true; break; }
+        if (in_bin <= BK_EDGE) break;
+        // crowded: one more level inside the class; the bins start from zero again
+        for (uint64_t b = gid; b < BK_BINS; b += gthreads) p.bins[b] = 0;
+        if (!grid_barrier(fb.header, gen)) return;
+    }
+    // Kept outright: D >= keep_from.  Boundary list: cls_lo <= D < keep_from (empty when the whole class is kept).
+    const bool top_class = cls_w >= 64 || cls_lo + (1ull << cls_w) < cls_lo;      // the class reaches the largest D there is
+    const uint64_t keep_from = whole ? cls_lo : cls_lo + (1ull << (cls_w & 63));
+    const uint32_t n_outright = K - (whole ? 0u : need);
+
+    // ---- emit ----
+    auto emit = [&](uint64_t rec, uint32_t pos) {
+        const uint32_t idx = record_idx(rec);
+        const T val = Elem<T>::from_key(record_key(rec));
+        if (p.sel_idx) { p.sel_vals[pos] = val; p.sel_idx[pos] = (int64_t)idx; }
+        if (p.mask) atomicOr(&p.mask[idx >> 5], 1u << (idx & 31u));
+        if (p.dense) p.dense[idx] = val;
+    };
+    for (uint32_t it = 0; it < iters; ++it) {
+        const uint64_t i = (uint64_t)it * gthreads + gid;
+        uint64_t rec = 0;
+        bool kept = false, boundary = false;
+        if (i < total) {
+            rec = record_at(i);
+            const uint64_t D = top - rec;
+            kept = keep_all || (whole ? D >= keep_from : (!top_class && D >= keep_from));
+            boundary = !kept && !whole && D >= cls_lo;
+        }
+        const unsigned bal = __ballot_sync(FULL_MASK, kept);
+        if (lane == 0) s_warp_count[warp] = __popc(bal);
+        const unsigned ebal = __ballot_sync(FULL_MASK, boundary);
+        if (ebal) {
+            uint32_t ebase = 0;
+            if (lane == 0) ebase = atomicAdd(&flags[1], (uint32_t)__popc(ebal));
+            ebase = __shfl_sync(FULL_MASK, ebase, 0);
+            const uint32_t epos = ebase + __popc(ebal & ((1u << lane) - 1u));
+            if (boundary && epos < BK_EDGE) p.edge[epos] = rec;
+        }
+        __syncthreads();
+        if (warp == 0) {                           // one atomic per CTA and pass
+            const uint32_t c = s_warp_count[lane];
+            uint32_t incl = c;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t v = __shfl_up_sync(FULL_MASK, incl, d);
+                if (lane >= (unsigned)d) incl += v;
+            }
+            uint32_t base = 0;
+            if (lane == 31 && incl) base = atomicAdd(&flags[0], incl);
+            base = __shfl_sync(FULL_MASK, base, 31);
+            s_warp_count[lane] = base + incl - c;  // first position of the warp's records
+        }
+        __syncthreads();
+        if (kept) {
+            const uint32_t pos = s_warp_count[warp] + __popc(bal & ((1u << lane) - 1u));
+            if (pos < n_outright) emit(rec, pos);
+        }
+        __syncthreads();                           // s_warp_count is rewritten by the next pass
+    }
+    if (whole) return;
+
+    // ---- the boundary class: rank its records, keep the best `need` ----
+    if (!grid_barrier(fb.header, gen)) return;
+    if (cta != 0) return;
+    const uint32_t n_edge = min(__ldcg(&flags[1]), BK_EDGE);
+    uint64_t* list = sh.edge;                      // RF_EDGE_CAP == BK_EDGE records of shared memory
+    static_assert(RF_EDGE_CAP >= BK_EDGE, "the boundary list fits SelectShared::edge");
+    for (uint32_t i = tid; i < n_edge; i += BK_THREADS) list[i] = __ldcg(&p.edge[i]);
+    __syncthreads();
+    for (uint32_t i = tid; i < n_edge; i += BK_THREADS) {
+        const uint64_t mine = list[i];
+        uint32_t rank = 0;
+        for (uint32_t j = 0; j < n_edge; ++j) rank += list[j] < mine;
+        if (rank < need) emit(mine, n_outright + rank);
+    }
+}
+
+}  // namespace profk

@@ -81,13 +81,95 @@ __device__ __forceinline__ void for_each_record(const FallbackParams<T>& p, uint
     }
 }
 
+// Exact selection of the k smallest records of `row` by the whole grid (FB_THREADS threads per CTA, all CTAs
+// co-resident): a most-significant-digit radix select over the row's elements as 64-bit records, 11 bits per pass,
+// a grid barrier after each, then one more read of the row that appends the k winners to the row's buffer (counter:
+// the row's `collect` word, zero on entry).  Called by every thread of every CTA; `gen` is the caller's copy of the
+// grid barrier's generation.  Returns false when a bounded wait gave up (the caller leaves the kernel); on a true
+// return the last barrier has been passed and the k records are in p.buf + row * p.buf_stride, in no particular order.
+template <typename T>
+__device__ __noinline__ bool grid_exact_select_row(const FallbackParams<T>& p, uint64_t row, uint32_t& gen, uint32_t* sh_hist,
+                                                   uint32_t* warp_sums) {
+    __shared__ uint32_t s_digit, s_before, s_cnt;
+    const unsigned tid = threadIdx.x, lane = lane_id();
+    if (!grid_barrier(p.header, gen)) return false;          // a previous row's histogram reads are over
+    for (uint32_t i = blockIdx.x * FB_THREADS + tid; i < FB_PASSES * FB_BINS; i += gridDim.x * FB_THREADS)
+        p.ghist[i] = 0;
+    if (!grid_barrier(p.header, gen)) return false;
+
+    uint64_t prefix = 0;       // selected high bits, right-aligned
+    uint32_t need = p.k;       // rank (from the smallest record) inside the prefix class
+    uint64_t limit = ~0ull;    // records <= limit are the answer
+    for (int pass = 0; pass < FB_PASSES; ++pass) {
+        const int shift = pass < 5 ? 53 - 11 * pass : 0;
+        const int width = pass < 5 ? 11 : 9;
+        const uint32_t nbins = 1u << width;
+        for (uint32_t i = tid; i < nbins; i += FB_THREADS) sh_hist[i] = 0;
+        __syncthreads();
+        for_each_record(p, row, [&](uint64_t rec, bool valid) {
+            const bool in_class = valid && (pass == 0 || (rec >> (shift + width)) == prefix);
+            const uint32_t digit = in_class ? (uint32_t)(rec >> shift) & (nbins - 1) : 0xFFFFFFFFu;
+            const unsigned peers = __match_any_sync(FULL_MASK, digit);
+            if (in_class && lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&sh_hist[digit], __popc(peers));
+        });
+        __syncthreads();
+        uint32_t* gh = p.ghist + pass * FB_BINS;
+        for (uint32_t i = tid; i < nbins; i += FB_THREADS) {
+            const uint32_t c = sh_hist[i];
+            if (c) atomicAdd(&gh[i], c);
+        }
+        if (!grid_barrier(p.header, gen)) return false;
+
+        // Every CTA finds the bin that holds the need-th smallest record of the class.
+        constexpr int PER = FB_BINS / FB_THREADS;                   // bins per thread
+        uint32_t c[PER], sum = 0;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            const uint32_t bin = tid * PER + j;
+            c[j] = bin < nbins ? __ldcg(&gh[bin]) : 0;
+            sum += c[j];
+        }
+        uint32_t before = block_inclusive_scan(sum, warp_sums) - sum;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            if (before < need && need <= before + c[j]) { s_digit = tid * PER + j; s_before = before; s_cnt = c[j]; }
+            before += c[j];
+        }
+        __syncthreads();
+        prefix = (prefix << width) | s_digit;
+        need -= s_before;
+        const bool whole_bin = (s_cnt == need);
+        __syncthreads();
+        if (whole_bin || pass == FB_PASSES - 1) {
+            limit = ((prefix + 1) << shift) - 1;        // wraps to all-ones when the class is the last one
+            break;
+        }
+    }
+
+    // ---- collect the k records <= limit into the row's buffer ----
+    uint64_t* dst = p.buf + row * p.buf_stride;
+    uint32_t* counter = &p.ctl[row].collect;
+    const unsigned lt_mask = (1u << lane) - 1u;
+    for_each_record(p, row, [&](uint64_t rec, bool valid) {
+        const bool take = valid && rec <= limit;
+        const unsigned bal = __ballot_sync(FULL_MASK, take);
+        if (bal) {
+            unsigned base = 0;
+            if (lane == 0) base = atomicAdd(counter, __popc(bal));
+            base = __shfl_sync(FULL_MASK, base, 0);
+            const unsigned pos = base + __popc(bal & lt_mask);
+            if (take && pos < p.capacity) dst[pos] = rec;
+        }
+    });
+    return grid_barrier(p.header, gen);
+}
+
 template <typename T>
 __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackParams<T> p) {
     __shared__ SelectShared sh;                 // the per-CTA selection's state; its arrays also serve the grid-wide one
     uint32_t* sh_hist = sh.hist;                // FB_BINS <= RF_BINS words
     uint32_t* warp_sums = sh.warp_sums;
     __shared__ uint32_t flag_masks[FB_THREADS / 32];
-    __shared__ uint32_t s_digit, s_before, s_cnt;
 
     const unsigned tid = threadIdx.x, lane = lane_id(), warp = tid >> 5;
     pdl_launch_dependents();
@@ -140,80 +222,12 @@ __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackPara
                 mask &= mask - 1;
                 const uint64_t row = chunk + w * 32 + b;
 
-                // ---- exact selection of the k smallest records of `row` ----
-                if (!grid_barrier(p.header, gen)) return;          // previous row's histogram reads are over
-                for (uint32_t i = blockIdx.x * FB_THREADS + tid; i < FB_PASSES * FB_BINS; i += gridDim.x * FB_THREADS)
-                    p.ghist[i] = 0;
-                if (!grid_barrier(p.header, gen)) return;
-
-                uint64_t prefix = 0;       // selected high bits, right-aligned
-                uint32_t need = p.k;       // rank (from the smallest record) inside the prefix class
-                uint64_t limit = ~0ull;    // records <= limit are the answer
-                for (int pass = 0; pass < FB_PASSES; ++pass) {
-                    const int shift = pass < 5 ? 53 - 11 * pass : 0;
-                    const int width = pass < 5 ? 11 : 9;
-                    const uint32_t nbins = 1u << width;
-                    for (uint32_t i = tid; i < nbins; i += FB_THREADS) sh_hist[i] = 0;
-                    __syncthreads();
-                    for_each_record(p, row, [&](uint64_t rec, bool valid) {
-                        const bool in_class = valid && (pass == 0 || (rec >> (shift + width)) == prefix);
-                        const uint32_t digit = in_class ? (uint32_t)(rec >> shift) & (nbins - 1) : 0xFFFFFFFFu;
-                        const unsigned peers = __match_any_sync(FULL_MASK, digit);
-                        if (in_class && lane == (unsigned)(__ffs(peers) - 1)) atomicAdd(&sh_hist[digit], __popc(peers));
-                    });
-                    __syncthreads();
-                    uint32_t* gh = p.ghist + pass * FB_BINS;
-                    for (uint32_t i = tid; i < nbins; i += FB_THREADS) {
-                        const uint32_t c = sh_hist[i];
-                        if (c) atomicAdd(&gh[i], c);
-                    }
-                    if (!grid_barrier(p.header, gen)) return;
-
-                    // Every CTA finds the bin that holds the need-th smallest record of the class.
-                    constexpr int PER = FB_BINS / FB_THREADS;                   // bins per thread
-                    uint32_t c[PER], sum = 0;
-#pragma unroll
-                    for (int j = 0; j < PER; ++j) {
-                        const uint32_t bin = tid * PER + j;
-                        c[j] = bin < nbins ? __ldcg(&gh[bin]) : 0;
-                        sum += c[j];
-                    }
-                    uint32_t before = block_inclusive_scan(sum, warp_sums) - sum;
-#pragma unroll
-                    for (int j = 0; j < PER; ++j) {
-                        if (before < need && need <= before + c[j]) { s_digit = tid * PER + j; s_before = before; s_cnt = c[j]; }
-                        before += c[j];
-                    }
-                    __syncthreads();
-                    prefix = (prefix << width) | s_digit;
-                    need -= s_before;
-                    const bool whole_bin = (s_cnt == need);
-                    __syncthreads();
-                    if (whole_bin || pass == FB_PASSES - 1) {
-                        limit = ((prefix + 1) << shift) - 1;        // wraps to all-ones when the class is the last one
-                        break;
-                    }
-                }
-
-                // ---- collect the k records <= limit into the row's buffer ----
+                // ---- exact selection of the k smallest records of `row` into the row's buffer ----
+                if (!grid_exact_select_row<T>(p, row, gen, sh_hist, warp_sums)) return;
                 uint64_t* dst = p.buf + row * p.buf_stride;
-                uint32_t* counter = &p.ctl[row].collect;
-                const unsigned lt_mask = (1u << lane) - 1u;
-                for_each_record(p, row, [&](uint64_t rec, bool valid) {
-                    const bool take = valid && rec <= limit;
-                    const unsigned bal = __ballot_sync(FULL_MASK, take);
-                    if (bal) {
-                        unsigned base = 0;
-                        if (lane == 0) base = atomicAdd(counter, __popc(bal));
-                        base = __shfl_sync(FULL_MASK, base, 0);
-                        const unsigned pos = base + __popc(bal & lt_mask);
-                        if (take && pos < p.capacity) dst[pos] = rec;
-                    }
-                });
 
                 // ---- order the k records and write the row's output (first CTA; the others move on
                 //      and meet it again at the next row's barrier) ----
-                if (!grid_barrier(p.header, gen)) return;
                 if (p.sort_rows && blockIdx.x == 0) {
                     extern __shared__ __align__(16) unsigned char fb_smem[];
                     uint64_t* sortbuf = reinterpret_cast<uint64_t*>(fb_smem);

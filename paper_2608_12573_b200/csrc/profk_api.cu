@@ -11,6 +11,7 @@
 #include <tuple>
 #include <vector>
 
+#include "batchtopk.cuh"
 #include "fallback.cuh"
 #include "filter.cuh"
 #include "profk.h"
@@ -79,21 +80,22 @@ struct WsLayout {
 
 // Records reserved per row: the capacity itself, or -- when k is too large for the single-CTA
 // refine -- twice the power of two the cluster sort pads the row to (records, then scratch).
-uint64_t row_stride_for(int64_t rows, int64_t capacity, int64_t k) {
-    if (!large_selection(rows, k)) return (uint64_t)capacity;
+uint64_t row_stride_for(int64_t capacity, bool large) {
+    if (!large) return (uint64_t)capacity;
     uint64_t p = BT_TILE;
     while (p < (uint64_t)capacity) p <<= 1;
     return 2 * p;
 }
 
-WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k) {
+// `large` = the layout of large selections (bins, partitioned append counters, doubled row pitch): whenever
+// large_selection(rows, k) says so, and always for the flattened BatchTopK calls, whose select works on the bins.
+WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k, bool large) {
     WsLayout l;
     l.off_header = 0;
     l.off_ghist = sizeof(WsHeader);
     l.off_ctl = align_up(l.off_ghist + (size_t)FB_PASSES * FB_BINS * sizeof(uint32_t), 256);
     l.off_tau = align_up(l.off_ctl + (size_t)rows * sizeof(RowCtl), 256);
     l.off_bins = align_up(l.off_tau + (size_t)rows * sizeof(uint4), 256);
-    const bool large = large_selection(rows, k);
     const size_t bins_bytes = large ? (size_t)rows * (LG_BINS + 8) * sizeof(uint32_t) : 0;
     // scratch of the in-refine exact selection (few rows, k within the single-CTA refine): up to
     // XS_MAX_SEGMENTS segments in all, each with a counter and k + XS_EDGE records
@@ -109,7 +111,7 @@ WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k) {
     // counters of the partitioned append (large selections only), each in a 256-byte line of its own
     l.off_parts = align_up(l.off_fb_records + (fbp ? (size_t)FB_MAX_CTAS * (size_t)(k + XS_EDGE) * sizeof(uint64_t) : 0), 256);
     l.off_buf = align_up(l.off_parts + (large ? (size_t)rows * FILTER_PARTS * FILTER_PART_STRIDE * sizeof(uint32_t) : 0), 256);
-    l.total = align_up(l.off_buf + (size_t)rows * (size_t)row_stride_for(rows, capacity, k) * sizeof(uint64_t), 256);
+    l.total = align_up(l.off_buf + (size_t)rows * (size_t)row_stride_for(capacity, large) * sizeof(uint64_t), 256);
     return l;
 }
 
@@ -335,8 +337,11 @@ int launch_cooperative(cudaLaunchConfig_t cfg, Kernel kernel, Params params, boo
 template <typename T>
 int launch_refine_large(const DeviceInfo& di, RowCtl* ctl, WsHeader* header, uint64_t* buf, uint64_t row_pitch, uint32_t* bins,
                         unsigned long long* slots, bool parts, uint32_t part_cap, const uint32_t* part_counts, int64_t rows,
-                        int64_t capacity, int64_t k, int64_t k_accept, int phase, T* out_vals, int64_t* out_idx, cudaStream_t st) {
+                        int64_t capacity, int64_t k, int64_t k_accept, int phase, T* out_vals, int64_t* out_idx, cudaStream_t st,
+                        const FallbackParams<T>* fused_fb = nullptr, bool after_kernel = true) {
     LargeParams<T> lp;
+    lp.fused = fused_fb ? 1 : 0;
+    if (fused_fb) lp.fb = *fused_fb; else lp.fb = FallbackParams<T>{};
     lp.ctl = ctl; lp.header = header; lp.buf = buf; lp.row_stride = row_pitch / 2; lp.bins = bins; lp.slots = slots;
     lp.parts = (phase == 0 && parts) ? FILTER_PARTS : 1u; lp.part_cap = part_cap; lp.part_counts = part_counts;
     lp.rows = (uint64_t)rows; lp.capacity = (uint32_t)capacity;
@@ -351,7 +356,7 @@ int launch_refine_large(const DeviceInfo& di, RowCtl* ctl, WsHeader* header, uin
     cfg.blockDim = dim3(BT_THREADS);
     cfg.dynamicSmemBytes = (size_t)BT_TILE * 8;
     cfg.stream = st;
-    return launch_cooperative(cfg, refine_large_kernel<T>, lp, true, [](LargeParams<T>& q, int v) { q.use_pdl = v; });
+    return launch_cooperative(cfg, refine_large_kernel<T>, lp, after_kernel, [](LargeParams<T>& q, int v) { q.use_pdl = v; });
 }
 
 // Who replaces a row that fails the count check.  With few rows each row gets a cluster of CTAs in
@@ -448,10 +453,10 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         std::lock_guard<std::mutex> lock(g_mutex);
         ws = g_workspace[dev];
     }
-    const WsLayout lay = ws_layout(rows, capacity, k);
-    if (!ws.ptr || ws.bytes < lay.total) return PROFK_EWORKSPACE;
-    const uint64_t row_stride = row_stride_for(rows, capacity, k);
     const bool large = large_selection(rows, k);
+    const WsLayout lay = ws_layout(rows, capacity, k, large);
+    if (!ws.ptr || ws.bytes < lay.total) return PROFK_EWORKSPACE;
+    const uint64_t row_stride = row_stride_for(capacity, large);
     unsigned char* base = static_cast<unsigned char*>(ws.ptr);
     WsHeader* header = reinterpret_cast<WsHeader*>(base + lay.off_header);
     uint32_t* ghist = reinterpret_cast<uint32_t*>(base + lay.off_ghist);
@@ -483,6 +488,23 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     uint32_t fb_sort_cap = 32;
     while (fb_sort_cap < (uint32_t)k && fb_sort_cap < SORT_CAP_MAX) fb_sort_cap <<= 1;
 
+    // What the grid-wide exact selection needs (the kernel of its own, or the large refine when it does that itself).
+    FallbackParams<T> fb;
+    fb.in = in; fb.N = (uint64_t)N; fb.rows = (uint64_t)rows; fb.k = (uint32_t)k;
+    fb.capacity = (uint32_t)capacity; fb.ctl = ctl; fb.header = header; fb.ghist = ghist; fb.buf = buf;
+    fb.buf_stride = row_stride; fb.sort_rows = large ? 0 : 1;
+    fb.tiles_per_row = tiles_per_row<T>((uint64_t)N, FB_THREADS * FB_UNROLL);
+    fb.use_pdl = 0;
+    fb.out_vals = out_vals; fb.out_idx = out_idx;
+    const bool fbp = rows > XS_MAX_ROWS && !large;
+    fb.cta_records = fbp ? reinterpret_cast<uint64_t*>(base + lay.off_fb_records) : nullptr;
+    fb.cta_counters = fbp ? reinterpret_cast<uint32_t*>(base + lay.off_fb_counters) : nullptr;
+    fb.sort_cap = fb_sort_cap;
+    fb.parallel = (fbp || large) ? 1 : 0;      // large selections write into the rows' own buffers
+    // A large selection from a single row: the count check, the exact replacement of a row that fails it and the
+    // ordering are one cooperative kernel (three launches otherwise, two of which do nothing when no row failed).
+    const bool fused_large = large && rows == 1;
+
     if (plan->mode == 0) {
         rc = launch_sample_select<T>(di, in, rows, N, plan->m, plan->r, seed, nullptr, ctl, header, (uint32_t)capacity, nullptr,
                                      rows <= GATHER_MAX_ROWS ? keys_scratch : nullptr, parts ? part_counts : nullptr, plan->tie_rule == PROFK_TIES_BY_INDEX, thr, st);
@@ -493,8 +515,8 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
 
         if (large) {
             rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, reinterpret_cast<unsigned long long*>(ghist), parts, part_cap, part_counts, rows,
-                                        capacity, k, plan->k_accept, 0,
-                                        out_vals, out_idx, st);
+                                        capacity, k, plan->k_accept, 0, out_vals, out_idx, st, fused_large ? &fb : nullptr);
+            if (fused_large) return rc;
         } else {
             // count check and refine; with clusters, also the exact selection of the rows that fail the check
             rc = launch_refine<T>(di, in, rows, N, ctl, header, buf, row_stride, capacity, k, plan->k_accept, false, csize, xs_records, xs_counters, out_vals, out_idx, st);
@@ -506,24 +528,15 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         ++g_launches;
         if (exact_in_refine)
             return launch_refine<T>(di, in, rows, N, ctl, header, buf, row_stride, capacity, k, k, true, csize, xs_records, xs_counters, out_vals, out_idx, st);
+        if (fused_large)
+            return launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, reinterpret_cast<unsigned long long*>(ghist), false, part_cap, part_counts, rows,
+                                          capacity, k, k, 0, out_vals, out_idx, st, &fb, false);
     }
 
     if (!exact_in_refine) {
         // Exact selection of the rows that failed the check (or, in direct mode, of all rows) by a grid-wide
         // cooperative kernel: all CTAs co-resident.  For large selections it runs between the two phases
-        // of the cluster refine.
-        FallbackParams<T> fb;
-        fb.in = in; fb.N = (uint64_t)N; fb.rows = (uint64_t)rows; fb.k = (uint32_t)k;
-        fb.capacity = (uint32_t)capacity; fb.ctl = ctl; fb.header = header; fb.ghist = ghist; fb.buf = buf;
-        fb.buf_stride = row_stride; fb.sort_rows = large ? 0 : 1;
-        fb.tiles_per_row = tiles_per_row<T>((uint64_t)N, FB_THREADS * FB_UNROLL);
-        fb.use_pdl = 0;
-        fb.out_vals = out_vals; fb.out_idx = out_idx;
-        const bool fbp = rows > XS_MAX_ROWS && !large;
-        fb.cta_records = fbp ? reinterpret_cast<uint64_t*>(base + lay.off_fb_records) : nullptr;
-        fb.cta_counters = fbp ? reinterpret_cast<uint32_t*>(base + lay.off_fb_counters) : nullptr;
-        fb.sort_cap = fb_sort_cap;
-        fb.parallel = (fbp || large) ? 1 : 0;      // large selections write into the rows' own buffers
+        // of the large refine.
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(std::min<unsigned>((unsigned)di.sm_count, FB_MAX_CTAS));
         cfg.blockDim = dim3(FB_THREADS);
@@ -541,26 +554,122 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     return PROFK_OK;
 }
 
+// The library's plan for a shape, kept for the shapes seen (the plan costs some host time: tail sums, bisections).
+int cached_plan(int64_t rows, int64_t N, int64_t k, double eps, double recall, profk_plan_t* plan) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    const int64_t plan_rows = rows <= GATHER_MAX_ROWS ? 1 : GATHER_MAX_ROWS + 1;     // the two classes the tuning knows
+    const auto key = std::make_tuple(plan_rows, N, k, eps, recall);
+    auto it = g_plan_cache.find(key);
+    if (it == g_plan_cache.end()) {
+        const int rc = profk_plan_batch(plan_rows, N, k, eps, recall, plan);
+        if (rc != PROFK_OK) return rc;
+        if (g_plan_cache.size() > 4096) g_plan_cache.clear();
+        g_plan_cache[key] = *plan;
+    } else {
+        *plan = it->second;
+    }
+    return PROFK_OK;
+}
+
 template <typename T>
 int topk_auto(const T* in, int64_t rows, int64_t N, int64_t k, double eps, double recall, uint64_t seed, void* stream,
               T* out_vals, int64_t* out_idx) {
     g_launches = 0;
     profk_plan_t plan;
+    const int rc = cached_plan(rows, N, k, eps, recall, &plan);
+    if (rc != PROFK_OK) return rc;
+    return topk_planned<T>(in, rows, N, k, &plan, seed, stream, out_vals, out_idx);
+}
+
+// Flattened BatchTopK: stages 1-3 as in topk_planned (one row), then the kept set without ordering (batchtopk.cuh).
+template <typename T>
+int batchtopk_planned(const T* in, int64_t N, int64_t K, const profk_plan_t* plan, uint64_t seed, void* stream, T* sel_vals,
+                      int64_t* sel_idx, uint32_t* mask, T* dense) {
+    g_launches = 0;
+    if (!in || !plan) return PROFK_EINVAL;
+    if ((sel_vals == nullptr) != (sel_idx == nullptr)) return PROFK_EINVAL;
+    if (!sel_vals && !mask && !dense) return PROFK_EINVAL;
+    if (N < 1 || N > N_MAX || K < 1 || K > N) return PROFK_EINVAL;
+    if (((uintptr_t)in % sizeof(T)) || ((uintptr_t)sel_vals % sizeof(T)) || ((uintptr_t)sel_idx % 8) || ((uintptr_t)mask % 4) ||
+        ((uintptr_t)dense % sizeof(T)))
+        return PROFK_EINVAL;
+    const int64_t capacity = plan->capacity;
+    if (capacity < K || capacity > N) return PROFK_EINVAL;
+    if (plan->mode != 0 && plan->mode != 1) return PROFK_EINVAL;
+    if (plan->tie_rule != PROFK_TIES_KEEP_ALL && plan->tie_rule != PROFK_TIES_BY_INDEX) return PROFK_EINVAL;
+    if (plan->mode == 0) {
+        if (plan->m < 1 || plan->m > std::min<int64_t>(N, M_MAX) || plan->r < 1 || plan->r > plan->m) return PROFK_EINVAL;
+        if (plan->k_accept != K) return PROFK_EINVAL;          // the kept set has exactly K members: no relaxed mode
+    }
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    DeviceInfo di;
+    int rc = ensure_device_info<T>(dev, &di);
+    if (rc != PROFK_OK) return rc;
+    Workspace ws;
     {
         std::lock_guard<std::mutex> lock(g_mutex);
-        const int64_t plan_rows = rows <= GATHER_MAX_ROWS ? 1 : GATHER_MAX_ROWS + 1;     // the two classes the tuning knows
-        const auto key = std::make_tuple(plan_rows, N, k, eps, recall);
-        auto it = g_plan_cache.find(key);
-        if (it == g_plan_cache.end()) {
-            const int rc = profk_plan_batch(plan_rows, N, k, eps, recall, &plan);
-            if (rc != PROFK_OK) return rc;
-            if (g_plan_cache.size() > 4096) g_plan_cache.clear();
-            g_plan_cache[key] = plan;
-        } else {
-            plan = it->second;
-        }
+        ws = g_workspace[dev];
     }
-    return topk_planned<T>(in, rows, N, k, &plan, seed, stream, out_vals, out_idx);
+    const WsLayout lay = ws_layout(1, capacity, K, true);
+    if (!ws.ptr || ws.bytes < lay.total) return PROFK_EWORKSPACE;
+    const uint64_t row_stride = row_stride_for(capacity, true);
+    unsigned char* base = static_cast<unsigned char*>(ws.ptr);
+    WsHeader* header = reinterpret_cast<WsHeader*>(base + lay.off_header);
+    uint32_t* ghist = reinterpret_cast<uint32_t*>(base + lay.off_ghist);
+    RowCtl* ctl = reinterpret_cast<RowCtl*>(base + lay.off_ctl);
+    uint4* thr = reinterpret_cast<uint4*>(base + lay.off_tau);
+    uint64_t* buf = reinterpret_cast<uint64_t*>(base + lay.off_buf);
+    uint32_t* bins = reinterpret_cast<uint32_t*>(base + lay.off_bins);
+    uint32_t* keys_scratch = reinterpret_cast<uint32_t*>(base + lay.off_keys);
+    uint32_t* part_counts = reinterpret_cast<uint32_t*>(base + lay.off_parts);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    const double per_warp_tile = (double)plan->r / (double)std::max<int64_t>(plan->m, 1) * 32.0 * FILTER_UNROLL * Elem<T>::VEC;
+    const bool staged = plan->mode == 0 && per_warp_tile > 2.0;       // as in topk_planned
+    const bool parts = !staged && plan->mode == 0;
+    const uint32_t part_cap = (uint32_t)(row_stride / 2 / FILTER_PARTS);
+
+    if (plan->mode == 0) {
+        rc = launch_sample_select<T>(di, in, 1, N, plan->m, plan->r, seed, nullptr, ctl, header, (uint32_t)capacity, nullptr, keys_scratch,
+                                     parts ? part_counts : nullptr, plan->tie_rule == PROFK_TIES_BY_INDEX, thr, st);
+        if (rc != PROFK_OK) return rc;
+        rc = launch_filter<T>(di, in, 1, N, nullptr, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, &header->tile_counter,
+                              parts, part_cap, part_counts, thr, st);
+        if (rc != PROFK_OK) return rc;
+    } else {
+        init_ctl_kernel<<<1, 256, 0, st>>>(ctl, 1, header, (uint32_t)capacity, (uint32_t)K);
+        CUDA_TRY(cudaGetLastError());
+        ++g_launches;
+    }
+    BatchTopkParams<T> bp;
+    bp.fb.in = in; bp.fb.N = (uint64_t)N; bp.fb.rows = 1; bp.fb.k = (uint32_t)K; bp.fb.capacity = (uint32_t)capacity;
+    bp.fb.ctl = ctl; bp.fb.header = header; bp.fb.ghist = ghist; bp.fb.buf = buf; bp.fb.buf_stride = row_stride; bp.fb.sort_rows = 0;
+    bp.fb.tiles_per_row = tiles_per_row<T>((uint64_t)N, FB_THREADS * FB_UNROLL);
+    bp.fb.use_pdl = 0; bp.fb.out_vals = nullptr; bp.fb.out_idx = nullptr; bp.fb.cta_records = nullptr; bp.fb.cta_counters = nullptr;
+    bp.fb.sort_cap = 0; bp.fb.parallel = 0;
+    bp.bins = bins;
+    bp.seg_totals = ghist;                                        // (the exact selection and the select levels never both run)
+    bp.edge = buf + row_stride / 2;                               // the scratch half of the row's buffer
+    bp.parts = parts ? FILTER_PARTS : 1u; bp.part_cap = part_cap; bp.part_counts = part_counts;
+    bp.sel_vals = sel_vals; bp.sel_idx = sel_idx; bp.mask = mask; bp.dense = dense;
+    bp.use_pdl = 0; bp.direct = plan->mode == 1 ? 1 : 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(std::min<unsigned>((unsigned)di.sm_count, FB_MAX_CTAS));
+    cfg.blockDim = dim3(BK_THREADS);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    return launch_cooperative(cfg, batchtopk_emit_kernel<T>, bp, plan->mode == 0, [](BatchTopkParams<T>& q, int v) { q.use_pdl = v; });
+}
+
+template <typename T>
+int batchtopk_auto(const T* in, int64_t N, int64_t K, double eps, uint64_t seed, void* stream, T* sel_vals, int64_t* sel_idx,
+                   uint32_t* mask, T* dense) {
+    g_launches = 0;
+    profk_plan_t plan;
+    const int rc = cached_plan(1, N, K, eps, 1.0, &plan);
+    if (rc != PROFK_OK) return rc;
+    return batchtopk_planned<T>(in, N, K, &plan, seed, stream, sel_vals, sel_idx, mask, dense);
 }
 
 template <typename T>
@@ -602,7 +711,7 @@ extern "C" {
 int profk_workspace_bytes(int64_t rows, int64_t capacity, int64_t k, size_t* bytes) {
     if (!bytes || rows < 1 || capacity < 1 || k < 1 || capacity < k || capacity > N_MAX || rows * capacity >= (1LL << 40))
         return PROFK_EINVAL;
-    *bytes = ws_layout(rows, capacity, k).total;
+    *bytes = ws_layout(rows, capacity, k, large_selection(rows, k)).total;
     return PROFK_OK;
 }
 
@@ -619,6 +728,34 @@ int profk_set_workspace(void* dev_ptr, size_t bytes) {
 int profk_topk_f32(const float* in, int64_t rows, int64_t N, int64_t k, double eps, double recall, uint64_t seed,
                    void* stream, float* out_vals, int64_t* out_idx) {
     return topk_auto<float>(in, rows, N, k, eps, recall, seed, stream, out_vals, out_idx);
+}
+
+int profk_batchtopk_workspace_bytes(int64_t capacity, int64_t K, size_t* bytes) {
+    if (!bytes || capacity < 1 || K < 1 || capacity < K || capacity > N_MAX) return PROFK_EINVAL;
+    *bytes = ws_layout(1, capacity, K, true).total;
+    return PROFK_OK;
+}
+
+int profk_batchtopk_f32(const float* in, int64_t N, int64_t K, double eps, uint64_t seed, void* stream, float* sel_vals,
+                        int64_t* sel_idx, uint32_t* mask, float* dense) {
+    return batchtopk_auto<float>(in, N, K, eps, seed, stream, sel_vals, sel_idx, mask, dense);
+}
+
+int profk_batchtopk_bf16(const void* in, int64_t N, int64_t K, double eps, uint64_t seed, void* stream, void* sel_vals,
+                         int64_t* sel_idx, uint32_t* mask, void* dense) {
+    return batchtopk_auto<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(in), N, K, eps, seed, stream,
+                                         static_cast<__nv_bfloat16*>(sel_vals), sel_idx, mask, static_cast<__nv_bfloat16*>(dense));
+}
+
+int profk_batchtopk_planned_f32(const float* in, int64_t N, int64_t K, const profk_plan_t* plan, uint64_t seed, void* stream,
+                                float* sel_vals, int64_t* sel_idx, uint32_t* mask, float* dense) {
+    return batchtopk_planned<float>(in, N, K, plan, seed, stream, sel_vals, sel_idx, mask, dense);
+}
+
+int profk_batchtopk_planned_bf16(const void* in, int64_t N, int64_t K, const profk_plan_t* plan, uint64_t seed, void* stream,
+                                 void* sel_vals, int64_t* sel_idx, uint32_t* mask, void* dense) {
+    return batchtopk_planned<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(in), N, K, plan, seed, stream,
+                                            static_cast<__nv_bfloat16*>(sel_vals), sel_idx, mask, static_cast<__nv_bfloat16*>(dense));
 }
 
 int profk_topk_bf16(const void* in, int64_t rows, int64_t N, int64_t k, double eps, double recall, uint64_t seed,
@@ -708,7 +845,7 @@ int profk_topk_noalloc_f32(const float* in, int64_t rows, int64_t N, int64_t k, 
         }
     }
     if (rows * plan.capacity >= (1LL << 40)) return PROFK_EINVAL;
-    if (ws_layout(rows, plan.capacity, k).total > NOALLOC_SCRATCH_BYTES) return PROFK_ETOOLARGE;
+    if (ws_layout(rows, plan.capacity, k, large_selection(rows, k)).total > NOALLOC_SCRATCH_BYTES) return PROFK_ETOOLARGE;
     g_ws_override_ptr = scratch;
     g_ws_override_bytes = NOALLOC_SCRATCH_BYTES;
     const int rc = topk_planned<float>(in, rows, N, k, &plan, seed, stream, out_vals, out_idx);
@@ -726,7 +863,7 @@ int profk_read_stats(void* stream, int64_t rows, profk_row_stats_t* out) {
         std::lock_guard<std::mutex> lock(g_mutex);
         ws = g_workspace[dev];
     }
-    const WsLayout lay = ws_layout(rows, 1, 1);
+    const WsLayout lay = ws_layout(rows, 1, 1, false);
     if (!ws.ptr || ws.bytes < lay.off_ctl + (size_t)rows * sizeof(RowCtl)) return PROFK_EWORKSPACE;
     std::vector<RowCtl> host((size_t)rows);
     WsHeader hdr;

@@ -17,6 +17,7 @@
 // up sets the workspace's error flag and the kernel returns.
 #pragma once
 
+#include "fallback.cuh"
 #include "grid_barrier.cuh"
 #include "refine.cuh"
 
@@ -47,6 +48,10 @@ template <typename T> struct LargeParams {
     T* out_vals;             // rows x k
     int64_t* out_idx;        // rows x k
     int use_pdl;
+    // A single row (fused == 1; one group of CTAs): a row that fails the count check, or a row in direct mode, is replaced
+    // inside this kernel by the grid-wide exact selection and ordered right away -- one launch instead of three.
+    int fused;
+    FallbackParams<T> fb;    // what that selection needs (fused == 1 only)
 };
 
 // All exchanges of the network with stride < BT_TILE, for one tile held in shared memory.
@@ -94,6 +99,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
     pdl_launch_dependents();
     if (p.use_pdl) pdl_wait();
     uint32_t gen = *((volatile uint32_t*)bar_gen);                   // read before this CTA's first arrival
+    uint32_t grid_gen = *((volatile uint32_t*)&p.header->bar_gen);   // the same for the grid-wide barrier of the exact selection
 
     for (uint64_t row = group; row < p.rows; row += p.groups) {
         // ---- is this row for this launch?  (the decision is the same in every CTA) ----
@@ -117,15 +123,24 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
             } else {
                 pcount[0] = R;
             }
-            const uint32_t status = (R > p.capacity || part_full) ? ROW_OVERFLOW : R < p.k_accept ? ROW_RECALL : ROW_OK;
-            if (cta == 0 && tid == 0) {
+            const bool direct = ctl.status == ROW_DIRECT;          // marked by the initialisation kernel: no filter ran
+            const uint32_t status = direct ? ROW_DIRECT : (R > p.capacity || part_full) ? ROW_OVERFLOW : R < p.k_accept ? ROW_RECALL : ROW_OK;
+            if (cta == 0 && tid == 0 && !direct) {
                 if (p.parts > 1) p.ctl[row].count = part_full && R <= p.capacity ? p.capacity + 1 : R;   // what the statistics report
                 p.ctl[row].status = status;
                 p.ctl[row].n_final = status ? p.k : R;
                 if (status) atomicAdd(&p.header->n_failed, 1u);
             }
-            if (status != ROW_OK) continue;      // the exact-selection kernel and the second phase take this row
             n = R;
+            if (status != ROW_OK) {
+                if (!p.fused) continue;          // the exact-selection kernel and the second phase take this row
+                // the k best records of the whole row into the row's buffer, then ordered below like any buffer
+                if (!grid_exact_select_row<T>(p.fb, row, grid_gen, reinterpret_cast<uint32_t*>(tile), s_warp)) return;
+                nparts = 1;
+#pragma unroll
+                for (int j = 0; j < (int)FILTER_PARTS; ++j) pcount[j] = 0;
+                pcount[0] = n = p.k;
+            }
         } else {
             if (ctl.status == ROW_OK) continue;  // already written by the first phase
             n = p.k;                             // the exact selection left exactly k records

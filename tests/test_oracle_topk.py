@@ -109,3 +109,51 @@ def test_checker_accepts_truth_and_rejects_corruptions():
     # duplicate index
     i6 = i.copy(); i6[1] = i6[0]
     assert topk.verify_topk(x, k, x[i6], i6) != []
+
+
+# ----------------------------------------------------------------------------- BatchTopK forms (Section 5, "Application")
+def test_kept_set_equals_brute_force_on_tiny_tied_inputs():
+    rng = np.random.default_rng(11)
+    for n in (1, 2, 7, 33, 64):
+        for trial in range(6):
+            x = rng.integers(0, 4, size=n).astype(np.float32)           # heavy ties
+            if trial == 0:
+                x[:] = 2.0                                               # all equal: the kept set is the first k indices
+            for k in sorted({1, n // 2 or 1, n}):
+                mask = topk.kept_mask(x, k)
+                _, bi = topk.topk_brute(x, k)
+                want = np.zeros(n, dtype=bool)
+                want[bi] = True
+                assert np.array_equal(mask, want), (n, trial, k)
+                if trial == 0:
+                    assert np.array_equal(np.flatnonzero(mask), np.arange(k))
+                # the defining properties: k kept; no dropped entry beats a kept one; ties at the k-th value go to the lowest indices
+                keys = topk.order_key(x).astype(np.int64)
+                assert mask.sum() == k
+                if k < n:
+                    kth = keys[mask].min()
+                    assert keys[~mask].max() <= kth
+                    tied = np.flatnonzero(keys == kth)
+                    n_tied_kept = int(mask[tied].sum())
+                    assert np.array_equal(tied[:n_tied_kept], tied[mask[tied]])
+
+
+def test_kept_dense_and_packed_mask():
+    x = np.array([[0.5, -1.0, 3.0, 0.5], [0.5, 2.0, -0.0, 0.5]], dtype=np.float32)       # a 2 x 4 "activation matrix"
+    dense = topk.kept_dense(x, 4)                                       # top 4 of the 8 flattened entries: 3.0, 2.0, then the two first 0.5
+    assert dense.shape == x.shape
+    assert np.array_equal(dense, np.array([[0.5, 0.0, 3.0, 0.5], [0.0, 2.0, 0.0, 0.0]], dtype=np.float32))
+    assert not np.signbit(dense).any()                                  # dropped entries are +0.0, also where the input held -0.0
+    mask = topk.kept_mask(x, 4)
+    assert np.flatnonzero(mask).tolist() == [0, 2, 3, 5]
+    assert topk.pack_mask(mask).tolist() == [0b101101]
+    # bf16 bit patterns: zero is the all-zero pattern there too
+    xb = np.array([0x3F80, 0x4000, 0xBF80, 0x3F80], dtype=np.uint16)    # 1, 2, -1, 1
+    assert topk.kept_dense(xb, 2).tolist() == [0x3F80, 0x4000, 0, 0]
+    # packing against NumPy's own bit packing (little-endian bit order inside little-endian words)
+    rng = np.random.default_rng(12)
+    for n in (1, 31, 32, 33, 1000):
+        m = rng.random(n) < 0.3
+        padded = np.zeros((n + 31) // 32 * 32, dtype=bool)
+        padded[:n] = m
+        assert np.array_equal(topk.pack_mask(m), np.packbits(padded, bitorder="little").view("<u4"))
