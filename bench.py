@@ -313,6 +313,51 @@ def measure_extra_config(profk, torch, name, dev, peak):
     return res
 
 
+def run_one_row_sharded(args, cfg, profk, sharding, torch, dev, rank, world):
+    """Strong scaling of one long row: every rank holds one shard (drawn on its GPU, seeded by the shard), each step is
+    one `sharding.topk_one_row` call (stage 1, all-gather of the sample keys, stage 2, stage 3, all-gather of the
+    candidate buffers, stage 4).  Timed with CUDA events, max over ranks; each call ends with an 8-byte read of the count
+    check's outcome, which is inside the timed region."""
+    rows, n, dt, recipe, seed, k, eps, recall = cfg
+    assert rows == 1, "--one-row-sharded needs a single-row configuration"
+    elem = 4 if dt == "f32" else 2
+    lo, hi = sharding.shard_layout(n, k, world, eps, recall)[rank]
+    shard_cfg = (1, hi - lo) + tuple(cfg[2:])
+    copies = 2
+    shards = [make_input(shard_cfg, seed_offset=1000 * c + 31 * rank, device=str(dev)).view(-1) for c in range(copies)]
+    gather = sharding.dist_gather(world, rank) if world > 1 else sharding.local_gather(1)
+    warmup, steps = max(args.warmup, 3), args.steps
+
+    def step(i):
+        return sharding.topk_one_row({rank: shards[i % copies]}, world, n, k, eps, recall, seed=i, gather=gather)
+
+    repaired = 0
+    for i in range(warmup):
+        step(i)
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        repaired += int(step(warmup + i)[2]["repaired"])
+    e1.record()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ms = sharding.max_over_ranks(e0.elapsed_time(e1), dev) / steps
+    if rank != 0:
+        return
+    gbs = n * elem / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": "top-k elements/s", "value": n / (ms * 1e-3), "unit": "elements/s", "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": dt, "data": "synthetic",
+        "config": {"workload": describe(args.config, cfg) + f"; ONE row cut into {world} shard(s), one per GPU",
+                   "parallelism": f"{world} shard(s) of one row; two all-gathers per call (sample keys, candidate buffers)"},
+        "extra": {"whole_row_GBps": gbs, "frac_of_8TBps_read_once_per_gpu": gbs / world / 8000.0, "calls_repaired": repaired}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -323,6 +368,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra-configs", action="store_true", help="skip the brief timing of the other configurations")
     ap.add_argument("--blocks", type=int, default=25, help="timed blocks of --steps calls (the first is the headline)")
+    ap.add_argument("--one-row-sharded", action="store_true",
+                    help="strong scaling instead of replicas: ONE row of the configuration's length cut into one shard per GPU "
+                         "(sharding.topk_one_row: two all-gathers per call); with --gpus 1 the same path on a single shard")
     ap.add_argument("--hot-path-only", action="store_true",
                     help="run only warm-up + timed steps of the hot path (for profiler captures) and exit")
     ap.add_argument("--rows", type=int, default=0,
@@ -359,6 +407,11 @@ def main():
     in_bytes = rows * n * elem
     warmup = max(args.warmup, 3)
     steps = args.steps
+    if args.one_row_sharded:
+        run_one_row_sharded(args, cfg, profk, sharding, torch, dev, rank, world)
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # Inputs: enough distinct copies that no step finds its input in L2 (126 MB).
     copies = max(2, min(8, -(-3 * L2_BYTES // in_bytes)))

@@ -277,6 +277,54 @@ int profk_sample_threshold_bf16(const void* in, int64_t rows, int64_t N, int64_t
                                 void* tau, uint32_t* sample_idx, void* stream);
 
 /*
+ * ONE ROW SPLIT OVER SEVERAL GPUS.  The paper runs on a single GPU and leaves distributed settings to future work
+ * (Section "Limitations"); the four stages of Section 3 split at two exchange points, and these stage calls are the
+ * pieces between them.  Every GPU holds a contiguous shard of the row made of whole sampling strata
+ * (profk_shard_bounds), so the sample -- and with it the threshold -- is the one the unsharded call draws for the same
+ * seed.  The caller makes the two exchanges (an all-gather each) into LOCAL buffers; no call here touches another
+ * GPU's memory.  Per row:
+ *   1. profk_shard_sample_keys_*      stage 1 on the shard: the order keys of the samples of its strata
+ *      -> all-gather the m keys (in stratum order)
+ *   2. profk_threshold_from_keys_*    stage 2: the r-th largest sampled record, as a 16-byte threshold record
+ *                                     {bits of tau, bits of the next value up, index of the record or 0xFFFFFFFF, 0}
+ *   3. profk_filter_shard_*           stage 3 on the shard, indices local to the shard; state = 8 uint32 words,
+ *                                     [0] = the shard's survivor count on return (the call zeroes it first)
+ *      -> all-gather (state, records), `capacity` records per shard
+ *   4. profk_refine_gathered_*        the count check on the summed counts and stage 4 on the merged records (global
+ *                                     index = local index + bases[g]); status_out[0] = PROFK_ROW_OK / _RECALL /
+ *                                     _OVERFLOW, status_out[1] = R.  Needs the registered workspace of
+ *                                     profk_workspace_bytes(1, capacity, k).  On a status other than OK the outputs
+ *                                     are not written: the exact replacement needs the whole row, which no single GPU
+ *                                     holds -- the caller repairs the row (e.g. the exact top-k of every shard with
+ *                                     profk_topk_*, gathered and selected from once more).
+ * Arguments: shard [device] the shard's elements, shard_base / shard_len its position in the row of length N;
+ * j_lo, j_hi the shard's strata [j_lo, j_hi) of m (j_lo even; j_hi even or m); keys_out / keys [device] uint32;
+ * thr_record [device] 4 uint32, 16-byte aligned; records [device] uint64; state / states [device] 16-byte aligned;
+ * bases [host] `shards` int64; shards <= 16.  m, r, capacity, k_accept, tie_rule come from profk_plan(N, k, ...).
+ * Errors: PROFK_EINVAL, PROFK_EWORKSPACE, PROFK_ECUDA.
+ */
+int profk_shard_bounds(int64_t N, int64_t m, int64_t shards, int64_t shard,
+                       int64_t* j_lo, int64_t* j_hi, int64_t* elem_lo, int64_t* elem_hi /* [host] out */);
+int profk_shard_sample_keys_f32(const float* shard, int64_t shard_base, int64_t shard_len, int64_t N, int64_t m,
+                                int64_t j_lo, int64_t j_hi, uint64_t seed, uint32_t* keys_out, void* stream);
+int profk_shard_sample_keys_bf16(const void* shard, int64_t shard_base, int64_t shard_len, int64_t N, int64_t m,
+                                 int64_t j_lo, int64_t j_hi, uint64_t seed, uint32_t* keys_out, void* stream);
+int profk_threshold_from_keys_f32(const uint32_t* keys, int64_t N, int64_t m, int64_t r, uint64_t seed, int tie_rule,
+                                  uint32_t* thr_record, void* stream);
+int profk_threshold_from_keys_bf16(const uint32_t* keys, int64_t N, int64_t m, int64_t r, uint64_t seed, int tie_rule,
+                                   uint32_t* thr_record, void* stream);
+int profk_filter_shard_f32(const float* shard, int64_t shard_base, int64_t shard_len, const uint32_t* thr_record,
+                           int64_t capacity, uint64_t* records, uint32_t* state, void* stream);
+int profk_filter_shard_bf16(const void* shard, int64_t shard_base, int64_t shard_len, const uint32_t* thr_record,
+                            int64_t capacity, uint64_t* records, uint32_t* state, void* stream);
+int profk_refine_gathered_f32(const uint64_t* records, const uint32_t* states, const int64_t* bases, int64_t shards,
+                              int64_t shard_capacity, const uint32_t* thr_record, int64_t capacity, int64_t k,
+                              int64_t k_accept, float* out_vals, int64_t* out_idx, uint32_t* status_out, void* stream);
+int profk_refine_gathered_bf16(const uint64_t* records, const uint32_t* states, const int64_t* bases, int64_t shards,
+                               int64_t shard_capacity, const uint32_t* thr_record, int64_t capacity, int64_t k,
+                               int64_t k_accept, void* out_vals, int64_t* out_idx, uint32_t* status_out, void* stream);
+
+/*
  * (This entry point has no counterpart in the paper; it exists for callers that must not
  * allocate.)  Same result as profk_topk_f32, but no workspace has to be registered and the
  * entry point calls no allocator, neither cudaMalloc / cudaFree nor an allocating library

@@ -23,6 +23,9 @@ EXPORTS = [
     "profk_debug_set_prefetch_wait_polls",
     "profk_batchtopk_workspace_bytes", "profk_batchtopk_f32", "profk_batchtopk_bf16", "profk_batchtopk_planned_f32",
     "profk_batchtopk_planned_bf16",
+    "profk_shard_bounds", "profk_shard_sample_keys_f32", "profk_shard_sample_keys_bf16", "profk_threshold_from_keys_f32",
+    "profk_threshold_from_keys_bf16", "profk_filter_shard_f32", "profk_filter_shard_bf16", "profk_refine_gathered_f32",
+    "profk_refine_gathered_bf16",
 ]
 
 ROW_OK, ROW_RECALL, ROW_OVERFLOW, ROW_DIRECT = 0, 1, 2, 3
@@ -296,6 +299,76 @@ def batchtopk(x, k: int, eps: float = 1e-3, seed: int = 0, want_pairs: bool = Tr
                                                                   ptr(dense))
     _check(code, "profk_batchtopk")
     return out
+
+
+# ---- one row over several GPUs: the stage calls (argument marshalling only; sharding.py makes the exchanges) ----
+def shard_bounds(n: int, m: int, shards: int, shard: int) -> tuple[int, int, int, int]:
+    """`profk_shard_bounds`: (j_lo, j_hi, elem_lo, elem_hi) of shard `shard` of `shards`: whole pairs of sampling strata."""
+    out = [ctypes.c_int64() for _ in range(4)]
+    _check(lib().profk_shard_bounds(ctypes.c_int64(n), ctypes.c_int64(m), ctypes.c_int64(shards), ctypes.c_int64(shard),
+                                    *[ctypes.byref(o) for o in out]), "profk_shard_bounds")
+    return tuple(int(o.value) for o in out)
+
+
+def shard_sample_keys(shard, shard_base: int, n: int, m: int, j_lo: int, j_hi: int, seed: int):
+    """`profk_shard_sample_keys_*`: uint32 order keys (as an int32 tensor) of the samples of strata [j_lo, j_hi)."""
+    import torch
+
+    keys = torch.empty(j_hi - j_lo, dtype=torch.int32, device=shard.device)
+    fn = getattr(lib(), f"profk_shard_sample_keys_{_suffix(shard)}")
+    with torch.cuda.device(shard.device):
+        _check(fn(ctypes.c_void_p(shard.data_ptr()), ctypes.c_int64(shard_base), ctypes.c_int64(shard.numel()), ctypes.c_int64(n),
+                  ctypes.c_int64(m), ctypes.c_int64(j_lo), ctypes.c_int64(j_hi), ctypes.c_uint64(seed),
+                  ctypes.c_void_p(keys.data_ptr()), _stream_ptr()), "profk_shard_sample_keys")
+    return keys
+
+
+def threshold_from_keys(keys, dtype, n: int, m: int, r: int, seed: int, tie_rule: int = TIES_BY_INDEX):
+    """`profk_threshold_from_keys_*`: the 4-word threshold record (int32 tensor) from the m gathered keys."""
+    import torch
+
+    thr = torch.empty(4, dtype=torch.int32, device=keys.device)
+    sfx = "f32" if dtype == torch.float32 else "bf16"
+    with torch.cuda.device(keys.device):
+        _check(getattr(lib(), f"profk_threshold_from_keys_{sfx}")(ctypes.c_void_p(keys.data_ptr()), ctypes.c_int64(n), ctypes.c_int64(m),
+                                                                ctypes.c_int64(r), ctypes.c_uint64(seed), ctypes.c_int(tie_rule),
+                                                                ctypes.c_void_p(thr.data_ptr()), _stream_ptr()), "profk_threshold_from_keys")
+    return thr
+
+
+def filter_shard(shard, shard_base: int, thr, capacity: int):
+    """`profk_filter_shard_*`: (records int64 (capacity,), state int32 (8,)) -- indices local to the shard."""
+    import torch
+
+    records = torch.empty(capacity, dtype=torch.int64, device=shard.device)
+    state = torch.empty(8, dtype=torch.int32, device=shard.device)
+    fn = getattr(lib(), f"profk_filter_shard_{_suffix(shard)}")
+    with torch.cuda.device(shard.device):
+        _check(fn(ctypes.c_void_p(shard.data_ptr()), ctypes.c_int64(shard_base), ctypes.c_int64(shard.numel()), ctypes.c_void_p(thr.data_ptr()),
+                  ctypes.c_int64(capacity), ctypes.c_void_p(records.data_ptr()), ctypes.c_void_p(state.data_ptr()), _stream_ptr()),
+               "profk_filter_shard")
+    return records, state
+
+
+def refine_gathered(records, states, bases, thr, dtype, capacity: int, k: int, k_accept: int):
+    """`profk_refine_gathered_*`: records (shards, shard_capacity) int64, states (shards, 8) int32, bases: list of int.
+    Returns (values (k,), indices (k,), status int32 (2,) = [PROFK_ROW_*, R]); nothing is synchronised."""
+    import torch
+
+    shards, shard_cap = records.shape
+    ensure_workspace(1, capacity, k, records.device)
+    vals = torch.empty(k, dtype=dtype, device=records.device)
+    idx = torch.empty(k, dtype=torch.int64, device=records.device)
+    status = torch.empty(2, dtype=torch.int32, device=records.device)
+    arr = (ctypes.c_int64 * shards)(*[int(b) for b in bases])
+    sfx = "f32" if dtype == torch.float32 else "bf16"
+    with torch.cuda.device(records.device):
+        _check(getattr(lib(), f"profk_refine_gathered_{sfx}")(ctypes.c_void_p(records.data_ptr()), ctypes.c_void_p(states.data_ptr()), arr,
+                                                            ctypes.c_int64(shards), ctypes.c_int64(shard_cap), ctypes.c_void_p(thr.data_ptr()),
+                                                            ctypes.c_int64(capacity), ctypes.c_int64(k), ctypes.c_int64(k_accept),
+                                                            ctypes.c_void_p(vals.data_ptr()), ctypes.c_void_p(idx.data_ptr()),
+                                                            ctypes.c_void_p(status.data_ptr()), _stream_ptr()), "profk_refine_gathered")
+    return vals, idx, status
 
 
 def topk_noalloc(x, k: int, eps: float = 1e-3, recall: float = 1.0, seed: int = 0, out=None):

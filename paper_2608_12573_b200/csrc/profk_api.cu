@@ -18,6 +18,7 @@
 #include "refine.cuh"
 #include "refine_large.cuh"
 #include "sample_select.cuh"
+#include "shard.cuh"
 
 using namespace profk;
 
@@ -206,16 +207,17 @@ int pick_cluster(int64_t rows, int64_t m, int max_cluster) {
 template <typename T>
 int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, int64_t m, int64_t r, uint64_t seed, T* tau, RowCtl* ctl,
                          WsHeader* header, uint32_t capacity, uint32_t* sample_idx, uint32_t* keys_scratch, uint32_t* part_counts,
-                         bool by_record, uint4* thr, cudaStream_t st) {
+                         bool by_record, uint4* thr, cudaStream_t st, const uint32_t* keys_given = nullptr) {
     const int csize = pick_cluster(rows, m, di.max_cluster[dtype_index<T>()]);
     // A large sample, or a sample of a very long row (every element on a page of its own), is gathered by a
-    // kernel over all SMs first; the cluster then only selects.
-    const bool spread_gather = keys_scratch != nullptr && rows <= GATHER_MAX_ROWS &&
+    // kernel over all SMs first; the cluster then only selects.  (keys_given: the caller already holds the sample's keys.)
+    const bool spread_gather = !keys_given && keys_scratch != nullptr && rows <= GATHER_MAX_ROWS &&
                                (m > GATHER_MIN_SAMPLE || (int64_t)N * (int64_t)sizeof(T) >= (512LL << 20));
     if (spread_gather) {
         GatherParams<T> gp;
         gp.in = in; gp.N = (uint64_t)N; gp.rows = (uint64_t)rows; gp.S = (uint32_t)m; gp.seed = seed;
         gp.q = (uint64_t)(N / m); gp.rem = (uint32_t)(N % m); gp.inv_s = 1.0f / (float)m; gp.keys_out = keys_scratch;
+        gp.pair_lo = 0; gp.pairs = (uint64_t)((m + 1) / 2); gp.base = 0;
         const int64_t pairs = rows * ((m + 1) / 2);
         cudaLaunchConfig_t gcfg = {};
         gcfg.gridDim = dim3((unsigned)((pairs + GATHER_THREADS - 1) / GATHER_THREADS));
@@ -229,7 +231,7 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
         ++g_launches;
     }
     SelectParams<T> sp;
-    sp.keys_in = spread_gather ? keys_scratch : nullptr;
+    sp.keys_in = keys_given ? keys_given : spread_gather ? keys_scratch : nullptr;
     sp.part_counts = part_counts;
     sp.by_record = by_record ? 1 : 0;
     sp.thr = thr;
@@ -703,6 +705,112 @@ int sample_threshold(const T* in, int64_t rows, int64_t N, int64_t m, int64_t r,
                                    static_cast<cudaStream_t>(stream));
 }
 
+// ---- one row over several GPUs: the stage calls (shard.cuh) ----
+
+// floor(j * N / m) on the host, as the kernels compute it.
+int64_t stratum_start_host(int64_t j, int64_t N, int64_t m) { return (int64_t)(((unsigned __int128)j * (unsigned __int128)N) / (unsigned __int128)m); }
+
+template <typename T>
+int shard_sample_keys(const T* shard, int64_t shard_base, int64_t shard_len, int64_t N, int64_t m, int64_t j_lo, int64_t j_hi, uint64_t seed,
+                      uint32_t* keys_out, void* stream) {
+    if (!shard || !keys_out) return PROFK_EINVAL;
+    if (N < 1 || N > N_MAX || m < 1 || m > std::min<int64_t>(N, M_MAX) || shard_len < 1 || shard_base < 0 || shard_base + shard_len > N) return PROFK_EINVAL;
+    if (j_lo < 0 || j_hi <= j_lo || j_hi > m || (j_lo & 1) || ((j_hi & 1) && j_hi != m)) return PROFK_EINVAL;      // whole pairs of strata
+    if (stratum_start_host(j_lo, N, m) < shard_base || stratum_start_host(j_hi, N, m) > shard_base + shard_len) return PROFK_EINVAL;
+    if ((uintptr_t)shard % sizeof(T) || (uintptr_t)keys_out % 4) return PROFK_EINVAL;
+    GatherParams<T> gp;
+    gp.in = shard; gp.N = (uint64_t)N; gp.rows = 1; gp.S = (uint32_t)m; gp.seed = seed;
+    gp.q = (uint64_t)(N / m); gp.rem = (uint32_t)(N % m); gp.inv_s = 1.0f / (float)m; gp.keys_out = keys_out;
+    gp.pair_lo = (uint64_t)(j_lo / 2); gp.pairs = (uint64_t)((j_hi - j_lo + 1) / 2); gp.base = (uint64_t)shard_base;
+    gather_kernel<T><<<(unsigned)((gp.pairs + GATHER_THREADS - 1) / GATHER_THREADS), GATHER_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(gp);
+    CUDA_TRY(cudaGetLastError());
+    return PROFK_OK;
+}
+
+template <typename T>
+int threshold_from_keys(const uint32_t* keys, int64_t N, int64_t m, int64_t r, uint64_t seed, int tie_rule, uint32_t* thr_record, void* stream) {
+    if (!keys || !thr_record) return PROFK_EINVAL;
+    if (N < 1 || N > N_MAX || m < 1 || m > std::min<int64_t>(N, M_MAX) || r < 1 || r > m) return PROFK_EINVAL;
+    if (tie_rule != PROFK_TIES_KEEP_ALL && tie_rule != PROFK_TIES_BY_INDEX) return PROFK_EINVAL;
+    if ((uintptr_t)keys % 4 || (uintptr_t)thr_record % 16) return PROFK_EINVAL;
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    DeviceInfo di;
+    const int rc = ensure_device_info<T>(dev, &di);
+    if (rc != PROFK_OK) return rc;
+    return launch_sample_select<T>(di, nullptr, 1, N, m, r, seed, nullptr, nullptr, nullptr, 0, nullptr, nullptr, nullptr,
+                                   tie_rule == PROFK_TIES_BY_INDEX, reinterpret_cast<uint4*>(thr_record), static_cast<cudaStream_t>(stream), keys);
+}
+
+template <typename T>
+int filter_shard(const T* shard, int64_t shard_base, int64_t shard_len, const uint32_t* thr_record, int64_t capacity, uint64_t* records,
+                 uint32_t* state, void* stream) {
+    if (!shard || !thr_record || !records || !state) return PROFK_EINVAL;
+    if (shard_len < 1 || shard_base < 0 || shard_base + shard_len > N_MAX || capacity < 1 || capacity > N_MAX) return PROFK_EINVAL;
+    if ((uintptr_t)shard % sizeof(T) || (uintptr_t)thr_record % 16 || (uintptr_t)records % 8 || (uintptr_t)state % 16) return PROFK_EINVAL;
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    DeviceInfo di;
+    const int rc = ensure_device_info<T>(dev, &di);
+    if (rc != PROFK_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    localize_threshold_kernel<<<1, 32, 0, st>>>(reinterpret_cast<const uint4*>(thr_record), (unsigned long long)shard_base,
+                                                (unsigned long long)shard_len, state);
+    CUDA_TRY(cudaGetLastError());
+    return launch_filter<T>(di, shard, 1, shard_len, nullptr, capacity, records, (uint64_t)capacity, state, 1, false, false, nullptr, false, 0u,
+                            nullptr, reinterpret_cast<const uint4*>(state + 4), st);
+}
+
+template <typename T>
+int refine_gathered(const uint64_t* records, const uint32_t* states, const int64_t* bases, int64_t shards, int64_t shard_capacity,
+                    const uint32_t* thr_record, int64_t capacity, int64_t k, int64_t k_accept, T* out_vals, int64_t* out_idx,
+                    uint32_t* status_out, void* stream) {
+    g_launches = 0;
+    if (!records || !states || !bases || !thr_record || !out_vals || !out_idx || !status_out) return PROFK_EINVAL;
+    if (shards < 1 || shards > SHARD_MAX || shard_capacity < 1 || capacity < k || k < 1 || k_accept < 1 || k_accept > k || capacity > N_MAX) return PROFK_EINVAL;
+    if ((uintptr_t)records % 8 || (uintptr_t)states % 16 || (uintptr_t)thr_record % 16 || (uintptr_t)out_vals % sizeof(T) || (uintptr_t)out_idx % 8 ||
+        (uintptr_t)status_out % 4)
+        return PROFK_EINVAL;
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    DeviceInfo di;
+    int rc = ensure_device_info<T>(dev, &di);
+    if (rc != PROFK_OK) return rc;
+    Workspace ws;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        ws = g_workspace[dev];
+    }
+    const bool large = large_selection(1, k);
+    const WsLayout lay = ws_layout(1, capacity, k, large);
+    if (!ws.ptr || ws.bytes < lay.total) return PROFK_EWORKSPACE;
+    const uint64_t row_stride = row_stride_for(capacity, large);
+    unsigned char* base = static_cast<unsigned char*>(ws.ptr);
+    WsHeader* header = reinterpret_cast<WsHeader*>(base + lay.off_header);
+    uint32_t* ghist = reinterpret_cast<uint32_t*>(base + lay.off_ghist);
+    RowCtl* ctl = reinterpret_cast<RowCtl*>(base + lay.off_ctl);
+    uint64_t* buf = reinterpret_cast<uint64_t*>(base + lay.off_buf);
+    uint32_t* bins = reinterpret_cast<uint32_t*>(base + lay.off_bins);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    ShardBases sb = {};
+    for (int64_t g = 0; g < shards; ++g) {
+        if (bases[g] < 0 || bases[g] > N_MAX) return PROFK_EINVAL;
+        sb.base[g] = bases[g];
+    }
+    merge_shards_kernel<<<di.sm_count, 256, 0, st>>>(records, states, sb, (uint32_t)shards, (uint32_t)std::min<int64_t>(shard_capacity, 0xFFFFFFFFll),
+                                                     (uint32_t)capacity, (uint32_t)k, (uint32_t)k_accept, reinterpret_cast<const uint4*>(thr_record),
+                                                     buf, ctl, header, status_out);
+    CUDA_TRY(cudaGetLastError());
+    ++g_launches;
+    // The ordinary count check and refinement of one row.  A row that fails the check is left alone here (its exact
+    // replacement needs the whole row, which no single GPU holds): the caller reads status_out and repairs it.
+    if (large)
+        return launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, reinterpret_cast<unsigned long long*>(ghist), false, 0u, nullptr, 1,
+                                      capacity, k, k_accept, 0, out_vals, out_idx, st);
+    return launch_refine<T>(di, static_cast<const T*>(nullptr), 1, 1, ctl, header, buf, row_stride, capacity, k, k_accept, false, 1, nullptr, nullptr,
+                            out_vals, out_idx, st);
+}
+
 }  // namespace
 
 // --------------------------------------------------------------------------------------- C ABI
@@ -852,6 +960,52 @@ int profk_topk_noalloc_f32(const float* in, int64_t rows, int64_t N, int64_t k, 
     g_ws_override_ptr = nullptr;
     g_ws_override_bytes = 0;
     return rc;
+}
+
+int profk_shard_bounds(int64_t N, int64_t m, int64_t shards, int64_t shard, int64_t* j_lo, int64_t* j_hi, int64_t* elem_lo, int64_t* elem_hi) {
+    if (!j_lo || !j_hi || !elem_lo || !elem_hi) return PROFK_EINVAL;
+    if (N < 1 || N > N_MAX || m < 1 || m > std::min<int64_t>(N, M_MAX) || shards < 1 || shards > SHARD_MAX || shard < 0 || shard >= shards) return PROFK_EINVAL;
+    const int64_t pairs = (m + 1) / 2;                    // strata travel in pairs (one Philox block serves two)
+    if (pairs < shards) return PROFK_EINVAL;
+    const int64_t lo = 2 * (pairs * shard / shards), hi = shard + 1 == shards ? m : 2 * (pairs * (shard + 1) / shards);
+    *j_lo = lo; *j_hi = hi;
+    *elem_lo = stratum_start_host(lo, N, m);
+    *elem_hi = stratum_start_host(hi, N, m);
+    return PROFK_OK;
+}
+
+int profk_shard_sample_keys_f32(const float* shard, int64_t shard_base, int64_t shard_len, int64_t N, int64_t m, int64_t j_lo, int64_t j_hi,
+                                uint64_t seed, uint32_t* keys_out, void* stream) {
+    return shard_sample_keys<float>(shard, shard_base, shard_len, N, m, j_lo, j_hi, seed, keys_out, stream);
+}
+int profk_shard_sample_keys_bf16(const void* shard, int64_t shard_base, int64_t shard_len, int64_t N, int64_t m, int64_t j_lo, int64_t j_hi,
+                                 uint64_t seed, uint32_t* keys_out, void* stream) {
+    return shard_sample_keys<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(shard), shard_base, shard_len, N, m, j_lo, j_hi, seed, keys_out, stream);
+}
+int profk_threshold_from_keys_f32(const uint32_t* keys, int64_t N, int64_t m, int64_t r, uint64_t seed, int tie_rule, uint32_t* thr_record, void* stream) {
+    return threshold_from_keys<float>(keys, N, m, r, seed, tie_rule, thr_record, stream);
+}
+int profk_threshold_from_keys_bf16(const uint32_t* keys, int64_t N, int64_t m, int64_t r, uint64_t seed, int tie_rule, uint32_t* thr_record, void* stream) {
+    return threshold_from_keys<__nv_bfloat16>(keys, N, m, r, seed, tie_rule, thr_record, stream);
+}
+int profk_filter_shard_f32(const float* shard, int64_t shard_base, int64_t shard_len, const uint32_t* thr_record, int64_t capacity,
+                           uint64_t* records, uint32_t* state, void* stream) {
+    return filter_shard<float>(shard, shard_base, shard_len, thr_record, capacity, records, state, stream);
+}
+int profk_filter_shard_bf16(const void* shard, int64_t shard_base, int64_t shard_len, const uint32_t* thr_record, int64_t capacity,
+                            uint64_t* records, uint32_t* state, void* stream) {
+    return filter_shard<__nv_bfloat16>(static_cast<const __nv_bfloat16*>(shard), shard_base, shard_len, thr_record, capacity, records, state, stream);
+}
+int profk_refine_gathered_f32(const uint64_t* records, const uint32_t* states, const int64_t* bases, int64_t shards, int64_t shard_capacity,
+                              const uint32_t* thr_record, int64_t capacity, int64_t k, int64_t k_accept, float* out_vals, int64_t* out_idx,
+                              uint32_t* status_out, void* stream) {
+    return refine_gathered<float>(records, states, bases, shards, shard_capacity, thr_record, capacity, k, k_accept, out_vals, out_idx, status_out, stream);
+}
+int profk_refine_gathered_bf16(const uint64_t* records, const uint32_t* states, const int64_t* bases, int64_t shards, int64_t shard_capacity,
+                               const uint32_t* thr_record, int64_t capacity, int64_t k, int64_t k_accept, void* out_vals, int64_t* out_idx,
+                               uint32_t* status_out, void* stream) {
+    return refine_gathered<__nv_bfloat16>(records, states, bases, shards, shard_capacity, thr_record, capacity, k, k_accept,
+                                          static_cast<__nv_bfloat16*>(out_vals), out_idx, status_out, stream);
 }
 
 int profk_read_stats(void* stream, int64_t rows, profk_row_stats_t* out) {

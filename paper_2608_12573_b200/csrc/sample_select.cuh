@@ -105,8 +105,8 @@ template <typename T>
 __device__ __forceinline__ void publish_threshold(const SelectParams<T>& p, uint64_t row, uint32_t tau_key, uint32_t j) {
     const T tau = Elem<T>::from_key(tau_key);
     if (p.tau) p.tau[row] = tau;
-    if (p.ctl) {
-        p.ctl[row].tau_bits = Elem<T>::bits(tau);
+    if (p.ctl || p.thr) {
+        if (p.ctl) p.ctl[row].tau_bits = Elem<T>::bits(tau);
         uint32_t idx = 0xFFFFFFFFu;
         if (p.by_record) {
             const Philox4 r = philox4x32_10(j >> 1, (uint32_t)row, (uint32_t)(row >> 32), 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32));
@@ -115,7 +115,7 @@ __device__ __forceinline__ void publish_threshold(const SelectParams<T>& p, uint
             const uint64_t u = (j & 1u) ? (((uint64_t)r.w << 32) | r.z) : (((uint64_t)r.y << 32) | r.x);
             idx = (uint32_t)(b0 + __umul64hi(u, b1 - b0));
         }
-        p.ctl[row].tau_idx = idx;
+        if (p.ctl) p.ctl[row].tau_idx = idx;
         if (p.thr) {
             const uint32_t top = Elem<T>::KEY_BITS == 32 ? 0xFFFFFFFFu : 0xFFFFu;
             const uint32_t next_key = tau_key == top ? tau_key : tau_key + 1u;
@@ -162,18 +162,23 @@ template <typename T> struct GatherParams {
     uint64_t q;            // N / S
     uint32_t rem;          // N % S
     float inv_s;           // 1 / S
-    uint32_t* keys_out;    // rows x S
+    uint32_t* keys_out;    // rows x S (a shard: the keys of its strata only, pairs * 2 of them)
+    // A shard of one row (the whole row: pair_lo = 0, pairs = ceil(S / 2), base = 0): `in` points at element `base` of the
+    // row and the kernel takes strata 2 * pair_lo ... 2 * (pair_lo + pairs) - 1, all of which lie inside the shard.
+    uint64_t pair_lo;
+    uint64_t pairs;
+    uint64_t base;
 };
 
 template <typename T>
 __global__ void __launch_bounds__(GATHER_THREADS) gather_kernel(const GatherParams<T> p) {
-    const uint64_t pairs = ((uint64_t)p.S + 1) / 2;
+    const uint64_t pairs = p.pairs;
     const uint64_t g = (uint64_t)blockIdx.x * GATHER_THREADS + threadIdx.x;
     const bool active = g < p.rows * pairs;
     const uint64_t row = active ? g / pairs : 0;
-    const uint64_t j = active ? 2 * (g % pairs) : 0;                 // even sample of the pair
+    const uint64_t j = active ? 2 * (p.pair_lo + g % pairs) : 0;     // even sample of the pair
     const bool second = active && j + 1 < p.S;
-    const T* rowp = p.in + row * p.N;
+    const T* rowp = p.in + row * p.N - p.base;
     uint32_t idx0 = 0, idx1 = 0;
     if (active) {
         const Philox4 r = philox4x32_10((uint32_t)(j >> 1), (uint32_t)row, (uint32_t)(row >> 32), 0u,
@@ -195,7 +200,7 @@ __global__ void __launch_bounds__(GATHER_THREADS) gather_kernel(const GatherPara
     if (active) {
         const T v0 = rowp[idx0];
         const T v1 = second ? rowp[idx1] : v0;
-        uint32_t* out = p.keys_out + row * p.S + j;
+        uint32_t* out = p.keys_out + row * p.S + (j - 2 * p.pair_lo);
         out[0] = Elem<T>::key(v0);
         if (second) out[1] = Elem<T>::key(v1);
     }
