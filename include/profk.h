@@ -70,7 +70,10 @@ enum {
     PROFK_ROW_OK = 0,       /* k_accept <= R <= capacity: answer refined from the buffer   */
     PROFK_ROW_RECALL = 1,   /* R < k_accept: too few candidates, exact selection ran       */
     PROFK_ROW_OVERFLOW = 2, /* R > capacity: buffer overflowed, exact selection ran        */
-    PROFK_ROW_DIRECT = 3    /* plan mode 1: exact selection without sampling or filtering  */
+    PROFK_ROW_DIRECT = 3,   /* plan mode 1: exact selection without sampling or filtering  */
+    PROFK_ROW_RECALL_REFILTERED = 4,   /* R < k_accept, then k <= R' <= capacity with the looser rank r_loose:
+                                          answer refined from the second filtering pass (tau, R report that pass) */
+    PROFK_ROW_OVERFLOW_REFILTERED = 5  /* R > capacity, then k <= R' <= capacity with the tighter rank r_tight */
 };
 
 /* How the filter of stage 3 treats copies of the threshold value (profk_plan_t.tie_rule).
@@ -103,6 +106,17 @@ enum {
  *   tie_rule  PROFK_TIES_*; profk_plan and profk_plan_ex set PROFK_TIES_BY_INDEX.
  *   z, alpha  Algorithm 1's z = 2 Phi^{-1}(1 - eps/2) and alpha = k / N.
  *   p_recall_fail, p_overflow   the two bounds for the returned (m, r, capacity).
+ *   r_tight, r_loose   second-chance ranks (0 = none).  Section 3, "Refinement", sends a row that fails the count
+ *             check to an exact top-k of the full input; the appendix ("Fallback as a Safety Mechanism") argues
+ *             that this is rare enough not to matter.  It is also avoidable most of the time: the sample is still
+ *             there, so after an overflow the row is filtered once more with the threshold of the TIGHTER rank
+ *             r_tight < r, after a recall failure with that of the LOOSER rank r_loose > r, into the same buffer
+ *             with the same check k <= R <= M -- one more read of the row at streaming speed -- and only a row
+ *             that fails again is selected exactly.  The ranks aim midway between k and M:
+ *             r_tight = floor(r (k + M) / (2 M)), r_loose = r + ceil((M - k) m / (2 N)).  Used for calls of up
+ *             to 18 rows with k <= 16384 (<= 8192 for up to four rows), where the exact selection runs inside
+ *             the refine kernel, and only when the sample's keys are kept (up to four rows, or m <= 32768);
+ *             other shapes go straight to the exact selection.
  * Both bounds are binomial tail bounds valid for the stratified sampler the
  * library uses (one uniform draw from each of m equal strata of the row).
  */
@@ -117,6 +131,8 @@ typedef struct profk_plan {
     double alpha;
     double p_recall_fail;
     double p_overflow;
+    int64_t r_tight;
+    int64_t r_loose;
 } profk_plan_t;
 
 /* Tuning inputs of Algorithm 1.  The paper's values (Section 4) are

@@ -153,6 +153,8 @@ class Plan:
     alpha: float
     p_recall_fail: float  # bound on Pr(R < k_accept) for (m, r)
     p_overflow: float     # bound on Pr(R > capacity) for (m, r)
+    r_tight: int = 0      # second-chance rank after an overflow (0 = none), see second_chance_ranks
+    r_loose: int = 0      # second-chance rank after a recall failure (0 = none)
 
 
 def accept_count(k: int, recall: float) -> int:
@@ -186,6 +188,20 @@ def guarded_capacity(N: int, S: int, t: int, k: int, eps_b: float) -> int:
     return lo
 
 
+def second_chance_ranks(N: int, k: int, S: int, t: int, capacity: int) -> tuple[int, int]:
+    """Ranks for one more filtering pass before the exact fallback (a reading: Section 3, "Refinement", and the
+    appendix "Fallback as a Safety Mechanism" only say that a failed row falls back to an exact top-k of the input).
+
+    The sample outlives the failure.  Seen from a threshold of rank t that kept just over M elements, the threshold of
+    a tighter rank t' keeps about M t'/t of them (the sampled ranks below a given one are spread like uniform order
+    statistics); aiming midway between k and M gives r_tight = floor(t (k + M) / (2 M)).  Seen from one that kept just
+    under k, each further sample rank adds about N/S survivors; midway again: r_loose = t + ceil((M - k) S / (2 N)).
+    A rank that does not exist (r_tight < 1 or not below t; r_loose above S or not above t) is reported as 0."""
+    tight = t * (k + capacity) // (2 * capacity)
+    loose = t + -(-((capacity - k) * S) // (2 * N))
+    return (tight if 1 <= tight < t else 0), (loose if t < loose <= S else 0)
+
+
 def plan_guarded(N: int, k: int, eps: float = EPS_DEFAULT, recall: float = 1.0,
                  s_min: int = S_MIN_DEFAULT, s_max: int = S_MAX_DEFAULT,
                  cost_ratio: float = COST_RATIO_DEFAULT) -> Plan:
@@ -200,6 +216,7 @@ def plan_guarded(N: int, k: int, eps: float = EPS_DEFAULT, recall: float = 1.0,
     m_paper = math.ceil(eq_M(N, k, S, z))
     capacity = min(N, max(m_exact, m_paper))
     mode = 1 if (2 * capacity >= N or N <= 2 * S) else 0
+    r_tight, r_loose = second_chance_ranks(N, k, S, t, capacity)
     return Plan(m=S, r=t, capacity=capacity, k_accept=k_acc, mode=mode, z=z, alpha=k / N,
                 p_recall_fail=rank_law.p_recall_fail_bound(N, S, t, k_acc),
-                p_overflow=rank_law.p_overflow_bound(N, S, t, capacity))
+                p_overflow=rank_law.p_overflow_bound(N, S, t, capacity), r_tight=r_tight, r_loose=r_loose)

@@ -29,6 +29,14 @@ are distinct, so R is the rank of the threshold record among all records of the 
 Lemma 1's law holds for any input, ties included; on rows without ties at tau nothing
 changes.
 
+Second chance before the exact fallback (`r_tight`, `r_loose`; a reading of "Refinement": the
+paper sends a failed row straight to an exact top-k of the full input): the sample is still there,
+so a row whose buffer overflowed is filtered once more with the threshold of the tighter sample rank
+r_tight, a row with too few candidates with that of the looser rank r_loose -- same buffer, same
+tie rule, and the check k <= R' <= M (the full k also in relaxed mode).  If it passes, the answer is
+refined from that pass (it is the same exact top-k) and the status says so; if not, or if the plan
+names no such rank (0), the exact top-k of the whole row replaces it as before.
+
 Status codes mirror the library's per-row statistics.
 
 Pins (tests/test_oracle_stages.py): whenever k <= R <= M the refined answer
@@ -48,6 +56,8 @@ STATUS_OK = 0            # k_accept <= R <= M: answer came from the buffer
 STATUS_RECALL = 1        # R < k_accept: fewer candidates than needed -> exact selection
 STATUS_OVERFLOW = 2      # R > M: buffer too small -> exact selection
 STATUS_DIRECT = 3        # plan mode 1: exact selection without sampling
+STATUS_RECALL_REFILTERED = 4      # R < k_accept, then k <= R' <= M under the looser rank: answer from the second pass
+STATUS_OVERFLOW_REFILTERED = 5    # R > M, then k <= R' <= M under the tighter rank: answer from the second pass
 
 
 @dataclass
@@ -96,27 +106,37 @@ def survivor_set_record(x: np.ndarray, tau, tau_idx: int) -> np.ndarray:
     return np.flatnonzero((keys > tk) | ((keys == tk) & (np.arange(x.shape[0]) <= tau_idx)))
 
 
+def _filter_with_rank(x: np.ndarray, s_idx: np.ndarray, rank: int, composite: bool):
+    """Stages 2 and 3 for one sample rank: (tau, indices kept)."""
+    if composite:
+        tau, tau_idx = threshold_record(x, s_idx, rank)              # stage 2, on records
+        return tau, survivor_set_record(x, tau, tau_idx)             # stage 3, tie-proof
+    tau = threshold(x, s_idx, rank)                                  # stage 2
+    return tau, survivor_set(x, tau)                                 # stage 3
+
+
 def run_row(x: np.ndarray, k: int, m: int, r: int, capacity: int, k_accept: int,
-            seed: int, row: int = 0, mode: int = 0, composite: bool = False) -> StageResult:
-    """All four stages on one row with an explicit plan (m, r, capacity, k_accept)."""
+            seed: int, row: int = 0, mode: int = 0, composite: bool = False,
+            r_tight: int = 0, r_loose: int = 0) -> StageResult:
+    """All four stages on one row with an explicit plan (m, r, capacity, k_accept[, r_tight, r_loose])."""
     n = x.shape[0]
     if mode == 1:
         vals, idx = topk.topk_row(x, k)
         return StageResult(np.empty(0, np.int64), None, 0, STATUS_DIRECT, vals, idx)
     s_idx = philox.sample_indices(n, m, seed, row)                  # stage 1
-    if composite:
-        tau, tau_idx = threshold_record(x, s_idx, r)                 # stage 2, on records
-        kept = survivor_set_record(x, tau, tau_idx)                  # stage 3, tie-proof
-    else:
-        tau = threshold(x, s_idx, r)                                 # stage 2
-        kept = survivor_set(x, tau)                                  # stage 3
+    tau, kept = _filter_with_rank(x, s_idx, r, composite)            # stages 2 and 3
     R = int(kept.size)
-    if R > capacity:                                                 # stage 4, failure branches
+    if R > capacity or R < k_accept:                                 # stage 4, failure branches
+        failed = STATUS_OVERFLOW if R > capacity else STATUS_RECALL
+        second = r_tight if R > capacity else r_loose
+        if second:                                                   # one more filtering pass with the other rank
+            tau2, kept2 = _filter_with_rank(x, s_idx, second, composite)
+            if k <= kept2.size <= capacity:
+                bvals, bpos = topk.topk_row(x[kept2], k)
+                status = STATUS_OVERFLOW_REFILTERED if failed == STATUS_OVERFLOW else STATUS_RECALL_REFILTERED
+                return StageResult(s_idx, tau2, int(kept2.size), status, bvals, kept2[bpos].astype(np.int64))
         vals, idx = topk.topk_row(x, k)
-        return StageResult(s_idx, tau, R, STATUS_OVERFLOW, vals, idx)
-    if R < k_accept:
-        vals, idx = topk.topk_row(x, k)
-        return StageResult(s_idx, tau, R, STATUS_RECALL, vals, idx)
+        return StageResult(s_idx, tau, R, failed, vals, idx)
     kk = min(k, R)                                                   # stage 4 on the buffer
     bvals, bpos = topk.topk_row(x[kept], kk)
     vals = np.empty(k, dtype=x.dtype)

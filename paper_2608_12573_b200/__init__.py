@@ -29,6 +29,7 @@ EXPORTS = [
 ]
 
 ROW_OK, ROW_RECALL, ROW_OVERFLOW, ROW_DIRECT = 0, 1, 2, 3
+ROW_RECALL_REFILTERED, ROW_OVERFLOW_REFILTERED = 4, 5    # repaired by a second filtering pass (plan.r_loose / plan.r_tight)
 TIES_KEEP_ALL, TIES_BY_INDEX = 0, 1      # profk_plan_t.tie_rule: the filter as printed / the threshold as a (value, index) record
 
 
@@ -40,7 +41,8 @@ class _PlanStruct(ctypes.Structure):
     _fields_ = [("m", ctypes.c_int64), ("r", ctypes.c_int64), ("capacity", ctypes.c_int64),
                 ("k_accept", ctypes.c_int64), ("mode", ctypes.c_int32), ("tie_rule", ctypes.c_int32),
                 ("z", ctypes.c_double), ("alpha", ctypes.c_double),
-                ("p_recall_fail", ctypes.c_double), ("p_overflow", ctypes.c_double)]
+                ("p_recall_fail", ctypes.c_double), ("p_overflow", ctypes.c_double),
+                ("r_tight", ctypes.c_int64), ("r_loose", ctypes.c_int64)]
 
 
 class _TuningStruct(ctypes.Structure):
@@ -64,10 +66,12 @@ class Plan:
     p_recall_fail: float = 0.0
     p_overflow: float = 0.0
     tie_rule: int = TIES_BY_INDEX
+    r_tight: int = 0      # second-chance ranks: 0 = none (a row that fails the count check is selected exactly at once)
+    r_loose: int = 0
 
     def _struct(self) -> _PlanStruct:
         return _PlanStruct(self.m, self.r, self.capacity, self.k_accept, self.mode, self.tie_rule,
-                           self.z, self.alpha, self.p_recall_fail, self.p_overflow)
+                           self.z, self.alpha, self.p_recall_fail, self.p_overflow, self.r_tight, self.r_loose)
 
 
 def lib() -> ctypes.CDLL:
@@ -132,7 +136,7 @@ def _plan_uncached(N, k, eps, recall, s_min, s_max, cost_ratio, rows) -> Plan:
                                    ctypes.c_double(recall), ctypes.byref(tun), ctypes.byref(out))
     _check(code, "profk_plan")
     return Plan(out.m, out.r, out.capacity, out.k_accept, out.mode, out.z, out.alpha,
-                out.p_recall_fail, out.p_overflow, out.tie_rule)
+                out.p_recall_fail, out.p_overflow, out.tie_rule, out.r_tight, out.r_loose)
 
 
 def workspace_bytes(rows: int, capacity: int, k: int) -> int:

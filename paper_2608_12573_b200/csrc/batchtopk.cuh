@@ -85,7 +85,7 @@ __device__ __forceinline__ void bk_zero_fill(E* p, uint64_t n, uint64_t gid, uin
 template <typename T>
 __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const BatchTopkParams<T> p) {
     __shared__ SelectShared sh;                  // hist / start / warp_sums serve the scans here and the exact selection
-    __shared__ uint32_t s_seg, s_seg_before, s_bin, s_bin_before, s_bin_count, s_base;
+    __shared__ uint32_t s_seg, s_seg_before, s_bin, s_bin_before, s_bin_count;
     __shared__ uint32_t s_warp_count[BK_THREADS / 32];
 
     const unsigned tid = threadIdx.x, lane = lane_id(), warp = tid >> 5;

@@ -151,6 +151,12 @@ extern "C" int profk_plan_ex(int64_t N, int64_t k, double eps, double recall, co
     out->alpha = alpha;
     out->p_recall_fail = recall_fail_bound(N, S, t, k_acc);
     out->p_overflow = overflow_bound(N, S, t, capacity);
+    // Second-chance ranks (see profk_plan_t): the sample ranks whose expected survivor count lies midway between k and
+    // the capacity, seen from a threshold that kept just too many (tight) or just too few (loose).
+    const int64_t tight = (int64_t)(((__int128)t * (__int128)(k + capacity)) / ((__int128)2 * capacity));
+    out->r_tight = (tight >= 1 && tight < t) ? tight : 0;
+    const int64_t loose = t + (int64_t)((((__int128)(capacity - k) * (__int128)S) + (__int128)2 * N - 1) / ((__int128)2 * N));
+    out->r_loose = (loose > t && loose <= S) ? loose : 0;
     return PROFK_OK;
 }
 

@@ -50,6 +50,7 @@ constexpr unsigned REFINE_CLUSTER_THREADS = 512;   // fewest threads of a refine
 constexpr size_t REFINE_SMEM_MAX = 160 * 1024;   // dynamic shared memory the refine kernel may ask for (it has ~41 KB static)
 constexpr int64_t N_MAX = 4278190080LL;          // 2^32 - 2^24
 constexpr int64_t M_MAX = 262144;                // largest sample the cluster select holds (8 CTAs x 32768 keys)
+constexpr int64_t KEPT_SAMPLE_MAX = 32768;       // largest sample whose keys are kept for a second filtering pass when there are more than GATHER_MAX_ROWS rows
 
 thread_local int g_launches = 0;
 thread_local void* g_ws_override_ptr = nullptr;   // set by the allocation-free entry point for the duration of its call
@@ -76,7 +77,7 @@ std::map<std::tuple<int64_t, int64_t, int64_t, double, double>, profk_plan_t> g_
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-    size_t off_header, off_ghist, off_ctl, off_tau, off_bins, off_xs_counters, off_xs_records, off_keys, off_fb_counters, off_fb_records, off_parts, off_buf, total;
+    size_t off_header, off_ghist, off_ctl, off_tau, off_tau2, off_bins, off_xs_counters, off_xs_records, off_keys, off_fb_counters, off_fb_records, off_parts, off_buf, total;
 };
 
 // Records reserved per row: the capacity itself, or -- when k is too large for the single-CTA
@@ -96,7 +97,8 @@ WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k, bool large) {
     l.off_ghist = sizeof(WsHeader);
     l.off_ctl = align_up(l.off_ghist + (size_t)FB_PASSES * FB_BINS * sizeof(uint32_t), 256);
     l.off_tau = align_up(l.off_ctl + (size_t)rows * sizeof(RowCtl), 256);
-    l.off_bins = align_up(l.off_tau + (size_t)rows * sizeof(uint4), 256);
+    l.off_tau2 = align_up(l.off_tau + (size_t)rows * sizeof(uint4), 256);       // threshold records of a second filtering pass
+    l.off_bins = align_up(l.off_tau2 + (size_t)rows * sizeof(uint4), 256);
     const size_t bins_bytes = large ? (size_t)rows * (LG_BINS + 8) * sizeof(uint32_t) : 0;
     // scratch of the in-refine exact selection (few rows, k within the single-CTA refine): up to
     // XS_MAX_SEGMENTS segments in all, each with a counter and k + XS_EDGE records
@@ -107,7 +109,10 @@ WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k, bool large) {
     l.off_keys = align_up(l.off_xs_records + (xs ? (size_t)XS_MAX_SEGMENTS * (size_t)(k + XS_EDGE) * sizeof(uint64_t) : 0), 256);
     // scratch of the grid-wide exact selection when it deals failed rows out one per CTA (many rows only)
     const bool fbp = rows > XS_MAX_ROWS && !large;
-    l.off_fb_counters = align_up(l.off_keys + (rows <= GATHER_MAX_ROWS ? (size_t)rows * (size_t)M_MAX * sizeof(uint32_t) : 0), 256);
+    // (up to GATHER_MAX_ROWS rows: room for the largest sample; up to XS_MAX_ROWS rows: for samples up to KEPT_SAMPLE_MAX,
+    // kept for the second filtering pass of a row that fails the count check)
+    const size_t keys_per_row = rows <= GATHER_MAX_ROWS ? (size_t)M_MAX : xs ? (size_t)KEPT_SAMPLE_MAX : 0;
+    l.off_fb_counters = align_up(l.off_keys + (size_t)rows * keys_per_row * sizeof(uint32_t), 256);
     l.off_fb_records = align_up(l.off_fb_counters + (fbp ? FB_MAX_CTAS * sizeof(uint32_t) : 0), 256);
     // counters of the partitioned append (large selections only), each in a 256-byte line of its own
     l.off_parts = align_up(l.off_fb_records + (fbp ? (size_t)FB_MAX_CTAS * (size_t)(k + XS_EDGE) * sizeof(uint64_t) : 0), 256);
@@ -207,7 +212,7 @@ int pick_cluster(int64_t rows, int64_t m, int max_cluster) {
 template <typename T>
 int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, int64_t m, int64_t r, uint64_t seed, T* tau, RowCtl* ctl,
                          WsHeader* header, uint32_t capacity, uint32_t* sample_idx, uint32_t* keys_scratch, uint32_t* part_counts,
-                         bool by_record, uint4* thr, cudaStream_t st, const uint32_t* keys_given = nullptr) {
+                         bool by_record, uint4* thr, cudaStream_t st, const uint32_t* keys_given = nullptr, uint32_t* keys_store = nullptr) {
     const int csize = pick_cluster(rows, m, di.max_cluster[dtype_index<T>()]);
     // A large sample, or a sample of a very long row (every element on a page of its own), is gathered by a
     // kernel over all SMs first; the cluster then only selects.  (keys_given: the caller already holds the sample's keys.)
@@ -232,6 +237,7 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
     }
     SelectParams<T> sp;
     sp.keys_in = keys_given ? keys_given : spread_gather ? keys_scratch : nullptr;
+    sp.keys_store = sp.keys_in ? nullptr : keys_store;       // (keys gathered by the kernel before are in memory already)
     sp.part_counts = part_counts;
     sp.by_record = by_record ? 1 : 0;
     sp.thr = thr;
@@ -378,7 +384,8 @@ template <typename T> int refine_cluster_size(const DeviceInfo& di, int64_t rows
 template <typename T>
 int launch_refine(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, RowCtl* ctl, WsHeader* header, uint64_t* buf,
                   uint64_t row_stride, int64_t capacity, int64_t k, int64_t k_accept, bool direct, int csize, uint64_t* xs_records,
-                  uint32_t* xs_counters, T* out_vals, int64_t* out_idx, cudaStream_t st) {
+                  uint32_t* xs_counters, T* out_vals, int64_t* out_idx, cudaStream_t st, const SampleInfo* sample = nullptr,
+                  uint4* thr2 = nullptr) {
     uint32_t sort_cap = 32;
     while (sort_cap < (uint32_t)k && sort_cap < SORT_CAP_MAX) sort_cap <<= 1;
     RefineParams<T> rp;
@@ -402,6 +409,8 @@ int launch_refine(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, Ro
     }
     rp.clusters_per_row = (uint32_t)nseg;
     rp.xs_records = xs_records; rp.xs_counters = xs_counters;
+    rp.sample = sample ? *sample : SampleInfo{};
+    rp.thr2 = thr2;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(rows * nseg * csize));
     cfg.blockDim = dim3(threads);
@@ -440,6 +449,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     if (plan->mode == 0) {
         if (plan->m < 1 || plan->m > std::min<int64_t>(N, M_MAX) || plan->r < 1 || plan->r > plan->m) return PROFK_EINVAL;
         if (plan->k_accept < 1 || plan->k_accept > k) return PROFK_EINVAL;
+        if (plan->r_tight < 0 || plan->r_tight > plan->m || plan->r_loose < 0 || plan->r_loose > plan->m) return PROFK_EINVAL;
     }
 
     int dev = 0;
@@ -490,6 +500,19 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     uint32_t fb_sort_cap = 32;
     while (fb_sort_cap < (uint32_t)k && fb_sort_cap < SORT_CAP_MAX) fb_sort_cap <<= 1;
 
+    // A second filtering pass for rows that fail the count check (plan->r_tight / r_loose) needs the sample's keys: they
+    // are kept when the refine kernel's clusters do the repair and the workspace has room for them.
+    const bool keep_keys = exact_in_refine && plan->mode == 0 && (plan->r_tight > 0 || plan->r_loose > 0) &&
+                           (rows <= GATHER_MAX_ROWS || plan->m <= KEPT_SAMPLE_MAX);
+    SampleInfo sample = {};
+    if (keep_keys) {
+        sample.keys = keys_scratch; sample.S = (uint32_t)plan->m; sample.seed = seed;
+        sample.q = (uint64_t)(N / plan->m); sample.rem = (uint32_t)(N % plan->m); sample.inv_s = 1.0f / (float)plan->m;
+        sample.by_record = plan->tie_rule == PROFK_TIES_BY_INDEX ? 1 : 0;
+        sample.r_tight = (uint32_t)plan->r_tight; sample.r_loose = (uint32_t)plan->r_loose;
+    }
+    uint4* thr2 = reinterpret_cast<uint4*>(base + lay.off_tau2);
+
     // What the grid-wide exact selection needs (the kernel of its own, or the large refine when it does that itself).
     FallbackParams<T> fb;
     fb.in = in; fb.N = (uint64_t)N; fb.rows = (uint64_t)rows; fb.k = (uint32_t)k;
@@ -509,7 +532,8 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
 
     if (plan->mode == 0) {
         rc = launch_sample_select<T>(di, in, rows, N, plan->m, plan->r, seed, nullptr, ctl, header, (uint32_t)capacity, nullptr,
-                                     rows <= GATHER_MAX_ROWS ? keys_scratch : nullptr, parts ? part_counts : nullptr, plan->tie_rule == PROFK_TIES_BY_INDEX, thr, st);
+                                     rows <= GATHER_MAX_ROWS ? keys_scratch : nullptr, parts ? part_counts : nullptr, plan->tie_rule == PROFK_TIES_BY_INDEX, thr, st,
+                                     nullptr, keep_keys ? keys_scratch : nullptr);
         if (rc != PROFK_OK) return rc;
         rc = launch_filter<T>(di, in, rows, N, nullptr, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, &header->tile_counter,
                               parts, part_cap, part_counts, thr, st);
@@ -521,7 +545,8 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
             if (fused_large) return rc;
         } else {
             // count check and refine; with clusters, also the exact selection of the rows that fail the check
-            rc = launch_refine<T>(di, in, rows, N, ctl, header, buf, row_stride, capacity, k, plan->k_accept, false, csize, xs_records, xs_counters, out_vals, out_idx, st);
+            rc = launch_refine<T>(di, in, rows, N, ctl, header, buf, row_stride, capacity, k, plan->k_accept, false, csize, xs_records, xs_counters, out_vals, out_idx, st,
+                                  keep_keys ? &sample : nullptr, thr2);
         }
         if (rc != PROFK_OK) return rc;
     } else {

@@ -19,6 +19,7 @@
 #pragma once
 
 #include "exact_select.cuh"
+#include "second_chance.cuh"
 #include "select_sort.cuh"
 
 namespace profk {
@@ -28,7 +29,7 @@ template <typename T> struct RefineParams {
     uint64_t N;
     RowCtl* ctl;
     WsHeader* header;
-    const uint64_t* buf;     // row r's records start at buf + r * buf_stride
+    uint64_t* buf;           // row r's records start at buf + r * buf_stride
     uint64_t buf_stride;
     uint32_t capacity;
     uint32_t k;
@@ -44,6 +45,8 @@ template <typename T> struct RefineParams {
     uint32_t clusters_per_row;   // segments a failed row is cut into for its exact selection, one cluster each
     uint64_t* xs_records;    // rows x clusters_per_row x (k + XS_EDGE) records selected from the segments
     uint32_t* xs_counters;   // rows x clusters_per_row append counters
+    SampleInfo sample;       // the kept sample and the second-chance ranks (sample.keys == null: none; clusters only)
+    uint4* thr2;             // rows threshold records of the second filtering pass
 };
 
 // Records selected from the segments of a row, read through L2 (other clusters wrote them); unused
@@ -88,14 +91,96 @@ __device__ __forceinline__ void finish_from_segments(const uint64_t* recs, uint3
 // Cluster `seg` of the row's clusters selects the k smallest records (and a few more) of its segment of
 // the row; the cluster that finishes last merges: the k smallest of all segments' records, ordered, are
 // the row's output.  The ticket is the row's `collect` word, zero on entry and zero again on exit.
+// The second chance (second_chance.cuh) of a row that failed the count check, run by all clusters of the row, each over
+// its own segment: the threshold of the plan's tighter (after an overflow) or looser (after too few candidates) sample
+// rank is selected from the kept keys -- by every CTA for itself, nobody waits for anybody -- the segment is filtered with
+// it into the row's buffer (counter: the row's `pad` word), and the cluster that finishes last takes the check
+// k <= R' <= M on the new count.  Returns, the same in every CTA of a cluster: 0 = not the last cluster, or the last one
+// and the row is answered (by its first CTA, from the buffer); 2 = the last cluster and the check failed again.
 template <typename T>
-__device__ __noinline__ void exact_row(const RefineParams<T>& p, uint64_t row, unsigned seg, unsigned crank, uint64_t* sortbuf,
-                                       SelectShared& sh, bool overflowed, uint32_t tau_key) {
+__device__ __noinline__ int second_chance_row(const RefineParams<T>& p, uint64_t row, unsigned seg, unsigned crank, uint32_t rung,
+                                              uint32_t failed_status, uint64_t* sortbuf, SelectShared& sh) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
     const unsigned tid = threadIdx.x, nthr = blockDim.x;
     const unsigned csize = p.cluster_size, nseg = p.clusters_per_row;
+    const SampleInfo& sm = p.sample;
+    uint32_t key2, j2;
+    kth_sample_record<T>(sm.keys + row * sm.S, sm.S, rung, sh, &key2, &j2);
+    const uint32_t idx2 = sm.by_record ? sample_element_index(j2, row, sm.seed, sm.q, sm.rem, sm.S, sm.inv_s) : 0xFFFFFFFFu;
+    const T tau2 = Elem<T>::from_key(key2);
+    if (tid == 0) {                              // (every CTA of the row writes the same sixteen bytes)
+        const uint32_t top = Elem<T>::KEY_BITS == 32 ? 0xFFFFFFFFu : 0xFFFFu;
+        p.thr2[row] = make_uint4(Elem<T>::bits(tau2), Elem<T>::bits(Elem<T>::from_key(key2 == top ? key2 : key2 + 1u)), idx2, 0u);
+    }
+    __syncthreads();
+
+    FilterParams<T> fp = {};
+    fp.in = p.in; fp.N = p.N; fp.rows = row + 1; fp.tau = nullptr; fp.capacity = p.capacity;
+    fp.buf = p.buf; fp.buf_stride = p.buf_stride;
+    fp.counts = &p.ctl[0].pad; fp.count_stride = sizeof(RowCtl) / 4;
+    fp.thr = p.thr2;
     const uint64_t tiles = tiles_per_row<T>(p.N, nthr * XS_UNROLL);
     const uint64_t seg_lo = tiles * seg / nseg, seg_hi = tiles * (seg + 1) / nseg;
+    if (nthr == 512) refilter_tiles<T, 512>(fp, (uint32_t)row, seg_lo, seg_hi, crank, csize, tau2);
+    else refilter_tiles<T, 1024>(fp, (uint32_t)row, seg_lo, seg_hi, crank, csize, tau2);
+    __threadfence();
+    cluster.sync();                              // the whole cluster's records and counts are out
+
+    // the last cluster to get here sees all of them
+    if (crank == 0 && tid == 0) {
+        const uint32_t ticket = atomicAdd(&p.ctl[row].collect, 1u);
+        uint32_t decision = 0;
+        if (ticket == nseg - 1) {
+            p.ctl[row].collect = 0;
+            __threadfence();
+            const uint32_t R2 = __ldcg(&p.ctl[row].pad);
+            decision = (R2 >= p.k && R2 <= p.capacity) ? 1u : 2u;
+            if (decision == 1u) {
+                p.ctl[row].status = failed_status == ROW_OVERFLOW ? ROW_OVERFLOW_REFILTERED : ROW_RECALL_REFILTERED;
+                p.ctl[row].count = R2;
+                p.ctl[row].tau_bits = Elem<T>::bits(tau2);
+                p.ctl[row].tau_idx = idx2;
+            }
+        }
+        sh.crowded = decision;
+    }
+    cluster.sync();
+    const uint32_t decision = *cluster.map_shared_rank(&sh.crowded, 0);
+    cluster.sync();                              // the first CTA's word has been read by all: it may go on
+    if (decision == 1u && crank == 0) {
+        const uint32_t R2 = __ldcg(&p.ctl[row].count);
+        finish_from_segments<T>(p.buf + row * p.buf_stride, R2, p.k, p.sort_cap, sortbuf, sh, row, p.out_vals, p.out_idx);
+    }
+    return decision == 2u ? 2 : 0;
+}
+
+// The exact top-k of the full row, for a row that failed the count check (Section 3, "Refinement").
+// Cluster `seg` of the row's clusters selects the k smallest records (and a few more) of its segment of
+// the row; the cluster that finishes last merges: the k smallest of all segments' records, ordered, are
+// the row's output.  The ticket is the row's `collect` word, zero on entry and zero again on exit.
+// When the plan names a second-chance rank for this kind of failure and the sample was kept, that comes first; the
+// exact selection then runs only if the second pass fails too, by the one cluster that found out, over the whole row.
+template <typename T>
+__device__ __noinline__ void exact_row(const RefineParams<T>& p, uint64_t row, unsigned seg, unsigned crank, uint64_t* sortbuf,
+                                       SelectShared& sh, uint32_t status, uint32_t tau_key) {
+    const unsigned tid = threadIdx.x, nthr = blockDim.x;
+    const unsigned csize = p.cluster_size, nseg = p.clusters_per_row;
+    const bool overflowed = status == ROW_OVERFLOW;
+    const uint64_t tiles = tiles_per_row<T>(p.N, nthr * XS_UNROLL);
     const uint32_t slots = p.k + XS_EDGE;                // per segment: a superset of its k smallest records
+    const uint32_t rung = status == ROW_OVERFLOW ? p.sample.r_tight : status == ROW_RECALL ? p.sample.r_loose : 0u;
+    if (rung != 0 && p.sample.keys != nullptr && csize > 1 && (nthr == 512 || nthr == 1024)) {
+        if (second_chance_row<T>(p, row, seg, crank, rung, status, sortbuf, sh) != 2) return;
+        // failed again: this cluster alone selects from the whole row, into its own scratch
+        const uint64_t* mine = p.xs_records + (row * nseg + seg) * (uint64_t)slots;
+        exact_select_cluster<T>(p.in, p.N, row, p.k, 0, tiles, p.xs_records + (row * nseg + seg) * (uint64_t)slots,
+                                p.xs_counters + row * nseg + seg, sh, csize, crank, false, 0u);
+        if (crank != 0) return;
+        finish_from_segments<T>(mine, slots, p.k, p.sort_cap, sortbuf, sh, row, p.out_vals, p.out_idx);
+        return;
+    }
+    const uint64_t seg_lo = tiles * seg / nseg, seg_hi = tiles * (seg + 1) / nseg;
     const uint64_t* recs = p.xs_records + (row * nseg) * (uint64_t)slots;
     exact_select_cluster<T>(p.in, p.N, row, p.k, seg_lo, seg_hi, p.xs_records + (row * nseg + seg) * (uint64_t)slots,
                             p.xs_counters + row * nseg + seg, sh, csize, crank, overflowed, tau_key);
@@ -170,7 +255,7 @@ __global__ void __maxnreg__(MAXREG) refine_kernel(const __grid_constant__ Refine
     }
     if (status != ROW_OK) {
         if (csize == 1) return;              // the exact-selection kernel that follows takes this row
-        exact_row<T>(p, row, seg, crank, sortbuf, sh, status == ROW_OVERFLOW, Elem<T>::key(Elem<T>::from_bits(ctl.tau_bits)));
+        exact_row<T>(p, row, seg, crank, sortbuf, sh, status, Elem<T>::key(Elem<T>::from_bits(ctl.tau_bits)));
         return;
     }
     if (!refiner) return;

@@ -45,7 +45,7 @@ struct RowCtl {
     uint32_t n_final;    // records the refine step has to order
     uint32_t capacity;
     uint32_t tau_idx;    // index of the threshold record; 0xFFFFFFFF = the threshold is the value alone
-    uint32_t pad;
+    uint32_t pad;        // survivors appended by a second filtering pass (second_chance.cuh)
 };
 static_assert(sizeof(RowCtl) == 32, "RowCtl is 32 bytes");
 
@@ -84,6 +84,7 @@ template <typename T> struct SelectParams {
     const uint32_t* keys_in;   // null, or rows x S keys of the sample gathered by gather_kernel before this one
     uint32_t* part_counts;     // null, or the counters of the partitioned append (FILTER_PARTS per row, FILTER_PART_STRIDE words apart) to reset with the row's
     int by_record;             // 1 = the threshold is the t-th sampled record (value descending, index ascending), 0 = its value
+    uint32_t* keys_store;      // null, or rows x S: the sample's keys are kept here for a second filtering pass (when this kernel gathers them itself)
 };
 
 // floor(j * N / S) = j * (N / S) + floor(j * (N % S) / S).  The second quotient is below S
@@ -98,6 +99,15 @@ __device__ __forceinline__ uint64_t stratum_start(uint64_t j, uint64_t q, uint32
     return j * q + (uint64_t)e;
 }
 
+// Element index of sample j of `row`: the Philox draw of stratum j again (one block serves samples 2p and 2p + 1).
+__device__ __forceinline__ uint32_t sample_element_index(uint32_t j, uint64_t row, uint64_t seed, uint64_t q, uint32_t rem, uint32_t S, float inv_s) {
+    const Philox4 r = philox4x32_10(j >> 1, (uint32_t)row, (uint32_t)(row >> 32), 0u, (uint32_t)seed, (uint32_t)(seed >> 32));
+    const uint64_t b0 = stratum_start(j, q, rem, S, inv_s);
+    const uint64_t b1 = stratum_start((uint64_t)j + 1, q, rem, S, inv_s);
+    const uint64_t u = (j & 1u) ? (((uint64_t)r.w << 32) | r.z) : (((uint64_t)r.y << 32) | r.x);
+    return (uint32_t)(b0 + __umul64hi(u, b1 - b0));
+}
+
 // Writes tau for one row: the key of the threshold and the number j of the sample that holds it.  Samples are
 // stratified, so among samples "smaller index" and "smaller sample number" are the same order; the element
 // index of sample j is drawn again here by the one thread that publishes.
@@ -108,13 +118,7 @@ __device__ __forceinline__ void publish_threshold(const SelectParams<T>& p, uint
     if (p.ctl || p.thr) {
         if (p.ctl) p.ctl[row].tau_bits = Elem<T>::bits(tau);
         uint32_t idx = 0xFFFFFFFFu;
-        if (p.by_record) {
-            const Philox4 r = philox4x32_10(j >> 1, (uint32_t)row, (uint32_t)(row >> 32), 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32));
-            const uint64_t b0 = stratum_start(j, p.q, p.rem, p.S, p.inv_s);
-            const uint64_t b1 = stratum_start((uint64_t)j + 1, p.q, p.rem, p.S, p.inv_s);
-            const uint64_t u = (j & 1u) ? (((uint64_t)r.w << 32) | r.z) : (((uint64_t)r.y << 32) | r.x);
-            idx = (uint32_t)(b0 + __umul64hi(u, b1 - b0));
-        }
+        if (p.by_record) idx = sample_element_index(j, row, p.seed, p.q, p.rem, p.S, p.inv_s);
         if (p.ctl) p.ctl[row].tau_idx = idx;
         if (p.thr) {
             const uint32_t top = Elem<T>::KEY_BITS == 32 ? 0xFFFFFFFFu : 0xFFFFu;
@@ -297,6 +301,7 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
                 const uint32_t local = 2 * pp + (s & 1);
                 const uint32_t k = Elem<T>::key(val[s]);
                 keys[local] = k;
+                if (p.keys_store) p.keys_store[row * p.S + j0 + local] = k;
                 my_max = max(my_max, k);
                 if (p.sample_idx) p.sample_idx[row * p.S + j0 + local] = idx[s];
             }
@@ -311,7 +316,7 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
     if (crank == 0 && tid == 0) {
         if (p.ctl) {
             RowCtl* c = p.ctl + row;
-            c->count = 0; c->collect = 0; c->status = 0; c->n_final = 0; c->capacity = p.capacity;
+            c->count = 0; c->collect = 0; c->status = 0; c->n_final = 0; c->capacity = p.capacity; c->pad = 0;
             if (p.part_counts)
                 for (int j = 0; j < (int)FILTER_PARTS; ++j) p.part_counts[(row * FILTER_PARTS + j) * FILTER_PART_STRIDE] = 0;
         }

@@ -14,7 +14,7 @@ constexpr int RF_BITS = 12;                 // digit width of the general select
 constexpr int RF_BINS = 1 << RF_BITS;
 constexpr uint32_t RF_EDGE_CAP = 1024;      // boundary bins up to this size are ranked directly
 
-enum : uint32_t { ROW_OK = 0, ROW_RECALL = 1, ROW_OVERFLOW = 2, ROW_DIRECT = 3 };
+enum : uint32_t { ROW_OK = 0, ROW_RECALL = 1, ROW_OVERFLOW = 2, ROW_DIRECT = 3, ROW_RECALL_REFILTERED = 4, ROW_OVERFLOW_REFILTERED = 5 };
 
 __device__ __forceinline__ uint64_t shr64(uint64_t x, int s) { return s >= 64 ? 0ull : (x >> s); }
 

@@ -1,0 +1,132 @@
+"""The second filtering pass before the exact fallback (profk_plan_t.r_tight / r_loose): a row that fails the count
+check is filtered once more with the threshold of a tighter or looser sample rank; only if that fails too is it
+selected exactly.  Outputs are bit-exact either way; status, threshold and survivor count follow the oracle's run of
+the same stages (oracle/stages.py)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_12573_b200 as profk
+from oracle import stages as o_stages
+from oracle import topk as o_topk
+from paper_2608_12573_b200 import _build, workloads
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    _build.build()
+    profk.lib()
+    torch.cuda.set_device(0)
+
+
+def bits(a):
+    return a.view(np.uint32) if a.dtype == np.float32 else a.view(np.uint16)
+
+
+def check(x, k, pl, seed, want_status=None):
+    """One call under plan `pl`: exact output, and per-row status / tau / R equal to the oracle's."""
+    v, i = profk.topk(x.cuda(), k, plan_override=pl, seed=seed)
+    torch.cuda.synchronize()
+    xn = workloads.as_numpy(x)
+    xn2 = xn[None, :] if xn.ndim == 1 else xn
+    ov, oi = o_topk.topk(xn2, k)
+    assert np.array_equal(i.cpu().numpy().reshape(ov.shape[0], k), oi), "indices differ from the oracle"
+    assert np.array_equal(bits(workloads.as_numpy(v)).reshape(ov.shape[0], k), bits(ov)), "values differ from the oracle"
+    stats = profk.read_stats(xn2.shape[0])
+    for r in range(xn2.shape[0]):
+        res = o_stages.run_row(xn2[r], k, pl.m, pl.r, pl.capacity, pl.k_accept, seed=seed, row=r, composite=pl.tie_rule == profk.TIES_BY_INDEX,
+                               r_tight=pl.r_tight, r_loose=pl.r_loose)
+        tau_bits, R, cap, status = stats[r]
+        assert status == res.status, (r, status, res.status)
+        assert tau_bits == int(bits(np.asarray([res.tau]))[0]), r
+        assert R == res.survivors or (res.survivors > cap and R > cap), (r, R, res.survivors)
+        if want_status is not None:
+            assert status == want_status, (r, status)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("rows,n", [(1, 1 << 22), (3, 1_000_003), (12, 300_001)])
+def test_overflow_then_the_tighter_rank(dtype, rows, n):
+    x = workloads.normal(rows, n, seed=80, dtype=dtype)
+    k = 64
+    m, r = 4096, 40                                                           # about 40 n / 4096 survivors
+    cap = 25 * n // 4096                                                      # too small for them, enough for rank 20
+    check(x, k, profk.Plan(m=m, r=r, capacity=cap, k_accept=k, mode=0, r_tight=20), seed=1, want_status=profk.ROW_OVERFLOW_REFILTERED)
+    # a rank that is hardly tighter overflows again: the exact selection answers
+    check(x, k, profk.Plan(m=m, r=r, capacity=cap, k_accept=k, mode=0, r_tight=39), seed=1, want_status=profk.ROW_OVERFLOW)
+    # no tighter rank named: as before
+    check(x, k, profk.Plan(m=m, r=r, capacity=cap, k_accept=k, mode=0), seed=1, want_status=profk.ROW_OVERFLOW)
+    # the filter as printed (value-only threshold) takes the same route
+    check(x, k, profk.Plan(m=m, r=r, capacity=cap, k_accept=k, mode=0, r_tight=20, tie_rule=profk.TIES_KEEP_ALL), seed=2)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("rows,n", [(1, 1 << 22), (4, 1_000_003), (9, 300_001)])
+def test_recall_failure_then_the_looser_rank(dtype, rows, n):
+    x = workloads.normal(rows, n, seed=81, dtype=dtype)
+    k = 1000
+    m = 32768                                                                 # rank 1: about n / 32768 survivors, far fewer than k
+    cap = 5 * k
+    loose = -(-5 * k * m // (2 * n))                                          # about 2.5 k survivors expected
+    check(x, k, profk.Plan(m=m, r=1, capacity=cap, k_accept=k, mode=0, r_loose=loose), seed=3, want_status=profk.ROW_RECALL_REFILTERED)
+    check(x, k, profk.Plan(m=m, r=1, capacity=cap, k_accept=k, mode=0, r_loose=2), seed=3, want_status=profk.ROW_RECALL)
+    check(x, k, profk.Plan(m=m, r=1, capacity=cap, k_accept=k, mode=0), seed=3, want_status=profk.ROW_RECALL)
+
+
+def test_ties_and_special_values_in_the_second_pass():
+    n, k = 1 << 21, 200
+    rows = {"constant": torch.full((n,), 3.0), "few values": workloads.few_values(n, seed=82, distinct=4),
+            "relu bf16": workloads.relu_gaussian(n, seed=83, dtype=torch.bfloat16)}
+    special = workloads.normal(1, n, seed=84)[0]
+    special[::1000] = float("nan")
+    special[1::1000] = -float("nan")
+    special[2::3000] = float("inf")
+    special[3::5000] = -0.0
+    rows["special"] = special
+    for name, x in rows.items():
+        for rule in (profk.TIES_BY_INDEX, profk.TIES_KEEP_ALL):
+            check(x, k, profk.Plan(m=4096, r=60, capacity=40 * n // 4096, k_accept=k, mode=0, r_tight=25, tie_rule=rule), seed=4)
+            check(x, k, profk.Plan(m=65536, r=1, capacity=20_000, k_accept=k, mode=0, r_loose=200, tie_rule=rule), seed=5)
+
+
+def test_the_librarys_own_plan_names_the_ranks_and_larger_samples_of_many_rows_skip_them():
+    pl = profk.plan(1 << 26, 256, 1e-4)
+    assert 0 < pl.r_tight < pl.r < pl.r_loose
+    # more than four rows and a sample above 32768: the keys are not kept, the exact selection answers at once
+    x = workloads.normal(6, 1 << 20, seed=85)
+    pl = profk.Plan(m=65536, r=640, capacity=8000, k_accept=64, mode=0, r_tight=320)
+    v, i = profk.topk(x.cuda(), 64, plan_override=pl, seed=6)
+    torch.cuda.synchronize()
+    ov, oi = o_topk.topk(workloads.as_numpy(x), 64)
+    assert np.array_equal(i.cpu().numpy(), oi) and np.array_equal(bits(v.cpu().numpy()), bits(ov))
+    assert all(s[3] == profk.ROW_OVERFLOW for s in profk.read_stats(6))
+
+
+def test_a_billion_element_row_overflows_and_is_repaired_in_one_more_scan():
+    n, k = 1 << 30, 64
+    xd = workloads.cauchy(n, 4, device="cuda")
+    xn = xd.cpu().numpy()
+    keys = o_topk.order_key(xn)
+    pl = profk.plan(n, k, 1e-3)
+    tight = profk.Plan(m=pl.m, r=8 * pl.r, capacity=pl.capacity, k_accept=k, mode=0, r_tight=pl.r)      # rank 8 t overflows M, rank t fits
+    v, i = profk.topk(xd, k, plan_override=tight, seed=7)
+    torch.cuda.synchronize()
+    assert o_topk.verify_topk(xn, k, v.cpu().numpy(), i.cpu().numpy(), keys=keys) == []
+    assert profk.read_stats(1)[0][3] == profk.ROW_OVERFLOW_REFILTERED
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    times = {}
+    for name, plan in (("second pass", tight), ("exact selection", profk.Plan(m=pl.m, r=8 * pl.r, capacity=pl.capacity, k_accept=k, mode=0))):
+        for _ in range(2):
+            profk.topk(xd, k, plan_override=plan, seed=7)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(5):
+            profk.topk(xd, k, plan_override=plan, seed=7)
+        e1.record()
+        torch.cuda.synchronize()
+        times[name] = e0.elapsed_time(e1) / 5
+    print("forced overflow at 2^30, ms per call:", times)
+    assert times["second pass"] < 0.6 * times["exact selection"]

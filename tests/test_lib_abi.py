@@ -56,6 +56,7 @@ def test_host_plan_equals_oracle_plan(lib, N, k, eps, recall, tuning):
         got = profk.plan(N, k, eps, recall, rows=rows)
         want = oracle_plan.plan_guarded(N, k, eps, recall, s_min=s_min, s_max=s_max, cost_ratio=ratio)
     assert (got.m, got.r, got.capacity, got.k_accept, got.mode) == (want.m, want.r, want.capacity, want.k_accept, want.mode)
+    assert (got.r_tight, got.r_loose) == (want.r_tight, want.r_loose)
     assert got.z == pytest.approx(want.z, rel=1e-12)
     assert got.alpha == want.alpha
     assert got.p_recall_fail == pytest.approx(want.p_recall_fail, rel=1e-6, abs=1e-300)

@@ -183,3 +183,23 @@ def test_relaxed_mode_and_direct_mode():
     assert plan.plan_guarded(2 ** 20, 64, 1e-3).mode == 0
     with pytest.raises(ValueError):
         plan.plan_guarded(10, 11)
+
+
+@pytest.mark.parametrize("N,k,eps", SHAPES)
+def test_second_chance_ranks_aim_between_k_and_the_capacity(N, k, eps):
+    """The ranks of the second filtering pass: integers on either side of t whose survivor counts, by Lemma 1's mean
+    E[R] = (N+1) r / (S+1), lie inside [k, M] -- a second pass that starts from there can pass the check."""
+    p = plan.plan_guarded(N, k, eps)
+    tight, loose = plan.second_chance_ranks(N, k, p.m, p.r, p.capacity)
+    assert (p.r_tight, p.r_loose) == (tight, loose)
+    assert tight == 0 or 1 <= tight < p.r
+    assert loose == 0 or p.r < loose <= p.m
+    assert tight == p.r * (k + p.capacity) // (2 * p.capacity) or tight == 0
+    if tight:
+        assert k <= rank_law.nhg_mean(N, p.m, tight) * 1.0 or tight == 1          # mean count of the tighter rank is not below k ...
+        assert rank_law.nhg_mean(N, p.m, tight) <= p.capacity                      # ... and fits the buffer
+    if loose:
+        mean = rank_law.nhg_mean(N, p.m, loose)
+        assert k <= mean <= p.capacity + N / p.m                                   # within one stratum of the buffer at most
+    if p.r == 1:
+        assert tight == 0                                                          # nothing is tighter than the sample maximum

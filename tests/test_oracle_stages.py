@@ -171,3 +171,44 @@ def test_filter_comparison_is_the_total_order_on_zeros_and_nans():
         assert np.array_equal(res.idx, i)
         statuses.add(res.status)
     assert stages.STATUS_RECALL in statuses
+
+
+# ----------------------------------------------------------------------------- second chance before the exact fallback
+def test_second_chance_ranks_and_the_second_filtering_pass_by_hand():
+    """A row built by hand, N = 64, sample of S = 16 (one index per stratum of four).  The thresholds of the three
+    ranks are read off the sorted sample, the survivor counts by counting, and the branch taken follows from them."""
+    from oracle import philox
+    rng = np.random.default_rng(21)
+    x = rng.permutation(64).astype(np.float32)                       # distinct values 0..63
+    s_idx = philox.sample_indices(64, 16, seed=9, row=0)
+    sample_desc = np.sort(x[s_idx])[::-1]
+    count = lambda tau: int(np.count_nonzero(x >= tau))              # distinct values: R is a plain count
+    k = 6
+    # overflow with rank 8, buffer of 20: the tighter rank 3 must bring the count back into [k, 20]
+    R8, R3 = count(sample_desc[7]), count(sample_desc[2])
+    assert R8 > 20 and k <= R3 <= 20, (R8, R3)                       # (the hand-picked seed makes it so)
+    res = stages.run_row(x, k, 16, 8, 20, k, seed=9, r_tight=3)
+    assert res.status == stages.STATUS_OVERFLOW_REFILTERED and res.survivors == R3 and res.tau == sample_desc[2]
+    ov, oi = topk.topk_brute(x, k)
+    assert np.array_equal(res.idx, oi) and np.array_equal(res.vals, ov)
+    # without a tighter rank, or with one that still overflows, the exact fallback answers, reporting the first pass
+    for tight in (0, 7):
+        res = stages.run_row(x, k, 16, 8, 20, k, seed=9, r_tight=tight)
+        assert res.status == stages.STATUS_OVERFLOW and res.survivors == R8 and res.tau == sample_desc[7]
+        assert np.array_equal(res.idx, oi)
+    # recall failure with rank 1 (the sample maximum) and k = 12: the looser rank 5 repairs it, rank 2 does not
+    k = 12
+    R1, R2, R5 = count(sample_desc[0]), count(sample_desc[1]), count(sample_desc[4])
+    assert R1 < k and R2 < k and k <= R5 <= 40, (R1, R2, R5)
+    ov, oi = topk.topk_brute(x, k)
+    res = stages.run_row(x, k, 16, 1, 40, k, seed=9, r_loose=5)
+    assert res.status == stages.STATUS_RECALL_REFILTERED and res.survivors == R5 and res.tau == sample_desc[4]
+    assert np.array_equal(res.idx, oi) and np.array_equal(res.vals, ov)
+    res = stages.run_row(x, k, 16, 1, 40, k, seed=9, r_loose=2)
+    assert res.status == stages.STATUS_RECALL and res.survivors == R1 and np.array_equal(res.idx, oi)
+    # the tie-proof variant takes the same branches on distinct values
+    res = stages.run_row(x, k, 16, 1, 40, k, seed=9, r_loose=5, composite=True)
+    assert res.status == stages.STATUS_RECALL_REFILTERED and res.survivors == R5 and np.array_equal(res.idx, oi)
+    # relaxed mode: the second pass is checked against the full k
+    res = stages.run_row(x, 12, 16, 1, 40, 3, seed=9, r_loose=2)     # k_accept = 3: R1 decides
+    assert (res.status == stages.STATUS_OK) == (R1 >= 3)
