@@ -199,11 +199,13 @@ def describe(name, cfg):
 
 
 def count_fallbacks(profk, inputs, rows, k, eps, recall, out, n_calls, seed0=10_000):
-    """Rows (over n_calls calls, each with its own seed) whose count check failed and were repaired by the exact path."""
+    """Rows (over n_calls calls, each with its own seed) whose count check failed and were repaired (by a second filtering
+    pass or by the exact selection)."""
     failed = 0
     for s in range(n_calls):
         profk.topk(inputs[s % len(inputs)], k, eps=eps, recall=recall, seed=seed0 + s, out=out)
-        failed += sum(1 for st in profk.read_stats(rows) if (st[3] & 0xFF) in (profk.ROW_RECALL, profk.ROW_OVERFLOW))
+        failed += sum(1 for st in profk.read_stats(rows) if (st[3] & 0xFF) in (profk.ROW_RECALL, profk.ROW_OVERFLOW, profk.ROW_RECALL_REFILTERED,
+                                                                               profk.ROW_OVERFLOW_REFILTERED))
     return failed
 
 
@@ -371,6 +373,8 @@ def main():
     ap.add_argument("--one-row-sharded", action="store_true",
                     help="strong scaling instead of replicas: ONE row of the configuration's length cut into one shard per GPU "
                          "(sharding.topk_one_row: two all-gathers per call); with --gpus 1 the same path on a single shard")
+    ap.add_argument("--entry", default="topk", choices=["topk", "batchtopk"],
+                    help="with --hot-path-only: the entry point a step calls (batchtopk: the kept set as unordered pairs; single-row configurations)")
     ap.add_argument("--hot-path-only", action="store_true",
                     help="run only warm-up + timed steps of the hot path (for profiler captures) and exit")
     ap.add_argument("--rows", type=int, default=0,
@@ -435,7 +439,10 @@ def main():
         torch.cuda.synchronize()
 
     def step(i):
-        profk.topk(dev_inputs[i % copies], k, eps=eps, recall=recall, seed=i, out=(out_vals, out_idx))
+        if args.hot_path_only and args.entry == "batchtopk":
+            profk.batchtopk(dev_inputs[i % copies], k, eps=eps, seed=i, want_pairs=True)
+        else:
+            profk.topk(dev_inputs[i % copies], k, eps=eps, recall=recall, seed=i, out=(out_vals, out_idx))
 
     # ---- device-resident timing: the headline value ----
     sampler = ClockSampler(local_rank)

@@ -10,12 +10,12 @@
 //   * otherwise a histogram select over the R candidate records.  A record r is at distance D = T - r below the
 //     largest record the filter can have kept (T = tau's key with an all-ones index), larger D = better record.
 //     Level 0 bins D on a logarithmic scale (6 bits of exponent, 12 of mantissa: 2^18 bins in global memory, fine
-//     where records are dense); the bin that holds the K-th best record is found by a two-step scan (128 segment
-//     totals, then the one segment); if that bin is crowded (many equal values: its records differ only in the index)
+//     where records are dense) and, through shared memory, into 512 coarse bins; after ONE grid barrier every CTA
+//     scans the coarse bins and then the 512 fine bins of the one that holds the K-th best record; if that bin is crowded (many equal values: its records differ only in the index)
 //     the next levels bin its D range linearly, 18 bits at a time, until at most BK_EDGE records are left in the
 //     boundary class;
-//   * the emit pass: every record of a better class is kept; the boundary class is copied to a short list and ranked
-//     there, its best `need` records are kept as well.  Kept records are appended to the pair list (one atomic per CTA
+//   * the emit pass: every record of a better class is kept; the boundary class is copied to a short list, and the CTA
+//     that finishes last (a ticket; nobody waits) ranks that list and keeps its best `need` records as well.  Kept records are appended to the pair list (one atomic per CTA
 //     and pass), set their bit in the mask and are written to the dense array, which the kernel has zeroed before.
 #pragma once
 
@@ -26,17 +26,18 @@ namespace profk {
 constexpr int BK_THREADS = FB_THREADS;          // the exact selection it may call is written for this CTA size
 constexpr int BK_BITS = 18;
 constexpr uint32_t BK_BINS = 1u << BK_BITS;
-constexpr uint32_t BK_FLAGS = 8;                // words after the bins: [0] pairs appended, [1] records in the boundary list
+constexpr uint32_t BK_FLAGS = 8;                // words after the bins: [0] pairs appended, [1] records in the boundary list, [2] CTAs done emitting
 constexpr uint32_t BK_EDGE = 1024;              // a boundary class up to this size is ranked directly
-constexpr uint32_t BK_SEGMENTS = 128;           // the scan cuts the bins into this many segments ...
-constexpr uint32_t BK_SEG_BINS = BK_BINS / BK_SEGMENTS;      // ... of 2048 bins, two per thread
-static_assert(BK_SEG_BINS == 2 * BK_THREADS, "a CTA scans one segment with two bins per thread");
+constexpr uint32_t BK_COARSE = 512;             // coarse bins, each the sum of BK_BINS / BK_COARSE = 512 fine ones
+constexpr uint32_t BK_PER_COARSE = BK_BINS / BK_COARSE;
+static_assert(BK_COARSE <= BK_THREADS && BK_PER_COARSE <= BK_THREADS, "one thread per coarse bin, then per fine bin of one coarse bin");
+constexpr uint32_t BK_WAIT_LIMIT = 1u << 22;    // polls of the "all CTAs have zeroed their share of the bins" counter
 constexpr int BK_MAX_LEVELS = 6;                // 12 + 18 * 3 > 64 bits: more levels than any input needs
 
 template <typename T> struct BatchTopkParams {
     FallbackParams<T> fb;        // the row (rows == 1), K, capacity, control block, header, histogram area, buffer
     uint32_t* bins;              // BK_BINS + BK_FLAGS words
-    uint32_t* seg_totals;        // BK_SEGMENTS words
+    uint32_t* coarse;            // BK_COARSE words: the coarse histogram
     uint64_t* edge;              // BK_EDGE records: the boundary class
     uint32_t parts;              // 1, or FILTER_PARTS: the filter appended to that many parts of the buffer
     uint32_t part_cap;
@@ -95,7 +96,13 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
     uint32_t* flags = p.bins + BK_BINS;
 
     // Prologue, before the wait for the filter kernel: the workspace's bins and flags (nobody else uses them).
+    // Each CTA then reports in through the header's `done` word (zeroed by the call's first kernel, long finished): the
+    // histogram pass below needs every CTA's share to be zero, and by then all have reported -- a wait that does not wait.
     for (uint64_t b = gid; b < BK_BINS + BK_FLAGS; b += gthreads) p.bins[b] = 0;
+    for (uint64_t b = gid; b < BK_COARSE; b += gthreads) p.coarse[b] = 0;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) atomicAdd(&fb.header->done, 1u);
     pdl_launch_dependents();
     if (p.use_pdl) pdl_wait();
     uint32_t gen = *((volatile uint32_t*)&fb.header->bar_gen);          // read before this CTA's first arrival
@@ -169,7 +176,25 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
     uint32_t need = K;            // ... and its `need` best records are kept, with every record of a better class
     bool whole = keep_all;        // the whole boundary class is kept: nothing to rank
     if (keep_all) need = 0;
-    if (!grid_barrier(fb.header, gen)) return;                            // bins are zero, in every CTA's view
+    __shared__ uint32_t s_coarse[BK_COARSE];
+    __shared__ uint32_t s_ok;
+    if (keep_all) {
+        // (the exact selection ended on a grid barrier, but the zero fill above came after it)
+        if (!grid_barrier(fb.header, gen)) return;
+    } else {
+        // every CTA has zeroed its share of the bins: reported before the wait for the filter kernel, so this returns at once
+        if (tid == 0) {
+            uint32_t ok = 1, polls = 0;
+            while (*((volatile uint32_t*)&fb.header->done) < nctas) {
+                __nanosleep(64);
+                if (++polls > BK_WAIT_LIMIT) { atomicExch(&fb.header->error, 1u); ok = 0; break; }
+            }
+            __threadfence();
+            s_ok = ok;
+        }
+        __syncthreads();
+        if (!s_ok) return;
+    }
     for (int level = 0; !whole && level < BK_MAX_LEVELS; ++level) {
         const int sh_bits = cls_w > BK_BITS ? cls_w - BK_BITS : 0;       // linear levels: D's bits below the bin
         auto bin_of = [&](uint64_t D, bool* in_class) {
@@ -177,47 +202,36 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
             *in_class = D >= cls_lo && ((D - cls_lo) >> cls_w) == 0;
             return (uint32_t)((D - cls_lo) >> sh_bits) & (BK_BINS - 1);
         };
-        // histogram, best records in the lowest bins
+        // histogram, best records in the lowest bins: fine bins in global memory, coarse bins through shared memory
+        for (uint32_t c = tid; c < BK_COARSE; c += BK_THREADS) s_coarse[c] = 0;
+        __syncthreads();
         for (uint64_t i = gid; i < total; i += gthreads) {
             bool in_class;
-            const uint32_t b = bin_of(top - record_at(i), &in_class);
-            if (in_class) atomicAdd(&p.bins[BK_BINS - 1 - b], 1u);
-        }
-        if (!grid_barrier(fb.header, gen)) return;
-        // totals of the segments
-        for (uint32_t s = cta; s < BK_SEGMENTS; s += nctas) {
-            const uint2 c = __ldcg(reinterpret_cast<const uint2*>(p.bins + s * BK_SEG_BINS) + tid);
-            const uint32_t incl = block_inclusive_scan(c.x + c.y, sh.warp_sums);
-            if (tid == BK_THREADS - 1) p.seg_totals[s] = incl;
-            __syncthreads();
-        }
-        if (!grid_barrier(fb.header, gen)) return;
-        // every CTA: the segment, then the bin, of the need-th best record of the class
-        if (warp == 0) {
-            uint32_t t[BK_SEGMENTS / 32], sum = 0;
-#pragma unroll
-            for (int j = 0; j < (int)(BK_SEGMENTS / 32); ++j) { t[j] = __ldcg(&p.seg_totals[lane * (BK_SEGMENTS / 32) + j]); sum += t[j]; }
-            uint32_t incl = sum;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t v = __shfl_up_sync(FULL_MASK, incl, d);
-                if (lane >= (unsigned)d) incl += v;
-            }
-            uint32_t before = incl - sum;
-#pragma unroll
-            for (int j = 0; j < (int)(BK_SEGMENTS / 32); ++j) {
-                if (before < need && need <= before + t[j]) { s_seg = lane * (BK_SEGMENTS / 32) + j; s_seg_before = before; }
-                before += t[j];
+            const uint32_t f = BK_BINS - 1 - bin_of(top - record_at(i), &in_class);
+            if (in_class) {
+                atomicAdd(&p.bins[f], 1u);
+                atomicAdd(&s_coarse[f / BK_PER_COARSE], 1u);
             }
         }
         __syncthreads();
+        for (uint32_t c = tid; c < BK_COARSE; c += BK_THREADS) {
+            const uint32_t n = s_coarse[c];
+            if (n) atomicAdd(&p.coarse[c], n);
+        }
+        if (!grid_barrier(fb.header, gen)) return;
+        // every CTA: the coarse bin, then the fine bin, of the need-th best record of the class
+        {
+            const uint32_t c = tid < BK_COARSE ? __ldcg(&p.coarse[tid]) : 0u;
+            const uint32_t incl = block_inclusive_scan(c, sh.warp_sums);
+            if (incl - c < need && need <= incl) { s_seg = tid; s_seg_before = incl - c; }
+            __syncthreads();
+        }
         {
             const uint32_t seg = s_seg, seg_before = s_seg_before;
-            const uint2 c = __ldcg(reinterpret_cast<const uint2*>(p.bins + seg * BK_SEG_BINS) + tid);
-            const uint32_t incl = block_inclusive_scan(c.x + c.y, sh.warp_sums);
-            const uint32_t b0 = seg_before + incl - c.x - c.y, b1 = b0 + c.x;
-            if (b0 < need && need <= b0 + c.x) { s_bin = seg * BK_SEG_BINS + 2 * tid; s_bin_before = b0; s_bin_count = c.x; }
-            else if (b1 < need && need <= b1 + c.y) { s_bin = seg * BK_SEG_BINS + 2 * tid + 1; s_bin_before = b1; s_bin_count = c.y; }
+            const uint32_t c = tid < BK_PER_COARSE ? __ldcg(&p.bins[seg * BK_PER_COARSE + tid]) : 0u;
+            const uint32_t incl = block_inclusive_scan(c, sh.warp_sums);
+            const uint32_t b0 = seg_before + incl - c;
+            if (tid < BK_PER_COARSE && b0 < need && need <= b0 + c) { s_bin = seg * BK_PER_COARSE + tid; s_bin_before = b0; s_bin_count = c; }
             __syncthreads();
         }
         const uint32_t bin = BK_BINS - 1 - s_bin, in_bin = s_bin_count;
@@ -228,7 +242,9 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
         if (in_bin == need) { whole = true; break; }
         if (in_bin <= BK_EDGE) break;
         // crowded: one more level inside the class; the bins start from zero again
+        if (!grid_barrier(fb.header, gen)) return;                        // everybody has read this level's bins
         for (uint64_t b = gid; b < BK_BINS; b += gthreads) p.bins[b] = 0;
+        for (uint64_t b = gid; b < BK_COARSE; b += gthreads) p.coarse[b] = 0;
         if (!grid_barrier(fb.header, gen)) return;
     }
     // Kept outright: D >= keep_from.  Boundary list: cls_lo <= D < keep_from (empty when the whole class is kept).
@@ -287,9 +303,13 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
     }
     if (whole) return;
 
-    // ---- the boundary class: rank its records, keep the best `need` ----
-    if (!grid_barrier(fb.header, gen)) return;
-    if (cta != 0) return;
+    // ---- the boundary class: the CTA that finishes last ranks its records and keeps the best `need` ----
+    __threadfence();                               // this thread's appends to the boundary list are out ...
+    __syncthreads();                               // ... for every thread of the CTA
+    if (tid == 0) s_ok = atomicAdd(&flags[2], 1u) == nctas - 1 ? 1u : 0u;
+    __syncthreads();
+    if (!s_ok) return;
+    __threadfence();
     const uint32_t n_edge = min(__ldcg(&flags[1]), BK_EDGE);
     uint64_t* list = sh.edge;                      // RF_EDGE_CAP == BK_EDGE records of shared memory
     static_assert(RF_EDGE_CAP >= BK_EDGE, "the boundary list fits SelectShared::edge");

@@ -676,7 +676,7 @@ int batchtopk_planned(const T* in, int64_t N, int64_t K, const profk_plan_t* pla
     bp.fb.use_pdl = 0; bp.fb.out_vals = nullptr; bp.fb.out_idx = nullptr; bp.fb.cta_records = nullptr; bp.fb.cta_counters = nullptr;
     bp.fb.sort_cap = 0; bp.fb.parallel = 0;
     bp.bins = bins;
-    bp.seg_totals = ghist;                                        // (the exact selection and the select levels never both run)
+    bp.coarse = ghist;                                            // (the exact selection and the select levels never both run)
     bp.edge = buf + row_stride / 2;                               // the scratch half of the row's buffer
     bp.parts = parts ? FILTER_PARTS : 1u; bp.part_cap = part_cap; bp.part_counts = part_counts;
     bp.sel_vals = sel_vals; bp.sel_idx = sel_idx; bp.mask = mask; bp.dense = dense;

@@ -44,9 +44,13 @@ def assert_stats_match(x: torch.Tensor, k: int, pl, seed: int, stats, rows=None)
     xn = workloads.as_numpy(x)
     xn = xn[None, :] if xn.ndim == 1 else xn
     for r in (range(xn.shape[0]) if rows is None else rows):
-        res = o_stages.run_row(xn[r], k, pl.m, pl.r, pl.capacity, pl.k_accept, seed=seed, row=r,
-                               composite=getattr(pl, "tie_rule", profk.TIES_BY_INDEX) == profk.TIES_BY_INDEX)
         tau_bits, R, cap, status = stats[r]
+        # A row repaired by the second filtering pass (statuses 4 and 5; only calls whose refine kernel repairs rows
+        # itself take it) is compared with the oracle's run of that pass, any other row with the run without it.
+        second = status in (profk.ROW_RECALL_REFILTERED, profk.ROW_OVERFLOW_REFILTERED)
+        res = o_stages.run_row(xn[r], k, pl.m, pl.r, pl.capacity, pl.k_accept, seed=seed, row=r,
+                               composite=getattr(pl, "tie_rule", profk.TIES_BY_INDEX) == profk.TIES_BY_INDEX,
+                               r_tight=getattr(pl, "r_tight", 0) if second else 0, r_loose=getattr(pl, "r_loose", 0) if second else 0)
         assert cap == pl.capacity
         assert tau_bits == int(bits(np.asarray([res.tau]))[0]), f"row {r}: threshold differs"     # same sample, same threshold
         assert status == res.status, f"row {r}: status {status}, oracle {res.status}"
