@@ -365,6 +365,94 @@ __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T
     return (uint64_t)base + total > cap ? row : 0xFFFFFFFFu;
 }
 
+// DEFER build (many survivors: batches of short rows, dense selections).  With one or two survivors per warp-tile most
+// tiles would take the slow path above, whose few hundred warp instructions -- executed for the sake of one or two lanes
+// -- make the scan instruction-bound (359 warp instructions per bf16 warp-tile on 2^20-element rows with k = 32, against
+// 96 on the fast path).  Here a warp whose tile holds a candidate only NOTES it: four votes say which lanes hold an
+// element not below the threshold in which of their vectors, one shared-memory atomic reserves room, and each such lane
+// writes the number of its vector into a list in the CTA's shared memory -- a few dozen instructions, no global memory.
+// When the CTA has streamed all its tiles it works the list off with every lane busy: thread i reads candidate vector i
+// again (the candidates are a fraction of a percent of the input), decides its elements exactly and appends the
+// survivors.  A warp that finds the list full takes the slow path above instead.
+#ifndef PROFK_DEFER_CAP
+#define PROFK_DEFER_CAP 6144
+#endif
+constexpr uint32_t DEFER_CAP = PROFK_DEFER_CAP;      // candidate vectors per CTA: 24 KB of shared memory
+constexpr uint32_t DEFER_NONE = 0xFFFFFFFFu;          // a reserved slot that was not used
+
+// One round of working the list off: lane by lane a candidate vector (number `vid` among the vectors of the launch,
+// tiles in order; DEFER_NONE = none) is read again and decided in the total order of the keys; the survivors are
+// appended with one atomic per warp when all of the warp's survivors belong to one row (the list is in tile order, so
+// they nearly always do), else with one per lane.  All 32 lanes call it.
+template <typename T, int THREADS, int UNROLL, bool PARTS>
+__device__ __forceinline__ void defer_process_round(const FilterParams<T>& p, uint32_t vid) {
+    using V = typename Elem<T>::vec_t;
+    constexpr int VEC = Elem<T>::VEC;
+    constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
+    const unsigned lane = lane_id();
+    uint32_t row = 0;
+    unsigned m = 0;
+    V v = {};
+    int64_t i0 = 0;
+    if (vid != DEFER_NONE) {
+        const uint32_t tile = vid / TILE_VECTORS, within = vid % TILE_VECTORS;
+        const uint32_t tiles_per_row = (uint32_t)p.tiles_per_row;
+        uint32_t tin = tile;
+        if (tiles_per_row != (uint32_t)p.total_tiles) { row = tile / tiles_per_row; tin = tile - row * tiles_per_row; }
+        const RowView<T> rv = row_view(p.in, p.N, row);
+        const T tau = p.thr ? Elem<T>::from_bits(reinterpret_cast<const uint32_t*>(p.thr + row)[0]) : p.tau[row];
+        const uint64_t q = (uint64_t)tin * TILE_VECTORS + within;
+        bool in;
+        v = load_row_vector(rv, p.N, q, &in);
+        if (in) {
+            i0 = (int64_t)(q * VEC) - (int64_t)rv.mis;
+            m = vec_pass_mask(v, tau);
+            if (i0 < 0 || i0 + VEC > (int64_t)p.N) {
+#pragma unroll
+                for (int j = 0; j < VEC; ++j)
+                    if (i0 + j < 0 || i0 + j >= (int64_t)p.N) m &= ~(1u << j);
+            }
+            m = confirm_survivors<T>(p, row, v, m, i0, tau);
+        }
+    }
+    const unsigned cnt = __popc(m);
+    const unsigned has = __ballot_sync(FULL_MASK, cnt != 0);
+    if (has == 0) return;
+    const uint32_t row0 = __shfl_sync(FULL_MASK, row, __ffs(has) - 1);
+    const bool one_row = __all_sync(FULL_MASK, cnt == 0 || row == row0);
+    const uint32_t my_row = one_row ? row0 : row;
+    uint32_t* counter = p.counts + (uint64_t)my_row * p.count_stride;
+    uint64_t* dst = p.buf + (uint64_t)my_row * p.buf_stride;
+    uint32_t cap = p.capacity;
+    if (PARTS) {
+        const uint32_t part = blockIdx.x % FILTER_PARTS;
+        counter = p.part_counts + ((uint64_t)my_row * FILTER_PARTS + part) * FILTER_PART_STRIDE;
+        dst += (uint64_t)part * p.part_cap;
+        cap = p.part_cap;
+    }
+    unsigned pos;
+    if (one_row) {
+        unsigned incl = cnt;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned nb = __shfl_up_sync(FULL_MASK, incl, d);
+            if (lane >= (unsigned)d) incl += nb;
+        }
+        const unsigned total = __shfl_sync(FULL_MASK, incl, 31);
+        unsigned base = 0;
+        if (lane == 0) base = atomicAdd(counter, total);
+        pos = __shfl_sync(FULL_MASK, base, 0) + incl - cnt;
+    } else {
+        pos = cnt ? atomicAdd(counter, cnt) : 0u;
+    }
+    while (m) {
+        const int b = __ffs(m) - 1;
+        m &= m - 1;
+        if (pos < cap) dst[pos] = make_record(Elem<T>::key(vec_elem(v, b)), (uint32_t)(i0 + b));
+        ++pos;
+    }
+}
+
 // STAGED = collect survivors in per-warp shared-memory stages (dense survivors, one row at a time);
 // otherwise append them directly (sparse survivors or many short rows).
 //
@@ -374,11 +462,18 @@ __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T
 // tiles of the launch (from dyn_start on) come from a global counter instead, so that SMs that saw
 // less bandwidth take fewer of them and all CTAs finish together.  The counter is read one tile
 // ahead, so its round trip hides behind the loads; only this tail needs a CTA barrier per tile.
-template <typename T, int THREADS, int UNROLL, bool STAGED, bool PARTS = false>
+template <typename T, int THREADS, int UNROLL, bool STAGED, bool PARTS = false, bool DEFER = false>
 __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGED : sizeof(T) == 4 ? PROFK_FILTER_MINBLOCKS_F32 : PROFK_FILTER_MINBLOCKS_BF16) filter_kernel(const __grid_constant__ FilterParams<T> p) {
+    static_assert(!(STAGED && DEFER), "one way of handling dense survivors at a time");
     using V = typename Elem<T>::vec_t;
     constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
     __shared__ WarpStage stages[STAGED ? THREADS / 32 : 1];
+    __shared__ uint32_t hits[DEFER ? DEFER_CAP : 1];
+    __shared__ uint32_t s_nhits;
+    if (DEFER) {
+        if (threadIdx.x == 0) s_nhits = 0;
+        __syncthreads();
+    }
     __shared__ uint32_t s_next[2];
     __shared__ __align__(8) uint64_t pf_bar;                         // counts the bytes of the prefetched tiles
     extern __shared__ __align__(128) unsigned char pf_smem[];        // p.prefetch_tiles tiles of 32 KB (or nothing)
@@ -524,9 +619,32 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
         }
 
         if (__any_sync(FULL_MASK, hit) && row != skip_row) {
-            uint32_t o;
-            if (STAGED) o = filter_slow_path<T, THREADS, UNROLL>(p, st, v[0], v[1], v[2], v[3], inside_mask, row, qbase, rv.mis, tau_lo);
-            else o = filter_slow_path_direct<T, THREADS, UNROLL, PARTS>(p, v, inside_mask, row, qbase, rv.mis, tau_lo);
+            uint32_t o = 0xFFFFFFFFu;
+            bool noted = false;
+            if (DEFER) {
+                // note the candidate vectors: which lanes, which of their vectors; one reservation for the warp
+                bool h[UNROLL];
+                uint32_t before[UNROLL], total = 0;
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) {
+                    h[u] = ((inside_mask >> u) & 1u) && vec_any_pass(v[u], tau);
+                    const uint32_t b = __ballot_sync(FULL_MASK, h[u]);
+                    before[u] = total + __popc(b & ((1u << lane) - 1u));
+                    total += __popc(b);
+                }
+                uint32_t base = 0;
+                if (lane == 0) base = atomicAdd(&s_nhits, total);
+                base = __shfl_sync(FULL_MASK, base, 0);
+                noted = base + total <= DEFER_CAP;               // (a warp that does not fit leaves its slots unused)
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u)
+                    if (h[u] && base + before[u] < DEFER_CAP)
+                        hits[base + before[u]] = noted ? tile * TILE_VECTORS + (uint32_t)u * THREADS + threadIdx.x : DEFER_NONE;
+            }
+            if (!noted) {
+                if (STAGED) o = filter_slow_path<T, THREADS, UNROLL>(p, st, v[0], v[1], v[2], v[3], inside_mask, row, qbase, rv.mis, tau_lo);
+                else o = filter_slow_path_direct<T, THREADS, UNROLL, PARTS>(p, v, inside_mask, row, qbase, rv.mis, tau_lo);
+            }
             if (o != 0xFFFFFFFFu) skip_row = o;
         }
 
@@ -547,6 +665,15 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
         if (row != tau_row) { tau_row = row; load_threshold(); }
     }
     if (STAGED && st->fill) flush_stage(p, st);
+    if (DEFER) {
+        // every tile of this CTA has been streamed: work the list off, one entry per thread
+        __syncthreads();
+        const uint32_t n = s_nhits < DEFER_CAP ? s_nhits : DEFER_CAP;
+        for (uint32_t e0 = 0; e0 < n; e0 += THREADS) {          // whole warps take part in every round
+            const uint32_t e = e0 + threadIdx.x;
+            if (e0 + (threadIdx.x & ~31u) < n) defer_process_round<T, THREADS, UNROLL, PARTS>(p, e < n ? hits[e] : DEFER_NONE);
+        }
+    }
     if (pf_pending) prefetch_landed(PREFETCH_SPIN_LIMIT);
 }
 

@@ -62,6 +62,7 @@ struct DeviceInfo {
     int sm_count = 0;
     int filter_blocks_per_sm[2] = {0, 0};     // by dtype
     int filter_staged_blocks_per_sm[2] = {0, 0};
+    int filter_defer_blocks_per_sm[2] = {0, 0};
     int max_cluster[2] = {8, 8};              // 16 when the device can co-schedule 16 CTAs of the threshold kernel
     int refine_cluster[2] = {8, 8};           // same for the refine kernel at its largest footprint
     bool ready = false;
@@ -145,6 +146,9 @@ template <typename T> int ensure_device_info(int dev, DeviceInfo* out) {
         CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, true>,
                                                                  FILTER_THREADS, 0));
         di.filter_staged_blocks_per_sm[d] = std::max(nb, 1);
+        CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false, false, true>,
+                                                                 FILTER_THREADS, 0));
+        di.filter_defer_blocks_per_sm[d] = std::max(nb, 1);
         CUDA_TRY(cudaFuncSetAttribute(sample_select_kernel<T, SEL_THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
         const int prefetch_bytes = (int)(FILTER_PREFETCH * FILTER_THREADS * FILTER_UNROLL * 16u);
         CUDA_TRY(cudaFuncSetAttribute(filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, prefetch_bytes));
@@ -274,7 +278,7 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
 template <typename T>
 int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, const T* tau, int64_t capacity, uint64_t* buf,
                   uint64_t buf_stride, uint32_t* counts, uint32_t count_stride, bool pdl, bool staged, uint32_t* tile_counter, bool parts,
-                  uint32_t part_cap, uint32_t* part_counts, const uint4* thr, cudaStream_t st) {
+                  uint32_t part_cap, uint32_t* part_counts, const uint4* thr, cudaStream_t st, bool deferred = false) {
     FilterParams<T> fp;
     fp.thr = thr;
     fp.in = in; fp.N = (uint64_t)N; fp.rows = (uint64_t)rows; fp.tau = tau; fp.capacity = (uint32_t)capacity;
@@ -285,8 +289,9 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     fp.use_pdl = pdl ? 1 : 0;
     fp.tile_counter = tile_counter;
     fp.part_cap = part_cap; fp.part_counts = part_counts;
+    if (staged || parts || fp.total_tiles * (uint64_t)(FILTER_THREADS * FILTER_UNROLL) >= (1ull << 32)) deferred = false;   // vectors are numbered in 32 bits
     const uint64_t max_grid = (uint64_t)di.sm_count *
-        (staged ? di.filter_staged_blocks_per_sm[dtype_index<T>()] : di.filter_blocks_per_sm[dtype_index<T>()]);
+        (staged ? di.filter_staged_blocks_per_sm[dtype_index<T>()] : deferred ? di.filter_defer_blocks_per_sm[dtype_index<T>()] : di.filter_blocks_per_sm[dtype_index<T>()]);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)std::min<uint64_t>(fp.total_tiles, max_grid));
     // all but the last ~PROFK_DYNAMIC_ROUNDS tiles per CTA follow the fixed stride
@@ -296,7 +301,8 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     cfg.blockDim = dim3(FILTER_THREADS);
     // A single row scanned behind the threshold kernel: each CTA copies its next tiles into shared memory while it waits.
     // (Not the staged build: its two CTAs per SM spill already, and the copies cost the 2^29 bf16 row 3 us.)
-    const bool prefetch = pdl && !staged && rows == 1 && fp.dyn_start >= (FILTER_PREFETCH + 1) * cfg.gridDim.x;
+    // (nor the build that defers its candidates: their list takes the shared memory)
+    const bool prefetch = pdl && !staged && !deferred && rows == 1 && fp.dyn_start >= (FILTER_PREFETCH + 1) * cfg.gridDim.x;
     fp.prefetch_tiles = prefetch ? FILTER_PREFETCH : 0u;
     fp.prefetch_spin_limit = g_prefetch_spin_limit.load();
     cfg.dynamicSmemBytes = prefetch ? FILTER_PREFETCH * FILTER_THREADS * FILTER_UNROLL * 16u : 0;
@@ -306,6 +312,7 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
     if (staged) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, true>, fp));
+    else if (deferred) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false, false, true>, fp));
     else if (parts) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false, true>, fp));
     else CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false>, fp));
     ++g_launches;
@@ -435,6 +442,17 @@ int launch_refine(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, Ro
     return PROFK_OK;
 }
 
+// Which build of the filter takes a launch with this many survivors expected per warp-tile.  From about one survivor per
+// warp-tile on, most tiles would run the slow path and the scan becomes instruction-bound; the build that only notes its
+// candidates in shared memory and decides them after streaming (DEFER, filter.cuh) then wins for bf16 (twice the
+// elements per warp-tile): 512 rows of 2^20, k = 32 (1.46 per warp-tile) 298 -> 279 us; the paper's SAE shape (3.2)
+// 112 -> 99, where it also replaces the staged build.  fp32: the SAE shape (1.6) 93.4 -> 89.8; batches of fp32 rows
+// (0.73) lose 2 % and stay on the direct build; 2^29 bf16, K = 131072 (0.4) is indifferent.
+template <typename T> bool defer_candidates(int64_t rows, double per_warp_tile) {
+    if (sizeof(T) == 2) return per_warp_tile > 0.8;
+    return rows == 1 && per_warp_tile > 1.0;
+}
+
 template <typename T>
 int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_plan_t* plan, uint64_t seed, void* stream,
                  T* out_vals, int64_t* out_idx) {
@@ -487,11 +505,13 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         // (The direct append has three CTAs per SM, eight counters for large selections and the prefetch behind the threshold
     // kernel; it holds up to about two survivors per warp-tile: 2^29 bf16, K = 131072 at 0.4: 248 -> 237 us; 50 M fp32,
     // K = 131072 at 1.6: 124 -> 114; 50 M bf16 at 3.2 stays staged, 120 against 127.)
-    const bool staged = plan->mode == 0 && rows == 1 && per_warp_tile > 2.0;
+    const bool deferred = plan->mode == 0 && defer_candidates<T>(rows, per_warp_tile);
+    const bool staged = plan->mode == 0 && !deferred && rows == 1 && per_warp_tile > 2.0;
 
     // Large selections keep so many survivors that a row's single append counter would hold the scan up:
     // the direct variant then appends to FILTER_PARTS parts of the buffer, each with a counter of its own.
-    const bool parts = large && !staged && plan->mode == 0;
+    // (The deferring build appends once per 32 candidates, after streaming: one counter is enough for it.)
+    const bool parts = large && !staged && !deferred && plan->mode == 0;
     const uint32_t part_cap = (uint32_t)(row_stride / 2 / FILTER_PARTS);
     uint32_t* part_counts = reinterpret_cast<uint32_t*>(base + lay.off_parts);
 
@@ -536,7 +556,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
                                      nullptr, keep_keys ? keys_scratch : nullptr);
         if (rc != PROFK_OK) return rc;
         rc = launch_filter<T>(di, in, rows, N, nullptr, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, &header->tile_counter,
-                              parts, part_cap, part_counts, thr, st);
+                              parts, part_cap, part_counts, thr, st, deferred);
         if (rc != PROFK_OK) return rc;
 
         if (large) {
@@ -653,8 +673,9 @@ int batchtopk_planned(const T* in, int64_t N, int64_t K, const profk_plan_t* pla
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
     const double per_warp_tile = (double)plan->r / (double)std::max<int64_t>(plan->m, 1) * 32.0 * FILTER_UNROLL * Elem<T>::VEC;
-    const bool staged = plan->mode == 0 && per_warp_tile > 2.0;       // as in topk_planned
-    const bool parts = !staged && plan->mode == 0;
+    const bool deferred = plan->mode == 0 && defer_candidates<T>(1, per_warp_tile);       // as in topk_planned
+    const bool staged = plan->mode == 0 && !deferred && per_warp_tile > 2.0;
+    const bool parts = !staged && !deferred && plan->mode == 0;
     const uint32_t part_cap = (uint32_t)(row_stride / 2 / FILTER_PARTS);
 
     if (plan->mode == 0) {
@@ -662,7 +683,7 @@ int batchtopk_planned(const T* in, int64_t N, int64_t K, const profk_plan_t* pla
                                      parts ? part_counts : nullptr, plan->tie_rule == PROFK_TIES_BY_INDEX, thr, st);
         if (rc != PROFK_OK) return rc;
         rc = launch_filter<T>(di, in, 1, N, nullptr, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, &header->tile_counter,
-                              parts, part_cap, part_counts, thr, st);
+                              parts, part_cap, part_counts, thr, st, deferred);
         if (rc != PROFK_OK) return rc;
     } else {
         init_ctl_kernel<<<1, 256, 0, st>>>(ctl, 1, header, (uint32_t)capacity, (uint32_t)K);

@@ -441,3 +441,38 @@ def test_call_captured_in_a_cuda_graph():
             graph.replay()
             torch.cuda.synchronize()
             assert_exact(x.cpu(), k, workloads.as_numpy(out[0]), out[1].cpu().numpy())
+
+
+# ----------------------------------------------------------------------------- dense survivors: the deferring build of the filter
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_dense_survivors_noted_in_shared_memory_and_decided_after_streaming(dtype):
+    """Plans with one to a dozen survivors per warp-tile (rank / sample size): the filter only notes candidate vectors
+    while it streams and decides them afterwards.  Ragged and unaligned rows, batches and single rows, floods of copies
+    of the threshold (the list in shared memory fills up and the warps fall back to the direct slow path), both tie
+    rules; status, threshold and survivor count follow the oracle."""
+    k = 40
+    cases = []
+    for rows, n in ((1, 1 << 22), (1, 3_000_001), (7, 300_001), (40, 1 << 17)):
+        cases.append((f"normal {rows}x{n}", workloads.normal(rows, n, seed=90 + rows, dtype=dtype)))
+    cases.append(("constant", torch.full((3, 1 << 19), 1.25).to(dtype)))
+    cases.append(("few values", workloads.few_values(1 << 21, seed=91, distinct=4).to(dtype).view(1, -1)))
+    cases.append(("relu", workloads.relu_gaussian(1 << 21, seed=92, dtype=torch.float32).to(dtype).view(2, -1)))
+    for name, x in cases:
+        rows, n = x.shape
+        for m, r in ((2048, 24), (1024, 6)):                 # 12 / 6 expected survivors per bf16 warp-tile, half of that for fp32
+            cap = min(n // 2 - 1, 3 * r * (n // m))
+            for rule in (profk.TIES_BY_INDEX, profk.TIES_KEEP_ALL):
+                pl = profk.Plan(m=m, r=r, capacity=cap, k_accept=k, mode=0, tie_rule=rule)
+                v, i = profk.topk(x.cuda(), k, plan_override=pl, seed=13)
+                torch.cuda.synchronize()
+                assert_exact(x, k, workloads.as_numpy(v), i.cpu().numpy())
+                assert_stats_match(x, k, pl, 13, profk.read_stats(rows))
+    # an unaligned view of a batch
+    big = workloads.normal(1, 5 * 100_003 + 8, seed=93, dtype=dtype)[0].cuda()
+    for off in (1, 3):
+        x = big[off: off + 5 * 100_003].view(5, 100_003)
+        pl = profk.Plan(m=1024, r=12, capacity=4000, k_accept=k, mode=0)
+        v, i = profk.topk(x, k, plan_override=pl, seed=14)
+        torch.cuda.synchronize()
+        assert_exact(x.cpu(), k, workloads.as_numpy(v), i.cpu().numpy())
+        assert_stats_match(x.cpu(), k, pl, 14, profk.read_stats(5))
