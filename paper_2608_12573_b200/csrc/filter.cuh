@@ -415,41 +415,45 @@ __device__ __forceinline__ void defer_process_round(const FilterParams<T>& p, ui
             m = confirm_survivors<T>(p, row, v, m, i0, tau);
         }
     }
+    // Append, one atomic per row that has survivors in this round (a round of 32 consecutive entries spans a tile or two,
+    // so one or two rows): the lanes of the first row with survivors form a group, scan their counts, their first lane
+    // reserves the room; then the next row's lanes, until none is left.
     const unsigned cnt = __popc(m);
-    const unsigned has = __ballot_sync(FULL_MASK, cnt != 0);
-    if (has == 0) return;
-    const uint32_t row0 = __shfl_sync(FULL_MASK, row, __ffs(has) - 1);
-    const bool one_row = __all_sync(FULL_MASK, cnt == 0 || row == row0);
-    const uint32_t my_row = one_row ? row0 : row;
-    uint32_t* counter = p.counts + (uint64_t)my_row * p.count_stride;
-    uint64_t* dst = p.buf + (uint64_t)my_row * p.buf_stride;
-    uint32_t cap = p.capacity;
-    if (PARTS) {
-        const uint32_t part = blockIdx.x % FILTER_PARTS;
-        counter = p.part_counts + ((uint64_t)my_row * FILTER_PARTS + part) * FILTER_PART_STRIDE;
-        dst += (uint64_t)part * p.part_cap;
-        cap = p.part_cap;
-    }
-    unsigned pos;
-    if (one_row) {
-        unsigned incl = cnt;
+    unsigned left = __ballot_sync(FULL_MASK, cnt != 0);
+    while (left) {
+        const uint32_t row0 = __shfl_sync(FULL_MASK, row, __ffs(left) - 1);
+        const bool mine = cnt != 0 && row == row0;
+        const unsigned group = __ballot_sync(FULL_MASK, mine);
+        unsigned incl = mine ? cnt : 0u;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
             const unsigned nb = __shfl_up_sync(FULL_MASK, incl, d);
             if (lane >= (unsigned)d) incl += nb;
         }
         const unsigned total = __shfl_sync(FULL_MASK, incl, 31);
+        uint32_t* counter = p.counts + (uint64_t)row0 * p.count_stride;
+        uint64_t* dst = p.buf + (uint64_t)row0 * p.buf_stride;
+        uint32_t cap = p.capacity;
+        if (PARTS) {
+            const uint32_t part = blockIdx.x % FILTER_PARTS;
+            counter = p.part_counts + ((uint64_t)row0 * FILTER_PARTS + part) * FILTER_PART_STRIDE;
+            dst += (uint64_t)part * p.part_cap;
+            cap = p.part_cap;
+        }
         unsigned base = 0;
-        if (lane == 0) base = atomicAdd(counter, total);
-        pos = __shfl_sync(FULL_MASK, base, 0) + incl - cnt;
-    } else {
-        pos = cnt ? atomicAdd(counter, cnt) : 0u;
-    }
-    while (m) {
-        const int b = __ffs(m) - 1;
-        m &= m - 1;
-        if (pos < cap) dst[pos] = make_record(Elem<T>::key(vec_elem(v, b)), (uint32_t)(i0 + b));
-        ++pos;
+        if (lane == (unsigned)(__ffs(group) - 1)) base = atomicAdd(counter, total);
+        base = __shfl_sync(FULL_MASK, base, __ffs(group) - 1);
+        if (mine) {
+            unsigned pos = base + incl - cnt;
+            unsigned mm = m;
+            while (mm) {
+                const int b = __ffs(mm) - 1;
+                mm &= mm - 1;
+                if (pos < cap) dst[pos] = make_record(Elem<T>::key(vec_elem(v, b)), (uint32_t)(i0 + b));
+                ++pos;
+            }
+        }
+        left &= ~group;
     }
 }
 
@@ -610,7 +614,14 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
         }
 
         bool hit = false;
-        if (inside_mask == ALL_INSIDE) {
+        bool h[UNROLL];                          // (DEFER) vector u holds an element that is not below tau
+        if (DEFER) {
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                h[u] = (inside_mask == ALL_INSIDE || ((inside_mask >> u) & 1u)) && vec_any_pass(v[u], tau);
+                hit |= h[u];
+            }
+        } else if (inside_mask == ALL_INSIDE) {
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) hit |= vec_any_pass(v[u], tau);
         } else {
@@ -622,24 +633,24 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
             uint32_t o = 0xFFFFFFFFu;
             bool noted = false;
             if (DEFER) {
-                // note the candidate vectors: which lanes, which of their vectors; one reservation for the warp
-                bool h[UNROLL];
-                uint32_t before[UNROLL], total = 0;
+                // Note the candidate vectors.  Only the lanes that hold one do anything: each reserves room for its own
+                // (one shared-memory atomic; a tile rarely has more than two such lanes) and writes their numbers.
+                uint32_t slot = 0, cnt = 0;
+                if (hit) {
 #pragma unroll
-                for (int u = 0; u < UNROLL; ++u) {
-                    h[u] = ((inside_mask >> u) & 1u) && vec_any_pass(v[u], tau);
-                    const uint32_t b = __ballot_sync(FULL_MASK, h[u]);
-                    before[u] = total + __popc(b & ((1u << lane) - 1u));
-                    total += __popc(b);
+                    for (int u = 0; u < UNROLL; ++u) cnt += h[u] ? 1u : 0u;
+                    slot = atomicAdd(&s_nhits, cnt);
                 }
-                uint32_t base = 0;
-                if (lane == 0) base = atomicAdd(&s_nhits, total);
-                base = __shfl_sync(FULL_MASK, base, 0);
-                noted = base + total <= DEFER_CAP;               // (a warp that does not fit leaves its slots unused)
+                noted = !__any_sync(FULL_MASK, hit && slot + cnt > DEFER_CAP);      // (a warp that does not fit leaves its slots unused)
+                if (hit) {
 #pragma unroll
-                for (int u = 0; u < UNROLL; ++u)
-                    if (h[u] && base + before[u] < DEFER_CAP)
-                        hits[base + before[u]] = noted ? tile * TILE_VECTORS + (uint32_t)u * THREADS + threadIdx.x : DEFER_NONE;
+                    for (int u = 0; u < UNROLL; ++u) {
+                        if (h[u]) {
+                            if (slot < DEFER_CAP) hits[slot] = noted ? tile * TILE_VECTORS + (uint32_t)u * THREADS + threadIdx.x : DEFER_NONE;
+                            ++slot;
+                        }
+                    }
+                }
             }
             if (!noted) {
                 if (STAGED) o = filter_slow_path<T, THREADS, UNROLL>(p, st, v[0], v[1], v[2], v[3], inside_mask, row, qbase, rv.mis, tau_lo);

@@ -445,9 +445,9 @@ int launch_refine(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, Ro
 // Which build of the filter takes a launch with this many survivors expected per warp-tile.  From about one survivor per
 // warp-tile on, most tiles would run the slow path and the scan becomes instruction-bound; the build that only notes its
 // candidates in shared memory and decides them after streaming (DEFER, filter.cuh) then wins for bf16 (twice the
-// elements per warp-tile): 512 rows of 2^20, k = 32 (1.46 per warp-tile) 298 -> 279 us; the paper's SAE shape (3.2)
-// 112 -> 99, where it also replaces the staged build.  fp32: the SAE shape (1.6) 93.4 -> 89.8; batches of fp32 rows
-// (0.73) lose 2 % and stay on the direct build; 2^29 bf16, K = 131072 (0.4) is indifferent.
+// elements per warp-tile): 512 rows of 2^20, k = 32 (1.46 per warp-tile) 298 -> 260 us; the paper's SAE shape (3.2)
+// 112 -> 97, where it also replaces the staged build.  fp32: the SAE shape (1.6) 93.4 -> 89.3; batches of fp32 rows
+// (0.73) lose 6 % (397 -> 422 us) and stay on the direct build; 2^29 bf16, K = 131072 (0.4) is indifferent.
 template <typename T> bool defer_candidates(int64_t rows, double per_warp_tile) {
     if (sizeof(T) == 2) return per_warp_tile > 0.8;
     return rows == 1 && per_warp_tile > 1.0;
