@@ -219,16 +219,17 @@ def time_filter_alone(profk, torch, inputs, rows, n, dt, pl, launches, warmup):
         return None
     dev = inputs[0].device
     elem = 4 if dt == "f32" else 2
-    taus = profk.sample_threshold(inputs[0], pl.m, pl.r, seed=0)
+    taus = [profk.sample_threshold(x, pl.m, pl.r, seed=0) for x in inputs]       # every input copy with its own thresholds
     buf = torch.empty((rows, pl.capacity), dtype=torch.int64, device=dev)
-    many = torch.zeros((launches + warmup) * rows, dtype=torch.int32, device=dev)
+    stride = profk.FILTER_COUNT_STRIDE           # one counter per 32 bytes
+    many = torch.zeros(((launches + warmup) * rows, stride), dtype=torch.int32, device=dev)
     fn = getattr(profk.lib(), "profk_filter_f32" if dt == "f32" else "profk_filter_bf16")
     stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
 
     def launch(i):
         code = fn(ctypes.c_void_p(inputs[i % len(inputs)].data_ptr()), ctypes.c_int64(rows), ctypes.c_int64(n),
-                  ctypes.c_void_p(taus.data_ptr()), ctypes.c_int64(pl.capacity), ctypes.c_void_p(buf.data_ptr()),
-                  ctypes.c_void_p(many.data_ptr() + 4 * i * rows), stream)
+                  ctypes.c_void_p(taus[i % len(inputs)].data_ptr()), ctypes.c_int64(pl.capacity), ctypes.c_void_p(buf.data_ptr()),
+                  ctypes.c_void_p(many.data_ptr() + 4 * stride * i * rows), stream)
         assert code == 0
 
     for i in range(warmup):
@@ -241,10 +242,10 @@ def time_filter_alone(profk, torch, inputs, rows, n, dt, pl, launches, warmup):
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / launches
-    survivors = float(many[:rows].sum().item())
+    survivors = float(many[:launches * rows, 0].sum().item()) / launches        # per launch, averaged over the launches
     # The stand-alone filter takes the threshold as a value alone: on a row flooded with copies of tau its buffer
     # overflows and the launch stops early, so its duration is not that of a scan.
-    overflowed = bool((many[:rows] > pl.capacity).any().item())
+    overflowed = bool((many[:launches * rows, 0] > pl.capacity).any().item())
     algo = rows * n * elem + survivors * 8            # read every element once + one 8-byte record per survivor
     return {"ms_per_launch": ms, "algorithmic_bytes": algo, "overflowed": overflowed, "survivors_per_launch": survivors,
             "GBps": None if overflowed else algo / (ms * 1e-3) / 1e9}

@@ -28,6 +28,7 @@ EXPORTS = [
     "profk_refine_gathered_bf16",
 ]
 
+FILTER_COUNT_STRIDE = 8      # PROFK_FILTER_COUNT_STRIDE: uint32 words per row in the counts array of profk_filter_*
 ROW_OK, ROW_RECALL, ROW_OVERFLOW, ROW_DIRECT = 0, 1, 2, 3
 ROW_RECALL_REFILTERED, ROW_OVERFLOW_REFILTERED = 4, 5    # repaired by a second filtering pass (plan.r_loose / plan.r_tight)
 TIES_KEEP_ALL, TIES_BY_INDEX = 0, 1      # profk_plan_t.tie_rule: the filter as printed / the threshold as a (value, index) record
@@ -408,13 +409,13 @@ def filter_pass(x, tau, capacity: int):
     rows, n = x2.shape
     tau = tau.reshape(rows).contiguous()
     buf = torch.empty((rows, capacity), dtype=torch.int64, device=x2.device)
-    counts = torch.zeros(rows, dtype=torch.int32, device=x2.device)
+    counts = torch.zeros((rows, FILTER_COUNT_STRIDE), dtype=torch.int32, device=x2.device)       # one counter per 32 bytes
     fn = getattr(lib(), f"profk_filter_{_suffix(x2)}")
     with torch.cuda.device(x2.device):
         code = fn(ctypes.c_void_p(x2.data_ptr()), ctypes.c_int64(rows), ctypes.c_int64(n), ctypes.c_void_p(tau.data_ptr()),
                   ctypes.c_int64(capacity), ctypes.c_void_p(buf.data_ptr()), ctypes.c_void_p(counts.data_ptr()), _stream_ptr())
     _check(code, "profk_filter")
-    return buf, counts
+    return buf, counts[:, 0]
 
 
 def sample_threshold(x, m: int, r: int, seed: int, want_indices: bool = False):

@@ -725,15 +725,18 @@ int filter_only(const T* in, int64_t rows, int64_t N, const T* tau, int64_t capa
                 void* stream) {
     if (!in || !tau || !buf_keys || !counts) return PROFK_EINVAL;
     if (rows < 1 || N < 1 || N > N_MAX || capacity < 1 || capacity > N_MAX) return PROFK_EINVAL;
-    if ((uintptr_t)in % sizeof(T) || (uintptr_t)tau % sizeof(T) || (uintptr_t)buf_keys % 8 || (uintptr_t)counts % 4)
+    if ((uintptr_t)in % sizeof(T) || (uintptr_t)tau % sizeof(T) || (uintptr_t)buf_keys % 8 || (uintptr_t)counts % 32)
         return PROFK_EINVAL;
     int dev = 0;
     CUDA_TRY(cudaGetDevice(&dev));
     DeviceInfo di;
     const int rc = ensure_device_info<T>(dev, &di);
     if (rc != PROFK_OK) return rc;
-    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, (uint64_t)capacity, counts, 1, false, false, nullptr, false, 0u, nullptr, nullptr,
-                            static_cast<cudaStream_t>(stream));
+    // The same build of the kernel a whole call would pick for this density of survivors, estimated from the capacity
+    // (a plan's capacity is about twice the survivors it expects).
+    const double per_warp_tile = 0.5 * (double)capacity / (double)N * 32.0 * FILTER_UNROLL * Elem<T>::VEC;
+    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, (uint64_t)capacity, counts, PROFK_FILTER_COUNT_STRIDE, false, false, nullptr, false,
+                            0u, nullptr, nullptr, static_cast<cudaStream_t>(stream), defer_candidates<T>(rows, per_warp_tile));
 }
 
 template <typename T>
