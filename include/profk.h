@@ -113,10 +113,11 @@ enum {
  *             r_tight < r, after a recall failure with that of the LOOSER rank r_loose > r, into the same buffer
  *             with the same check k <= R <= M -- one more read of the row at streaming speed -- and only a row
  *             that fails again is selected exactly.  The ranks aim midway between k and M:
- *             r_tight = floor(r (k + M) / (2 M)), r_loose = r + ceil((M - k) m / (2 N)).  Used for calls of up
- *             to 18 rows with k <= 16384 (<= 8192 for up to four rows), where the exact selection runs inside
- *             the refine kernel, and only when the sample's keys are kept (up to four rows, or m <= 32768);
- *             other shapes go straight to the exact selection.
+ *             r_tight = floor(r (k + M) / (2 M)), r_loose = r + ceil((M - k) m / (2 N)).  Used for selections the
+ *             single-CTA refine orders (k <= 16384; <= 8192 for up to four rows) when the sample's keys are kept:
+ *             any sample for up to four rows, m <= 32768 for up to 18 rows, m <= 4096 for larger batches (there the
+ *             grid-wide repair kernel takes the pass, as long as fewer than eight rows of the call failed).  Larger
+ *             selections, the BatchTopK entry points and anything else go straight to the exact selection.
  * Both bounds are binomial tail bounds valid for the stratified sampler the
  * library uses (one uniform draw from each of m equal strata of the row).
  */

@@ -48,6 +48,10 @@ template <typename T> struct FallbackParams {
     uint32_t* cta_counters;   // gridDim.x counters
     uint32_t sort_cap;        // power of two >= k: records the dynamic shared memory holds
     int parallel;             // 1 = the one-row-per-CTA mode may be used (its scratch is there, or none is needed)
+    // The second filtering pass (second_chance.cuh) of a row that failed the check, taken by the whole grid before the
+    // exact selection when the rows are repaired one after the other here and ordered here (sort_rows == 1).
+    SampleInfo sample;        // sample.keys == null: none
+    uint4* thr2;              // rows threshold records of that pass
 };
 
 static_assert(FB_BINS <= RF_BINS, "the grid-wide selection's histogram lives in SelectShared::hist");
@@ -222,6 +226,46 @@ __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackPara
                 mask &= mask - 1;
                 const uint64_t row = chunk + w * 32 + b;
 
+                // ---- first another filtering pass with the plan's tighter / looser sample rank, if it names one ----
+                if (p.sort_rows && p.sample.keys != nullptr) {
+                    const uint32_t status = __ldcg(&p.ctl[row].status);
+                    const uint32_t rung = status == ROW_OVERFLOW ? p.sample.r_tight : status == ROW_RECALL ? p.sample.r_loose : 0u;
+                    if (rung != 0) {
+                        const SampleInfo& sm = p.sample;
+                        uint32_t key2, j2;
+                        kth_sample_record<T>(sm.keys + row * sm.S, sm.S, rung, sh, &key2, &j2);       // every CTA for itself
+                        const uint32_t idx2 = sm.by_record ? sample_element_index(j2, row, sm.seed, sm.q, sm.rem, sm.S, sm.inv_s) : 0xFFFFFFFFu;
+                        const T tau2 = Elem<T>::from_key(key2);
+                        if (tid == 0) {
+                            const uint32_t top = Elem<T>::KEY_BITS == 32 ? 0xFFFFFFFFu : 0xFFFFu;
+                            p.thr2[row] = make_uint4(Elem<T>::bits(tau2), Elem<T>::bits(Elem<T>::from_key(key2 == top ? key2 : key2 + 1u)), idx2, 0u);
+                        }
+                        __syncthreads();
+                        FilterParams<T> fp = {};
+                        fp.in = p.in; fp.N = p.N; fp.rows = row + 1; fp.tau = nullptr; fp.capacity = p.capacity;
+                        fp.buf = p.buf; fp.buf_stride = p.buf_stride;
+                        fp.counts = &p.ctl[0].pad; fp.count_stride = sizeof(RowCtl) / 4;
+                        fp.thr = p.thr2;
+                        refilter_tiles<T, FB_THREADS>(fp, (uint32_t)row, 0, p.tiles_per_row, blockIdx.x, gridDim.x, tau2);
+                        if (!grid_barrier(p.header, gen)) return;
+                        const uint32_t R2 = __ldcg(&p.ctl[row].pad);
+                        if (R2 >= p.k && R2 <= p.capacity) {           // (the same decision in every CTA)
+                            if (blockIdx.x == 0) {
+                                if (tid == 0) {
+                                    p.ctl[row].status = status == ROW_OVERFLOW ? ROW_OVERFLOW_REFILTERED : ROW_RECALL_REFILTERED;
+                                    p.ctl[row].count = R2;
+                                    p.ctl[row].tau_bits = Elem<T>::bits(tau2);
+                                    p.ctl[row].tau_idx = idx2;
+                                }
+                                extern __shared__ __align__(16) unsigned char fb_smem[];
+                                finish_from_segments<T>(p.buf + row * p.buf_stride, R2, p.k, p.sort_cap, reinterpret_cast<uint64_t*>(fb_smem), sh,
+                                                        row, p.out_vals, p.out_idx);
+                                __syncthreads();
+                            }
+                            continue;
+                        }
+                    }
+                }
                 // ---- exact selection of the k smallest records of `row` into the row's buffer ----
                 if (!grid_exact_select_row<T>(p, row, gen, sh_hist, warp_sums)) return;
                 uint64_t* dst = p.buf + row * p.buf_stride;

@@ -51,6 +51,7 @@ constexpr size_t REFINE_SMEM_MAX = 160 * 1024;   // dynamic shared memory the re
 constexpr int64_t N_MAX = 4278190080LL;          // 2^32 - 2^24
 constexpr int64_t M_MAX = 262144;                // largest sample the cluster select holds (8 CTAs x 32768 keys)
 constexpr int64_t KEPT_SAMPLE_MAX = 32768;       // largest sample whose keys are kept for a second filtering pass when there are more than GATHER_MAX_ROWS rows
+constexpr int64_t KEPT_SAMPLE_BATCH_MAX = 4096;  // the same for batches of more than XS_MAX_ROWS rows
 
 thread_local int g_launches = 0;
 thread_local void* g_ws_override_ptr = nullptr;   // set by the allocation-free entry point for the duration of its call
@@ -111,8 +112,8 @@ WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k, bool large) {
     // scratch of the grid-wide exact selection when it deals failed rows out one per CTA (many rows only)
     const bool fbp = rows > XS_MAX_ROWS && !large;
     // (up to GATHER_MAX_ROWS rows: room for the largest sample; up to XS_MAX_ROWS rows: for samples up to KEPT_SAMPLE_MAX,
-    // kept for the second filtering pass of a row that fails the count check)
-    const size_t keys_per_row = rows <= GATHER_MAX_ROWS ? (size_t)M_MAX : xs ? (size_t)KEPT_SAMPLE_MAX : 0;
+    // larger batches: up to KEPT_SAMPLE_BATCH_MAX -- kept for the second filtering pass of a row that fails the count check)
+    const size_t keys_per_row = rows <= GATHER_MAX_ROWS ? (size_t)M_MAX : xs ? (size_t)KEPT_SAMPLE_MAX : !large ? (size_t)KEPT_SAMPLE_BATCH_MAX : 0;
     l.off_fb_counters = align_up(l.off_keys + (size_t)rows * keys_per_row * sizeof(uint32_t), 256);
     l.off_fb_records = align_up(l.off_fb_counters + (fbp ? FB_MAX_CTAS * sizeof(uint32_t) : 0), 256);
     // counters of the partitioned append (large selections only), each in a 256-byte line of its own
@@ -522,8 +523,8 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
 
     // A second filtering pass for rows that fail the count check (plan->r_tight / r_loose) needs the sample's keys: they
     // are kept when the refine kernel's clusters do the repair and the workspace has room for them.
-    const bool keep_keys = exact_in_refine && plan->mode == 0 && (plan->r_tight > 0 || plan->r_loose > 0) &&
-                           (rows <= GATHER_MAX_ROWS || plan->m <= KEPT_SAMPLE_MAX);
+    const bool keep_keys = !large && plan->mode == 0 && (plan->r_tight > 0 || plan->r_loose > 0) &&
+                           (rows <= GATHER_MAX_ROWS || plan->m <= (rows <= XS_MAX_ROWS ? KEPT_SAMPLE_MAX : KEPT_SAMPLE_BATCH_MAX));
     SampleInfo sample = {};
     if (keep_keys) {
         sample.keys = keys_scratch; sample.S = (uint32_t)plan->m; sample.seed = seed;
@@ -546,6 +547,8 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     fb.cta_counters = fbp ? reinterpret_cast<uint32_t*>(base + lay.off_fb_counters) : nullptr;
     fb.sort_cap = fb_sort_cap;
     fb.parallel = (fbp || large) ? 1 : 0;      // large selections write into the rows' own buffers
+    fb.sample = keep_keys ? sample : SampleInfo{};
+    fb.thr2 = thr2;
     // A large selection from a single row: the count check, the exact replacement of a row that fails it and the
     // ordering are one cooperative kernel (three launches otherwise, two of which do nothing when no row failed).
     const bool fused_large = large && rows == 1;
@@ -695,7 +698,7 @@ int batchtopk_planned(const T* in, int64_t N, int64_t K, const profk_plan_t* pla
     bp.fb.ctl = ctl; bp.fb.header = header; bp.fb.ghist = ghist; bp.fb.buf = buf; bp.fb.buf_stride = row_stride; bp.fb.sort_rows = 0;
     bp.fb.tiles_per_row = tiles_per_row<T>((uint64_t)N, FB_THREADS * FB_UNROLL);
     bp.fb.use_pdl = 0; bp.fb.out_vals = nullptr; bp.fb.out_idx = nullptr; bp.fb.cta_records = nullptr; bp.fb.cta_counters = nullptr;
-    bp.fb.sort_cap = 0; bp.fb.parallel = 0;
+    bp.fb.sort_cap = 0; bp.fb.parallel = 0; bp.fb.sample = SampleInfo{}; bp.fb.thr2 = nullptr;
     bp.bins = bins;
     bp.coarse = ghist;                                            // (the exact selection and the select levels never both run)
     bp.edge = buf + row_stride / 2;                               // the scratch half of the row's buffer

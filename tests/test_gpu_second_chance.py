@@ -130,3 +130,44 @@ def test_a_billion_element_row_overflows_and_is_repaired_in_one_more_scan():
         times[name] = e0.elapsed_time(e1) / 5
     print("forced overflow at 2^30, ms per call:", times)
     assert times["second pass"] < 0.6 * times["exact selection"]
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_batches_repaired_by_the_grid_wide_kernel_take_the_second_pass_too(dtype):
+    """More than 18 rows: failed rows are repaired by the grid-wide kernel, one after the other when fewer than eight
+    failed.  A capacity just above the expected survivor count makes a few rows of the batch overflow; the tighter rank
+    brings most of them back, and every row's status, threshold and count follow the oracle."""
+    rows, n, k = 40, 1 << 18, 64
+    x = workloads.normal(rows, n, seed=86, dtype=dtype)
+    xn = workloads.as_numpy(x)
+    m, r = 2048, 16                                                           # 2048 survivors expected, sigma 512
+    found = None
+    for cap in (2560, 2688, 2816, 2944, 3072):                                # pick a capacity that 1..7 rows exceed
+        pl = profk.Plan(m=m, r=r, capacity=cap, k_accept=k, mode=0, r_tight=8)
+        first = [o_stages.run_row(xn[row], k, m, r, cap, k, seed=21, row=row, composite=True).status for row in range(rows)]
+        if 1 <= sum(s != o_stages.STATUS_OK for s in first) <= 7:
+            found = pl
+            break
+    assert found is not None, "no capacity with 1..7 failing rows: change the seed"
+    check(x, k, found, seed=21)
+    stats = profk.read_stats(rows)
+    assert any(s[3] == profk.ROW_OVERFLOW_REFILTERED for s in stats)
+    # recall failures in a few rows: rank 4 of 2048 keeps about 512, k = 250 is within reach of bad luck
+    k2 = 250
+    found = None
+    for r2 in (4, 3):
+        pl = profk.Plan(m=m, r=r2, capacity=4000, k_accept=k2, mode=0, r_loose=12)
+        first = [o_stages.run_row(xn[row], k2, m, r2, 4000, k2, seed=22, row=row, composite=True).status for row in range(rows)]
+        if 1 <= sum(s != o_stages.STATUS_OK for s in first) <= 7:
+            found = pl
+            break
+    assert found is not None, "no rank with 1..7 failing rows: change the seed"
+    check(x, k2, found, seed=22)
+    assert any(s[3] == profk.ROW_RECALL_REFILTERED for s in profk.read_stats(rows))
+    # eight or more failed rows are dealt out one per CTA and selected exactly at once: statuses 1 / 2 as before
+    pl = profk.Plan(m=m, r=r, capacity=1024, k_accept=k, mode=0, r_tight=8)
+    v, i = profk.topk(x.cuda(), k, plan_override=pl, seed=23)
+    torch.cuda.synchronize()
+    ov, oi = o_topk.topk(xn, k)
+    assert np.array_equal(i.cpu().numpy(), oi) and np.array_equal(bits(workloads.as_numpy(v)), bits(ov))
+    assert all(s[3] == profk.ROW_OVERFLOW for s in profk.read_stats(rows))
