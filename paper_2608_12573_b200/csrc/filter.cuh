@@ -368,24 +368,23 @@ __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T
 // DEFER build (many survivors: batches of short rows, dense selections).  With one or two survivors per warp-tile most
 // tiles would take the slow path above, whose few hundred warp instructions -- executed for the sake of one or two lanes
 // -- make the scan instruction-bound (359 warp instructions per bf16 warp-tile on 2^20-element rows with k = 32, against
-// 96 on the fast path).  Here a warp whose tile holds a candidate only NOTES it: four votes say which lanes hold an
-// element not below the threshold in which of their vectors, one shared-memory atomic reserves room, and each such lane
-// writes the number of its vector into a list in the CTA's shared memory -- a few dozen instructions, no global memory.
-// When the CTA has streamed all its tiles it works the list off with every lane busy: thread i reads candidate vector i
-// again (the candidates are a fraction of a percent of the input), decides its elements exactly and appends the
-// survivors.  A warp that finds the list full takes the slow path above instead.
+// 164 with no survivor at all).  Here a warp whose tile holds a candidate only NOTES it: the lanes that hold an element
+// not below the threshold -- one or two of the 32 as a rule -- reserve room with a shared-memory atomic and write the
+// numbers of their candidate vectors into a list in the CTA's shared memory; the other lanes do nothing, and no global
+// memory is touched.  When the CTA has streamed all its tiles it works the list off with every lane busy: thread i reads
+// candidate vector i again (the candidates are a few percent of the input at most), decides its elements exactly and
+// appends the survivors.  A warp that finds the list full takes the slow path above instead.
 #ifndef PROFK_DEFER_CAP
 #define PROFK_DEFER_CAP 6144
 #endif
 constexpr uint32_t DEFER_CAP = PROFK_DEFER_CAP;      // candidate vectors per CTA: 24 KB of shared memory
 constexpr uint32_t DEFER_NONE = 0xFFFFFFFFu;          // a reserved slot that was not used
 
-// One round of working the list off: lane by lane a candidate vector (number `vid` among the vectors of the launch,
+// One batch of 32 list entries worked off: lane by lane a candidate vector (number `vid` among the vectors of the launch,
 // tiles in order; DEFER_NONE = none) is read again and decided in the total order of the keys; the survivors are
-// appended with one atomic per warp when all of the warp's survivors belong to one row (the list is in tile order, so
-// they nearly always do), else with one per lane.  All 32 lanes call it.
+// appended with one atomic per row that has survivors among them.  All 32 lanes call it.
 template <typename T, int THREADS, int UNROLL, bool PARTS>
-__device__ __forceinline__ void defer_process_round(const FilterParams<T>& p, uint32_t vid) {
+__device__ __forceinline__ void defer_process_batch(const FilterParams<T>& p, uint32_t vid) {
     using V = typename Elem<T>::vec_t;
     constexpr int VEC = Elem<T>::VEC;
     constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
@@ -415,7 +414,7 @@ __device__ __forceinline__ void defer_process_round(const FilterParams<T>& p, ui
             m = confirm_survivors<T>(p, row, v, m, i0, tau);
         }
     }
-    // Append, one atomic per row that has survivors in this round (a round of 32 consecutive entries spans a tile or two,
+    // Append, one atomic per row that has survivors in this batch (32 consecutive entries of the list span a tile or two,
     // so one or two rows): the lanes of the first row with survivors form a group, scan their counts, their first lane
     // reserves the room; then the next row's lanes, until none is left.
     const unsigned cnt = __popc(m);
@@ -680,9 +679,9 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
         // every tile of this CTA has been streamed: work the list off, one entry per thread
         __syncthreads();
         const uint32_t n = s_nhits < DEFER_CAP ? s_nhits : DEFER_CAP;
-        for (uint32_t e0 = 0; e0 < n; e0 += THREADS) {          // whole warps take part in every round
+        for (uint32_t e0 = 0; e0 < n; e0 += THREADS) {          // whole warps take part in every batch
             const uint32_t e = e0 + threadIdx.x;
-            if (e0 + (threadIdx.x & ~31u) < n) defer_process_round<T, THREADS, UNROLL, PARTS>(p, e < n ? hits[e] : DEFER_NONE);
+            if (e0 + (threadIdx.x & ~31u) < n) defer_process_batch<T, THREADS, UNROLL, PARTS>(p, e < n ? hits[e] : DEFER_NONE);
         }
     }
     if (pf_pending) prefetch_landed(PREFETCH_SPIN_LIMIT);
