@@ -354,8 +354,10 @@ template <typename T>
 int launch_refine_large(const DeviceInfo& di, RowCtl* ctl, WsHeader* header, uint64_t* buf, uint64_t row_pitch, uint32_t* bins,
                         unsigned long long* slots, bool parts, uint32_t part_cap, const uint32_t* part_counts, int64_t rows,
                         int64_t capacity, int64_t k, int64_t k_accept, int phase, T* out_vals, int64_t* out_idx, cudaStream_t st,
-                        const FallbackParams<T>* fused_fb = nullptr, bool after_kernel = true) {
+                        const FallbackParams<T>* fused_fb = nullptr, bool after_kernel = true, int64_t N = 0) {
     LargeParams<T> lp;
+    lp.idx_bits = 32;                            // (N unknown: every bit of the index word may be used)
+    if (N > 1) { lp.idx_bits = 1; while (((int64_t)1 << lp.idx_bits) < N) ++lp.idx_bits; }
     lp.fused = fused_fb ? 1 : 0;
     if (fused_fb) lp.fb = *fused_fb; else lp.fb = FallbackParams<T>{};
     lp.ctl = ctl; lp.header = header; lp.buf = buf; lp.row_stride = row_pitch / 2; lp.bins = bins; lp.slots = slots;
@@ -564,7 +566,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
 
         if (large) {
             rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, reinterpret_cast<unsigned long long*>(ghist), parts, part_cap, part_counts, rows,
-                                        capacity, k, plan->k_accept, 0, out_vals, out_idx, st, fused_large ? &fb : nullptr);
+                                        capacity, k, plan->k_accept, 0, out_vals, out_idx, st, fused_large ? &fb : nullptr, true, N);
             if (fused_large) return rc;
         } else {
             // count check and refine; with clusters, also the exact selection of the rows that fail the check
@@ -580,7 +582,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
             return launch_refine<T>(di, in, rows, N, ctl, header, buf, row_stride, capacity, k, k, true, csize, xs_records, xs_counters, out_vals, out_idx, st);
         if (fused_large)
             return launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, reinterpret_cast<unsigned long long*>(ghist), false, part_cap, part_counts, rows,
-                                          capacity, k, k, 0, out_vals, out_idx, st, &fb, false);
+                                          capacity, k, k, 0, out_vals, out_idx, st, &fb, false, N);
     }
 
     if (!exact_in_refine) {
@@ -598,7 +600,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     if (large) {   // the rows the exact selection repaired still have to be ordered and written
         rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, reinterpret_cast<unsigned long long*>(ghist), false, part_cap, part_counts, rows,
                                     capacity, k, k, 1, out_vals,
-                                    out_idx, st);
+                                    out_idx, st, nullptr, true, N);
         if (rc != PROFK_OK) return rc;
     }
     return PROFK_OK;

@@ -52,6 +52,7 @@ template <typename T> struct LargeParams {
     // inside this kernel by the grid-wide exact selection and ordered right away -- one launch instead of three.
     int fused;
     FallbackParams<T> fb;    // what that selection needs (fused == 1 only)
+    int idx_bits;            // bits an index of the row occupies (1 .. 32)
 };
 
 // All exchanges of the network with stride < BT_TILE, for one tile held in shared memory.
@@ -214,9 +215,17 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
             rmin = l2 < rmin ? l2 : rmin;
             rmax = h2 > rmax ? h2 : rmax;
         }
-        const int rbits = 64 - __clzll((long long)(rmax - rmin));    // range < 2^rbits
+        // Bins on the top LG_BITS bits of the records' range.  A record holds the value key above a 32-bit index, but the
+        // indices of a row only need idx_bits bits: the unused bits in between are squeezed out first (the order is kept),
+        // so that they go to the index instead -- equal values, which differ in the index alone, then spread over 2^(32 -
+        // idx_bits) times as many bins (bf16 rows hold thousands of copies of one value near the threshold: at the
+        // paper's SAE shape a bin held about 800 records and ranking inside the bins took most of the kernel).
+        const int ib = p.idx_bits;
+        const unsigned long long hmin = rmin >> 32;
+        auto squeeze = [&](unsigned long long rec) { return (((rec >> 32) - hmin) << ib) | (rec & 0xFFFFFFFFull); };
+        const int rbits = 64 - __clzll((long long)squeeze(rmax));    // squeezed records < 2^rbits
         const int shift = rbits > LG_BITS ? rbits - LG_BITS : 0;
-        auto bin_of = [&](unsigned long long rec) { return (uint32_t)((rec - rmin) >> shift); };
+        auto bin_of = [&](unsigned long long rec) { return (uint32_t)(squeeze(rec) >> shift); };
 
         // histogram (global atomics spread over the bins)
         for_each_record([&](unsigned long long rec) { atomicAdd(&bins[bin_of(rec)], 1u); });
