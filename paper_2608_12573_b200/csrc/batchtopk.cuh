@@ -7,8 +7,9 @@
 // One cooperative kernel (one CTA per SM, all co-resident, bounded grid barriers) does stage 4 in that form:
 //   * the count check of Section 3, "Refinement"; a row that fails it is replaced on the spot by the exact selection
 //     of the whole row (grid_exact_select_row), which leaves exactly K records -- all of them kept;
-//   * otherwise a histogram select over the R candidate records.  A record r is at distance D = T - r below the
-//     largest record the filter can have kept (T = tau's key with an all-ones index), larger D = better record.
+//   * otherwise a histogram select over the R candidate records.  A record r is at distance D below the largest
+//     record the filter can have kept (tau's key with the last index; the index word's unused bits squeezed out),
+//     larger D = better record.
 //     Level 0 bins D on a logarithmic scale (6 bits of exponent, 12 of mantissa: 2^18 bins in global memory, fine
 //     where records are dense) and, through shared memory, into 512 coarse bins; after ONE grid barrier every CTA
 //     scans the coarse bins and then the 512 fine bins of the one that holds the K-th best record; if that bin is crowded (many equal values: its records differ only in the index)
@@ -168,9 +169,16 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
     if (p.dense) bk_zero_fill(p.dense, fb.N, gid, gthreads);
 
     // ---- the class of the K-th best record ----
-    // D = top - record >= 0 for every record the filter kept (their keys are >= tau's); larger D = better record.
+    // D = distance of a record below `top`, the largest record the filter can have kept (tau's key, the last index);
+    // D >= 0 for every kept record (their keys are >= tau's), larger D = better record.  A record holds the key above a
+    // 32-bit index word of which a row only uses idx_bits bits; the unused bits are squeezed out of D, so that the bits
+    // right below the key difference are real index bits: thousands of copies of one bf16 value then spread over the
+    // logarithmic level's bins instead of crowding one (which costs further levels).
     const uint32_t tau_key = Elem<T>::key(Elem<T>::from_bits(__ldcg(&fb.ctl[0].tau_bits)));
     const uint64_t top = make_record(tau_key, 0xFFFFFFFFu);
+    const int idx_bits = fb.N > 1 ? 64 - __clzll((long long)(fb.N - 1)) : 1;
+    const uint64_t idx_top = (1ull << idx_bits) - 1ull;
+    auto dist = [&](uint64_t rec) { return (((top >> 32) - (rec >> 32)) << idx_bits) | (idx_top - (rec & 0xFFFFFFFFull)); };
     uint64_t cls_lo = 0;          // the boundary class is cls_lo <= D < cls_lo + 2^cls_w ...
     int cls_w = 64;               // ... (64: every D)
     uint32_t need = K;            // ... and its `need` best records are kept, with every record of a better class
@@ -207,7 +215,7 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
         __syncthreads();
         for (uint64_t i = gid; i < total; i += gthreads) {
             bool in_class;
-            const uint32_t f = BK_BINS - 1 - bin_of(top - record_at(i), &in_class);
+            const uint32_t f = BK_BINS - 1 - bin_of(dist(record_at(i)), &in_class);
             if (in_class) {
                 atomicAdd(&p.bins[f], 1u);
                 atomicAdd(&s_coarse[f / BK_PER_COARSE], 1u);
@@ -266,7 +274,7 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
         bool kept = false, boundary = false;
         if (i < total) {
             rec = record_at(i);
-            const uint64_t D = top - rec;
+            const uint64_t D = dist(rec);
             kept = keep_all || (whole ? D >= keep_from : (!top_class && D >= keep_from));
             boundary = !kept && !whole && D >= cls_lo;
         }
