@@ -113,11 +113,13 @@ enum {
  *             r_tight < r, after a recall failure with that of the LOOSER rank r_loose > r, into the same buffer
  *             with the same check k <= R <= M -- one more read of the row at streaming speed -- and only a row
  *             that fails again is selected exactly.  The ranks aim midway between k and M:
- *             r_tight = floor(r (k + M) / (2 M)), r_loose = r + ceil((M - k) m / (2 N)).  Used for selections the
- *             single-CTA refine orders (k <= 16384; <= 8192 for up to four rows) when the sample's keys are kept:
- *             any sample for up to four rows, m <= 32768 for up to 18 rows, m <= 4096 for larger batches (there the
- *             grid-wide repair kernel takes the pass, as long as fewer than eight rows of the call failed).  Larger
- *             selections, the BatchTopK entry points and anything else go straight to the exact selection.
+ *             r_tight = floor(r (k + M) / (2 M)), r_loose = r + ceil((M - k) m / (2 N)).  Used when the sample's keys
+ *             are kept: for selections the single-CTA refine orders (k <= 16384; <= 8192 for up to four rows) any
+ *             sample for up to four rows, m <= 32768 for up to 18 rows, m <= 4096 for larger batches (there the
+ *             grid-wide repair kernel takes the pass, as long as fewer than eight rows of the call failed); for
+ *             larger selections a single row (profk_topk_* with rows == 1, and the BatchTopK entry points, whose
+ *             one kernel after the filter takes the pass itself).  Larger selections from several rows and
+ *             anything else go straight to the exact selection.
  * Both bounds are binomial tail bounds valid for the stratified sampler the
  * library uses (one uniform draw from each of m equal strata of the row).
  */

@@ -139,13 +139,20 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
         }
     }
     bool keep_all = false;                        // every record in the buffer is kept (it holds exactly K)
+    uint32_t tau_key = 0;
     if (status != ROW_OK) {
-        // The exact replacement (Section 3, "Refinement"): the K best records of the whole row, into the buffer.
-        if (!grid_exact_select_row<T>(fb, 0, gen, sh.hist, sh.warp_sums)) return;
+        // A second filtering pass with the plan's tighter / looser sample rank first, if it names one ...
+        uint32_t R2 = 0;
+        const int again = p.direct ? 0 : grid_second_chance_row<T>(fb, 0, status, gen, sh, &R2, &tau_key);
+        if (again < 0) return;
+        // ... else the exact replacement (Section 3, "Refinement"): the K best records of the whole row, into the buffer.
+        if (again == 0 && !grid_exact_select_row<T>(fb, 0, gen, sh.hist, sh.warp_sums)) return;
 #pragma unroll
         for (int j = 0; j < (int)FILTER_PARTS; ++j) pcount[j] = 0;
-        pcount[0] = K;
-        keep_all = true;
+        pcount[0] = again == 1 ? R2 : K;
+        keep_all = again == 0;
+    } else {
+        tau_key = Elem<T>::key(Elem<T>::from_bits(__ldcg(&fb.ctl[0].tau_bits)));
     }
     uint32_t pend[FILTER_PARTS];                  // pend[j] = records in parts 0..j
     {
@@ -174,7 +181,6 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
     // 32-bit index word of which a row only uses idx_bits bits; the unused bits are squeezed out of D, so that the bits
     // right below the key difference are real index bits: thousands of copies of one bf16 value then spread over the
     // logarithmic level's bins instead of crowding one (which costs further levels).
-    const uint32_t tau_key = Elem<T>::key(Elem<T>::from_bits(__ldcg(&fb.ctl[0].tau_bits)));
     const uint64_t top = make_record(tau_key, 0xFFFFFFFFu);
     const int idx_bits = fb.N > 1 ? 64 - __clzll((long long)(fb.N - 1)) : 1;
     const uint64_t idx_top = (1ull << idx_bits) - 1ull;

@@ -49,7 +49,8 @@ template <typename T> struct FallbackParams {
     uint32_t sort_cap;        // power of two >= k: records the dynamic shared memory holds
     int parallel;             // 1 = the one-row-per-CTA mode may be used (its scratch is there, or none is needed)
     // The second filtering pass (second_chance.cuh) of a row that failed the check, taken by the whole grid before the
-    // exact selection when the rows are repaired one after the other here and ordered here (sort_rows == 1).
+    // exact selection: when the rows are repaired one after the other by the kernel below and ordered there
+    // (sort_rows == 1), and by the fused large-selection kernels for their single row.
     SampleInfo sample;        // sample.keys == null: none
     uint4* thr2;              // rows threshold records of that pass
 };
@@ -168,6 +169,50 @@ __device__ __noinline__ bool grid_exact_select_row(const FallbackParams<T>& p, u
     return grid_barrier(p.header, gen);
 }
 
+// The second filtering pass (second_chance.cuh) of a row that failed the count check with `status`, by the whole grid:
+// every CTA selects the plan's tighter (overflow) or looser (too few candidates) sample rank from the kept keys for
+// itself, the grid filters the row once more into the row's buffer (from its start; counter: the row's `pad` word, zero
+// on entry), one grid barrier, and every CTA takes the same count check.  Returns 1 when the row passed it: the buffer
+// holds *R2 records, k <= *R2 <= capacity, *key2 is the order key of the threshold used, and the row's control block
+// says so; 0 when no second pass applies (no keys kept, no such rank in the plan) or the row failed again; -1 when a
+// bounded wait gave up (the caller leaves the kernel).  Called by every thread of every CTA (FB_THREADS threads).
+template <typename T>
+__device__ __noinline__ int grid_second_chance_row(const FallbackParams<T>& p, uint64_t row, uint32_t status, uint32_t& gen, SelectShared& sh,
+                                                   uint32_t* R2_out, uint32_t* key2_out) {
+    const SampleInfo& sm = p.sample;
+    if (sm.keys == nullptr) return 0;
+    const uint32_t rung = status == ROW_OVERFLOW ? sm.r_tight : status == ROW_RECALL ? sm.r_loose : 0u;
+    if (rung == 0) return 0;
+    const unsigned tid = threadIdx.x;
+    uint32_t key2, j2;
+    kth_sample_record<T>(sm.keys + row * sm.S, sm.S, rung, sh, &key2, &j2);       // every CTA for itself
+    const uint32_t idx2 = sm.by_record ? sample_element_index(j2, row, sm.seed, sm.q, sm.rem, sm.S, sm.inv_s) : 0xFFFFFFFFu;
+    const T tau2 = Elem<T>::from_key(key2);
+    if (tid == 0) {
+        const uint32_t top = Elem<T>::KEY_BITS == 32 ? 0xFFFFFFFFu : 0xFFFFu;
+        p.thr2[row] = make_uint4(Elem<T>::bits(tau2), Elem<T>::bits(Elem<T>::from_key(key2 == top ? key2 : key2 + 1u)), idx2, 0u);
+    }
+    __syncthreads();
+    FilterParams<T> fp = {};
+    fp.in = p.in; fp.N = p.N; fp.rows = row + 1; fp.tau = nullptr; fp.capacity = p.capacity;
+    fp.buf = p.buf; fp.buf_stride = p.buf_stride;
+    fp.counts = &p.ctl[0].pad; fp.count_stride = sizeof(RowCtl) / 4;
+    fp.thr = p.thr2;
+    refilter_tiles<T, FB_THREADS>(fp, (uint32_t)row, 0, p.tiles_per_row, blockIdx.x, gridDim.x, tau2);
+    if (!grid_barrier(p.header, gen)) return -1;
+    const uint32_t R2 = __ldcg(&p.ctl[row].pad);
+    if (R2 < p.k || R2 > p.capacity) return 0;                 // (the same decision in every CTA)
+    if (blockIdx.x == 0 && tid == 0) {
+        p.ctl[row].status = status == ROW_OVERFLOW ? ROW_OVERFLOW_REFILTERED : ROW_RECALL_REFILTERED;
+        p.ctl[row].count = R2;
+        p.ctl[row].tau_bits = Elem<T>::bits(tau2);
+        p.ctl[row].tau_idx = idx2;
+    }
+    *R2_out = R2;
+    *key2_out = key2;
+    return 1;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackParams<T> p) {
     __shared__ SelectShared sh;                 // the per-CTA selection's state; its arrays also serve the grid-wide one
@@ -227,43 +272,18 @@ __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackPara
                 const uint64_t row = chunk + w * 32 + b;
 
                 // ---- first another filtering pass with the plan's tighter / looser sample rank, if it names one ----
-                if (p.sort_rows && p.sample.keys != nullptr) {
-                    const uint32_t status = __ldcg(&p.ctl[row].status);
-                    const uint32_t rung = status == ROW_OVERFLOW ? p.sample.r_tight : status == ROW_RECALL ? p.sample.r_loose : 0u;
-                    if (rung != 0) {
-                        const SampleInfo& sm = p.sample;
-                        uint32_t key2, j2;
-                        kth_sample_record<T>(sm.keys + row * sm.S, sm.S, rung, sh, &key2, &j2);       // every CTA for itself
-                        const uint32_t idx2 = sm.by_record ? sample_element_index(j2, row, sm.seed, sm.q, sm.rem, sm.S, sm.inv_s) : 0xFFFFFFFFu;
-                        const T tau2 = Elem<T>::from_key(key2);
-                        if (tid == 0) {
-                            const uint32_t top = Elem<T>::KEY_BITS == 32 ? 0xFFFFFFFFu : 0xFFFFu;
-                            p.thr2[row] = make_uint4(Elem<T>::bits(tau2), Elem<T>::bits(Elem<T>::from_key(key2 == top ? key2 : key2 + 1u)), idx2, 0u);
+                if (p.sort_rows) {
+                    uint32_t R2 = 0, key2 = 0;
+                    const int again = grid_second_chance_row<T>(p, row, __ldcg(&p.ctl[row].status), gen, sh, &R2, &key2);
+                    if (again < 0) return;
+                    if (again == 1) {
+                        if (blockIdx.x == 0) {
+                            extern __shared__ __align__(16) unsigned char fb_smem[];
+                            finish_from_segments<T>(p.buf + row * p.buf_stride, R2, p.k, p.sort_cap, reinterpret_cast<uint64_t*>(fb_smem), sh,
+                                                    row, p.out_vals, p.out_idx);
+                            __syncthreads();
                         }
-                        __syncthreads();
-                        FilterParams<T> fp = {};
-                        fp.in = p.in; fp.N = p.N; fp.rows = row + 1; fp.tau = nullptr; fp.capacity = p.capacity;
-                        fp.buf = p.buf; fp.buf_stride = p.buf_stride;
-                        fp.counts = &p.ctl[0].pad; fp.count_stride = sizeof(RowCtl) / 4;
-                        fp.thr = p.thr2;
-                        refilter_tiles<T, FB_THREADS>(fp, (uint32_t)row, 0, p.tiles_per_row, blockIdx.x, gridDim.x, tau2);
-                        if (!grid_barrier(p.header, gen)) return;
-                        const uint32_t R2 = __ldcg(&p.ctl[row].pad);
-                        if (R2 >= p.k && R2 <= p.capacity) {           // (the same decision in every CTA)
-                            if (blockIdx.x == 0) {
-                                if (tid == 0) {
-                                    p.ctl[row].status = status == ROW_OVERFLOW ? ROW_OVERFLOW_REFILTERED : ROW_RECALL_REFILTERED;
-                                    p.ctl[row].count = R2;
-                                    p.ctl[row].tau_bits = Elem<T>::bits(tau2);
-                                    p.ctl[row].tau_idx = idx2;
-                                }
-                                extern __shared__ __align__(16) unsigned char fb_smem[];
-                                finish_from_segments<T>(p.buf + row * p.buf_stride, R2, p.k, p.sort_cap, reinterpret_cast<uint64_t*>(fb_smem), sh,
-                                                        row, p.out_vals, p.out_idx);
-                                __syncthreads();
-                            }
-                            continue;
-                        }
+                        continue;
                     }
                 }
                 // ---- exact selection of the k smallest records of `row` into the row's buffer ----

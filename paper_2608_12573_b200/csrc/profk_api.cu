@@ -524,8 +524,9 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     while (fb_sort_cap < (uint32_t)k && fb_sort_cap < SORT_CAP_MAX) fb_sort_cap <<= 1;
 
     // A second filtering pass for rows that fail the count check (plan->r_tight / r_loose) needs the sample's keys: they
-    // are kept when the refine kernel's clusters do the repair and the workspace has room for them.
-    const bool keep_keys = !large && plan->mode == 0 && (plan->r_tight > 0 || plan->r_loose > 0) &&
+    // are kept when the workspace has room for them and a kernel that takes that pass does the repair: the refine
+    // kernel's clusters, the grid-wide repair kernel, or the fused kernel of a large selection from a single row.
+    const bool keep_keys = (!large || rows == 1) && plan->mode == 0 && (plan->r_tight > 0 || plan->r_loose > 0) &&
                            (rows <= GATHER_MAX_ROWS || plan->m <= (rows <= XS_MAX_ROWS ? KEPT_SAMPLE_MAX : KEPT_SAMPLE_BATCH_MAX));
     SampleInfo sample = {};
     if (keep_keys) {
@@ -652,6 +653,7 @@ int batchtopk_planned(const T* in, int64_t N, int64_t K, const profk_plan_t* pla
     if (plan->mode == 0) {
         if (plan->m < 1 || plan->m > std::min<int64_t>(N, M_MAX) || plan->r < 1 || plan->r > plan->m) return PROFK_EINVAL;
         if (plan->k_accept != K) return PROFK_EINVAL;          // the kept set has exactly K members: no relaxed mode
+        if (plan->r_tight < 0 || plan->r_tight > plan->m || plan->r_loose < 0 || plan->r_loose > plan->m) return PROFK_EINVAL;
     }
     int dev = 0;
     CUDA_TRY(cudaGetDevice(&dev));
@@ -685,7 +687,8 @@ int batchtopk_planned(const T* in, int64_t N, int64_t K, const profk_plan_t* pla
 
     if (plan->mode == 0) {
         rc = launch_sample_select<T>(di, in, 1, N, plan->m, plan->r, seed, nullptr, ctl, header, (uint32_t)capacity, nullptr, keys_scratch,
-                                     parts ? part_counts : nullptr, plan->tie_rule == PROFK_TIES_BY_INDEX, thr, st);
+                                     parts ? part_counts : nullptr, plan->tie_rule == PROFK_TIES_BY_INDEX, thr, st, nullptr,
+                                     (plan->r_tight > 0 || plan->r_loose > 0) ? keys_scratch : nullptr);
         if (rc != PROFK_OK) return rc;
         rc = launch_filter<T>(di, in, 1, N, nullptr, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, &header->tile_counter,
                               parts, part_cap, part_counts, thr, st, deferred);
@@ -700,7 +703,18 @@ int batchtopk_planned(const T* in, int64_t N, int64_t K, const profk_plan_t* pla
     bp.fb.ctl = ctl; bp.fb.header = header; bp.fb.ghist = ghist; bp.fb.buf = buf; bp.fb.buf_stride = row_stride; bp.fb.sort_rows = 0;
     bp.fb.tiles_per_row = tiles_per_row<T>((uint64_t)N, FB_THREADS * FB_UNROLL);
     bp.fb.use_pdl = 0; bp.fb.out_vals = nullptr; bp.fb.out_idx = nullptr; bp.fb.cta_records = nullptr; bp.fb.cta_counters = nullptr;
-    bp.fb.sort_cap = 0; bp.fb.parallel = 0; bp.fb.sample = SampleInfo{}; bp.fb.thr2 = nullptr;
+    bp.fb.sort_cap = 0; bp.fb.parallel = 0;
+    // the sample's keys stay in the workspace for a second filtering pass of a row that fails the count check
+    const bool keep_keys = plan->mode == 0 && (plan->r_tight > 0 || plan->r_loose > 0);
+    bp.fb.sample = SampleInfo{};
+    if (keep_keys) {
+        SampleInfo& sm = bp.fb.sample;
+        sm.keys = keys_scratch; sm.S = (uint32_t)plan->m; sm.seed = seed;
+        sm.q = (uint64_t)(N / plan->m); sm.rem = (uint32_t)(N % plan->m); sm.inv_s = 1.0f / (float)plan->m;
+        sm.by_record = plan->tie_rule == PROFK_TIES_BY_INDEX ? 1 : 0;
+        sm.r_tight = (uint32_t)plan->r_tight; sm.r_loose = (uint32_t)plan->r_loose;
+    }
+    bp.fb.thr2 = reinterpret_cast<uint4*>(base + lay.off_tau2);
     bp.bins = bins;
     bp.coarse = ghist;                                            // (the exact selection and the select levels never both run)
     bp.edge = buf + row_stride / 2;                               // the scratch half of the row's buffer

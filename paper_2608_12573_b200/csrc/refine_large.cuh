@@ -135,12 +135,17 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
             n = R;
             if (status != ROW_OK) {
                 if (!p.fused) continue;          // the exact-selection kernel and the second phase take this row
-                // the k best records of the whole row into the row's buffer, then ordered below like any buffer
-                if (!grid_exact_select_row<T>(p.fb, row, grid_gen, reinterpret_cast<uint32_t*>(tile), s_warp)) return;
+                // first a second filtering pass with the plan's tighter / looser sample rank, if it names one (the tile in
+                // shared memory, unused so far, holds that pass's selection state) ...
+                uint32_t R2 = 0, key2 = 0;
+                const int again = direct ? 0 : grid_second_chance_row<T>(p.fb, row, status, grid_gen, *reinterpret_cast<SelectShared*>(smem_raw), &R2, &key2);
+                if (again < 0) return;
+                // ... else the k best records of the whole row into the row's buffer; ordered below like any buffer
+                if (again == 0 && !grid_exact_select_row<T>(p.fb, row, grid_gen, reinterpret_cast<uint32_t*>(tile), s_warp)) return;
                 nparts = 1;
 #pragma unroll
                 for (int j = 0; j < (int)FILTER_PARTS; ++j) pcount[j] = 0;
-                pcount[0] = n = p.k;
+                pcount[0] = n = again == 1 ? R2 : p.k;
             }
         } else {
             if (ctl.status == ROW_OK) continue;  // already written by the first phase

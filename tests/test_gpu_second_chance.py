@@ -171,3 +171,46 @@ def test_batches_repaired_by_the_grid_wide_kernel_take_the_second_pass_too(dtype
     ov, oi = o_topk.topk(xn, k)
     assert np.array_equal(i.cpu().numpy(), oi) and np.array_equal(bits(workloads.as_numpy(v)), bits(ov))
     assert all(s[3] == profk.ROW_OVERFLOW for s in profk.read_stats(rows))
+
+
+def _btk_forms(xn, k, out):
+    """The BatchTopK forms in `out` against the oracle's kept set of the host row xn."""
+    want = o_topk.kept_mask(xn, k)
+    idx = out["indices"].cpu().numpy()
+    assert np.array_equal(np.sort(idx), np.flatnonzero(want)), "kept indices differ from the oracle's set"
+    assert np.array_equal(bits(workloads.as_numpy(out["values"])), bits(xn[idx]))
+    assert np.array_equal(out["mask"].cpu().numpy().view(np.uint32), o_topk.pack_mask(want))
+    dense = np.zeros_like(xn)
+    dense[want] = xn[want]
+    assert np.array_equal(bits(workloads.as_numpy(out["dense"]).reshape(-1)), bits(dense))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_large_selections_from_one_row_take_the_second_pass_inside_their_fused_kernels(dtype):
+    """k beyond what one CTA orders: the ordering kernel of `profk_topk_*` and the emit kernel of `profk_batchtopk_*`
+    repair their single row themselves, with the same second filtering pass before the exact selection."""
+    n, k, m = 3_000_001, 20_000, 65536                                        # a sample rank keeps about 45.8 elements
+    x = workloads.normal(1, n, seed=87, dtype=dtype)[0]
+    xn = workloads.as_numpy(x)
+    cap = 34_000
+    cases = [
+        (profk.Plan(m=m, r=1000, capacity=cap, k_accept=k, mode=0, r_tight=600), profk.ROW_OVERFLOW_REFILTERED),   # 45.8 K, then 27.5 K
+        (profk.Plan(m=m, r=1000, capacity=cap, k_accept=k, mode=0, r_tight=990), profk.ROW_OVERFLOW),              # overflows again
+        (profk.Plan(m=m, r=1000, capacity=cap, k_accept=k, mode=0), profk.ROW_OVERFLOW),                           # no rank named
+        (profk.Plan(m=m, r=300, capacity=cap, k_accept=k, mode=0, r_loose=600), profk.ROW_RECALL_REFILTERED),      # 13.7 K, then 27.5 K
+        (profk.Plan(m=m, r=300, capacity=cap, k_accept=k, mode=0, r_loose=310), profk.ROW_RECALL),                 # too few again
+        (profk.Plan(m=m, r=1000, capacity=cap, k_accept=k, mode=0, r_tight=600, tie_rule=profk.TIES_KEEP_ALL), None),
+    ]
+    for seed, (pl, want) in enumerate(cases):
+        check(x, k, pl, seed=30 + seed, want_status=want)
+        ordered = profk.read_stats(1)[0]
+        out = profk.batchtopk(x.cuda(), k, seed=30 + seed, want_pairs=True, want_mask=True, want_dense=True, plan_override=pl)
+        torch.cuda.synchronize()
+        _btk_forms(xn, k, out)
+        assert profk.read_stats(1)[0] == ordered                             # same stages, same threshold, count and status
+    # in place: the second pass and the exact selection read the input before the dense form overwrites it
+    xc = x.cuda().clone()
+    out = profk.batchtopk(xc, k, seed=30, want_pairs=True, want_mask=True, in_place=True, plan_override=cases[0][0])
+    torch.cuda.synchronize()
+    _btk_forms(xn, k, out)
+    assert profk.read_stats(1)[0][3] == profk.ROW_OVERFLOW_REFILTERED
