@@ -7,12 +7,13 @@
 // One cooperative kernel (one CTA per SM, all co-resident, bounded grid barriers) does stage 4 in that form:
 //   * the count check of Section 3, "Refinement"; a row that fails it is replaced on the spot by the exact selection
 //     of the whole row (grid_exact_select_row), which leaves exactly K records -- all of them kept;
-//   * otherwise a histogram select over the R candidate records.  A record r is at distance D below the largest
-//     record the filter can have kept (tau's key with the last index; the index word's unused bits squeezed out),
-//     larger D = better record.
-//     Level 0 bins D on a logarithmic scale (6 bits of exponent, 12 of mantissa: 2^18 bins in global memory, fine
-//     where records are dense) and, through shared memory, into 512 coarse bins; after ONE grid barrier every CTA
-//     scans the coarse bins and then the 512 fine bins of the one that holds the K-th best record; if that bin is crowded (many equal values: its records differ only in the index)
+//   * otherwise a histogram select over the R candidate records in the bins of bins.cuh (distance D below the largest
+//     record the filter can have kept, on a logarithmic scale: 2^18 fine bins in global memory, 512 coarse ones).
+//     Level 0 is counted by the filter kernel itself as it appends the records (its HIST build), so this kernel starts
+//     with the histogram made and no grid barrier at all when only the pairs are wanted; a call whose filter did not
+//     count (or whose row was filtered a second time) counts here: fine bins with global atomics, coarse bins through
+//     shared memory, ONE grid barrier.  Every CTA then scans the coarse bins and the 512 fine bins of the one that
+//     holds the K-th best record; if that bin is crowded (many equal values: its records differ only in the index)
 //     the next levels bin its D range linearly, 18 bits at a time, until at most BK_EDGE records are left in the
 //     boundary class;
 //   * the emit pass: every record of a better class is kept; the boundary class is copied to a short list, and the CTA
@@ -25,20 +26,20 @@
 namespace profk {
 
 constexpr int BK_THREADS = FB_THREADS;          // the exact selection it may call is written for this CTA size
-constexpr int BK_BITS = 18;
-constexpr uint32_t BK_BINS = 1u << BK_BITS;
-constexpr uint32_t BK_FLAGS = 8;                // words after the bins: [0] pairs appended, [1] records in the boundary list, [2] CTAs done emitting
+constexpr int BK_BITS = BIN_BITS;
+constexpr uint32_t BK_BINS = BIN_COUNT;
+// the flag words after the bins: [0] pairs appended, [1] records in the boundary list, [2] CTAs done emitting
 constexpr uint32_t BK_EDGE = 1024;              // a boundary class up to this size is ranked directly
-constexpr uint32_t BK_COARSE = 512;             // coarse bins, each the sum of BK_BINS / BK_COARSE = 512 fine ones
-constexpr uint32_t BK_PER_COARSE = BK_BINS / BK_COARSE;
+constexpr uint32_t BK_COARSE = BIN_COARSE;
+constexpr uint32_t BK_PER_COARSE = BIN_PER_COARSE;
 static_assert(BK_COARSE <= BK_THREADS && BK_PER_COARSE <= BK_THREADS, "one thread per coarse bin, then per fine bin of one coarse bin");
 constexpr uint32_t BK_WAIT_LIMIT = 1u << 22;    // polls of the "all CTAs have zeroed their share of the bins" counter
 constexpr int BK_MAX_LEVELS = 6;                // 12 + 18 * 3 > 64 bits: more levels than any input needs
 
 template <typename T> struct BatchTopkParams {
     FallbackParams<T> fb;        // the row (rows == 1), K, capacity, control block, header, histogram area, buffer
-    uint32_t* bins;              // BK_BINS + BK_FLAGS words
-    uint32_t* coarse;            // BK_COARSE words: the coarse histogram
+    uint32_t* bins;              // BIN_ROW_WORDS words: fine bins, flags, coarse bins
+    int hist_ready;              // 1 = the filter kernel counted the records it appended in them (all else zero); 0 = nobody has touched them
     uint64_t* edge;              // BK_EDGE records: the boundary class
     uint32_t parts;              // 1, or FILTER_PARTS: the filter appended to that many parts of the buffer
     uint32_t part_cap;
@@ -50,24 +51,6 @@ template <typename T> struct BatchTopkParams {
     int use_pdl;
     int direct;                  // 1 = no threshold / filter ran: the row is selected exactly
 };
-
-// Bin of the logarithmic level: exponent e = floor(log2 D) in the top 6 bits, the 12 bits after the leading one below.
-// Monotone in D.  D = 0 shares bin 0 with D = 1.
-__device__ __forceinline__ uint32_t bk_log_bin(uint64_t D) {
-    if (D < 2) return 0;
-    const int e = 63 - __clzll((long long)D);
-    const uint64_t frac = D ^ (1ull << e);
-    const uint32_t m = e >= 12 ? (uint32_t)(frac >> (e - 12)) : (uint32_t)(frac << (12 - e));
-    return ((uint32_t)e << 12) | m;
-}
-// The D range of a bin of the logarithmic level: [lo, lo + 2^w).
-__device__ __forceinline__ void bk_log_bin_range(uint32_t bin, uint64_t* lo, int* w) {
-    if (bin == 0) { *lo = 0; *w = 1; return; }
-    const int e = (int)(bin >> 12);
-    const uint64_t m = bin & 4095u;
-    if (e >= 12) { *lo = (1ull << e) | (m << (e - 12)); *w = e - 12; }
-    else { *lo = (1ull << e) + (m >> (12 - e)); *w = 0; }
-}
 
 // Zeroes n elements at p (aligned to the element size only) with 16-byte stores where the address allows.
 template <typename E>
@@ -94,16 +77,19 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
     const unsigned nctas = gridDim.x, cta = blockIdx.x;
     const uint64_t gid = (uint64_t)cta * BK_THREADS + tid, gthreads = (uint64_t)nctas * BK_THREADS;
     const FallbackParams<T>& fb = p.fb;
-    uint32_t* flags = p.bins + BK_BINS;
+    uint32_t* flags = p.bins + BIN_COUNT;
+    uint32_t* coarse = flags + BIN_FLAGS;
 
     // Prologue, before the wait for the filter kernel: the workspace's bins and flags (nobody else uses them).
     // Each CTA then reports in through the header's `done` word (zeroed by the call's first kernel, long finished): the
     // histogram pass below needs every CTA's share to be zero, and by then all have reported -- a wait that does not wait.
-    for (uint64_t b = gid; b < BK_BINS + BK_FLAGS; b += gthreads) p.bins[b] = 0;
-    for (uint64_t b = gid; b < BK_COARSE; b += gthreads) p.coarse[b] = 0;
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) atomicAdd(&fb.header->done, 1u);
+    // (Not when the filter kernel counts in them: then the threshold kernels have cleared them.)
+    if (!p.hist_ready) {
+        for (uint64_t b = gid; b < BIN_ROW_WORDS; b += gthreads) p.bins[b] = 0;
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) atomicAdd(&fb.header->done, 1u);
+    }
     pdl_launch_dependents();
     if (p.use_pdl) pdl_wait();
     uint32_t gen = *((volatile uint32_t*)&fb.header->bar_gen);          // read before this CTA's first arrival
@@ -181,10 +167,9 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
     // 32-bit index word of which a row only uses idx_bits bits; the unused bits are squeezed out of D, so that the bits
     // right below the key difference are real index bits: thousands of copies of one bf16 value then spread over the
     // logarithmic level's bins instead of crowding one (which costs further levels).
-    const uint64_t top = make_record(tau_key, 0xFFFFFFFFu);
-    const int idx_bits = fb.N > 1 ? 64 - __clzll((long long)(fb.N - 1)) : 1;
-    const uint64_t idx_top = (1ull << idx_bits) - 1ull;
-    auto dist = [&](uint64_t rec) { return (((top >> 32) - (rec >> 32)) << idx_bits) | (idx_top - (rec & 0xFFFFFFFFull)); };
+    const uint32_t top_hi = ~tau_key;
+    const int idx_bits = index_bits(fb.N);
+    auto dist = [&](uint64_t rec) { return record_dist(rec, top_hi, idx_bits); };
     uint64_t cls_lo = 0;          // the boundary class is cls_lo <= D < cls_lo + 2^cls_w ...
     int cls_w = 64;               // ... (64: every D)
     uint32_t need = K;            // ... and its `need` best records are kept, with every record of a better class
@@ -192,8 +177,19 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
     if (keep_all) need = 0;
     __shared__ uint32_t s_coarse[BK_COARSE];
     __shared__ uint32_t s_ok;
+    // level 0 has been counted by the filter kernel (all of it: no record went in uncounted)
+    const bool have_hist = p.hist_ready && status == ROW_OK && __ldcg(&flags[BIN_FLAG_UNCOUNTED]) == 0;
     if (keep_all) {
         // (the exact selection ended on a grid barrier, but the zero fill above came after it)
+        if (!grid_barrier(fb.header, gen)) return;
+    } else if (have_hist) {
+        // nothing to count; only the zero fill above has to be over everywhere before anybody emits
+        if ((p.mask || p.dense) && !grid_barrier(fb.header, gen)) return;
+    } else if (p.hist_ready) {
+        // the bins hold the counts of the first filtering pass, the buffer the records of the second: start again
+        // (nobody has read the bins yet; the flags behind them are still zero)
+        for (uint64_t b = gid; b < BIN_COUNT; b += gthreads) p.bins[b] = 0;
+        for (uint64_t b = gid; b < BIN_COARSE; b += gthreads) coarse[b] = 0;
         if (!grid_barrier(fb.header, gen)) return;
     } else {
         // every CTA has zeroed its share of the bins: reported before the wait for the filter kernel, so this returns at once
@@ -212,30 +208,32 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
     for (int level = 0; !whole && level < BK_MAX_LEVELS; ++level) {
         const int sh_bits = cls_w > BK_BITS ? cls_w - BK_BITS : 0;       // linear levels: D's bits below the bin
         auto bin_of = [&](uint64_t D, bool* in_class) {
-            if (level == 0) { *in_class = true; return bk_log_bin(D); }
+            if (level == 0) { *in_class = true; return log_bin(D); }
             *in_class = D >= cls_lo && ((D - cls_lo) >> cls_w) == 0;
             return (uint32_t)((D - cls_lo) >> sh_bits) & (BK_BINS - 1);
         };
         // histogram, best records in the lowest bins: fine bins in global memory, coarse bins through shared memory
-        for (uint32_t c = tid; c < BK_COARSE; c += BK_THREADS) s_coarse[c] = 0;
-        __syncthreads();
-        for (uint64_t i = gid; i < total; i += gthreads) {
-            bool in_class;
-            const uint32_t f = BK_BINS - 1 - bin_of(dist(record_at(i)), &in_class);
-            if (in_class) {
-                atomicAdd(&p.bins[f], 1u);
-                atomicAdd(&s_coarse[f / BK_PER_COARSE], 1u);
+        if (!(level == 0 && have_hist)) {
+            for (uint32_t c = tid; c < BK_COARSE; c += BK_THREADS) s_coarse[c] = 0;
+            __syncthreads();
+            for (uint64_t i = gid; i < total; i += gthreads) {
+                bool in_class;
+                const uint32_t f = BK_BINS - 1 - bin_of(dist(record_at(i)), &in_class);
+                if (in_class) {
+                    atomicAdd(&p.bins[f], 1u);
+                    atomicAdd(&s_coarse[f / BK_PER_COARSE], 1u);
+                }
             }
+            __syncthreads();
+            for (uint32_t c = tid; c < BK_COARSE; c += BK_THREADS) {
+                const uint32_t n = s_coarse[c];
+                if (n) atomicAdd(&coarse[c], n);
+            }
+            if (!grid_barrier(fb.header, gen)) return;
         }
-        __syncthreads();
-        for (uint32_t c = tid; c < BK_COARSE; c += BK_THREADS) {
-            const uint32_t n = s_coarse[c];
-            if (n) atomicAdd(&p.coarse[c], n);
-        }
-        if (!grid_barrier(fb.header, gen)) return;
         // every CTA: the coarse bin, then the fine bin, of the need-th best record of the class
         {
-            const uint32_t c = tid < BK_COARSE ? __ldcg(&p.coarse[tid]) : 0u;
+            const uint32_t c = tid < BK_COARSE ? __ldcg(&coarse[tid]) : 0u;
             const uint32_t incl = block_inclusive_scan(c, sh.warp_sums);
             if (incl - c < need && need <= incl) { s_seg = tid; s_seg_before = incl - c; }
             __syncthreads();
@@ -250,7 +248,7 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
         }
         const uint32_t bin = BK_BINS - 1 - s_bin, in_bin = s_bin_count;
         need -= s_bin_before;
-        if (level == 0) bk_log_bin_range(bin, &cls_lo, &cls_w);
+        if (level == 0) log_bin_range(bin, &cls_lo, &cls_w);
         else { cls_lo += (uint64_t)bin << sh_bits; cls_w = sh_bits; }
         __syncthreads();                           // the shared words are rewritten by the next level
         if (in_bin == need) { whole = true; break; }
@@ -258,7 +256,7 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
         // crowded: one more level inside the class; the bins start from zero again
         if (!grid_barrier(fb.header, gen)) return;                        // everybody has read this level's bins
         for (uint64_t b = gid; b < BK_BINS; b += gthreads) p.bins[b] = 0;
-        for (uint64_t b = gid; b < BK_COARSE; b += gthreads) p.coarse[b] = 0;
+        for (uint64_t b = gid; b < BK_COARSE; b += gthreads) coarse[b] = 0;
         if (!grid_barrier(fb.header, gen)) return;
     }
     // Kept outright: D >= keep_from.  Boundary list: cls_lo <= D < keep_from (empty when the whole class is kept).

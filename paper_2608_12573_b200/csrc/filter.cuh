@@ -11,6 +11,7 @@
 // streaming loop.
 #pragma once
 
+#include "bins.cuh"
 #include "rowscan.cuh"
 
 // Launch shape of the filter kernel (tuned on B200; overridable at build time for experiments).
@@ -65,6 +66,25 @@ template <typename T> struct FilterParams {
     // loads (PREFETCH_SPIN_LIMIT; a test sets 0 to take that branch).  The wait before the CTA leaves always has the
     // full limit: shared memory must not be handed on while a copy into it is in flight.
     uint32_t prefetch_spin_limit;
+    // The HIST build (one row, large selections): every record appended is also counted in the bins of bins.cuh -- the
+    // fine bins at hist[0 .. BIN_COUNT) with one global atomic, the coarse ones through the CTA's shared memory -- so that
+    // the kernel behind this one finds its histogram made (unless the flag word BIN_FLAG_UNCOUNTED says that some records
+    // went uncounted).  All BIN_ROW_WORDS words are zero when the scan starts.
+    uint32_t* hist;
+    int idx_bits;            // bits an index of the row occupies
+};
+
+// What the appending code of the HIST build needs to count a record (an empty shell otherwise).
+struct HistCtx {
+    uint32_t* fine;          // global
+    uint32_t* coarse;        // shared memory of the CTA
+    uint32_t top_hi;         // high word of the largest record the filter keeps: tau's key, inverted
+    int idx_bits;
+    __device__ __forceinline__ void count(uint64_t rec) const {
+        const uint32_t b = record_bin(rec, top_hi, idx_bits);
+        atomicAdd(&fine[b], 1u);
+        atomicAdd(&coarse[b / BIN_PER_COARSE], 1u);
+    }
 };
 
 constexpr uint32_t FILTER_PREFETCH = 2;
@@ -192,9 +212,9 @@ __device__ __forceinline__ unsigned warp_exclusive_count(unsigned cnt, unsigned 
 
 // Writes one thread's survivors as records to out[pos], out[pos + 1], ... (positions >= limit are dropped).
 // Survivors are few: a loop over the set bits, each picking its element out of the registers.
-template <typename T, int THREADS, int UNROLL>
+template <typename T, int THREADS, int UNROLL, bool HIST = false>
 __device__ __forceinline__ void emit_survivors(const typename Elem<T>::vec_t (&v)[UNROLL], uint32_t mine, uint64_t qbase,
-                                               uint32_t mis, uint64_t* out, unsigned pos, unsigned limit) {
+                                               uint32_t mis, uint64_t* out, unsigned pos, unsigned limit, const HistCtx& hc = HistCtx{}) {
     constexpr int VEC = Elem<T>::VEC;
     static_assert(UNROLL == 4, "four vectors per thread and tile");
     while (mine) {
@@ -204,7 +224,11 @@ __device__ __forceinline__ void emit_survivors(const typename Elem<T>::vec_t (&v
         const T x = u == 0 ? vec_elem(v[0], l) : u == 1 ? vec_elem(v[1], l) : u == 2 ? vec_elem(v[2], l) : vec_elem(v[3], l);
         const uint64_t q = qbase + (uint64_t)u * THREADS + threadIdx.x;
         const uint32_t i = (uint32_t)((int64_t)(q * VEC) - (int64_t)mis) + (uint32_t)l;
-        if (pos < limit) out[pos] = make_record(Elem<T>::key(x), i);
+        if (pos < limit) {
+            const uint64_t rec = make_record(Elem<T>::key(x), i);
+            out[pos] = rec;
+            if (HIST) hc.count(rec);
+        }
         ++pos;
     }
 }
@@ -340,9 +364,10 @@ __device__ __noinline__ uint32_t filter_slow_path(const FilterParams<T>& p, Warp
 
 // The slow path without staging (sparse survivors): one global atomic per warp and tile, records
 // written straight to the row buffer.  Returns the row if its buffer has overflowed, else ~0.
-template <typename T, int THREADS, int UNROLL, bool PARTS>
+template <typename T, int THREADS, int UNROLL, bool PARTS, bool HIST = false>
 __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T>& p, const typename Elem<T>::vec_t (&v)[UNROLL],
-                                                            uint32_t inside_mask, uint32_t row, uint64_t qbase, uint32_t mis, T tau) {
+                                                            uint32_t inside_mask, uint32_t row, uint64_t qbase, uint32_t mis, T tau,
+                                                            uint32_t* hist_coarse = nullptr) {
     const unsigned lane = lane_id();
     const uint32_t mine = survivor_mask<T, THREADS, UNROLL>(v, inside_mask, p.N, qbase, mis, tau, p, row);
     const unsigned cnt = __popc(mine);
@@ -361,7 +386,10 @@ __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T
     unsigned base = 0;
     if (lane == 0) base = atomicAdd(counter, total);
     base = __shfl_sync(FULL_MASK, base, 0);
-    if (cnt) emit_survivors<T, THREADS, UNROLL>(v, mine, qbase, mis, dst, base + before, cap);
+    if (cnt) {
+        if (HIST) emit_survivors<T, THREADS, UNROLL, true>(v, mine, qbase, mis, dst, base + before, cap, HistCtx{p.hist, hist_coarse, ~Elem<T>::key(tau), p.idx_bits});
+        else emit_survivors<T, THREADS, UNROLL>(v, mine, qbase, mis, dst, base + before, cap);
+    }
     return (uint64_t)base + total > cap ? row : 0xFFFFFFFFu;
 }
 
@@ -383,37 +411,56 @@ constexpr uint32_t DEFER_NONE = 0xFFFFFFFFu;          // a reserved slot that wa
 // One batch of 32 list entries worked off: lane by lane a candidate vector (number `vid` among the vectors of the launch,
 // tiles in order; DEFER_NONE = none) is read again and decided in the total order of the keys; the survivors are
 // appended with one atomic per row that has survivors among them.  All 32 lanes call it.
-template <typename T, int THREADS, int UNROLL, bool PARTS>
-__device__ __forceinline__ void defer_process_batch(const FilterParams<T>& p, uint32_t vid) {
-    using V = typename Elem<T>::vec_t;
+// A list entry decided: candidate vector number `vid` among the vectors of the launch (tiles in order; DEFER_NONE = none)
+// is read again and its elements are tested in the total order of the keys.
+template <typename T> struct DeferDecided {
+    typename Elem<T>::vec_t v;
+    int64_t i0;        // index of the vector's first element in its row
+    uint32_t row;
+    unsigned m;        // bit j: element j is kept
+    uint32_t top_hi;   // (HIST) what HistCtx needs of the row's threshold
+};
+template <typename T, int THREADS, int UNROLL>
+__device__ __forceinline__ DeferDecided<T> defer_decide(const FilterParams<T>& p, uint32_t vid) {
     constexpr int VEC = Elem<T>::VEC;
     constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
-    const unsigned lane = lane_id();
-    uint32_t row = 0;
-    unsigned m = 0;
-    V v = {};
-    int64_t i0 = 0;
+    DeferDecided<T> d = {};
     if (vid != DEFER_NONE) {
         const uint32_t tile = vid / TILE_VECTORS, within = vid % TILE_VECTORS;
         const uint32_t tiles_per_row = (uint32_t)p.tiles_per_row;
         uint32_t tin = tile;
-        if (tiles_per_row != (uint32_t)p.total_tiles) { row = tile / tiles_per_row; tin = tile - row * tiles_per_row; }
-        const RowView<T> rv = row_view(p.in, p.N, row);
-        const T tau = p.thr ? Elem<T>::from_bits(reinterpret_cast<const uint32_t*>(p.thr + row)[0]) : p.tau[row];
+        if (tiles_per_row != (uint32_t)p.total_tiles) { d.row = tile / tiles_per_row; tin = tile - d.row * tiles_per_row; }
+        const RowView<T> rv = row_view(p.in, p.N, d.row);
+        const T tau = p.thr ? Elem<T>::from_bits(reinterpret_cast<const uint32_t*>(p.thr + d.row)[0]) : p.tau[d.row];
         const uint64_t q = (uint64_t)tin * TILE_VECTORS + within;
         bool in;
-        v = load_row_vector(rv, p.N, q, &in);
+        d.v = load_row_vector(rv, p.N, q, &in);
         if (in) {
-            i0 = (int64_t)(q * VEC) - (int64_t)rv.mis;
-            m = vec_pass_mask(v, tau);
-            if (i0 < 0 || i0 + VEC > (int64_t)p.N) {
+            d.i0 = (int64_t)(q * VEC) - (int64_t)rv.mis;
+            d.m = vec_pass_mask(d.v, tau);
+            if (d.i0 < 0 || d.i0 + VEC > (int64_t)p.N) {
 #pragma unroll
                 for (int j = 0; j < VEC; ++j)
-                    if (i0 + j < 0 || i0 + j >= (int64_t)p.N) m &= ~(1u << j);
+                    if (d.i0 + j < 0 || d.i0 + j >= (int64_t)p.N) d.m &= ~(1u << j);
             }
-            m = confirm_survivors<T>(p, row, v, m, i0, tau);
+            d.m = confirm_survivors<T>(p, d.row, d.v, d.m, d.i0, tau);
+            d.top_hi = ~Elem<T>::key(tau);
         }
     }
+    return d;
+}
+
+// One batch of 32 list entries worked off, lane by lane one entry; the survivors are appended with one atomic per row
+// that has survivors among them.  All 32 lanes call it.
+template <typename T, int THREADS, int UNROLL, bool PARTS, bool HIST = false>
+__device__ __forceinline__ void defer_process_batch(const FilterParams<T>& p, uint32_t vid, uint32_t* hist_coarse = nullptr) {
+    const unsigned lane = lane_id();
+    const DeferDecided<T> d = defer_decide<T, THREADS, UNROLL>(p, vid);
+    const uint32_t row = d.row;
+    const unsigned m = d.m;
+    const typename Elem<T>::vec_t v = d.v;
+    const int64_t i0 = d.i0;
+    const HistCtx hc = {p.hist, hist_coarse, d.top_hi, p.idx_bits};
     // Append, one atomic per row that has survivors in this batch (32 consecutive entries of the list span a tile or two,
     // so one or two rows): the lanes of the first row with survivors form a group, scan their counts, their first lane
     // reserves the room; then the next row's lanes, until none is left.
@@ -448,12 +495,71 @@ __device__ __forceinline__ void defer_process_batch(const FilterParams<T>& p, ui
             while (mm) {
                 const int b = __ffs(mm) - 1;
                 mm &= mm - 1;
-                if (pos < cap) dst[pos] = make_record(Elem<T>::key(vec_elem(v, b)), (uint32_t)(i0 + b));
+                if (pos < cap) {
+                    const uint64_t rec = make_record(Elem<T>::key(vec_elem(v, b)), (uint32_t)(i0 + b));
+                    dst[pos] = rec;
+                    if (HIST) hc.count(rec);
+                }
                 ++pos;
             }
         }
         left &= ~group;
     }
+}
+
+// The same for a launch over ONE row, by the whole CTA: THREADS entries, one atomic.  When the scan ends every CTA of
+// the grid works its list off at the same moment, and an atomic per warp -- seven thousand on the row's one counter --
+// took longer than the rest of that work.  `scratch` holds THREADS / 32 + 1 words of shared memory; all threads call.
+template <typename T, int THREADS, int UNROLL, bool HIST>
+__device__ __noinline__ void defer_process_block(const FilterParams<T>& p, uint32_t vid, uint32_t* hist_coarse, uint32_t* scratch) {
+    static_assert(THREADS / 32 <= 32, "one lane of the first warp per warp of the CTA");
+    const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
+    const DeferDecided<T> d = defer_decide<T, THREADS, UNROLL>(p, vid);
+    const unsigned cnt = __popc(d.m);
+    unsigned incl = cnt;
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+        const unsigned nb = __shfl_up_sync(FULL_MASK, incl, s);
+        if (lane >= (unsigned)s) incl += nb;
+    }
+    if (lane == 31) scratch[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        const unsigned w = lane < THREADS / 32 ? scratch[lane] : 0u;
+        unsigned wi = w;
+#pragma unroll
+        for (int s = 1; s < 32; s <<= 1) {
+            const unsigned nb = __shfl_up_sync(FULL_MASK, wi, s);
+            if (lane >= (unsigned)s) wi += nb;
+        }
+        unsigned base = 0;
+        if (lane == 31 && wi) base = atomicAdd(p.counts, wi);           // (row 0's counter)
+        base = __shfl_sync(FULL_MASK, base, 31);
+        if (lane < THREADS / 32) scratch[lane] = base + wi - w;         // first position of the warp's records
+    }
+    __syncthreads();
+    if (cnt) {
+        const HistCtx hc = {p.hist, hist_coarse, d.top_hi, p.idx_bits};
+        unsigned pos = scratch[warp] + incl - cnt;
+        unsigned mm = d.m;
+        while (mm) {
+            const int b = __ffs(mm) - 1;
+            mm &= mm - 1;
+            if (pos < p.capacity) {
+                const uint64_t rec = make_record(Elem<T>::key(vec_elem(d.v, b)), (uint32_t)(d.i0 + b));
+                p.buf[pos] = rec;
+                if (HIST) hc.count(rec);
+            }
+            ++pos;
+        }
+    }
+    __syncthreads();                   // scratch is rewritten by the next batch
+}
+
+// The HIST build's: out of line, so that the counting costs the streaming loop no registers.
+template <typename T, int THREADS, int UNROLL, bool PARTS>
+__device__ __noinline__ void defer_process_batch_counting(const FilterParams<T>& p, uint32_t vid, uint32_t* hist_coarse) {
+    defer_process_batch<T, THREADS, UNROLL, PARTS, true>(p, vid, hist_coarse);
 }
 
 // STAGED = collect survivors in per-warp shared-memory stages (dense survivors, one row at a time);
@@ -465,16 +571,21 @@ __device__ __forceinline__ void defer_process_batch(const FilterParams<T>& p, ui
 // tiles of the launch (from dyn_start on) come from a global counter instead, so that SMs that saw
 // less bandwidth take fewer of them and all CTAs finish together.  The counter is read one tile
 // ahead, so its round trip hides behind the loads; only this tail needs a CTA barrier per tile.
-template <typename T, int THREADS, int UNROLL, bool STAGED, bool PARTS = false, bool DEFER = false>
+template <typename T, int THREADS, int UNROLL, bool STAGED, bool PARTS = false, bool DEFER = false, bool HIST = false>
 __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGED : sizeof(T) == 4 ? PROFK_FILTER_MINBLOCKS_F32 : PROFK_FILTER_MINBLOCKS_BF16) filter_kernel(const __grid_constant__ FilterParams<T> p) {
     static_assert(!(STAGED && DEFER), "one way of handling dense survivors at a time");
+    static_assert(!HIST || (DEFER && !PARTS), "only the deferring build counts its records");
     using V = typename Elem<T>::vec_t;
     constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
     __shared__ WarpStage stages[STAGED ? THREADS / 32 : 1];
     __shared__ uint32_t hits[DEFER ? DEFER_CAP : 1];
     __shared__ uint32_t s_nhits;
-    if (DEFER) {
+    __shared__ uint32_t s_scan[DEFER ? THREADS / 32 + 1 : 1];
+    __shared__ uint32_t s_hcoarse[HIST ? BIN_COARSE : 1];       // (HIST) this CTA's share of the coarse histogram
+    if (DEFER || HIST) {
         if (threadIdx.x == 0) s_nhits = 0;
+        if (HIST)
+            for (uint32_t c = threadIdx.x; c < BIN_COARSE; c += THREADS) s_hcoarse[c] = 0;
         __syncthreads();
     }
     __shared__ uint32_t s_next[2];
@@ -654,6 +765,8 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
             if (!noted) {
                 if (STAGED) o = filter_slow_path<T, THREADS, UNROLL>(p, st, v[0], v[1], v[2], v[3], inside_mask, row, qbase, rv.mis, tau_lo);
                 else o = filter_slow_path_direct<T, THREADS, UNROLL, PARTS>(p, v, inside_mask, row, qbase, rv.mis, tau_lo);
+                // (HIST) records appended on this way out of a full list are not counted: the kernel behind is told so
+                if (HIST && lane == 0) p.hist[BIN_COUNT + BIN_FLAG_UNCOUNTED] = 1u;
             }
             if (o != 0xFFFFFFFFu) skip_row = o;
         }
@@ -681,7 +794,21 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
         const uint32_t n = s_nhits < DEFER_CAP ? s_nhits : DEFER_CAP;
         for (uint32_t e0 = 0; e0 < n; e0 += THREADS) {          // whole warps take part in every batch
             const uint32_t e = e0 + threadIdx.x;
-            if (e0 + (threadIdx.x & ~31u) < n) defer_process_batch<T, THREADS, UNROLL, PARTS>(p, e < n ? hits[e] : DEFER_NONE);
+            if (one_row && !PARTS) {
+                defer_process_block<T, THREADS, UNROLL, HIST>(p, e < n ? hits[e] : DEFER_NONE, s_hcoarse, s_scan);
+            } else if (e0 + (threadIdx.x & ~31u) < n) {
+                if (HIST) defer_process_batch_counting<T, THREADS, UNROLL, PARTS>(p, e < n ? hits[e] : DEFER_NONE, s_hcoarse);
+                else defer_process_batch<T, THREADS, UNROLL, PARTS>(p, e < n ? hits[e] : DEFER_NONE);
+            }
+        }
+    }
+    if (HIST) {
+        // this CTA's coarse counts join the row's (the fine bins were counted record by record)
+        __syncthreads();
+        uint32_t* coarse = p.hist + BIN_COUNT + BIN_FLAGS;
+        for (uint32_t c = threadIdx.x; c < BIN_COARSE; c += THREADS) {
+            const uint32_t n = s_hcoarse[c];
+            if (n) atomicAdd(&coarse[c], n);
         }
     }
     if (pf_pending) prefetch_landed(PREFETCH_SPIN_LIMIT);

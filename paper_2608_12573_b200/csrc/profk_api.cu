@@ -101,7 +101,7 @@ WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k, bool large) {
     l.off_tau = align_up(l.off_ctl + (size_t)rows * sizeof(RowCtl), 256);
     l.off_tau2 = align_up(l.off_tau + (size_t)rows * sizeof(uint4), 256);       // threshold records of a second filtering pass
     l.off_bins = align_up(l.off_tau2 + (size_t)rows * sizeof(uint4), 256);
-    const size_t bins_bytes = large ? (size_t)rows * (LG_BINS + 8) * sizeof(uint32_t) : 0;
+    const size_t bins_bytes = large ? (size_t)rows * BIN_ROW_WORDS * sizeof(uint32_t) : 0;
     // scratch of the in-refine exact selection (few rows, k within the single-CTA refine): up to
     // XS_MAX_SEGMENTS segments in all, each with a counter and k + XS_EDGE records
     const bool xs = rows <= XS_MAX_ROWS && !large;
@@ -217,7 +217,8 @@ int pick_cluster(int64_t rows, int64_t m, int max_cluster) {
 template <typename T>
 int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, int64_t m, int64_t r, uint64_t seed, T* tau, RowCtl* ctl,
                          WsHeader* header, uint32_t capacity, uint32_t* sample_idx, uint32_t* keys_scratch, uint32_t* part_counts,
-                         bool by_record, uint4* thr, cudaStream_t st, const uint32_t* keys_given = nullptr, uint32_t* keys_store = nullptr) {
+                         bool by_record, uint4* thr, cudaStream_t st, const uint32_t* keys_given = nullptr, uint32_t* keys_store = nullptr,
+                         uint32_t* zero = nullptr, uint32_t zero_words = 0) {
     const int csize = pick_cluster(rows, m, di.max_cluster[dtype_index<T>()]);
     // A large sample, or a sample of a very long row (every element on a page of its own), is gathered by a
     // kernel over all SMs first; the cluster then only selects.  (keys_given: the caller already holds the sample's keys.)
@@ -228,6 +229,7 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
         gp.in = in; gp.N = (uint64_t)N; gp.rows = (uint64_t)rows; gp.S = (uint32_t)m; gp.seed = seed;
         gp.q = (uint64_t)(N / m); gp.rem = (uint32_t)(N % m); gp.inv_s = 1.0f / (float)m; gp.keys_out = keys_scratch;
         gp.pair_lo = 0; gp.pairs = (uint64_t)((m + 1) / 2); gp.base = 0;
+        gp.zero = reinterpret_cast<uint4*>(zero); gp.zero_vecs = zero_words / 4;      // cleared by the wider of the two kernels
         const int64_t pairs = rows * ((m + 1) / 2);
         cudaLaunchConfig_t gcfg = {};
         gcfg.gridDim = dim3((unsigned)((pairs + GATHER_THREADS - 1) / GATHER_THREADS));
@@ -245,6 +247,7 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
     sp.keys_store = sp.keys_in ? nullptr : keys_store;       // (keys gathered by the kernel before are in memory already)
     sp.part_counts = part_counts;
     sp.by_record = by_record ? 1 : 0;
+    sp.zero = spread_gather ? nullptr : reinterpret_cast<uint4*>(zero); sp.zero_vecs = zero_words / 4;
     sp.thr = thr;
     sp.in = in; sp.N = (uint64_t)N; sp.S = (uint32_t)m; sp.t = (uint32_t)r; sp.seed = seed;
     sp.per_cta = (uint32_t)(((m + csize - 1) / csize + 1) & ~1LL);      // even: samples are drawn in pairs
@@ -279,8 +282,9 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
 template <typename T>
 int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, const T* tau, int64_t capacity, uint64_t* buf,
                   uint64_t buf_stride, uint32_t* counts, uint32_t count_stride, bool pdl, bool staged, uint32_t* tile_counter, bool parts,
-                  uint32_t part_cap, uint32_t* part_counts, const uint4* thr, cudaStream_t st, bool deferred = false) {
+                  uint32_t part_cap, uint32_t* part_counts, const uint4* thr, cudaStream_t st, bool deferred = false, uint32_t* hist = nullptr) {
     FilterParams<T> fp;
+    fp.hist = hist; fp.idx_bits = index_bits((uint64_t)N);
     fp.thr = thr;
     fp.in = in; fp.N = (uint64_t)N; fp.rows = (uint64_t)rows; fp.tau = tau; fp.capacity = (uint32_t)capacity;
     fp.buf = buf; fp.buf_stride = buf_stride; fp.counts = counts; fp.count_stride = count_stride;
@@ -312,7 +316,9 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
-    if (staged) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, true>, fp));
+    if (hist && (rows != 1 || !deferred)) return PROFK_EINVAL;      // (no caller asks for that)
+    if (hist) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false, false, true, true>, fp));
+    else if (staged) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, true>, fp));
     else if (deferred) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false, false, true>, fp));
     else if (parts) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false, true>, fp));
     else CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false>, fp));
@@ -684,14 +690,16 @@ int batchtopk_planned(const T* in, int64_t N, int64_t K, const profk_plan_t* pla
     const bool staged = plan->mode == 0 && !deferred && per_warp_tile > 2.0;
     const bool parts = !staged && !deferred && plan->mode == 0;
     const uint32_t part_cap = (uint32_t)(row_stride / 2 / FILTER_PARTS);
+    const bool hist = deferred;
 
     if (plan->mode == 0) {
+        // The filter counts the records it appends in the bins the emit kernel selects from (cleared by the threshold kernels).
         rc = launch_sample_select<T>(di, in, 1, N, plan->m, plan->r, seed, nullptr, ctl, header, (uint32_t)capacity, nullptr, keys_scratch,
                                      parts ? part_counts : nullptr, plan->tie_rule == PROFK_TIES_BY_INDEX, thr, st, nullptr,
-                                     (plan->r_tight > 0 || plan->r_loose > 0) ? keys_scratch : nullptr);
+                                     (plan->r_tight > 0 || plan->r_loose > 0) ? keys_scratch : nullptr, hist ? bins : nullptr, BIN_ROW_WORDS);
         if (rc != PROFK_OK) return rc;
         rc = launch_filter<T>(di, in, 1, N, nullptr, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, &header->tile_counter,
-                              parts, part_cap, part_counts, thr, st, deferred);
+                              parts, part_cap, part_counts, thr, st, deferred, hist ? bins : nullptr);
         if (rc != PROFK_OK) return rc;
     } else {
         init_ctl_kernel<<<1, 256, 0, st>>>(ctl, 1, header, (uint32_t)capacity, (uint32_t)K);
@@ -716,7 +724,7 @@ int batchtopk_planned(const T* in, int64_t N, int64_t K, const profk_plan_t* pla
     }
     bp.fb.thr2 = reinterpret_cast<uint4*>(base + lay.off_tau2);
     bp.bins = bins;
-    bp.coarse = ghist;                                            // (the exact selection and the select levels never both run)
+    bp.hist_ready = hist ? 1 : 0;
     bp.edge = buf + row_stride / 2;                               // the scratch half of the row's buffer
     bp.parts = parts ? FILTER_PARTS : 1u; bp.part_cap = part_cap; bp.part_counts = part_counts;
     bp.sel_vals = sel_vals; bp.sel_idx = sel_idx; bp.mask = mask; bp.dense = dense;
@@ -790,6 +798,7 @@ int shard_sample_keys(const T* shard, int64_t shard_base, int64_t shard_len, int
     gp.in = shard; gp.N = (uint64_t)N; gp.rows = 1; gp.S = (uint32_t)m; gp.seed = seed;
     gp.q = (uint64_t)(N / m); gp.rem = (uint32_t)(N % m); gp.inv_s = 1.0f / (float)m; gp.keys_out = keys_out;
     gp.pair_lo = (uint64_t)(j_lo / 2); gp.pairs = (uint64_t)((j_hi - j_lo + 1) / 2); gp.base = (uint64_t)shard_base;
+    gp.zero = nullptr; gp.zero_vecs = 0;
     gather_kernel<T><<<(unsigned)((gp.pairs + GATHER_THREADS - 1) / GATHER_THREADS), GATHER_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(gp);
     CUDA_TRY(cudaGetLastError());
     return PROFK_OK;

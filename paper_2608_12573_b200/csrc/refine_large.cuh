@@ -34,7 +34,7 @@ template <typename T> struct LargeParams {
     WsHeader* header;
     uint64_t* buf;           // row r: records at buf + r * 2 * row_stride, then row_stride records of scratch;
     uint64_t row_stride;     //        row_stride is a power of two >= capacity, >= BT_TILE
-    uint32_t* bins;          // rows x (LG_BINS + 8) words: bin counts / positions, then flags
+    uint32_t* bins;          // rows x BIN_ROW_WORDS words: bin counts / positions, then flags
     unsigned long long* slots;   // 2 words per CTA of the grid, then one per CTA: per-CTA minima / maxima and scan totals
     uint32_t groups;         // CTA groups the grid is cut into (<= WS_GROUPS; gridDim.x is a multiple of it)
     uint32_t parts;          // 1, or FILTER_PARTS: the filter appended to that many parts of the row's buffer (first phase only)
@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         const uint32_t kk = n < p.k ? n : p.k;
         uint64_t* G = p.buf + row * 2 * p.row_stride;
         uint64_t* G2 = G + p.row_stride;
-        uint32_t* bins = p.bins + row * (uint64_t)(LG_BINS + 8);
+        uint32_t* bins = p.bins + row * (uint64_t)BIN_ROW_WORDS;
         uint32_t* flags = bins + LG_BINS;                                // [0] = some bin that matters is crowded
         // every record of the row once, spread over the grid's threads
         // (The parts are walked as one run of sum(pcount) positions: part by part, a part of 20 K records would

@@ -85,6 +85,8 @@ template <typename T> struct SelectParams {
     uint32_t* part_counts;     // null, or the counters of the partitioned append (FILTER_PARTS per row, FILTER_PART_STRIDE words apart) to reset with the row's
     int by_record;             // 1 = the threshold is the t-th sampled record (value descending, index ascending), 0 = its value
     uint32_t* keys_store;      // null, or rows x S: the sample's keys are kept here for a second filtering pass (when this kernel gathers them itself)
+    uint4* zero;               // null, or zero_vecs 16-byte vectors to clear for the kernels behind this one (the bins the filter counts in)
+    uint32_t zero_vecs;
 };
 
 // floor(j * N / S) = j * (N / S) + floor(j * (N % S) / S).  The second quotient is below S
@@ -172,6 +174,8 @@ template <typename T> struct GatherParams {
     uint64_t pair_lo;
     uint64_t pairs;
     uint64_t base;
+    uint4* zero;           // null, or zero_vecs 16-byte vectors to clear for the kernels behind this one (the bins the filter counts in)
+    uint32_t zero_vecs;
 };
 
 template <typename T>
@@ -201,6 +205,8 @@ __global__ void __launch_bounds__(GATHER_THREADS) gather_kernel(const GatherPara
     // Dependents are released only now, after the wait: the kernels behind this one read the input before their
     // own wait (which covers this kernel alone), so they must not start before whatever wrote the input has finished.
     pdl_launch_dependents();
+    if (p.zero)        // (after the wait: the previous call's last kernel has read these words)
+        for (uint64_t i = g; i < p.zero_vecs; i += (uint64_t)gridDim.x * GATHER_THREADS) p.zero[i] = make_uint4(0u, 0u, 0u, 0u);
     if (active) {
         const T v0 = rowp[idx0];
         const T v1 = second ? rowp[idx1] : v0;
@@ -313,6 +319,8 @@ __global__ void __launch_bounds__(THREADS, THREADS == SEL_THREADS ? 1 : 4) sampl
     // finished, even a producer that released its own dependents early.  The filter's prologue still overlaps the
     // whole selection below.
     pdl_launch_dependents();
+    if (p.zero)
+        for (uint32_t i = blockIdx.x * THREADS + tid; i < p.zero_vecs; i += gridDim.x * THREADS) p.zero[i] = make_uint4(0u, 0u, 0u, 0u);
     if (crank == 0 && tid == 0) {
         if (p.ctl) {
             RowCtl* c = p.ctl + row;
