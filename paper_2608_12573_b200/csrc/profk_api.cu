@@ -360,8 +360,9 @@ template <typename T>
 int launch_refine_large(const DeviceInfo& di, RowCtl* ctl, WsHeader* header, uint64_t* buf, uint64_t row_pitch, uint32_t* bins,
                         unsigned long long* slots, bool parts, uint32_t part_cap, const uint32_t* part_counts, int64_t rows,
                         int64_t capacity, int64_t k, int64_t k_accept, int phase, T* out_vals, int64_t* out_idx, cudaStream_t st,
-                        const FallbackParams<T>* fused_fb = nullptr, bool after_kernel = true, int64_t N = 0) {
+                        const FallbackParams<T>* fused_fb = nullptr, bool after_kernel = true, int64_t N = 0, bool hist_ready = false) {
     LargeParams<T> lp;
+    lp.hist_ready = hist_ready ? 1 : 0;
     lp.idx_bits = 32;                            // (N unknown: every bit of the index word may be used)
     if (N > 1) { lp.idx_bits = 1; while (((int64_t)1 << lp.idx_bits) < N) ++lp.idx_bits; }
     lp.fused = fused_fb ? 1 : 0;
@@ -562,18 +563,22 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     // ordering are one cooperative kernel (three launches otherwise, two of which do nothing when no row failed).
     const bool fused_large = large && rows == 1;
 
+    // ... and when its filter is the deferring build, that counts the records it appends in the bins the ordering starts
+    // from (cleared by the threshold kernels).
+    const bool hist = fused_large && deferred;
+
     if (plan->mode == 0) {
         rc = launch_sample_select<T>(di, in, rows, N, plan->m, plan->r, seed, nullptr, ctl, header, (uint32_t)capacity, nullptr,
                                      rows <= GATHER_MAX_ROWS ? keys_scratch : nullptr, parts ? part_counts : nullptr, plan->tie_rule == PROFK_TIES_BY_INDEX, thr, st,
-                                     nullptr, keep_keys ? keys_scratch : nullptr);
+                                     nullptr, keep_keys ? keys_scratch : nullptr, hist ? bins : nullptr, BIN_ROW_WORDS);
         if (rc != PROFK_OK) return rc;
         rc = launch_filter<T>(di, in, rows, N, nullptr, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, &header->tile_counter,
-                              parts, part_cap, part_counts, thr, st, deferred);
+                              parts, part_cap, part_counts, thr, st, deferred, hist ? bins : nullptr);
         if (rc != PROFK_OK) return rc;
 
         if (large) {
             rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, reinterpret_cast<unsigned long long*>(ghist), parts, part_cap, part_counts, rows,
-                                        capacity, k, plan->k_accept, 0, out_vals, out_idx, st, fused_large ? &fb : nullptr, true, N);
+                                        capacity, k, plan->k_accept, 0, out_vals, out_idx, st, fused_large ? &fb : nullptr, true, N, hist);
             if (fused_large) return rc;
         } else {
             // count check and refine; with clusters, also the exact selection of the rows that fail the check

@@ -4,13 +4,14 @@
 // descending, index ascending" -- by the whole grid, launched cooperatively (one CTA per SM, all
 // co-resident), one row after the other.
 //
-// Main path: the records are binned on the top 18 bits of their distance above the smallest
-// record (262144 bins in global memory; because a record holds the value key above the index,
-// equal values are spread over bins by index), a cluster-wide scan turns the counts into
-// first positions, the records are scattered into a second buffer grouped by bin, and every
-// record of a bin that reaches into the first k positions ranks itself inside its bin -- a
-// handful of comparisons -- to find its place in the output.
-// Reserve path, taken when a bin is too crowded for that (an outlier stretches the range):
+// Main path: the records are counted in the bins of bins.cuh (262144 bins in global memory on a
+// logarithmic scale of the distance from the threshold record, 512 coarse bins over them; the
+// filter kernel makes this histogram itself where it can), a scan over the coarse and then the
+// fine bins turns the counts into first positions, the records are scattered into a second
+// buffer grouped by bin, and every record of a bin that reaches into the first k positions
+// ranks itself inside its bin -- a handful of comparisons -- to find its place in the output.
+// Two grid barriers when the histogram comes with the buffer, three or four otherwise.
+// Reserve path, taken when a bin is too crowded for that (very many equal records far from the threshold):
 // a bitonic network over P = 2^j records in the row's buffer, exchanges below one tile
 // (16384 records = 128 KB) in shared memory, the longer ones on the buffer in global memory.
 // The steps of both paths are separated by grid barriers whose waits are bounded: a wait that gives
@@ -25,8 +26,7 @@ namespace profk {
 
 constexpr uint32_t BT_TILE = 16384;          // records per shared-memory tile
 constexpr int BT_THREADS = 1024;
-constexpr int LG_BITS = 18;                  // digit width of the binning
-constexpr uint32_t LG_BINS = 1u << LG_BITS;
+constexpr uint32_t LG_WAIT_LIMIT = 1u << 22;  // polls of the "all CTAs have zeroed their share of the bins" counter
 constexpr uint32_t LG_CROWDED = 1024;        // a bin this full (among those that matter) sends the row to the reserve path
 
 template <typename T> struct LargeParams {
@@ -53,6 +53,8 @@ template <typename T> struct LargeParams {
     int fused;
     FallbackParams<T> fb;    // what that selection needs (fused == 1 only)
     int idx_bits;            // bits an index of the row occupies (1 .. 32)
+    int hist_ready;          // 1 = (fused) the filter kernel counted the records it appended in the row's bins; the rest of
+                             // the row's BIN_ROW_WORDS words are zero.  0 = nobody has touched them
 };
 
 // All exchanges of the network with stride < BT_TILE, for one tile held in shared memory.
@@ -78,8 +80,10 @@ template <typename T>
 __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const LargeParams<T> p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint64_t* tile = reinterpret_cast<uint64_t*>(smem_raw);          // BT_TILE records
-    __shared__ unsigned long long s_min[32], s_max[32];
+    __shared__ unsigned long long s_max[32];
     __shared__ uint32_t s_warp[32];
+    __shared__ uint32_t s_coarse[BIN_COARSE];
+    static_assert(BIN_COARSE <= BT_THREADS && BIN_PER_COARSE <= BT_THREADS, "one thread per coarse bin, then per fine bin of one coarse bin");
 
     // The grid works as p.groups groups of CTAs (one for a single row); a group takes rows group, group + groups, ...
     // one after the other, all its CTAs on one row, with a barrier of its own.
@@ -87,16 +91,20 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
     const unsigned tid = threadIdx.x;
     const uint64_t gid = (uint64_t)cta * BT_THREADS + tid;           // thread index inside the group
     const uint64_t gthreads = (uint64_t)nctas * BT_THREADS;
-    unsigned long long* slot_min = p.slots + group * nctas;
     unsigned long long* slot_max = p.slots + gridDim.x + group * nctas;
-    unsigned long long* slot_total = p.slots + 2 * gridDim.x + group * nctas;
     uint32_t* bar_count = &p.header->group_bar[group][0];
     uint32_t* bar_gen = &p.header->group_bar[group][1];
     auto barrier = [&](uint32_t& g) { return cta_group_barrier(bar_count, bar_gen, &p.header->error, nctas, g); };
-    // The scan is shared by a power-of-two number of CTAs (at most 256, so that a thread owns a whole bin).
-    unsigned scan_ctas = 1;
-    while (scan_ctas * 2 <= nctas && scan_ctas < 256) scan_ctas *= 2;
 
+    // A single row whose filter did not count: the bins are cleared here, before the wait for the filter kernel, and each
+    // CTA reports in through the header's `done` word (zeroed by the call's first kernel, long finished).
+    bool clean_bins = p.fused && !p.hist_ready;
+    if (clean_bins) {
+        for (uint64_t b = gid; b < BIN_ROW_WORDS; b += gthreads) p.bins[b] = 0;
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) atomicAdd(&p.header->done, 1u);
+    }
     pdl_launch_dependents();
     if (p.use_pdl) pdl_wait();
     uint32_t gen = *((volatile uint32_t*)bar_gen);                   // read before this CTA's first arrival
@@ -107,6 +115,9 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         const RowCtl ctl = p.ctl[row];
         uint32_t n;
         uint32_t nparts = 1, pcount[FILTER_PARTS] = {};      // the records are pcount[j] at G + j * part_cap
+        uint32_t tau_key = Elem<T>::key(Elem<T>::from_bits(ctl.tau_bits));
+        bool from_filter = false;        // the buffer is what a filtering pass with threshold tau_key left
+        bool status_ok = false;          // ... the first one
         if (p.phase == 0) {
             uint32_t R = ctl.count;
             bool part_full = false;
@@ -133,6 +144,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
                 if (status) atomicAdd(&p.header->n_failed, 1u);
             }
             n = R;
+            from_filter = status_ok = status == ROW_OK;
             if (status != ROW_OK) {
                 if (!p.fused) continue;          // the exact-selection kernel and the second phase take this row
                 // first a second filtering pass with the plan's tighter / looser sample rank, if it names one (the tile in
@@ -146,6 +158,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
 #pragma unroll
                 for (int j = 0; j < (int)FILTER_PARTS; ++j) pcount[j] = 0;
                 pcount[0] = n = again == 1 ? R2 : p.k;
+                if (again == 1) { from_filter = true; tau_key = key2; }
             }
         } else {
             if (ctl.status == ROW_OK) continue;  // already written by the first phase
@@ -156,7 +169,8 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         uint64_t* G = p.buf + row * 2 * p.row_stride;
         uint64_t* G2 = G + p.row_stride;
         uint32_t* bins = p.bins + row * (uint64_t)BIN_ROW_WORDS;
-        uint32_t* flags = bins + LG_BINS;                                // [0] = some bin that matters is crowded
+        uint32_t* flags = bins + BIN_COUNT;                              // [0] = some bin that matters is crowded
+        uint32_t* coarse = flags + BIN_FLAGS;
         // every record of the row once, spread over the grid's threads
         // (The parts are walked as one run of sum(pcount) positions: part by part, a part of 20 K records would
         // keep one thread in seven of the grid busy and cost a memory round trip of its own, eight per pass.)
@@ -182,67 +196,93 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         }
 
         // ================= main path: bin, scan, scatter, rank inside bins =================
-        // smallest and largest record of the row; clear the bins meanwhile
-        for (uint64_t b = gid; b < LG_BINS + 8; b += gthreads) bins[b] = 0;
-        unsigned long long lo = ~0ull, hi = 0ull;
-        for_each_record([&](unsigned long long rec) {
-            lo = rec < lo ? rec : lo;
-            hi = rec > hi ? rec : hi;
-        });
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) {
-            const unsigned long long l2 = __shfl_xor_sync(FULL_MASK, lo, d), h2 = __shfl_xor_sync(FULL_MASK, hi, d);
-            lo = l2 < lo ? l2 : lo;
-            hi = h2 > hi ? h2 : hi;
-        }
-        if ((tid & 31) == 0) { s_min[tid >> 5] = lo; s_max[tid >> 5] = hi; }
-        __syncthreads();
-        if (tid < 32) {
-            lo = s_min[tid]; hi = s_max[tid];
+        // The bins of bins.cuh measure a record from the largest record the buffer can hold.  For a row that passed the
+        // check that is the threshold's key with the last index (its histogram may have been made by the filter kernel);
+        // for a row that was selected exactly, the largest record of the buffer: one pass and a barrier more.
+        uint32_t top_hi;
+        bool counted = false;            // the bins hold this buffer's histogram already
+        if (from_filter) {
+            top_hi = ~tau_key;
+            counted = p.hist_ready && status_ok && __ldcg(&flags[BIN_FLAG_UNCOUNTED]) == 0;
+        } else {
+            unsigned long long hi = 0ull;
+            for_each_record([&](unsigned long long rec) { hi = rec > hi ? rec : hi; });
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) {
-                const unsigned long long l2 = __shfl_xor_sync(FULL_MASK, lo, d), h2 = __shfl_xor_sync(FULL_MASK, hi, d);
-                lo = l2 < lo ? l2 : lo;
+                const unsigned long long h2 = __shfl_xor_sync(FULL_MASK, hi, d);
                 hi = h2 > hi ? h2 : hi;
             }
-            if (tid == 0) { slot_min[cta] = lo; slot_max[cta] = hi; }
-        }
-        if (!barrier(gen)) return;
-        unsigned long long rmin = ~0ull, rmax = 0ull;
-        for (unsigned c = tid & 31; c < nctas; c += 32) {
-            const unsigned long long l2 = __ldcg(&slot_min[c]), h2 = __ldcg(&slot_max[c]);
-            rmin = l2 < rmin ? l2 : rmin;
-            rmax = h2 > rmax ? h2 : rmax;
-        }
+            if ((tid & 31) == 0) s_max[tid >> 5] = hi;
+            __syncthreads();
+            if (tid < 32) {
+                hi = s_max[tid];
 #pragma unroll
-        for (int d = 16; d > 0; d >>= 1) {
-            const unsigned long long l2 = __shfl_xor_sync(FULL_MASK, rmin, d), h2 = __shfl_xor_sync(FULL_MASK, rmax, d);
-            rmin = l2 < rmin ? l2 : rmin;
-            rmax = h2 > rmax ? h2 : rmax;
+                for (int d = 16; d > 0; d >>= 1) {
+                    const unsigned long long h2 = __shfl_xor_sync(FULL_MASK, hi, d);
+                    hi = h2 > hi ? h2 : hi;
+                }
+                if (tid == 0) slot_max[cta] = hi;
+            }
+            if (!barrier(gen)) return;
+            unsigned long long rmax = 0ull;
+            for (unsigned c = tid & 31; c < nctas; c += 32) {
+                const unsigned long long h2 = __ldcg(&slot_max[c]);
+                rmax = h2 > rmax ? h2 : rmax;
+            }
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+                const unsigned long long h2 = __shfl_xor_sync(FULL_MASK, rmax, d);
+                rmax = h2 > rmax ? h2 : rmax;
+            }
+            top_hi = (uint32_t)(rmax >> 32);
         }
-        // Bins on the top LG_BITS bits of the records' range.  A record holds the value key above a 32-bit index, but the
-        // indices of a row only need idx_bits bits: the unused bits in between are squeezed out first (the order is kept),
-        // so that they go to the index instead -- equal values, which differ in the index alone, then spread over 2^(32 -
-        // idx_bits) times as many bins (bf16 rows hold thousands of copies of one value near the threshold: at the
-        // paper's SAE shape a bin held about 800 records and ranking inside the bins took most of the kernel).
         const int ib = p.idx_bits;
-        const unsigned long long hmin = rmin >> 32;
-        auto squeeze = [&](unsigned long long rec) { return (((rec >> 32) - hmin) << ib) | (rec & 0xFFFFFFFFull); };
-        const int rbits = 64 - __clzll((long long)squeeze(rmax));    // squeezed records < 2^rbits
-        const int shift = rbits > LG_BITS ? rbits - LG_BITS : 0;
-        auto bin_of = [&](unsigned long long rec) { return (uint32_t)(squeeze(rec) >> shift); };
+        auto bin_of = [&](unsigned long long rec) { return record_bin(rec, top_hi, ib); };
 
-        // histogram (global atomics spread over the bins)
-        for_each_record([&](unsigned long long rec) { atomicAdd(&bins[bin_of(rec)], 1u); });
-        if (!barrier(gen)) return;
+        if (!counted) {
+            if (clean_bins) {
+                // every CTA zeroed its share of the bins before it waited for the filter kernel and reported in: by now all
+                // have, so this returns at once
+                if (tid == 0) {
+                    uint32_t ok = 1, polls = 0;
+                    while (*((volatile uint32_t*)&p.header->done) < gridDim.x) {
+                        __nanosleep(64);
+                        if (++polls > LG_WAIT_LIMIT) { atomicExch(&p.header->error, 1u); ok = 0; break; }
+                    }
+                    __threadfence();
+                    s_warp[0] = ok;
+                }
+                __syncthreads();
+                const uint32_t ok = s_warp[0];
+                __syncthreads();
+                if (!ok) return;
+                clean_bins = false;
+            } else {
+                for (uint64_t b = gid; b < BIN_ROW_WORDS; b += gthreads)
+                    if (b < BIN_COUNT + 1 || b >= BIN_COUNT + BIN_FLAGS) bins[b] = 0;      // the bins, the "crowded" flag, the coarse bins
+                if (!barrier(gen)) return;
+            }
+            // histogram: fine bins in global memory, coarse bins through shared memory
+            for (uint32_t c = tid; c < BIN_COARSE; c += BT_THREADS) s_coarse[c] = 0;
+            __syncthreads();
+            for_each_record([&](unsigned long long rec) {
+                const uint32_t b = bin_of(rec);
+                atomicAdd(&bins[b], 1u);
+                atomicAdd(&s_coarse[b / BIN_PER_COARSE], 1u);
+            });
+            __syncthreads();
+            for (uint32_t c = tid; c < BIN_COARSE; c += BT_THREADS) {
+                const uint32_t cn = s_coarse[c];
+                if (cn) atomicAdd(&coarse[c], cn);
+            }
+            if (!barrier(gen)) return;
+        }
 
-        // scan: CTA c < scan_ctas owns bins [c, c+1) * LG_BINS / scan_ctas; counts become first positions
-        const uint32_t per_cta = LG_BINS / scan_ctas, per_thr = per_cta / BT_THREADS;
-        const uint32_t b0 = cta * per_cta + tid * per_thr;
-        uint32_t sum = 0, incl = 0;
-        if (cta < scan_ctas) {
-            for (uint32_t j = 0; j < per_thr; ++j) sum += __ldcg(&bins[b0 + j]);
-            incl = sum;
+        // scan: every CTA sums the coarse bins before each of its own; CTA c turns the counts of the fine bins of coarse
+        // bins c, c + nctas, ... into first positions
+        {
+            const uint32_t c = tid < BIN_COARSE ? __ldcg(&coarse[tid]) : 0u;
+            uint32_t incl = c;
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
                 const uint32_t v = __shfl_up_sync(FULL_MASK, incl, d);
@@ -250,30 +290,28 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
             }
             if ((tid & 31) == 31) s_warp[tid >> 5] = incl;
             __syncthreads();
-            if (tid < 32) {
-                uint32_t w = s_warp[tid];
-#pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    const uint32_t v = __shfl_up_sync(FULL_MASK, w, d);
-                    if (tid >= (unsigned)d) w += v;
-                }
-                s_warp[tid] = w;
-                if (tid == 31) slot_total[cta] = w;
-            }
+            uint32_t before = incl - c;
+            for (unsigned w = 0; w < (tid >> 5); ++w) before += s_warp[w];
+            if (tid < BIN_COARSE) s_coarse[tid] = before;                // records in the coarse bins before this one
+            __syncthreads();
         }
-        if (!barrier(gen)) return;
-        if (cta < scan_ctas) {
-            uint32_t before = incl - sum + ((tid >> 5) ? s_warp[(tid >> 5) - 1] : 0);
-            uint32_t ahead = 0;                                      // records in the bins of the CTAs before this one
-            for (unsigned c = tid & 31; c < cta; c += 32) ahead += (uint32_t)__ldcg(&slot_total[c]);
+        for (uint32_t seg = cta; seg < BIN_COARSE; seg += nctas) {
+            const uint32_t b = seg * BIN_PER_COARSE + tid;
+            const uint32_t c = tid < BIN_PER_COARSE ? __ldcg(&bins[b]) : 0u;
+            uint32_t incl = c;
 #pragma unroll
-            for (int d = 16; d > 0; d >>= 1) ahead += __shfl_xor_sync(FULL_MASK, ahead, d);
-            before += ahead;
-            for (uint32_t j = 0; j < per_thr; ++j) {
-                const uint32_t c = __ldcg(&bins[b0 + j]);
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t v = __shfl_up_sync(FULL_MASK, incl, d);
+                if ((tid & 31) >= (unsigned)d) incl += v;
+            }
+            __syncthreads();                                             // s_warp of the round before
+            if ((tid & 31) == 31) s_warp[tid >> 5] = incl;
+            __syncthreads();
+            uint32_t before = s_coarse[seg] + incl - c;
+            for (unsigned w = 0; w < (tid >> 5); ++w) before += s_warp[w];
+            if (tid < BIN_PER_COARSE) {
                 if (before < kk && c > LG_CROWDED) atomicOr(&flags[0], 1u);
-                bins[b0 + j] = before;                               // first position; the scatter advances it to the end
-                before += c;
+                bins[b] = before;                                        // first position; the scatter advances it to the end
             }
         }
         if (!barrier(gen)) return;
