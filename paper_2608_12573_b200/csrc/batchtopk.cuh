@@ -92,7 +92,6 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
     }
     pdl_launch_dependents();
     if (p.use_pdl) pdl_wait();
-    uint32_t gen = *((volatile uint32_t*)&fb.header->bar_gen);          // read before this CTA's first arrival
 
     // ---- the count check of stage 4 (the same in every CTA) ----
     const uint32_t K = fb.k;
@@ -129,10 +128,10 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
     if (status != ROW_OK) {
         // A second filtering pass with the plan's tighter / looser sample rank first, if it names one ...
         uint32_t R2 = 0;
-        const int again = p.direct ? 0 : grid_second_chance_row<T>(fb, 0, status, gen, sh, &R2, &tau_key);
+        const int again = p.direct ? 0 : grid_second_chance_row<T>(fb, 0, status, sh, &R2, &tau_key);
         if (again < 0) return;
         // ... else the exact replacement (Section 3, "Refinement"): the K best records of the whole row, into the buffer.
-        if (again == 0 && !grid_exact_select_row<T>(fb, 0, gen, sh.hist, sh.warp_sums)) return;
+        if (again == 0 && !grid_exact_select_row<T>(fb, 0, sh.hist, sh.warp_sums)) return;
 #pragma unroll
         for (int j = 0; j < (int)FILTER_PARTS; ++j) pcount[j] = 0;
         pcount[0] = again == 1 ? R2 : K;
@@ -181,16 +180,16 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
     const bool have_hist = p.hist_ready && status == ROW_OK && __ldcg(&flags[BIN_FLAG_UNCOUNTED]) == 0;
     if (keep_all) {
         // (the exact selection ended on a grid barrier, but the zero fill above came after it)
-        if (!grid_barrier(fb.header, gen)) return;
+        if (!grid_barrier(fb.header)) return;
     } else if (have_hist) {
         // nothing to count; only the zero fill above has to be over everywhere before anybody emits
-        if ((p.mask || p.dense) && !grid_barrier(fb.header, gen)) return;
+        if ((p.mask || p.dense) && !grid_barrier(fb.header)) return;
     } else if (p.hist_ready) {
         // the bins hold the counts of the first filtering pass, the buffer the records of the second: start again
         // (nobody has read the bins yet; the flags behind them are still zero)
         for (uint64_t b = gid; b < BIN_COUNT; b += gthreads) p.bins[b] = 0;
         for (uint64_t b = gid; b < BIN_COARSE; b += gthreads) coarse[b] = 0;
-        if (!grid_barrier(fb.header, gen)) return;
+        if (!grid_barrier(fb.header)) return;
     } else {
         // every CTA has zeroed its share of the bins: reported before the wait for the filter kernel, so this returns at once
         if (tid == 0) {
@@ -229,7 +228,7 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
                 const uint32_t n = s_coarse[c];
                 if (n) atomicAdd(&coarse[c], n);
             }
-            if (!grid_barrier(fb.header, gen)) return;
+            if (!grid_barrier(fb.header)) return;
         }
         // every CTA: the coarse bin, then the fine bin, of the need-th best record of the class
         {
@@ -254,10 +253,10 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
         if (in_bin == need) { whole = true; break; }
         if (in_bin <= BK_EDGE) break;
         // crowded: one more level inside the class; the bins start from zero again
-        if (!grid_barrier(fb.header, gen)) return;                        // everybody has read this level's bins
+        if (!grid_barrier(fb.header)) return;                        // everybody has read this level's bins
         for (uint64_t b = gid; b < BK_BINS; b += gthreads) p.bins[b] = 0;
         for (uint64_t b = gid; b < BK_COARSE; b += gthreads) coarse[b] = 0;
-        if (!grid_barrier(fb.header, gen)) return;
+        if (!grid_barrier(fb.header)) return;
     }
     // Kept outright: D >= keep_from.  Boundary list: cls_lo <= D < keep_from (empty when the whole class is kept).
     const bool top_class = cls_w >= 64 || cls_lo + (1ull << cls_w) < cls_lo;      // the class reaches the largest D there is
@@ -272,50 +271,73 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
         if (p.mask) atomicOr(&p.mask[idx >> 5], 1u << (idx & 31u));
         if (p.dense) p.dense[idx] = val;
     };
-    for (uint32_t it = 0; it < iters; ++it) {
-        const uint64_t i = (uint64_t)it * gthreads + gid;
-        uint64_t rec = 0;
-        bool kept = false, boundary = false;
-        if (i < total) {
-            rec = record_at(i);
-            const uint64_t D = dist(rec);
-            kept = keep_all || (whole ? D >= keep_from : (!top_class && D >= keep_from));
-            boundary = !kept && !whole && D >= cls_lo;
+    // Each thread takes up to EM records at a time (their loads in flight together); the CTA reserves room in the pair list
+    // for all of them with one atomic.
+    constexpr int EM = 4;
+    for (uint32_t it0 = 0; it0 < iters; it0 += EM) {
+        uint64_t rec[EM];
+        bool valid[EM];
+#pragma unroll
+        for (int u = 0; u < EM; ++u) {
+            const uint64_t i = (uint64_t)(it0 + u) * gthreads + gid;
+            valid[u] = it0 + u < iters && i < total;
+            rec[u] = valid[u] ? record_at(i) : 0ull;
         }
-        const unsigned bal = __ballot_sync(FULL_MASK, kept);
-        if (lane == 0) s_warp_count[warp] = __popc(bal);
-        const unsigned ebal = __ballot_sync(FULL_MASK, boundary);
-        if (ebal) {
-            uint32_t ebase = 0;
-            if (lane == 0) ebase = atomicAdd(&flags[1], (uint32_t)__popc(ebal));
-            ebase = __shfl_sync(FULL_MASK, ebase, 0);
-            const uint32_t epos = ebase + __popc(ebal & ((1u << lane) - 1u));
-            if (boundary && epos < BK_EDGE) p.edge[epos] = rec;
+        unsigned keptm = 0, cnt = 0;               // bit u: record u is kept outright
+#pragma unroll
+        for (int u = 0; u < EM; ++u) {
+            bool kept = false, boundary = false;
+            if (valid[u]) {
+                const uint64_t D = dist(rec[u]);
+                kept = keep_all || (whole ? D >= keep_from : (!top_class && D >= keep_from));
+                boundary = !kept && !whole && D >= cls_lo;
+            }
+            keptm |= kept ? 1u << u : 0u;
+            cnt += kept ? 1u : 0u;
+            const unsigned ebal = __ballot_sync(FULL_MASK, boundary);
+            if (ebal) {
+                uint32_t ebase = 0;
+                if (lane == 0) ebase = atomicAdd(&flags[1], (uint32_t)__popc(ebal));
+                ebase = __shfl_sync(FULL_MASK, ebase, 0);
+                const uint32_t epos = ebase + __popc(ebal & ((1u << lane) - 1u));
+                if (boundary && epos < BK_EDGE) p.edge[epos] = rec[u];
+            }
         }
+        uint32_t incl = cnt;                       // prefix of the counts over the warp, then over the CTA
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t v = __shfl_up_sync(FULL_MASK, incl, d);
+            if (lane >= (unsigned)d) incl += v;
+        }
+        if (lane == 31) s_warp_count[warp] = incl;
         __syncthreads();
-        if (warp == 0) {                           // one atomic per CTA and pass
+        if (warp == 0) {
             const uint32_t c = s_warp_count[lane];
-            uint32_t incl = c;
+            uint32_t wi = c;
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t v = __shfl_up_sync(FULL_MASK, incl, d);
-                if (lane >= (unsigned)d) incl += v;
+                const uint32_t v = __shfl_up_sync(FULL_MASK, wi, d);
+                if (lane >= (unsigned)d) wi += v;
             }
             uint32_t base = 0;
-            if (lane == 31 && incl) base = atomicAdd(&flags[0], incl);
+            if (lane == 31 && wi) base = atomicAdd(&flags[0], wi);
             base = __shfl_sync(FULL_MASK, base, 31);
-            s_warp_count[lane] = base + incl - c;  // first position of the warp's records
+            s_warp_count[lane] = base + wi - c;    // first position of the warp's records
         }
         __syncthreads();
-        if (kept) {
-            const uint32_t pos = s_warp_count[warp] + __popc(bal & ((1u << lane) - 1u));
-            if (pos < n_outright) emit(rec, pos);
+        uint32_t pos = s_warp_count[warp] + incl - cnt;
+#pragma unroll
+        for (int u = 0; u < EM; ++u) {
+            if ((keptm >> u) & 1u) {
+                if (pos < n_outright) emit(rec[u], pos);
+                ++pos;
+            }
         }
-        __syncthreads();                           // s_warp_count is rewritten by the next pass
+        __syncthreads();                           // s_warp_count is rewritten by the next round
     }
     if (whole) return;
 
-    // ---- the boundary class: the CTA that finishes last ranks its records and keeps the best `need` ----
+    // ---- the boundary class: the CTA that finishes last keeps its best `need` records ----
     __threadfence();                               // this thread's appends to the boundary list are out ...
     __syncthreads();                               // ... for every thread of the CTA
     if (tid == 0) s_ok = atomicAdd(&flags[2], 1u) == nctas - 1 ? 1u : 0u;
@@ -323,15 +345,36 @@ __global__ void __launch_bounds__(BK_THREADS, 1) batchtopk_emit_kernel(const Bat
     if (!s_ok) return;
     __threadfence();
     const uint32_t n_edge = min(__ldcg(&flags[1]), BK_EDGE);
-    uint64_t* list = sh.edge;                      // RF_EDGE_CAP == BK_EDGE records of shared memory
-    static_assert(RF_EDGE_CAP >= BK_EDGE, "the boundary list fits SelectShared::edge");
-    for (uint32_t i = tid; i < n_edge; i += BK_THREADS) list[i] = __ldcg(&p.edge[i]);
+    static_assert(BK_EDGE <= BK_THREADS && BK_EDGE <= RF_BINS && RF_EDGE_CAP >= BK_EDGE, "one thread, one bin and one slot per boundary record");
+    // One more level in shared memory: the class's D range cut into BK_EDGE slices, best first.  Slices before the one
+    // that holds the need-th best record are kept whole; of that slice -- a record or two as a rule -- the best are
+    // found by comparing its records with one another.
+    const int sl_shift = cls_w > 10 ? cls_w - 10 : 0;
+    const uint64_t mine = tid < n_edge ? __ldcg(&p.edge[tid]) : 0ull;
+    const uint32_t slice = tid < n_edge ? BK_EDGE - 1 - (uint32_t)(((dist(mine) - cls_lo) >> sl_shift) & (BK_EDGE - 1)) : 0u;
+    sh.hist[tid] = 0;
+    if (tid == 0) { sh.fill = 0; sh.n_edge = 0; }
     __syncthreads();
-    for (uint32_t i = tid; i < n_edge; i += BK_THREADS) {
-        const uint64_t mine = list[i];
+    if (tid < n_edge) atomicAdd(&sh.hist[slice], 1u);
+    __syncthreads();
+    {
+        const uint32_t c = sh.hist[tid];
+        const uint32_t incl = block_inclusive_scan(c, sh.warp_sums);
+        if (incl - c < need && need <= incl) { s_bin = tid; s_bin_before = incl - c; }
+        __syncthreads();
+    }
+    const uint32_t edge_slice = s_bin, edge_before = s_bin_before;
+    uint64_t* list = sh.edge;                      // the records of that slice
+    if (tid < n_edge) {
+        if (slice < edge_slice) emit(mine, n_outright + atomicAdd(&sh.fill, 1u));
+        else if (slice == edge_slice) list[atomicAdd(&sh.n_edge, 1u)] = mine;
+    }
+    __syncthreads();
+    const uint32_t n_list = sh.n_edge;
+    if (tid < n_edge && slice == edge_slice) {
         uint32_t rank = 0;
-        for (uint32_t j = 0; j < n_edge; ++j) rank += list[j] < mine;
-        if (rank < need) emit(mine, n_outright + rank);
+        for (uint32_t j = 0; j < n_list; ++j) rank += list[j] < mine;
+        if (rank < need - edge_before) emit(mine, n_outright + edge_before + rank);
     }
 }
 

@@ -89,18 +89,17 @@ __device__ __forceinline__ void for_each_record(const FallbackParams<T>& p, uint
 // Exact selection of the k smallest records of `row` by the whole grid (FB_THREADS threads per CTA, all CTAs
 // co-resident): a most-significant-digit radix select over the row's elements as 64-bit records, 11 bits per pass,
 // a grid barrier after each, then one more read of the row that appends the k winners to the row's buffer (counter:
-// the row's `collect` word, zero on entry).  Called by every thread of every CTA; `gen` is the caller's copy of the
-// grid barrier's generation.  Returns false when a bounded wait gave up (the caller leaves the kernel); on a true
+// the row's `collect` word, zero on entry).  Called by every thread of every CTA.  Returns false when a bounded wait gave up (the caller leaves the kernel); on a true
 // return the last barrier has been passed and the k records are in p.buf + row * p.buf_stride, in no particular order.
 template <typename T>
-__device__ __noinline__ bool grid_exact_select_row(const FallbackParams<T>& p, uint64_t row, uint32_t& gen, uint32_t* sh_hist,
+__device__ __noinline__ bool grid_exact_select_row(const FallbackParams<T>& p, uint64_t row, uint32_t* sh_hist,
                                                    uint32_t* warp_sums) {
     __shared__ uint32_t s_digit, s_before, s_cnt;
     const unsigned tid = threadIdx.x, lane = lane_id();
-    if (!grid_barrier(p.header, gen)) return false;          // a previous row's histogram reads are over
+    if (!grid_barrier(p.header)) return false;          // a previous row's histogram reads are over
     for (uint32_t i = blockIdx.x * FB_THREADS + tid; i < FB_PASSES * FB_BINS; i += gridDim.x * FB_THREADS)
         p.ghist[i] = 0;
-    if (!grid_barrier(p.header, gen)) return false;
+    if (!grid_barrier(p.header)) return false;
 
     uint64_t prefix = 0;       // selected high bits, right-aligned
     uint32_t need = p.k;       // rank (from the smallest record) inside the prefix class
@@ -123,7 +122,7 @@ __device__ __noinline__ bool grid_exact_select_row(const FallbackParams<T>& p, u
             const uint32_t c = sh_hist[i];
             if (c) atomicAdd(&gh[i], c);
         }
-        if (!grid_barrier(p.header, gen)) return false;
+        if (!grid_barrier(p.header)) return false;
 
         // Every CTA finds the bin that holds the need-th smallest record of the class.
         constexpr int PER = FB_BINS / FB_THREADS;                   // bins per thread
@@ -166,7 +165,7 @@ __device__ __noinline__ bool grid_exact_select_row(const FallbackParams<T>& p, u
             if (take && pos < p.capacity) dst[pos] = rec;
         }
     });
-    return grid_barrier(p.header, gen);
+    return grid_barrier(p.header);
 }
 
 // The second filtering pass (second_chance.cuh) of a row that failed the count check with `status`, by the whole grid:
@@ -177,7 +176,7 @@ __device__ __noinline__ bool grid_exact_select_row(const FallbackParams<T>& p, u
 // says so; 0 when no second pass applies (no keys kept, no such rank in the plan) or the row failed again; -1 when a
 // bounded wait gave up (the caller leaves the kernel).  Called by every thread of every CTA (FB_THREADS threads).
 template <typename T>
-__device__ __noinline__ int grid_second_chance_row(const FallbackParams<T>& p, uint64_t row, uint32_t status, uint32_t& gen, SelectShared& sh,
+__device__ __noinline__ int grid_second_chance_row(const FallbackParams<T>& p, uint64_t row, uint32_t status, SelectShared& sh,
                                                    uint32_t* R2_out, uint32_t* key2_out) {
     const SampleInfo& sm = p.sample;
     if (sm.keys == nullptr) return 0;
@@ -199,7 +198,7 @@ __device__ __noinline__ int grid_second_chance_row(const FallbackParams<T>& p, u
     fp.counts = &p.ctl[0].pad; fp.count_stride = sizeof(RowCtl) / 4;
     fp.thr = p.thr2;
     refilter_tiles<T, FB_THREADS>(fp, (uint32_t)row, 0, p.tiles_per_row, blockIdx.x, gridDim.x, tau2);
-    if (!grid_barrier(p.header, gen)) return -1;
+    if (!grid_barrier(p.header)) return -1;
     const uint32_t R2 = __ldcg(&p.ctl[row].pad);
     if (R2 < p.k || R2 > p.capacity) return 0;                 // (the same decision in every CTA)
     if (blockIdx.x == 0 && tid == 0) {
@@ -254,7 +253,6 @@ __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackPara
         return;
     }
 
-    uint32_t gen = *((volatile uint32_t*)&p.header->bar_gen);   // read before this CTA's first arrival
 
     for (uint64_t chunk = 0; chunk < p.rows; chunk += FB_THREADS) {
         // ---- FB_THREADS rows at a time; every CTA reads the same status words ----
@@ -274,7 +272,7 @@ __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackPara
                 // ---- first another filtering pass with the plan's tighter / looser sample rank, if it names one ----
                 if (p.sort_rows) {
                     uint32_t R2 = 0, key2 = 0;
-                    const int again = grid_second_chance_row<T>(p, row, __ldcg(&p.ctl[row].status), gen, sh, &R2, &key2);
+                    const int again = grid_second_chance_row<T>(p, row, __ldcg(&p.ctl[row].status), sh, &R2, &key2);
                     if (again < 0) return;
                     if (again == 1) {
                         if (blockIdx.x == 0) {
@@ -287,7 +285,7 @@ __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackPara
                     }
                 }
                 // ---- exact selection of the k smallest records of `row` into the row's buffer ----
-                if (!grid_exact_select_row<T>(p, row, gen, sh_hist, warp_sums)) return;
+                if (!grid_exact_select_row<T>(p, row, sh_hist, warp_sums)) return;
                 uint64_t* dst = p.buf + row * p.buf_stride;
 
                 // ---- order the k records and write the row's output (first CTA; the others move on

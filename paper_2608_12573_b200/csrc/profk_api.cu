@@ -458,7 +458,12 @@ int launch_refine(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, Ro
 // elements per warp-tile): 512 rows of 2^20, k = 32 (1.46 per warp-tile) 298 -> 260 us; the paper's SAE shape (3.2)
 // 112 -> 97, where it also replaces the staged build.  fp32: the SAE shape (1.6) 93.4 -> 89.3; batches of fp32 rows
 // (0.73) lose 6 % (397 -> 422 us) and stay on the direct build; 2^29 bf16, K = 131072 (0.4) is indifferent.
-template <typename T> bool defer_candidates(int64_t rows, double per_warp_tile) {
+// A large selection from a single row (and the BatchTopK entry points) gains more: the deferring build also hands the
+// kernel behind it a finished histogram (HIST, filter.cuh) and needs no partitioned append; from 0.1 survivors per
+// warp-tile on it wins (2^29 bf16, K = 131072 at 0.41: 218 -> 212 us; 2^26 fp32, k = 32768 at 0.36: 89 -> 81; 2^28 bf16,
+// k = 20000 at 0.18: 127 -> 120; at 0.05 it loses half a percent to the direct build with its prefetched tiles).
+template <typename T> bool defer_candidates(int64_t rows, double per_warp_tile, bool large_one_row = false) {
+    if (large_one_row) return per_warp_tile > 0.1;
     if (sizeof(T) == 2) return per_warp_tile > 0.8;
     return rows == 1 && per_warp_tile > 1.0;
 }
@@ -515,7 +520,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         // (The direct append has three CTAs per SM, eight counters for large selections and the prefetch behind the threshold
     // kernel; it holds up to about two survivors per warp-tile: 2^29 bf16, K = 131072 at 0.4: 248 -> 237 us; 50 M fp32,
     // K = 131072 at 1.6: 124 -> 114; 50 M bf16 at 3.2 stays staged, 120 against 127.)
-    const bool deferred = plan->mode == 0 && defer_candidates<T>(rows, per_warp_tile);
+    const bool deferred = plan->mode == 0 && defer_candidates<T>(rows, per_warp_tile, large && rows == 1);
     const bool staged = plan->mode == 0 && !deferred && rows == 1 && per_warp_tile > 2.0;
 
     // Large selections keep so many survivors that a row's single append counter would hold the scan up:
@@ -691,7 +696,7 @@ int batchtopk_planned(const T* in, int64_t N, int64_t K, const profk_plan_t* pla
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
     const double per_warp_tile = (double)plan->r / (double)std::max<int64_t>(plan->m, 1) * 32.0 * FILTER_UNROLL * Elem<T>::VEC;
-    const bool deferred = plan->mode == 0 && defer_candidates<T>(1, per_warp_tile);       // as in topk_planned
+    const bool deferred = plan->mode == 0 && defer_candidates<T>(1, per_warp_tile, true);       // as in topk_planned for a large selection
     const bool staged = plan->mode == 0 && !deferred && per_warp_tile > 2.0;
     const bool parts = !staged && !deferred && plan->mode == 0;
     const uint32_t part_cap = (uint32_t)(row_stride / 2 / FILTER_PARTS);

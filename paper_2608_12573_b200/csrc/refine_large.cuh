@@ -93,8 +93,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
     const uint64_t gthreads = (uint64_t)nctas * BT_THREADS;
     unsigned long long* slot_max = p.slots + gridDim.x + group * nctas;
     uint32_t* bar_count = &p.header->group_bar[group][0];
-    uint32_t* bar_gen = &p.header->group_bar[group][1];
-    auto barrier = [&](uint32_t& g) { return cta_group_barrier(bar_count, bar_gen, &p.header->error, nctas, g); };
+    auto barrier = [&]() { return cta_group_barrier(bar_count, &p.header->error, nctas); };
 
     // A single row whose filter did not count: the bins are cleared here, before the wait for the filter kernel, and each
     // CTA reports in through the header's `done` word (zeroed by the call's first kernel, long finished).
@@ -107,8 +106,6 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
     }
     pdl_launch_dependents();
     if (p.use_pdl) pdl_wait();
-    uint32_t gen = *((volatile uint32_t*)bar_gen);                   // read before this CTA's first arrival
-    uint32_t grid_gen = *((volatile uint32_t*)&p.header->bar_gen);   // the same for the grid-wide barrier of the exact selection
 
     for (uint64_t row = group; row < p.rows; row += p.groups) {
         // ---- is this row for this launch?  (the decision is the same in every CTA) ----
@@ -150,10 +147,10 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
                 // first a second filtering pass with the plan's tighter / looser sample rank, if it names one (the tile in
                 // shared memory, unused so far, holds that pass's selection state) ...
                 uint32_t R2 = 0, key2 = 0;
-                const int again = direct ? 0 : grid_second_chance_row<T>(p.fb, row, status, grid_gen, *reinterpret_cast<SelectShared*>(smem_raw), &R2, &key2);
+                const int again = direct ? 0 : grid_second_chance_row<T>(p.fb, row, status, *reinterpret_cast<SelectShared*>(smem_raw), &R2, &key2);
                 if (again < 0) return;
                 // ... else the k best records of the whole row into the row's buffer; ordered below like any buffer
-                if (again == 0 && !grid_exact_select_row<T>(p.fb, row, grid_gen, reinterpret_cast<uint32_t*>(tile), s_warp)) return;
+                if (again == 0 && !grid_exact_select_row<T>(p.fb, row, reinterpret_cast<uint32_t*>(tile), s_warp)) return;
                 nparts = 1;
 #pragma unroll
                 for (int j = 0; j < (int)FILTER_PARTS; ++j) pcount[j] = 0;
@@ -180,13 +177,20 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
 #pragma unroll
             for (int j = 0; j < (int)FILTER_PARTS; ++j) { acc += pcount[j]; pend[j] = acc; }
         }
-        auto for_each_record = [&](auto&& f) {
-            for (uint64_t i = gid; i < pend[FILTER_PARTS - 1]; i += gthreads) {
-                uint32_t j = 0, before = 0;
+        auto record_at = [&](uint64_t i) {
+            uint32_t j = 0, before = 0;
 #pragma unroll
-                for (int q = 0; q < (int)FILTER_PARTS - 1; ++q)
-                    if (i >= pend[q]) { j = q + 1; before = pend[q]; }
-                f((unsigned long long)__ldcg(G + (uint64_t)j * p.part_cap + (i - before)));
+            for (int q = 0; q < (int)FILTER_PARTS - 1; ++q)
+                if (i >= pend[q]) { j = q + 1; before = pend[q]; }
+            return (unsigned long long)__ldcg(G + (uint64_t)j * p.part_cap + (i - before));
+        };
+        auto for_each_record = [&](auto&& f) {           // (two loads in flight per thread: a pass is one or two rounds long)
+            const uint64_t total = pend[FILTER_PARTS - 1];
+            for (uint64_t i = gid; i < total; i += 2 * gthreads) {
+                const bool two = i + gthreads < total;
+                const unsigned long long r0 = record_at(i), r1 = two ? record_at(i + gthreads) : 0ull;
+                f(r0);
+                if (two) f(r1);
             }
         };
 
@@ -223,7 +227,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
                 }
                 if (tid == 0) slot_max[cta] = hi;
             }
-            if (!barrier(gen)) return;
+            if (!barrier()) return;
             unsigned long long rmax = 0ull;
             for (unsigned c = tid & 31; c < nctas; c += 32) {
                 const unsigned long long h2 = __ldcg(&slot_max[c]);
@@ -260,7 +264,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
             } else {
                 for (uint64_t b = gid; b < BIN_ROW_WORDS; b += gthreads)
                     if (b < BIN_COUNT + 1 || b >= BIN_COUNT + BIN_FLAGS) bins[b] = 0;      // the bins, the "crowded" flag, the coarse bins
-                if (!barrier(gen)) return;
+                if (!barrier()) return;
             }
             // histogram: fine bins in global memory, coarse bins through shared memory
             for (uint32_t c = tid; c < BIN_COARSE; c += BT_THREADS) s_coarse[c] = 0;
@@ -275,51 +279,48 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
                 const uint32_t cn = s_coarse[c];
                 if (cn) atomicAdd(&coarse[c], cn);
             }
-            if (!barrier(gen)) return;
+            if (!barrier()) return;
         }
 
         // scan: every CTA sums the coarse bins before each of its own; CTA c turns the counts of the fine bins of coarse
         // bins c, c + nctas, ... into first positions
         {
             const uint32_t c = tid < BIN_COARSE ? __ldcg(&coarse[tid]) : 0u;
-            uint32_t incl = c;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t v = __shfl_up_sync(FULL_MASK, incl, d);
-                if ((tid & 31) >= (unsigned)d) incl += v;
-            }
-            if ((tid & 31) == 31) s_warp[tid >> 5] = incl;
-            __syncthreads();
-            uint32_t before = incl - c;
-            for (unsigned w = 0; w < (tid >> 5); ++w) before += s_warp[w];
-            if (tid < BIN_COARSE) s_coarse[tid] = before;                // records in the coarse bins before this one
+            const uint32_t incl = block_inclusive_scan(c, s_warp);
+            if (tid < BIN_COARSE) s_coarse[tid] = incl - c;              // records in the coarse bins before this one
             __syncthreads();
         }
-        for (uint32_t seg = cta; seg < BIN_COARSE; seg += nctas) {
-            const uint32_t b = seg * BIN_PER_COARSE + tid;
-            const uint32_t c = tid < BIN_PER_COARSE ? __ldcg(&bins[b]) : 0u;
-            uint32_t incl = c;
+        constexpr int SEG_AHEAD = 4;                                     // counts loaded ahead: a CTA of a full grid has at most four coarse bins
+        uint32_t ahead[SEG_AHEAD];
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t v = __shfl_up_sync(FULL_MASK, incl, d);
-                if ((tid & 31) >= (unsigned)d) incl += v;
+        for (int a = 0; a < SEG_AHEAD; ++a) {
+            const uint32_t seg = cta + a * nctas;
+            ahead[a] = seg < BIN_COARSE && tid < BIN_PER_COARSE ? __ldcg(&bins[seg * BIN_PER_COARSE + tid]) : 0u;
+        }
+        int turn = 0;
+        for (uint32_t seg = cta; seg < BIN_COARSE; seg += nctas, ++turn) {
+            const uint32_t b = seg * BIN_PER_COARSE + tid;
+            uint32_t c = 0;
+            if (turn < SEG_AHEAD) {
+#pragma unroll
+                for (int a = 0; a < SEG_AHEAD; ++a)
+                    if (a == turn) c = ahead[a];
+            } else if (tid < BIN_PER_COARSE) {
+                c = __ldcg(&bins[b]);
             }
             __syncthreads();                                             // s_warp of the round before
-            if ((tid & 31) == 31) s_warp[tid >> 5] = incl;
-            __syncthreads();
-            uint32_t before = s_coarse[seg] + incl - c;
-            for (unsigned w = 0; w < (tid >> 5); ++w) before += s_warp[w];
+            const uint32_t before = s_coarse[seg] + block_inclusive_scan(c, s_warp) - c;
             if (tid < BIN_PER_COARSE) {
                 if (before < kk && c > LG_CROWDED) atomicOr(&flags[0], 1u);
                 bins[b] = before;                                        // first position; the scatter advances it to the end
             }
         }
-        if (!barrier(gen)) return;
+        if (!barrier()) return;
 
         if (__ldcg(&flags[0]) == 0) {
             // scatter into the second buffer, grouped by bin
             for_each_record([&](unsigned long long rec) { G2[atomicAdd(&bins[bin_of(rec)], 1u)] = rec; });
-            if (!barrier(gen)) return;
+            if (!barrier()) return;
             // rank inside the bin: bin b now occupies [end of bin b-1, bins[b])
             // (only positions below the end of the bin that holds position kk-1 matter; they are a prefix)
             const uint64_t g_end = (uint64_t)kk + LG_CROWDED < n ? (uint64_t)kk + LG_CROWDED : n;
@@ -344,9 +345,9 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
                 for (uint64_t i = gid; i < pcount[j]; i += gthreads) G2[first + i] = __ldcg(&part[i]);
                 first += pcount[j];
             }
-            if (!barrier(gen)) return;
+            if (!barrier()) return;
             for (uint64_t i = gid; i < n; i += gthreads) G[i] = __ldcg(&G2[i]);
-            if (!barrier(gen)) return;
+            if (!barrier()) return;
         }
         uint64_t P = BT_TILE;
         while (P < n) P <<= 1;
@@ -361,7 +362,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
             for (uint32_t i = tid; i < BT_TILE; i += BT_THREADS) G[base + i] = tile[i];
             __syncthreads();
         }
-        if (!barrier(gen)) return;
+        if (!barrier()) return;
 
         // ---- merge: exchanges at distance >= BT_TILE on the buffer, the rest tile by tile ----
         for (uint64_t size = 2ull * BT_TILE; size <= P; size <<= 1) {
@@ -373,7 +374,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
                     const uint64_t x = __ldcg(&G[lo2]), y = __ldcg(&G[hi2]);
                     if ((x > y) == ascending) { G[lo2] = y; G[hi2] = x; }
                 }
-                if (!barrier(gen)) return;
+                if (!barrier()) return;
             }
             for (uint64_t t = cta; t < tiles; t += nctas) {
                 const uint64_t base = t * BT_TILE;
@@ -383,7 +384,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
                 for (uint32_t i = tid; i < BT_TILE; i += BT_THREADS) G[base + i] = tile[i];
                 __syncthreads();
             }
-            if (!barrier(gen)) return;
+            if (!barrier()) return;
         }
 
         for (uint64_t j = gid; j < kk; j += gthreads) write_output(p.out_vals, p.out_idx, p.k, row, (uint32_t)j, __ldcg(&G[j]));

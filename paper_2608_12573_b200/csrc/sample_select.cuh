@@ -53,14 +53,14 @@ constexpr int WS_GROUPS = 32;            // most CTA groups of the large-k refin
 
 // Header of the workspace: state of the grid barrier used by the exact-selection kernel.
 struct WsHeader {
-    uint32_t bar_count;
-    uint32_t bar_gen;
+    uint32_t bar_count;  // arrivals at the grid barrier since the start of the call (grid_barrier.cuh)
+    uint32_t bar_gen;    // (unused)
     uint32_t error;      // non-zero = a bounded wait gave up
     uint32_t done;       // CTAs of the filter kernel that have finished (ticket for its last CTA)
     uint32_t n_failed;   // rows whose count check failed
     uint32_t tile_counter;  // hands out the filter kernel's tiles
     uint32_t pad[58];
-    uint32_t group_bar[WS_GROUPS][2];   // barriers of the CTA groups of the large-k refine: {arrivals, generation}
+    uint32_t group_bar[WS_GROUPS][2];   // barriers of the CTA groups of the large-k refine: {arrivals, unused}
 };
 static_assert(sizeof(WsHeader) == 512, "WsHeader is 512 bytes");
 

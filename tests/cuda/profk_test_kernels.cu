@@ -20,8 +20,7 @@ __global__ void early_trigger_copy_kernel(const float* src, float* dst, int64_t 
 // wait runs out after `polls` polls, sets the workspace's error flag and returns.  returned[cta] = 1 + what the
 // barrier reported (so 1 = "gave up", and 0 would mean the CTA never came back).
 __global__ void barrier_timeout_kernel(profk::WsHeader* header, uint32_t members, uint32_t polls, uint32_t* returned) {
-    uint32_t gen = *((volatile uint32_t*)&header->bar_gen);
-    const bool ok = profk::cta_group_barrier(&header->bar_count, &header->bar_gen, &header->error, members, gen, polls);
+    const bool ok = profk::cta_group_barrier(&header->bar_count, &header->error, members, polls);
     if (threadIdx.x == 0) returned[blockIdx.x] = 1u + (ok ? 1u : 0u);
 }
 
