@@ -4,11 +4,12 @@
 // The kernel is bound by HBM bandwidth: one 128-bit load per VEC elements, one compare
 // per element, and nothing else on the common path.  Survivors are rare (1e-3 .. 1e-5 of
 // the elements), so the append is a warp-cooperative slow path taken only when some lane
-// of the warp saw a survivor.  Survivors are first collected in a small per-warp stage in
-// shared memory and appended to the row buffer 32 or more at a time, so the round trip of
-// the global counter atomic is paid once per flush, not once per tile with a survivor; the
-// slow path is a separate function so that its registers do not limit the occupancy of the
-// streaming loop.
+// of the warp saw a survivor: one atomic on the row's counter per warp and tile, records
+// written straight to the row's buffer (eight counters and eight parts of the buffer for
+// large selections from long rows).  Where survivors are dense -- one or more per
+// warp-tile -- the DEFER build only notes its candidates while it streams and decides them
+// afterwards, with every lane busy; its HIST form also counts the records it appends in
+// the bins that the kernel behind it selects from.
 #pragma once
 
 #include "bins.cuh"
@@ -26,9 +27,6 @@
 #endif
 #ifndef PROFK_FILTER_MINBLOCKS_BF16
 #define PROFK_FILTER_MINBLOCKS_BF16 3            // the direct-append variant fits 40 registers without spills
-#endif
-#ifndef PROFK_FILTER_MINBLOCKS_STAGED
-#define PROFK_FILTER_MINBLOCKS_STAGED 2          // the staged variants do not: they spill at 40 and lose more than they gain
 #endif
 
 namespace profk {
@@ -233,137 +231,7 @@ __device__ __forceinline__ void emit_survivors(const typename Elem<T>::vec_t (&v
     }
 }
 
-constexpr uint32_t STAGE_CAP = 64;       // records a warp collects in shared memory ...
-constexpr uint32_t STAGE_FLUSH = 32;     // ... and the fill at which it appends them to the row buffer
-
-// Per-warp staging state, kept in shared memory so that the streaming loop carries none of it.
-struct WarpStage {
-    uint64_t rec[STAGE_CAP];
-    uint32_t fill;        // records waiting
-    uint32_t row;         // the row they belong to
-};
-
-// Appends a warp's staged records to their row's buffer: one global atomic and a few coalesced
-// stores per STAGE_FLUSH survivors.  Returns the row if its buffer has overflowed, else ~0.
-template <typename T>
-__device__ __noinline__ uint32_t flush_stage(const FilterParams<T>& p, WarpStage* st) {
-    const unsigned lane = lane_id();
-    const uint32_t fill = st->fill, row = st->row;
-    unsigned base = 0;
-    if (lane == 0) base = atomicAdd(p.counts + (uint64_t)row * p.count_stride, fill);
-    base = __shfl_sync(FULL_MASK, base, 0);
-    uint64_t* dst = p.buf + (uint64_t)row * p.buf_stride;
-    for (uint32_t i = lane; i < fill; i += 32)
-        if (base + i < p.capacity) dst[base + i] = st->rec[i];
-    __syncwarp();
-    if (lane == 0) st->fill = 0;
-    __syncwarp();
-    return (uint64_t)base + fill > p.capacity ? row : 0xFFFFFFFFu;
-}
-
-// The slow path of one warp and one tile: exact per-element test, records into the warp's stage
-// (or straight into the buffer when the tile is full of survivors).  Kept out of line so that its
-// registers do not weigh on the streaming loop.  Returns a row whose buffer has overflowed, or ~0.
-template <typename T, int THREADS, int UNROLL>
-__device__ __noinline__ uint32_t filter_slow_path(const FilterParams<T>& p, WarpStage* st,
-                                                  typename Elem<T>::vec_t v0, typename Elem<T>::vec_t v1,
-                                                  typename Elem<T>::vec_t v2, typename Elem<T>::vec_t v3,
-                                                  uint32_t inside_mask, uint32_t row, uint64_t qbase, uint32_t mis, T tau) {
-    using V = typename Elem<T>::vec_t;
-    constexpr int VEC = Elem<T>::VEC;
-    static_assert(UNROLL == 4, "the slow path takes four vectors");
-    const V v[4] = {v0, v1, v2, v3};
-    const unsigned lane = lane_id();
-    // Per element: a survivor mask, the warp's prefix of the counts, then the records.  With four elements
-    // per vector the straight-line form (every element tested and written under a predicate) is the cheaper
-    // one, also in registers; with eight it is a loop over the set bits of the mask.
-    constexpr bool STRAIGHT = VEC <= 4;
-    unsigned mine_u[UNROLL];        // STRAIGHT: per vector, bit l set = element l survives
-    uint32_t mine = 0;              // otherwise: bit u * VEC + l
-    unsigned cnt = 0, total, before;
-    if constexpr (STRAIGHT) {
-        const float tau_f = Elem<T>::as_float(tau);
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-            mine_u[u] = 0;
-            if (((inside_mask >> u) & 1u) && vec_any_pass(v[u], tau)) {      // most vectors hold no survivor
-                const uint64_t q = qbase + (uint64_t)u * THREADS + threadIdx.x;
-                const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
-#pragma unroll
-                for (int l = 0; l < VEC; ++l) {
-                    const int64_t i = i0 + l;
-                    const bool ok = i >= 0 && i < (int64_t)p.N && !(Elem<T>::as_float(vec_elem(v[u], l)) < tau_f);
-                    if (ok) mine_u[u] |= 1u << l;
-                }
-                mine_u[u] = confirm_survivors<T>(p, row, v[u], mine_u[u], i0, tau);
-            }
-            cnt += __popc(mine_u[u]);
-        }
-        unsigned incl = cnt;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const unsigned nb = __shfl_up_sync(FULL_MASK, incl, d);
-            if (lane >= (unsigned)d) incl += nb;
-        }
-        total = __shfl_sync(FULL_MASK, incl, 31);
-        before = incl - cnt;
-    } else {
-        mine = survivor_mask<T, THREADS, UNROLL>(v, inside_mask, p.N, qbase, mis, tau, p, row);
-        cnt = __popc(mine);
-        before = warp_exclusive_count(cnt, lane, &total);
-    }
-    if (total == 0) return 0xFFFFFFFFu;
-
-    uint32_t overflowed = 0xFFFFFFFFu;
-    uint32_t fill = st->fill;
-    if (fill && (st->row != row || fill + total > STAGE_CAP)) {
-        overflowed = flush_stage(p, st);
-        fill = 0;
-    }
-    uint64_t* out;
-    unsigned pos, limit;
-    const bool to_stage = total <= STAGE_CAP;
-    if (to_stage) {                           // the usual case
-        out = st->rec; pos = fill + before; limit = STAGE_CAP;
-    } else {                                  // a tile full of survivors: straight to the buffer
-        unsigned base = 0;
-        if (lane == 0) base = atomicAdd(p.counts + (uint64_t)row * p.count_stride, total);
-        base = __shfl_sync(FULL_MASK, base, 0);
-        out = p.buf + (uint64_t)row * p.buf_stride; pos = base + before; limit = p.capacity;
-        if ((uint64_t)base + total > p.capacity) overflowed = row;
-    }
-    if constexpr (STRAIGHT) {
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-            if (mine_u[u]) {
-                const uint64_t q = qbase + (uint64_t)u * THREADS + threadIdx.x;
-                const int64_t i0 = (int64_t)(q * VEC) - (int64_t)mis;
-#pragma unroll
-                for (int l = 0; l < VEC; ++l) {
-                    if (mine_u[u] & (1u << l)) {
-                        if (pos < limit) out[pos] = make_record(Elem<T>::key(vec_elem(v[u], l)), (uint32_t)(i0 + l));
-                        ++pos;
-                    }
-                }
-            }
-        }
-    } else {
-        if (cnt) emit_survivors<T, THREADS, UNROLL>(v, mine, qbase, mis, out, pos, limit);
-    }
-    if (to_stage) {
-        __syncwarp();
-        if (lane == 0) { st->fill = fill + total; st->row = row; }
-        __syncwarp();
-        if (fill + total >= STAGE_FLUSH) {
-            const uint32_t o = flush_stage(p, st);
-            if (o != 0xFFFFFFFFu) overflowed = o;
-        }
-    }
-    return overflowed;
-}
-
-// The slow path without staging (sparse survivors): one global atomic per warp and tile, records
-// written straight to the row buffer.  Returns the row if its buffer has overflowed, else ~0.
+// The slow path: one global atomic per warp and tile, records written straight to the row buffer.  Returns the row if its buffer has overflowed, else ~0.
 template <typename T, int THREADS, int UNROLL, bool PARTS, bool HIST = false>
 __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T>& p, const typename Elem<T>::vec_t (&v)[UNROLL],
                                                             uint32_t inside_mask, uint32_t row, uint64_t qbase, uint32_t mis, T tau,
@@ -562,22 +430,17 @@ __device__ __noinline__ void defer_process_batch_counting(const FilterParams<T>&
     defer_process_batch<T, THREADS, UNROLL, PARTS, true>(p, vid, hist_coarse);
 }
 
-// STAGED = collect survivors in per-warp shared-memory stages (dense survivors, one row at a time);
-// otherwise append them directly (sparse survivors or many short rows).
-//
 // Work distribution: a tile is TILE_VECTORS consecutive vectors of one row (32 KB), loaded by the
 // whole CTA at once (every warp-level load is one contiguous 512-byte run, the CTA's loads one 32 KB
 // run).  A CTA takes tiles blockIdx.x, + gridDim.x, ... with its warps running freely; the last few
 // tiles of the launch (from dyn_start on) come from a global counter instead, so that SMs that saw
 // less bandwidth take fewer of them and all CTAs finish together.  The counter is read one tile
 // ahead, so its round trip hides behind the loads; only this tail needs a CTA barrier per tile.
-template <typename T, int THREADS, int UNROLL, bool STAGED, bool PARTS = false, bool DEFER = false, bool HIST = false>
-__global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGED : sizeof(T) == 4 ? PROFK_FILTER_MINBLOCKS_F32 : PROFK_FILTER_MINBLOCKS_BF16) filter_kernel(const __grid_constant__ FilterParams<T> p) {
-    static_assert(!(STAGED && DEFER), "one way of handling dense survivors at a time");
+template <typename T, int THREADS, int UNROLL, bool PARTS = false, bool DEFER = false, bool HIST = false>
+__global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOCKS_F32 : PROFK_FILTER_MINBLOCKS_BF16) filter_kernel(const __grid_constant__ FilterParams<T> p) {
     static_assert(!HIST || (DEFER && !PARTS), "only the deferring build counts its records");
     using V = typename Elem<T>::vec_t;
     constexpr uint32_t TILE_VECTORS = THREADS * UNROLL;
-    __shared__ WarpStage stages[STAGED ? THREADS / 32 : 1];
     __shared__ uint32_t hits[DEFER ? DEFER_CAP : 1];
     __shared__ uint32_t s_nhits;
     __shared__ uint32_t s_scan[DEFER ? THREADS / 32 + 1 : 1];
@@ -593,11 +456,6 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
     extern __shared__ __align__(128) unsigned char pf_smem[];        // p.prefetch_tiles tiles of 32 KB (or nothing)
 
     const unsigned lane = lane_id();
-    WarpStage* st = &stages[STAGED ? threadIdx.x >> 5 : 0];
-    if (STAGED) {
-        if (lane == 0) { st->fill = 0; st->row = 0; }
-        __syncwarp();
-    }
 
     constexpr int VEC = Elem<T>::VEC;
     constexpr uint32_t ALL_INSIDE = (1u << UNROLL) - 1u;
@@ -763,8 +621,7 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
                 }
             }
             if (!noted) {
-                if (STAGED) o = filter_slow_path<T, THREADS, UNROLL>(p, st, v[0], v[1], v[2], v[3], inside_mask, row, qbase, rv.mis, tau_lo);
-                else o = filter_slow_path_direct<T, THREADS, UNROLL, PARTS>(p, v, inside_mask, row, qbase, rv.mis, tau_lo);
+                o = filter_slow_path_direct<T, THREADS, UNROLL, PARTS>(p, v, inside_mask, row, qbase, rv.mis, tau_lo);
                 // (HIST) records appended on this way out of a full list are not counted: the kernel behind is told so
                 if (HIST && lane == 0) p.hist[BIN_COUNT + BIN_FLAG_UNCOUNTED] = 1u;
             }
@@ -787,7 +644,6 @@ __global__ void __launch_bounds__(THREADS, STAGED ? PROFK_FILTER_MINBLOCKS_STAGE
         decode_and_load(false);
         if (row != tau_row) { tau_row = row; load_threshold(); }
     }
-    if (STAGED && st->fill) flush_stage(p, st);
     if (DEFER) {
         // every tile of this CTA has been streamed: work the list off, one entry per thread
         __syncthreads();

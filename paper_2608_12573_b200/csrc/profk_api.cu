@@ -62,7 +62,6 @@ std::atomic<int> g_coop_pdl{-1};                 // -1 untried, 1 accepted, 0 re
 struct DeviceInfo {
     int sm_count = 0;
     int filter_blocks_per_sm[2] = {0, 0};     // by dtype
-    int filter_staged_blocks_per_sm[2] = {0, 0};
     int filter_defer_blocks_per_sm[2] = {0, 0};
     int max_cluster[2] = {8, 8};              // 16 when the device can co-schedule 16 CTAs of the threshold kernel
     int refine_cluster[2] = {8, 8};           // same for the refine kernel at its largest footprint
@@ -141,19 +140,16 @@ template <typename T> int ensure_device_info(int dev, DeviceInfo* out) {
     const int d = dtype_index<T>();
     if (di.filter_blocks_per_sm[d] == 0) {
         int nb = 0;
-        CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false>,
+        CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL>,
                                                                  FILTER_THREADS, 0));
         di.filter_blocks_per_sm[d] = std::max(nb, 1);
-        CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, true>,
-                                                                 FILTER_THREADS, 0));
-        di.filter_staged_blocks_per_sm[d] = std::max(nb, 1);
-        CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false, false, true>,
+        CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false, true>,
                                                                  FILTER_THREADS, 0));
         di.filter_defer_blocks_per_sm[d] = std::max(nb, 1);
         CUDA_TRY(cudaFuncSetAttribute(sample_select_kernel<T, SEL_THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
         const int prefetch_bytes = (int)(FILTER_PREFETCH * FILTER_THREADS * FILTER_UNROLL * 16u);
-        CUDA_TRY(cudaFuncSetAttribute(filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, prefetch_bytes));
-        CUDA_TRY(cudaFuncSetAttribute(filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, prefetch_bytes));
+        CUDA_TRY(cudaFuncSetAttribute(filter_kernel<T, FILTER_THREADS, FILTER_UNROLL>, cudaFuncAttributeMaxDynamicSharedMemorySize, prefetch_bytes));
+        CUDA_TRY(cudaFuncSetAttribute(filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, prefetch_bytes));
         // (the small build holds 33 KB of static shared memory: with 4096 keys it passes the 48 KB that need no opt-in)
         CUDA_TRY(cudaFuncSetAttribute(sample_select_kernel<T, SEL_SMALL_THREADS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * 1024));
         CUDA_TRY(cudaFuncSetAttribute(refine_kernel<T, 48>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)REFINE_SMEM_MAX));
@@ -281,7 +277,7 @@ int launch_sample_select(const DeviceInfo& di, const T* in, int64_t rows, int64_
 
 template <typename T>
 int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, const T* tau, int64_t capacity, uint64_t* buf,
-                  uint64_t buf_stride, uint32_t* counts, uint32_t count_stride, bool pdl, bool staged, uint32_t* tile_counter, bool parts,
+                  uint64_t buf_stride, uint32_t* counts, uint32_t count_stride, bool pdl, uint32_t* tile_counter, bool parts,
                   uint32_t part_cap, uint32_t* part_counts, const uint4* thr, cudaStream_t st, bool deferred = false, uint32_t* hist = nullptr) {
     FilterParams<T> fp;
     fp.hist = hist; fp.idx_bits = index_bits((uint64_t)N);
@@ -294,9 +290,9 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     fp.use_pdl = pdl ? 1 : 0;
     fp.tile_counter = tile_counter;
     fp.part_cap = part_cap; fp.part_counts = part_counts;
-    if (staged || parts || fp.total_tiles * (uint64_t)(FILTER_THREADS * FILTER_UNROLL) >= (1ull << 32)) deferred = false;   // vectors are numbered in 32 bits
+    if (parts || fp.total_tiles * (uint64_t)(FILTER_THREADS * FILTER_UNROLL) >= (1ull << 32)) deferred = false;   // vectors are numbered in 32 bits
     const uint64_t max_grid = (uint64_t)di.sm_count *
-        (staged ? di.filter_staged_blocks_per_sm[dtype_index<T>()] : deferred ? di.filter_defer_blocks_per_sm[dtype_index<T>()] : di.filter_blocks_per_sm[dtype_index<T>()]);
+        (deferred ? di.filter_defer_blocks_per_sm[dtype_index<T>()] : di.filter_blocks_per_sm[dtype_index<T>()]);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)std::min<uint64_t>(fp.total_tiles, max_grid));
     // all but the last ~PROFK_DYNAMIC_ROUNDS tiles per CTA follow the fixed stride
@@ -305,9 +301,8 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     if (rounds <= PROFK_DYNAMIC_ROUNDS) fp.tile_counter = nullptr;
     cfg.blockDim = dim3(FILTER_THREADS);
     // A single row scanned behind the threshold kernel: each CTA copies its next tiles into shared memory while it waits.
-    // (Not the staged build: its two CTAs per SM spill already, and the copies cost the 2^29 bf16 row 3 us.)
-    // (nor the build that defers its candidates: their list takes the shared memory)
-    const bool prefetch = pdl && !staged && !deferred && rows == 1 && fp.dyn_start >= (FILTER_PREFETCH + 1) * cfg.gridDim.x;
+    // (Not the build that defers its candidates: their list takes the shared memory.)
+    const bool prefetch = pdl && !deferred && rows == 1 && fp.dyn_start >= (FILTER_PREFETCH + 1) * cfg.gridDim.x;
     fp.prefetch_tiles = prefetch ? FILTER_PREFETCH : 0u;
     fp.prefetch_spin_limit = g_prefetch_spin_limit.load();
     cfg.dynamicSmemBytes = prefetch ? FILTER_PREFETCH * FILTER_THREADS * FILTER_UNROLL * 16u : 0;
@@ -317,11 +312,10 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
     if (hist && (rows != 1 || !deferred)) return PROFK_EINVAL;      // (no caller asks for that)
-    if (hist) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false, false, true, true>, fp));
-    else if (staged) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, true>, fp));
-    else if (deferred) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false, false, true>, fp));
-    else if (parts) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false, true>, fp));
-    else CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false>, fp));
+    if (hist) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false, true, true>, fp));
+    else if (deferred) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, false, true>, fp));
+    else if (parts) CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL, true>, fp));
+    else CUDA_TRY(cudaLaunchKernelEx(&cfg, filter_kernel<T, FILTER_THREADS, FILTER_UNROLL>, fp));
     ++g_launches;
     return PROFK_OK;
 }
@@ -456,8 +450,9 @@ int launch_refine(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, Ro
 // warp-tile on, most tiles would run the slow path and the scan becomes instruction-bound; the build that only notes its
 // candidates in shared memory and decides them after streaming (DEFER, filter.cuh) then wins for bf16 (twice the
 // elements per warp-tile): 512 rows of 2^20, k = 32 (1.46 per warp-tile) 298 -> 260 us; the paper's SAE shape (3.2)
-// 112 -> 97, where it also replaces the staged build.  fp32: the SAE shape (1.6) 93.4 -> 89.3; batches of fp32 rows
-// (0.73) lose 6 % (397 -> 422 us) and stay on the direct build; 2^29 bf16, K = 131072 (0.4) is indifferent.
+// 112 -> 97.  fp32: the SAE shape (1.6) 93.4 -> 89.3; batches of fp32 rows (0.73) lose 6 % (397 -> 422 us) and stay on
+// the direct build.  (An earlier build that staged survivors per warp in shared memory has gone: this one beat it
+// wherever it was chosen.)
 // A large selection from a single row (and the BatchTopK entry points) gains more: the deferring build also hands the
 // kernel behind it a finished histogram (HIST, filter.cuh) and needs no partitioned append; from 0.1 survivors per
 // warp-tile on it wins (2^29 bf16, K = 131072 at 0.41: 218 -> 212 us; 2^26 fp32, k = 32768 at 0.36: 89 -> 81; 2^28 bf16,
@@ -514,19 +509,15 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     uint32_t* keys_scratch = reinterpret_cast<uint32_t*>(base + lay.off_keys);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-    // Survivors are staged per warp when a warp's tile is expected to hold a good fraction of one
-    // (expected survivors per element ~ r / m); sparse survivors are appended directly.
+    // Survivors expected per warp-tile (expected survivors per element ~ r / m) decide the build of the filter: sparse
+    // survivors are appended directly, dense ones noted and decided after streaming.
     const double per_warp_tile = (double)plan->r / (double)std::max<int64_t>(plan->m, 1) * 32.0 * FILTER_UNROLL * Elem<T>::VEC;
-        // (The direct append has three CTAs per SM, eight counters for large selections and the prefetch behind the threshold
-    // kernel; it holds up to about two survivors per warp-tile: 2^29 bf16, K = 131072 at 0.4: 248 -> 237 us; 50 M fp32,
-    // K = 131072 at 1.6: 124 -> 114; 50 M bf16 at 3.2 stays staged, 120 against 127.)
     const bool deferred = plan->mode == 0 && defer_candidates<T>(rows, per_warp_tile, large && rows == 1);
-    const bool staged = plan->mode == 0 && !deferred && rows == 1 && per_warp_tile > 2.0;
 
     // Large selections keep so many survivors that a row's single append counter would hold the scan up:
     // the direct variant then appends to FILTER_PARTS parts of the buffer, each with a counter of its own.
     // (The deferring build appends once per 32 candidates, after streaming: one counter is enough for it.)
-    const bool parts = large && !staged && !deferred && plan->mode == 0;
+    const bool parts = large && !deferred && plan->mode == 0;
     const uint32_t part_cap = (uint32_t)(row_stride / 2 / FILTER_PARTS);
     uint32_t* part_counts = reinterpret_cast<uint32_t*>(base + lay.off_parts);
 
@@ -577,7 +568,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
                                      rows <= GATHER_MAX_ROWS ? keys_scratch : nullptr, parts ? part_counts : nullptr, plan->tie_rule == PROFK_TIES_BY_INDEX, thr, st,
                                      nullptr, keep_keys ? keys_scratch : nullptr, hist ? bins : nullptr, BIN_ROW_WORDS);
         if (rc != PROFK_OK) return rc;
-        rc = launch_filter<T>(di, in, rows, N, nullptr, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, &header->tile_counter,
+        rc = launch_filter<T>(di, in, rows, N, nullptr, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, &header->tile_counter,
                               parts, part_cap, part_counts, thr, st, deferred, hist ? bins : nullptr);
         if (rc != PROFK_OK) return rc;
 
@@ -697,8 +688,7 @@ int batchtopk_planned(const T* in, int64_t N, int64_t K, const profk_plan_t* pla
 
     const double per_warp_tile = (double)plan->r / (double)std::max<int64_t>(plan->m, 1) * 32.0 * FILTER_UNROLL * Elem<T>::VEC;
     const bool deferred = plan->mode == 0 && defer_candidates<T>(1, per_warp_tile, true);       // as in topk_planned for a large selection
-    const bool staged = plan->mode == 0 && !deferred && per_warp_tile > 2.0;
-    const bool parts = !staged && !deferred && plan->mode == 0;
+    const bool parts = !deferred && plan->mode == 0;
     const uint32_t part_cap = (uint32_t)(row_stride / 2 / FILTER_PARTS);
     const bool hist = deferred;
 
@@ -708,7 +698,7 @@ int batchtopk_planned(const T* in, int64_t N, int64_t K, const profk_plan_t* pla
                                      parts ? part_counts : nullptr, plan->tie_rule == PROFK_TIES_BY_INDEX, thr, st, nullptr,
                                      (plan->r_tight > 0 || plan->r_loose > 0) ? keys_scratch : nullptr, hist ? bins : nullptr, BIN_ROW_WORDS);
         if (rc != PROFK_OK) return rc;
-        rc = launch_filter<T>(di, in, 1, N, nullptr, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, staged, &header->tile_counter,
+        rc = launch_filter<T>(di, in, 1, N, nullptr, capacity, buf, row_stride, &ctl[0].count, sizeof(RowCtl) / 4, true, &header->tile_counter,
                               parts, part_cap, part_counts, thr, st, deferred, hist ? bins : nullptr);
         if (rc != PROFK_OK) return rc;
     } else {
@@ -772,7 +762,7 @@ int filter_only(const T* in, int64_t rows, int64_t N, const T* tau, int64_t capa
     // The same build of the kernel a whole call would pick for this density of survivors, estimated from the capacity
     // (a plan's capacity is about twice the survivors it expects).
     const double per_warp_tile = 0.5 * (double)capacity / (double)N * 32.0 * FILTER_UNROLL * Elem<T>::VEC;
-    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, (uint64_t)capacity, counts, PROFK_FILTER_COUNT_STRIDE, false, false, nullptr, false,
+    return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, (uint64_t)capacity, counts, PROFK_FILTER_COUNT_STRIDE, false, nullptr, false,
                             0u, nullptr, nullptr, static_cast<cudaStream_t>(stream), defer_candidates<T>(rows, per_warp_tile));
 }
 
@@ -844,7 +834,7 @@ int filter_shard(const T* shard, int64_t shard_base, int64_t shard_len, const ui
     localize_threshold_kernel<<<1, 32, 0, st>>>(reinterpret_cast<const uint4*>(thr_record), (unsigned long long)shard_base,
                                                 (unsigned long long)shard_len, state);
     CUDA_TRY(cudaGetLastError());
-    return launch_filter<T>(di, shard, 1, shard_len, nullptr, capacity, records, (uint64_t)capacity, state, 1, false, false, nullptr, false, 0u,
+    return launch_filter<T>(di, shard, 1, shard_len, nullptr, capacity, records, (uint64_t)capacity, state, 1, false, nullptr, false, 0u,
                             nullptr, reinterpret_cast<const uint4*>(state + 4), st);
 }
 
