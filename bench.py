@@ -309,8 +309,8 @@ def measure_extra_config(profk, torch, name, dev, peak):
         res["batchtopk_note"] = ("outputs are allocated through torch inside the timed loop (caching allocator); the dense form also "
                                  "writes N elements of zeros")
     if k > 8192 and rows <= 4:
-        res["filter_note"] = ("the stand-alone filter launch appends to one counter per row; inside the call a selection this large "
-                              "appends to eight (or stages per warp), so the call's own filter pass is faster than this figure")
+        res["filter_note"] = ("the stand-alone filter launch takes the build of the kernel that the call takes at this density of survivors, "
+                              "without the histogram the call's own launch also makes for the kernel behind it")
     del inputs, out
     torch.cuda.empty_cache()
     return res

@@ -282,8 +282,9 @@ int profk_batchtopk_planned_bf16(const void* in, int64_t N, int64_t K, const pro
  * index ascending".  Records are
  * appended in no particular order.  Needs no workspace.  The launch takes the build of the kernel a whole call would
  * take for the density of survivors that `capacity` suggests (a plan's capacity is about twice the survivors it
- * expects): from about one survivor per warp-tile on, bf16 rows use the build that notes candidates in shared memory
- * while streaming and decides them afterwards.
+ * expects): from about one survivor per warp-tile on (a tenth of one for a single row with a capacity beyond 32768
+ * records, as for a large selection), the build that notes candidates in shared memory while streaming and decides
+ * them afterwards.
  */
 #define PROFK_FILTER_COUNT_STRIDE 8
 int profk_filter_f32(const float* in, int64_t rows, int64_t N, const float* tau, int64_t capacity,

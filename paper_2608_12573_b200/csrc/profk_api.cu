@@ -761,9 +761,10 @@ int filter_only(const T* in, int64_t rows, int64_t N, const T* tau, int64_t capa
     if (rc != PROFK_OK) return rc;
     // The same build of the kernel a whole call would pick for this density of survivors, estimated from the capacity
     // (a plan's capacity is about twice the survivors it expects).
+    // (a single row whose capacity is beyond what one CTA refines: a whole call would treat it as a large selection)
     const double per_warp_tile = 0.5 * (double)capacity / (double)N * 32.0 * FILTER_UNROLL * Elem<T>::VEC;
     return launch_filter<T>(di, in, rows, N, tau, capacity, buf_keys, (uint64_t)capacity, counts, PROFK_FILTER_COUNT_STRIDE, false, nullptr, false,
-                            0u, nullptr, nullptr, static_cast<cudaStream_t>(stream), defer_candidates<T>(rows, per_warp_tile));
+                            0u, nullptr, nullptr, static_cast<cudaStream_t>(stream), defer_candidates<T>(rows, per_warp_tile, rows == 1 && capacity > 32768));
 }
 
 template <typename T>
