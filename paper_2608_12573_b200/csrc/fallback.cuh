@@ -184,7 +184,9 @@ __device__ __noinline__ int grid_second_chance_row(const FallbackParams<T>& p, u
     if (rung == 0) return 0;
     const unsigned tid = threadIdx.x;
     uint32_t key2, j2;
-    kth_sample_record<T>(sm.keys + row * sm.S, sm.S, rung, sh, &key2, &j2);       // every CTA for itself
+    // (every CTA for itself; a tighter rank lies among the keys at or above the first pass's threshold)
+    kth_sample_record<T>(sm.keys + row * sm.S, sm.S, rung, sh, &key2, &j2,
+                         status == ROW_OVERFLOW ? Elem<T>::key(Elem<T>::from_bits(__ldcg(&p.ctl[row].tau_bits))) : 0u);
     const uint32_t idx2 = sm.by_record ? sample_element_index(j2, row, sm.seed, sm.q, sm.rem, sm.S, sm.inv_s) : 0xFFFFFFFFu;
     const T tau2 = Elem<T>::from_key(key2);
     if (tid == 0) {

@@ -87,178 +87,14 @@ __device__ __forceinline__ void finish_from_segments(const uint64_t* recs, uint3
     sort_and_write<T>(sortbuf, k, k, k, row, out_vals, out_idx);
 }
 
-// The exact top-k of the full row, for a row that failed the count check (Section 3, "Refinement").
-// Cluster `seg` of the row's clusters selects the k smallest records (and a few more) of its segment of
-// the row; the cluster that finishes last merges: the k smallest of all segments' records, ordered, are
-// the row's output.  The ticket is the row's `collect` word, zero on entry and zero again on exit.
-// The second chance (second_chance.cuh) of a row that failed the count check, run by all clusters of the row, each over
-// its own segment: the threshold of the plan's tighter (after an overflow) or looser (after too few candidates) sample
-// rank is selected from the kept keys -- by every CTA for itself, nobody waits for anybody -- the segment is filtered with
-// it into the row's buffer (counter: the row's `pad` word), and the cluster that finishes last takes the check
-// k <= R' <= M on the new count.  Returns, the same in every CTA of a cluster: 0 = not the last cluster, or the last one
-// and the row is answered (by its first CTA, from the buffer); 2 = the last cluster and the check failed again.
-template <typename T>
-__device__ __noinline__ int second_chance_row(const RefineParams<T>& p, uint64_t row, unsigned seg, unsigned crank, uint32_t rung,
-                                              uint32_t failed_status, uint64_t* sortbuf, SelectShared& sh) {
-    namespace cg = cooperative_groups;
-    cg::cluster_group cluster = cg::this_cluster();
-    const unsigned tid = threadIdx.x, nthr = blockDim.x;
-    const unsigned csize = p.cluster_size, nseg = p.clusters_per_row;
-    const SampleInfo& sm = p.sample;
-    uint32_t key2, j2;
-    kth_sample_record<T>(sm.keys + row * sm.S, sm.S, rung, sh, &key2, &j2);
-    const uint32_t idx2 = sm.by_record ? sample_element_index(j2, row, sm.seed, sm.q, sm.rem, sm.S, sm.inv_s) : 0xFFFFFFFFu;
-    const T tau2 = Elem<T>::from_key(key2);
-    if (tid == 0) {                              // (every CTA of the row writes the same sixteen bytes)
-        const uint32_t top = Elem<T>::KEY_BITS == 32 ? 0xFFFFFFFFu : 0xFFFFu;
-        p.thr2[row] = make_uint4(Elem<T>::bits(tau2), Elem<T>::bits(Elem<T>::from_key(key2 == top ? key2 : key2 + 1u)), idx2, 0u);
-    }
-    __syncthreads();
-
-    FilterParams<T> fp = {};
-    fp.in = p.in; fp.N = p.N; fp.rows = row + 1; fp.tau = nullptr; fp.capacity = p.capacity;
-    fp.buf = p.buf; fp.buf_stride = p.buf_stride;
-    fp.counts = &p.ctl[0].pad; fp.count_stride = sizeof(RowCtl) / 4;
-    fp.thr = p.thr2;
-    const uint64_t tiles = tiles_per_row<T>(p.N, nthr * XS_UNROLL);
-    const uint64_t seg_lo = tiles * seg / nseg, seg_hi = tiles * (seg + 1) / nseg;
-    if (nthr == 512) refilter_tiles<T, 512>(fp, (uint32_t)row, seg_lo, seg_hi, crank, csize, tau2);
-    else refilter_tiles<T, 1024>(fp, (uint32_t)row, seg_lo, seg_hi, crank, csize, tau2);
-    __threadfence();
-    cluster.sync();                              // the whole cluster's records and counts are out
-
-    // the last cluster to get here sees all of them
-    if (crank == 0 && tid == 0) {
-        const uint32_t ticket = atomicAdd(&p.ctl[row].collect, 1u);
-        uint32_t decision = 0;
-        if (ticket == nseg - 1) {
-            p.ctl[row].collect = 0;
-            __threadfence();
-            const uint32_t R2 = __ldcg(&p.ctl[row].pad);
-            decision = (R2 >= p.k && R2 <= p.capacity) ? 1u : 2u;
-            if (decision == 1u) {
-                p.ctl[row].status = failed_status == ROW_OVERFLOW ? ROW_OVERFLOW_REFILTERED : ROW_RECALL_REFILTERED;
-                p.ctl[row].count = R2;
-                p.ctl[row].tau_bits = Elem<T>::bits(tau2);
-                p.ctl[row].tau_idx = idx2;
-            }
-        }
-        sh.crowded = decision;
-    }
-    cluster.sync();
-    const uint32_t decision = *cluster.map_shared_rank(&sh.crowded, 0);
-    cluster.sync();                              // the first CTA's word has been read by all: it may go on
-    if (decision == 1u && crank == 0) {
-        const uint32_t R2 = __ldcg(&p.ctl[row].count);
-        finish_from_segments<T>(p.buf + row * p.buf_stride, R2, p.k, p.sort_cap, sortbuf, sh, row, p.out_vals, p.out_idx);
-    }
-    return decision == 2u ? 2 : 0;
-}
-
-// The exact top-k of the full row, for a row that failed the count check (Section 3, "Refinement").
-// Cluster `seg` of the row's clusters selects the k smallest records (and a few more) of its segment of
-// the row; the cluster that finishes last merges: the k smallest of all segments' records, ordered, are
-// the row's output.  The ticket is the row's `collect` word, zero on entry and zero again on exit.
-// When the plan names a second-chance rank for this kind of failure and the sample was kept, that comes first; the
-// exact selection then runs only if the second pass fails too, by the one cluster that found out, over the whole row.
-template <typename T>
-__device__ __noinline__ void exact_row(const RefineParams<T>& p, uint64_t row, unsigned seg, unsigned crank, uint64_t* sortbuf,
-                                       SelectShared& sh, uint32_t status, uint32_t tau_key) {
-    const unsigned tid = threadIdx.x, nthr = blockDim.x;
-    const unsigned csize = p.cluster_size, nseg = p.clusters_per_row;
-    const bool overflowed = status == ROW_OVERFLOW;
-    const uint64_t tiles = tiles_per_row<T>(p.N, nthr * XS_UNROLL);
-    const uint32_t slots = p.k + XS_EDGE;                // per segment: a superset of its k smallest records
-    const uint32_t rung = status == ROW_OVERFLOW ? p.sample.r_tight : status == ROW_RECALL ? p.sample.r_loose : 0u;
-    if (rung != 0 && p.sample.keys != nullptr && csize > 1 && (nthr == 512 || nthr == 1024)) {
-        if (second_chance_row<T>(p, row, seg, crank, rung, status, sortbuf, sh) != 2) return;
-        // failed again: this cluster alone selects from the whole row, into its own scratch
-        const uint64_t* mine = p.xs_records + (row * nseg + seg) * (uint64_t)slots;
-        exact_select_cluster<T>(p.in, p.N, row, p.k, 0, tiles, p.xs_records + (row * nseg + seg) * (uint64_t)slots,
-                                p.xs_counters + row * nseg + seg, sh, csize, crank, false, 0u);
-        if (crank != 0) return;
-        finish_from_segments<T>(mine, slots, p.k, p.sort_cap, sortbuf, sh, row, p.out_vals, p.out_idx);
-        return;
-    }
-    const uint64_t seg_lo = tiles * seg / nseg, seg_hi = tiles * (seg + 1) / nseg;
-    const uint64_t* recs = p.xs_records + (row * nseg) * (uint64_t)slots;
-    exact_select_cluster<T>(p.in, p.N, row, p.k, seg_lo, seg_hi, p.xs_records + (row * nseg + seg) * (uint64_t)slots,
-                            p.xs_counters + row * nseg + seg, sh, csize, crank, overflowed, tau_key);
-    if (crank != 0) return;
-
-    // every thread of this cluster has fenced its records; the last cluster to get here sees them all
-    if (tid == 0) {
-        const uint32_t ticket = atomicAdd(&p.ctl[row].collect, 1u);
-        const bool last = ticket == nseg - 1;
-        if (last) { p.ctl[row].collect = 0; __threadfence(); }
-        sh.cnt = last ? 1u : 0u;
-    }
-    __syncthreads();
-    if (sh.cnt == 0) return;
-    __syncthreads();                         // sh.cnt is rewritten by the select below
-
-    finish_from_segments<T>(recs, nseg * slots, p.k, p.sort_cap, sortbuf, sh, row, p.out_vals, p.out_idx);
-}
-
-// Two builds of the kernel.  With up to 512 threads a refine CTA has to start beside the last CTAs
-// of the filter kernel on an SM, and 48 registers per thread is what fits there; the (rare) exact
-// selection then runs with spills.  A CTA of 1024 threads does not fit there anyway and gets the
-// registers the exact selection wants.
-template <typename T, int MAXREG>
-__global__ void __maxnreg__(MAXREG) refine_kernel(const __grid_constant__ RefineParams<T> p) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    uint64_t* sortbuf = reinterpret_cast<uint64_t*>(smem_raw);                 // sort_cap + RF_EDGE_CAP records
-    uint64_t* staged = sortbuf + p.sort_cap + RF_EDGE_CAP;                     // stage_cap records
-    __shared__ SelectShared sh;
-
-    // CTAs of a row are consecutive: clusters_per_row clusters (along x) of cluster_size CTAs.
-    const unsigned csize = p.cluster_size, nseg = p.clusters_per_row;
-    const unsigned cta_in_row = blockIdx.x % (csize * nseg);
-    const unsigned seg = cta_in_row / csize, crank = cta_in_row % csize;
-    const bool refiner = cta_in_row == 0;            // the CTA that refines the row's buffer
+// Stage 4 proper: the k best of the R = ctl.count candidate records of `row`, in order, written to the output.  One CTA;
+// sh.hist zero, sh.or_bits = sh.fill = sh.n_edge = sh.crowded = 0 on entry.  PRELOADED: r[] holds the first batch of
+// records already (8 per thread, requested before the survivor count was known; slots beyond the capacity all ones).
+template <typename T, bool PRELOADED>
+__device__ __forceinline__ void refine_row(const RefineParams<T>& p, uint64_t row, const RowCtl& ctl, uint64_t (&r)[8], uint64_t* sortbuf,
+                                           uint64_t* staged, SelectShared& sh) {
     const unsigned tid = threadIdx.x, nthr = blockDim.x, lane = lane_id();
-    const uint64_t row = blockIdx.x / (csize * nseg);
-    if (refiner) {
-        if (tid == 0) { sh.or_bits = 0ull; sh.fill = 0; sh.n_edge = 0; sh.crowded = 0; }
-        for (uint32_t i = tid; i < RF_BINS; i += nthr) sh.hist[i] = 0;
-        __syncthreads();
-    }
-    pdl_launch_dependents();
-    if (p.use_pdl) pdl_wait();
-
-    // The first batch of records (8 per thread, kept in registers) is requested at once, together with
-    // the row's control block: which of them are real is known when the survivor count arrives.
     const uint64_t* src = p.buf + row * p.buf_stride;
-    uint64_t r[8];
-    if (refiner && !p.direct) {
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const uint32_t i = u * nthr + tid;
-            r[u] = i < p.capacity ? src[i] : ~0ull;
-        }
-    }
-
-    // ---- the count check of stage 4 ----
-    RowCtl ctl;
-    uint32_t status;
-    if (p.direct) {                          // the row's control block was set up by the initialisation kernel
-        ctl.tau_bits = 0; ctl.count = 0;
-        status = ROW_DIRECT;
-    } else {
-        ctl = p.ctl[row];
-        status = ctl.count > p.capacity ? ROW_OVERFLOW : ctl.count < p.k_accept ? ROW_RECALL : ROW_OK;
-        if (refiner && tid == 0) {
-            p.ctl[row].status = status;
-            p.ctl[row].n_final = status ? p.k : ctl.count;
-            if (status) atomicAdd(&p.header->n_failed, 1u);
-        }
-    }
-    if (status != ROW_OK) {
-        if (csize == 1) return;              // the exact-selection kernel that follows takes this row
-        exact_row<T>(p, row, seg, crank, sortbuf, sh, status, Elem<T>::key(Elem<T>::from_bits(ctl.tau_bits)));
-        return;
-    }
-    if (!refiner) return;
     const uint32_t R = ctl.count;
 
     const uint32_t n = R;
@@ -291,7 +127,7 @@ __global__ void __maxnreg__(MAXREG) refine_kernel(const __grid_constant__ Refine
     };
 
     for (uint32_t b = 0; b < nbatch; ++b) {
-        if (b > 0) load_batch(b);
+        if (b > 0 || !PRELOADED) load_batch(b);
 #pragma unroll
         for (int u = 0; u < 8; ++u)
             if (valid(b, u)) atomicAdd(&sh.hist[bin_of(r[u])], 1u);
@@ -401,6 +237,190 @@ __global__ void __maxnreg__(MAXREG) refine_kernel(const __grid_constant__ Refine
         m = kk;
     }
     sort_and_write<T>(sortbuf, m, kk, p.k, row, p.out_vals, p.out_idx);
+}
+
+// The same out of line, for the one CTA that refines a row after a second filtering pass (second_chance_row): the refine
+// kernel's own path keeps its registers.
+template <typename T>
+__device__ __noinline__ void refine_row_again(const RefineParams<T>& p, uint64_t row, uint64_t* sortbuf, uint64_t* staged, SelectShared& sh) {
+    const unsigned tid = threadIdx.x, nthr = blockDim.x;
+    __syncthreads();
+    if (tid == 0) { sh.or_bits = 0ull; sh.fill = 0; sh.n_edge = 0; sh.crowded = 0; }
+    for (uint32_t i = tid; i < RF_BINS; i += nthr) sh.hist[i] = 0;
+    __syncthreads();
+    const RowCtl ctl = p.ctl[row];               // the count and the threshold of the second pass (this CTA wrote them)
+    uint64_t r[8];
+    refine_row<T, false>(p, row, ctl, r, sortbuf, staged, sh);
+}
+
+// The second chance (second_chance.cuh) of a row that failed the count check, run by all clusters of the row, each over
+// its own segment: the threshold of the plan's tighter (after an overflow) or looser (after too few candidates) sample
+// rank is selected from the kept keys -- by every CTA for itself, nobody waits for anybody -- the segment is filtered with
+// it into the row's buffer (counter: the row's `pad` word), and the cluster that finishes last takes the check
+// k <= R' <= M on the new count.  Returns, the same in every CTA of a cluster: 0 = not the last cluster, or the last one
+// and the row is answered (its first CTA refines it from the buffer like any row); 2 = the last cluster and the check
+// failed again.
+template <typename T>
+__device__ __noinline__ int second_chance_row(const RefineParams<T>& p, uint64_t row, unsigned seg, unsigned crank, uint32_t rung,
+                                              uint32_t failed_status, uint64_t* sortbuf, SelectShared& sh, uint32_t tau_key) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned tid = threadIdx.x, nthr = blockDim.x;
+    const unsigned csize = p.cluster_size, nseg = p.clusters_per_row;
+    const SampleInfo& sm = p.sample;
+    uint32_t key2, j2;
+    // (a tighter rank lies among the keys at or above the first pass's threshold)
+    kth_sample_record<T>(sm.keys + row * sm.S, sm.S, rung, sh, &key2, &j2, failed_status == ROW_OVERFLOW ? tau_key : 0u);
+    const uint32_t idx2 = sm.by_record ? sample_element_index(j2, row, sm.seed, sm.q, sm.rem, sm.S, sm.inv_s) : 0xFFFFFFFFu;
+    const T tau2 = Elem<T>::from_key(key2);
+    if (tid == 0) {                              // (every CTA of the row writes the same sixteen bytes)
+        const uint32_t top = Elem<T>::KEY_BITS == 32 ? 0xFFFFFFFFu : 0xFFFFu;
+        p.thr2[row] = make_uint4(Elem<T>::bits(tau2), Elem<T>::bits(Elem<T>::from_key(key2 == top ? key2 : key2 + 1u)), idx2, 0u);
+    }
+    __syncthreads();
+
+    FilterParams<T> fp = {};
+    fp.in = p.in; fp.N = p.N; fp.rows = row + 1; fp.tau = nullptr; fp.capacity = p.capacity;
+    fp.buf = p.buf; fp.buf_stride = p.buf_stride;
+    fp.counts = &p.ctl[0].pad; fp.count_stride = sizeof(RowCtl) / 4;
+    fp.thr = p.thr2;
+    const uint64_t tiles = tiles_per_row<T>(p.N, nthr * XS_UNROLL);
+    const uint64_t seg_lo = tiles * seg / nseg, seg_hi = tiles * (seg + 1) / nseg;
+    if (nthr == 512) refilter_tiles<T, 512>(fp, (uint32_t)row, seg_lo, seg_hi, crank, csize, tau2);
+    else refilter_tiles<T, 1024>(fp, (uint32_t)row, seg_lo, seg_hi, crank, csize, tau2);
+    __threadfence();
+    cluster.sync();                              // the whole cluster's records and counts are out
+
+    // the last cluster to get here sees all of them
+    if (crank == 0 && tid == 0) {
+        const uint32_t ticket = atomicAdd(&p.ctl[row].collect, 1u);
+        uint32_t decision = 0;
+        if (ticket == nseg - 1) {
+            p.ctl[row].collect = 0;
+            __threadfence();
+            const uint32_t R2 = __ldcg(&p.ctl[row].pad);
+            decision = (R2 >= p.k && R2 <= p.capacity) ? 1u : 2u;
+            if (decision == 1u) {
+                p.ctl[row].status = failed_status == ROW_OVERFLOW ? ROW_OVERFLOW_REFILTERED : ROW_RECALL_REFILTERED;
+                p.ctl[row].count = R2;
+                p.ctl[row].tau_bits = Elem<T>::bits(tau2);
+                p.ctl[row].tau_idx = idx2;
+            }
+        }
+        sh.crowded = decision;
+    }
+    cluster.sync();
+    const uint32_t decision = *cluster.map_shared_rank(&sh.crowded, 0);
+    cluster.sync();                              // the first CTA's word has been read by all: it may go on
+    if (decision == 1u && crank == 0) refine_row_again<T>(p, row, sortbuf, sortbuf + p.sort_cap + RF_EDGE_CAP, sh);
+    return decision == 2u ? 2 : 0;
+}
+
+// The exact top-k of the full row, for a row that failed the count check (Section 3, "Refinement").
+// Cluster `seg` of the row's clusters selects the k smallest records (and a few more) of its segment of
+// the row; the cluster that finishes last merges: the k smallest of all segments' records, ordered, are
+// the row's output.  The ticket is the row's `collect` word, zero on entry and zero again on exit.
+// When the plan names a second-chance rank for this kind of failure and the sample was kept, that comes first; the
+// exact selection then runs only if the second pass fails too, by the one cluster that found out, over the whole row.
+template <typename T>
+__device__ __noinline__ void exact_row(const RefineParams<T>& p, uint64_t row, unsigned seg, unsigned crank, uint64_t* sortbuf,
+                                       SelectShared& sh, uint32_t status, uint32_t tau_key) {
+    const unsigned tid = threadIdx.x, nthr = blockDim.x;
+    const unsigned csize = p.cluster_size, nseg = p.clusters_per_row;
+    const bool overflowed = status == ROW_OVERFLOW;
+    const uint64_t tiles = tiles_per_row<T>(p.N, nthr * XS_UNROLL);
+    const uint32_t slots = p.k + XS_EDGE;                // per segment: a superset of its k smallest records
+    const uint32_t rung = status == ROW_OVERFLOW ? p.sample.r_tight : status == ROW_RECALL ? p.sample.r_loose : 0u;
+    if (rung != 0 && p.sample.keys != nullptr && csize > 1 && (nthr == 512 || nthr == 1024)) {
+        if (second_chance_row<T>(p, row, seg, crank, rung, status, sortbuf, sh, tau_key) != 2) return;
+        // failed again: this cluster alone selects from the whole row, into its own scratch
+        const uint64_t* mine = p.xs_records + (row * nseg + seg) * (uint64_t)slots;
+        exact_select_cluster<T>(p.in, p.N, row, p.k, 0, tiles, p.xs_records + (row * nseg + seg) * (uint64_t)slots,
+                                p.xs_counters + row * nseg + seg, sh, csize, crank, false, 0u);
+        if (crank != 0) return;
+        finish_from_segments<T>(mine, slots, p.k, p.sort_cap, sortbuf, sh, row, p.out_vals, p.out_idx);
+        return;
+    }
+    const uint64_t seg_lo = tiles * seg / nseg, seg_hi = tiles * (seg + 1) / nseg;
+    const uint64_t* recs = p.xs_records + (row * nseg) * (uint64_t)slots;
+    exact_select_cluster<T>(p.in, p.N, row, p.k, seg_lo, seg_hi, p.xs_records + (row * nseg + seg) * (uint64_t)slots,
+                            p.xs_counters + row * nseg + seg, sh, csize, crank, overflowed, tau_key);
+    if (crank != 0) return;
+
+    // every thread of this cluster has fenced its records; the last cluster to get here sees them all
+    if (tid == 0) {
+        const uint32_t ticket = atomicAdd(&p.ctl[row].collect, 1u);
+        const bool last = ticket == nseg - 1;
+        if (last) { p.ctl[row].collect = 0; __threadfence(); }
+        sh.cnt = last ? 1u : 0u;
+    }
+    __syncthreads();
+    if (sh.cnt == 0) return;
+    __syncthreads();                         // sh.cnt is rewritten by the select below
+
+    finish_from_segments<T>(recs, nseg * slots, p.k, p.sort_cap, sortbuf, sh, row, p.out_vals, p.out_idx);
+}
+
+// Two builds of the kernel.  With up to 512 threads a refine CTA has to start beside the last CTAs
+// of the filter kernel on an SM, and 48 registers per thread is what fits there; the (rare) exact
+// selection then runs with spills.  A CTA of 1024 threads does not fit there anyway and gets the
+// registers the exact selection wants.
+template <typename T, int MAXREG>
+__global__ void __maxnreg__(MAXREG) refine_kernel(const __grid_constant__ RefineParams<T> p) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint64_t* sortbuf = reinterpret_cast<uint64_t*>(smem_raw);                 // sort_cap + RF_EDGE_CAP records
+    uint64_t* staged = sortbuf + p.sort_cap + RF_EDGE_CAP;                     // stage_cap records
+    __shared__ SelectShared sh;
+
+    // CTAs of a row are consecutive: clusters_per_row clusters (along x) of cluster_size CTAs.
+    const unsigned csize = p.cluster_size, nseg = p.clusters_per_row;
+    const unsigned cta_in_row = blockIdx.x % (csize * nseg);
+    const unsigned seg = cta_in_row / csize, crank = cta_in_row % csize;
+    const bool refiner = cta_in_row == 0;            // the CTA that refines the row's buffer
+    const unsigned tid = threadIdx.x, nthr = blockDim.x, lane = lane_id();
+    const uint64_t row = blockIdx.x / (csize * nseg);
+    if (refiner) {
+        if (tid == 0) { sh.or_bits = 0ull; sh.fill = 0; sh.n_edge = 0; sh.crowded = 0; }
+        for (uint32_t i = tid; i < RF_BINS; i += nthr) sh.hist[i] = 0;
+        __syncthreads();
+    }
+    pdl_launch_dependents();
+    if (p.use_pdl) pdl_wait();
+
+    // The first batch of records (8 per thread, kept in registers) is requested at once, together with
+    // the row's control block: which of them are real is known when the survivor count arrives.
+    const uint64_t* src = p.buf + row * p.buf_stride;
+    uint64_t r[8];
+    if (refiner && !p.direct) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t i = u * nthr + tid;
+            r[u] = i < p.capacity ? src[i] : ~0ull;
+        }
+    }
+
+    // ---- the count check of stage 4 ----
+    RowCtl ctl;
+    uint32_t status;
+    if (p.direct) {                          // the row's control block was set up by the initialisation kernel
+        ctl.tau_bits = 0; ctl.count = 0;
+        status = ROW_DIRECT;
+    } else {
+        ctl = p.ctl[row];
+        status = ctl.count > p.capacity ? ROW_OVERFLOW : ctl.count < p.k_accept ? ROW_RECALL : ROW_OK;
+        if (refiner && tid == 0) {
+            p.ctl[row].status = status;
+            p.ctl[row].n_final = status ? p.k : ctl.count;
+            if (status) atomicAdd(&p.header->n_failed, 1u);
+        }
+    }
+    if (status != ROW_OK) {
+        if (csize == 1) return;              // the exact-selection kernel that follows takes this row
+        exact_row<T>(p, row, seg, crank, sortbuf, sh, status, Elem<T>::key(Elem<T>::from_bits(ctl.tau_bits)));
+        return;
+    }
+    if (!refiner) return;
+    refine_row<T, true>(p, row, ctl, r, sortbuf, staged, sh);
 }
 
 }  // namespace profk

@@ -26,10 +26,86 @@ struct SampleInfo {
 };
 
 // The rank-th largest of the S sample keys at `keys`, as a record under (key descending, sample number ascending):
-// its key and its sample number.  All threads of the CTA call it; uses sh.hist, sh.warp_sums, sh.digit, sh.before, sh.cnt.
+// its key and its sample number.  All threads of the CTA call it (whole warps); uses sh.hist, sh.start, sh.edge,
+// sh.warp_sums, sh.digit, sh.before, sh.cnt, sh.fill, sh.n_edge (the last two left zero).
+// `lower` is a key with at least `rank` sample keys at or above it, if the caller knows one (the first pass's threshold
+// when a tighter rank is wanted), else 0.
+// Ranks up to the CTA's thread count -- all that the plans ask for -- are found without a histogram: a key that has
+// `rank` keys at or above it bounds the answer from below (the caller's, or the rank-th largest of the threads' own
+// maxima after one pass over the keys); the keys at or above the bound, a few times `rank` of them, are collected in
+// shared memory and compared with one another.  (A radix select over all keys, the general path below, spends its
+// first pass on shared-memory atomics into the handful of bins that the keys of a sample crowd: 94 us for 2^17 keys.)
 template <typename T>
 __device__ __noinline__ void kth_sample_record(const uint32_t* keys, uint32_t S, uint32_t rank, SelectShared& sh, uint32_t* key_out,
-                                               uint32_t* j_out) {
+                                               uint32_t* j_out, uint32_t lower = 0) {
+    {
+        const unsigned tid = threadIdx.x, nthr = blockDim.x;
+        constexpr int KU = 8;                    // loads in flight per thread
+        if (rank <= nthr && nthr <= RF_BINS) {
+            if (lower == 0) {
+                // the threads' maxima, and the rank-th largest of them (ties by thread number)
+                uint32_t mx = 0;
+                for (uint32_t i0 = 0; i0 < S; i0 += KU * nthr) {
+                    uint32_t kk[KU];
+#pragma unroll
+                    for (int u = 0; u < KU; ++u) {
+                        const uint32_t i = i0 + u * nthr + tid;
+                        kk[u] = i < S ? __ldcg(&keys[i]) : 0u;
+                    }
+#pragma unroll
+                    for (int u = 0; u < KU; ++u) mx = kk[u] > mx ? kk[u] : mx;
+                }
+                sh.start[tid] = mx;
+                __syncthreads();
+                uint32_t above = 0;
+                for (uint32_t j = 0; j < nthr; ++j) {
+                    const uint32_t o = sh.start[j];
+                    above += (o > mx) || (o == mx && j < tid);
+                }
+                if (above == rank - 1) sh.digit = mx;
+                __syncthreads();
+                lower = sh.digit;
+                __syncthreads();
+            }
+            // collect the records at or above the bound: (key << 32) | ~(sample number), larger = better
+            if (tid == 0) sh.fill = 0;
+            __syncthreads();
+            for (uint32_t i0 = 0; i0 < S; i0 += KU * nthr) {
+                uint32_t kk[KU];
+#pragma unroll
+                for (int u = 0; u < KU; ++u) {
+                    const uint32_t i = i0 + u * nthr + tid;
+                    kk[u] = i < S ? __ldcg(&keys[i]) : 0u;
+                }
+#pragma unroll
+                for (int u = 0; u < KU; ++u) {
+                    const uint32_t i = i0 + u * nthr + tid;
+                    if (i < S && kk[u] >= lower) {
+                        const uint32_t slot = atomicAdd(&sh.fill, 1u);
+                        if (slot < RF_EDGE_CAP) sh.edge[slot] = ((uint64_t)kk[u] << 32) | (uint64_t)(0xFFFFFFFFu - i);
+                    }
+                }
+            }
+            __syncthreads();
+            const uint32_t ncand = sh.fill;
+            __syncthreads();
+            if (tid == 0) sh.fill = 0;
+            if (ncand <= RF_EDGE_CAP) {
+                for (uint32_t c = tid; c < ncand; c += nthr) {
+                    const uint64_t mine = sh.edge[c];
+                    uint32_t above = 0;
+                    for (uint32_t j = 0; j < ncand; ++j) above += sh.edge[j] > mine;
+                    if (above == rank - 1) { sh.digit = (uint32_t)(mine >> 32); sh.cnt = 0xFFFFFFFFu - (uint32_t)mine; }
+                }
+                __syncthreads();
+                *key_out = sh.digit;
+                *j_out = sh.cnt;
+                __syncthreads();
+                return;
+            }
+            __syncthreads();                     // more candidates than the list holds (a sample of equal keys): the general path
+        }
+    }
     constexpr int KB = Elem<T>::KEY_BITS;
     const unsigned tid = threadIdx.x, nthr = blockDim.x;
     uint32_t prefix = 0, need = rank;
@@ -40,9 +116,26 @@ __device__ __noinline__ void kth_sample_record(const uint32_t* keys, uint32_t S,
         const uint32_t nbins = 1u << width;
         for (uint32_t b = tid; b < nbins; b += nthr) sh.hist[b] = 0;
         __syncthreads();
-        for (uint32_t i = tid; i < S; i += nthr) {
-            const uint32_t k = __ldcg(&keys[i]);
-            if (consumed == 0 || (k >> (KB - consumed)) == prefix) atomicAdd(&sh.hist[(k >> shift) & (nbins - 1)], 1u);
+        // (whole warps together: the keys of a sample crowd a few bins of the first pass, and the lanes that meet in a
+        // bin add once for all of them -- one shared-memory atomic per key took a 2^17-key sample 100 us a pass)
+        // (eight loads in flight per thread: one at a time, a 2^17-key sample took 128 round trips to L2 a pass)
+        constexpr int KU = 8;
+        for (uint32_t i0 = 0; i0 < S; i0 += KU * nthr) {
+            uint32_t kk[KU];
+#pragma unroll
+            for (int u = 0; u < KU; ++u) {
+                const uint32_t i = i0 + u * nthr + tid;
+                kk[u] = i < S ? __ldcg(&keys[i]) : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < KU; ++u) {
+                const uint32_t i = i0 + u * nthr + tid;
+                const uint32_t k = kk[u];
+                const bool in_class = i < S && (consumed == 0 || (k >> (KB - consumed)) == prefix);
+                const uint32_t digit = in_class ? (k >> shift) & (nbins - 1) : 0xFFFFFFFFu;
+                const unsigned peers = __match_any_sync(FULL_MASK, digit);
+                if (in_class && lane_id() == (unsigned)(__ffs(peers) - 1)) atomicAdd(&sh.hist[digit], (uint32_t)__popc(peers));
+            }
         }
         __syncthreads();
         // the digit of the need-th largest key of the class: bins from the top
@@ -65,20 +158,64 @@ __device__ __noinline__ void kth_sample_record(const uint32_t* keys, uint32_t S,
         consumed += width;
         __syncthreads();
     }
-    // of the samples with exactly this key, the need-th in sample order
+    // Of the samples with exactly this key, the need-th in sample order.  Sample i is looked at in round i / nthr by
+    // thread i % nthr: every warp votes on its 32 samples of a round and notes the count; the counts, in (round, warp)
+    // order, are scanned once, and the warp whose vote holds the need-th match votes again to find the lane.  (Up to
+    // RF_BINS counts at a time: the rounds are taken in groups.)
+    const unsigned lane = lane_id(), warp = tid >> 5, nwarps = nthr >> 5;
+    const uint32_t rounds = (S + nthr - 1) / nthr, rounds_per_group = RF_BINS / nwarps;
     uint32_t seen = 0;
-    for (uint32_t base = 0; base < S; base += nthr) {
-        const uint32_t i = base + tid;
-        const uint32_t flag = i < S && __ldcg(&keys[i]) == prefix;
-        const uint32_t in_run = (uint32_t)__syncthreads_count((int)flag);
-        const uint32_t incl = block_scan_any(flag, sh.warp_sums);
-        if (flag && seen + incl == need) sh.cnt = i;
-        seen += in_run;
-        if (seen >= need) break;
+    for (uint32_t g0 = 0; g0 < rounds; g0 += rounds_per_group) {
+        const uint32_t g1 = g0 + rounds_per_group < rounds ? g0 + rounds_per_group : rounds;
+        for (uint32_t r0 = g0; r0 < g1; r0 += 8) {                        // (eight loads in flight)
+            uint32_t kk[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const uint32_t i = (r0 + u) * nthr + tid;
+                kk[u] = (r0 + u < g1 && i < S) ? __ldcg(&keys[i]) : ~prefix;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const uint32_t i = (r0 + u) * nthr + tid;
+                const unsigned bal = __ballot_sync(FULL_MASK, r0 + u < g1 && i < S && kk[u] == prefix);
+                if (lane == 0 && r0 + u < g1) sh.hist[(r0 + u - g0) * nwarps + warp] = (uint32_t)__popc(bal);
+            }
+        }
+        __syncthreads();
+        const uint32_t ncounts = (g1 - g0) * nwarps, per = (ncounts + nthr - 1) / nthr;
+        uint32_t sum = 0;
+        for (uint32_t j = 0; j < per; ++j) {
+            const uint32_t c = tid * per + j;
+            sum += c < ncounts ? sh.hist[c] : 0u;
+        }
+        uint32_t before = seen + block_scan_any(sum, sh.warp_sums) - sum;
+        for (uint32_t j = 0; j < per; ++j) {
+            const uint32_t c = tid * per + j;
+            const uint32_t cnt = c < ncounts ? sh.hist[c] : 0u;
+            if (before < need && need <= before + cnt) { sh.digit = c; sh.before = before; }
+            before += cnt;
+        }
+        if (tid == nthr - 1) sh.n_edge = before;             // matches up to the end of this group
+        __syncthreads();
+        const uint32_t upto = sh.n_edge;
+        if (need <= upto) {
+            const uint32_t c = sh.digit, r = g0 + c / nwarps, off = need - sh.before;      // the off-th match of that vote
+            if (warp == c % nwarps) {
+                const uint32_t i = r * nthr + tid;
+                const bool flag = i < S && __ldcg(&keys[i]) == prefix;
+                const unsigned bal = __ballot_sync(FULL_MASK, flag);
+                if (flag && (uint32_t)__popc(bal & ((2u << lane) - 1u)) == off) sh.cnt = i;
+            }
+            break;
+        }
+        seen = upto;
+        __syncthreads();                                     // the counts are rewritten by the next group
     }
     __syncthreads();
     *key_out = prefix;
     *j_out = sh.cnt;
+    __syncthreads();
+    if (tid == 0) sh.n_edge = 0;                             // as the callers' kernels set it at their start
     __syncthreads();
 }
 
