@@ -172,3 +172,24 @@ def test_config4_flattened_2p29_bf16():
     mask = np.zeros(n, dtype=bool)
     mask[idx] = True
     assert np.array_equal(out["mask"].cpu().numpy().view(np.uint32), o_topk.pack_mask(mask))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_a_selection_so_dense_that_the_filters_candidate_list_overflows(dtype):
+    """A quarter of the row is kept: every CTA of the deferring filter notes more candidates than its list holds, the
+    rest leave through the inline slow path without being counted in the bins, and the kernel behind the filter is told to
+    count for itself.  Both entry points stay exact."""
+    n, k = 1 << 24, 1 << 22
+    pl = profk.plan(n, k, 1e-3)
+    assert pl.mode == 0 and pl.capacity > 444 * 6144          # more candidates than all lists together
+    x = workloads.normal(1, n, seed=63, dtype=dtype)[0]
+    xn = workloads.as_numpy(x)
+    xd = x.cuda()
+    check_forms(xn, k, run(xd, k, seed=1, want_pairs=True, want_mask=True, want_dense=True))
+    assert profk.read_stats(1)[0][3] == profk.ROW_OK
+    v, i = profk.topk(xd, k, seed=2)
+    torch.cuda.synchronize()
+    ov, oi = o_topk.topk(xn[None, :], k)
+    assert np.array_equal(i.cpu().numpy(), oi[0])
+    assert np.array_equal(bits(workloads.as_numpy(v)), bits(ov[0]))
+    assert profk.read_stats(1)[0][3] == profk.ROW_OK
