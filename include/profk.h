@@ -117,9 +117,9 @@ enum {
  *             are kept: for selections the single-CTA refine orders (k <= 16384; <= 8192 for up to four rows) any
  *             sample for up to four rows, m <= 32768 for up to 18 rows, m <= 4096 for larger batches (there the
  *             grid-wide repair kernel takes the pass, as long as fewer than eight rows of the call failed); for
- *             larger selections a single row (profk_topk_* with rows == 1, and the BatchTopK entry points, whose
- *             one kernel after the filter takes the pass itself).  Larger selections from several rows and
- *             anything else go straight to the exact selection.
+ *             larger selections up to four rows (a single row, and the BatchTopK entry points: the one kernel after
+ *             the filter takes the pass itself; two to four rows: the repair kernel).  Larger selections from more
+ *             rows and anything else go straight to the exact selection.
  * Both bounds are binomial tail bounds valid for the stratified sampler the
  * library uses (one uniform draw from each of m equal strata of the row).
  */

@@ -49,8 +49,8 @@ template <typename T> struct FallbackParams {
     uint32_t sort_cap;        // power of two >= k: records the dynamic shared memory holds
     int parallel;             // 1 = the one-row-per-CTA mode may be used (its scratch is there, or none is needed)
     // The second filtering pass (second_chance.cuh) of a row that failed the check, taken by the whole grid before the
-    // exact selection: when the rows are repaired one after the other by the kernel below and ordered there
-    // (sort_rows == 1), and by the fused large-selection kernels for their single row.
+    // exact selection: when the rows are repaired one after the other by the kernel below, and by the fused
+    // large-selection kernels for their single row.
     SampleInfo sample;        // sample.keys == null: none
     uint4* thr2;              // rows threshold records of that pass
 };
@@ -272,12 +272,12 @@ __global__ void __launch_bounds__(FB_THREADS) fallback_kernel(const FallbackPara
                 const uint64_t row = chunk + w * 32 + b;
 
                 // ---- first another filtering pass with the plan's tighter / looser sample rank, if it names one ----
-                if (p.sort_rows) {
+                {
                     uint32_t R2 = 0, key2 = 0;
                     const int again = grid_second_chance_row<T>(p, row, __ldcg(&p.ctl[row].status), sh, &R2, &key2);
                     if (again < 0) return;
                     if (again == 1) {
-                        if (blockIdx.x == 0) {
+                        if (p.sort_rows && blockIdx.x == 0) {      // (large selections: the kernel behind this one orders the row)
                             extern __shared__ __align__(16) unsigned char fb_smem[];
                             finish_from_segments<T>(p.buf + row * p.buf_stride, R2, p.k, p.sort_cap, reinterpret_cast<uint64_t*>(fb_smem), sh,
                                                     row, p.out_vals, p.out_idx);

@@ -528,8 +528,9 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
 
     // A second filtering pass for rows that fail the count check (plan->r_tight / r_loose) needs the sample's keys: they
     // are kept when the workspace has room for them and a kernel that takes that pass does the repair: the refine
-    // kernel's clusters, the grid-wide repair kernel, or the fused kernel of a large selection from a single row.
-    const bool keep_keys = (!large || rows == 1) && plan->mode == 0 && (plan->r_tight > 0 || plan->r_loose > 0) &&
+    // kernel's clusters, the grid-wide repair kernel (large selections: up to four rows), or the fused kernel of a large
+    // selection from a single row.
+    const bool keep_keys = (!large || rows <= GATHER_MAX_ROWS) && plan->mode == 0 && (plan->r_tight > 0 || plan->r_loose > 0) &&
                            (rows <= GATHER_MAX_ROWS || plan->m <= (rows <= XS_MAX_ROWS ? KEPT_SAMPLE_MAX : KEPT_SAMPLE_BATCH_MAX));
     SampleInfo sample = {};
     if (keep_keys) {

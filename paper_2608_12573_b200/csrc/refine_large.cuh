@@ -159,7 +159,12 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
             }
         } else {
             if (ctl.status == ROW_OK) continue;  // already written by the first phase
-            n = p.k;                             // the exact selection left exactly k records
+            if (ctl.status == ROW_OVERFLOW_REFILTERED || ctl.status == ROW_RECALL_REFILTERED) {
+                n = ctl.count;                   // what a second filtering pass left (its threshold is in the control block)
+                from_filter = true;
+            } else {
+                n = p.k;                         // the exact selection left exactly k records
+            }
             pcount[0] = n;
         }
         const uint32_t kk = n < p.k ? n : p.k;

@@ -214,3 +214,19 @@ def test_large_selections_from_one_row_take_the_second_pass_inside_their_fused_k
     torch.cuda.synchronize()
     _btk_forms(xn, k, out)
     assert profk.read_stats(1)[0][3] == profk.ROW_OVERFLOW_REFILTERED
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_large_selections_from_a_few_rows_take_the_second_pass_in_the_repair_kernel(dtype):
+    """Two to four rows with k beyond what one CTA orders: the grid-wide repair kernel between the two phases of the large
+    refine filters a failed row once more; the second phase orders what that pass left."""
+    rows, n, k, m = 3, 2_000_003, 20_000, 65536                               # a sample rank keeps about 30.5 elements
+    x = workloads.normal(rows, n, seed=88, dtype=dtype)
+    cap = 34_000
+    check(x, k, profk.Plan(m=m, r=1500, capacity=cap, k_accept=k, mode=0, r_tight=900), seed=40, want_status=profk.ROW_OVERFLOW_REFILTERED)
+    check(x, k, profk.Plan(m=m, r=1500, capacity=cap, k_accept=k, mode=0, r_tight=1490), seed=41, want_status=profk.ROW_OVERFLOW)
+    check(x, k, profk.Plan(m=m, r=450, capacity=cap, k_accept=k, mode=0, r_loose=900), seed=42, want_status=profk.ROW_RECALL_REFILTERED)
+    check(x, k, profk.Plan(m=m, r=450, capacity=cap, k_accept=k, mode=0), seed=43, want_status=profk.ROW_RECALL)
+    # a mix: one row's own capacity problem only (the others pass): a capacity between the rows' survivor counts
+    pl = profk.Plan(m=m, r=1000, capacity=cap, k_accept=k, mode=0, r_tight=800)        # about 30.5 K survivors: all pass
+    check(x, k, pl, seed=44, want_status=profk.ROW_OK)
