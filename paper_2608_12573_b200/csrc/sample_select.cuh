@@ -56,7 +56,7 @@ struct WsHeader {
     uint32_t bar_count;  // arrivals at the grid barrier since the start of the call (grid_barrier.cuh)
     uint32_t bar_gen;    // (unused)
     uint32_t error;      // non-zero = a bounded wait gave up
-    uint32_t done;       // CTAs of the filter kernel that have finished (ticket for its last CTA)
+    uint32_t done;       // CTAs of the emit / large-refine kernel that have cleared their share of the bins
     uint32_t n_failed;   // rows whose count check failed
     uint32_t tile_counter;  // hands out the filter kernel's tiles
     uint32_t pad[58];
