@@ -25,7 +25,7 @@ using namespace profk;
 namespace {
 
 #ifndef PROFK_DYNAMIC_ROUNDS
-#define PROFK_DYNAMIC_ROUNDS 2      // tiles per CTA (on average) that the filter hands out dynamically at the end
+#define PROFK_DYNAMIC_ROUNDS 2      // fewest tiles per CTA (on average) that the filter hands out dynamically at the end
 #endif
 constexpr int FILTER_THREADS = PROFK_FILTER_THREADS;
 constexpr int FILTER_UNROLL = PROFK_FILTER_UNROLL;
@@ -295,10 +295,17 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
         (deferred ? di.filter_defer_blocks_per_sm[dtype_index<T>()] : di.filter_blocks_per_sm[dtype_index<T>()]);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)std::min<uint64_t>(fp.total_tiles, max_grid));
-    // all but the last ~PROFK_DYNAMIC_ROUNDS tiles per CTA follow the fixed stride
+    // All but the last few tiles per CTA follow the fixed stride; the rest come from a counter, so that all CTAs finish
+    // together.  The longer the launch, the more of them: the three CTAs of an SM do not advance at the same rate (the
+    // one that arrived first is a few per cent ahead: after 148 tiles its neighbours were 10-20 us behind), and two
+    // rounds cannot level that.  An eighth of a single row's rounds, at most 32; a sixteenth of a batch's, at most 12
+    // (a batch pays a division per dynamic tile): 2^30 fp32 605 -> 595 us, 2^29 bf16 K = 131072 207 -> 196, 512 rows of
+    // 2^20 400 -> 394 (bf16 253 -> 248); 2^26 (18 rounds) keeps its two.
     const uint64_t rounds = fp.total_tiles / cfg.gridDim.x;
-    fp.dyn_start = (uint32_t)((rounds > PROFK_DYNAMIC_ROUNDS ? rounds - PROFK_DYNAMIC_ROUNDS : 0) * cfg.gridDim.x);
-    if (rounds <= PROFK_DYNAMIC_ROUNDS) fp.tile_counter = nullptr;
+    const uint64_t dyn_rounds = rows > 1 ? std::min<uint64_t>(std::max<uint64_t>(rounds / 16, PROFK_DYNAMIC_ROUNDS), 12)
+                                         : std::min<uint64_t>(std::max<uint64_t>(rounds / 8, PROFK_DYNAMIC_ROUNDS), 32);
+    fp.dyn_start = (uint32_t)((rounds > dyn_rounds ? rounds - dyn_rounds : 0) * cfg.gridDim.x);
+    if (rounds <= dyn_rounds) fp.tile_counter = nullptr;
     cfg.blockDim = dim3(FILTER_THREADS);
     // A single row scanned behind the threshold kernel: each CTA copies its next tiles into shared memory while it waits.
     // (Not the build that defers its candidates: their list takes the shared memory.)
