@@ -46,6 +46,7 @@ template <typename T> struct FilterParams {
     int use_pdl;             // 1 = launched as a programmatic dependent of the threshold kernel
     uint32_t* tile_counter;  // zeroed counter that hands out the tiles from dyn_start on (null = fixed stride throughout)
     uint32_t dyn_start;      // first tile handed out dynamically (a multiple of the grid size)
+    uint32_t dyn_chunk;      // consecutive tiles a CTA takes from the counter at a time (>= 1)
     // Partitioned append (the PARTS build of the kernel only).  With very many survivors the single counter of a
     // row becomes the bottleneck -- atomics on one address retire about 2 ns apart, 164 K of them are a quarter of
     // a 2^30-element scan -- so the row's buffer is cut into FILTER_PARTS equal parts, each with a counter in a
@@ -435,7 +436,8 @@ __device__ __noinline__ void defer_process_batch_counting(const FilterParams<T>&
 // run).  A CTA takes tiles blockIdx.x, + gridDim.x, ... with its warps running freely; the last few
 // tiles of the launch (from dyn_start on) come from a global counter instead, so that SMs that saw
 // less bandwidth take fewer of them and all CTAs finish together.  The counter is read one tile
-// ahead, so its round trip hides behind the loads; only this tail needs a CTA barrier per tile.
+// ahead, so its round trip hides behind the loads; only this tail needs a CTA barrier per tile
+// (per chunk of dyn_chunk consecutive tiles: batches take four at a time).
 template <typename T, int THREADS, int UNROLL, bool PARTS = false, bool DEFER = false, bool HIST = false>
 __global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOCKS_F32 : PROFK_FILTER_MINBLOCKS_BF16) filter_kernel(const __grid_constant__ FilterParams<T> p) {
     static_assert(!HIST || (DEFER && !PARTS), "only the deferring build counts its records");
@@ -575,9 +577,10 @@ __global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOC
         // the launch are handed out by the counter.  Thread 0 asks for the next one now; the answer is
         // needed only after this tile.
         const bool dynamic = p.tile_counter != nullptr && tile + gridDim.x >= p.dyn_start;
+        const bool claim = dynamic && (parity >> 1) == 0;        // (parity: bit 0 = which word of s_next, the rest = tiles left of the chunk)
         uint32_t upcoming = 0;
-        if (dynamic && threadIdx.x == 0) {
-            const uint32_t t = p.dyn_start + atomicAdd(p.tile_counter, 1u);
+        if (claim && threadIdx.x == 0) {
+            const uint32_t t = p.dyn_start + atomicAdd(p.tile_counter, p.dyn_chunk);
             upcoming = t < total_tiles ? t : total_tiles;
         }
 
@@ -628,11 +631,14 @@ __global__ void __launch_bounds__(THREADS, sizeof(T) == 4 ? PROFK_FILTER_MINBLOC
             if (o != 0xFFFFFFFFu) skip_row = o;
         }
 
-        if (dynamic) {
-            if (threadIdx.x == 0) s_next[parity] = upcoming;
+        if (claim) {
+            if (threadIdx.x == 0) s_next[parity & 1u] = upcoming;
             __syncthreads();
-            tile = s_next[parity];
-            parity ^= 1u;
+            tile = s_next[parity & 1u];
+            parity = ((parity & 1u) ^ 1u) | ((p.dyn_chunk - 1u) << 1);
+        } else if (dynamic) {
+            tile = tile + 1u;                    // the next tile of the chunk this CTA holds
+            parity -= 2u;
         } else {
             tile = total_tiles - tile <= gridDim.x ? total_tiles : tile + gridDim.x;
         }

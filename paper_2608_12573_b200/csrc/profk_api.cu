@@ -298,12 +298,14 @@ int launch_filter(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, co
     // All but the last few tiles per CTA follow the fixed stride; the rest come from a counter, so that all CTAs finish
     // together.  The longer the launch, the more of them: the three CTAs of an SM do not advance at the same rate (the
     // one that arrived first is a few per cent ahead: after 148 tiles its neighbours were 10-20 us behind), and two
-    // rounds cannot level that.  An eighth of a single row's rounds, at most 32; a sixteenth of a batch's, at most 12
-    // (a batch pays a division per dynamic tile): 2^30 fp32 605 -> 595 us, 2^29 bf16 K = 131072 207 -> 196, 512 rows of
-    // 2^20 400 -> 394 (bf16 253 -> 248); 2^26 (18 rounds) keeps its two.
+    // rounds cannot level that.  An eighth of a single row's rounds, at most 32, one tile at a time; a quarter of a
+    // batch's, at most 32, and there a CTA takes four consecutive tiles from the counter at a time (a dynamic tile costs a
+    // batch a CTA barrier and a division): 2^30 fp32 605 -> 595 us, 2^29 bf16 K = 131072 207 -> 196, 512 rows of 2^20
+    // 400 -> 386 (bf16 253 -> 242); 2^26 (18 rounds) keeps its two.
     const uint64_t rounds = fp.total_tiles / cfg.gridDim.x;
-    const uint64_t dyn_rounds = rows > 1 ? std::min<uint64_t>(std::max<uint64_t>(rounds / 16, PROFK_DYNAMIC_ROUNDS), 12)
+    const uint64_t dyn_rounds = rows > 1 ? std::min<uint64_t>(std::max<uint64_t>(rounds / 4, PROFK_DYNAMIC_ROUNDS), 32)
                                          : std::min<uint64_t>(std::max<uint64_t>(rounds / 8, PROFK_DYNAMIC_ROUNDS), 32);
+    fp.dyn_chunk = rows > 1 ? (dyn_rounds >= 16 ? 4u : dyn_rounds >= 8 ? 2u : 1u) : 1u;
     fp.dyn_start = (uint32_t)((rounds > dyn_rounds ? rounds - dyn_rounds : 0) * cfg.gridDim.x);
     if (rounds <= dyn_rounds) fp.tile_counter = nullptr;
     cfg.blockDim = dim3(FILTER_THREADS);
