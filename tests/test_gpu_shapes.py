@@ -75,3 +75,19 @@ def test_shape(case, rows, n, k, dtype, eps, recall, recipe):
         assert np.array_equal(i[r, :n_real], oi[r, :n_real]), f"row {r}: indices differ from the oracle"
         assert np.array_equal(bits(v[r, :n_real]), bits(ov[r, :n_real])), f"row {r}: values differ from the oracle"
         assert np.all(i[r, n_real:] == -1)
+
+
+@pytest.mark.parametrize("rows,n,dtype", [(128, (1 << 20) + 12_345, torch.float32), (256, (1 << 20) - 77, torch.bfloat16),
+                                          (300, 1 << 20, torch.float32)])
+def test_batches_long_enough_for_every_way_the_filter_deals_its_last_tiles(rows, n, dtype):
+    """The filter hands the last rounds of a launch out from a counter, one tile at a time for short launches and two or
+    four consecutive tiles at a time for long batches.  These launches have 37 to 87 rounds of tiles (chunks of two and of
+    four; the 512-row configuration tests cover longer ones) and ragged rows, so that chunks end inside the last tile."""
+    k = 50
+    x = workloads.normal(rows, n, seed=rows, dtype=dtype)
+    v, i = profk.topk(x.cuda(), k, eps=1e-3, seed=5)
+    torch.cuda.synchronize()
+    xn = workloads.as_numpy(x)
+    ov, oi = o_topk.topk(xn, k)
+    assert np.array_equal(i.cpu().numpy(), oi)
+    assert np.array_equal(bits(workloads.as_numpy(v)), bits(ov))
