@@ -52,7 +52,7 @@ CONFIGS = {
 
 # DRAM bytes (read + write) of one filter launch at cfg2, from the ncu capture summarised in
 # profiles/filter_kernel_f32_2p26.md (dram__bytes_read.sum + dram__bytes_write.sum).
-FILTER_TRAFFIC_BYTES = {"cfg2": 272.39e6}
+FILTER_TRAFFIC_BYTES = {"cfg2": 272.20e6}
 
 L2_BYTES = 126 * 1024 * 1024
 
