@@ -420,6 +420,10 @@ int launch_refine(const DeviceInfo& di, const T* in, int64_t rows, int64_t N, Ro
     rp.cluster_size = (uint32_t)csize;
     unsigned threads = csize > 1 ? REFINE_CLUSTER_THREADS : 128;      // a cluster may have to read whole rows
     while (threads < 1024 && threads * 8 < (unsigned)capacity) threads <<= 1;
+    // More rows than SMs, one CTA per row: CTAs of 1024 threads run one to an SM, wave after wave (512 rows: 3.4 us a
+    // row, the last done 17 us after the filter); CTAs of 256 threads all start at once.  A buffer is a third full as a
+    // rule, so 256 threads hold a row's records in one batch of eight when the capacity is within 6144.
+    if (csize == 1 && !direct && rows > di.sm_count && capacity <= 6144) threads = 256;
     // A failed row is cut into segments, one cluster each, so that all SMs read it: as many clusters per
     // row as the SMs hold at once, but no more than the row has tiles for.
     int64_t nseg = 1;

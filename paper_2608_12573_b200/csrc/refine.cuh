@@ -107,8 +107,11 @@ __device__ __forceinline__ void refine_row(const RefineParams<T>& p, uint64_t ro
     // ---- bin the records by the distance d of their key above tau, on a logarithmic scale: the bin is
     //      the exponent and the top seven mantissa bits of d as a float (monotone in d, 32 x 128 = 4096
     //      bins, fine where the records are dense -- just above tau -- and coarse where they are rare).
-    //      Bin 0 holds the largest keys. ----
+    //      Bin 0 holds the largest keys.  A CTA of 256 threads (the rows of a large batch, a thousand or two records
+    //      each) takes five mantissa bits, 1024 bins: four bins per thread again, and a quarter of the scan. ----
     const uint32_t tau_key = Elem<T>::key(Elem<T>::from_bits(ctl.tau_bits));
+    const uint32_t nbins = nthr == 256 ? RF_BINS / 4 : RF_BINS;
+    const int bin_shift = nthr == 256 ? 18 : 16;
     const uint32_t nbatch = (n + 8 * nthr - 1) / (8 * nthr);   // one batch = 8 records per thread
     auto load_batch = [&](uint32_t b) {
 #pragma unroll
@@ -122,8 +125,8 @@ __device__ __forceinline__ void refine_row(const RefineParams<T>& p, uint64_t ro
         const uint32_t key = record_key(rec);
         const uint32_t d = key > tau_key ? key - tau_key : 0u;
         const uint32_t f = __float_as_uint((float)d);           // 0 for d = 0, exponent >= 127 otherwise
-        const uint32_t level = f > (127u << 23) ? (f >> 16) - (127u << 7) : 0u;     // 0 .. 4095
-        return (uint32_t)(RF_BINS - 1) - level;
+        const uint32_t level = f > (127u << 23) ? (f >> bin_shift) - (127u << (23 - bin_shift)) : 0u;     // 0 .. nbins - 1
+        return (nbins - 1u) - level;
     };
 
     for (uint32_t b = 0; b < nbatch; ++b) {
@@ -135,7 +138,7 @@ __device__ __forceinline__ void refine_row(const RefineParams<T>& p, uint64_t ro
     __syncthreads();
 
     // ---- scan the bin counts: first position of every bin, and the bin of the kk-th best record ----
-    if (nthr * 4 == RF_BINS) {
+    if (nthr * 4 == nbins) {
         // four bins per thread, read and written as one 16-byte vector; two barriers in all
         const uint4 c = reinterpret_cast<const uint4*>(sh.hist)[tid];
         const uint32_t sum = c.x + c.y + c.z + c.w;
@@ -147,7 +150,7 @@ __device__ __forceinline__ void refine_row(const RefineParams<T>& p, uint64_t ro
         }
         if (lane == 31) sh.warp_sums[tid >> 5] = incl;
         __syncthreads();
-        uint32_t w = sh.warp_sums[lane];                       // every warp scans the 32 warp totals itself
+        uint32_t w = lane < (nthr >> 5) ? sh.warp_sums[lane] : 0u;       // every warp scans the warps' totals itself
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
             const uint32_t v = __shfl_up_sync(FULL_MASK, w, d);
@@ -165,16 +168,16 @@ __device__ __forceinline__ void refine_row(const RefineParams<T>& p, uint64_t ro
         reinterpret_cast<uint4*>(sh.start)[tid] = make_uint4(b0, b1, b2, b3);
         reinterpret_cast<uint4*>(sh.hist)[tid] = make_uint4(b0, b1, b2, b3);     // the bins' write cursors
     } else {
-        const uint32_t per = (RF_BINS + nthr - 1) / nthr;
+        const uint32_t per = (nbins + nthr - 1) / nthr;
         uint32_t sum = 0;
         for (uint32_t j = 0; j < per; ++j) {
             const uint32_t bin = tid * per + j;
-            sum += bin < RF_BINS ? sh.hist[bin] : 0;
+            sum += bin < nbins ? sh.hist[bin] : 0;
         }
         uint32_t before = block_scan_any(sum, sh.warp_sums) - sum;
         for (uint32_t j = 0; j < per; ++j) {
             const uint32_t bin = tid * per + j;
-            if (bin < RF_BINS) {
+            if (bin < nbins) {
                 const uint32_t c = sh.hist[bin];
                 if (before < kk && kk <= before + c) { sh.digit = bin; sh.before = before; sh.cnt = c; }
                 if (before < kk && c > RF_EDGE_CAP) sh.crowded = 1;         // a bin that matters is too full to rank
