@@ -31,13 +31,16 @@ constexpr int FILTER_THREADS = PROFK_FILTER_THREADS;
 constexpr int FILTER_UNROLL = PROFK_FILTER_UNROLL;
 constexpr uint32_t SORT_CAP_MAX = 16384;         // largest k the single-CTA refine orders in shared memory
 // Selections the whole grid refines (refine_large_kernel) instead of one CTA per row: beyond the single-CTA limit, and
-// from 8193 on when there are at most LARGE_FEW_ROWS rows -- one CTA takes 100-280 us over 12000-16384 records of a
-// long row (bf16, whose equal keys send the selection through the index digits, worst), the grid 80-100; with many
-// rows the CTAs work side by side and win.
+// from 8193 on (bf16: from 3073 on) when there are at most LARGE_FEW_ROWS rows -- one CTA takes 100-280 us over
+// 12000-16384 records of a long row (bf16, whose equal keys send the selection through the index digits, worst), the
+// grid 80-100; with many rows the CTAs work side by side and win.  Since the grid-wide path starts from the filter's
+// histogram a bf16 row is better off there from a few thousand on (2^28 bf16: k = 4096 137 -> 118 us, k = 8192
+// 245 -> 114; 2^26: 58 -> 56, 106 -> 57; k = 2048 still 103 against 118); fp32 rows are not (k = 8192: 186 against 193).
 constexpr int64_t LARGE_FEW_ROWS = 4;
 constexpr int64_t LARGE_FEW_K = 8192;
-inline bool large_selection(int64_t rows, int64_t k) {
-    return k > (int64_t)SORT_CAP_MAX || (rows <= LARGE_FEW_ROWS && k > LARGE_FEW_K);
+constexpr int64_t LARGE_FEW_K_HALF = 3072;
+inline bool large_selection(int64_t rows, int64_t k, size_t elem_size) {
+    return k > (int64_t)SORT_CAP_MAX || (rows <= LARGE_FEW_ROWS && k > (elem_size == 2 ? LARGE_FEW_K_HALF : LARGE_FEW_K));
 }
 constexpr unsigned FB_MAX_CTAS = 256;             // most CTAs of the grid-wide exact selection (its per-CTA scratch is sized for them)
 // Samples above this size are gathered by a kernel over all SMs (65536: 2^26, k = 16, S = 40529 took 49.7 us, not 47.0).
@@ -506,7 +509,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         std::lock_guard<std::mutex> lock(g_mutex);
         ws = g_workspace[dev];
     }
-    const bool large = large_selection(rows, k);
+    const bool large = large_selection(rows, k, sizeof(T));
     const WsLayout lay = ws_layout(rows, capacity, k, large);
     if (!ws.ptr || ws.bytes < lay.total) return PROFK_EWORKSPACE;
     const uint64_t row_stride = row_stride_for(capacity, large);
@@ -873,7 +876,7 @@ int refine_gathered(const uint64_t* records, const uint32_t* states, const int64
         std::lock_guard<std::mutex> lock(g_mutex);
         ws = g_workspace[dev];
     }
-    const bool large = large_selection(1, k);
+    const bool large = large_selection(1, k, sizeof(T));
     const WsLayout lay = ws_layout(1, capacity, k, large);
     if (!ws.ptr || ws.bytes < lay.total) return PROFK_EWORKSPACE;
     const uint64_t row_stride = row_stride_for(capacity, large);
@@ -911,7 +914,8 @@ extern "C" {
 int profk_workspace_bytes(int64_t rows, int64_t capacity, int64_t k, size_t* bytes) {
     if (!bytes || rows < 1 || capacity < 1 || k < 1 || capacity < k || capacity > N_MAX || rows * capacity >= (1LL << 40))
         return PROFK_EINVAL;
-    *bytes = ws_layout(rows, capacity, k, large_selection(rows, k)).total;
+    // (enough for either element type: the two take the grid-wide layout from different k on)
+    *bytes = std::max(ws_layout(rows, capacity, k, large_selection(rows, k, 4)).total, ws_layout(rows, capacity, k, large_selection(rows, k, 2)).total);
     return PROFK_OK;
 }
 
@@ -1045,7 +1049,7 @@ int profk_topk_noalloc_f32(const float* in, int64_t rows, int64_t N, int64_t k, 
         }
     }
     if (rows * plan.capacity >= (1LL << 40)) return PROFK_EINVAL;
-    if (ws_layout(rows, plan.capacity, k, large_selection(rows, k)).total > NOALLOC_SCRATCH_BYTES) return PROFK_ETOOLARGE;
+    if (ws_layout(rows, plan.capacity, k, large_selection(rows, k, sizeof(float))).total > NOALLOC_SCRATCH_BYTES) return PROFK_ETOOLARGE;
     g_ws_override_ptr = scratch;
     g_ws_override_bytes = NOALLOC_SCRATCH_BYTES;
     const int rc = topk_planned<float>(in, rows, N, k, &plan, seed, stream, out_vals, out_idx);
