@@ -114,7 +114,7 @@ enum {
  *             with the same check k <= R <= M -- one more read of the row at streaming speed -- and only a row
  *             that fails again is selected exactly.  The ranks aim midway between k and M:
  *             r_tight = floor(r (k + M) / (2 M)), r_loose = r + ceil((M - k) m / (2 N)).  Used when the sample's keys
- *             are kept: for selections the single-CTA refine orders (k <= 16384; for up to four rows <= 8192, bf16 <= 3072) any
+ *             are kept: for selections the single-CTA refine orders (k <= 16384; <= 8192 for up to four rows, <= 3072 for one bf16 row) any
  *             sample for up to four rows, m <= 32768 for up to 18 rows, m <= 4096 for larger batches (there the
  *             grid-wide repair kernel takes the pass, as long as fewer than eight rows of the call failed); for
  *             larger selections up to four rows (a single row, and the BatchTopK entry points: the one kernel after

@@ -31,7 +31,7 @@ constexpr int FILTER_THREADS = PROFK_FILTER_THREADS;
 constexpr int FILTER_UNROLL = PROFK_FILTER_UNROLL;
 constexpr uint32_t SORT_CAP_MAX = 16384;         // largest k the single-CTA refine orders in shared memory
 // Selections the whole grid refines (refine_large_kernel) instead of one CTA per row: beyond the single-CTA limit, and
-// from 8193 on (bf16: from 3073 on) when there are at most LARGE_FEW_ROWS rows -- one CTA takes 100-280 us over
+// from 8193 on (a single bf16 row: from 3073 on) when there are at most LARGE_FEW_ROWS rows -- one CTA takes 100-280 us over
 // 12000-16384 records of a long row (bf16, whose equal keys send the selection through the index digits, worst), the
 // grid 80-100; with many rows the CTAs work side by side and win.  Since the grid-wide path starts from the filter's
 // histogram a bf16 row is better off there from a few thousand on (2^28 bf16: k = 4096 137 -> 118 us, k = 8192
@@ -40,7 +40,9 @@ constexpr int64_t LARGE_FEW_ROWS = 4;
 constexpr int64_t LARGE_FEW_K = 8192;
 constexpr int64_t LARGE_FEW_K_HALF = 3072;
 inline bool large_selection(int64_t rows, int64_t k, size_t elem_size) {
-    return k > (int64_t)SORT_CAP_MAX || (rows <= LARGE_FEW_ROWS && k > (elem_size == 2 ? LARGE_FEW_K_HALF : LARGE_FEW_K));
+    // (the lower switch of bf16 is for a single row: only there the grid-wide path is one launch that starts from the
+    // filter's histogram; two rows of 2^22 bf16 with k = 4096 took 68 us through it against 34)
+    return k > (int64_t)SORT_CAP_MAX || (rows <= LARGE_FEW_ROWS && k > LARGE_FEW_K) || (rows == 1 && elem_size == 2 && k > LARGE_FEW_K_HALF);
 }
 constexpr unsigned FB_MAX_CTAS = 256;             // most CTAs of the grid-wide exact selection (its per-CTA scratch is sized for them)
 // Samples above this size are gathered by a kernel over all SMs (65536: 2^26, k = 16, S = 40529 took 49.7 us, not 47.0).
