@@ -114,12 +114,15 @@ enum {
  *             with the same check k <= R <= M -- one more read of the row at streaming speed -- and only a row
  *             that fails again is selected exactly.  The ranks aim midway between k and M:
  *             r_tight = floor(r (k + M) / (2 M)), r_loose = r + ceil((M - k) m / (2 N)).  Used when the sample's keys
- *             are kept: for selections the single-CTA refine orders (k <= 16384; <= 8192 for up to four rows, <= 3072 for one bf16 row) any
- *             sample for up to four rows, m <= 32768 for up to 18 rows, m <= 4096 for larger batches (there the
- *             grid-wide repair kernel takes the pass, as long as fewer than eight rows of the call failed); for
- *             larger selections up to four rows (a single row, and the BatchTopK entry points: the one kernel after
- *             the filter takes the pass itself; two to four rows: the repair kernel).  Larger selections from more
- *             rows and anything else go straight to the exact selection.
+ *             are kept: any sample for up to four rows, m <= 32768 for up to 18 rows; for larger batches m <= 4096,
+ *             when one CTA orders each row's selection (k <= 16384; there the grid-wide repair kernel takes the
+ *             pass, as long as fewer than eight rows of the call failed).  Which kernel takes the pass follows from
+ *             who orders the selection: the refine kernel's clusters where one CTA orders a row (k <= 16384; from
+ *             one to 18 rows the library hands selections above 8192 -- one bf16 row: above 3072 -- to the whole
+ *             grid where that measured faster, by element type and row length), the one kernel after the filter
+ *             for a grid-ordered selection from a single row and for the BatchTopK entry points, the repair kernel
+ *             for grid-ordered selections from 2 to 18 rows.  Grid-ordered selections from more rows and anything
+ *             else go straight to the exact selection.
  * Both bounds are binomial tail bounds valid for the stratified sampler the
  * library uses (one uniform draw from each of m equal strata of the row).
  */

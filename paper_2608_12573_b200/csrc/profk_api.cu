@@ -31,18 +31,37 @@ constexpr int FILTER_THREADS = PROFK_FILTER_THREADS;
 constexpr int FILTER_UNROLL = PROFK_FILTER_UNROLL;
 constexpr uint32_t SORT_CAP_MAX = 16384;         // largest k the single-CTA refine orders in shared memory
 // Selections the whole grid refines (refine_large_kernel) instead of one CTA per row: beyond the single-CTA limit, and
-// from 8193 on (a single bf16 row: from 3073 on) when there are at most LARGE_FEW_ROWS rows -- one CTA takes 100-280 us over
-// 12000-16384 records of a long row (bf16, whose equal keys send the selection through the index digits, worst), the
-// grid 80-100; with many rows the CTAs work side by side and win.  Since the grid-wide path starts from the filter's
-// histogram a bf16 row is better off there from a few thousand on (2^28 bf16: k = 4096 137 -> 118 us, k = 8192
-// 245 -> 114; 2^26: 58 -> 56, 106 -> 57; k = 2048 still 103 against 118); fp32 rows are not (k = 8192: 186 against 193).
+// below it where that measured faster.  One CTA takes 100-280 us over 12000-16384 records (bf16, whose equal keys send
+// the selection through the index digits, worst), the CTAs of several rows side by side; the grid takes 30-40 us per
+// row, one row after the other, behind two launches more.
+//   one row: from k = 8193 on; bf16 from 3073 on, since the grid-wide path is then one launch that starts from the
+//     filter's histogram (2^28 bf16: k = 4096 137 -> 118 us, k = 8192 245 -> 114; 2^26: 58 -> 56, 106 -> 57; k = 2048
+//     still 103 against 118; fp32 k = 8192: 186 against 193).
+//   2 to 18 rows, k > 8192: bf16 (5 rows of 2^22, k = 16384: 222 -> 86 us; 18 rows of 2^26: 1048 -> 555), except
+//     more than 8 rows shorter than 2^24 up to k = 10240 (16 rows of 2^22, k = 8193: 119 through one CTA each, 159
+//     through the grid); fp32 for rows of 2^26 and more, and of 2^24 and more from k = 10241 on (18 rows of 2^24,
+//     k = 16384: 472 -> 365; 2 rows of 2^22, k = 8500: 42 through one CTA each, 71 through the grid).
+//   more rows: the CTAs work side by side and win.
 constexpr int64_t LARGE_FEW_ROWS = 4;
+constexpr int64_t LARGE_SOME_ROWS = 18;
 constexpr int64_t LARGE_FEW_K = 8192;
 constexpr int64_t LARGE_FEW_K_HALF = 3072;
-inline bool large_selection(int64_t rows, int64_t k, size_t elem_size) {
-    // (the lower switch of bf16 is for a single row: only there the grid-wide path is one launch that starts from the
-    // filter's histogram; two rows of 2^22 bf16 with k = 4096 took 68 us through it against 34)
+constexpr int64_t LARGE_SOME_K = 10240;
+inline bool large_selection(int64_t rows, int64_t k, size_t elem_size, int64_t N) {
+    if (k > (int64_t)SORT_CAP_MAX) return true;
+    if (rows == 1) return k > (elem_size == 2 ? LARGE_FEW_K_HALF : LARGE_FEW_K);
+    if (rows > LARGE_SOME_ROWS || k <= LARGE_FEW_K) return false;
+    if (elem_size == 2) return rows <= 8 || N >= (1LL << 24) || k > LARGE_SOME_K;
+    return N >= (1LL << 26) || (N >= (1LL << 24) && k > LARGE_SOME_K);
+}
+// The rule without the row length, as the allocation-free entry point applies it (its scratch holds the grid-wide
+// layout of at most LARGE_FEW_ROWS rows).
+inline bool large_selection_few(int64_t rows, int64_t k, size_t elem_size) {
     return k > (int64_t)SORT_CAP_MAX || (rows <= LARGE_FEW_ROWS && k > LARGE_FEW_K) || (rows == 1 && elem_size == 2 && k > LARGE_FEW_K_HALF);
+}
+// Whether some element type and row length send (rows, k) through the grid-wide layout.
+inline bool large_possible(int64_t rows, int64_t k) {
+    return k > (int64_t)SORT_CAP_MAX || (rows == 1 && k > LARGE_FEW_K_HALF) || (rows <= LARGE_SOME_ROWS && k > LARGE_FEW_K);
 }
 constexpr unsigned FB_MAX_CTAS = 256;             // most CTAs of the grid-wide exact selection (its per-CTA scratch is sized for them)
 // Samples above this size are gathered by a kernel over all SMs (65536: 2^26, k = 16, S = 40529 took 49.7 us, not 47.0).
@@ -117,7 +136,7 @@ WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k, bool large) {
     const bool fbp = rows > XS_MAX_ROWS && !large;
     // (up to GATHER_MAX_ROWS rows: room for the largest sample; up to XS_MAX_ROWS rows: for samples up to KEPT_SAMPLE_MAX,
     // larger batches: up to KEPT_SAMPLE_BATCH_MAX -- kept for the second filtering pass of a row that fails the count check)
-    const size_t keys_per_row = rows <= GATHER_MAX_ROWS ? (size_t)M_MAX : xs ? (size_t)KEPT_SAMPLE_MAX : !large ? (size_t)KEPT_SAMPLE_BATCH_MAX : 0;
+    const size_t keys_per_row = rows <= GATHER_MAX_ROWS ? (size_t)M_MAX : rows <= XS_MAX_ROWS ? (size_t)KEPT_SAMPLE_MAX : !large ? (size_t)KEPT_SAMPLE_BATCH_MAX : 0;
     l.off_fb_counters = align_up(l.off_keys + (size_t)rows * keys_per_row * sizeof(uint32_t), 256);
     l.off_fb_records = align_up(l.off_fb_counters + (fbp ? FB_MAX_CTAS * sizeof(uint32_t) : 0), 256);
     // counters of the partitioned append (large selections only), each in a 256-byte line of its own
@@ -511,7 +530,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         std::lock_guard<std::mutex> lock(g_mutex);
         ws = g_workspace[dev];
     }
-    const bool large = large_selection(rows, k, sizeof(T));
+    const bool large = g_ws_override_ptr ? large_selection_few(rows, k, sizeof(T)) : large_selection(rows, k, sizeof(T), N);
     const WsLayout lay = ws_layout(rows, capacity, k, large);
     if (!ws.ptr || ws.bytes < lay.total) return PROFK_EWORKSPACE;
     const uint64_t row_stride = row_stride_for(capacity, large);
@@ -546,9 +565,9 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
 
     // A second filtering pass for rows that fail the count check (plan->r_tight / r_loose) needs the sample's keys: they
     // are kept when the workspace has room for them and a kernel that takes that pass does the repair: the refine
-    // kernel's clusters, the grid-wide repair kernel (large selections: up to four rows), or the fused kernel of a large
-    // selection from a single row.
-    const bool keep_keys = (!large || rows <= GATHER_MAX_ROWS) && plan->mode == 0 && (plan->r_tight > 0 || plan->r_loose > 0) &&
+    // kernel's clusters, the grid-wide repair kernel (large selections: up to XS_MAX_ROWS rows), or the fused kernel of a
+    // large selection from a single row.
+    const bool keep_keys = (!large || rows <= XS_MAX_ROWS) && plan->mode == 0 && (plan->r_tight > 0 || plan->r_loose > 0) &&
                            (rows <= GATHER_MAX_ROWS || plan->m <= (rows <= XS_MAX_ROWS ? KEPT_SAMPLE_MAX : KEPT_SAMPLE_BATCH_MAX));
     SampleInfo sample = {};
     if (keep_keys) {
@@ -878,7 +897,7 @@ int refine_gathered(const uint64_t* records, const uint32_t* states, const int64
         std::lock_guard<std::mutex> lock(g_mutex);
         ws = g_workspace[dev];
     }
-    const bool large = large_selection(1, k, sizeof(T));
+    const bool large = large_selection(1, k, sizeof(T), 0);
     const WsLayout lay = ws_layout(1, capacity, k, large);
     if (!ws.ptr || ws.bytes < lay.total) return PROFK_EWORKSPACE;
     const uint64_t row_stride = row_stride_for(capacity, large);
@@ -916,8 +935,11 @@ extern "C" {
 int profk_workspace_bytes(int64_t rows, int64_t capacity, int64_t k, size_t* bytes) {
     if (!bytes || rows < 1 || capacity < 1 || k < 1 || capacity < k || capacity > N_MAX || rows * capacity >= (1LL << 40))
         return PROFK_EINVAL;
-    // (enough for either element type: the two take the grid-wide layout from different k on)
-    *bytes = std::max(ws_layout(rows, capacity, k, large_selection(rows, k, 4)).total, ws_layout(rows, capacity, k, large_selection(rows, k, 2)).total);
+    // (enough for either element type and any row length: they take the grid-wide layout from different k on)
+    size_t need = 0;
+    if (k <= (int64_t)SORT_CAP_MAX) need = ws_layout(rows, capacity, k, false).total;
+    if (large_possible(rows, k)) need = std::max(need, ws_layout(rows, capacity, k, true).total);
+    *bytes = need;
     return PROFK_OK;
 }
 
@@ -1051,7 +1073,7 @@ int profk_topk_noalloc_f32(const float* in, int64_t rows, int64_t N, int64_t k, 
         }
     }
     if (rows * plan.capacity >= (1LL << 40)) return PROFK_EINVAL;
-    if (ws_layout(rows, plan.capacity, k, large_selection(rows, k, sizeof(float))).total > NOALLOC_SCRATCH_BYTES) return PROFK_ETOOLARGE;
+    if (ws_layout(rows, plan.capacity, k, large_selection_few(rows, k, sizeof(float))).total > NOALLOC_SCRATCH_BYTES) return PROFK_ETOOLARGE;
     g_ws_override_ptr = scratch;
     g_ws_override_bytes = NOALLOC_SCRATCH_BYTES;
     const int rc = topk_planned<float>(in, rows, N, k, &plan, seed, stream, out_vals, out_idx);

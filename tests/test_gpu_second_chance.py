@@ -230,3 +230,26 @@ def test_large_selections_from_a_few_rows_take_the_second_pass_in_the_repair_ker
     # a mix: one row's own capacity problem only (the others pass): a capacity between the rows' survivor counts
     pl = profk.Plan(m=m, r=1000, capacity=cap, k_accept=k, mode=0, r_tight=800)        # about 30.5 K survivors: all pass
     check(x, k, pl, seed=44, want_status=profk.ROW_OK)
+
+
+@pytest.mark.parametrize("dtype,n", [(torch.bfloat16, 500_009), (torch.float32, (1 << 24) + 5)])
+def test_large_selections_from_up_to_eighteen_rows_take_the_second_pass_when_the_sample_is_small(dtype, n):
+    """Five to eighteen rows whose k (above 8192) the grid refines -- bf16 at any row length, fp32 from 2^24 elements on:
+    the repair kernel takes the second pass when the sample has at most 32768 keys, the exact selection otherwise."""
+    rows, k, m = 6, 9000, 32768
+    x = workloads.normal(rows, n, seed=89, dtype=dtype)
+    per = n / m                                                               # survivors per sample rank
+    r, cap = int(30_000 / per) + 1, 22_000                                    # about 30 K survivors: too many
+    check(x, k, profk.Plan(m=m, r=r, capacity=cap, k_accept=k, mode=0, r_tight=int(15_000 / per) + 1), seed=50,
+          want_status=profk.ROW_OVERFLOW_REFILTERED)
+    check(x, k, profk.Plan(m=m, r=r, capacity=cap, k_accept=k, mode=0), seed=50, want_status=profk.ROW_OVERFLOW)
+    r = max(int(4_000 / per), 1)                                              # about 4 K survivors: too few
+    check(x, k, profk.Plan(m=m, r=r, capacity=cap, k_accept=k, mode=0, r_loose=int(15_000 / per) + 1), seed=51,
+          want_status=profk.ROW_RECALL_REFILTERED)
+    # 65536 keys are not kept: the exact selection answers
+    pl = profk.Plan(m=2 * m, r=2 * r, capacity=cap, k_accept=k, mode=0, r_loose=2 * int(15_000 / per) + 2)
+    v, i = profk.topk(x.cuda(), k, plan_override=pl, seed=52)
+    torch.cuda.synchronize()
+    ov, oi = o_topk.topk(workloads.as_numpy(x), k)
+    assert np.array_equal(i.cpu().numpy(), oi) and np.array_equal(bits(workloads.as_numpy(v)), bits(ov))
+    assert all(s[3] == profk.ROW_RECALL for s in profk.read_stats(rows))
