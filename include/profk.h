@@ -118,11 +118,11 @@ enum {
  *             when one CTA orders each row's selection (k <= 16384; there the grid-wide repair kernel takes the
  *             pass, as long as fewer than eight rows of the call failed).  Which kernel takes the pass follows from
  *             who orders the selection: the refine kernel's clusters where one CTA orders a row (k <= 16384; from
- *             one to 18 rows the library hands selections above 8192 -- one bf16 row: above 3072 -- to the whole
- *             grid where that measured faster, by element type and row length), the one kernel after the filter
- *             for a grid-ordered selection from a single row and for the BatchTopK entry points, the repair kernel
- *             for grid-ordered selections from 2 to 18 rows.  Grid-ordered selections from more rows and anything
- *             else go straight to the exact selection.
+ *             one to 18 rows the library hands selections above 4096 -- one row: above 8192, bf16 above 3072 --
+ *             to the whole grid where that measured faster, by element type, row count and row length), the one
+ *             kernel after the filter for a grid-ordered selection from 1 to 18 rows and for the BatchTopK entry
+ *             points.  Grid-ordered selections from more rows and anything else go straight to the exact
+ *             selection.
  * Both bounds are binomial tail bounds valid for the stratified sampler the
  * library uses (one uniform draw from each of m equal strata of the row).
  */

@@ -32,27 +32,39 @@ constexpr int FILTER_UNROLL = PROFK_FILTER_UNROLL;
 constexpr uint32_t SORT_CAP_MAX = 16384;         // largest k the single-CTA refine orders in shared memory
 // Selections the whole grid refines (refine_large_kernel) instead of one CTA per row: beyond the single-CTA limit, and
 // below it where that measured faster.  One CTA takes 100-280 us over 12000-16384 records (bf16, whose equal keys send
-// the selection through the index digits, worst), the CTAs of several rows side by side; the grid takes 30-40 us per
-// row, one row after the other, behind two launches more.
-//   one row: from k = 8193 on; bf16 from 3073 on, since the grid-wide path is then one launch that starts from the
-//     filter's histogram (2^28 bf16: k = 4096 137 -> 118 us, k = 8192 245 -> 114; 2^26: 58 -> 56, 106 -> 57; k = 2048
-//     still 103 against 118; fp32 k = 8192: 186 against 193).
-//   2 to 18 rows, k > 8192: bf16 (5 rows of 2^22, k = 16384: 222 -> 86 us; 18 rows of 2^26: 1048 -> 555), except
-//     more than 8 rows shorter than 2^24 up to k = 10240 (16 rows of 2^22, k = 8193: 119 through one CTA each, 159
-//     through the grid); fp32 for rows of 2^26 and more, and of 2^24 and more from k = 10241 on (18 rows of 2^24,
-//     k = 16384: 472 -> 365; 2 rows of 2^22, k = 8500: 42 through one CTA each, 71 through the grid).
+// the selection through the index digits, worst), the CTAs of several rows side by side; the grid takes 10-40 us per
+// row, in up to 18 groups side by side, and its launch costs 7-9 us more.
+//   one row: from k = 8193 on; bf16 from 3073 on, since the grid-wide path then starts from the filter's histogram
+//     (2^28 bf16: k = 4096 137 -> 118 us, k = 8192 245 -> 114; 2^26: 58 -> 56, 106 -> 57; k = 2048 still 103 against
+//     118; fp32 k = 8192: 186 against 193).
+//   2 to 18 rows: from the k of large_switch_k on, read off sweeps over rows x k x N (2^20 .. 2^26) of both paths: the
+//     longer the rows and the more of them, the earlier (8 fp32 rows of 2^24, k = 6000: 203 us through one CTA each, 178
+//     through the grid; of 2^22: 74 against 103; 4 bf16 rows of 2^26, k = 4500: 180 against 142; 2 of 2^20: 39 against 49).
 //   more rows: the CTAs work side by side and win.
 constexpr int64_t LARGE_FEW_ROWS = 4;
 constexpr int64_t LARGE_SOME_ROWS = 18;
 constexpr int64_t LARGE_FEW_K = 8192;
 constexpr int64_t LARGE_FEW_K_HALF = 3072;
-constexpr int64_t LARGE_SOME_K = 10240;
+constexpr int64_t LARGE_SOME_K_MIN = 4096;       // no call of 2 to 18 rows switches at or below this k
+// 2 to 18 rows: the largest k one CTA per row still orders.
+inline int64_t large_switch_k(int64_t rows, size_t elem_size, int64_t N) {
+    const int64_t never = (int64_t)SORT_CAP_MAX;
+    if (elem_size == 2) {
+        if (N >= (1LL << 26)) return LARGE_SOME_K_MIN;
+        if (N >= (1LL << 24)) return rows <= 4 ? 6144 : 7168;
+        return rows <= 4 ? 6656 : rows <= 8 ? 8192 : 10240;
+    }
+    if (N >= (1LL << 26)) return 6144;
+    if (N >= (1LL << 25)) return rows <= 3 ? 8192 : 6144;
+    if (N >= (1LL << 24)) return rows <= 4 ? 10240 : 6144;
+    if (N >= (1LL << 23)) return 13312;
+    return never;
+}
 inline bool large_selection(int64_t rows, int64_t k, size_t elem_size, int64_t N) {
     if (k > (int64_t)SORT_CAP_MAX) return true;
     if (rows == 1) return k > (elem_size == 2 ? LARGE_FEW_K_HALF : LARGE_FEW_K);
-    if (rows > LARGE_SOME_ROWS || k <= LARGE_FEW_K) return false;
-    if (elem_size == 2) return rows <= 8 || N >= (1LL << 24) || k > LARGE_SOME_K;
-    return N >= (1LL << 26) || (N >= (1LL << 24) && k > LARGE_SOME_K);
+    if (rows > LARGE_SOME_ROWS) return false;
+    return k > large_switch_k(rows, elem_size, N);
 }
 // The rule without the row length, as the allocation-free entry point applies it (its scratch holds the grid-wide
 // layout of at most LARGE_FEW_ROWS rows).
@@ -61,7 +73,7 @@ inline bool large_selection_few(int64_t rows, int64_t k, size_t elem_size) {
 }
 // Whether some element type and row length send (rows, k) through the grid-wide layout.
 inline bool large_possible(int64_t rows, int64_t k) {
-    return k > (int64_t)SORT_CAP_MAX || (rows == 1 && k > LARGE_FEW_K_HALF) || (rows <= LARGE_SOME_ROWS && k > LARGE_FEW_K);
+    return k > (int64_t)SORT_CAP_MAX || (rows == 1 && k > LARGE_FEW_K_HALF) || (rows <= LARGE_SOME_ROWS && k > LARGE_SOME_K_MIN);
 }
 constexpr unsigned FB_MAX_CTAS = 256;             // most CTAs of the grid-wide exact selection (its per-CTA scratch is sized for them)
 // Samples above this size are gathered by a kernel over all SMs (65536: 2^26, k = 16, S = 40529 took 49.7 us, not 47.0).
@@ -392,7 +404,7 @@ int launch_refine_large(const DeviceInfo& di, RowCtl* ctl, WsHeader* header, uin
     lp.hist_ready = hist_ready ? 1 : 0;
     lp.idx_bits = 32;                            // (N unknown: every bit of the index word may be used)
     if (N > 1) { lp.idx_bits = 1; while (((int64_t)1 << lp.idx_bits) < N) ++lp.idx_bits; }
-    lp.fused = fused_fb ? 1 : 0;
+    lp.fused = fused_fb ? (rows == 1 ? 1 : 2) : 0;
     if (fused_fb) lp.fb = *fused_fb; else lp.fb = FallbackParams<T>{};
     lp.ctl = ctl; lp.header = header; lp.buf = buf; lp.row_stride = row_pitch / 2; lp.bins = bins; lp.slots = slots;
     lp.parts = (phase == 0 && parts) ? FILTER_PARTS : 1u; lp.part_cap = part_cap; lp.part_counts = part_counts;
@@ -596,6 +608,9 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     // A large selection from a single row: the count check, the exact replacement of a row that fails it and the
     // ordering are one cooperative kernel (three launches otherwise, two of which do nothing when no row failed).
     const bool fused_large = large && rows == 1;
+    // ... and from a few rows (not in direct mode): the groups of the grid order the rows that passed, then the whole
+    // grid repairs and orders the rest -- the two cooperative launches saved cost 7-9 us each behind their predecessors.
+    const bool fused_some = large && rows > 1 && rows <= XS_MAX_ROWS && plan->mode == 0;
 
     // ... and when its filter is the deferring build, that counts the records it appends in the bins the ordering starts
     // from (cleared by the threshold kernels).
@@ -612,8 +627,8 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
 
         if (large) {
             rc = launch_refine_large<T>(di, ctl, header, buf, row_stride, bins, reinterpret_cast<unsigned long long*>(ghist), parts, part_cap, part_counts, rows,
-                                        capacity, k, plan->k_accept, 0, out_vals, out_idx, st, fused_large ? &fb : nullptr, true, N, hist);
-            if (fused_large) return rc;
+                                        capacity, k, plan->k_accept, 0, out_vals, out_idx, st, fused_large || fused_some ? &fb : nullptr, true, N, hist);
+            if (fused_large || fused_some) return rc;
         } else {
             // count check and refine; with clusters, also the exact selection of the rows that fail the check
             rc = launch_refine<T>(di, in, rows, N, ctl, header, buf, row_stride, capacity, k, plan->k_accept, false, csize, xs_records, xs_counters, out_vals, out_idx, st,

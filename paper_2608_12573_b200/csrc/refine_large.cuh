@@ -50,8 +50,11 @@ template <typename T> struct LargeParams {
     int use_pdl;
     // A single row (fused == 1; one group of CTAs): a row that fails the count check, or a row in direct mode, is replaced
     // inside this kernel by the grid-wide exact selection and ordered right away -- one launch instead of three.
+    // A few rows (fused == 2; phase 0, no direct mode): the groups order the rows that pass side by side; then the whole
+    // grid meets at one barrier and, if some row failed, takes the failed rows one after the other as a single group --
+    // second filtering pass or exact selection, then the ordering -- again in this one launch.
     int fused;
-    FallbackParams<T> fb;    // what that selection needs (fused == 1 only)
+    FallbackParams<T> fb;    // what that selection needs (fused != 0 only)
     int idx_bits;            // bits an index of the row occupies (1 .. 32)
     int hist_ready;          // 1 = (fused) the filter kernel counted the records it appended in the row's bins; the rest of
                              // the row's BIN_ROW_WORDS words are zero.  0 = nobody has touched them
@@ -87,17 +90,18 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
 
     // The grid works as p.groups groups of CTAs (one for a single row); a group takes rows group, group + groups, ...
     // one after the other, all its CTAs on one row, with a barrier of its own.
-    const unsigned nctas = gridDim.x / p.groups, group = blockIdx.x / nctas, cta = blockIdx.x % nctas;
+    // (not constants: the repair round of fused == 2 regroups the grid into one group)
+    unsigned ngroups = p.groups, nctas = gridDim.x / ngroups, group = blockIdx.x / nctas, cta = blockIdx.x % nctas;
     const unsigned tid = threadIdx.x;
-    const uint64_t gid = (uint64_t)cta * BT_THREADS + tid;           // thread index inside the group
-    const uint64_t gthreads = (uint64_t)nctas * BT_THREADS;
+    uint64_t gid = (uint64_t)cta * BT_THREADS + tid;                 // thread index inside the group
+    uint64_t gthreads = (uint64_t)nctas * BT_THREADS;
     unsigned long long* slot_max = p.slots + gridDim.x + group * nctas;
     uint32_t* bar_count = &p.header->group_bar[group][0];
     auto barrier = [&]() { return cta_group_barrier(bar_count, &p.header->error, nctas); };
 
     // A single row whose filter did not count: the bins are cleared here, before the wait for the filter kernel, and each
     // CTA reports in through the header's `done` word (zeroed by the call's first kernel, long finished).
-    bool clean_bins = p.fused && !p.hist_ready;
+    bool clean_bins = p.fused == 1 && !p.hist_ready;
     if (clean_bins) {
         for (uint64_t b = gid; b < BIN_ROW_WORDS; b += gthreads) p.bins[b] = 0;
         __threadfence();
@@ -107,7 +111,19 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
     pdl_launch_dependents();
     if (p.use_pdl) pdl_wait();
 
-    for (uint64_t row = group; row < p.rows; row += p.groups) {
+    for (int round = 0; round < 2; ++round) {
+    if (round == 1) {
+        // ---- fused == 2: the groups are through with the rows that passed; the whole grid, as one group, takes the rest ----
+        if (p.fused != 2) break;
+        if (!grid_barrier(p.header)) return;
+        if (__ldcg(&p.header->n_failed) == 0) break;
+        ngroups = 1; nctas = gridDim.x; group = 0; cta = blockIdx.x;
+        gid = (uint64_t)cta * BT_THREADS + tid;
+        gthreads = (uint64_t)nctas * BT_THREADS;
+        slot_max = p.slots + gridDim.x;
+        bar_count = &p.header->bar_count;          // (the counter of grid_barrier: the same members from here on)
+    }
+    for (uint64_t row = group; row < p.rows; row += ngroups) {
         // ---- is this row for this launch?  (the decision is the same in every CTA) ----
         const RowCtl ctl = p.ctl[row];
         uint32_t n;
@@ -116,34 +132,43 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         bool from_filter = false;        // the buffer is what a filtering pass with threshold tau_key left
         bool status_ok = false;          // ... the first one
         if (p.phase == 0) {
-            uint32_t R = ctl.count;
-            bool part_full = false;
-            if (p.parts > 1) {                   // partitioned append: the row's count is the sum of its parts'
-                nparts = FILTER_PARTS;
-                uint64_t sum = 0;
+            uint32_t status;
+            bool direct = false;
+            if (round == 0) {
+                uint32_t R = ctl.count;
+                bool part_full = false;
+                if (p.parts > 1) {                   // partitioned append: the row's count is the sum of its parts'
+                    nparts = FILTER_PARTS;
+                    uint64_t sum = 0;
 #pragma unroll
-                for (int j = 0; j < (int)FILTER_PARTS; ++j) {
-                    const uint32_t c = p.part_counts[(row * FILTER_PARTS + j) * FILTER_PART_STRIDE];
-                    part_full |= c > p.part_cap;
-                    pcount[j] = c < p.part_cap ? c : p.part_cap;
-                    sum += c;
+                    for (int j = 0; j < (int)FILTER_PARTS; ++j) {
+                        const uint32_t c = p.part_counts[(row * FILTER_PARTS + j) * FILTER_PART_STRIDE];
+                        part_full |= c > p.part_cap;
+                        pcount[j] = c < p.part_cap ? c : p.part_cap;
+                        sum += c;
+                    }
+                    R = sum > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)sum;
+                } else {
+                    pcount[0] = R;
                 }
-                R = sum > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)sum;
+                direct = ctl.status == ROW_DIRECT;                     // marked by the initialisation kernel: no filter ran
+                status = direct ? ROW_DIRECT : (R > p.capacity || part_full) ? ROW_OVERFLOW : R < p.k_accept ? ROW_RECALL : ROW_OK;
+                if (cta == 0 && tid == 0 && !direct) {
+                    if (p.parts > 1) p.ctl[row].count = part_full && R <= p.capacity ? p.capacity + 1 : R;   // what the statistics report
+                    p.ctl[row].status = status;
+                    p.ctl[row].n_final = status ? p.k : R;
+                    if (status) atomicAdd(&p.header->n_failed, 1u);
+                }
+                n = R;
+                from_filter = status_ok = status == ROW_OK;
             } else {
-                pcount[0] = R;
+                // (the status another group's CTA wrote before the barrier: read past this SM's L1)
+                status = __ldcg(&p.ctl[row].status);
+                if (status == ROW_OK) continue;                    // ordered in the first round
+                n = 0;
             }
-            const bool direct = ctl.status == ROW_DIRECT;          // marked by the initialisation kernel: no filter ran
-            const uint32_t status = direct ? ROW_DIRECT : (R > p.capacity || part_full) ? ROW_OVERFLOW : R < p.k_accept ? ROW_RECALL : ROW_OK;
-            if (cta == 0 && tid == 0 && !direct) {
-                if (p.parts > 1) p.ctl[row].count = part_full && R <= p.capacity ? p.capacity + 1 : R;   // what the statistics report
-                p.ctl[row].status = status;
-                p.ctl[row].n_final = status ? p.k : R;
-                if (status) atomicAdd(&p.header->n_failed, 1u);
-            }
-            n = R;
-            from_filter = status_ok = status == ROW_OK;
             if (status != ROW_OK) {
-                if (!p.fused) continue;          // the exact-selection kernel and the second phase take this row
+                if (p.fused == 0 || (p.fused == 2 && round == 0)) continue;   // the exact-selection kernel and the second phase, or the second round, take this row
                 // first a second filtering pass with the plan's tighter / looser sample rank, if it names one (the tile in
                 // shared memory, unused so far, holds that pass's selection state) ...
                 uint32_t R2 = 0, key2 = 0;
@@ -393,6 +418,7 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
         }
 
         for (uint64_t j = gid; j < kk; j += gthreads) write_output(p.out_vals, p.out_idx, p.k, row, (uint32_t)j, __ldcg(&G[j]));
+    }
     }
 }
 

@@ -253,3 +253,24 @@ def test_large_selections_from_up_to_eighteen_rows_take_the_second_pass_when_the
     ov, oi = o_topk.topk(workloads.as_numpy(x), k)
     assert np.array_equal(i.cpu().numpy(), oi) and np.array_equal(bits(workloads.as_numpy(v)), bits(ov))
     assert all(s[3] == profk.ROW_RECALL for s in profk.read_stats(rows))
+
+
+def test_a_few_rows_of_a_grid_ordered_call_fail_and_the_others_pass():
+    """Seven rows, k above what one CTA orders for them: the groups of the grid order the rows that pass, then the whole
+    grid repairs the others -- some by the second pass, one (no room even for the tighter rank) exactly."""
+    rows, n, k, m = 7, 400_003, 9000, 32768
+    x = workloads.normal(rows, n, seed=90, dtype=torch.bfloat16)
+    xn = workloads.as_numpy(x)
+    per = n / m
+    r = int(20_000 / per) + 1
+    tight = int(14_000 / per) + 1
+    first = sorted(o_stages.run_row(xn[i], k, m, r, n, k, seed=60, row=i, composite=True).survivors for i in range(rows))
+    cap = (first[2] + first[3]) // 2                                          # three rows fit, four overflow
+    assert first[2] < cap < first[3]
+    pl = profk.Plan(m=m, r=r, capacity=cap, k_accept=k, mode=0, r_tight=tight)
+    check(x, k, pl, seed=60)
+    got = sorted(s[3] for s in profk.read_stats(rows))
+    assert got == [profk.ROW_OK] * 3 + [profk.ROW_OVERFLOW_REFILTERED] * 4
+    # no tighter rank named: the four rows are selected exactly
+    check(x, k, profk.Plan(m=m, r=r, capacity=cap, k_accept=k, mode=0), seed=60)
+    assert sorted(s[3] for s in profk.read_stats(rows)) == [profk.ROW_OK] * 3 + [profk.ROW_OVERFLOW] * 4
