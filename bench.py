@@ -40,6 +40,8 @@ CONFIGS = {
     # the shape of Section 5's sparse-autoencoder measurement: N = 50,331,648 flattened activations, K = 131,072
     "cfg4_sae_f32": (1, 50331648, "f32", "relu_gaussian", 3, 131072, 1e-3, 1.0),
     "cfg4_sae_bf16": (1, 50331648, "bf16", "relu_gaussian", 3, 131072, 1e-3, 1.0),
+    # a few rows whose selection the whole grid orders (one cooperative launch after the filter): for launch lists
+    "rows4_bf16_k8192": (4, 1 << 24, "bf16", "normal", 9, 8192, 1e-3, 1.0),
     "cfg5_cauchy_k64": (1, 1 << 30, "f32", "cauchy", 4, 64, 1e-3, 1.0),
     "cfg5_cauchy_k65536": (1, 1 << 30, "f32", "cauchy", 4, 65536, 1e-3, 1.0),
     "cfg5_pareto_k1": (1, 1 << 30, "f32", "pareto", 5, 1, 1e-3, 1.0),
