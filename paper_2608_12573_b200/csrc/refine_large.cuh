@@ -320,27 +320,36 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
             if (tid < BIN_COARSE) s_coarse[tid] = incl - c;              // records in the coarse bins before this one
             __syncthreads();
         }
-        constexpr int SEG_AHEAD = 4;                                     // counts loaded ahead: a CTA of a full grid has at most four coarse bins
-        uint32_t ahead[SEG_AHEAD];
+        // (two coarse bins a round, one per half of the CTA; the counts of the first two rounds are loaded ahead: a CTA
+        // of a full grid has at most four coarse bins)
+        constexpr int SEG_PER_ROUND = BT_THREADS / BIN_PER_COARSE;
+        constexpr int ROUNDS_AHEAD = 2;
+        static_assert(SEG_PER_ROUND == 2, "a round of the scan covers two coarse bins");
+        const uint32_t half = tid / BIN_PER_COARSE, fine = tid % BIN_PER_COARSE;
+        uint32_t ahead[ROUNDS_AHEAD];
 #pragma unroll
-        for (int a = 0; a < SEG_AHEAD; ++a) {
-            const uint32_t seg = cta + a * nctas;
-            ahead[a] = seg < BIN_COARSE && tid < BIN_PER_COARSE ? __ldcg(&bins[seg * BIN_PER_COARSE + tid]) : 0u;
+        for (int a = 0; a < ROUNDS_AHEAD; ++a) {
+            const uint32_t seg = cta + (a * SEG_PER_ROUND + half) * nctas;
+            ahead[a] = seg < BIN_COARSE ? __ldcg(&bins[seg * BIN_PER_COARSE + fine]) : 0u;
         }
         int turn = 0;
-        for (uint32_t seg = cta; seg < BIN_COARSE; seg += nctas, ++turn) {
-            const uint32_t b = seg * BIN_PER_COARSE + tid;
+        for (uint32_t seg0 = cta; seg0 < BIN_COARSE; seg0 += SEG_PER_ROUND * nctas, ++turn) {
+            const uint32_t seg = seg0 + half * nctas;
+            const uint32_t b = seg * BIN_PER_COARSE + fine;
             uint32_t c = 0;
-            if (turn < SEG_AHEAD) {
+            if (turn < ROUNDS_AHEAD) {
 #pragma unroll
-                for (int a = 0; a < SEG_AHEAD; ++a)
+                for (int a = 0; a < ROUNDS_AHEAD; ++a)
                     if (a == turn) c = ahead[a];
-            } else if (tid < BIN_PER_COARSE) {
+            } else if (seg < BIN_COARSE) {
                 c = __ldcg(&bins[b]);
             }
             __syncthreads();                                             // s_warp of the round before
-            const uint32_t before = s_coarse[seg] + block_inclusive_scan(c, s_warp) - c;
-            if (tid < BIN_PER_COARSE) {
+            // records of this round's first coarse bin: they precede the second half's bins in the block-wide scan
+            const uint32_t first_total = seg0 + 1 < BIN_COARSE ? s_coarse[seg0 + 1] - s_coarse[seg0] : 0u;
+            const uint32_t excl = block_inclusive_scan(c, s_warp) - c;
+            if (seg < BIN_COARSE) {
+                const uint32_t before = s_coarse[seg] + excl - (half ? first_total : 0u);
                 if (before < kk && c > LG_CROWDED) atomicOr(&flags[0], 1u);
                 bins[b] = before;                                        // first position; the scatter advances it to the end
             }
