@@ -114,7 +114,7 @@ enum {
  *             with the same check k <= R <= M -- one more read of the row at streaming speed -- and only a row
  *             that fails again is selected exactly.  The ranks aim midway between k and M:
  *             r_tight = floor(r (k + M) / (2 M)), r_loose = r + ceil((M - k) m / (2 N)).  Used when the sample's keys
- *             are kept: any sample for up to four rows, m <= 32768 for up to 18 rows; for larger batches m <= 4096,
+ *             are kept: any sample for up to four rows, m <= 131072 for up to 18 rows; for larger batches m <= 4096,
  *             when one CTA orders each row's selection (k <= 16384; there the grid-wide repair kernel takes the
  *             pass, as long as fewer than eight rows of the call failed).  Which kernel takes the pass follows from
  *             who orders the selection: the refine kernel's clusters where one CTA orders a row (k <= 16384; from
@@ -363,8 +363,11 @@ int profk_refine_gathered_bf16(const uint64_t* records, const uint32_t* states, 
  * pool that is itself inside an allocation, a real-time or plug-in context that was handed
  * its buffers up front, a host that has already given all device memory to another
  * allocator -- and still needs a top-k of buffers it already owns.
- *   - Limit: the workspace the shape needs (profk_workspace_bytes for rows, the plan's
- *     capacity and k) must fit 16 MiB; roughly rows * capacity <= 2,000,000 records, e.g.
+ *   - Limit: the workspace the call lays out in the array (never more than profk_workspace_bytes
+ *     for rows, the plan's capacity and k; this entry point keeps samples of 5 to 18 rows for the
+ *     second filtering pass up to 32768 keys only, and hands selections from 2 to 4 rows to the
+ *     whole grid from k = 8193 on whatever the rows' length) must fit 16 MiB; roughly
+ *     rows * capacity <= 2,000,000 records, e.g.
  *     one row of any length up to the library limit with small k, or 512 rows of 2^20
  *     elements with k = 32.  Anything larger returns PROFK_ETOOLARGE and does nothing.
  *   - Every GPU that loads the library holds the 16 MiB until the process exits.

@@ -86,7 +86,8 @@ constexpr unsigned REFINE_CLUSTER_THREADS = 512;   // fewest threads of a refine
 constexpr size_t REFINE_SMEM_MAX = 160 * 1024;   // dynamic shared memory the refine kernel may ask for (it has ~41 KB static)
 constexpr int64_t N_MAX = 4278190080LL;          // 2^32 - 2^24
 constexpr int64_t M_MAX = 262144;                // largest sample the cluster select holds (8 CTAs x 32768 keys)
-constexpr int64_t KEPT_SAMPLE_MAX = 32768;       // largest sample whose keys are kept for a second filtering pass when there are more than GATHER_MAX_ROWS rows
+constexpr int64_t KEPT_SAMPLE_MAX = 131072;      // largest sample whose keys are kept for a second filtering pass when there are more than GATHER_MAX_ROWS rows
+constexpr int64_t KEPT_SAMPLE_NOALLOC_MAX = 32768;   // ... in the scratch of the allocation-free entry point
 constexpr int64_t KEPT_SAMPLE_BATCH_MAX = 4096;  // the same for batches of more than XS_MAX_ROWS rows
 
 thread_local int g_launches = 0;
@@ -128,7 +129,7 @@ uint64_t row_stride_for(int64_t capacity, bool large) {
 
 // `large` = the layout of large selections (bins, partitioned append counters, doubled row pitch): whenever
 // large_selection(rows, k) says so, and always for the flattened BatchTopK calls, whose select works on the bins.
-WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k, bool large) {
+WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k, bool large, int64_t kept_sample_max = KEPT_SAMPLE_MAX) {
     WsLayout l;
     l.off_header = 0;
     l.off_ghist = sizeof(WsHeader);
@@ -148,7 +149,7 @@ WsLayout ws_layout(int64_t rows, int64_t capacity, int64_t k, bool large) {
     const bool fbp = rows > XS_MAX_ROWS && !large;
     // (up to GATHER_MAX_ROWS rows: room for the largest sample; up to XS_MAX_ROWS rows: for samples up to KEPT_SAMPLE_MAX,
     // larger batches: up to KEPT_SAMPLE_BATCH_MAX -- kept for the second filtering pass of a row that fails the count check)
-    const size_t keys_per_row = rows <= GATHER_MAX_ROWS ? (size_t)M_MAX : rows <= XS_MAX_ROWS ? (size_t)KEPT_SAMPLE_MAX : !large ? (size_t)KEPT_SAMPLE_BATCH_MAX : 0;
+    const size_t keys_per_row = rows <= GATHER_MAX_ROWS ? (size_t)M_MAX : rows <= XS_MAX_ROWS ? (size_t)kept_sample_max : !large ? (size_t)KEPT_SAMPLE_BATCH_MAX : 0;
     l.off_fb_counters = align_up(l.off_keys + (size_t)rows * keys_per_row * sizeof(uint32_t), 256);
     l.off_fb_records = align_up(l.off_fb_counters + (fbp ? FB_MAX_CTAS * sizeof(uint32_t) : 0), 256);
     // counters of the partitioned append (large selections only), each in a 256-byte line of its own
@@ -543,7 +544,8 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
         ws = g_workspace[dev];
     }
     const bool large = g_ws_override_ptr ? large_selection_few(rows, k, sizeof(T)) : large_selection(rows, k, sizeof(T), N);
-    const WsLayout lay = ws_layout(rows, capacity, k, large);
+    const int64_t kept_sample_max = g_ws_override_ptr ? KEPT_SAMPLE_NOALLOC_MAX : KEPT_SAMPLE_MAX;
+    const WsLayout lay = ws_layout(rows, capacity, k, large, kept_sample_max);
     if (!ws.ptr || ws.bytes < lay.total) return PROFK_EWORKSPACE;
     const uint64_t row_stride = row_stride_for(capacity, large);
     unsigned char* base = static_cast<unsigned char*>(ws.ptr);
@@ -580,7 +582,7 @@ int topk_planned(const T* in, int64_t rows, int64_t N, int64_t k, const profk_pl
     // kernel's clusters, the grid-wide repair kernel (large selections: up to XS_MAX_ROWS rows), or the fused kernel of a
     // large selection from a single row.
     const bool keep_keys = (!large || rows <= XS_MAX_ROWS) && plan->mode == 0 && (plan->r_tight > 0 || plan->r_loose > 0) &&
-                           (rows <= GATHER_MAX_ROWS || plan->m <= (rows <= XS_MAX_ROWS ? KEPT_SAMPLE_MAX : KEPT_SAMPLE_BATCH_MAX));
+                           (rows <= GATHER_MAX_ROWS || plan->m <= (rows <= XS_MAX_ROWS ? kept_sample_max : KEPT_SAMPLE_BATCH_MAX));
     SampleInfo sample = {};
     if (keep_keys) {
         sample.keys = keys_scratch; sample.S = (uint32_t)plan->m; sample.seed = seed;
@@ -1088,7 +1090,7 @@ int profk_topk_noalloc_f32(const float* in, int64_t rows, int64_t N, int64_t k, 
         }
     }
     if (rows * plan.capacity >= (1LL << 40)) return PROFK_EINVAL;
-    if (ws_layout(rows, plan.capacity, k, large_selection_few(rows, k, sizeof(float))).total > NOALLOC_SCRATCH_BYTES) return PROFK_ETOOLARGE;
+    if (ws_layout(rows, plan.capacity, k, large_selection_few(rows, k, sizeof(float)), KEPT_SAMPLE_NOALLOC_MAX).total > NOALLOC_SCRATCH_BYTES) return PROFK_ETOOLARGE;
     g_ws_override_ptr = scratch;
     g_ws_override_bytes = NOALLOC_SCRATCH_BYTES;
     const int rc = topk_planned<float>(in, rows, N, k, &plan, seed, stream, out_vals, out_idx);

@@ -92,12 +92,12 @@ def test_ties_and_special_values_in_the_second_pass():
             check(x, k, profk.Plan(m=65536, r=1, capacity=20_000, k_accept=k, mode=0, r_loose=200, tie_rule=rule), seed=5)
 
 
-def test_the_librarys_own_plan_names_the_ranks_and_larger_samples_of_many_rows_skip_them():
+def test_the_librarys_own_plan_names_the_ranks_and_the_largest_samples_of_many_rows_skip_them():
     pl = profk.plan(1 << 26, 256, 1e-4)
     assert 0 < pl.r_tight < pl.r < pl.r_loose
-    # more than four rows and a sample above 32768: the keys are not kept, the exact selection answers at once
+    # more than four rows and a sample above 131072: the keys are not kept, the exact selection answers at once
     x = workloads.normal(6, 1 << 20, seed=85)
-    pl = profk.Plan(m=65536, r=640, capacity=8000, k_accept=64, mode=0, r_tight=320)
+    pl = profk.Plan(m=262144, r=2560, capacity=8000, k_accept=64, mode=0, r_tight=1280)
     v, i = profk.topk(x.cuda(), 64, plan_override=pl, seed=6)
     torch.cuda.synchronize()
     ov, oi = o_topk.topk(workloads.as_numpy(x), 64)
@@ -235,7 +235,7 @@ def test_large_selections_from_a_few_rows_take_the_second_pass_in_the_repair_ker
 @pytest.mark.parametrize("dtype,n", [(torch.bfloat16, 500_009), (torch.float32, (1 << 24) + 5)])
 def test_large_selections_from_up_to_eighteen_rows_take_the_second_pass_when_the_sample_is_small(dtype, n):
     """Five to eighteen rows whose k (above 8192) the grid refines -- bf16 at any row length, fp32 from 2^24 elements on:
-    the repair kernel takes the second pass when the sample has at most 32768 keys, the exact selection otherwise."""
+    the second pass is taken when the sample has at most 131072 keys, the exact selection otherwise."""
     rows, k, m = 6, 9000, 32768
     x = workloads.normal(rows, n, seed=89, dtype=dtype)
     per = n / m                                                               # survivors per sample rank
@@ -246,8 +246,8 @@ def test_large_selections_from_up_to_eighteen_rows_take_the_second_pass_when_the
     r = max(int(4_000 / per), 1)                                              # about 4 K survivors: too few
     check(x, k, profk.Plan(m=m, r=r, capacity=cap, k_accept=k, mode=0, r_loose=int(15_000 / per) + 1), seed=51,
           want_status=profk.ROW_RECALL_REFILTERED)
-    # 65536 keys are not kept: the exact selection answers
-    pl = profk.Plan(m=2 * m, r=2 * r, capacity=cap, k_accept=k, mode=0, r_loose=2 * int(15_000 / per) + 2)
+    # 262144 keys are not kept: the exact selection answers
+    pl = profk.Plan(m=8 * m, r=8 * r, capacity=cap, k_accept=k, mode=0, r_loose=8 * int(15_000 / per) + 8)
     v, i = profk.topk(x.cuda(), k, plan_override=pl, seed=52)
     torch.cuda.synchronize()
     ov, oi = o_topk.topk(workloads.as_numpy(x), k)
@@ -274,3 +274,12 @@ def test_a_few_rows_of_a_grid_ordered_call_fail_and_the_others_pass():
     # no tighter rank named: the four rows are selected exactly
     check(x, k, profk.Plan(m=m, r=r, capacity=cap, k_accept=k, mode=0), seed=60)
     assert sorted(s[3] for s in profk.read_stats(rows)) == [profk.ROW_OK] * 3 + [profk.ROW_OVERFLOW] * 4
+
+
+def test_twelve_long_rows_with_the_largest_kept_sample():
+    """12 rows of 2^22 under a 131072-key sample: one CTA orders each row, its clusters take the second pass."""
+    rows, n, k, m = 12, 1 << 22, 256, 131072
+    x = workloads.normal(rows, n, seed=91)
+    per = n / m                                                               # 32 survivors per sample rank
+    check(x, k, profk.Plan(m=m, r=200, capacity=4000, k_accept=k, mode=0, r_tight=60), seed=70, want_status=profk.ROW_OVERFLOW_REFILTERED)
+    check(x, k, profk.Plan(m=m, r=2, capacity=4000, k_accept=k, mode=0, r_loose=40), seed=71, want_status=profk.ROW_RECALL_REFILTERED)
