@@ -50,7 +50,7 @@ template <typename T> struct FilterParams {
     // Partitioned append (the PARTS build of the kernel only).  With very many survivors the single counter of a
     // row becomes the bottleneck -- atomics on one address retire about 2 ns apart, 164 K of them are a quarter of
     // a 2^30-element scan -- so the row's buffer is cut into FILTER_PARTS equal parts, each with a counter in a
-    // cache line of its own, and a CTA appends to part blockIdx.x mod FILTER_PARTS.
+    // cache line of its own, and the survivors of a tile go to part (tile index in the row) mod FILTER_PARTS.
     uint32_t part_cap;       // records per part
     uint32_t* part_counts;   // row r, part j: part_counts[(r * FILTER_PARTS + j) * FILTER_PART_STRIDE] (zeroed)
     // Threshold records written by the threshold kernel (null = take `tau`, a value alone): row r's is {bits of tau,
@@ -247,7 +247,9 @@ __device__ __forceinline__ uint32_t filter_slow_path_direct(const FilterParams<T
     uint64_t* dst = p.buf + (uint64_t)row * p.buf_stride;
     uint32_t cap = p.capacity;
     if (PARTS) {
-        const uint32_t part = blockIdx.x % FILTER_PARTS;
+        // (the part follows the tile, not the CTA: every part gets an eighth of the row's tiles whoever scans them --
+        // with the tiles dealt from the counter, a few CTAs take most of a late row and their parts overflowed)
+        const uint32_t part = (uint32_t)(qbase / ((uint64_t)THREADS * UNROLL)) % FILTER_PARTS;
         counter = p.part_counts + ((uint64_t)row * FILTER_PARTS + part) * FILTER_PART_STRIDE;
         dst += (uint64_t)part * p.part_cap;
         cap = p.part_cap;

@@ -79,13 +79,82 @@ __device__ __forceinline__ void bitonic_tile_steps(uint64_t* tile, uint64_t base
     }
 }
 
+// Shared-memory state of the scan over the bins (refine_large_kernel).
+struct ScanShared {
+    uint32_t coarse[BIN_COARSE];     // records in the coarse bins before each one
+    uint32_t ccount[BIN_COARSE];     // records in each coarse bin
+    uint16_t listed[BIN_COARSE];     // the coarse bins that matter, in order
+    uint32_t nlisted;                // how many are listed
+    uint32_t scattered;              // positions the scatter fills: [0, scattered)
+};
+
+// The scan of one row's bins by one group of `nctas` CTAs (this one: `cta`); all BT_THREADS threads call it.  Every CTA
+// sums the coarse bins before each of its own and lists the coarse bins that matter -- not empty, and starting below
+// position kk: the fine bins of the others are never looked at, and their records stay where they are.  CTA c turns
+// the counts of the fine bins of the c-th, (c + nctas)-th, ... listed coarse bin into first positions (bins[b]) and
+// flags a crowded bin among them.  On return the lists are in shared memory for every thread of the block (the loop's
+// block-wide scans come after the last write to them).
+__device__ __noinline__ void scan_bins(uint32_t* bins, const uint32_t* coarse, uint32_t* flags, ScanShared& ss, uint32_t* s_warp,
+                                       unsigned cta, unsigned nctas, uint32_t kk) {
+    const unsigned tid = threadIdx.x;
+    {
+        const uint32_t c = tid < BIN_COARSE ? __ldcg(&coarse[tid]) : 0u;
+        const uint32_t incl = block_inclusive_scan(c, s_warp);
+        if (tid < BIN_COARSE) { ss.coarse[tid] = incl - c; ss.ccount[tid] = c; }
+        const bool listed = c != 0 && incl - c < kk;
+        if (tid == 0) ss.scattered = 0;
+        __syncthreads();
+        const uint32_t at = block_inclusive_scan(listed ? 1u : 0u, s_warp);
+        if (listed) { ss.listed[at - 1] = (uint16_t)tid; atomicMax(&ss.scattered, incl); }   // (incl: the end of the last listed one)
+        if (tid == BT_THREADS - 1) ss.nlisted = at;
+        __syncthreads();
+    }
+    // (two coarse bins a round, one per half of the CTA; the counts of the first two rounds are loaded ahead)
+    constexpr int SEG_PER_ROUND = BT_THREADS / BIN_PER_COARSE;
+    constexpr int ROUNDS_AHEAD = 2;
+    static_assert(SEG_PER_ROUND == 2, "a round of the scan covers two coarse bins");
+    const uint32_t nlisted = ss.nlisted;
+    const uint32_t half = tid / BIN_PER_COARSE, fine = tid % BIN_PER_COARSE;
+    uint32_t ahead[ROUNDS_AHEAD];
+#pragma unroll
+    for (int a = 0; a < ROUNDS_AHEAD; ++a) {
+        const uint32_t li = cta + (a * SEG_PER_ROUND + half) * nctas;
+        ahead[a] = li < nlisted ? __ldcg(&bins[(uint32_t)ss.listed[li] * BIN_PER_COARSE + fine]) : 0u;
+    }
+    int turn = 0;
+    for (uint32_t li0 = cta; li0 < nlisted; li0 += SEG_PER_ROUND * nctas, ++turn) {
+        const uint32_t li = li0 + half * nctas;
+        const bool mine = li < nlisted;
+        const uint32_t seg = mine ? ss.listed[li] : 0u;
+        const uint32_t b = seg * BIN_PER_COARSE + fine;
+        uint32_t c = 0;
+        if (turn < ROUNDS_AHEAD) {
+#pragma unroll
+            for (int a = 0; a < ROUNDS_AHEAD; ++a)
+                if (a == turn) c = ahead[a];
+        } else if (mine) {
+            c = __ldcg(&bins[b]);
+        }
+        __syncthreads();                                             // s_warp of the round before
+        // records of this round's first coarse bin: they precede the second half's bins in the block-wide scan
+        const uint32_t first_total = ss.ccount[ss.listed[li0]];
+        const uint32_t excl = block_inclusive_scan(c, s_warp) - c;
+        if (mine) {
+            const uint32_t before = ss.coarse[seg] + excl - (half ? first_total : 0u);
+            if (before < kk && c > LG_CROWDED) atomicOr(&flags[0], 1u);
+            bins[b] = before;                                        // first position; the scatter advances it to the end
+        }
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const LargeParams<T> p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint64_t* tile = reinterpret_cast<uint64_t*>(smem_raw);          // BT_TILE records
     __shared__ unsigned long long s_max[32];
     __shared__ uint32_t s_warp[32];
-    __shared__ uint32_t s_coarse[BIN_COARSE];
+    __shared__ ScanShared ss;
+    uint32_t* const s_coarse = ss.coarse;
     static_assert(BIN_COARSE <= BT_THREADS && BIN_PER_COARSE <= BT_THREADS, "one thread per coarse bin, then per fine bin of one coarse bin");
 
     // The grid works as p.groups groups of CTAs (one for a single row); a group takes rows group, group + groups, ...
@@ -312,61 +381,27 @@ __global__ void __launch_bounds__(BT_THREADS, 1) refine_large_kernel(const Large
             if (!barrier()) return;
         }
 
-        // scan: every CTA sums the coarse bins before each of its own; CTA c turns the counts of the fine bins of coarse
-        // bins c, c + nctas, ... into first positions
-        {
-            const uint32_t c = tid < BIN_COARSE ? __ldcg(&coarse[tid]) : 0u;
-            const uint32_t incl = block_inclusive_scan(c, s_warp);
-            if (tid < BIN_COARSE) s_coarse[tid] = incl - c;              // records in the coarse bins before this one
-            __syncthreads();
-        }
-        // (two coarse bins a round, one per half of the CTA; the counts of the first two rounds are loaded ahead: a CTA
-        // of a full grid has at most four coarse bins)
-        constexpr int SEG_PER_ROUND = BT_THREADS / BIN_PER_COARSE;
-        constexpr int ROUNDS_AHEAD = 2;
-        static_assert(SEG_PER_ROUND == 2, "a round of the scan covers two coarse bins");
-        const uint32_t half = tid / BIN_PER_COARSE, fine = tid % BIN_PER_COARSE;
-        uint32_t ahead[ROUNDS_AHEAD];
-#pragma unroll
-        for (int a = 0; a < ROUNDS_AHEAD; ++a) {
-            const uint32_t seg = cta + (a * SEG_PER_ROUND + half) * nctas;
-            ahead[a] = seg < BIN_COARSE ? __ldcg(&bins[seg * BIN_PER_COARSE + fine]) : 0u;
-        }
-        int turn = 0;
-        for (uint32_t seg0 = cta; seg0 < BIN_COARSE; seg0 += SEG_PER_ROUND * nctas, ++turn) {
-            const uint32_t seg = seg0 + half * nctas;
-            const uint32_t b = seg * BIN_PER_COARSE + fine;
-            uint32_t c = 0;
-            if (turn < ROUNDS_AHEAD) {
-#pragma unroll
-                for (int a = 0; a < ROUNDS_AHEAD; ++a)
-                    if (a == turn) c = ahead[a];
-            } else if (seg < BIN_COARSE) {
-                c = __ldcg(&bins[b]);
-            }
-            __syncthreads();                                             // s_warp of the round before
-            // records of this round's first coarse bin: they precede the second half's bins in the block-wide scan
-            const uint32_t first_total = seg0 + 1 < BIN_COARSE ? s_coarse[seg0 + 1] - s_coarse[seg0] : 0u;
-            const uint32_t excl = block_inclusive_scan(c, s_warp) - c;
-            if (seg < BIN_COARSE) {
-                const uint32_t before = s_coarse[seg] + excl - (half ? first_total : 0u);
-                if (before < kk && c > LG_CROWDED) atomicOr(&flags[0], 1u);
-                bins[b] = before;                                        // first position; the scatter advances it to the end
-            }
-        }
+        // scan (out of line: its registers are its own): the coarse bins' first positions, the list of the coarse bins that
+        // matter, and the first positions of their fine bins
+        scan_bins(bins, coarse, flags, ss, s_warp, cta, nctas, kk);
         if (!barrier()) return;
 
         if (__ldcg(&flags[0]) == 0) {
-            // scatter into the second buffer, grouped by bin
-            for_each_record([&](unsigned long long rec) { G2[atomicAdd(&bins[bin_of(rec)], 1u)] = rec; });
+            // scatter into the second buffer, grouped by bin: the records of the listed coarse bins
+            for_each_record([&](unsigned long long rec) {
+                const uint32_t b = bin_of(rec);
+                if (s_coarse[b / BIN_PER_COARSE] < kk) G2[atomicAdd(&bins[b], 1u)] = rec;
+            });
             if (!barrier()) return;
-            // rank inside the bin: bin b now occupies [end of bin b-1, bins[b])
+            // rank inside the bin: bin b now occupies [end of the bin before it, bins[b]); the first fine bin of a coarse bin
+            // starts where the coarse bin does
             // (only positions below the end of the bin that holds position kk-1 matter; they are a prefix)
-            const uint64_t g_end = (uint64_t)kk + LG_CROWDED < n ? (uint64_t)kk + LG_CROWDED : n;
+            uint64_t g_end = (uint64_t)kk + LG_CROWDED < n ? (uint64_t)kk + LG_CROWDED : n;
+            g_end = g_end < ss.scattered ? g_end : ss.scattered;
             for (uint64_t g = gid; g < g_end; g += gthreads) {
                 const unsigned long long rec = __ldcg(&G2[g]);
                 const uint32_t b = bin_of(rec);
-                const uint32_t first = b ? __ldcg(&bins[b - 1]) : 0u, last = __ldcg(&bins[b]);
+                const uint32_t first = b % BIN_PER_COARSE ? __ldcg(&bins[b - 1]) : s_coarse[b / BIN_PER_COARSE], last = __ldcg(&bins[b]);
                 if (first < kk) {
                     uint32_t pos = first;
                     for (uint32_t j = first; j < last; ++j) pos += __ldcg(&G2[j]) < rec;
