@@ -37,9 +37,10 @@ constexpr uint32_t SORT_CAP_MAX = 16384;         // largest k the single-CTA ref
 //   one row: from k = 8193 on; bf16 from 3073 on, since the grid-wide path then starts from the filter's histogram
 //     (2^28 bf16: k = 4096 137 -> 118 us, k = 8192 245 -> 114; 2^26: 58 -> 56, 106 -> 57; k = 2048 still 103 against
 //     118; fp32 k = 8192: 186 against 193).
-//   2 to 18 rows: from the k of large_switch_k on, read off sweeps over rows x k x N (2^20 .. 2^26) of both paths: the
-//     longer the rows and the more of them, the earlier (8 fp32 rows of 2^24, k = 6000: 203 us through one CTA each, 178
-//     through the grid; of 2^22: 74 against 103; 4 bf16 rows of 2^26, k = 4500: 180 against 142; 2 of 2^20: 39 against 49).
+//   2 to 18 rows: from the k of large_switch_k on, read off sweeps over rows x k x N (2^20 .. 2^26) of both paths.  fp32:
+//     the longer the rows and the more of them, the earlier (8 rows of 2^24, k = 6000: 203 us through one CTA each, 178
+//     through the grid; of 2^22: 74 against 103).  bf16: near k = 6000 whatever the length (8 rows of 2^22: k = 5000 69
+//     against 74, k = 6000 78 against 75, k = 8192 102 against 77, k = 16384 246 against 87).
 //   more rows: the CTAs work side by side and win.
 constexpr int64_t LARGE_FEW_ROWS = 4;
 constexpr int64_t LARGE_SOME_ROWS = 18;
@@ -49,11 +50,7 @@ constexpr int64_t LARGE_SOME_K_MIN = 4096;       // no call of 2 to 18 rows swit
 // 2 to 18 rows: the largest k one CTA per row still orders.
 inline int64_t large_switch_k(int64_t rows, size_t elem_size, int64_t N) {
     const int64_t never = (int64_t)SORT_CAP_MAX;
-    if (elem_size == 2) {
-        if (N >= (1LL << 26)) return LARGE_SOME_K_MIN;
-        if (N >= (1LL << 24)) return rows <= 4 ? 6144 : 7168;
-        return rows <= 4 ? 6656 : rows <= 8 ? 8192 : 10240;
-    }
+    if (elem_size == 2) return rows <= 8 ? 5632 : 6656;        // (at every row length from 2^20 to 2^26)
     if (N >= (1LL << 26)) return 6144;
     if (N >= (1LL << 25)) return rows <= 3 ? 8192 : 6144;
     if (N >= (1LL << 24)) return rows <= 4 ? 10240 : 6144;
